@@ -1,0 +1,161 @@
+/* resist.h -- C boundary of the ResIST sub-ResNet training library (CUDA, sm_100a).
+ *
+ * The calls follow the protocol of Algorithm 1 of "ResIST: Layer-Wise Decomposition of ResNets for
+ * Distributed Training" (arXiv 2107.00961): per synchronisation round, subResNets(.) partitions the
+ * residual blocks of a global pre-activation ResNet among S shallow sub-ResNets (Sec. 2.2), each
+ * sub-ResNet takes l local SGD steps (Algorithm 1, inner loops), and aggregate(.) sets every global
+ * parameter to its mean over the sub-ResNets that held it (Sec. 2.3; Appendix B).  Here the S
+ * "workers" are S independent problems on ONE GPU; nothing crosses a link.
+ *
+ * Conventions
+ *  - Every function returns 0 (RESIST_OK) or a negative resist_status; nothing throws or aborts.
+ *    resist_last_error() gives a human-readable reason for the last failure on that context.
+ *  - "dev" pointers are CUDA device pointers owned by the caller; "host" pointers are ordinary memory.
+ *  - Activations are NHWC, convolution weights [Cout][kh][kw][Cin], both contiguous.
+ *  - The library owns parameters, momentum, gradients, activations and scratch; it obtains device
+ *    memory only through the resist_allocator given at init (or cudaMalloc when that is NULL).
+ *  - Work is enqueued on the given stream; calls that return host data synchronise that stream.
+ *  - State machine: init -> partition -> (local_step)* -> aggregate -> partition ...; a call out of
+ *    order returns RESIST_ESTATE.
+ *
+ * Flat parameter order (all fp32 on the boundary): stem conv; stem BN gamma, beta (if any); per block in
+ * network order: basic = bn1 g,b | conv1 3x3 | bn2 g,b | conv2 3x3 | projection 1x1 (if any);
+ * bottleneck = bn1 g,b | conv1 1x1 | bn2 g,b | conv2 3x3 | bn3 g,b | conv3 1x1 | projection (if any);
+ * final BN g,b; head weight [classes][C]; head bias.  Buffers: per BN in that order, running mean then
+ * running variance.
+ */
+#ifndef RESIST_H
+#define RESIST_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    RESIST_OK = 0,
+    RESIST_EINVAL = -1,       /* bad argument */
+    RESIST_ESTATE = -2,       /* call out of order */
+    RESIST_ENOMEM = -3,       /* the allocator returned NULL */
+    RESIST_ECUDA = -4,        /* a CUDA call failed; see resist_last_error */
+    RESIST_ETIMEOUT = -5,     /* a bounded device-side wait gave up */
+    RESIST_EUNSUPPORTED = -6
+} resist_status;
+
+enum { RESIST_BASIC = 0, RESIST_BOTTLENECK = 1 };
+enum { RESIST_F32 = 0, RESIST_BF16 = 1 };
+enum { RESIST_MOMENTUM_RESTART = 0, RESIST_MOMENTUM_KEEP = 1 };
+enum { RESIST_CONV_AUTO = 0, RESIST_CONV_CUDA_CORES = 1 };
+#define RESIST_MAX_SUBNETS 32
+
+typedef struct resist_ctx resist_ctx;
+typedef void* resist_stream;                 /* a cudaStream_t */
+
+/* One residual block (Sec. 2.1, pre-activation order BN -> ReLU -> conv).  `partitionable` marks the blocks
+ * that subResNets(.) deals out (Sec. 2.2: the non-strided blocks of the third section); all others are
+ * held by every sub-ResNet. */
+typedef struct {
+    int32_t kind;            /* RESIST_BASIC (3x3,3x3) or RESIST_BOTTLENECK (1x1,3x3,1x1; stride on the 3x3) */
+    int32_t stage;
+    int32_t cin, cmid, cout; /* basic: cmid = cout */
+    int32_t stride;          /* 1 or 2 */
+    int32_t has_projection;  /* 1x1 strided conv on the skip path, reading relu(bn1(x)) */
+    int32_t partitionable;
+} resist_block;
+
+typedef struct {
+    int32_t in_h, in_w, in_c, classes;
+    int32_t stem_k, stem_stride, stem_cout;
+    int32_t stem_bn_relu;    /* stem conv followed by BN + ReLU */
+    int32_t stem_maxpool;    /* then a 3x3 stride-2 max-pool, padding 1 */
+    int32_t num_blocks;
+    const resist_block* blocks;   /* host, num_blocks entries, copied at init */
+} resist_arch;
+
+typedef struct {
+    int32_t dtype;           /* RESIST_F32: everything fp32 on CUDA cores.  RESIST_BF16: activations, activation
+                                gradients and the convolutions' weight copy are bf16, accumulation and all
+                                parameters, statistics and gradients of parameters fp32 */
+    float momentum;          /* SGD momentum mu: v = mu*v + g; w -= lr*v */
+    float weight_decay;      /* g += wd*w */
+    float bn_eps;
+    float bn_momentum;       /* running = (1-m)*running + m*batch (variance unbiased) */
+    int32_t min_depth;       /* >0: top sub-ResNets up to this many partitioned blocks (Sec. 2.6) */
+    int32_t momentum_policy; /* RESIST_MOMENTUM_RESTART: zero the momentum at every partition */
+    int32_t conv_backend;    /* RESIST_CONV_AUTO: tensor cores where the shape allows; _CUDA_CORES: never */
+} resist_opts;
+
+/* Device-memory source.  alloc returns a device pointer aligned to >= 256 bytes or NULL; release frees it.
+ * Both are called on the host from inside resist_* calls (never from another thread). */
+typedef struct {
+    void* (*alloc)(void* user, size_t bytes);
+    void (*release)(void* user, void* dev_ptr);
+    void* user;
+} resist_allocator;
+
+/* Creates a context holding the global ResNet h(W) (Algorithm 1, "randomly initialized ResNet"): He-normal
+ * conv and head weights drawn from a splitmix64 stream seeded with `seed`, gamma 1, beta 0, bias 0, running
+ * mean 0, running var 1.  arch, opts: host.  alloc may be NULL.  *out receives the context. */
+int resist_init(const resist_arch* arch, const resist_opts* opts, uint64_t seed, const resist_allocator* alloc,
+                resist_ctx** out);
+int resist_destroy(resist_ctx* ctx);
+
+/* subResNets(h(W), S) of Algorithm 1 (Sec. 2.2): permutes the partitionable block indices with Fisher-Yates
+ * driven by splitmix64(round_seed) (i from P-1 down to 1, j = next() mod (i+1)), deals position j of the
+ * permutation to sub-ResNet j mod S, gives every other block to all S; then copies the global parameters into
+ * the S working copies ("distribute each h_s(W_s) to a different worker") and restarts their momentum.
+ * member_mask: host, [num_blocks], bit s set = block is in sub-ResNet s (may be NULL).
+ * Errors: S < 1 or S > 32, or S > P with min_depth == 0 -> RESIST_EINVAL. */
+int resist_partition(resist_ctx* ctx, uint64_t round_seed, int32_t S, uint32_t* member_mask, resist_stream stream);
+
+/* One local SGD iteration of sub-ResNet `subnet` (Algorithm 1: W_s = W_s - eta dL/dW_s): forward and backward
+ * of its blocks on one minibatch (batch-statistics BN, mean softmax cross-entropy), then the momentum update.
+ * images: dev, [B][in_h][in_w][in_c], fp32 or bf16 according to opts.dtype.  labels: dev int32 [B].
+ * loss_out: dev float[1] or NULL.  B >= 2. */
+int resist_local_step(resist_ctx* ctx, int32_t subnet, const void* images, const int32_t* labels, int32_t B,
+                      float lr, float* loss_out, resist_stream stream);
+
+/* The same iteration for all S sub-ResNets at once: each layer slot is one launch over the S problems.
+ * images, labels: host arrays of S dev pointers.  loss_out: dev float[S] or NULL. */
+int resist_local_step_grouped(resist_ctx* ctx, const void* const* images, const int32_t* const* labels, int32_t B,
+                              float lr, float* loss_out, resist_stream stream);
+
+/* aggregate({h_s(W_s)}) of Algorithm 1 (Sec. 2.3; Appendix B): every global parameter and BN running statistic
+ * becomes the mean over the sub-ResNets that held it, evaluated in fp32 as first + (sum_s (w_s - first))/count
+ * with owners in ascending order; a single owner is copied bit for bit. */
+int resist_aggregate(resist_ctx* ctx, resist_stream stream);
+
+/* Evaluates the global network (Sec. 2.6): all blocks, BN with running statistics, the residual branch of every
+ * partitionable block scaled by 1/S (S of the last partition; 1 before any).  logits_out: dev float
+ * [B][classes] or NULL; loss_out: dev float[1] or NULL; correct_out: dev int32[1] (top-1 hits) or NULL. */
+int resist_eval(resist_ctx* ctx, const void* images, const int32_t* labels, int32_t B, float* logits_out,
+                float* loss_out, int32_t* correct_out, resist_stream stream);
+
+/* Parity and checkpoint taps (host buffers, fp32, flat order above; they synchronise the device). */
+int resist_param_count(resist_ctx* ctx, int64_t* n_params, int64_t* n_buffers);
+int resist_get_params(resist_ctx* ctx, int32_t subnet /* -1 = global */, float* host_params, float* host_buffers);
+int resist_set_params(resist_ctx* ctx, const float* host_params, const float* host_buffers);   /* global */
+int resist_get_grads(resist_ctx* ctx, int32_t subnet, float* host_grads);    /* last step's dL/dW; absent blocks 0 */
+int resist_get_logits(resist_ctx* ctx, int32_t subnet, float* host_logits);  /* last step's [B][classes] */
+
+/* Work counters of the last local step call (grouped or single). */
+typedef struct {
+    int64_t kernel_launches;   /* kernels enqueued */
+    int64_t conv_flops;        /* 2*M*N*K summed over forward, dgrad and wgrad convolutions */
+    int64_t tensor_core_convs; /* convolution problems run on tcgen05 */
+    int64_t cuda_core_convs;   /* convolution problems run on CUDA cores */
+    int64_t workspace_bytes;   /* device memory held for activations and scratch */
+} resist_step_info;
+int resist_get_step_info(resist_ctx* ctx, resist_step_info* out);
+
+/* The library's own splitmix64 (the stream that drives the partition), for cross-checking: host out[n]. */
+void resist_splitmix64(uint64_t seed, int64_t n, uint64_t* out);
+
+const char* resist_last_error(resist_ctx* ctx);   /* ctx may be NULL: the last init failure */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RESIST_H */

@@ -1,0 +1,108 @@
+// Internal declarations shared by the runtime and the kernel files of the ResIST library.
+// Every kernel is a "grouped" kernel: it receives a device array of problem descriptors and
+// blockIdx.y selects the problem, so the S sub-ResNets of one layer slot run in one launch.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+namespace resist {
+
+enum ConvMode { CONV_FWD = 0, CONV_DGRAD = 1, CONV_WGRAD = 2 };
+
+// One convolution problem, any mode.  Geometry always describes the FORWARD convolution:
+// input [N,H,W,C], weights [K,ksz,ksz,C], output [N,P,Q,K].
+struct ConvProb {
+    const void* act;      // fwd: input a;      dgrad: dy;            wgrad: input a
+    const void* wgt;      // fwd: weights;      dgrad: weights;       wgrad: dy
+    const void* add;      // optional tensor added to the result (shape of out), or nullptr
+    void* out;            // fwd: y (T);        dgrad: da (T);        wgrad: dw (fp32, [K][ksz][ksz][C])
+    float* partial;       // wgrad split-K workspace [splits][K*ksz*ksz*C], or nullptr
+    double* stat_partial; // fwd (tensor-core path): per-tile column sums for the next BN, or nullptr
+    int N, H, W, C, K, ksz, stride, pad, P, Q;
+    int M, Ncol, Kred;    // GEMM extents of this mode
+    int tiles_m, tiles_n, splits, ktiles_per_split;
+    float scale;          // result = scale*acc + add
+    int pad_;
+};
+
+// One batch-normalisation + ReLU problem over x [m, C] (forward or backward).
+struct BnProb {
+    const void* x;        // pre-normalisation tensor (T)
+    void* a;              // forward output relu(bn(x)) (T)
+    const void* da;       // backward: gradient w.r.t. a (T)
+    void* dx;             // backward: gradient w.r.t. x (T)
+    const void* add;      // backward: tensor added to dx (skip-path gradient), or nullptr
+    const float* gamma; const float* beta;
+    float* dgamma; float* dbeta;
+    float* run_mean; float* run_var;   // forward: updated when non-null
+    double* partial;      // [chunks][2][C]
+    float* stat;          // [4][C]: mean, invstd, sum dz, sum dz*xhat
+    long long m;
+    int C, chunks, rows_per_chunk;
+    float eps, momentum;
+    int eval;             // 1: use running statistics (no batch statistics)
+    int pad_;
+};
+
+struct PoolProb {         // 3x3 stride-2 max-pool, pad 1: x [N,H,W,C] -> y [N,P,Q,C]
+    const void* x; void* y; int* arg; const void* dy; void* dx;
+    int N, H, W, C, P, Q;
+};
+
+struct HeadProb {         // global average pool + linear head + mean softmax cross-entropy
+    const void* a;        // final activation (T) [B, HW, C]
+    void* da;             // its gradient (T)
+    const float* w; const float* b; float* dw; float* db;
+    float* pooled;        // [B, C]
+    float* dpooled;       // [B, C]
+    float* logits;        // [B, classes]
+    float* dlogits;       // [B, classes]
+    const int* labels;
+    float* loss;          // [1]
+    float* loss_user;     // optional copy for the caller
+    int* correct;         // optional top-1 count
+    float* logits_user;   // optional copy for the caller
+    int B, HW, C, classes;
+};
+
+// A contiguous run of parameters treated alike by the bandwidth kernels.
+struct Segment {
+    long long begin;      // offset in the flat vector
+    long long len;
+    long long chunk0;     // first chunk index of this segment in the launch
+    unsigned mask;        // aggregate: owners; scatter/sgd: unused
+    int sub;              // scatter/sgd: sub-ResNet index
+};
+
+struct ParamArrays {      // device pointers of the flat arrays
+    float* global; float* global_buf;
+    float* w;  float* v;  float* g;  __nv_bfloat16* wb;  float* buf;   // [S][n] each (buf: [S][n_buffers])
+    long long n, nbuf;
+};
+
+constexpr int SEG_CHUNK = 4096;   // elements per CTA in the segment kernels
+
+// ---- launchers (kernels_ref.cu)
+void launch_conv_ref(const ConvProb* d, int nprob, int max_tiles, int mode, bool bf16, cudaStream_t s);
+void launch_splitk_reduce(const ConvProb* d, int nprob, int max_elems, cudaStream_t s);
+void launch_bn_stats(const BnProb* d, int nprob, int max_chunks, int max_c, bool bf16, cudaStream_t s);
+void launch_bn_apply(const BnProb* d, int nprob, long long max_elems, bool bf16, cudaStream_t s);
+void launch_bn_bwd_reduce(const BnProb* d, int nprob, int max_chunks, int max_c, bool bf16, cudaStream_t s);
+void launch_bn_bwd_apply(const BnProb* d, int nprob, long long max_elems, bool bf16, cudaStream_t s);
+void launch_maxpool_fwd(const PoolProb* d, int nprob, long long max_elems, bool bf16, cudaStream_t s);
+void launch_maxpool_bwd(const PoolProb* d, int nprob, long long max_elems, bool bf16, cudaStream_t s);
+void launch_head_fwd(const HeadProb* d, int nprob, int maxB, int maxC, int max_classes, bool bf16, cudaStream_t s);
+void launch_head_bwd(const HeadProb* d, int nprob, int maxB, int maxC, int max_classes, long long max_elems,
+                     bool bf16, cudaStream_t s);
+
+// ---- launchers (kernels_bw.cu)
+void launch_sgd(const Segment* d, int nseg, long long nchunks, ParamArrays pa, float lr, float mu, float wd,
+                bool shadow, cudaStream_t s);
+void launch_scatter(const Segment* d, int nseg, long long nchunks, ParamArrays pa, bool zero_momentum, bool shadow,
+                    cudaStream_t s);
+void launch_scatter_buffers(const Segment* d, int nseg, long long nchunks, ParamArrays pa, cudaStream_t s);
+void launch_aggregate(const Segment* d, int nseg, long long nchunks, const float* sub, long long stride,
+                      float* global, int S, cudaStream_t s);
+
+}  // namespace resist

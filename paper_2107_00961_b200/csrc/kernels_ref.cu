@@ -1,0 +1,420 @@
+// CUDA-core kernel family: every layer of the sub-ResNet step for storage type T = float or bf16,
+// fp32 arithmetic.  It is the whole path of the fp32 mode, and in bf16 mode it runs whatever the
+// tensor-core kernels do not take (3-channel stems, odd shapes) and the small head/loss kernels.
+// All reductions have a fixed order: results are reproducible run to run.
+#include "internal.h"
+
+namespace resist {
+
+template <class T> __device__ __forceinline__ float ldf(const void* p, long long i);
+template <> __device__ __forceinline__ float ldf<float>(const void* p, long long i) { return ((const float*)p)[i]; }
+template <> __device__ __forceinline__ float ldf<__nv_bfloat16>(const void* p, long long i) {
+    return __bfloat162float(((const __nv_bfloat16*)p)[i]);
+}
+template <class T> __device__ __forceinline__ void stf(void* p, long long i, float v);
+template <> __device__ __forceinline__ void stf<float>(void* p, long long i, float v) { ((float*)p)[i] = v; }
+template <> __device__ __forceinline__ void stf<__nv_bfloat16>(void* p, long long i, float v) {
+    ((__nv_bfloat16*)p)[i] = __float2bfloat16_rn(v);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Implicit-GEMM convolution on CUDA cores: 64x64 output tile, 16-deep slices, 256 threads, 4x4 per thread.
+//   forward: rows = output pixels (n,p,q), cols = output channels, reduction = (r,s,c)
+//   dgrad:   rows = input pixels (n,h,w),  cols = input channels,  reduction = (r,s,k)
+//   wgrad:   rows = output channels,       cols = (r,s,c),         reduction = output pixels; split over
+//            `splits` CTAs along the reduction, partial sums reduced afterwards in a fixed order.
+// ------------------------------------------------------------------------------------------------
+constexpr int BM = 64, BN = 64, BK = 16;
+
+template <class T, int MODE>
+__device__ __forceinline__ float load_a(const ConvProb& p, int row, int kk) {
+    if (row >= p.M || kk >= p.Kred) return 0.f;
+    if (MODE == CONV_FWD) {
+        int q = row % p.Q, t = row / p.Q, pp = t % p.P, n = t / p.P;
+        int c = kk % p.C, t2 = kk / p.C, s = t2 % p.ksz, r = t2 / p.ksz;
+        int h = pp * p.stride + r - p.pad, x = q * p.stride + s - p.pad;
+        if (h < 0 || h >= p.H || x < 0 || x >= p.W) return 0.f;
+        return ldf<T>(p.act, (((long long)n * p.H + h) * p.W + x) * p.C + c);
+    } else if (MODE == CONV_DGRAD) {
+        int x = row % p.W, t = row / p.W, h = t % p.H, n = t / p.H;
+        int ko = kk % p.K, t2 = kk / p.K, s = t2 % p.ksz, r = t2 / p.ksz;
+        int ph = h + p.pad - r, qx = x + p.pad - s;
+        if (ph < 0 || qx < 0 || ph % p.stride || qx % p.stride) return 0.f;
+        int pp = ph / p.stride, q = qx / p.stride;
+        if (pp >= p.P || q >= p.Q) return 0.f;
+        return ldf<T>(p.act, (((long long)n * p.P + pp) * p.Q + q) * p.K + ko);
+    } else {   // wgrad: A[ko, t] = dy[t, ko]
+        return ldf<T>(p.wgt, (long long)kk * p.K + row);
+    }
+}
+template <class T, int MODE>
+__device__ __forceinline__ float load_b(const ConvProb& p, int kk, int col) {
+    if (col >= p.Ncol || kk >= p.Kred) return 0.f;
+    if (MODE == CONV_FWD) {
+        return ldf<T>(p.wgt, (long long)col * p.Kred + kk);
+    } else if (MODE == CONV_DGRAD) {
+        int ko = kk % p.K, t2 = kk / p.K, s = t2 % p.ksz, r = t2 / p.ksz;
+        return ldf<T>(p.wgt, (((long long)ko * p.ksz + r) * p.ksz + s) * p.C + col);
+    } else {   // wgrad: B[t, (r,s,c)] = a[n, p*stride+r-pad, q*stride+s-pad, c]
+        int q = kk % p.Q, t = kk / p.Q, pp = t % p.P, n = t / p.P;
+        int c = col % p.C, t2 = col / p.C, s = t2 % p.ksz, r = t2 / p.ksz;
+        int h = pp * p.stride + r - p.pad, x = q * p.stride + s - p.pad;
+        if (h < 0 || h >= p.H || x < 0 || x >= p.W) return 0.f;
+        return ldf<T>(p.act, (((long long)n * p.H + h) * p.W + x) * p.C + c);
+    }
+}
+
+template <class T, int MODE>
+__global__ void __launch_bounds__(256) conv_ref_kernel(const ConvProb* __restrict__ probs) {
+    const ConvProb& p = probs[blockIdx.y];
+    const int tiles = p.tiles_m * p.tiles_n;
+    int tile = blockIdx.x;
+    if (tile >= tiles * p.splits) return;
+    const int split = tile / tiles; tile -= split * tiles;
+    const int tm = tile / p.tiles_n, tn = tile % p.tiles_n;
+    __shared__ float As[BK][BM + 4];
+    __shared__ float Bs[BK][BN + 4];
+    const int tid = threadIdx.x, ty = tid / 16, tx = tid % 16;
+    float acc[4][4] = {};
+    const int kt0 = split * p.ktiles_per_split;
+    int kt1 = kt0 + p.ktiles_per_split;
+    const int ktiles = (p.Kred + BK - 1) / BK;
+    if (kt1 > ktiles) kt1 = ktiles;
+    for (int kt = kt0; kt < kt1; ++kt) {
+        const int k0 = kt * BK;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            int e = tid + 256 * i;
+            if (MODE == CONV_WGRAD) { int r = e % BM, kc = e / BM; As[kc][r] = load_a<T, MODE>(p, tm * BM + r, k0 + kc); }
+            else { int kc = e % BK, r = e / BK; As[kc][r] = load_a<T, MODE>(p, tm * BM + r, k0 + kc); }
+            if (MODE == CONV_FWD) { int kc = e % BK, c = e / BK; Bs[kc][c] = load_b<T, MODE>(p, k0 + kc, tn * BN + c); }
+            else { int c = e % BN, kc = e / BN; Bs[kc][c] = load_b<T, MODE>(p, k0 + kc, tn * BN + c); }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kc = 0; kc < BK; ++kc) {
+            float a[4], b[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { a[i] = As[kc][ty * 4 + i]; b[i] = Bs[kc][tx * 4 + i]; }
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int row = tm * BM + ty * 4 + i;
+        if (row >= p.M) continue;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int col = tn * BN + tx * 4 + j;
+            if (col >= p.Ncol) continue;
+            const long long o = (long long)row * p.Ncol + col;
+            if (MODE == CONV_WGRAD) {
+                if (p.splits > 1) p.partial[(long long)split * p.M * p.Ncol + o] = acc[i][j];
+                else ((float*)p.out)[o] = acc[i][j];
+            } else {
+                float v = acc[i][j] * p.scale;
+                if (p.add) v += ldf<T>(p.add, o);
+                stf<T>(p.out, o, v);
+            }
+        }
+    }
+}
+
+__global__ void splitk_reduce_kernel(const ConvProb* __restrict__ probs) {
+    const ConvProb& p = probs[blockIdx.y];
+    if (p.splits <= 1) return;
+    const long long n = (long long)p.M * p.Ncol;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+        float s = 0.f;
+        for (int k = 0; k < p.splits; ++k) s += p.partial[(long long)k * n + i];
+        ((float*)p.out)[i] = s;
+    }
+}
+
+void launch_conv_ref(const ConvProb* d, int nprob, int max_tiles, int mode, bool bf16, cudaStream_t s) {
+    dim3 g(max_tiles, nprob);
+    if (!bf16) {
+        if (mode == CONV_FWD) conv_ref_kernel<float, CONV_FWD><<<g, 256, 0, s>>>(d);
+        else if (mode == CONV_DGRAD) conv_ref_kernel<float, CONV_DGRAD><<<g, 256, 0, s>>>(d);
+        else conv_ref_kernel<float, CONV_WGRAD><<<g, 256, 0, s>>>(d);
+    } else {
+        if (mode == CONV_FWD) conv_ref_kernel<__nv_bfloat16, CONV_FWD><<<g, 256, 0, s>>>(d);
+        else if (mode == CONV_DGRAD) conv_ref_kernel<__nv_bfloat16, CONV_DGRAD><<<g, 256, 0, s>>>(d);
+        else conv_ref_kernel<__nv_bfloat16, CONV_WGRAD><<<g, 256, 0, s>>>(d);
+    }
+}
+void launch_splitk_reduce(const ConvProb* d, int nprob, int max_elems, cudaStream_t s) {
+    int gx = (max_elems + 255) / 256; if (gx > 1184) gx = 1184; if (gx < 1) gx = 1;
+    splitk_reduce_kernel<<<dim3(gx, nprob), 256, 0, s>>>(d);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Batch normalisation + ReLU.  Statistics: each CTA reduces `rows_per_chunk` rows of all C channels
+// (fp32 per thread, fp64 across threads), a finalise kernel adds the chunk partials in order.
+// ------------------------------------------------------------------------------------------------
+// MODE 0: sums of x and x^2.  MODE 1: sums of dz and dz*xhat (backward).
+template <class T, int MODE>
+__global__ void __launch_bounds__(256) bn_reduce_kernel(const BnProb* __restrict__ probs) {
+    const BnProb& p = probs[blockIdx.y];
+    if ((int)blockIdx.x >= p.chunks || p.eval) return;
+    __shared__ double part[2][256];
+    const int C = p.C, nl = C < 256 ? C : 256, R = 256 / nl;
+    const int rg = threadIdx.x / nl, lane = threadIdx.x % nl;
+    const long long r0 = (long long)blockIdx.x * p.rows_per_chunk;
+    long long r1 = r0 + p.rows_per_chunk; if (r1 > p.m) r1 = p.m;
+    for (int cb = 0; cb < C; cb += nl) {
+        const int c = cb + lane;
+        float s0 = 0.f, s1 = 0.f;
+        if (rg < R && c < C) {
+            float mean = 0.f, istd = 0.f, g = 0.f, b = 0.f;
+            if (MODE == 1) { mean = p.stat[c]; istd = p.stat[C + c]; g = p.gamma[c]; b = p.beta[c]; }
+            for (long long r = r0 + rg; r < r1; r += R) {
+                float x = ldf<T>(p.x, r * C + c);
+                if (MODE == 0) { s0 += x; s1 += x * x; }
+                else {
+                    float xh = (x - mean) * istd;
+                    float dz = (xh * g + b > 0.f) ? ldf<T>(p.da, r * C + c) : 0.f;
+                    s0 += dz; s1 += dz * xh;
+                }
+            }
+        }
+        __syncthreads();
+        part[0][threadIdx.x] = s0; part[1][threadIdx.x] = s1;
+        __syncthreads();
+        if (rg == 0 && c < C) {
+            double a0 = 0.0, a1 = 0.0;
+            for (int k = 0; k < R; ++k) { a0 += part[0][k * nl + lane]; a1 += part[1][k * nl + lane]; }
+            p.partial[((long long)blockIdx.x * 2 + 0) * C + c] = a0;
+            p.partial[((long long)blockIdx.x * 2 + 1) * C + c] = a1;
+        }
+    }
+}
+
+template <int MODE>
+__global__ void bn_finalize_kernel(const BnProb* __restrict__ probs) {
+    const BnProb& p = probs[blockIdx.y];
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= p.C) return;
+    if (p.eval) {
+        if (MODE == 0) { p.stat[c] = p.run_mean[c]; p.stat[p.C + c] = (float)(1.0 / sqrt((double)p.run_var[c] + (double)p.eps)); }
+        return;
+    }
+    double a0 = 0.0, a1 = 0.0;
+    for (int k = 0; k < p.chunks; ++k) { a0 += p.partial[((long long)k * 2 + 0) * p.C + c]; a1 += p.partial[((long long)k * 2 + 1) * p.C + c]; }
+    if (MODE == 0) {
+        const double m = (double)p.m, mean = a0 / m;
+        double var = a1 / m - mean * mean; if (var < 0.0) var = 0.0;
+        p.stat[c] = (float)mean;
+        p.stat[p.C + c] = (float)(1.0 / sqrt(var + (double)p.eps));
+        if (p.run_mean) {
+            const double unb = p.m > 1 ? var * m / (m - 1.0) : var, mo = (double)p.momentum;
+            p.run_mean[c] = (float)((1.0 - mo) * (double)p.run_mean[c] + mo * mean);
+            p.run_var[c] = (float)((1.0 - mo) * (double)p.run_var[c] + mo * unb);
+        }
+    } else {
+        p.stat[2 * p.C + c] = (float)a0; p.stat[3 * p.C + c] = (float)a1;
+        p.dbeta[c] = (float)a0; p.dgamma[c] = (float)a1;
+    }
+}
+
+template <class T>
+__global__ void __launch_bounds__(256) bn_apply_kernel(const BnProb* __restrict__ probs) {
+    const BnProb& p = probs[blockIdx.y];
+    const long long n = p.m * p.C;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+        const int c = (int)(i % p.C);
+        float z = (ldf<T>(p.x, i) - p.stat[c]) * p.stat[p.C + c] * p.gamma[c] + p.beta[c];
+        stf<T>(p.a, i, z > 0.f ? z : 0.f);
+    }
+}
+
+template <class T>
+__global__ void __launch_bounds__(256) bn_bwd_apply_kernel(const BnProb* __restrict__ probs) {
+    const BnProb& p = probs[blockIdx.y];
+    const long long n = p.m * p.C;
+    const float inv_m = 1.f / (float)p.m;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+        const int c = (int)(i % p.C);
+        const float istd = p.stat[p.C + c], g = p.gamma[c];
+        const float xh = (ldf<T>(p.x, i) - p.stat[c]) * istd;
+        const float dz = (xh * g + p.beta[c] > 0.f) ? ldf<T>(p.da, i) : 0.f;
+        float v = g * istd * (dz - p.stat[2 * p.C + c] * inv_m - xh * p.stat[3 * p.C + c] * inv_m);
+        if (p.add) v += ldf<T>(p.add, i);
+        stf<T>(p.dx, i, v);
+    }
+}
+
+static int ew_grid(long long n) { long long g = (n + 255) / 256; if (g > 148 * 16) g = 148 * 16; if (g < 1) g = 1; return (int)g; }
+
+void launch_bn_stats(const BnProb* d, int nprob, int max_chunks, int max_c, bool bf16, cudaStream_t s) {
+    if (bf16) bn_reduce_kernel<__nv_bfloat16, 0><<<dim3(max_chunks, nprob), 256, 0, s>>>(d);
+    else bn_reduce_kernel<float, 0><<<dim3(max_chunks, nprob), 256, 0, s>>>(d);
+    bn_finalize_kernel<0><<<dim3((max_c + 127) / 128, nprob), 128, 0, s>>>(d);
+}
+void launch_bn_apply(const BnProb* d, int nprob, long long max_elems, bool bf16, cudaStream_t s) {
+    if (bf16) bn_apply_kernel<__nv_bfloat16><<<dim3(ew_grid(max_elems), nprob), 256, 0, s>>>(d);
+    else bn_apply_kernel<float><<<dim3(ew_grid(max_elems), nprob), 256, 0, s>>>(d);
+}
+void launch_bn_bwd_reduce(const BnProb* d, int nprob, int max_chunks, int max_c, bool bf16, cudaStream_t s) {
+    if (bf16) bn_reduce_kernel<__nv_bfloat16, 1><<<dim3(max_chunks, nprob), 256, 0, s>>>(d);
+    else bn_reduce_kernel<float, 1><<<dim3(max_chunks, nprob), 256, 0, s>>>(d);
+    bn_finalize_kernel<1><<<dim3((max_c + 127) / 128, nprob), 128, 0, s>>>(d);
+}
+void launch_bn_bwd_apply(const BnProb* d, int nprob, long long max_elems, bool bf16, cudaStream_t s) {
+    if (bf16) bn_bwd_apply_kernel<__nv_bfloat16><<<dim3(ew_grid(max_elems), nprob), 256, 0, s>>>(d);
+    else bn_bwd_apply_kernel<float><<<dim3(ew_grid(max_elems), nprob), 256, 0, s>>>(d);
+}
+
+// ------------------------------------------------------------------------------------------------
+// 3x3 stride-2 max-pool (padding 1, padded cells never win; first maximum in row-major window order)
+// ------------------------------------------------------------------------------------------------
+template <class T>
+__global__ void maxpool_fwd_kernel(const PoolProb* __restrict__ probs) {
+    const PoolProb& p = probs[blockIdx.y];
+    const long long n = (long long)p.N * p.P * p.Q * p.C;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+        int c = (int)(i % p.C); long long t = i / p.C; int q = (int)(t % p.Q); t /= p.Q; int pp = (int)(t % p.P); int nn = (int)(t / p.P);
+        bool have = false; float best = 0.f; int bi = -1;
+        for (int r = 0; r < 3; ++r) { int h = 2 * pp + r - 1; if (h < 0 || h >= p.H) continue;
+            for (int s = 0; s < 3; ++s) { int w = 2 * q + s - 1; if (w < 0 || w >= p.W) continue;
+                float v = ldf<T>(p.x, (((long long)nn * p.H + h) * p.W + w) * p.C + c);
+                if (!have || v > best) { have = true; best = v; bi = h * p.W + w; } } }
+        stf<T>(p.y, i, best);
+        if (p.arg) p.arg[i] = bi;
+    }
+}
+template <class T>
+__global__ void maxpool_bwd_kernel(const PoolProb* __restrict__ probs) {
+    const PoolProb& p = probs[blockIdx.y];
+    const long long n = (long long)p.N * p.H * p.W * p.C;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+        int c = (int)(i % p.C); long long t = i / p.C; int w = (int)(t % p.W); t /= p.W; int h = (int)(t % p.H); int nn = (int)(t / p.H);
+        float acc = 0.f;
+        for (int pp = h / 2; pp <= (h + 1) / 2; ++pp) { if (pp >= p.P) continue;          // windows with 2p-1 <= h <= 2p+1
+            for (int q = w / 2; q <= (w + 1) / 2; ++q) { if (q >= p.Q) continue;
+                long long o = (((long long)nn * p.P + pp) * p.Q + q) * p.C + c;
+                if (p.arg[o] == h * p.W + w) acc += ldf<T>(p.dy, o); } }
+        stf<T>(p.dx, i, acc);
+    }
+}
+void launch_maxpool_fwd(const PoolProb* d, int nprob, long long max_elems, bool bf16, cudaStream_t s) {
+    if (bf16) maxpool_fwd_kernel<__nv_bfloat16><<<dim3(ew_grid(max_elems), nprob), 256, 0, s>>>(d);
+    else maxpool_fwd_kernel<float><<<dim3(ew_grid(max_elems), nprob), 256, 0, s>>>(d);
+}
+void launch_maxpool_bwd(const PoolProb* d, int nprob, long long max_elems, bool bf16, cudaStream_t s) {
+    if (bf16) maxpool_bwd_kernel<__nv_bfloat16><<<dim3(ew_grid(max_elems), nprob), 256, 0, s>>>(d);
+    else maxpool_bwd_kernel<float><<<dim3(ew_grid(max_elems), nprob), 256, 0, s>>>(d);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Global average pool, linear head, mean softmax cross-entropy and their gradients (fp32 math)
+// ------------------------------------------------------------------------------------------------
+template <class T>
+__global__ void avgpool_kernel(const HeadProb* __restrict__ probs) {
+    const HeadProb& p = probs[blockIdx.y];
+    const int n = p.B * p.C;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+        const int c = i % p.C, b = i / p.C;
+        float s = 0.f;
+        for (int k = 0; k < p.HW; ++k) s += ldf<T>(p.a, ((long long)b * p.HW + k) * p.C + c);
+        p.pooled[i] = s / (float)p.HW;
+    }
+}
+// one warp per logit
+__global__ void head_logits_kernel(const HeadProb* __restrict__ probs) {
+    const HeadProb& p = probs[blockIdx.y];
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) / 32, lane = threadIdx.x % 32;
+    const int nw = gridDim.x * blockDim.x / 32;
+    for (int o = warp; o < p.B * p.classes; o += nw) {
+        const int k = o % p.classes, b = o / p.classes;
+        float s = 0.f;
+        for (int c = lane; c < p.C; c += 32) s = fmaf(p.w[(long long)k * p.C + c], p.pooled[(long long)b * p.C + c], s);
+        for (int d = 16; d; d >>= 1) s += __shfl_xor_sync(0xffffffffu, s, d);
+        if (lane == 0) { s += p.b[k]; p.logits[o] = s; if (p.logits_user) p.logits_user[o] = s; }
+    }
+}
+// one CTA per problem; one warp per sample, samples strided over the warps; fixed-order loss sum
+__global__ void __launch_bounds__(256) loss_kernel(const HeadProb* __restrict__ probs) {
+    const HeadProb& p = probs[blockIdx.x];
+    __shared__ float sl[1024]; __shared__ int sc[1024];
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    for (int b = warp; b < p.B; b += 8) {
+        const float* lg = p.logits + (long long)b * p.classes;
+        float mx = -INFINITY; int arg = 0x7fffffff;
+        for (int k = lane; k < p.classes; k += 32) { float v = lg[k]; if (v > mx) { mx = v; arg = k; } }
+        for (int d = 16; d; d >>= 1) {
+            float om = __shfl_xor_sync(0xffffffffu, mx, d); int oa = __shfl_xor_sync(0xffffffffu, arg, d);
+            if (om > mx || (om == mx && oa < arg)) { mx = om; arg = oa; }
+        }
+        float se = 0.f;
+        for (int k = lane; k < p.classes; k += 32) se += expf(lg[k] - mx);
+        for (int d = 16; d; d >>= 1) se += __shfl_xor_sync(0xffffffffu, se, d);
+        const float lse = mx + logf(se);
+        const int y = p.labels ? p.labels[b] : -1;
+        if (p.dlogits)
+            for (int k = lane; k < p.classes; k += 32)
+                p.dlogits[(long long)b * p.classes + k] = (expf(lg[k] - lse) - (k == y ? 1.f : 0.f)) / (float)p.B;
+        if (lane == 0) { sl[b] = y >= 0 ? lse - lg[y] : 0.f; sc[b] = (arg == y); }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float s = 0.f; int c = 0;
+        for (int b = 0; b < p.B; ++b) { s += sl[b]; c += sc[b]; }
+        s /= (float)p.B;
+        if (p.loss) *p.loss = s;
+        if (p.loss_user) *p.loss_user = s;
+        if (p.correct) *p.correct = c;
+    }
+}
+__global__ void head_bwd_w_kernel(const HeadProb* __restrict__ probs) {
+    const HeadProb& p = probs[blockIdx.y];
+    const int n = p.classes * p.C;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n + p.classes; i += gridDim.x * blockDim.x) {
+        float s = 0.f;
+        if (i < n) { const int c = i % p.C, k = i / p.C;
+            for (int b = 0; b < p.B; ++b) s = fmaf(p.dlogits[(long long)b * p.classes + k], p.pooled[(long long)b * p.C + c], s);
+            p.dw[i] = s;
+        } else { const int k = i - n;
+            for (int b = 0; b < p.B; ++b) s += p.dlogits[(long long)b * p.classes + k];
+            p.db[k] = s; }
+    }
+}
+__global__ void head_bwd_x_kernel(const HeadProb* __restrict__ probs) {
+    const HeadProb& p = probs[blockIdx.y];
+    const int n = p.B * p.C;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+        const int c = i % p.C, b = i / p.C;
+        float s = 0.f;
+        for (int k = 0; k < p.classes; ++k) s = fmaf(p.dlogits[(long long)b * p.classes + k], p.w[(long long)k * p.C + c], s);
+        p.dpooled[i] = s / (float)p.HW;
+    }
+}
+template <class T>
+__global__ void avgpool_bwd_kernel(const HeadProb* __restrict__ probs) {
+    const HeadProb& p = probs[blockIdx.y];
+    const long long n = (long long)p.B * p.HW * p.C;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+        const int c = (int)(i % p.C); const long long b = i / ((long long)p.HW * p.C);
+        stf<T>(p.da, i, p.dpooled[b * p.C + c]);
+    }
+}
+
+void launch_head_fwd(const HeadProb* d, int nprob, int maxB, int maxC, int max_classes, bool bf16, cudaStream_t s) {
+    if (bf16) avgpool_kernel<__nv_bfloat16><<<dim3(ew_grid((long long)maxB * maxC), nprob), 256, 0, s>>>(d);
+    else avgpool_kernel<float><<<dim3(ew_grid((long long)maxB * maxC), nprob), 256, 0, s>>>(d);
+    head_logits_kernel<<<dim3(ew_grid((long long)maxB * max_classes * 32), nprob), 256, 0, s>>>(d);
+    loss_kernel<<<nprob, 256, 0, s>>>(d);
+}
+void launch_head_bwd(const HeadProb* d, int nprob, int maxB, int maxC, int max_classes, long long max_elems,
+                     bool bf16, cudaStream_t s) {
+    head_bwd_w_kernel<<<dim3(ew_grid((long long)max_classes * (maxC + 1)), nprob), 256, 0, s>>>(d);
+    head_bwd_x_kernel<<<dim3(ew_grid((long long)maxB * maxC), nprob), 256, 0, s>>>(d);
+    if (bf16) avgpool_bwd_kernel<__nv_bfloat16><<<dim3(ew_grid(max_elems), nprob), 256, 0, s>>>(d);
+    else avgpool_bwd_kernel<float><<<dim3(ew_grid(max_elems), nprob), 256, 0, s>>>(d);
+}
+
+}  // namespace resist

@@ -1,0 +1,535 @@
+// Launch plans of the local training step (Algorithm 1, inner loop) and of evaluation (Sec. 2.6).
+// For a given partition and batch size every sub-ResNet is unrolled into a list of keyed operations;
+// operations of different sub-ResNets with the same key become ONE grouped launch whose blockIdx.y
+// selects the sub-ResNet, so that S shallow networks fill the GPU together.
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include "runtime.h"
+
+namespace resist {
+
+void* ctx_alloc(resist_ctx* ctx, size_t bytes);
+void ctx_free(resist_ctx* ctx, void* p);
+void held_segments(const resist_ctx* ctx, int sub, uint32_t bit, bool buffers, std::vector<Segment>& out, long long& chunks);
+int ensure_param_arrays(resist_ctx* ctx, int S);
+int ensure_seg_table(resist_ctx* ctx, int n);
+bool conv_tc_supported(const ConvProb& p, int mode);                                   // conv_tc.cu
+void launch_conv_tc(const ConvProb* d, int nprob, int max_tiles, int mode, cudaStream_t s);
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+static int out_dim(int h, int k, int stride) { return (h + 2 * ((k - 1) / 2) - k) / stride + 1; }
+
+void free_plan(resist_ctx* ctx, Plan& p) {
+    ctx_free(ctx, p.d_blob);
+    p = Plan();
+}
+
+struct PatchArgs {
+    const void* images[RESIST_MAX_SUBNETS]; const int* labels[RESIST_MAX_SUBNETS];
+    float* loss_out; float* logits_out; int* correct;
+};
+__global__ void patch_kernel(const PatchSite* sites, int n, PatchArgs a) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const PatchSite s = sites[i];
+    void* v = nullptr;
+    if (s.what == 0) v = (void*)a.images[s.sub];
+    else if (s.what == 1) v = (void*)a.labels[s.sub];
+    else if (s.what == 2) v = a.loss_out ? (void*)(a.loss_out + s.sub) : nullptr;
+    else if (s.what == 3) v = (void*)a.logits_out;
+    else v = (void*)a.correct;
+    *s.where = v;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Unrolling one sub-ResNet into operations.  Device memory comes from a bump allocator over the
+// sub-ResNet's workspace slice; with base == nullptr the pass only measures.
+// ------------------------------------------------------------------------------------------------
+struct Builder {
+    resist_ctx* ctx; int B; int sub; int copy; bool eval; int slot_for_patch;
+    char* base; size_t off = 0; size_t es;
+    std::vector<Op>* ops;
+    // scratch shared by the operations of this sub-ResNet (they run one after another)
+    double* bn_partial = nullptr; float* wgrad_partial = nullptr; size_t bn_partial_need = 0, wgrad_partial_need = 0;
+    char* gbuf[6] = {}; bool gused[6] = {}; size_t gbig = 0;
+    float* logits = nullptr;
+    long long flops = 0; int n_tc = 0, n_cc = 0;
+
+    void* take(size_t bytes) { off = align_up(off, 256); void* p = base ? base + off : nullptr; off += bytes; return p; }
+    void* act(long long elems) { size_t b = (size_t)elems * es; if (b > gbig) gbig = b; return take(b); }
+    int gtake() { for (int i = 0; i < 6; ++i) if (!gused[i]) { gused[i] = true; return i; } return -1; }
+    void grel(int i) { if (i >= 0) gused[i] = false; }
+
+    float* W() const { return ctx->pa.w + (long long)copy * ctx->pa.n; }
+    float* G() const { return ctx->pa.g + (long long)copy * ctx->pa.n; }
+    float* Bf() const { return ctx->pa.buf + (long long)copy * ctx->pa.nbuf; }
+    const void* CW(long long o) const {           // the convolutions' copy of the weights
+        if (ctx->opts.dtype == RESIST_BF16) return ctx->pa.wb + (long long)copy * ctx->pa.n + o;
+        return W() + o;
+    }
+
+    void conv(long long key, int mode, const void* a, const ConvRef& cr, const void* dy_or_null, const void* add, void* out,
+              int N, int H, int Wd, float scale, bool patch = false) {
+        Op op{}; op.key = key; op.sub = sub; op.patch_images = patch ? 1 : 0;
+        op.kind = mode == CONV_FWD ? OP_CONV_FWD : mode == CONV_DGRAD ? OP_CONV_DGRAD : OP_CONV_WGRAD;
+        ConvProb& p = op.conv;
+        p.N = N; p.H = H; p.W = Wd; p.C = cr.cin; p.K = cr.cout; p.ksz = cr.k; p.stride = cr.stride; p.pad = (cr.k - 1) / 2;
+        p.P = out_dim(H, cr.k, cr.stride); p.Q = out_dim(Wd, cr.k, cr.stride);
+        p.scale = scale; p.add = add; p.out = out; p.partial = nullptr; p.stat_partial = nullptr;
+        const long long rows_out = (long long)N * p.P * p.Q, rows_in = (long long)N * H * Wd;
+        if (mode == CONV_FWD) { p.act = a; p.wgt = CW(cr.w); p.M = (int)rows_out; p.Ncol = p.K; p.Kred = p.ksz * p.ksz * p.C; }
+        else if (mode == CONV_DGRAD) { p.act = dy_or_null; p.wgt = CW(cr.w); p.M = (int)rows_in; p.Ncol = p.C; p.Kred = p.ksz * p.ksz * p.K; }
+        else { p.act = a; p.wgt = dy_or_null; p.M = p.K; p.Ncol = p.ksz * p.ksz * p.C; p.Kred = (int)rows_out; p.out = G() + cr.w; }
+        p.tiles_m = (p.M + 63) / 64; p.tiles_n = (p.Ncol + 63) / 64; p.splits = 1;
+        const int ktiles = (p.Kred + 15) / 16; p.ktiles_per_split = ktiles;
+        flops += 2LL * rows_out * p.K * p.ksz * p.ksz * p.C;
+        op.backend = (ctx->opts.dtype == RESIST_BF16 && ctx->opts.conv_backend == RESIST_CONV_AUTO && conv_tc_supported(p, mode)) ? 1 : 0;
+        if (op.backend) ++n_tc; else ++n_cc;
+        if (mode == CONV_WGRAD && !op.backend) {
+            const int tiles = p.tiles_m * p.tiles_n;
+            int want = (2 * ctx->sm_count + tiles - 1) / tiles; if (want > 64) want = 64; if (want > ktiles) want = ktiles; if (want < 1) want = 1;
+            p.ktiles_per_split = (ktiles + want - 1) / want; p.splits = (ktiles + p.ktiles_per_split - 1) / p.ktiles_per_split;
+            if (p.splits > 1) {
+                wgrad_partial_need = std::max(wgrad_partial_need, (size_t)p.splits * p.M * p.Ncol * 4);
+                p.partial = wgrad_partial;
+            }
+        }
+        ops->push_back(op);
+        if (mode == CONV_WGRAD && p.splits > 1) { Op r = op; r.key = key + 1; r.kind = OP_SPLITK; r.patch_images = 0; ops->push_back(r); }
+    }
+
+    // forward BN+ReLU: statistics (or running statistics in evaluation) then apply
+    float* bn_fwd(long long key, const void* x, void* a, const BNRef& r, long long m) {
+        float* stat = (float*)take((size_t)4 * r.c * 4);
+        Op op{}; op.key = key; op.sub = sub; op.kind = OP_BN_STATS;
+        BnProb& p = op.bn;
+        p.x = x; p.a = a; p.gamma = W() + r.g; p.beta = W() + r.b; p.dgamma = G() + r.g; p.dbeta = G() + r.b;
+        p.run_mean = Bf() + r.buf; p.run_var = Bf() + r.buf + r.c; p.stat = stat; p.m = m; p.C = r.c;
+        p.eps = ctx->opts.bn_eps; p.momentum = ctx->opts.bn_momentum; p.eval = eval ? 1 : 0;
+        const int nl = r.c < 256 ? r.c : 256, R = 256 / nl;
+        long long rpc = (long long)R * 32; const long long lim = (m + 1023) / 1024; if (rpc < lim) rpc = lim;
+        p.rows_per_chunk = (int)rpc; p.chunks = (int)((m + rpc - 1) / rpc);
+        bn_partial_need = std::max(bn_partial_need, (size_t)p.chunks * 2 * r.c * 8);
+        p.partial = bn_partial;
+        ops->push_back(op);
+        op.key = key + 1; op.kind = OP_BN_APPLY; ops->push_back(op);
+        return stat;
+    }
+    void bn_bwd(long long key, const void* x, const void* da, void* dx, const void* add, const BNRef& r, float* stat, long long m) {
+        Op op{}; op.key = key; op.sub = sub; op.kind = OP_BN_BWD_REDUCE;
+        BnProb& p = op.bn;
+        p.x = x; p.da = da; p.dx = dx; p.add = add; p.gamma = W() + r.g; p.beta = W() + r.b; p.dgamma = G() + r.g; p.dbeta = G() + r.b;
+        p.stat = stat; p.m = m; p.C = r.c; p.eps = ctx->opts.bn_eps; p.momentum = ctx->opts.bn_momentum; p.eval = 0;
+        const int nl = r.c < 256 ? r.c : 256, R = 256 / nl;
+        long long rpc = (long long)R * 32; const long long lim = (m + 1023) / 1024; if (rpc < lim) rpc = lim;
+        p.rows_per_chunk = (int)rpc; p.chunks = (int)((m + rpc - 1) / rpc);
+        p.partial = bn_partial;
+        ops->push_back(op);
+        op.key = key + 1; op.kind = OP_BN_BWD_APPLY; ops->push_back(op);
+    }
+};
+
+struct BlockMem { int H, W, Ho, Wo; void *x, *a1, *y1, *a2, *y2, *a3; float* stat[3]; };
+
+// Returns the workspace bytes this sub-ResNet needs.  `present` has one entry per block.
+static size_t unroll_subnet(resist_ctx* ctx, Builder& bd, const std::vector<char>& present, float inv_S) {
+    const resist_arch& A = ctx->arch; const Layout& L = ctx->L; const int B = bd.B; const int nb = A.num_blocks;
+    const long long KEY_BLOCK0 = 100, FWD_END = KEY_BLOCK0 + 20LL * nb, BWD0 = FWD_END + 10, BWD_BLOCK0 = BWD0 + 10;
+    const long long BWD_END = BWD_BLOCK0 + 40LL * nb;
+    // scratch first, so that its addresses do not depend on the network above it
+    bd.bn_partial = (double*)bd.take(bd.bn_partial_need);
+    bd.wgrad_partial = (float*)bd.take(bd.wgrad_partial_need);
+    if (!bd.eval) for (int i = 0; i < 6; ++i) bd.gbuf[i] = (char*)bd.take(bd.gbig);
+
+    // ---- stem
+    const int Hs = out_dim(A.in_h, A.stem_k, A.stem_stride), Ws = out_dim(A.in_w, A.stem_k, A.stem_stride);
+    const long long m_stem = (long long)B * Hs * Ws;
+    void* stem_y = bd.act(m_stem * A.stem_cout); void* stem_a = nullptr; void* stem_p = nullptr; int* stem_arg = nullptr; float* stem_stat = nullptr;
+    bd.conv(0, CONV_FWD, nullptr, L.stem, nullptr, nullptr, stem_y, B, A.in_h, A.in_w, 1.f, true);
+    void* cur = stem_y; int cH = Hs, cW = Ws, cC = A.stem_cout;
+    if (A.stem_bn_relu) { stem_a = bd.act(m_stem * cC); stem_stat = bd.bn_fwd(1, stem_y, stem_a, L.stem_bn, m_stem); cur = stem_a; }
+    if (A.stem_maxpool) {
+        const int Hp = out_dim(cH, 3, 2), Wp = out_dim(cW, 3, 2);
+        stem_p = bd.act((long long)B * Hp * Wp * cC); stem_arg = (int*)bd.take((size_t)B * Hp * Wp * cC * 4);
+        Op op{}; op.key = 3; op.sub = bd.sub; op.kind = OP_POOL_FWD;
+        op.pool = PoolProb{cur, stem_p, stem_arg, nullptr, nullptr, B, cH, cW, cC, Hp, Wp};
+        bd.ops->push_back(op);
+        cur = stem_p; cH = Hp; cW = Wp;
+    }
+
+    // ---- blocks
+    std::vector<BlockMem> bm(nb); std::vector<int> order;
+    for (int b = 0; b < nb; ++b) if (present[b]) order.push_back(b);
+    for (size_t slot = 0; slot < order.size(); ++slot) {
+        const int b = order[slot]; const resist_block& K = ctx->blocks[b]; const BlockRef& r = L.blk[b]; BlockMem& s = bm[b];
+        const long long key = KEY_BLOCK0 + 20LL * (long long)slot;
+        s.H = cH; s.W = cW; s.Ho = out_dim(cH, 3, K.stride); s.Wo = out_dim(cW, 3, K.stride);
+        const long long m_in = (long long)B * s.H * s.W, m_out = (long long)B * s.Ho * s.Wo;
+        const float scale = (bd.eval && K.partitionable) ? inv_S : 1.f;
+        s.x = cur; s.a1 = bd.act(m_in * K.cin);
+        s.stat[0] = bd.bn_fwd(key + 0, s.x, s.a1, r.bn[0], m_in);
+        const void* sc = s.x;
+        if (K.has_projection) { void* scb = bd.act(m_out * K.cout); bd.conv(key + 2, CONV_FWD, s.a1, r.proj, nullptr, nullptr, scb, B, s.H, s.W, 1.f); sc = scb; }
+        void* out = bd.act(m_out * K.cout);
+        if (K.kind == RESIST_BASIC) {
+            s.y1 = bd.act(m_out * K.cout); s.a2 = bd.act(m_out * K.cout);
+            bd.conv(key + 3, CONV_FWD, s.a1, r.conv[0], nullptr, nullptr, s.y1, B, s.H, s.W, 1.f);
+            s.stat[1] = bd.bn_fwd(key + 4, s.y1, s.a2, r.bn[1], m_out);
+            bd.conv(key + 6, CONV_FWD, s.a2, r.conv[1], nullptr, sc, out, B, s.Ho, s.Wo, scale);
+        } else {
+            s.y1 = bd.act(m_in * K.cmid); s.a2 = bd.act(m_in * K.cmid); s.y2 = bd.act(m_out * K.cmid); s.a3 = bd.act(m_out * K.cmid);
+            bd.conv(key + 3, CONV_FWD, s.a1, r.conv[0], nullptr, nullptr, s.y1, B, s.H, s.W, 1.f);
+            s.stat[1] = bd.bn_fwd(key + 4, s.y1, s.a2, r.bn[1], m_in);
+            bd.conv(key + 6, CONV_FWD, s.a2, r.conv[1], nullptr, nullptr, s.y2, B, s.H, s.W, 1.f);
+            s.stat[2] = bd.bn_fwd(key + 7, s.y2, s.a3, r.bn[2], m_out);
+            bd.conv(key + 9, CONV_FWD, s.a3, r.conv[2], nullptr, sc, out, B, s.Ho, s.Wo, scale);
+        }
+        cur = out; cH = s.Ho; cW = s.Wo; cC = K.cout;
+    }
+
+    // ---- final BN + ReLU, pool, head, loss
+    const long long mF = (long long)B * cH * cW; const int HW = cH * cW;
+    void* xF = cur; void* aF = bd.act(mF * cC);
+    float* statF = bd.bn_fwd(FWD_END, xF, aF, L.final_bn, mF);
+    HeadProb hp{};
+    hp.a = aF; hp.w = bd.W() + L.head_w; hp.b = bd.W() + L.head_b; hp.dw = bd.G() + L.head_w; hp.db = bd.G() + L.head_b;
+    hp.pooled = (float*)bd.take((size_t)B * cC * 4); hp.dpooled = (float*)bd.take((size_t)B * cC * 4);
+    hp.logits = (float*)bd.take((size_t)B * A.classes * 4); hp.dlogits = bd.eval ? nullptr : (float*)bd.take((size_t)B * A.classes * 4);
+    hp.loss = (float*)bd.take(256); hp.B = B; hp.HW = HW; hp.C = cC; hp.classes = A.classes;
+    bd.logits = hp.logits;
+    { Op op{}; op.key = FWD_END + 2; op.sub = bd.sub; op.kind = OP_HEAD_FWD; op.head = hp; bd.ops->push_back(op); }
+    if (bd.eval) return bd.off;
+
+    // ---- backward
+    int g_cur = bd.gtake();                                   // gradient w.r.t. the current tensor
+    hp.da = bd.gbuf[g_cur];
+    { Op op{}; op.key = BWD0; op.sub = bd.sub; op.kind = OP_HEAD_BWD; op.head = hp; bd.ops->push_back(op); }
+    { int g = bd.gtake(); bd.bn_bwd(BWD0 + 1, xF, bd.gbuf[g_cur], bd.gbuf[g], nullptr, L.final_bn, statF, mF); bd.grel(g_cur); g_cur = g; }
+    for (int slot = (int)order.size() - 1; slot >= 0; --slot) {
+        const int b = order[slot]; const resist_block& K = ctx->blocks[b]; const BlockRef& r = L.blk[b]; BlockMem& s = bm[b];
+        const long long key = BWD_BLOCK0 + 40LL * ((long long)order.size() - 1 - slot);
+        const long long m_in = (long long)B * s.H * s.W, m_out = (long long)B * s.Ho * s.Wo;
+        const char* dout = bd.gbuf[g_cur];
+        int g_sc = -1;
+        if (K.has_projection) {
+            bd.conv(key + 0, CONV_WGRAD, s.a1, r.proj, dout, nullptr, nullptr, B, s.H, s.W, 1.f);
+            g_sc = bd.gtake();
+            bd.conv(key + 2, CONV_DGRAD, nullptr, r.proj, dout, nullptr, bd.gbuf[g_sc], B, s.H, s.W, 1.f);
+        }
+        int g_da1 = -1;
+        if (K.kind == RESIST_BASIC) {
+            const int g_da2 = bd.gtake();
+            bd.conv(key + 3, CONV_WGRAD, s.a2, r.conv[1], dout, nullptr, nullptr, B, s.Ho, s.Wo, 1.f);
+            bd.conv(key + 5, CONV_DGRAD, nullptr, r.conv[1], dout, nullptr, bd.gbuf[g_da2], B, s.Ho, s.Wo, 1.f);
+            const int g_dy1 = bd.gtake();
+            bd.bn_bwd(key + 6, s.y1, bd.gbuf[g_da2], bd.gbuf[g_dy1], nullptr, r.bn[1], s.stat[1], m_out);
+            bd.grel(g_da2);
+            bd.conv(key + 8, CONV_WGRAD, s.a1, r.conv[0], bd.gbuf[g_dy1], nullptr, nullptr, B, s.H, s.W, 1.f);
+            g_da1 = bd.gtake();
+            bd.conv(key + 10, CONV_DGRAD, nullptr, r.conv[0], bd.gbuf[g_dy1], g_sc >= 0 ? bd.gbuf[g_sc] : nullptr, bd.gbuf[g_da1], B, s.H, s.W, 1.f);
+            bd.grel(g_dy1);
+        } else {
+            const int g_da3 = bd.gtake();
+            bd.conv(key + 3, CONV_WGRAD, s.a3, r.conv[2], dout, nullptr, nullptr, B, s.Ho, s.Wo, 1.f);
+            bd.conv(key + 5, CONV_DGRAD, nullptr, r.conv[2], dout, nullptr, bd.gbuf[g_da3], B, s.Ho, s.Wo, 1.f);
+            const int g_dy2 = bd.gtake();
+            bd.bn_bwd(key + 6, s.y2, bd.gbuf[g_da3], bd.gbuf[g_dy2], nullptr, r.bn[2], s.stat[2], m_out);
+            bd.grel(g_da3);
+            bd.conv(key + 8, CONV_WGRAD, s.a2, r.conv[1], bd.gbuf[g_dy2], nullptr, nullptr, B, s.H, s.W, 1.f);
+            const int g_da2 = bd.gtake();
+            bd.conv(key + 10, CONV_DGRAD, nullptr, r.conv[1], bd.gbuf[g_dy2], nullptr, bd.gbuf[g_da2], B, s.H, s.W, 1.f);
+            bd.grel(g_dy2);
+            const int g_dy1 = bd.gtake();
+            bd.bn_bwd(key + 11, s.y1, bd.gbuf[g_da2], bd.gbuf[g_dy1], nullptr, r.bn[1], s.stat[1], m_in);
+            bd.grel(g_da2);
+            bd.conv(key + 13, CONV_WGRAD, s.a1, r.conv[0], bd.gbuf[g_dy1], nullptr, nullptr, B, s.H, s.W, 1.f);
+            g_da1 = bd.gtake();
+            bd.conv(key + 15, CONV_DGRAD, nullptr, r.conv[0], bd.gbuf[g_dy1], g_sc >= 0 ? bd.gbuf[g_sc] : nullptr, bd.gbuf[g_da1], B, s.H, s.W, 1.f);
+            bd.grel(g_dy1);
+        }
+        bd.grel(g_sc);
+        const int g_dx = bd.gtake();
+        // identity skip: the block's input also receives dout directly
+        bd.bn_bwd(key + 20, s.x, bd.gbuf[g_da1], bd.gbuf[g_dx], K.has_projection ? nullptr : dout, r.bn[0], s.stat[0], m_in);
+        bd.grel(g_da1); bd.grel(g_cur); g_cur = g_dx;
+    }
+    // ---- stem backward (no input gradient)
+    if (A.stem_maxpool) {
+        const int g = bd.gtake();
+        Op op{}; op.key = BWD_END; op.sub = bd.sub; op.kind = OP_POOL_BWD;
+        op.pool = PoolProb{stem_a ? stem_a : stem_y, nullptr, stem_arg, bd.gbuf[g_cur], bd.gbuf[g], B, Hs, Ws, A.stem_cout, cH, cW};
+        op.pool.P = out_dim(Hs, 3, 2); op.pool.Q = out_dim(Ws, 3, 2);
+        bd.ops->push_back(op); bd.grel(g_cur); g_cur = g;
+    }
+    if (A.stem_bn_relu) { const int g = bd.gtake(); bd.bn_bwd(BWD_END + 1, stem_y, bd.gbuf[g_cur], bd.gbuf[g], nullptr, L.stem_bn, stem_stat, m_stem); bd.grel(g_cur); g_cur = g; }
+    bd.conv(BWD_END + 3, CONV_WGRAD, nullptr, L.stem, bd.gbuf[g_cur], nullptr, nullptr, B, A.in_h, A.in_w, 1.f, true);
+    return bd.off;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Workspace: one slice per sub-ResNet, all slices the size of the largest.
+// ------------------------------------------------------------------------------------------------
+struct Needs { size_t bn_partial = 0, wgrad_partial = 0, gbig = 0, total = 0; };
+
+static Needs measure_subnet(resist_ctx* ctx, int sub, int copy, const std::vector<char>& present, int B, bool eval, float inv_S) {
+    std::vector<Op> scratch;
+    Builder b1{ctx, B, sub, copy, eval, 0, nullptr}; b1.es = ctx->opts.dtype == RESIST_BF16 ? 2 : 4; b1.ops = &scratch;
+    unroll_subnet(ctx, b1, present, inv_S);
+    Needs n; n.bn_partial = b1.bn_partial_need; n.wgrad_partial = b1.wgrad_partial_need; n.gbig = b1.gbig;
+    scratch.clear();
+    Builder b2{ctx, B, sub, copy, eval, 0, nullptr}; b2.es = b1.es; b2.ops = &scratch;
+    b2.bn_partial_need = n.bn_partial; b2.wgrad_partial_need = n.wgrad_partial; b2.gbig = n.gbig;
+    n.total = align_up(unroll_subnet(ctx, b2, present, inv_S), 256);
+    return n;
+}
+
+static std::vector<char> present_of(const resist_ctx* ctx, int sub) {
+    std::vector<char> p(ctx->arch.num_blocks);
+    for (int b = 0; b < ctx->arch.num_blocks; ++b) p[b] = (ctx->mask[b] >> sub & 1u) ? 1 : 0;
+    return p;
+}
+
+static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool single, cudaStream_t st) {
+    std::stable_sort(ops.begin(), ops.end(), [](const Op& a, const Op& b) { return a.key < b.key; });
+    std::vector<ConvProb> conv; std::vector<BnProb> bn; std::vector<PoolProb> pool; std::vector<HeadProb> head;
+    struct HostSite { int arr; int idx; int field; int what; int sub; };
+    std::vector<HostSite> sites;
+    plan.launches.clear();
+    for (size_t i = 0; i < ops.size();) {
+        size_t j = i;
+        while (j < ops.size() && ops[j].key == ops[i].key && ops[j].kind == ops[i].kind && ops[j].backend == ops[i].backend) ++j;
+        Launch L{}; L.kind = ops[i].kind; L.backend = ops[i].backend; L.count = (int)(j - i);
+        for (size_t k = i; k < j; ++k) {
+            const Op& o = ops[k]; const int slot = single ? 0 : o.sub;
+            switch (o.kind) {
+                case OP_CONV_FWD: case OP_CONV_DGRAD: case OP_CONV_WGRAD: case OP_SPLITK: {
+                    if (k == i) L.first = (int)conv.size();
+                    if (o.patch_images) sites.push_back({0, (int)conv.size(), 0, 0, slot});
+                    conv.push_back(o.conv);
+                    const ConvProb& p = o.conv;
+                    if (o.kind == OP_SPLITK) L.max_elems = std::max<long long>(L.max_elems, (long long)p.M * p.Ncol);
+                    else L.gx = std::max(L.gx, p.tiles_m * p.tiles_n * p.splits);
+                    break; }
+                case OP_BN_STATS: case OP_BN_APPLY: case OP_BN_BWD_REDUCE: case OP_BN_BWD_APPLY: {
+                    if (k == i) L.first = (int)bn.size();
+                    bn.push_back(o.bn);
+                    L.gx = std::max(L.gx, o.bn.chunks); L.max_c = std::max(L.max_c, o.bn.C);
+                    L.max_elems = std::max<long long>(L.max_elems, o.bn.m * o.bn.C);
+                    break; }
+                case OP_POOL_FWD: case OP_POOL_BWD: {
+                    if (k == i) L.first = (int)pool.size();
+                    pool.push_back(o.pool);
+                    const PoolProb& p = o.pool;
+                    L.max_elems = std::max<long long>(L.max_elems, (long long)p.N * (o.kind == OP_POOL_FWD ? p.P * p.Q : p.H * p.W) * p.C);
+                    break; }
+                case OP_HEAD_FWD: case OP_HEAD_BWD: {
+                    if (k == i) L.first = (int)head.size();
+                    sites.push_back({1, (int)head.size(), 0, 1, slot});
+                    if (o.kind == OP_HEAD_FWD) { sites.push_back({1, (int)head.size(), 1, 2, slot});
+                        if (plan.sub == -2) { sites.push_back({1, (int)head.size(), 2, 3, 0}); sites.push_back({1, (int)head.size(), 3, 4, 0}); } }
+                    head.push_back(o.head);
+                    const HeadProb& p = o.head;
+                    L.max_b = std::max(L.max_b, p.B); L.max_c = std::max(L.max_c, p.C); L.max_classes = std::max(L.max_classes, p.classes);
+                    L.max_elems = std::max<long long>(L.max_elems, (long long)p.B * p.HW * p.C);
+                    break; }
+            }
+        }
+        plan.launches.push_back(L);
+        i = j;
+    }
+    // one device blob: conv | bn | pool | head | sites | sgd segments
+    std::vector<Segment> segs; long long chunks = 0;
+    if (plan.sub >= 0) held_segments(ctx, plan.sub, 1u << plan.sub, false, segs, chunks);
+    else if (plan.sub == -1) for (int s = 0; s < ctx->S; ++s) held_segments(ctx, s, 1u << s, false, segs, chunks);
+    size_t off = 0;
+    const size_t o_conv = off; off += align_up(conv.size() * sizeof(ConvProb), 256);
+    const size_t o_bn = off;   off += align_up(bn.size() * sizeof(BnProb), 256);
+    const size_t o_pool = off; off += align_up(pool.size() * sizeof(PoolProb), 256);
+    const size_t o_head = off; off += align_up(head.size() * sizeof(HeadProb), 256);
+    const size_t o_site = off; off += align_up(sites.size() * sizeof(PatchSite), 256);
+    const size_t o_seg = off;  off += align_up(segs.size() * sizeof(Segment), 256);
+    ctx_free(ctx, plan.d_blob);
+    plan.d_blob = ctx_alloc(ctx, off + 256); plan.blob_bytes = off;
+    if (!plan.d_blob) { ctx->err = "allocator returned NULL for the launch plan"; return RESIST_ENOMEM; }
+    char* base = (char*)plan.d_blob;
+    plan.d_conv = (ConvProb*)(base + o_conv); plan.d_bn = (BnProb*)(base + o_bn); plan.d_pool = (PoolProb*)(base + o_pool);
+    plan.d_head = (HeadProb*)(base + o_head); plan.d_sites = (PatchSite*)(base + o_site); plan.d_sgd = (Segment*)(base + o_seg);
+    std::vector<PatchSite> dsites;
+    for (const HostSite& h : sites) {
+        PatchSite s{}; s.what = h.what; s.sub = h.sub;
+        if (h.arr == 0) s.where = (void**)&plan.d_conv[h.idx].act;
+        else if (h.field == 0) s.where = (void**)&plan.d_head[h.idx].labels;
+        else if (h.field == 1) s.where = (void**)&plan.d_head[h.idx].loss_user;
+        else if (h.field == 2) s.where = (void**)&plan.d_head[h.idx].logits_user;
+        else s.where = (void**)&plan.d_head[h.idx].correct;
+        dsites.push_back(s);
+    }
+    std::vector<char> host(off, 0);
+    if (!conv.empty()) memcpy(host.data() + o_conv, conv.data(), conv.size() * sizeof(ConvProb));
+    if (!bn.empty()) memcpy(host.data() + o_bn, bn.data(), bn.size() * sizeof(BnProb));
+    if (!pool.empty()) memcpy(host.data() + o_pool, pool.data(), pool.size() * sizeof(PoolProb));
+    if (!head.empty()) memcpy(host.data() + o_head, head.data(), head.size() * sizeof(HeadProb));
+    if (!dsites.empty()) memcpy(host.data() + o_site, dsites.data(), dsites.size() * sizeof(PatchSite));
+    if (!segs.empty()) memcpy(host.data() + o_seg, segs.data(), segs.size() * sizeof(Segment));
+    cudaError_t e = cudaMemcpyAsync(plan.d_blob, host.data(), off, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) { ctx->err = std::string("plan upload: ") + cudaGetErrorString(e); return RESIST_ECUDA; }
+    plan.nsites = (int)dsites.size(); plan.n_sgd_seg = (int)segs.size(); plan.sgd_chunks = chunks;
+    return RESIST_OK;
+}
+
+static int ensure_workspace(resist_ctx* ctx, int B, std::vector<Needs>& needs) {
+    needs.resize(ctx->S);
+    size_t slice = 0;
+    for (int s = 0; s < ctx->S; ++s) { needs[s] = measure_subnet(ctx, s, s, present_of(ctx, s), B, false, 1.f); slice = std::max(slice, needs[s].total); }
+    if (slice <= ctx->ws_slice && (size_t)ctx->S * ctx->ws_slice <= ctx->ws_bytes) return RESIST_OK;
+    if (slice <= ctx->ws_slice) slice = ctx->ws_slice;
+    slice = align_up(slice + slice / 16, 1 << 20);               // a little slack: partitions differ slightly in size
+    cudaDeviceSynchronize();
+    ctx_free(ctx, ctx->d_ws); ctx->d_ws = nullptr; ctx->ws_bytes = 0; ctx->ws_slice = 0;
+    for (Plan& p : ctx->plans) p.valid = false;
+    ctx->d_ws = ctx_alloc(ctx, slice * ctx->S);
+    if (!ctx->d_ws) { ctx->err = "allocator returned NULL for the activation workspace"; return RESIST_ENOMEM; }
+    ctx->ws_bytes = slice * ctx->S; ctx->ws_slice = slice;
+    return RESIST_OK;
+}
+
+// sub >= 0: one sub-ResNet; sub == -1: all S grouped
+static int build_plan(resist_ctx* ctx, Plan& plan, int sub, int B, cudaStream_t st) {
+    std::vector<Needs> needs;
+    int rc = ensure_workspace(ctx, B, needs);
+    if (rc) return rc;
+    std::vector<Op> ops; plan.info = resist_step_info{};
+    const int s0 = sub >= 0 ? sub : 0, s1 = sub >= 0 ? sub + 1 : ctx->S;
+    for (int s = s0; s < s1; ++s) {
+        Builder bd{ctx, B, s, s, false, 0, (char*)ctx->d_ws + (size_t)s * ctx->ws_slice};
+        bd.es = ctx->opts.dtype == RESIST_BF16 ? 2 : 4; bd.ops = &ops;
+        bd.bn_partial_need = needs[s].bn_partial; bd.wgrad_partial_need = needs[s].wgrad_partial; bd.gbig = needs[s].gbig;
+        const size_t used = unroll_subnet(ctx, bd, present_of(ctx, s), 1.f);
+        if (used > ctx->ws_slice) { ctx->err = "internal: workspace slice too small"; return RESIST_EINVAL; }
+        ctx->logits_dev[s] = bd.logits; ctx->logits_B[s] = B;
+        plan.info.conv_flops += bd.flops; plan.info.tensor_core_convs += bd.n_tc; plan.info.cuda_core_convs += bd.n_cc;
+    }
+    plan.sub = sub;
+    rc = upload_plan(ctx, plan, ops, sub >= 0, st);
+    if (rc) return rc;
+    plan.B = B; plan.generation = ctx->generation; plan.valid = true;
+    plan.info.workspace_bytes = (int64_t)ctx->ws_bytes;
+    return RESIST_OK;
+}
+
+static int run_plan(resist_ctx* ctx, Plan& plan, const PatchArgs& pa, bool update, float lr, cudaStream_t st) {
+    const bool bf = ctx->opts.dtype == RESIST_BF16;
+    long long n_launch = 0;
+    if (plan.nsites) { patch_kernel<<<(plan.nsites + 63) / 64, 64, 0, st>>>(plan.d_sites, plan.nsites, pa); ++n_launch; }
+    for (const Launch& L : plan.launches) {
+        switch (L.kind) {
+            case OP_CONV_FWD: case OP_CONV_DGRAD: case OP_CONV_WGRAD: {
+                const int mode = L.kind == OP_CONV_FWD ? CONV_FWD : L.kind == OP_CONV_DGRAD ? CONV_DGRAD : CONV_WGRAD;
+                if (L.backend) launch_conv_tc(plan.d_conv + L.first, L.count, L.gx, mode, st);
+                else launch_conv_ref(plan.d_conv + L.first, L.count, L.gx, mode, bf, st);
+                ++n_launch; break; }
+            case OP_SPLITK: launch_splitk_reduce(plan.d_conv + L.first, L.count, (int)L.max_elems, st); ++n_launch; break;
+            case OP_BN_STATS: launch_bn_stats(plan.d_bn + L.first, L.count, L.gx, L.max_c, bf, st); n_launch += 2; break;
+            case OP_BN_APPLY: launch_bn_apply(plan.d_bn + L.first, L.count, L.max_elems, bf, st); ++n_launch; break;
+            case OP_BN_BWD_REDUCE: launch_bn_bwd_reduce(plan.d_bn + L.first, L.count, L.gx, L.max_c, bf, st); n_launch += 2; break;
+            case OP_BN_BWD_APPLY: launch_bn_bwd_apply(plan.d_bn + L.first, L.count, L.max_elems, bf, st); ++n_launch; break;
+            case OP_POOL_FWD: launch_maxpool_fwd(plan.d_pool + L.first, L.count, L.max_elems, bf, st); ++n_launch; break;
+            case OP_POOL_BWD: launch_maxpool_bwd(plan.d_pool + L.first, L.count, L.max_elems, bf, st); ++n_launch; break;
+            case OP_HEAD_FWD: launch_head_fwd(plan.d_head + L.first, L.count, L.max_b, L.max_c, L.max_classes, bf, st); n_launch += 3; break;
+            case OP_HEAD_BWD: launch_head_bwd(plan.d_head + L.first, L.count, L.max_b, L.max_c, L.max_classes, L.max_elems, bf, st); n_launch += 3; break;
+        }
+    }
+    if (update && plan.sgd_chunks) {
+        launch_sgd(plan.d_sgd, plan.n_sgd_seg, plan.sgd_chunks, ctx->pa, lr, ctx->opts.momentum, ctx->opts.weight_decay, bf, st);
+        ++n_launch;
+    }
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { ctx->err = std::string("launch failed: ") + cudaGetErrorString(e); return RESIST_ECUDA; }
+    ctx->info = plan.info; ctx->info.kernel_launches = n_launch;
+    return RESIST_OK;
+}
+
+}  // namespace resist
+
+using namespace resist;
+
+extern "C" {
+
+int resist_local_step(resist_ctx* ctx, int32_t subnet, const void* images, const int32_t* labels, int32_t B, float lr,
+                      float* loss_out, resist_stream stream) {
+    if (!ctx) return RESIST_EINVAL;
+    if (ctx->state < 1) { ctx->err = "local step before partition"; return RESIST_ESTATE; }
+    if (subnet < 0 || subnet >= ctx->S) { ctx->err = "subnet out of range"; return RESIST_EINVAL; }
+    if (!images || !labels || B < 2 || B > 1024) { ctx->err = "need images, labels and 2 <= B <= 1024"; return RESIST_EINVAL; }
+    cudaStream_t st = (cudaStream_t)stream;
+    Plan& plan = ctx->plans[subnet];
+    if (!plan.valid || plan.B != B || plan.generation != ctx->generation) { int rc = build_plan(ctx, plan, subnet, B, st); if (rc) return rc; }
+    PatchArgs pa{}; pa.images[0] = images; pa.labels[0] = labels; pa.loss_out = loss_out;
+    int rc = run_plan(ctx, plan, pa, true, lr, st);
+    if (rc == RESIST_OK) ctx->state = 2;
+    return rc;
+}
+
+int resist_local_step_grouped(resist_ctx* ctx, const void* const* images, const int32_t* const* labels, int32_t B, float lr,
+                              float* loss_out, resist_stream stream) {
+    if (!ctx) return RESIST_EINVAL;
+    if (ctx->state < 1) { ctx->err = "local step before partition"; return RESIST_ESTATE; }
+    if (!images || !labels || B < 2 || B > 1024) { ctx->err = "need images, labels and 2 <= B <= 1024"; return RESIST_EINVAL; }
+    PatchArgs pa{};
+    for (int s = 0; s < ctx->S; ++s) { if (!images[s] || !labels[s]) { ctx->err = "null image or label pointer"; return RESIST_EINVAL; }
+        pa.images[s] = images[s]; pa.labels[s] = labels[s]; }
+    pa.loss_out = loss_out;
+    cudaStream_t st = (cudaStream_t)stream;
+    Plan& plan = ctx->plans[ctx->S_cap];
+    if (!plan.valid || plan.B != B || plan.generation != ctx->generation) { int rc = build_plan(ctx, plan, -1, B, st); if (rc) return rc; }
+    int rc = run_plan(ctx, plan, pa, true, lr, st);
+    if (rc == RESIST_OK) ctx->state = 2;
+    return rc;
+}
+
+int resist_eval(resist_ctx* ctx, const void* images, const int32_t* labels, int32_t B, float* logits_out, float* loss_out,
+                int32_t* correct_out, resist_stream stream) {
+    if (!ctx) return RESIST_EINVAL;
+    if (!images || B < 1 || B > 1024) { ctx->err = "need images and 1 <= B <= 1024"; return RESIST_EINVAL; }
+    cudaStream_t st = (cudaStream_t)stream;
+    int rc = ensure_param_arrays(ctx, std::max(ctx->S_cap, 1));
+    if (rc) return rc;
+    const int copy = ctx->S_cap;                               // the evaluation copy sits after the working copies
+    const int S = std::max(ctx->S, 1);
+    // refresh the evaluation copy from the global parameters
+    Segment sp{0, ctx->L.n_params, 0, 0u, copy}, sb{0, ctx->L.n_buffers, 0, 0u, copy};
+    rc = ensure_seg_table(ctx, 2); if (rc) return rc;
+    Segment both[2] = {sp, sb};
+    cudaError_t e = cudaMemcpyAsync(ctx->d_seg, both, sizeof(both), cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) { ctx->err = cudaGetErrorString(e); return RESIST_ECUDA; }
+    launch_scatter(ctx->d_seg, 1, (sp.len + SEG_CHUNK - 1) / SEG_CHUNK, ctx->pa, false, ctx->opts.dtype == RESIST_BF16, st);
+    launch_scatter_buffers(ctx->d_seg + 1, 1, (sb.len + SEG_CHUNK - 1) / SEG_CHUNK, ctx->pa, st);
+    cudaStreamSynchronize(st);
+    Plan& plan = ctx->plans[ctx->S_cap + 1];
+    if (!plan.valid || plan.B != B || plan.generation != (unsigned long long)S) {
+        std::vector<char> all(ctx->arch.num_blocks, 1);
+        Needs n = measure_subnet(ctx, 0, copy, all, B, true, 1.f / (float)S);
+        if (n.total > ctx->eval_ws_bytes) {
+            cudaDeviceSynchronize(); ctx_free(ctx, ctx->d_eval_ws);
+            ctx->d_eval_ws = ctx_alloc(ctx, n.total); ctx->eval_ws_bytes = ctx->d_eval_ws ? n.total : 0;
+            if (!ctx->d_eval_ws) { ctx->err = "allocator returned NULL for the evaluation workspace"; return RESIST_ENOMEM; }
+        }
+        std::vector<Op> ops;
+        Builder bd{ctx, B, 0, copy, true, 0, (char*)ctx->d_eval_ws}; bd.es = ctx->opts.dtype == RESIST_BF16 ? 2 : 4; bd.ops = &ops;
+        bd.bn_partial_need = n.bn_partial; bd.wgrad_partial_need = n.wgrad_partial; bd.gbig = n.gbig;
+        unroll_subnet(ctx, bd, all, 1.f / (float)S);
+        plan.sub = -2;
+        rc = upload_plan(ctx, plan, ops, true, st);
+        if (rc) return rc;
+        plan.B = B; plan.generation = (unsigned long long)S; plan.valid = true;
+    }
+    PatchArgs pa{}; pa.images[0] = images; pa.labels[0] = labels; pa.loss_out = loss_out; pa.logits_out = logits_out; pa.correct = correct_out;
+    const resist_step_info keep = ctx->info;
+    rc = run_plan(ctx, plan, pa, false, 0.f, st);
+    ctx->info = keep;
+    return rc;
+}
+
+}  // extern "C"

@@ -1,0 +1,74 @@
+// Host runtime of the ResIST library: context, parameter layout, per-round schedule and launch plans.
+#pragma once
+#include <string>
+#include <vector>
+#include "../../include/resist.h"
+#include "internal.h"
+
+namespace resist {
+
+struct BNRef { long long g, b, buf; int c; };                 // offsets of gamma, beta; running stats (mean, var)
+struct ConvRef { long long w; int k, cin, cout, stride; };
+struct BlockRef { BNRef bn[3]; ConvRef conv[3]; ConvRef proj; int nconv; long long begin, end, buf_begin, buf_end; };
+struct Layout {
+    ConvRef stem; BNRef stem_bn; std::vector<BlockRef> blk; BNRef final_bn;
+    long long head_w, head_b; int head_c; long long n_params, n_buffers;
+};
+Layout make_layout(const resist_arch& a, const std::vector<resist_block>& blocks);
+
+enum OpKind {
+    OP_CONV_FWD, OP_CONV_DGRAD, OP_CONV_WGRAD, OP_SPLITK, OP_BN_STATS, OP_BN_APPLY, OP_BN_BWD_REDUCE, OP_BN_BWD_APPLY,
+    OP_POOL_FWD, OP_POOL_BWD, OP_HEAD_FWD, OP_HEAD_BWD
+};
+
+// One operation of one sub-ResNet, keyed so that equal keys of different sub-ResNets share a launch.
+struct Op {
+    long long key; OpKind kind; int sub;
+    ConvProb conv; BnProb bn; PoolProb pool; HeadProb head;
+    int backend;          // convolutions: 0 = CUDA cores, 1 = tensor cores
+    int patch_images;     // conv.act must be replaced by the caller's image pointer
+};
+
+struct PatchSite { void** where; int what; int sub; };        // what: 0 images, 1 labels, 2 loss_out, 3 logits_out, 4 correct
+
+struct Launch {
+    OpKind kind; int backend; int first, count;               // range in the typed device array
+    int gx; long long max_elems; int max_b, max_c, max_classes;
+};
+
+struct Plan {
+    bool valid = false; int B = 0; unsigned long long generation = 0; int sub = -1;   // sub = -1: all sub-ResNets grouped
+    std::vector<Launch> launches;
+    void* d_blob = nullptr; size_t blob_bytes = 0;            // descriptor arrays in one device allocation
+    ConvProb* d_conv = nullptr; BnProb* d_bn = nullptr; PoolProb* d_pool = nullptr; HeadProb* d_head = nullptr;
+    PatchSite* d_sites = nullptr; int nsites = 0;
+    Segment* d_sgd = nullptr; int n_sgd_seg = 0; long long sgd_chunks = 0;
+    resist_step_info info{};
+};
+
+struct SubMem {           // device tensors of one sub-ResNet for one batch size (offsets into the workspace)
+    size_t bytes = 0;
+};
+
+}  // namespace resist
+
+struct resist_ctx {
+    resist_arch arch{}; std::vector<resist_block> blocks; resist_opts opts{};
+    resist::Layout L;
+    resist_allocator alloc{}; bool own_alloc = false;
+    int S = 0, S_cap = 0;                                      // current and allocated number of sub-ResNets
+    std::vector<uint32_t> mask;                                // member_mask of the current round
+    int state = 0;                                             // 0 = initialised, 1 = partitioned, 2 = stepped
+    unsigned long long generation = 0;                         // bumped by every partition
+    resist::ParamArrays pa{};                                  // arrays hold S_cap + 1 copies; the last is the evaluation copy
+    void* d_param_blob = nullptr;
+    // workspace: per sub-ResNet slices of one allocation
+    void* d_ws = nullptr; size_t ws_bytes = 0; size_t ws_slice = 0;
+    void* d_eval_ws = nullptr; size_t eval_ws_bytes = 0;
+    std::vector<resist::Plan> plans;                           // [S_cap] single plans, [S_cap] = grouped, [S_cap+1] = eval
+    resist::Segment* d_seg = nullptr; int seg_cap = 0;         // scratch table for scatter / aggregate
+    std::vector<float*> logits_dev; std::vector<int> logits_B; // last logits per sub-ResNet (device pointers into ws)
+    resist_step_info info{};
+    int sm_count = 148;
+    std::string err;
+};
