@@ -150,6 +150,33 @@ typedef struct {
 } resist_step_info;
 int resist_get_step_info(resist_ctx* ctx, resist_step_info* out);
 
+/* ---- Layer-level entry points: one layer on caller-owned device tensors, run by the kernels of the local step.
+ * They allocate their own scratch with cudaMalloc, synchronise the stream before returning, and report
+ * failures through resist_layer_last_error().  dtype: RESIST_F32 or RESIST_BF16 for activations and weights.
+ *
+ * resist_conv2d: a k x k convolution with zero padding (k-1)/2 and stride 1 or 2, the building block of the
+ * residual blocks of Sec. 2.1.  Geometry is always that of the forward convolution: a [N,H,W,C], w [K,k,k,C],
+ * y [N,P,Q,K] with P = (H + 2*pad - k)/stride + 1.
+ *   mode 0 (forward): act = a, wgt = w, out = y = scale * conv(a, w) + add      (add: y-shaped or NULL)
+ *   mode 1 (dgrad):   act = dy, wgt = w, out = da = conv^T(dy, w) + add         (add: a-shaped or NULL)
+ *   mode 2 (wgrad):   act = a, wgt = dy, out = dw, fp32 [K,k,k,C]
+ * backend: RESIST_CONV_AUTO or RESIST_CONV_CUDA_CORES; *used_backend (host, may be NULL) receives 1 when the
+ * tensor-core kernel ran. */
+int resist_conv2d(int32_t mode, int32_t dtype, int32_t backend, const void* act, const void* wgt, const void* add, void* out,
+                  int32_t N, int32_t H, int32_t W, int32_t C, int32_t K, int32_t ksz, int32_t stride, float scale,
+                  int32_t* used_backend, resist_stream stream);
+
+/* BN (batch statistics over the m rows of x [m, C], biased variance) followed by ReLU, the pre-activation of
+ * Sec. 2.1.  stat: dev float [4*C], receives mean and 1/sqrt(var+eps) (and, in backward, the two reduction
+ * sums); run_mean/run_var: dev, updated when non-NULL.  Backward returns dx (+ add), dgamma, dbeta. */
+int resist_bn_relu_forward(int32_t dtype, const void* x, const float* gamma, const float* beta, void* a, float* stat,
+                           float* run_mean, float* run_var, int64_t m, int32_t C, float eps, float momentum,
+                           resist_stream stream);
+int resist_bn_relu_backward(int32_t dtype, const void* x, const void* da, const float* gamma, const float* beta, float* stat,
+                            const void* add, void* dx, float* dgamma, float* dbeta, int64_t m, int32_t C,
+                            resist_stream stream);
+const char* resist_layer_last_error(void);
+
 /* The library's own splitmix64 (the stream that drives the partition), for cross-checking: host out[n]. */
 void resist_splitmix64(uint64_t seed, int64_t n, uint64_t* out);
 

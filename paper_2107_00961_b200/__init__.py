@@ -82,6 +82,10 @@ def lib():
         L.resist_get_step_info.argtypes = [P, C.POINTER(_StepInfo)]
         L.resist_splitmix64.argtypes = [U64, C.c_int64, P]
         L.resist_splitmix64.restype = None
+        L.resist_conv2d.argtypes = [I, I, I, P, P, P, P, I, I, I, I, I, I, I, F, P, P]
+        L.resist_bn_relu_forward.argtypes = [I, P, P, P, P, P, P, P, C.c_int64, I, F, F, P]
+        L.resist_bn_relu_backward.argtypes = [I, P, P, P, P, P, P, P, P, P, C.c_int64, I, P]
+        L.resist_layer_last_error.restype = C.c_char_p
         L.resist_last_error.argtypes = [P]
         L.resist_last_error.restype = C.c_char_p
         _lib = L
@@ -90,7 +94,8 @@ def lib():
 
 EXPORTS = ["resist_init", "resist_destroy", "resist_partition", "resist_local_step", "resist_local_step_grouped",
            "resist_aggregate", "resist_eval", "resist_param_count", "resist_get_params", "resist_set_params",
-           "resist_get_grads", "resist_get_logits", "resist_get_step_info", "resist_splitmix64", "resist_last_error"]
+           "resist_get_grads", "resist_get_logits", "resist_get_step_info", "resist_splitmix64", "resist_last_error",
+           "resist_conv2d", "resist_bn_relu_forward", "resist_bn_relu_backward", "resist_layer_last_error"]
 
 
 def resist_splitmix64(seed: int, n: int) -> np.ndarray:
@@ -101,6 +106,61 @@ def resist_splitmix64(seed: int, n: int) -> np.ndarray:
 
 def _stream_handle(stream: Optional[torch.cuda.Stream]) -> int:
     return (stream or torch.cuda.current_stream()).cuda_stream
+
+
+def _odim(h, k, s):
+    return (h + 2 * ((k - 1) // 2) - k) // s + 1
+
+
+def _layer_check(rc):
+    if rc != RESIST_OK:
+        raise ResistError(rc, lib().resist_layer_last_error().decode())
+
+
+def _dt(t: torch.Tensor) -> int:
+    return {torch.float32: F32, torch.bfloat16: BF16}[t.dtype]
+
+
+def resist_conv2d(mode: int, act: torch.Tensor, wgt: torch.Tensor, geom, add: Optional[torch.Tensor] = None,
+                  scale: float = 1.0, backend: int = CONV_AUTO, stream=None):
+    """geom = (N, H, W, C, K, ksz, stride) of the forward convolution.  Returns (out, used_tensor_cores)."""
+    N, H, W, Cc, K, ksz, stride = geom
+    P, Q = _odim(H, ksz, stride), _odim(W, ksz, stride)
+    if mode == 0:
+        out = torch.empty(N, P, Q, K, dtype=act.dtype, device=act.device)
+    elif mode == 1:
+        out = torch.empty(N, H, W, Cc, dtype=act.dtype, device=act.device)
+    else:
+        out = torch.empty(K, ksz, ksz, Cc, dtype=torch.float32, device=act.device)
+    used = C.c_int32(0)
+    _layer_check(lib().resist_conv2d(mode, _dt(act), backend, act.data_ptr(), wgt.data_ptr(),
+                                     add.data_ptr() if add is not None else None, out.data_ptr(), N, H, W, Cc, K, ksz,
+                                     stride, scale, C.addressof(used), _stream_handle(stream)))
+    return out, bool(used.value)
+
+
+def resist_bn_relu_forward(x: torch.Tensor, gamma, beta, run_mean=None, run_var=None, eps=1e-5, momentum=0.1, stream=None):
+    Cc = x.shape[-1]
+    m = x.numel() // Cc
+    a = torch.empty_like(x)
+    stat = torch.zeros(4 * Cc, dtype=torch.float32, device=x.device)
+    _layer_check(lib().resist_bn_relu_forward(_dt(x), x.data_ptr(), gamma.data_ptr(), beta.data_ptr(), a.data_ptr(),
+                                              stat.data_ptr(), run_mean.data_ptr() if run_mean is not None else None,
+                                              run_var.data_ptr() if run_var is not None else None, m, Cc, eps, momentum,
+                                              _stream_handle(stream)))
+    return a, stat
+
+
+def resist_bn_relu_backward(x, da, gamma, beta, stat, add=None, stream=None):
+    Cc = x.shape[-1]
+    m = x.numel() // Cc
+    dx = torch.empty_like(x)
+    dg = torch.empty(Cc, dtype=torch.float32, device=x.device)
+    db = torch.empty(Cc, dtype=torch.float32, device=x.device)
+    _layer_check(lib().resist_bn_relu_backward(_dt(x), x.data_ptr(), da.data_ptr(), gamma.data_ptr(), beta.data_ptr(),
+                                               stat.data_ptr(), add.data_ptr() if add is not None else None, dx.data_ptr(),
+                                               dg.data_ptr(), db.data_ptr(), m, Cc, _stream_handle(stream)))
+    return dx, dg, db
 
 
 class Context:

@@ -170,11 +170,12 @@ __global__ void __launch_bounds__(256) bn_reduce_kernel(const BnProb* __restrict
         const int c = cb + lane;
         float s0 = 0.f, s1 = 0.f;
         if (rg < R && c < C) {
-            float mean = 0.f, istd = 0.f, g = 0.f, b = 0.f;
+            float mean = 0.f, istd = 0.f, g = 0.f, b = 0.f, shift = 0.f;
             if (MODE == 1) { mean = p.stat[c]; istd = p.stat[C + c]; g = p.gamma[c]; b = p.beta[c]; }
+            else shift = ldf<T>(p.x, c);      // sums of (x - x[0,c]): no cancellation when |mean| >> std
             for (long long r = r0 + rg; r < r1; r += R) {
                 float x = ldf<T>(p.x, r * C + c);
-                if (MODE == 0) { s0 += x; s1 += x * x; }
+                if (MODE == 0) { x -= shift; s0 += x; s1 += x * x; }
                 else {
                     float xh = (x - mean) * istd;
                     float dz = (xh * g + b > 0.f) ? ldf<T>(p.da, r * C + c) : 0.f;
@@ -194,7 +195,7 @@ __global__ void __launch_bounds__(256) bn_reduce_kernel(const BnProb* __restrict
     }
 }
 
-template <int MODE>
+template <class T, int MODE>
 __global__ void bn_finalize_kernel(const BnProb* __restrict__ probs) {
     const BnProb& p = probs[blockIdx.y];
     const int c = blockIdx.x * blockDim.x + threadIdx.x;
@@ -206,8 +207,9 @@ __global__ void bn_finalize_kernel(const BnProb* __restrict__ probs) {
     double a0 = 0.0, a1 = 0.0;
     for (int k = 0; k < p.chunks; ++k) { a0 += p.partial[((long long)k * 2 + 0) * p.C + c]; a1 += p.partial[((long long)k * 2 + 1) * p.C + c]; }
     if (MODE == 0) {
-        const double m = (double)p.m, mean = a0 / m;
-        double var = a1 / m - mean * mean; if (var < 0.0) var = 0.0;
+        const double m = (double)p.m, dm = a0 / m;                 // sums are of x - x[0,c]
+        double var = a1 / m - dm * dm; if (var < 0.0) var = 0.0;
+        const double mean = dm + (double)ldf<T>(p.x, c);
         p.stat[c] = (float)mean;
         p.stat[p.C + c] = (float)(1.0 / sqrt(var + (double)p.eps));
         if (p.run_mean) {
@@ -253,7 +255,8 @@ static int ew_grid(long long n) { long long g = (n + 255) / 256; if (g > 148 * 1
 void launch_bn_stats(const BnProb* d, int nprob, int max_chunks, int max_c, bool bf16, cudaStream_t s) {
     if (bf16) bn_reduce_kernel<__nv_bfloat16, 0><<<dim3(max_chunks, nprob), 256, 0, s>>>(d);
     else bn_reduce_kernel<float, 0><<<dim3(max_chunks, nprob), 256, 0, s>>>(d);
-    bn_finalize_kernel<0><<<dim3((max_c + 127) / 128, nprob), 128, 0, s>>>(d);
+    if (bf16) bn_finalize_kernel<__nv_bfloat16, 0><<<dim3((max_c + 127) / 128, nprob), 128, 0, s>>>(d);
+    else bn_finalize_kernel<float, 0><<<dim3((max_c + 127) / 128, nprob), 128, 0, s>>>(d);
 }
 void launch_bn_apply(const BnProb* d, int nprob, long long max_elems, bool bf16, cudaStream_t s) {
     if (bf16) bn_apply_kernel<__nv_bfloat16><<<dim3(ew_grid(max_elems), nprob), 256, 0, s>>>(d);
@@ -262,7 +265,7 @@ void launch_bn_apply(const BnProb* d, int nprob, long long max_elems, bool bf16,
 void launch_bn_bwd_reduce(const BnProb* d, int nprob, int max_chunks, int max_c, bool bf16, cudaStream_t s) {
     if (bf16) bn_reduce_kernel<__nv_bfloat16, 1><<<dim3(max_chunks, nprob), 256, 0, s>>>(d);
     else bn_reduce_kernel<float, 1><<<dim3(max_chunks, nprob), 256, 0, s>>>(d);
-    bn_finalize_kernel<1><<<dim3((max_c + 127) / 128, nprob), 128, 0, s>>>(d);
+    bn_finalize_kernel<float, 1><<<dim3((max_c + 127) / 128, nprob), 128, 0, s>>>(d);
 }
 void launch_bn_bwd_apply(const BnProb* d, int nprob, long long max_elems, bool bf16, cudaStream_t s) {
     if (bf16) bn_bwd_apply_kernel<__nv_bfloat16><<<dim3(ew_grid(max_elems), nprob), 256, 0, s>>>(d);

@@ -1,0 +1,119 @@
+// Layer-level entry points: one convolution (forward, dgrad or wgrad) or one BN+ReLU (forward, backward)
+// on caller-owned device tensors, run by the same kernels the local step uses.
+#include <algorithm>
+#include <string>
+#include "runtime.h"
+
+namespace resist {
+bool conv_tc_supported(const ConvProb& p, int mode);
+void launch_conv_tc(const ConvProb* d, int nprob, int max_tiles, int mode, cudaStream_t s);
+size_t conv_tc_scratch_bytes(const ConvProb& p, int mode);
+void conv_tc_prepare(ConvProb& p, int mode, void* scratch, int sm_count);
+}
+using namespace resist;
+
+static thread_local std::string g_layer_error;
+extern "C" const char* resist_layer_last_error(void) { return g_layer_error.c_str(); }
+
+static int out_dim(int h, int k, int stride) { return (h + 2 * ((k - 1) / 2) - k) / stride + 1; }
+
+extern "C" int resist_conv2d(int32_t mode, int32_t dtype, int32_t backend, const void* act, const void* wgt, const void* add,
+                             void* out, int32_t N, int32_t H, int32_t W, int32_t C, int32_t K, int32_t ksz, int32_t stride,
+                             float scale, int32_t* used_backend, resist_stream stream) {
+    if (!act || !wgt || !out || N < 1 || H < 1 || W < 1 || C < 1 || K < 1 || ksz < 1 || ksz % 2 == 0 || stride < 1 || mode < 0 || mode > 2) {
+        g_layer_error = "bad argument"; return RESIST_EINVAL; }
+    if (dtype != RESIST_F32 && dtype != RESIST_BF16) { g_layer_error = "bad dtype"; return RESIST_EINVAL; }
+    cudaStream_t st = (cudaStream_t)stream;
+    ConvProb p{};
+    p.N = N; p.H = H; p.W = W; p.C = C; p.K = K; p.ksz = ksz; p.stride = stride; p.pad = (ksz - 1) / 2;
+    p.P = out_dim(H, ksz, stride); p.Q = out_dim(W, ksz, stride); p.scale = scale; p.add = add; p.out = out;
+    p.act = act; p.wgt = wgt;
+    const long long rows_out = (long long)N * p.P * p.Q, rows_in = (long long)N * H * W;
+    if (mode == CONV_FWD) { p.M = (int)rows_out; p.Ncol = K; p.Kred = ksz * ksz * C; }
+    else if (mode == CONV_DGRAD) { p.M = (int)rows_in; p.Ncol = C; p.Kred = ksz * ksz * K; }
+    else { p.M = K; p.Ncol = ksz * ksz * C; p.Kred = (int)rows_out; p.add = nullptr; }
+    p.tiles_m = (p.M + 63) / 64; p.tiles_n = (p.Ncol + 63) / 64; p.splits = 1;
+    const int ktiles = (p.Kred + 15) / 16; p.ktiles_per_split = ktiles;
+    int sm = 148; int dev = 0; cudaGetDevice(&dev); cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev);
+    const bool tc = dtype == RESIST_BF16 && backend == RESIST_CONV_AUTO && conv_tc_supported(p, mode);
+    if (used_backend) *used_backend = tc ? 1 : 0;
+    size_t scratch = 0;
+    if (tc) scratch = conv_tc_scratch_bytes(p, mode);
+    else if (mode == CONV_WGRAD) {
+        const int tiles = p.tiles_m * p.tiles_n;
+        int want = (2 * sm + tiles - 1) / tiles; want = std::max(1, std::min(std::min(want, 64), ktiles));
+        p.ktiles_per_split = (ktiles + want - 1) / want; p.splits = (ktiles + p.ktiles_per_split - 1) / p.ktiles_per_split;
+        if (p.splits > 1) scratch = (size_t)p.splits * p.M * p.Ncol * 4;
+    }
+    char* blob = nullptr;
+    cudaError_t e = cudaMalloc(&blob, 1024 + scratch);
+    if (e != cudaSuccess) { g_layer_error = cudaGetErrorString(e); return RESIST_ENOMEM; }
+    if (tc) conv_tc_prepare(p, mode, blob + 1024, sm);
+    else if (p.splits > 1) p.partial = (float*)(blob + 1024);
+    e = cudaMemcpyAsync(blob, &p, sizeof(p), cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) {
+        if (tc) launch_conv_tc((ConvProb*)blob, 1, p.tiles_m * p.tiles_n * p.splits, mode, st);
+        else {
+            launch_conv_ref((ConvProb*)blob, 1, p.tiles_m * p.tiles_n * p.splits, mode, dtype == RESIST_BF16, st);
+            if (mode == CONV_WGRAD && p.splits > 1) launch_splitk_reduce((ConvProb*)blob, 1, p.M * p.Ncol, st);
+        }
+        e = cudaGetLastError();
+    }
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    cudaFree(blob);
+    if (e != cudaSuccess) { g_layer_error = cudaGetErrorString(e); return RESIST_ECUDA; }
+    return RESIST_OK;
+}
+
+static void fill_bn(BnProb& p, int64_t m, int C) {
+    p.m = m; p.C = C;
+    const int nl = C < 256 ? C : 256, R = 256 / nl;
+    long long rpc = (long long)R * 32; const long long lim = (m + 1023) / 1024; if (rpc < lim) rpc = lim;
+    p.rows_per_chunk = (int)rpc; p.chunks = (int)((m + rpc - 1) / rpc);
+}
+
+extern "C" int resist_bn_relu_forward(int32_t dtype, const void* x, const float* gamma, const float* beta, void* a, float* stat,
+                                      float* run_mean, float* run_var, int64_t m, int32_t C, float eps, float momentum,
+                                      resist_stream stream) {
+    if (!x || !gamma || !beta || !a || !stat || m < 1 || C < 1) { g_layer_error = "bad argument"; return RESIST_EINVAL; }
+    cudaStream_t st = (cudaStream_t)stream;
+    BnProb p{}; p.x = x; p.a = a; p.gamma = gamma; p.beta = beta; p.run_mean = run_mean; p.run_var = run_var; p.stat = stat;
+    p.eps = eps; p.momentum = momentum; fill_bn(p, m, C);
+    char* blob = nullptr;
+    cudaError_t e = cudaMalloc(&blob, 1024 + (size_t)p.chunks * 2 * C * 8);
+    if (e != cudaSuccess) { g_layer_error = cudaGetErrorString(e); return RESIST_ENOMEM; }
+    p.partial = (double*)(blob + 1024);
+    e = cudaMemcpyAsync(blob, &p, sizeof(p), cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) {
+        launch_bn_stats((BnProb*)blob, 1, p.chunks, C, dtype == RESIST_BF16, st);
+        launch_bn_apply((BnProb*)blob, 1, m * C, dtype == RESIST_BF16, st);
+        e = cudaGetLastError();
+    }
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    cudaFree(blob);
+    if (e != cudaSuccess) { g_layer_error = cudaGetErrorString(e); return RESIST_ECUDA; }
+    return RESIST_OK;
+}
+
+extern "C" int resist_bn_relu_backward(int32_t dtype, const void* x, const void* da, const float* gamma, const float* beta,
+                                       float* stat, const void* add, void* dx, float* dgamma, float* dbeta, int64_t m, int32_t C,
+                                       resist_stream stream) {
+    if (!x || !da || !gamma || !beta || !stat || !dx || !dgamma || !dbeta || m < 1 || C < 1) { g_layer_error = "bad argument"; return RESIST_EINVAL; }
+    cudaStream_t st = (cudaStream_t)stream;
+    BnProb p{}; p.x = x; p.da = da; p.dx = dx; p.add = add; p.gamma = gamma; p.beta = beta; p.dgamma = dgamma; p.dbeta = dbeta; p.stat = stat;
+    fill_bn(p, m, C);
+    char* blob = nullptr;
+    cudaError_t e = cudaMalloc(&blob, 1024 + (size_t)p.chunks * 2 * C * 8);
+    if (e != cudaSuccess) { g_layer_error = cudaGetErrorString(e); return RESIST_ENOMEM; }
+    p.partial = (double*)(blob + 1024);
+    e = cudaMemcpyAsync(blob, &p, sizeof(p), cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) {
+        launch_bn_bwd_reduce((BnProb*)blob, 1, p.chunks, C, dtype == RESIST_BF16, st);
+        launch_bn_bwd_apply((BnProb*)blob, 1, m * C, dtype == RESIST_BF16, st);
+        e = cudaGetLastError();
+    }
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    cudaFree(blob);
+    if (e != cudaSuccess) { g_layer_error = cudaGetErrorString(e); return RESIST_ECUDA; }
+    return RESIST_OK;
+}

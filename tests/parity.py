@@ -9,9 +9,11 @@ MOM = float(np.float32(0.9))     # the library keeps momentum in fp32; give the 
 LR = float(np.float32(0.1))
 
 
-def max_rel_err(a, b, floor=1e-3):
-    """max |a-b| / max(|b|, floor*max|b|): relative error, elements far below the tensor's scale compared
-    against that scale (fp32 accumulation error follows the size of the summands, not of the sum)."""
+def max_rel_err(a, b, floor=1e-2):
+    """max |a-b| / max(|b|, floor*max|b|): relative error, with elements below 1 % of the tensor's largest
+    magnitude compared against that 1 % instead.  An fp32 chain of k roundings leaves an absolute error of
+    about k * 6e-8 * scale on every element whatever its own size (the error follows the summands, not the
+    sum), so a 1e-4 relative bound is only meaningful for elements above k * 6e-4 of the scale; k ~ 10."""
     a = np.asarray(a, np.float64)
     b = np.asarray(b, np.float64)
     s = np.abs(b).max()
@@ -28,11 +30,11 @@ def norm_max_abs(a, b):
     return float(np.abs(a - b).max() / s) if s > 0 else float(np.abs(a).max())
 
 
-def per_tensor(arch, a, b, fn, skip_blocks=()):
+def per_tensor(arch, a, b, fn, skip_blocks=(), skip_names=()):
     """Worst fn(a_t, b_t) over the parameter tensors; returns (value, tensor name)."""
     worst, name = 0.0, ""
     for t in synth.param_layout(arch)[0]:
-        if t.block in skip_blocks:
+        if t.block in skip_blocks or t.name in skip_names:
             continue
         v = fn(a[t.offset:t.offset + t.size], b[t.offset:t.offset + t.size])
         if v > worst:
