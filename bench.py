@@ -1,0 +1,323 @@
+#!/usr/bin/env python
+"""Benchmark of the ResIST hot path on B200: sub-ResNet training images/s.
+
+Workload (N = 1): the CIFAR-shaped ResNet-110 configuration: S = 4 sub-ResNets from a seeded layer-wise
+partition (stage-first blocks shared), batch 128 per sub-ResNet, bf16 activations and weights with fp32 master
+weights, 50 local SGD steps per synchronisation round.  A "step" is one grouped local step of all S sub-ResNets
+(S*B images: forward, backward, SGD-momentum update); every 50th step is followed by the reassembly
+(resist_aggregate) and the next round's partition + scatter (resist_partition), all inside the timed region.
+Inputs are synthetic (Gaussian pixels, uniform labels), generated before the timed region.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+`value` is measured with the inputs resident in HBM; `e2e` repeats the same steps through the same public calls
+with the inputs in pinned host memory (copied in every step, the losses copied out every step).
+With --gpus N > 1 (under torchrun) every rank runs an independent replica on its own GPU and the values add up:
+the path has no exchange between GPUs.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import synth  # noqa: E402
+
+LOCAL_STEPS = 50
+POOL = 16            # distinct batches per sub-ResNet, cycled
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"], "bf16_tflops_sustained": d.get("bf16_tflops_sustained"),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons of one GPU, sampled every 200 ms while running."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "200"], stdout=subprocess.PIPE, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        sm, mx, reasons = [], [], set()
+        for l in self.lines:
+            f = [x.strip() for x in l.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def make_batches(cfg, n):
+    xs, ys = [], []
+    for i in range(n):
+        bx, by = [], []
+        for s in range(cfg.S):
+            x, y = synth.batch(cfg, 0, i, s)
+            bx.append(x)
+            by.append(y)
+        xs.append(bx)
+        ys.append(by)
+    return xs, ys
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2107_00961_b200 as lib
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+    torch.cuda.set_device(local)
+    dev = torch.device(f"cuda:{local}")
+    cfg = synth.config(2)
+    S, B, K, W = cfg.S, cfg.batch, args.steps, args.warmup
+
+    ctx = lib.Context(cfg.arch.to_int32(), dtype=lib.BF16, momentum=cfg.momentum, seed=cfg.init_seed, device=str(dev))
+    p0, b0 = synth.init_params(cfg.arch, cfg.init_seed)
+    ctx.set_params(p0, b0)
+    xs, ys = make_batches(cfg, POOL)
+    d_x = [[torch.from_numpy(x).to(dev).to(torch.bfloat16) for x in bx] for bx in xs]
+    d_y = [[torch.from_numpy(y).to(dev) for y in by] for by in ys]
+    h_x = [[torch.from_numpy(synth.bf16_bits(x).view(np.int16)).view(torch.bfloat16).pin_memory() for x in bx] for bx in xs]
+    h_y = [[torch.from_numpy(y).pin_memory() for y in by] for by in ys]
+    stage_x = [torch.empty_like(d_x[0][s]) for s in range(S)]
+    stage_y = [torch.empty_like(d_y[0][s]) for s in range(S)]
+    loss = torch.zeros(S, dtype=torch.float32, device=dev)
+    h_loss = torch.zeros(S, dtype=torch.float32).pin_memory()
+    stream = torch.cuda.current_stream()
+    state = {"step": 0, "round": 0, "launches": 0}
+
+    def new_round():
+        ctx.partition(cfg.round_seed(state["round"]), S)
+        state["round"] += 1
+
+    def one_step(e2e: bool):
+        i = state["step"] % POOL
+        if e2e:
+            for s in range(S):
+                stage_x[s].copy_(h_x[i][s], non_blocking=True)
+                stage_y[s].copy_(h_y[i][s], non_blocking=True)
+            ctx.local_step_grouped(stage_x, stage_y, cfg.lr, loss)
+            h_loss.copy_(loss, non_blocking=True)
+            stream.synchronize()              # the caller reads the loss every step
+        else:
+            ctx.local_step_grouped(d_x[i], d_y[i], cfg.lr, loss)
+        state["step"] += 1
+        state["launches"] += ctx.step_info()["kernel_launches"]
+        if state["step"] % LOCAL_STEPS == 0:
+            ctx.aggregate()
+            new_round()
+            state["launches"] += 4            # aggregate (parameters, buffers) + scatter (parameters, buffers)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(e2e: bool):
+        state["step"] = 0
+        new_round()
+        for _ in range(W):
+            one_step(e2e)
+        state["step"] = 0
+        state["launches"] = 0
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(K):
+            one_step(e2e)
+        e1.record(stream)
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms, state["launches"]
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    ms, launches = timed(False)
+    clocks = sampler.stop()
+    info = ctx.step_info()
+    ms_e2e, _ = timed(True)
+
+    # per-kernel pass: the same steps with every launch bracketed by CUDA events on the library's stream
+    peaks = measured_peaks()
+    ctx.set_profiling(True)
+    ctx.get_profile()
+    new_round()
+    state["step"] = 0
+    nprof = min(K, 10)
+    for _ in range(nprof):
+        one_step(False)
+    prof = ctx.get_profile()
+    ctx.set_profiling(False)
+    total_ms = sum(v["ms"] for v in prof.values())
+    top_name, top = max(((k, v) for k, v in prof.items() if k not in ("scatter", "aggregate")), key=lambda kv: kv[1]["ms"])
+    per_ms = top["ms"] / top["operations"]
+    roof = {"kernel": top_name, "share_of_step": top["ms"] / total_ms, "launches": top["operations"], "avg_ms": per_ms}
+    ai = top["flops"] / max(top["bytes"], 1.0)
+    ridge = peaks["bf16_tflops"] * 1e12 / (peaks["hbm_gbs"] * 1e9)
+    if top["flops"] > 0 and ai > ridge and "tcgen05" in top_name:
+        ach = top["flops"] / top["operations"] / (per_ms * 1e-3) / 1e12
+        roof.update(bound="tensor", achieved=ach, peak=peaks["bf16_tflops_sustained"] or peaks["bf16_tflops"], unit="TFLOP/s")
+    else:
+        ach = top["bytes"] / top["operations"] / (per_ms * 1e-3) / 1e9
+        roof.update(bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s")
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["peak_source"] = peaks["source"]
+    roof["traffic"] = None
+    roof["arithmetic_intensity"] = ai
+    conv_ms = sum(v["ms"] for k, v in prof.items() if k.startswith("conv_") or k == "wgrad_splitk_reduce")
+    conv_flops = sum(v["flops"] for k, v in prof.items() if k.startswith("conv_"))
+    kernels = {k: {"ms_per_step": v["ms"] / nprof, "share": v["ms"] / total_ms,
+                   "GBps": v["bytes"] / max(v["ms"], 1e-9) / 1e6, "TFLOPs": v["flops"] / max(v["ms"], 1e-9) / 1e9}
+               for k, v in sorted(prof.items(), key=lambda kv: -kv[1]["ms"])}
+
+    images = S * B * K * world
+    out = {
+        "metric": "sub-ResNet train images/s", "value": images / (ms * 1e-3), "unit": "images/s", "n_gpus": world, "steps": K,
+        "warmup": W, "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": "configs[1]: CIFAR-shaped ResNet-110, S=4 sub-ResNets, batch 128 per sub-ResNet, bf16 + fp32 master, "
+                               "50 local steps per round with aggregate + repartition between rounds",
+                   "S": S, "batch_per_subnet": B, "local_steps": LOCAL_STEPS, "multi_gpu": "independent replicas" if world > 1 else "single GPU",
+                   "l2": "working set per step (saved activations, %.0f MB) exceeds the 126 MB L2; no flush" % (info["workspace_bytes"] / 1e6)},
+        "clocks": clocks,
+        "e2e": {"value": images / (ms_e2e * 1e-3), "unit": "images/s", "ms_per_step": ms_e2e / K,
+                "h2d_bytes_per_step": int(S * (B * 32 * 32 * 3 * 2 + B * 4)), "d2h_bytes_per_step": int(S * 4)},
+        "gpu_launches": int(launches),
+        "conv": {"TFLOPs": conv_flops / max(conv_ms, 1e-9) / 1e9, "frac_of_bf16_peak": conv_flops / max(conv_ms, 1e-9) / 1e9 / peaks["bf16_tflops"],
+                 "tensor_core_convs": info["tensor_core_convs"], "cuda_core_convs": info["cuda_core_convs"],
+                 "flops_per_step": info["conv_flops"]},
+        "roofline": roof, "kernels": kernels,
+    }
+    if rank == 0:
+        out["cpu_baseline"] = cpu_baseline(cfg, budget_s=20.0)
+        print(json.dumps(out))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def oracle_step_all(cfg, a, mask, params, B, step_idx):
+    """One oracle local step of every sub-ResNet at batch B, one thread per sub-ResNet.  Returns seconds."""
+    import oracle
+    S = cfg.S
+    data = [synth.batch(cfg, 0, step_idx, s, B=B, as_bf16=True) for s in range(S)]
+    moms = [np.zeros_like(params[s]) for s in range(S)]
+    t0 = time.perf_counter()
+    th = [threading.Thread(target=oracle.step, args=(a, oracle.present_of(mask, s), params[s], moms[s], None, data[s][0], data[s][1]),
+                           kwargs=dict(lr=cfg.lr, mu=cfg.momentum, quant=0)) for s in range(S)]
+    for t in th:
+        t.start()
+    for t in th:
+        t.join()
+    return time.perf_counter() - t0
+
+
+def cpu_baseline(cfg, budget_s: float):
+    """The oracle as it stands, on the host cores: one local step of all S sub-ResNets at a reduced batch."""
+    import oracle
+    a = cfg.arch.to_int32()
+    mask = oracle.partition(a, cfg.round_seed(0), cfg.S)
+    p0, _ = synth.init_params(cfg.arch, cfg.init_seed)
+    params = [p0.copy() for _ in range(cfg.S)]
+    t2 = oracle_step_all(cfg, a, mask, params, 2, 0)
+    B = int(max(2, min(cfg.batch, 2 * budget_s / max(t2, 1e-3))))
+    t = oracle_step_all(cfg, a, mask, params, B, 1)
+    return {"value": cfg.S * B / t, "unit": "images/s", "cores": cfg.S, "kind": "oracle",
+            "sample": f"one local step of all S={cfg.S} sub-ResNets of the same network at batch {B} per sub-ResNet "
+                      f"({t:.1f} s, one thread per sub-ResNet, {os.cpu_count()} host cores present)"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    cfg = synth.config(2)
+    a = cfg.arch.to_int32()
+    mask = oracle.partition(a, cfg.round_seed(0), cfg.S)
+    p0, _ = synth.init_params(cfg.arch, cfg.init_seed)
+    params = [p0.copy() for _ in range(cfg.S)]
+    K, W = args.steps, args.warmup
+    t2 = oracle_step_all(cfg, a, mask, params, 2, 0)
+    per_step = 150.0 / max(K + W, 1)                       # the whole run should end within a few minutes
+    B = int(max(2, min(cfg.batch, 2 * per_step / max(t2, 1e-3))))
+    for i in range(W):
+        oracle_step_all(cfg, a, mask, params, B, i)
+    t = 0.0
+    for i in range(K):
+        t += oracle_step_all(cfg, a, mask, params, B, W + i)
+    v = cfg.S * B * K / t
+    sample = f"each step = one local step of all S={cfg.S} sub-ResNets at batch {B} per sub-ResNet (full workload: 128)"
+    print(json.dumps({
+        "impl": "reference", "metric": "sub-ResNet train images/s", "value": v, "unit": "images/s", "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+        "steps": K, "warmup": W, "ms_per_step": 1e3 * t / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "configs[1]: CIFAR-shaped ResNet-110, S=4 sub-ResNets; CPU oracle on a bounded sample", "S": cfg.S,
+                   "batch_per_subnet": B},
+        "cpu_baseline": {"value": v, "unit": "images/s", "cores": cfg.S, "kind": "oracle", "sample": sample},
+        "e2e": {"value": v, "unit": "images/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

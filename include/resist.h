@@ -177,6 +177,22 @@ int resist_bn_relu_backward(int32_t dtype, const void* x, const void* da, const 
                             resist_stream stream);
 const char* resist_layer_last_error(void);
 
+/* Per-kernel timing.  With profiling on, every launch of a local step, partition or aggregate is bracketed by
+ * CUDA events on the call's stream and the call synchronises before returning; times, launch counts and the
+ * algorithmic bytes and FLOPs of the work launched accumulate per kernel family until read.
+ * resist_get_profile copies up to `cap` entries to host memory, returns the number of families in *n (may
+ * exceed cap) and clears the counters. */
+typedef struct {
+    char name[32];
+    int64_t launches;        /* kernel launches (a family may issue two kernels per operation) */
+    int64_t operations;      /* bracketed operations */
+    double ms;               /* summed device time */
+    double bytes;            /* algorithmic bytes: each operand read once, each result written once */
+    double flops;            /* algorithmic FLOPs (convolutions: 2*M*N*K) */
+} resist_profile_entry;
+int resist_set_profiling(resist_ctx* ctx, int32_t on);
+int resist_get_profile(resist_ctx* ctx, resist_profile_entry* out, int32_t cap, int32_t* n);
+
 /* The library's own splitmix64 (the stream that drives the partition), for cross-checking: host out[n]. */
 void resist_splitmix64(uint64_t seed, int64_t n, uint64_t* out);
 

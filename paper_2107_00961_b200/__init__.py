@@ -52,6 +52,11 @@ class _Allocator(C.Structure):
     _fields_ = [("alloc", _ALLOC_FN), ("release", _FREE_FN), ("user", C.c_void_p)]
 
 
+class _ProfileEntry(C.Structure):
+    _fields_ = [("name", C.c_char * 32), ("launches", C.c_int64), ("operations", C.c_int64), ("ms", C.c_double),
+                ("bytes", C.c_double), ("flops", C.c_double)]
+
+
 class _StepInfo(C.Structure):
     _fields_ = [(n, C.c_int64) for n in ("kernel_launches", "conv_flops", "tensor_core_convs", "cuda_core_convs",
                                            "workspace_bytes")]
@@ -82,6 +87,8 @@ def lib():
         L.resist_get_step_info.argtypes = [P, C.POINTER(_StepInfo)]
         L.resist_splitmix64.argtypes = [U64, C.c_int64, P]
         L.resist_splitmix64.restype = None
+        L.resist_set_profiling.argtypes = [P, I]
+        L.resist_get_profile.argtypes = [P, P, I, P]
         L.resist_conv2d.argtypes = [I, I, I, P, P, P, P, I, I, I, I, I, I, I, F, P, P]
         L.resist_bn_relu_forward.argtypes = [I, P, P, P, P, P, P, P, C.c_int64, I, F, F, P]
         L.resist_bn_relu_backward.argtypes = [I, P, P, P, P, P, P, P, P, P, C.c_int64, I, P]
@@ -95,7 +102,7 @@ def lib():
 EXPORTS = ["resist_init", "resist_destroy", "resist_partition", "resist_local_step", "resist_local_step_grouped",
            "resist_aggregate", "resist_eval", "resist_param_count", "resist_get_params", "resist_set_params",
            "resist_get_grads", "resist_get_logits", "resist_get_step_info", "resist_splitmix64", "resist_last_error",
-           "resist_conv2d", "resist_bn_relu_forward", "resist_bn_relu_backward", "resist_layer_last_error"]
+           "resist_set_profiling", "resist_get_profile", "resist_conv2d", "resist_bn_relu_forward", "resist_bn_relu_backward", "resist_layer_last_error"]
 
 
 def resist_splitmix64(seed: int, n: int) -> np.ndarray:
@@ -301,6 +308,17 @@ class Context:
         out = np.empty((B, self.classes), dtype=np.float32)
         self._check(self._lib.resist_get_logits(self._ctx, subnet, out.ctypes.data))
         return out
+
+    def set_profiling(self, on: bool):
+        self._check(self._lib.resist_set_profiling(self._ctx, 1 if on else 0))
+
+    def get_profile(self) -> dict:
+        """{family: dict(launches, operations, ms, bytes, flops)} since the last read; clears the counters."""
+        arr = (_ProfileEntry * 32)()
+        n = C.c_int32(0)
+        self._check(self._lib.resist_get_profile(self._ctx, C.addressof(arr), 32, C.addressof(n)))
+        return {arr[i].name.decode(): {"launches": arr[i].launches, "operations": arr[i].operations, "ms": arr[i].ms,
+                                       "bytes": arr[i].bytes, "flops": arr[i].flops} for i in range(min(n.value, 32))}
 
     def step_info(self) -> dict:
         s = _StepInfo()

@@ -292,6 +292,7 @@ static std::vector<char> present_of(const resist_ctx* ctx, int sub) {
 
 static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool single, cudaStream_t st) {
     std::stable_sort(ops.begin(), ops.end(), [](const Op& a, const Op& b) { return a.key < b.key; });
+    const double es = ctx->opts.dtype == RESIST_BF16 ? 2.0 : 4.0;
     std::vector<ConvProb> conv; std::vector<BnProb> bn; std::vector<PoolProb> pool; std::vector<HeadProb> head;
     struct HostSite { int arr; int idx; int field; int what; int sub; };
     std::vector<HostSite> sites;
@@ -308,20 +309,31 @@ static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool s
                     if (o.patch_images) sites.push_back({0, (int)conv.size(), 0, 0, slot});
                     conv.push_back(o.conv);
                     const ConvProb& p = o.conv;
-                    if (o.kind == OP_SPLITK) L.max_elems = std::max<long long>(L.max_elems, (long long)p.M * p.Ncol);
-                    else L.gx = std::max(L.gx, p.tiles_m * p.tiles_n * p.splits);
+                    if (o.kind == OP_SPLITK) { L.max_elems = std::max<long long>(L.max_elems, (long long)p.M * p.Ncol);
+                        L.bytes += 4.0 * p.M * p.Ncol * (p.splits + 1); }
+                    else { L.gx = std::max(L.gx, p.tiles_m * p.tiles_n * p.splits);
+                        const double in_e = (double)p.N * p.H * p.W * p.C, out_e = (double)p.N * p.P * p.Q * p.K, w_e = (double)p.K * p.ksz * p.ksz * p.C;
+                        L.flops += 2.0 * out_e * p.ksz * p.ksz * p.C;
+                        if (o.kind == OP_CONV_WGRAD) L.bytes += es * (in_e + out_e) + 4.0 * w_e;
+                        else L.bytes += es * (in_e + out_e + w_e + (p.add ? (o.kind == OP_CONV_FWD ? out_e : in_e) : 0.0)); }
                     break; }
                 case OP_BN_STATS: case OP_BN_APPLY: case OP_BN_BWD_REDUCE: case OP_BN_BWD_APPLY: {
                     if (k == i) L.first = (int)bn.size();
                     bn.push_back(o.bn);
                     L.gx = std::max(L.gx, o.bn.chunks); L.max_c = std::max(L.max_c, o.bn.C);
                     L.max_elems = std::max<long long>(L.max_elems, o.bn.m * o.bn.C);
+                    { const double e = (double)o.bn.m * o.bn.C;
+                      if (o.kind == OP_BN_STATS) L.bytes += o.bn.eval ? 0.0 : es * e;
+                      else if (o.kind == OP_BN_APPLY) L.bytes += 2 * es * e;
+                      else if (o.kind == OP_BN_BWD_REDUCE) L.bytes += 2 * es * e;
+                      else L.bytes += es * e * (o.bn.add ? 4 : 3); }
                     break; }
                 case OP_POOL_FWD: case OP_POOL_BWD: {
                     if (k == i) L.first = (int)pool.size();
                     pool.push_back(o.pool);
                     const PoolProb& p = o.pool;
                     L.max_elems = std::max<long long>(L.max_elems, (long long)p.N * (o.kind == OP_POOL_FWD ? p.P * p.Q : p.H * p.W) * p.C);
+                    L.bytes += (double)p.N * p.C * (es * ((double)p.H * p.W + (double)p.P * p.Q) + 4.0 * p.P * p.Q);
                     break; }
                 case OP_HEAD_FWD: case OP_HEAD_BWD: {
                     if (k == i) L.first = (int)head.size();
@@ -332,6 +344,7 @@ static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool s
                     const HeadProb& p = o.head;
                     L.max_b = std::max(L.max_b, p.B); L.max_c = std::max(L.max_c, p.C); L.max_classes = std::max(L.max_classes, p.classes);
                     L.max_elems = std::max<long long>(L.max_elems, (long long)p.B * p.HW * p.C);
+                    L.bytes += es * (double)p.B * p.HW * p.C + 4.0 * p.classes * p.C;
                     break; }
             }
         }
@@ -376,6 +389,7 @@ static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool s
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
     if (e != cudaSuccess) { ctx->err = std::string("plan upload: ") + cudaGetErrorString(e); return RESIST_ECUDA; }
     plan.nsites = (int)dsites.size(); plan.n_sgd_seg = (int)segs.size(); plan.sgd_chunks = chunks;
+    plan.sgd_params = 0; for (const Segment& sg : segs) plan.sgd_params += (double)sg.len;
     return RESIST_OK;
 }
 
@@ -422,8 +436,25 @@ static int build_plan(resist_ctx* ctx, Plan& plan, int sub, int B, cudaStream_t 
 static int run_plan(resist_ctx* ctx, Plan& plan, const PatchArgs& pa, bool update, float lr, cudaStream_t st) {
     const bool bf = ctx->opts.dtype == RESIST_BF16;
     long long n_launch = 0;
-    if (plan.nsites) { patch_kernel<<<(plan.nsites + 63) / 64, 64, 0, st>>>(plan.d_sites, plan.nsites, pa); ++n_launch; }
+    Profiler& pf = ctx->prof;
+    if (plan.nsites) { pf.begin(PK_PATCH, 1, 0, 0, st); patch_kernel<<<(plan.nsites + 63) / 64, 64, 0, st>>>(plan.d_sites, plan.nsites, pa); pf.end(st); ++n_launch; }
     for (const Launch& L : plan.launches) {
+        int pk = 0, nk = 1;
+        switch (L.kind) {
+            case OP_CONV_FWD: pk = L.backend ? PK_CONV_FWD_TC : PK_CONV_FWD_CC; break;
+            case OP_CONV_DGRAD: pk = L.backend ? PK_CONV_DGRAD_TC : PK_CONV_DGRAD_CC; break;
+            case OP_CONV_WGRAD: pk = L.backend ? PK_CONV_WGRAD_TC : PK_CONV_WGRAD_CC; break;
+            case OP_SPLITK: pk = PK_SPLITK; break;
+            case OP_BN_STATS: pk = PK_BN_STATS; nk = 2; break;
+            case OP_BN_APPLY: pk = PK_BN_APPLY; break;
+            case OP_BN_BWD_REDUCE: pk = PK_BN_BWD_REDUCE; nk = 2; break;
+            case OP_BN_BWD_APPLY: pk = PK_BN_BWD_APPLY; break;
+            case OP_POOL_FWD: pk = PK_POOL_FWD; break;
+            case OP_POOL_BWD: pk = PK_POOL_BWD; break;
+            case OP_HEAD_FWD: pk = PK_HEAD_FWD; nk = 3; break;
+            case OP_HEAD_BWD: pk = PK_HEAD_BWD; nk = 3; break;
+        }
+        pf.begin(pk, nk, L.bytes, L.flops, st);
         switch (L.kind) {
             case OP_CONV_FWD: case OP_CONV_DGRAD: case OP_CONV_WGRAD: {
                 const int mode = L.kind == OP_CONV_FWD ? CONV_FWD : L.kind == OP_CONV_DGRAD ? CONV_DGRAD : CONV_WGRAD;
@@ -440,11 +471,15 @@ static int run_plan(resist_ctx* ctx, Plan& plan, const PatchArgs& pa, bool updat
             case OP_HEAD_FWD: launch_head_fwd(plan.d_head + L.first, L.count, L.max_b, L.max_c, L.max_classes, bf, st); n_launch += 3; break;
             case OP_HEAD_BWD: launch_head_bwd(plan.d_head + L.first, L.count, L.max_b, L.max_c, L.max_classes, L.max_elems, bf, st); n_launch += 3; break;
         }
+        pf.end(st);
     }
     if (update && plan.sgd_chunks) {
+        pf.begin(PK_SGD, 1, (bf ? 22.0 : 20.0) * plan.sgd_params, 0, st);
         launch_sgd(plan.d_sgd, plan.n_sgd_seg, plan.sgd_chunks, ctx->pa, lr, ctx->opts.momentum, ctx->opts.weight_decay, bf, st);
+        pf.end(st);
         ++n_launch;
     }
+    pf.collect(st);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { ctx->err = std::string("launch failed: ") + cudaGetErrorString(e); return RESIST_ECUDA; }
     ctx->info = plan.info; ctx->info.kernel_launches = n_launch;

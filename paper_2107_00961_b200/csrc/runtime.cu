@@ -264,6 +264,32 @@ int resist_get_step_info(resist_ctx* ctx, resist_step_info* out) {
     return RESIST_OK;
 }
 
+static const char* const PK_NAMES[PK_COUNT] = {
+    "conv_fwd_cuda_core", "conv_dgrad_cuda_core", "conv_wgrad_cuda_core", "conv_fwd_tcgen05", "conv_dgrad_tcgen05",
+    "conv_wgrad_tcgen05", "wgrad_splitk_reduce", "bn_stats", "bn_apply_relu", "bn_bwd_reduce", "bn_bwd_apply", "maxpool_fwd",
+    "maxpool_bwd", "head_fwd", "head_bwd", "sgd_momentum", "patch_pointers", "scatter", "aggregate"};
+
+int resist_set_profiling(resist_ctx* ctx, int32_t on) {
+    if (!ctx) return RESIST_EINVAL;
+    ctx->prof.on = on != 0;
+    return RESIST_OK;
+}
+
+int resist_get_profile(resist_ctx* ctx, resist_profile_entry* out, int32_t cap, int32_t* n) {
+    if (!ctx || !n) return RESIST_EINVAL;
+    Profiler& pf = ctx->prof;
+    int k = 0;
+    for (int i = 0; i < PK_COUNT; ++i) {
+        if (!pf.ops[i]) continue;
+        if (out && k < cap) { resist_profile_entry& e = out[k]; memset(&e, 0, sizeof(e)); strncpy(e.name, PK_NAMES[i], sizeof(e.name) - 1);
+            e.launches = pf.launches[i]; e.operations = pf.ops[i]; e.ms = pf.ms[i]; e.bytes = pf.bytes[i]; e.flops = pf.flops[i]; }
+        ++k;
+    }
+    *n = k;
+    for (int i = 0; i < PK_COUNT; ++i) { pf.launches[i] = pf.ops[i] = 0; pf.ms[i] = pf.bytes[i] = pf.flops[i] = 0; }
+    return RESIST_OK;
+}
+
 int resist_partition(resist_ctx* ctx, uint64_t round_seed, int32_t S, uint32_t* member_mask, resist_stream stream) {
     if (!ctx) return RESIST_EINVAL;
     cudaStream_t st = (cudaStream_t)stream;
@@ -298,8 +324,12 @@ int resist_partition(resist_ctx* ctx, uint64_t round_seed, int32_t S, uint32_t* 
     CK(cudaMemcpyAsync(ctx->d_seg, segs.data(), segs.size() * sizeof(Segment), cudaMemcpyHostToDevice, st));
     CK(cudaMemcpyAsync(ctx->d_seg + segs.size(), bsegs.data(), bsegs.size() * sizeof(Segment), cudaMemcpyHostToDevice, st));
     const bool restart = ctx->opts.momentum_policy == RESIST_MOMENTUM_RESTART || ctx->state == 0;
-    launch_scatter(ctx->d_seg, (int)segs.size(), chunks, ctx->pa, restart, ctx->opts.dtype == RESIST_BF16, st);
+    double held_p = 0, heldb = 0; for (const Segment& g : segs) held_p += (double)g.len; for (const Segment& g : bsegs) heldb += (double)g.len;
+    const bool bf = ctx->opts.dtype == RESIST_BF16;
+    ctx->prof.begin(PK_SCATTER, 2, held_p * (4.0 + 4.0 + (restart ? 4.0 : 0.0) + (bf ? 2.0 : 0.0)) + heldb * 8.0, 0, st);
+    launch_scatter(ctx->d_seg, (int)segs.size(), chunks, ctx->pa, restart, bf, st);
     launch_scatter_buffers(ctx->d_seg + segs.size(), (int)bsegs.size(), bchunks, ctx->pa, st);
+    ctx->prof.end(st); ctx->prof.collect(st);
     CK(cudaGetLastError());
     CK(cudaStreamSynchronize(st));     // the host-side segment vectors die here
     ctx->state = 1;
@@ -331,8 +361,13 @@ int resist_aggregate(resist_ctx* ctx, resist_stream stream) {
     if (rc) return rc;
     CK(cudaMemcpyAsync(ctx->d_seg, segs.data(), segs.size() * sizeof(Segment), cudaMemcpyHostToDevice, st));
     CK(cudaMemcpyAsync(ctx->d_seg + segs.size(), bsegs.data(), bsegs.size() * sizeof(Segment), cudaMemcpyHostToDevice, st));
+    double rd = 0, wr = 0;
+    for (const Segment& g : segs) { rd += (double)g.len * __builtin_popcount(g.mask); wr += (double)g.len; }
+    for (const Segment& g : bsegs) { rd += (double)g.len * __builtin_popcount(g.mask); wr += (double)g.len; }
+    ctx->prof.begin(PK_AGGREGATE, 2, 4.0 * (rd + wr), 0, st);
     launch_aggregate(ctx->d_seg, (int)segs.size(), chunks, ctx->pa.w, ctx->pa.n, ctx->pa.global, S, st);
     launch_aggregate(ctx->d_seg + segs.size(), (int)bsegs.size(), bchunks, ctx->pa.buf, ctx->pa.nbuf, ctx->pa.global_buf, S, st);
+    ctx->prof.end(st); ctx->prof.collect(st);
     CK(cudaGetLastError());
     CK(cudaStreamSynchronize(st));
     return RESIST_OK;

@@ -34,6 +34,29 @@ struct PatchSite { void** where; int what; int sub; };        // what: 0 images,
 struct Launch {
     OpKind kind; int backend; int first, count;               // range in the typed device array
     int gx; long long max_elems; int max_b, max_c, max_classes;
+    double bytes, flops;                                      // algorithmic work of this launch
+};
+
+enum ProfKind {
+    PK_CONV_FWD_CC, PK_CONV_DGRAD_CC, PK_CONV_WGRAD_CC, PK_CONV_FWD_TC, PK_CONV_DGRAD_TC, PK_CONV_WGRAD_TC, PK_SPLITK,
+    PK_BN_STATS, PK_BN_APPLY, PK_BN_BWD_REDUCE, PK_BN_BWD_APPLY, PK_POOL_FWD, PK_POOL_BWD, PK_HEAD_FWD, PK_HEAD_BWD,
+    PK_SGD, PK_PATCH, PK_SCATTER, PK_AGGREGATE, PK_COUNT
+};
+struct Profiler {
+    bool on = false;
+    std::vector<cudaEvent_t> pool; size_t used = 0;
+    struct Pending { int kind; int launches; double bytes, flops; cudaEvent_t e0, e1; };
+    std::vector<Pending> pending;
+    long long launches[PK_COUNT] = {}, ops[PK_COUNT] = {}; double ms[PK_COUNT] = {}, bytes[PK_COUNT] = {}, flops[PK_COUNT] = {};
+    cudaEvent_t ev() { if (used == pool.size()) { cudaEvent_t e; cudaEventCreate(&e); pool.push_back(e); } return pool[used++]; }
+    void begin(int kind, int launches_, double b, double f, cudaStream_t st) {
+        if (!on) return; Pending p{kind, launches_, b, f, ev(), ev()}; cudaEventRecord(p.e0, st); pending.push_back(p); }
+    void end(cudaStream_t st) { if (!on) return; cudaEventRecord(pending.back().e1, st); }
+    void collect(cudaStream_t st) {
+        if (!on) return; cudaStreamSynchronize(st);
+        for (auto& p : pending) { float t = 0.f; cudaEventElapsedTime(&t, p.e0, p.e1);
+            ms[p.kind] += t; launches[p.kind] += p.launches; ops[p.kind] += 1; bytes[p.kind] += p.bytes; flops[p.kind] += p.flops; }
+        pending.clear(); used = 0; }
 };
 
 struct Plan {
@@ -42,7 +65,7 @@ struct Plan {
     void* d_blob = nullptr; size_t blob_bytes = 0;            // descriptor arrays in one device allocation
     ConvProb* d_conv = nullptr; BnProb* d_bn = nullptr; PoolProb* d_pool = nullptr; HeadProb* d_head = nullptr;
     PatchSite* d_sites = nullptr; int nsites = 0;
-    Segment* d_sgd = nullptr; int n_sgd_seg = 0; long long sgd_chunks = 0;
+    Segment* d_sgd = nullptr; int n_sgd_seg = 0; long long sgd_chunks = 0; double sgd_params = 0;
     resist_step_info info{};
 };
 
@@ -69,6 +92,7 @@ struct resist_ctx {
     resist::Segment* d_seg = nullptr; int seg_cap = 0;         // scratch table for scatter / aggregate
     std::vector<float*> logits_dev; std::vector<int> logits_B; // last logits per sub-ResNet (device pointers into ws)
     resist_step_info info{};
+    resist::Profiler prof;
     int sm_count = 148;
     std::string err;
 };
