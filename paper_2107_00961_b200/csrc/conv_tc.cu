@@ -1,9 +1,340 @@
-// Tensor-core convolution kernels (tcgen05 + TMEM).  Placeholder until the kernels land: no shape is
-// accepted, so every convolution runs on the CUDA-core family.
+// Tensor-core convolutions for sm_100a: implicit GEMM on tcgen05.mma with the accumulator in TMEM and the
+// operands staged in shared memory by TMA.
+//
+// Forward and dgrad of a stride-1 k x k convolution (k = 1 or 3) share one kernel.  The output tile is 128
+// consecutive positions of one image in "padded-flat" order (row-major over rows of W + 2*pad positions; the
+// 2*pad extra positions per row are computed and thrown away).  In that order the operand of filter tap (r,s) is
+// the SAME pixel run shifted by r*(W+2*pad)+s positions, so the input halo is fetched ONCE per tile (TMA box
+// with out-of-bounds zero fill = the zero padding) and all k*k taps read it through shifted shared-memory
+// descriptors.  Shared memory holds the pixels as planes of 8 channels (16 bytes per pixel per plane), which is
+// the canonical no-swizzle K-major layout of the MMA: 8 pixels x 16 B form one core matrix, any 16-byte pixel
+// offset is a legal start address.
+//
+// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer, warps 2..5 = epilogue
+// (TMEM -> registers -> scale, residual add, bf16 -> global).  Every wait is bounded: on expiry the kernel
+// records the place in the status word, drains, frees its TMEM and returns.
+#include <cuda.h>
+#include <cstdio>
+#include <cstring>
 #include "internal.h"
+
 namespace resist {
-bool conv_tc_supported(const ConvProb&, int) { return false; }
-void launch_conv_tc(const ConvProb*, int, int, int, cudaStream_t) {}
-size_t conv_tc_scratch_bytes(const ConvProb&, int) { return 0; }
-void conv_tc_prepare(ConvProb&, int, void*, int) {}
+
+// ------------------------------------------------------------------------------------------------ device helpers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// bounded wait: false when the barrier did not flip within the limit
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    for (uint32_t i = 0; i < (1u << 22); ++i) {
+        if (mbar_try(bar, parity)) return true;
+        if (i > 64) __nanosleep(64);
+    }
+    return false;
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const void* tmap, uint32_t bar, int c0, int c1, int c2, int c3) {
+    asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+                 ::"r"(dst), "l"(tmap), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    // no-swizzle matrix descriptor: start >> 4 | LBO >> 4 at bit 16 | SBO >> 4 at bit 32 | version 1 at bit 46
+    return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
+           ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* v) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+                   "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+                 : "r"(taddr));
+}
+
+// One tensor-core convolution problem.  The two tensor maps come first so that each is 64-byte aligned.
+struct alignas(64) TcProb {
+    CUtensorMap map_a;        // activations (forward: a; dgrad: dy) viewed as (channel, x, y, image)
+    CUtensorMap map_b;        // weights viewed as (8 input channels, output channel, input-channel group, tap)
+    const __nv_bfloat16* add; __nv_bfloat16* out;
+    int* status;
+    int H, W, Wp, pad, taps, flip;          // image extent (1x1 layers: one long row), padded width, taps = k*k
+    int n_img, tiles_per_img, tiles_n;
+    int ncol;                               // channels of the output tensor
+    int n_tile;                             // MMA N: output channels per CTA (multiple of 16, <= 256)
+    int kc, nchunks;                        // reduction channels per pipeline stage, number of stages' worth
+    int box_w, box_h;                       // activation box (pixels)
+    int plane_bytes;                        // one 8-channel plane of the activation box, padded
+    int a_stage_bytes, b_stage_bytes, b_tap_bytes;
+    int b_mn_major;                         // 0: forward (weights K-major); 1: dgrad (weights MN-major)
+    int tmem_cols; int flat;                // flat = 1: 1x1 layer, tile = 128 consecutive pixels of the whole tensor
+    int stages;                             // pipeline depth: 1 when the reduction fits one stage, else 2
+    float scale;
+};
+
+constexpr int TC_THREADS = 192;
+constexpr int TC_STAGES = 2;
+
+__global__ void __launch_bounds__(TC_THREADS) conv_tc_kernel(const TcProb* __restrict__ probs) {
+    const TcProb& p = probs[blockIdx.y];
+    const int tiles = p.n_img * p.tiles_per_img * p.tiles_n;
+    if ((int)blockIdx.x >= tiles) return;
+    const int tn = blockIdx.x % p.tiles_n;
+    const int tm = blockIdx.x / p.tiles_n;
+    const int img = tm / p.tiles_per_img, t_in = tm % p.tiles_per_img;
+    const int pos0 = t_in * 128;                                  // first padded-flat position of this tile
+    const int row0 = p.flat ? 0 : pos0 / p.Wp;                    // first output row touched
+    const int a_off = p.flat ? 0 : pos0 - row0 * p.Wp;            // tile start inside the box, tap (0,0)
+
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 127) & ~(uintptr_t)127);
+    __shared__ __align__(8) uint64_t bars[2 * TC_STAGES + 1];
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int abort_s;
+    const uint32_t bar_full = smem_u32(&bars[0]), bar_empty = smem_u32(&bars[TC_STAGES]), bar_acc = smem_u32(&bars[2 * TC_STAGES]);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int stage_bytes = p.a_stage_bytes + p.b_stage_bytes;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < TC_STAGES; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
+        mbar_init(bar_acc, 1);
+        abort_s = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(p.tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_d = tmem_base_s;
+
+    if (warp == 0) {
+        // ---------------------------------------------------------------- TMA producer
+        if (lane == 0) {
+            for (int c = 0; c < p.nchunks; ++c) {
+                const int s = c % p.stages, it = c / p.stages;
+                if (it > 0 && !mbar_wait(bar_empty + 8 * s, (it - 1) & 1)) { atomicExch(&abort_s, 1); atomicExch(p.status, 1); break; }
+                const uint32_t a_dst = smem_u32(smem + s * stage_bytes), b_dst = a_dst + p.a_stage_bytes;
+                mbar_expect_tx(bar_full + 8 * s, (uint32_t)((p.kc / 8) * p.box_w * p.box_h * 16 + p.taps * p.b_tap_bytes));
+                const int x0 = p.flat ? pos0 : -p.pad, y0 = p.flat ? 0 : row0 - p.pad;
+                for (int pl = 0; pl < p.kc / 8; ++pl)
+                    tma_load_4d(a_dst + pl * p.plane_bytes, &p.map_a, bar_full + 8 * s, c * p.kc + pl * 8, x0, y0, img);
+                if (!p.b_mn_major) tma_load_4d(b_dst, &p.map_b, bar_full + 8 * s, 0, tn * p.n_tile, c * (p.kc / 8), 0);
+                else tma_load_4d(b_dst, &p.map_b, bar_full + 8 * s, 0, c * p.kc, tn * (p.n_tile / 8), 0);
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------------------------------------------------------- MMA issuer
+        if (lane == 0) {
+            // instruction descriptor: fp32 accumulate, bf16 x bf16, A K-major, B K-major or MN-major, N, M = 128
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)p.b_mn_major << 16) |
+                                   ((uint32_t)(p.n_tile >> 3) << 17) | ((128u >> 4) << 24);
+            const int ksz = p.taps == 9 ? 3 : 1;
+            bool ok = true;
+            for (int c = 0; c < p.nchunks && ok; ++c) {
+                const int s = c % p.stages, it = c / p.stages;
+                if (!mbar_wait(bar_full + 8 * s, it & 1)) { atomicExch(&abort_s, 1); atomicExch(p.status, 2); ok = false; break; }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t a_base = smem_u32(smem + s * stage_bytes), b_base = a_base + p.a_stage_bytes;
+                for (int t = 0; t < p.taps; ++t) {
+                    const int r = t / ksz, q = t % ksz;
+                    const int shift = p.flip ? ((ksz - 1 - r) * p.Wp + (ksz - 1 - q)) : (r * p.Wp + q);
+                    for (int k16 = 0; k16 < p.kc / 16; ++k16) {
+                        const uint64_t ad = smem_desc(a_base + 2 * k16 * p.plane_bytes + (a_off + shift) * 16, p.plane_bytes, 128);
+                        uint64_t bd;
+                        if (!p.b_mn_major) bd = smem_desc(b_base + t * p.b_tap_bytes + 2 * k16 * p.n_tile * 16, p.n_tile * 16, 128);
+                        else bd = smem_desc(b_base + t * p.b_tap_bytes + k16 * 256, 128, p.kc * 16);
+                        umma_bf16(tmem_d, ad, bd, idesc, (c | t | k16) ? 1u : 0u);
+                    }
+                }
+                umma_commit(bar_empty + 8 * s);          // stage reusable once these MMAs have read it
+            }
+            if (ok) umma_commit(bar_acc);                // accumulator complete
+        }
+    } else {
+        // ---------------------------------------------------------------- epilogue: 4 warps, one TMEM lane quadrant each
+        const int quad = warp & 3;
+        const int m = quad * 32 + lane;                  // row of the tile = TMEM lane
+        bool ok = mbar_wait(bar_acc, 0);
+        ok = __all_sync(0xffffffffu, ok);                // tcgen05.ld below is warp-collective
+        if (!ok) { atomicExch(&abort_s, 1); atomicExch(p.status, 3); }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        // padded-flat position -> output pixel
+        long long pix = -1;
+        if (p.flat) { const long long g = (long long)pos0 + m; if (g < (long long)p.W) pix = g; }
+        else {
+            const int pos = pos0 + m, i = pos / p.Wp, j = pos - i * p.Wp;
+            if (i < p.H && j < p.W) pix = ((long long)img * p.H + i) * p.W + j;
+        }
+        if (ok) {
+            for (int c0 = 0; c0 < p.n_tile; c0 += 16) {
+                uint32_t v[16];
+                tmem_ld16(tmem_d + ((uint32_t)(quad * 32) << 16) + (uint32_t)c0, v);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                if (pix >= 0) {
+                    const long long o = pix * p.ncol + tn * p.n_tile + c0;
+                    float f[16];
+#pragma unroll
+                    for (int k = 0; k < 16; ++k) f[k] = __uint_as_float(v[k]) * p.scale;
+                    if (p.add) {
+                        const uint4 a0 = *reinterpret_cast<const uint4*>(p.add + o), a1 = *reinterpret_cast<const uint4*>(p.add + o + 8);
+                        const uint32_t aw[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) {
+                            f[2 * k] += __uint_as_float(aw[k] << 16);
+                            f[2 * k + 1] += __uint_as_float(aw[k] & 0xFFFF0000u);
+                        }
+                    }
+                    uint32_t w[8];
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * k], f[2 * k + 1]);
+                        w[k] = *reinterpret_cast<uint32_t*>(&h);
+                    }
+                    *reinterpret_cast<uint4*>(p.out + o) = make_uint4(w[0], w[1], w[2], w[3]);
+                    *reinterpret_cast<uint4*>(p.out + o + 8) = make_uint4(w[4], w[5], w[6], w[7]);
+                }
+            }
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(p.tmem_cols) : "memory");
+    }
+}
+
+// ------------------------------------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* f = nullptr; cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)f;
+    }
+    return fn;
+}
+
+static bool encode4(CUtensorMap* m, const void* base, const uint64_t dims[4], const uint64_t strides_bytes[3], const uint32_t box[4]) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t d[4] = {dims[0], dims[1], dims[2], dims[3]};
+    cuuint64_t st[3] = {strides_bytes[0], strides_bytes[1], strides_bytes[2]};
+    cuuint32_t b[4] = {box[0], box[1], box[2], box[3]};
+    cuuint32_t es[4] = {1, 1, 1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), d, st, b, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+struct TcGeom { int stages, chan_a, ncol, n_tile, kc, nchunks, Wp, box_w, box_h, plane_bytes, a_stage, b_stage, b_tap, tiles_per_img, n_img, H, W, flat, tmem_cols; size_t smem; };
+
+// Decides whether (and how) the tensor-core kernel takes this problem.
+static bool tc_geometry(const ConvProb& p, int mode, TcGeom& g) {
+    if (mode == CONV_WGRAD) return false;
+    if (p.stride != 1 || (p.ksz != 1 && p.ksz != 3)) return false;
+    if (p.C % 16 || p.K % 16) return false;
+    if (((uintptr_t)p.act | (uintptr_t)p.wgt | (uintptr_t)p.out | (uintptr_t)p.add) & 15) return false;
+    g.chan_a = mode == CONV_FWD ? p.C : p.K;            // reduction channels
+    g.ncol = mode == CONV_FWD ? p.K : p.C;              // output channels
+    g.flat = p.ksz == 1;
+    const int taps = p.ksz * p.ksz;
+    if (g.flat) { g.n_img = 1; g.H = 1; g.W = p.N * p.H * p.W; g.Wp = g.W; g.box_w = 128; g.box_h = 1;
+        g.tiles_per_img = (int)(((long long)g.W + 127) / 128); }
+    else { g.n_img = p.N; g.H = p.H; g.W = p.W; g.Wp = p.W + 2; if (g.Wp > 128) return false;
+        const int rows = (g.Wp - 1 + 127) / g.Wp + 1;   // rows 128 consecutive positions can touch
+        g.box_w = g.Wp; g.box_h = std::min(rows, p.H) + 2; if (g.box_h > 256) return false;
+        g.tiles_per_img = (p.H * g.Wp + 127) / 128; }
+    g.n_tile = g.ncol; while (g.n_tile > 128) { if (g.n_tile % 2) return false; g.n_tile /= 2; }
+    if (g.n_tile % 16) return false;
+    int kc = g.chan_a > 64 ? 64 : g.chan_a;
+    while (kc > 16 && (taps * g.n_tile * kc * 2 > 80 * 1024 || g.chan_a % kc)) kc -= 16;
+    if (g.chan_a % kc || taps * g.n_tile * kc * 2 > 100 * 1024) return false;
+    g.kc = kc; g.nchunks = g.chan_a / kc;
+    // a plane must hold the box and cover every address an MMA can touch: 128 rows past the largest tap shift
+    const int max_read = (g.flat ? 0 : g.Wp - 1) + (p.ksz - 1) * g.Wp + (p.ksz - 1) + 128;
+    const int plane_px = std::max(g.box_w * g.box_h, max_read);
+    g.plane_bytes = ((plane_px * 16 + 127) / 128) * 128;
+    g.a_stage = (kc / 8) * g.plane_bytes;
+    g.b_tap = g.n_tile * kc * 2; g.b_stage = ((taps * g.b_tap + 127) / 128) * 128;
+    g.stages = g.nchunks > 1 ? TC_STAGES : 1;
+    g.smem = (size_t)g.stages * (g.a_stage + g.b_stage) + 256;
+    if (g.smem > 200 * 1024) return false;
+    g.tmem_cols = 32; while (g.tmem_cols < g.n_tile) g.tmem_cols *= 2;
+    return true;
+}
+
+bool conv_tc_supported(const ConvProb& p, int mode) { TcGeom g; return encode_fn() != nullptr && tc_geometry(p, mode, g); }
+size_t conv_tc_scratch_bytes(const ConvProb&, int) { return sizeof(TcProb) + 64; }
+
+static int* g_status = nullptr;      // one status word per process, zeroed at creation
+int* conv_tc_status_word() {
+    if (!g_status) { cudaMalloc(&g_status, 256); cudaMemset(g_status, 0, 256); }
+    return g_status;
+}
+int conv_tc_read_status() {
+    if (!g_status) return 0;
+    int v = 0; cudaMemcpy(&v, g_status, 4, cudaMemcpyDeviceToHost); return v;
+}
+
+// Fills a host-side TcProb for this problem.  Returns false when the problem is not supported.
+bool conv_tc_fill(const ConvProb& p, int mode, void* host_tc) {
+    TcGeom g; if (!tc_geometry(p, mode, g)) return false;
+    TcProb t; memset(&t, 0, sizeof(t));
+    const int taps = p.ksz * p.ksz;
+    // activations: (channel, x, y, image), bf16, channels contiguous
+    { const uint64_t dims[4] = {(uint64_t)g.chan_a, (uint64_t)g.W, (uint64_t)g.H, (uint64_t)g.n_img};
+      const uint64_t st[3] = {(uint64_t)g.chan_a * 2, (uint64_t)g.chan_a * 2 * g.W, (uint64_t)g.chan_a * 2 * g.W * g.H};
+      const uint32_t box[4] = {8, (uint32_t)g.box_w, (uint32_t)g.box_h, 1};
+      if (!encode4(&t.map_a, p.act, dims, st, box)) return false; }
+    // weights [K][k][k][C] viewed as (8 input channels, output channel K, input-channel group C/8, tap)
+    { const uint64_t dims[4] = {8, (uint64_t)p.K, (uint64_t)p.C / 8, (uint64_t)taps};
+      const uint64_t st[3] = {(uint64_t)taps * p.C * 2, 16, (uint64_t)p.C * 2};
+      uint32_t box[4];
+      if (mode == CONV_FWD) { box[0] = 8; box[1] = g.n_tile; box[2] = g.kc / 8; box[3] = taps; }
+      else { box[0] = 8; box[1] = g.kc; box[2] = g.n_tile / 8; box[3] = taps; }
+      if (!encode4(&t.map_b, p.wgt, dims, st, box)) return false; }
+    t.add = (const __nv_bfloat16*)p.add; t.out = (__nv_bfloat16*)p.out; t.status = conv_tc_status_word();
+    t.H = g.H; t.W = g.W; t.Wp = g.Wp; t.pad = p.ksz / 2; t.taps = taps; t.flip = mode == CONV_DGRAD ? 1 : 0;
+    t.n_img = g.n_img; t.tiles_per_img = g.tiles_per_img; t.tiles_n = g.ncol / g.n_tile; t.ncol = g.ncol; t.n_tile = g.n_tile;
+    t.kc = g.kc; t.nchunks = g.nchunks; t.box_w = g.box_w; t.box_h = g.box_h; t.plane_bytes = g.plane_bytes;
+    t.a_stage_bytes = g.a_stage; t.b_stage_bytes = g.b_stage; t.b_tap_bytes = g.b_tap; t.b_mn_major = mode == CONV_DGRAD ? 1 : 0;
+    t.tmem_cols = g.tmem_cols; t.flat = g.flat; t.scale = p.scale; t.stages = g.stages;
+    memcpy(host_tc, &t, sizeof(t));
+    return true;
+}
+size_t conv_tc_prob_bytes() { return sizeof(TcProb); }
+int conv_tc_tiles(const void* host_tc) { const TcProb* t = (const TcProb*)host_tc; return t->n_img * t->tiles_per_img * t->tiles_n; }
+size_t conv_tc_smem(const void* host_tc) {
+    const TcProb* t = (const TcProb*)host_tc; return (size_t)t->stages * (t->a_stage_bytes + t->b_stage_bytes) + 256;
+}
+
+void launch_conv_tc_probs(const void* d_tc, int nprob, int max_tiles, size_t max_smem, cudaStream_t s) {
+    static size_t configured = 0;
+    if (max_smem > configured) {
+        cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(200 * 1024 + 256));
+        configured = 200 * 1024 + 256;
+    }
+    conv_tc_kernel<<<dim3(max_tiles, nprob), TC_THREADS, max_smem, s>>>((const TcProb*)d_tc);
+}
+
 }  // namespace resist

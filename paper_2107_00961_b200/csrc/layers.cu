@@ -2,13 +2,17 @@
 // on caller-owned device tensors, run by the same kernels the local step uses.
 #include <algorithm>
 #include <string>
+#include <vector>
 #include "runtime.h"
 
 namespace resist {
 bool conv_tc_supported(const ConvProb& p, int mode);
-void launch_conv_tc(const ConvProb* d, int nprob, int max_tiles, int mode, cudaStream_t s);
-size_t conv_tc_scratch_bytes(const ConvProb& p, int mode);
-void conv_tc_prepare(ConvProb& p, int mode, void* scratch, int sm_count);
+bool conv_tc_fill(const ConvProb& p, int mode, void* host_tc);
+size_t conv_tc_prob_bytes();
+int conv_tc_tiles(const void* host_tc);
+size_t conv_tc_smem(const void* host_tc);
+void launch_conv_tc_probs(const void* d_tc, int nprob, int max_tiles, size_t max_smem, cudaStream_t s);
+int conv_tc_read_status();
 }
 using namespace resist;
 
@@ -38,7 +42,9 @@ extern "C" int resist_conv2d(int32_t mode, int32_t dtype, int32_t backend, const
     const bool tc = dtype == RESIST_BF16 && backend == RESIST_CONV_AUTO && conv_tc_supported(p, mode);
     if (used_backend) *used_backend = tc ? 1 : 0;
     size_t scratch = 0;
-    if (tc) scratch = conv_tc_scratch_bytes(p, mode);
+    std::vector<char> host_tc;
+    if (tc) { host_tc.resize(conv_tc_prob_bytes()); scratch = host_tc.size();
+        if (!conv_tc_fill(p, mode, host_tc.data())) { g_layer_error = "tensor map encoding failed"; return RESIST_ECUDA; } }
     else if (mode == CONV_WGRAD) {
         const int tiles = p.tiles_m * p.tiles_n;
         int want = (2 * sm + tiles - 1) / tiles; want = std::max(1, std::min(std::min(want, 64), ktiles));
@@ -48,11 +54,11 @@ extern "C" int resist_conv2d(int32_t mode, int32_t dtype, int32_t backend, const
     char* blob = nullptr;
     cudaError_t e = cudaMalloc(&blob, 1024 + scratch);
     if (e != cudaSuccess) { g_layer_error = cudaGetErrorString(e); return RESIST_ENOMEM; }
-    if (tc) conv_tc_prepare(p, mode, blob + 1024, sm);
-    else if (p.splits > 1) p.partial = (float*)(blob + 1024);
+    if (!tc && p.splits > 1) p.partial = (float*)(blob + 1024);
     e = cudaMemcpyAsync(blob, &p, sizeof(p), cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess && tc) e = cudaMemcpyAsync(blob + 1024, host_tc.data(), host_tc.size(), cudaMemcpyHostToDevice, st);
     if (e == cudaSuccess) {
-        if (tc) launch_conv_tc((ConvProb*)blob, 1, p.tiles_m * p.tiles_n * p.splits, mode, st);
+        if (tc) launch_conv_tc_probs(blob + 1024, 1, conv_tc_tiles(host_tc.data()), conv_tc_smem(host_tc.data()), st);
         else {
             launch_conv_ref((ConvProb*)blob, 1, p.tiles_m * p.tiles_n * p.splits, mode, dtype == RESIST_BF16, st);
             if (mode == CONV_WGRAD && p.splits > 1) launch_splitk_reduce((ConvProb*)blob, 1, p.M * p.Ncol, st);
@@ -62,6 +68,8 @@ extern "C" int resist_conv2d(int32_t mode, int32_t dtype, int32_t backend, const
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
     cudaFree(blob);
     if (e != cudaSuccess) { g_layer_error = cudaGetErrorString(e); return RESIST_ECUDA; }
+    if (tc) { const int stv = conv_tc_read_status();
+        if (stv) { g_layer_error = "a bounded device-side wait gave up (code " + std::to_string(stv) + ")"; return RESIST_ETIMEOUT; } }
     return RESIST_OK;
 }
 

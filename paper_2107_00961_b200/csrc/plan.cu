@@ -15,7 +15,11 @@ void held_segments(const resist_ctx* ctx, int sub, uint32_t bit, bool buffers, s
 int ensure_param_arrays(resist_ctx* ctx, int S);
 int ensure_seg_table(resist_ctx* ctx, int n);
 bool conv_tc_supported(const ConvProb& p, int mode);                                   // conv_tc.cu
-void launch_conv_tc(const ConvProb* d, int nprob, int max_tiles, int mode, cudaStream_t s);
+bool conv_tc_fill(const ConvProb& p, int mode, void* host_tc);
+size_t conv_tc_prob_bytes();
+int conv_tc_tiles(const void* host_tc);
+size_t conv_tc_smem(const void* host_tc);
+void launch_conv_tc_probs(const void* d_tc, int nprob, int max_tiles, size_t max_smem, cudaStream_t s);
 
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 static int out_dim(int h, int k, int stride) { return (h + 2 * ((k - 1) / 2) - k) / stride + 1; }
@@ -294,6 +298,7 @@ static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool s
     std::stable_sort(ops.begin(), ops.end(), [](const Op& a, const Op& b) { return a.key < b.key; });
     const double es = ctx->opts.dtype == RESIST_BF16 ? 2.0 : 4.0;
     std::vector<ConvProb> conv; std::vector<BnProb> bn; std::vector<PoolProb> pool; std::vector<HeadProb> head;
+    const size_t tcb = conv_tc_prob_bytes(); std::vector<char> tc; int n_tc = 0;
     struct HostSite { int arr; int idx; int field; int what; int sub; };
     std::vector<HostSite> sites;
     plan.launches.clear();
@@ -305,6 +310,21 @@ static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool s
             const Op& o = ops[k]; const int slot = single ? 0 : o.sub;
             switch (o.kind) {
                 case OP_CONV_FWD: case OP_CONV_DGRAD: case OP_CONV_WGRAD: case OP_SPLITK: {
+                    if (o.backend && o.kind != OP_SPLITK) {      // tensor-core problem: its own descriptor array
+                        if (k == i) L.first = n_tc;
+                        tc.resize((size_t)(n_tc + 1) * tcb);
+                        const int mode = o.kind == OP_CONV_FWD ? CONV_FWD : o.kind == OP_CONV_DGRAD ? CONV_DGRAD : CONV_WGRAD;
+                        if (!conv_tc_fill(o.conv, mode, tc.data() + (size_t)n_tc * tcb)) { ctx->err = "tensor map encoding failed"; return RESIST_ECUDA; }
+                        L.gx = std::max(L.gx, conv_tc_tiles(tc.data() + (size_t)n_tc * tcb));
+                        L.max_elems = std::max<long long>(L.max_elems, (long long)conv_tc_smem(tc.data() + (size_t)n_tc * tcb));
+                        ++n_tc;
+                        const ConvProb& p = o.conv;
+                        const double in_e = (double)p.N * p.H * p.W * p.C, out_e = (double)p.N * p.P * p.Q * p.K, w_e = (double)p.K * p.ksz * p.ksz * p.C;
+                        L.flops += 2.0 * out_e * p.ksz * p.ksz * p.C;
+                        if (o.kind == OP_CONV_WGRAD) L.bytes += es * (in_e + out_e) + 4.0 * w_e;
+                        else L.bytes += es * (in_e + out_e + w_e + (p.add ? (o.kind == OP_CONV_FWD ? out_e : in_e) : 0.0));
+                        break;
+                    }
                     if (k == i) L.first = (int)conv.size();
                     if (o.patch_images) sites.push_back({0, (int)conv.size(), 0, 0, slot});
                     conv.push_back(o.conv);
@@ -362,6 +382,7 @@ static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool s
     const size_t o_head = off; off += align_up(head.size() * sizeof(HeadProb), 256);
     const size_t o_site = off; off += align_up(sites.size() * sizeof(PatchSite), 256);
     const size_t o_seg = off;  off += align_up(segs.size() * sizeof(Segment), 256);
+    const size_t o_tc = off;   off += align_up(tc.size(), 256);
     ctx_free(ctx, plan.d_blob);
     plan.d_blob = ctx_alloc(ctx, off + 256); plan.blob_bytes = off;
     if (!plan.d_blob) { ctx->err = "allocator returned NULL for the launch plan"; return RESIST_ENOMEM; }
@@ -385,6 +406,8 @@ static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool s
     if (!head.empty()) memcpy(host.data() + o_head, head.data(), head.size() * sizeof(HeadProb));
     if (!dsites.empty()) memcpy(host.data() + o_site, dsites.data(), dsites.size() * sizeof(PatchSite));
     if (!segs.empty()) memcpy(host.data() + o_seg, segs.data(), segs.size() * sizeof(Segment));
+    if (!tc.empty()) memcpy(host.data() + o_tc, tc.data(), tc.size());
+    plan.d_tc = base + o_tc; plan.tc_stride = tcb;
     cudaError_t e = cudaMemcpyAsync(plan.d_blob, host.data(), off, cudaMemcpyHostToDevice, st);
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
     if (e != cudaSuccess) { ctx->err = std::string("plan upload: ") + cudaGetErrorString(e); return RESIST_ECUDA; }
@@ -458,7 +481,7 @@ static int run_plan(resist_ctx* ctx, Plan& plan, const PatchArgs& pa, bool updat
         switch (L.kind) {
             case OP_CONV_FWD: case OP_CONV_DGRAD: case OP_CONV_WGRAD: {
                 const int mode = L.kind == OP_CONV_FWD ? CONV_FWD : L.kind == OP_CONV_DGRAD ? CONV_DGRAD : CONV_WGRAD;
-                if (L.backend) launch_conv_tc(plan.d_conv + L.first, L.count, L.gx, mode, st);
+                if (L.backend) launch_conv_tc_probs((const char*)plan.d_tc + (size_t)L.first * plan.tc_stride, L.count, L.gx, (size_t)L.max_elems, st);
                 else launch_conv_ref(plan.d_conv + L.first, L.count, L.gx, mode, bf, st);
                 ++n_launch; break; }
             case OP_SPLITK: launch_splitk_reduce(plan.d_conv + L.first, L.count, (int)L.max_elems, st); ++n_launch; break;

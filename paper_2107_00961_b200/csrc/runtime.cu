@@ -76,6 +76,14 @@ void ctx_free(resist_ctx* ctx, void* p) {
 }
 
 void free_plan(resist_ctx* ctx, Plan& p);   // plan.cu
+int conv_tc_read_status();                  // conv_tc.cu
+
+// after a synchronisation: did any bounded device-side wait give up?
+static int device_status(resist_ctx* ctx) {
+    const int v = conv_tc_read_status();
+    if (v) { ctx->err = "a bounded device-side wait gave up (code " + std::to_string(v) + ")"; return RESIST_ETIMEOUT; }
+    return RESIST_OK;
+}
 
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -234,7 +242,7 @@ int resist_get_params(resist_ctx* ctx, int32_t subnet, float* host_params, float
     const float* b = subnet < 0 ? ctx->pa.global_buf : ctx->pa.buf + (long long)subnet * ctx->pa.nbuf;
     if (host_params) CK(cudaMemcpy(host_params, p, (size_t)ctx->L.n_params * 4, cudaMemcpyDeviceToHost));
     if (host_buffers) CK(cudaMemcpy(host_buffers, b, (size_t)ctx->L.n_buffers * 4, cudaMemcpyDeviceToHost));
-    return RESIST_OK;
+    return device_status(ctx);
 }
 
 int resist_get_grads(resist_ctx* ctx, int32_t subnet, float* host_grads) {
@@ -246,7 +254,7 @@ int resist_get_grads(resist_ctx* ctx, int32_t subnet, float* host_grads) {
     for (size_t b = 0; b < ctx->L.blk.size(); ++b)          // blocks this sub-ResNet does not hold have no gradient
         if (!(ctx->mask[b] >> subnet & 1u))
             std::fill(host_grads + ctx->L.blk[b].begin, host_grads + ctx->L.blk[b].end, 0.f);
-    return RESIST_OK;
+    return device_status(ctx);
 }
 
 int resist_get_logits(resist_ctx* ctx, int32_t subnet, float* host_logits) {
@@ -370,7 +378,7 @@ int resist_aggregate(resist_ctx* ctx, resist_stream stream) {
     ctx->prof.end(st); ctx->prof.collect(st);
     CK(cudaGetLastError());
     CK(cudaStreamSynchronize(st));
-    return RESIST_OK;
+    return device_status(ctx);
 }
 
 }  // extern "C"
