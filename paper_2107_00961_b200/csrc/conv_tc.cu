@@ -221,6 +221,149 @@ __global__ void __launch_bounds__(TC_THREADS) conv_tc_kernel(const TcProb* __res
     }
 }
 
+// ------------------------------------------------------------------------------------------------ wgrad
+// dw[k][r][s][c] = sum over output pixels of dy[pix][k] * a[pix + shift(r,s)][c].  The reduction runs over the
+// padded-flat pixel positions of the forward kernel, 128 per pipeline stage: D[cout (128 lanes), cin] per tap,
+// A = dy^T and B = shifted a, both MN-major straight from their 8-channel planes.  dy is fetched with a box that
+// starts at column 0, so the pad positions of every row and the rows past the image read as zero and add nothing.
+// A CTA accumulates a range of pixel tiles for a group of taps and writes an fp32 partial; a second kernel adds
+// the partials in a fixed order.
+struct alignas(64) TcWgradProb {
+    CUtensorMap map_dy;       // (channel k, x, y, image)
+    CUtensorMap map_a;        // (channel c, x, y, image)
+    float* partial;           // [splits][taps][cout][cin]
+    float* out;               // [cout][taps][cin]
+    int* status;
+    int H, W, Wp, pad, taps, ksz, flat;
+    int n_img, tiles_per_img, pixel_tiles;       // pixel tiles in total = n_img * tiles_per_img
+    int cout, cin, m_tiles, n_tile, n_tiles;     // cout tiles of 128 rows, cin tiles of n_tile columns
+    int tap_groups, taps_per_group, splits, tiles_per_split;
+    int box_w, box_h_a, box_h_dy;
+    int plane_a, plane_dy;                       // bytes of one 8-channel plane
+    int dy_planes, a_planes;                     // planes fetched per stage
+    int stage_bytes, stages, tmem_cols;
+};
+
+__global__ void __launch_bounds__(TC_THREADS) conv_wgrad_tc_kernel(const TcWgradProb* __restrict__ probs) {
+    const TcWgradProb& p = probs[blockIdx.y];
+    const int ctas = p.m_tiles * p.n_tiles * p.tap_groups * p.splits;
+    if ((int)blockIdx.x >= ctas) return;
+    int id = blockIdx.x;
+    const int split = id % p.splits; id /= p.splits;
+    const int tg = id % p.tap_groups; id /= p.tap_groups;
+    const int tn = id % p.n_tiles; const int tm = id / p.n_tiles;
+    const int t_begin = split * p.tiles_per_split;
+    int t_end = t_begin + p.tiles_per_split; if (t_end > p.pixel_tiles) t_end = p.pixel_tiles;
+    const int tap0 = tg * p.taps_per_group;
+    int ntap = p.taps - tap0; if (ntap > p.taps_per_group) ntap = p.taps_per_group;
+    const int nt = t_end - t_begin;
+
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 127) & ~(uintptr_t)127);
+    __shared__ __align__(8) uint64_t bars[2 * 4 + 1];
+    __shared__ uint32_t tmem_base_s;
+    const uint32_t bar_full = smem_u32(&bars[0]), bar_empty = smem_u32(&bars[4]), bar_acc = smem_u32(&bars[8]);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.stages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
+        mbar_init(bar_acc, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(p.tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_d = tmem_base_s;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int i = 0; i < nt; ++i) {
+                const int s = i % p.stages, it = i / p.stages;
+                if (it > 0 && !mbar_wait(bar_empty + 8 * s, (it - 1) & 1)) { atomicExch(p.status, 11); break; }
+                const int t = t_begin + i, img = t / p.tiles_per_img, pos0 = (t % p.tiles_per_img) * 128;
+                const int row0 = p.flat ? 0 : pos0 / p.Wp;
+                const uint32_t dy_dst = smem_u32(smem + s * p.stage_bytes), a_dst = dy_dst + p.dy_planes * p.plane_dy;
+                mbar_expect_tx(bar_full + 8 * s, (uint32_t)(p.dy_planes * p.box_w * p.box_h_dy * 16 + p.a_planes * p.box_w * p.box_h_a * 16));
+                for (int pl = 0; pl < p.dy_planes; ++pl)
+                    tma_load_4d(dy_dst + pl * p.plane_dy, &p.map_dy, bar_full + 8 * s, tm * 128 + pl * 8, p.flat ? pos0 : 0, row0, img);
+                for (int pl = 0; pl < p.a_planes; ++pl)
+                    tma_load_4d(a_dst + pl * p.plane_a, &p.map_a, bar_full + 8 * s, tn * p.n_tile + pl * 8, p.flat ? pos0 : -p.pad,
+                                p.flat ? 0 : row0 - p.pad, img);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // fp32 accumulate, bf16 x bf16, A and B MN-major, N = n_tile, M = 128
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) | ((uint32_t)(p.n_tile >> 3) << 17) | ((128u >> 4) << 24);
+            bool ok = true;
+            for (int i = 0; i < nt && ok; ++i) {
+                const int s = i % p.stages, it = i / p.stages;
+                if (!mbar_wait(bar_full + 8 * s, it & 1)) { atomicExch(p.status, 12); ok = false; break; }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const int pos0 = ((t_begin + i) % p.tiles_per_img) * 128;
+                const int off = p.flat ? 0 : pos0 % p.Wp;
+                const uint32_t dy_base = smem_u32(smem + s * p.stage_bytes), a_base = dy_base + p.dy_planes * p.plane_dy;
+                for (int tt = 0; tt < ntap; ++tt) {
+                    const int t = tap0 + tt, r = t / p.ksz, q = t % p.ksz;
+                    for (int k16 = 0; k16 < 8; ++k16) {
+                        const uint64_t ad = smem_desc(dy_base + (off + k16 * 16) * 16, 128, p.plane_dy);
+                        const uint64_t bd = smem_desc(a_base + (off + r * p.Wp + q + k16 * 16) * 16, 128, p.plane_a);
+                        umma_bf16(tmem_d + (uint32_t)(tt * p.n_tile), ad, bd, idesc, (i | k16) ? 1u : 0u);
+                    }
+                }
+                umma_commit(bar_empty + 8 * s);
+            }
+            if (ok) umma_commit(bar_acc);
+        }
+    } else {
+        const int quad = warp & 3, m = quad * 32 + lane;
+        bool ok = nt > 0 ? mbar_wait(bar_acc, 0) : true;
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) atomicExch(p.status, 13);
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const int k = tm * 128 + m;
+        if (ok && quad * 32 < p.cout - tm * 128) {            // warp-uniform: this lane quadrant holds real output channels
+            for (int tt = 0; tt < ntap; ++tt) {
+                float* dst = p.partial + (((long long)split * p.taps + tap0 + tt) * p.cout + k) * p.cin + tn * p.n_tile;
+                for (int c0 = 0; c0 < p.n_tile; c0 += 16) {
+                    uint32_t v[16];
+                    if (nt > 0) { tmem_ld16(tmem_d + ((uint32_t)(quad * 32) << 16) + (uint32_t)(tt * p.n_tile + c0), v);
+                        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+                    else { for (int j = 0; j < 16; ++j) v[j] = 0u; }
+                    if (k < p.cout) {
+#pragma unroll
+                        for (int j = 0; j < 16; j += 4)
+                            *reinterpret_cast<uint4*>(dst + c0 + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                    }
+                }
+            }
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(p.tmem_cols) : "memory");
+    }
+}
+
+// out[k][t][c] = sum over splits (ascending) of partial[split][t][k][c]
+__global__ void __launch_bounds__(256) wgrad_tc_reduce_kernel(const TcWgradProb* __restrict__ probs) {
+    const TcWgradProb& p = probs[blockIdx.y];
+    const long long n = (long long)p.taps * p.cout * p.cin;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+        const int c = (int)(i % p.cin); const long long r = i / p.cin; const int t = (int)(r % p.taps); const int k = (int)(r / p.taps);
+        const long long src = ((long long)t * p.cout + k) * p.cin + c;
+        float s = 0.f;
+        for (int sp = 0; sp < p.splits; ++sp) s += p.partial[(long long)sp * n + src];
+        p.out[i] = s;
+    }
+}
+
 // ------------------------------------------------------------------------------------------------ host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
@@ -335,6 +478,94 @@ void launch_conv_tc_probs(const void* d_tc, int nprob, int max_tiles, size_t max
         configured = 200 * 1024 + 256;
     }
     conv_tc_kernel<<<dim3(max_tiles, nprob), TC_THREADS, max_smem, s>>>((const TcProb*)d_tc);
+}
+
+// ---- wgrad host side
+struct WgGeom { int flat, n_img, H, W, Wp, tiles_per_img, pixel_tiles, m_tiles, n_tile, n_tiles, tap_groups, taps_per_group, splits,
+                tiles_per_split, box_w, box_h_a, box_h_dy, plane_a, plane_dy, dy_planes, a_planes, stage_bytes, stages, tmem_cols; size_t smem, partial_bytes; };
+
+static bool wg_geometry(const ConvProb& p, int target_ctas, WgGeom& g) {
+    if (p.stride != 1 || (p.ksz != 1 && p.ksz != 3)) return false;
+    if (p.C % 16 || p.K % 8) return false;
+    if (p.K > 128 && p.K % 128) return false;
+    if (((uintptr_t)p.act | (uintptr_t)p.wgt) & 15) return false;
+    const int taps = p.ksz * p.ksz;
+    g.flat = p.ksz == 1;
+    int rows = 1;
+    if (g.flat) { g.n_img = 1; g.H = 1; g.W = p.N * p.H * p.W; g.Wp = g.W; g.box_w = 128; g.tiles_per_img = (int)(((long long)g.W + 127) / 128); }
+    else { g.n_img = p.N; g.H = p.H; g.W = p.W; g.Wp = p.W + 2; if (g.Wp > 128) return false;
+        // every one of the 128 positions of a stage enters the reduction, so all of them must hold data or the
+        // zero fill of the TMA box, never stale shared memory: the boxes cover every row 128 positions can touch
+        // (rows past the image come back as zeros), and the activation box has one row to spare for the two
+        // pixels the last tap reaches past its halo
+        rows = (g.Wp - 1 + 127) / g.Wp + 1; g.box_w = g.Wp; g.tiles_per_img = (p.H * g.Wp + 127) / 128; }
+    g.box_h_dy = rows; g.box_h_a = g.flat ? 1 : rows + 3;
+    if (g.box_h_a > 256) return false;
+    g.pixel_tiles = g.n_img * g.tiles_per_img;
+    g.m_tiles = (p.K + 127) / 128;
+    g.n_tile = p.C; while (g.n_tile > 256 || (g.n_tile > 64 && taps > 1 && g.n_tile * 3 > 512)) { if (g.n_tile % 32) return false; g.n_tile /= 2; }
+    g.n_tiles = p.C / g.n_tile;
+    g.taps_per_group = std::min(taps, 512 / g.n_tile); if (taps == 9 && g.taps_per_group < 9) g.taps_per_group = std::min(g.taps_per_group, 3);
+    if (g.taps_per_group < 1) return false;
+    g.tap_groups = (taps + g.taps_per_group - 1) / g.taps_per_group;
+    g.tmem_cols = 32; while (g.tmem_cols < g.taps_per_group * g.n_tile) g.tmem_cols *= 2;
+    if (g.tmem_cols > 512) return false;
+    // planes: the MMA addresses 16 planes of dy whatever cout is; the bytes past the real planes only have to exist
+    g.plane_a = ((g.box_w * g.box_h_a * 16 + 127) / 128) * 128;
+    g.plane_dy = ((g.box_w * g.box_h_dy * 16 + 127) / 128) * 128;
+    g.dy_planes = std::min(p.K, 128) / 8;
+    g.a_planes = g.n_tile / 8;
+    g.stage_bytes = g.dy_planes * g.plane_dy + g.a_planes * g.plane_a;
+    const int slack = 16 * g.plane_dy + 256;
+    g.stages = 4; while (g.stages > 1 && (size_t)g.stages * g.stage_bytes + slack > 200 * 1024) --g.stages;
+    g.smem = (size_t)g.stages * g.stage_bytes + slack;
+    if (g.smem > 200 * 1024) return false;
+    const int fixed = g.m_tiles * g.n_tiles * g.tap_groups;
+    int want = std::max(1, target_ctas / fixed); if (want > g.pixel_tiles) want = g.pixel_tiles; if (want > 256) want = 256;
+    g.tiles_per_split = (g.pixel_tiles + want - 1) / want; g.splits = (g.pixel_tiles + g.tiles_per_split - 1) / g.tiles_per_split;
+    g.partial_bytes = (size_t)g.splits * taps * p.K * p.C * 4;
+    return true;
+}
+
+bool conv_wgrad_tc_supported(const ConvProb& p, int target_ctas, size_t* partial_bytes) {
+    WgGeom g; if (!encode_fn() || !wg_geometry(p, target_ctas, g)) return false;
+    if (partial_bytes) *partial_bytes = g.partial_bytes;
+    return true;
+}
+
+// p.act = a, p.wgt = dy, p.out = dw (fp32), p.partial = workspace of at least partial_bytes
+bool conv_wgrad_tc_fill(const ConvProb& p, int target_ctas, void* host_tc) {
+    WgGeom g; if (!wg_geometry(p, target_ctas, g)) return false;
+    TcWgradProb t; memset(&t, 0, sizeof(t));
+    { const uint64_t dims[4] = {(uint64_t)p.K, (uint64_t)g.W, (uint64_t)g.H, (uint64_t)g.n_img};
+      const uint64_t st[3] = {(uint64_t)p.K * 2, (uint64_t)p.K * 2 * g.W, (uint64_t)p.K * 2 * g.W * g.H};
+      const uint32_t box[4] = {8, (uint32_t)g.box_w, (uint32_t)g.box_h_dy, 1};
+      if (!encode4(&t.map_dy, p.wgt, dims, st, box)) return false; }
+    { const uint64_t dims[4] = {(uint64_t)p.C, (uint64_t)g.W, (uint64_t)g.H, (uint64_t)g.n_img};
+      const uint64_t st[3] = {(uint64_t)p.C * 2, (uint64_t)p.C * 2 * g.W, (uint64_t)p.C * 2 * g.W * g.H};
+      const uint32_t box[4] = {8, (uint32_t)g.box_w, (uint32_t)g.box_h_a, 1};
+      if (!encode4(&t.map_a, p.act, dims, st, box)) return false; }
+    t.partial = p.partial; t.out = (float*)p.out; t.status = conv_tc_status_word();
+    t.H = g.H; t.W = g.W; t.Wp = g.Wp; t.pad = p.ksz / 2; t.taps = p.ksz * p.ksz; t.ksz = p.ksz; t.flat = g.flat;
+    t.n_img = g.n_img; t.tiles_per_img = g.tiles_per_img; t.pixel_tiles = g.pixel_tiles;
+    t.cout = p.K; t.cin = p.C; t.m_tiles = g.m_tiles; t.n_tile = g.n_tile; t.n_tiles = g.n_tiles;
+    t.tap_groups = g.tap_groups; t.taps_per_group = g.taps_per_group; t.splits = g.splits; t.tiles_per_split = g.tiles_per_split;
+    t.box_w = g.box_w; t.box_h_a = g.box_h_a; t.box_h_dy = g.box_h_dy; t.plane_a = g.plane_a; t.plane_dy = g.plane_dy;
+    t.dy_planes = g.dy_planes; t.a_planes = g.a_planes; t.stage_bytes = g.stage_bytes; t.stages = g.stages; t.tmem_cols = g.tmem_cols;
+    memcpy(host_tc, &t, sizeof(t));
+    return true;
+}
+size_t conv_wgrad_tc_prob_bytes() { return sizeof(TcWgradProb); }
+int conv_wgrad_tc_ctas(const void* h) { const TcWgradProb* t = (const TcWgradProb*)h; return t->m_tiles * t->n_tiles * t->tap_groups * t->splits; }
+size_t conv_wgrad_tc_smem(const void* h) { const TcWgradProb* t = (const TcWgradProb*)h; return (size_t)t->stages * t->stage_bytes + 16 * t->plane_dy + 256; }
+long long conv_wgrad_tc_out_elems(const void* h) { const TcWgradProb* t = (const TcWgradProb*)h; return (long long)t->taps * t->cout * t->cin; }
+
+void launch_conv_wgrad_tc_probs(const void* d_tc, int nprob, int max_ctas, size_t max_smem, long long max_out, cudaStream_t s) {
+    static bool configured = false;
+    if (!configured) { cudaFuncSetAttribute(conv_wgrad_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(200 * 1024 + 256)); configured = true; }
+    conv_wgrad_tc_kernel<<<dim3(max_ctas, nprob), TC_THREADS, max_smem, s>>>((const TcWgradProb*)d_tc);
+    long long gx = (max_out + 255) / 256; if (gx > 592) gx = 592; if (gx < 1) gx = 1;
+    wgrad_tc_reduce_kernel<<<dim3((unsigned)gx, nprob), 256, 0, s>>>((const TcWgradProb*)d_tc);
 }
 
 }  // namespace resist

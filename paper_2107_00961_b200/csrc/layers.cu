@@ -13,6 +13,13 @@ int conv_tc_tiles(const void* host_tc);
 size_t conv_tc_smem(const void* host_tc);
 void launch_conv_tc_probs(const void* d_tc, int nprob, int max_tiles, size_t max_smem, cudaStream_t s);
 int conv_tc_read_status();
+bool conv_wgrad_tc_supported(const ConvProb& p, int target_ctas, size_t* partial_bytes);
+bool conv_wgrad_tc_fill(const ConvProb& p, int target_ctas, void* host_tc);
+size_t conv_wgrad_tc_prob_bytes();
+int conv_wgrad_tc_ctas(const void* h);
+size_t conv_wgrad_tc_smem(const void* h);
+long long conv_wgrad_tc_out_elems(const void* h);
+void launch_conv_wgrad_tc_probs(const void* d_tc, int nprob, int max_ctas, size_t max_smem, long long max_out, cudaStream_t s);
 }
 using namespace resist;
 
@@ -39,11 +46,14 @@ extern "C" int resist_conv2d(int32_t mode, int32_t dtype, int32_t backend, const
     p.tiles_m = (p.M + 63) / 64; p.tiles_n = (p.Ncol + 63) / 64; p.splits = 1;
     const int ktiles = (p.Kred + 15) / 16; p.ktiles_per_split = ktiles;
     int sm = 148; int dev = 0; cudaGetDevice(&dev); cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev);
-    const bool tc = dtype == RESIST_BF16 && backend == RESIST_CONV_AUTO && conv_tc_supported(p, mode);
+    size_t wg_partial = 0;
+    const bool tc = dtype == RESIST_BF16 && backend == RESIST_CONV_AUTO &&
+                    (mode == CONV_WGRAD ? conv_wgrad_tc_supported(p, 2 * sm, &wg_partial) : conv_tc_supported(p, mode));
     if (used_backend) *used_backend = tc ? 1 : 0;
     size_t scratch = 0;
     std::vector<char> host_tc;
-    if (tc) { host_tc.resize(conv_tc_prob_bytes()); scratch = host_tc.size();
+    if (tc && mode == CONV_WGRAD) { host_tc.resize(conv_wgrad_tc_prob_bytes()); scratch = 1024 + wg_partial; }
+    else if (tc) { host_tc.resize(conv_tc_prob_bytes()); scratch = host_tc.size();
         if (!conv_tc_fill(p, mode, host_tc.data())) { g_layer_error = "tensor map encoding failed"; return RESIST_ECUDA; } }
     else if (mode == CONV_WGRAD) {
         const int tiles = p.tiles_m * p.tiles_n;
@@ -55,10 +65,14 @@ extern "C" int resist_conv2d(int32_t mode, int32_t dtype, int32_t backend, const
     cudaError_t e = cudaMalloc(&blob, 1024 + scratch);
     if (e != cudaSuccess) { g_layer_error = cudaGetErrorString(e); return RESIST_ENOMEM; }
     if (!tc && p.splits > 1) p.partial = (float*)(blob + 1024);
+    if (tc && mode == CONV_WGRAD) { p.partial = (float*)(blob + 2048);
+        if (!conv_wgrad_tc_fill(p, 2 * sm, host_tc.data())) { cudaFree(blob); g_layer_error = "tensor map encoding failed"; return RESIST_ECUDA; } }
     e = cudaMemcpyAsync(blob, &p, sizeof(p), cudaMemcpyHostToDevice, st);
     if (e == cudaSuccess && tc) e = cudaMemcpyAsync(blob + 1024, host_tc.data(), host_tc.size(), cudaMemcpyHostToDevice, st);
     if (e == cudaSuccess) {
-        if (tc) launch_conv_tc_probs(blob + 1024, 1, conv_tc_tiles(host_tc.data()), conv_tc_smem(host_tc.data()), st);
+        if (tc && mode == CONV_WGRAD) launch_conv_wgrad_tc_probs(blob + 1024, 1, conv_wgrad_tc_ctas(host_tc.data()), conv_wgrad_tc_smem(host_tc.data()),
+                                                                 conv_wgrad_tc_out_elems(host_tc.data()), st);
+        else if (tc) launch_conv_tc_probs(blob + 1024, 1, conv_tc_tiles(host_tc.data()), conv_tc_smem(host_tc.data()), st);
         else {
             launch_conv_ref((ConvProb*)blob, 1, p.tiles_m * p.tiles_n * p.splits, mode, dtype == RESIST_BF16, st);
             if (mode == CONV_WGRAD && p.splits > 1) launch_splitk_reduce((ConvProb*)blob, 1, p.M * p.Ncol, st);

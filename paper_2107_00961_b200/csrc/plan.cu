@@ -20,6 +20,14 @@ size_t conv_tc_prob_bytes();
 int conv_tc_tiles(const void* host_tc);
 size_t conv_tc_smem(const void* host_tc);
 void launch_conv_tc_probs(const void* d_tc, int nprob, int max_tiles, size_t max_smem, cudaStream_t s);
+bool conv_wgrad_tc_supported(const ConvProb& p, int target_ctas, size_t* partial_bytes);
+bool conv_wgrad_tc_fill(const ConvProb& p, int target_ctas, void* host_tc);
+size_t conv_wgrad_tc_prob_bytes();
+int conv_wgrad_tc_ctas(const void* h);
+size_t conv_wgrad_tc_smem(const void* h);
+long long conv_wgrad_tc_out_elems(const void* h);
+void launch_conv_wgrad_tc_probs(const void* d_tc, int nprob, int max_ctas, size_t max_smem, long long max_out, cudaStream_t s);
+static int wgrad_target_ctas(const resist_ctx* ctx) { return std::max(8, 2 * ctx->sm_count / std::max(1, ctx->S)); }
 
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 static int out_dim(int h, int k, int stride) { return (h + 2 * ((k - 1) / 2) - k) / stride + 1; }
@@ -88,7 +96,12 @@ struct Builder {
         p.tiles_m = (p.M + 63) / 64; p.tiles_n = (p.Ncol + 63) / 64; p.splits = 1;
         const int ktiles = (p.Kred + 15) / 16; p.ktiles_per_split = ktiles;
         flops += 2LL * rows_out * p.K * p.ksz * p.ksz * p.C;
-        op.backend = (ctx->opts.dtype == RESIST_BF16 && ctx->opts.conv_backend == RESIST_CONV_AUTO && conv_tc_supported(p, mode)) ? 1 : 0;
+        const bool tc_ok = ctx->opts.dtype == RESIST_BF16 && ctx->opts.conv_backend == RESIST_CONV_AUTO;
+        if (mode == CONV_WGRAD) {
+            size_t pb = 0;
+            op.backend = (tc_ok && !patch && conv_wgrad_tc_supported(p, wgrad_target_ctas(ctx), &pb)) ? 1 : 0;
+            if (op.backend) { wgrad_partial_need = std::max(wgrad_partial_need, pb); p.partial = wgrad_partial; }
+        } else op.backend = (tc_ok && conv_tc_supported(p, mode)) ? 1 : 0;
         if (op.backend) ++n_tc; else ++n_cc;
         if (mode == CONV_WGRAD && !op.backend) {
             const int tiles = p.tiles_m * p.tiles_n;
@@ -299,6 +312,7 @@ static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool s
     const double es = ctx->opts.dtype == RESIST_BF16 ? 2.0 : 4.0;
     std::vector<ConvProb> conv; std::vector<BnProb> bn; std::vector<PoolProb> pool; std::vector<HeadProb> head;
     const size_t tcb = conv_tc_prob_bytes(); std::vector<char> tc; int n_tc = 0;
+    const size_t wtcb = conv_wgrad_tc_prob_bytes(); std::vector<char> wtc; int n_wtc = 0;
     struct HostSite { int arr; int idx; int field; int what; int sub; };
     std::vector<HostSite> sites;
     plan.launches.clear();
@@ -310,6 +324,20 @@ static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool s
             const Op& o = ops[k]; const int slot = single ? 0 : o.sub;
             switch (o.kind) {
                 case OP_CONV_FWD: case OP_CONV_DGRAD: case OP_CONV_WGRAD: case OP_SPLITK: {
+                    if (o.backend && o.kind == OP_CONV_WGRAD) {  // tensor-core wgrad: its own descriptor array
+                        if (k == i) L.first = n_wtc;
+                        wtc.resize((size_t)(n_wtc + 1) * wtcb);
+                        char* h = wtc.data() + (size_t)n_wtc * wtcb;
+                        if (!conv_wgrad_tc_fill(o.conv, wgrad_target_ctas(ctx), h)) { ctx->err = "tensor map encoding failed"; return RESIST_ECUDA; }
+                        L.gx = std::max(L.gx, conv_wgrad_tc_ctas(h));
+                        L.max_elems = std::max<long long>(L.max_elems, (long long)conv_wgrad_tc_smem(h));
+                        L.max_b = (int)std::max<long long>(L.max_b, conv_wgrad_tc_out_elems(h));
+                        ++n_wtc;
+                        const ConvProb& p = o.conv;
+                        const double in_e = (double)p.N * p.H * p.W * p.C, out_e = (double)p.N * p.P * p.Q * p.K, w_e = (double)p.K * p.ksz * p.ksz * p.C;
+                        L.flops += 2.0 * out_e * p.ksz * p.ksz * p.C; L.bytes += es * (in_e + out_e) + 4.0 * w_e;
+                        break;
+                    }
                     if (o.backend && o.kind != OP_SPLITK) {      // tensor-core problem: its own descriptor array
                         if (k == i) L.first = n_tc;
                         tc.resize((size_t)(n_tc + 1) * tcb);
@@ -383,6 +411,7 @@ static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool s
     const size_t o_site = off; off += align_up(sites.size() * sizeof(PatchSite), 256);
     const size_t o_seg = off;  off += align_up(segs.size() * sizeof(Segment), 256);
     const size_t o_tc = off;   off += align_up(tc.size(), 256);
+    const size_t o_wtc = off;  off += align_up(wtc.size(), 256);
     ctx_free(ctx, plan.d_blob);
     plan.d_blob = ctx_alloc(ctx, off + 256); plan.blob_bytes = off;
     if (!plan.d_blob) { ctx->err = "allocator returned NULL for the launch plan"; return RESIST_ENOMEM; }
@@ -408,6 +437,8 @@ static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool s
     if (!segs.empty()) memcpy(host.data() + o_seg, segs.data(), segs.size() * sizeof(Segment));
     if (!tc.empty()) memcpy(host.data() + o_tc, tc.data(), tc.size());
     plan.d_tc = base + o_tc; plan.tc_stride = tcb;
+    if (!wtc.empty()) memcpy(host.data() + o_wtc, wtc.data(), wtc.size());
+    plan.d_wtc = base + o_wtc; plan.wtc_stride = wtcb;
     cudaError_t e = cudaMemcpyAsync(plan.d_blob, host.data(), off, cudaMemcpyHostToDevice, st);
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
     if (e != cudaSuccess) { ctx->err = std::string("plan upload: ") + cudaGetErrorString(e); return RESIST_ECUDA; }
@@ -481,7 +512,8 @@ static int run_plan(resist_ctx* ctx, Plan& plan, const PatchArgs& pa, bool updat
         switch (L.kind) {
             case OP_CONV_FWD: case OP_CONV_DGRAD: case OP_CONV_WGRAD: {
                 const int mode = L.kind == OP_CONV_FWD ? CONV_FWD : L.kind == OP_CONV_DGRAD ? CONV_DGRAD : CONV_WGRAD;
-                if (L.backend) launch_conv_tc_probs((const char*)plan.d_tc + (size_t)L.first * plan.tc_stride, L.count, L.gx, (size_t)L.max_elems, st);
+                if (L.backend && mode == CONV_WGRAD) { launch_conv_wgrad_tc_probs((const char*)plan.d_wtc + (size_t)L.first * plan.wtc_stride, L.count, L.gx, (size_t)L.max_elems, L.max_b, st); ++n_launch; }
+                else if (L.backend) launch_conv_tc_probs((const char*)plan.d_tc + (size_t)L.first * plan.tc_stride, L.count, L.gx, (size_t)L.max_elems, st);
                 else launch_conv_ref(plan.d_conv + L.first, L.count, L.gx, mode, bf, st);
                 ++n_launch; break; }
             case OP_SPLITK: launch_splitk_reduce(plan.d_conv + L.first, L.count, (int)L.max_elems, st); ++n_launch; break;

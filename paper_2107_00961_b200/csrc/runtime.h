@@ -66,6 +66,7 @@ struct Plan {
     ConvProb* d_conv = nullptr; BnProb* d_bn = nullptr; PoolProb* d_pool = nullptr; HeadProb* d_head = nullptr;
     PatchSite* d_sites = nullptr; int nsites = 0;
     void* d_tc = nullptr; size_t tc_stride = 0;              // tensor-core convolution descriptors
+    void* d_wtc = nullptr; size_t wtc_stride = 0;            // tensor-core wgrad descriptors
     Segment* d_sgd = nullptr; int n_sgd_seg = 0; long long sgd_chunks = 0; double sgd_params = 0;
     resist_step_info info{};
 };
