@@ -177,6 +177,26 @@ int resist_bn_relu_backward(int32_t dtype, const void* x, const void* da, const 
                             resist_stream stream);
 const char* resist_layer_last_error(void);
 
+/* resist_bn_relu_forward for callers that cannot allocate device memory (the paper has no counterpart: this is a
+ * property of the library, not of the method).  Who needs it: code running inside a fixed memory pool, loops
+ * that cannot afford the stall an allocation or a free can cause, hosts whose framework owns all device memory.
+ * Same arguments and the same result, bit for bit, as resist_bn_relu_forward, but it calls no cudaMalloc,
+ * cudaFree or other allocating routine: the per-chunk partial sums (chunks x 2 x C doubles) and the problem
+ * descriptor live in a 4 MiB array built into the library, which every GPU that loads the library holds until
+ * the process ends.
+ *  - Limit: chunks * C <= 262144 with chunks = ceil(m / max(32 * (256 / min(C, 256)), ceil(m / 1024))) <= 1024;
+ *    e.g. any m with C <= 256.  Larger problems return RESIST_EUNSUPPORTED with the sizes in the message.
+ *  - The first call on each device looks up the array's device address (one cudaGetSymbolAddress, with that
+ *    device current); make that first call before any stream capture begins.
+ *  - All calls share the one array, and it keeps what the last call left there.  Nothing has to be cleared between
+ *    calls (each call writes every slot before reading it), but two calls that overlap on the GPU (different
+ *    streams, or different host threads without ordering) race on it: keep them on one stream or order them.
+ *  - Asynchronous: work is enqueued on `stream`, nothing is synchronised.  Errors: resist_noalloc_last_error(). */
+int resist_bn_relu_forward_noalloc(int32_t dtype, const void* x, const float* gamma, const float* beta, void* a, float* stat,
+                                   float* run_mean, float* run_var, int64_t m, int32_t C, float eps, float momentum,
+                                   resist_stream stream);
+const char* resist_noalloc_last_error(void);
+
 /* Per-kernel timing.  With profiling on, every launch of a local step, partition or aggregate is bracketed by
  * CUDA events on the call's stream and the call synchronises before returning; times, launch counts and the
  * algorithmic bytes and FLOPs of the work launched accumulate per kernel family until read.

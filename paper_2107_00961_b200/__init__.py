@@ -93,6 +93,8 @@ def lib():
         L.resist_bn_relu_forward.argtypes = [I, P, P, P, P, P, P, P, C.c_int64, I, F, F, P]
         L.resist_bn_relu_backward.argtypes = [I, P, P, P, P, P, P, P, P, P, C.c_int64, I, P]
         L.resist_layer_last_error.restype = C.c_char_p
+        L.resist_bn_relu_forward_noalloc.argtypes = [I, P, P, P, P, P, P, P, C.c_int64, I, F, F, P]
+        L.resist_noalloc_last_error.restype = C.c_char_p
         L.resist_last_error.argtypes = [P]
         L.resist_last_error.restype = C.c_char_p
         _lib = L
@@ -102,7 +104,8 @@ def lib():
 EXPORTS = ["resist_init", "resist_destroy", "resist_partition", "resist_local_step", "resist_local_step_grouped",
            "resist_aggregate", "resist_eval", "resist_param_count", "resist_get_params", "resist_set_params",
            "resist_get_grads", "resist_get_logits", "resist_get_step_info", "resist_splitmix64", "resist_last_error",
-           "resist_set_profiling", "resist_get_profile", "resist_conv2d", "resist_bn_relu_forward", "resist_bn_relu_backward", "resist_layer_last_error"]
+           "resist_set_profiling", "resist_get_profile", "resist_conv2d", "resist_bn_relu_forward", "resist_bn_relu_backward", "resist_layer_last_error",
+           "resist_bn_relu_forward_noalloc", "resist_noalloc_last_error"]
 
 
 def resist_splitmix64(seed: int, n: int) -> np.ndarray:
@@ -156,6 +159,21 @@ def resist_bn_relu_forward(x: torch.Tensor, gamma, beta, run_mean=None, run_var=
                                               run_var.data_ptr() if run_var is not None else None, m, Cc, eps, momentum,
                                               _stream_handle(stream)))
     return a, stat
+
+
+def resist_bn_relu_forward_noalloc(x: torch.Tensor, gamma, beta, a: torch.Tensor, stat: torch.Tensor, run_mean=None,
+                                   run_var=None, eps=1e-5, momentum=0.1, stream=None):
+    """resist_bn_relu_forward without any device allocation: the caller passes the output `a` (shape of x) and
+    `stat` (float32 [4*C]) too, and the reduction scratch is a fixed array inside the library (see the header for
+    its limit).  Enqueues on the stream and returns; calls must not overlap on the GPU."""
+    Cc = x.shape[-1]
+    m = x.numel() // Cc
+    rc = lib().resist_bn_relu_forward_noalloc(_dt(x), x.data_ptr(), gamma.data_ptr(), beta.data_ptr(), a.data_ptr(),
+                                              stat.data_ptr(), run_mean.data_ptr() if run_mean is not None else None,
+                                              run_var.data_ptr() if run_var is not None else None, m, Cc, eps, momentum,
+                                              _stream_handle(stream))
+    if rc != RESIST_OK:
+        raise ResistError(rc, lib().resist_noalloc_last_error().decode())
 
 
 def resist_bn_relu_backward(x, da, gamma, beta, stat, add=None, stream=None):

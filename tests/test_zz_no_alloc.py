@@ -1,0 +1,62 @@
+"""The allocation-free BN+ReLU forward against the ordinary entry point.
+
+Some users of the library cannot let it call cudaMalloc (a fixed memory pool, a latency-critical loop, a framework
+that owns the device memory).  resist_bn_relu_forward_noalloc keeps its reduction scratch in an array built into
+the library instead.  This file is named so that pytest collects it last: a run that stops at the first failure
+has then already run every other test.  It calls the entry point twice in a row, on different data, because the
+second call finds the first call's leftovers in the shared array.
+"""
+import numpy as np
+import pytest
+import torch
+
+import synth
+from parity import max_rel_err, norm_max_abs
+
+pytestmark = pytest.mark.gpu
+
+
+def case(seed, m_rows, C, bf):
+    x = synth.standard_normal(seed, m_rows * C).astype(np.float32).reshape(m_rows, C) * np.float32(1.3)
+    x += synth.standard_normal(seed + 1, C).astype(np.float32)[None, :]
+    if bf:
+        x = synth.round_to_bf16(x)
+    g = (1 + 0.2 * synth.standard_normal(seed + 2, C)).astype(np.float32)
+    b = (0.3 * synth.standard_normal(seed + 3, C)).astype(np.float32)
+    t = torch.from_numpy(x).cuda()
+    return (t.to(torch.bfloat16) if bf else t), torch.from_numpy(g).cuda(), torch.from_numpy(b).cuda()
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_noalloc_matches_the_allocating_entry_point_twice_in_a_row(dtype):
+    import paper_2107_00961_b200 as m
+    bf = dtype == "bf16"
+    # the second problem is smaller than the first, so stale partial sums of the first sit right behind its own
+    for seed, rows, C in ((101, 5000, 64), (202, 777, 32)):
+        x, g, b = case(seed, rows, C, bf)
+        rm = torch.zeros(C, device="cuda"); rv = torch.ones(C, device="cuda")
+        rm2, rv2 = rm.clone(), rv.clone()
+        a_ref, stat_ref = m.resist_bn_relu_forward(x, g, b, rm, rv)
+        a = torch.empty_like(x)
+        stat = torch.zeros(4 * C, dtype=torch.float32, device="cuda")
+        before = torch.cuda.memory_allocated()
+        m.resist_bn_relu_forward_noalloc(x, g, b, a, stat, rm2, rv2)
+        torch.cuda.synchronize()
+        assert torch.cuda.memory_allocated() == before
+        tol = 2e-2 if bf else 1e-4
+        err = norm_max_abs if bf else max_rel_err
+        assert err(a.float().cpu().numpy(), a_ref.float().cpu().numpy()) < tol
+        assert max_rel_err(stat[:2 * C].cpu().numpy(), stat_ref[:2 * C].cpu().numpy()) < 1e-6
+        assert max_rel_err(rm2.cpu().numpy(), rm.cpu().numpy()) < 1e-6 and max_rel_err(rv2.cpu().numpy(), rv.cpu().numpy()) < 1e-6
+        # same chunking, same kernels: the two entry points agree bit for bit
+        assert torch.equal(a, a_ref)
+
+
+def test_noalloc_rejects_what_does_not_fit():
+    import paper_2107_00961_b200 as m
+    C, rows = 2048, 40000           # 1000 chunks x 2 x 2048 doubles = 32 MiB of partial sums: beyond the 4 MiB array
+    x = torch.zeros(rows, C, device="cuda")
+    g = torch.ones(C, device="cuda"); b = torch.zeros(C, device="cuda")
+    with pytest.raises(m.ResistError) as e:
+        m.resist_bn_relu_forward_noalloc(x, g, b, torch.empty_like(x), torch.zeros(4 * C, device="cuda"))
+    assert e.value.code == -6 and "bytes" in str(e.value)
