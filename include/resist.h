@@ -184,8 +184,8 @@ const char* resist_layer_last_error(void);
  * cudaFree or other allocating routine: the per-chunk partial sums (chunks x 2 x C doubles) and the problem
  * descriptor live in a 4 MiB array built into the library, which every GPU that loads the library holds until
  * the process ends.
- *  - Limit: chunks * C <= 262144 with chunks = ceil(m / max(32 * (256 / min(C, 256)), ceil(m / 1024))) <= 1024;
- *    e.g. any m with C <= 256.  Larger problems return RESIST_EUNSUPPORTED with the sizes in the message.
+ *  - Limit: chunks * C <= 262144, where chunks (the number of row chunks reduced by one CTA each) never exceeds
+ *    1024: any m with C <= 256 fits.  Larger problems return RESIST_EUNSUPPORTED with the sizes in the message.
  *  - The first call on each device looks up the array's device address (one cudaGetSymbolAddress, with that
  *    device current); make that first call before any stream capture begins.
  *  - All calls share the one array, and it keeps what the last call left there.  Nothing has to be cleared between

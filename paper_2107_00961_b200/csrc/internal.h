@@ -42,8 +42,23 @@ struct BnProb {
     int C, chunks, rows_per_chunk;
     float eps, momentum;
     int eval;             // 1: use running statistics (no batch statistics)
-    int pad_;
+    int vec;              // 1: bf16 fast path (16-byte accesses, 8 channels per thread)
 };
+
+// How the rows of a BN problem are cut into chunks (one CTA each) and whether the vector path applies.
+inline void bn_chunking(BnProb& p, bool bf16) {
+    const int C = p.C; const long long m = p.m;
+    const int G = C / 8;
+    const bool pow2 = G > 0 && (G & (G - 1)) == 0;
+    const bool aligned = ((((uintptr_t)p.x) | ((uintptr_t)p.a) | ((uintptr_t)p.da) | ((uintptr_t)p.dx) | ((uintptr_t)p.add) |
+                            ((uintptr_t)p.gamma) | ((uintptr_t)p.beta) | ((uintptr_t)p.stat)) & 15) == 0;
+    p.vec = (bf16 && C % 8 == 0 && pow2 && G <= 256 && aligned) ? 1 : 0;
+    long long rpc;
+    if (p.vec) { const int R = 256 / G; rpc = (long long)R * 16; }
+    else { const int nl = C < 256 ? C : 256, R = 256 / nl; rpc = (long long)R * 32; }
+    const long long lim = (m + 1023) / 1024; if (rpc < lim) rpc = lim;
+    p.rows_per_chunk = (int)rpc; p.chunks = (int)((m + rpc - 1) / rpc);
+}
 
 struct PoolProb {         // 3x3 stride-2 max-pool, pad 1: x [N,H,W,C] -> y [N,P,Q,C]
     const void* x; void* y; int* arg; const void* dy; void* dx;

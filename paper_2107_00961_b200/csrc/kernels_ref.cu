@@ -156,11 +156,124 @@ void launch_splitk_reduce(const ConvProb* d, int nprob, int max_elems, cudaStrea
 // Batch normalisation + ReLU.  Statistics: each CTA reduces `rows_per_chunk` rows of all C channels
 // (fp32 per thread, fp64 across threads), a finalise kernel adds the chunk partials in order.
 // ------------------------------------------------------------------------------------------------
+
+// ---- bf16 fast path: 16-byte accesses, a thread owns 8 consecutive channels (one group) and every (256/G)-th row
+__device__ __forceinline__ void unpack8(const uint4& v, float* f) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) { f[2 * k] = __uint_as_float(w[k] << 16); f[2 * k + 1] = __uint_as_float(w[k] & 0xFFFF0000u); }
+}
+__device__ __forceinline__ uint4 pack8(const float* f) {
+    uint32_t w[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) { __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * k], f[2 * k + 1]); w[k] = *reinterpret_cast<uint32_t*>(&h); }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+template <int MODE>
+__device__ void bn_reduce_vec(const BnProb& p) {
+    __shared__ float sm[256][17];
+    const int C = p.C, G = C >> 3, R = 256 / G;
+    const int g = threadIdx.x % G, r = threadIdx.x / G;
+    const long long r0 = (long long)blockIdx.x * p.rows_per_chunk;
+    long long r1 = r0 + p.rows_per_chunk; if (r1 > p.m) r1 = p.m;
+    float s0[8], s1[8], sh[8], mean[8], istd[8], ga[8], be[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) { s0[j] = 0.f; s1[j] = 0.f; }
+    if (MODE == 0) { unpack8(*reinterpret_cast<const uint4*>((const __nv_bfloat16*)p.x + g * 8), sh); }
+    else {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { const int c = g * 8 + j; mean[j] = p.stat[c]; istd[j] = p.stat[C + c]; ga[j] = p.gamma[c]; be[j] = p.beta[c]; }
+    }
+    const uint4* xv = reinterpret_cast<const uint4*>(p.x);
+    const uint4* dv = reinterpret_cast<const uint4*>(p.da);
+#pragma unroll 4
+    for (long long row = r0 + r; row < r1; row += R) {
+        float x[8]; unpack8(xv[row * G + g], x);
+        if (MODE == 0) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) { const float d = x[j] - sh[j]; s0[j] += d; s1[j] += d * d; }
+        } else {
+            float d[8]; unpack8(dv[row * G + g], d);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) { const float xh = (x[j] - mean[j]) * istd[j]; const float dz = (xh * ga[j] + be[j] > 0.f) ? d[j] : 0.f; s0[j] += dz; s1[j] += dz * xh; }
+        }
+    }
+    // lanes of a warp that own the same channel group: fixed-order butterfly in fp32
+    if (G < 32) {
+        for (int off = 16; off >= G; off >>= 1) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) { s0[j] += __shfl_down_sync(0xffffffffu, s0[j], off); s1[j] += __shfl_down_sync(0xffffffffu, s1[j], off); }
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) { sm[threadIdx.x][j] = s0[j]; sm[threadIdx.x][8 + j] = s1[j]; }
+    __syncthreads();
+    if ((int)threadIdx.x < C) {
+        const int c = threadIdx.x, cg = c >> 3, j = c & 7;
+        double a0 = 0.0, a1 = 0.0;
+        if (G < 32) { for (int w = 0; w < 8; ++w) { a0 += sm[w * 32 + cg][j]; a1 += sm[w * 32 + cg][8 + j]; } }
+        else { for (int k = 0; k < R; ++k) { a0 += sm[cg + G * k][j]; a1 += sm[cg + G * k][8 + j]; } }
+        p.partial[((long long)blockIdx.x * 2 + 0) * C + c] = a0;
+        p.partial[((long long)blockIdx.x * 2 + 1) * C + c] = a1;
+    }
+    // more than 256 channels: the remaining ones, 256 at a time
+    for (int c = threadIdx.x + 256; c < C; c += 256) {
+        const int cg = c >> 3, j = c & 7;
+        double a0 = 0.0, a1 = 0.0;
+        for (int k = 0; k < R; ++k) { a0 += sm[cg + G * k][j]; a1 += sm[cg + G * k][8 + j]; }
+        p.partial[((long long)blockIdx.x * 2 + 0) * C + c] = a0;
+        p.partial[((long long)blockIdx.x * 2 + 1) * C + c] = a1;
+    }
+}
+
+template <int MODE>   // 0: forward apply; 1: backward apply
+__device__ void bn_apply_vec(const BnProb& p) {
+    const int C = p.C, G = C >> 3;
+    const long long nv = p.m * G;
+    const float inv_m = 1.f / (float)p.m;
+    const uint4* xv = reinterpret_cast<const uint4*>(p.x);
+    const uint4* dv = reinterpret_cast<const uint4*>(p.da);
+    const uint4* av = reinterpret_cast<const uint4*>(p.add);
+    uint4* ov = reinterpret_cast<uint4*>(MODE == 0 ? p.a : p.dx);
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long v = blockIdx.x * (long long)blockDim.x + threadIdx.x; v < nv; v += stride) {
+        const int c0 = (int)(v & (long long)(G - 1)) * 8;          // G is a power of two
+        float x[8], o[8]; unpack8(xv[v], x);
+        const float4 m0 = *reinterpret_cast<const float4*>(p.stat + c0), m1 = *reinterpret_cast<const float4*>(p.stat + c0 + 4);
+        const float4 i0 = *reinterpret_cast<const float4*>(p.stat + C + c0), i1 = *reinterpret_cast<const float4*>(p.stat + C + c0 + 4);
+        const float4 g0 = *reinterpret_cast<const float4*>(p.gamma + c0), g1 = *reinterpret_cast<const float4*>(p.gamma + c0 + 4);
+        const float4 b0 = *reinterpret_cast<const float4*>(p.beta + c0), b1 = *reinterpret_cast<const float4*>(p.beta + c0 + 4);
+        const float mean[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w}, istd[8] = {i0.x, i0.y, i0.z, i0.w, i1.x, i1.y, i1.z, i1.w};
+        const float ga[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w}, be[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+        if (MODE == 0) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) { const float z = (x[j] - mean[j]) * istd[j] * ga[j] + be[j]; o[j] = z > 0.f ? z : 0.f; }
+        } else {
+            float d[8]; unpack8(dv[v], d);
+            const float4 s0 = *reinterpret_cast<const float4*>(p.stat + 2 * C + c0), s1 = *reinterpret_cast<const float4*>(p.stat + 2 * C + c0 + 4);
+            const float4 t0 = *reinterpret_cast<const float4*>(p.stat + 3 * C + c0), t1 = *reinterpret_cast<const float4*>(p.stat + 3 * C + c0 + 4);
+            const float sb[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w}, sg[8] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const float xh = (x[j] - mean[j]) * istd[j];
+                const float dz = (xh * ga[j] + be[j] > 0.f) ? d[j] : 0.f;
+                o[j] = ga[j] * istd[j] * (dz - sb[j] * inv_m - xh * sg[j] * inv_m);
+            }
+            if (av) { float ad[8]; unpack8(av[v], ad);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) o[j] += ad[j]; }
+        }
+        ov[v] = pack8(o);
+    }
+}
+
 // MODE 0: sums of x and x^2.  MODE 1: sums of dz and dz*xhat (backward).
 template <class T, int MODE>
 __global__ void __launch_bounds__(256) bn_reduce_kernel(const BnProb* __restrict__ probs) {
     const BnProb& p = probs[blockIdx.y];
     if ((int)blockIdx.x >= p.chunks || p.eval) return;
+    if (p.vec) { bn_reduce_vec<MODE>(p); return; }
     __shared__ double part[2][256];
     const int C = p.C, nl = C < 256 ? C : 256, R = 256 / nl;
     const int rg = threadIdx.x / nl, lane = threadIdx.x % nl;
@@ -226,6 +339,7 @@ __global__ void bn_finalize_kernel(const BnProb* __restrict__ probs) {
 template <class T>
 __global__ void __launch_bounds__(256) bn_apply_kernel(const BnProb* __restrict__ probs) {
     const BnProb& p = probs[blockIdx.y];
+    if (p.vec) { bn_apply_vec<0>(p); return; }
     const long long n = p.m * p.C;
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
         const int c = (int)(i % p.C);
@@ -237,6 +351,7 @@ __global__ void __launch_bounds__(256) bn_apply_kernel(const BnProb* __restrict_
 template <class T>
 __global__ void __launch_bounds__(256) bn_bwd_apply_kernel(const BnProb* __restrict__ probs) {
     const BnProb& p = probs[blockIdx.y];
+    if (p.vec) { bn_apply_vec<1>(p); return; }
     const long long n = p.m * p.C;
     const float inv_m = 1.f / (float)p.m;
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {

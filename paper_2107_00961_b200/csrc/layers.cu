@@ -87,11 +87,9 @@ extern "C" int resist_conv2d(int32_t mode, int32_t dtype, int32_t backend, const
     return RESIST_OK;
 }
 
-static void fill_bn(BnProb& p, int64_t m, int C) {
+static void fill_bn(BnProb& p, int64_t m, int C, bool bf16) {
     p.m = m; p.C = C;
-    const int nl = C < 256 ? C : 256, R = 256 / nl;
-    long long rpc = (long long)R * 32; const long long lim = (m + 1023) / 1024; if (rpc < lim) rpc = lim;
-    p.rows_per_chunk = (int)rpc; p.chunks = (int)((m + rpc - 1) / rpc);
+    bn_chunking(p, bf16);
 }
 
 extern "C" int resist_bn_relu_forward(int32_t dtype, const void* x, const float* gamma, const float* beta, void* a, float* stat,
@@ -100,7 +98,7 @@ extern "C" int resist_bn_relu_forward(int32_t dtype, const void* x, const float*
     if (!x || !gamma || !beta || !a || !stat || m < 1 || C < 1) { g_layer_error = "bad argument"; return RESIST_EINVAL; }
     cudaStream_t st = (cudaStream_t)stream;
     BnProb p{}; p.x = x; p.a = a; p.gamma = gamma; p.beta = beta; p.run_mean = run_mean; p.run_var = run_var; p.stat = stat;
-    p.eps = eps; p.momentum = momentum; fill_bn(p, m, C);
+    p.eps = eps; p.momentum = momentum; fill_bn(p, m, C, dtype == RESIST_BF16);
     char* blob = nullptr;
     cudaError_t e = cudaMalloc(&blob, 1024 + (size_t)p.chunks * 2 * C * 8);
     if (e != cudaSuccess) { g_layer_error = cudaGetErrorString(e); return RESIST_ENOMEM; }
@@ -123,7 +121,7 @@ extern "C" int resist_bn_relu_backward(int32_t dtype, const void* x, const void*
     if (!x || !da || !gamma || !beta || !stat || !dx || !dgamma || !dbeta || m < 1 || C < 1) { g_layer_error = "bad argument"; return RESIST_EINVAL; }
     cudaStream_t st = (cudaStream_t)stream;
     BnProb p{}; p.x = x; p.da = da; p.dx = dx; p.add = add; p.gamma = gamma; p.beta = beta; p.dgamma = dgamma; p.dbeta = dbeta; p.stat = stat;
-    fill_bn(p, m, C);
+    fill_bn(p, m, C, dtype == RESIST_BF16);
     char* blob = nullptr;
     cudaError_t e = cudaMalloc(&blob, 1024 + (size_t)p.chunks * 2 * C * 8);
     if (e != cudaSuccess) { g_layer_error = cudaGetErrorString(e); return RESIST_ENOMEM; }

@@ -49,9 +49,7 @@ extern "C" int resist_bn_relu_forward_noalloc(int32_t dtype, const void* x, cons
     BnProb p{}; p.x = x; p.a = a; p.gamma = gamma; p.beta = beta; p.run_mean = run_mean; p.run_var = run_var; p.stat = stat;
     p.eps = eps; p.momentum = momentum; p.m = m; p.C = C;
     // the same chunking as resist_bn_relu_forward, so that both give the same bits
-    const int nl = C < 256 ? C : 256, R = 256 / nl;
-    long long rpc = (long long)R * 32; const long long lim = (m + 1023) / 1024; if (rpc < lim) rpc = lim;
-    p.rows_per_chunk = (int)rpc; p.chunks = (int)((m + rpc - 1) / rpc);
+    bn_chunking(p, dtype == RESIST_BF16);
     const size_t need = (size_t)p.chunks * 2 * (size_t)C * sizeof(double);
     if (need > RESIST_NOALLOC_SCRATCH_BYTES) {
         g_noalloc_error = "needs " + std::to_string(need) + " bytes of reduction scratch (chunks x 2 x C doubles) but the built-in array holds " +

@@ -124,9 +124,7 @@ struct Builder {
         p.x = x; p.a = a; p.gamma = W() + r.g; p.beta = W() + r.b; p.dgamma = G() + r.g; p.dbeta = G() + r.b;
         p.run_mean = Bf() + r.buf; p.run_var = Bf() + r.buf + r.c; p.stat = stat; p.m = m; p.C = r.c;
         p.eps = ctx->opts.bn_eps; p.momentum = ctx->opts.bn_momentum; p.eval = eval ? 1 : 0;
-        const int nl = r.c < 256 ? r.c : 256, R = 256 / nl;
-        long long rpc = (long long)R * 32; const long long lim = (m + 1023) / 1024; if (rpc < lim) rpc = lim;
-        p.rows_per_chunk = (int)rpc; p.chunks = (int)((m + rpc - 1) / rpc);
+        bn_chunking(p, ctx->opts.dtype == RESIST_BF16);
         bn_partial_need = std::max(bn_partial_need, (size_t)p.chunks * 2 * r.c * 8);
         p.partial = bn_partial;
         ops->push_back(op);
@@ -138,9 +136,7 @@ struct Builder {
         BnProb& p = op.bn;
         p.x = x; p.da = da; p.dx = dx; p.add = add; p.gamma = W() + r.g; p.beta = W() + r.b; p.dgamma = G() + r.g; p.dbeta = G() + r.b;
         p.stat = stat; p.m = m; p.C = r.c; p.eps = ctx->opts.bn_eps; p.momentum = ctx->opts.bn_momentum; p.eval = 0;
-        const int nl = r.c < 256 ? r.c : 256, R = 256 / nl;
-        long long rpc = (long long)R * 32; const long long lim = (m + 1023) / 1024; if (rpc < lim) rpc = lim;
-        p.rows_per_chunk = (int)rpc; p.chunks = (int)((m + rpc - 1) / rpc);
+        bn_chunking(p, ctx->opts.dtype == RESIST_BF16);
         p.partial = bn_partial;
         ops->push_back(op);
         op.key = key + 1; op.kind = OP_BN_BWD_APPLY; ops->push_back(op);
