@@ -83,6 +83,7 @@ struct alignas(64) TcProb {
     int b_mn_major;                         // 0: forward (weights K-major); 1: dgrad (weights MN-major)
     int tmem_cols; int flat;                // flat = 1: 1x1 layer, tile = 128 consecutive pixels of the whole tensor
     int stages;                             // pipeline depth: 1 when the reduction fits one stage, else 2
+    int os, P, Q;                           // output stride: only positions (i,j) with i,j multiples of os are stored, as pixel (i/os, j/os) of a P x Q image
     float scale;
 };
 
@@ -180,7 +181,10 @@ __global__ void __launch_bounds__(TC_THREADS) conv_tc_kernel(const TcProb* __res
         if (p.flat) { const long long g = (long long)pos0 + m; if (g < (long long)p.W) pix = g; }
         else {
             const int pos = pos0 + m, i = pos / p.Wp, j = pos - i * p.Wp;
-            if (i < p.H && j < p.W) pix = ((long long)img * p.H + i) * p.W + j;
+            if (i < p.H && j < p.W) {
+                if (p.os == 1) pix = ((long long)img * p.H + i) * p.W + j;
+                else if (i % p.os == 0 && j % p.os == 0) pix = ((long long)img * p.P + i / p.os) * p.Q + j / p.os;   // strided layer
+            }
         }
         if (ok) {
             for (int c0 = 0; c0 < p.n_tile; c0 += 16) {
@@ -219,6 +223,28 @@ __global__ void __launch_bounds__(TC_THREADS) conv_tc_kernel(const TcProb* __res
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(p.tmem_cols) : "memory");
     }
+}
+
+// ------------------------------------------------------------------------------------------------ zero stuffing
+// Backward of a stride-2 layer runs as a stride-1 problem on dy spread out to the input resolution:
+// up[n, 2p, 2q, :] = dy[n, p, q, :], zero elsewhere.  Then dgrad(up) and wgrad(a, up) at stride 1 are the
+// stride-2 dgrad and wgrad, term for term.
+__global__ void __launch_bounds__(256) zero_stuff_kernel(const UpProb* __restrict__ probs) {
+    const UpProb& p = probs[blockIdx.y];
+    const int G = p.K >> 3;
+    const long long nv = (long long)p.N * p.H * p.W * G;
+    const uint4* src = reinterpret_cast<const uint4*>(p.src);
+    uint4* dst = reinterpret_cast<uint4*>(p.dst);
+    for (long long v = blockIdx.x * (long long)blockDim.x + threadIdx.x; v < nv; v += (long long)gridDim.x * blockDim.x) {
+        const int g = (int)(v % G); long long t = v / G; const int w = (int)(t % p.W); t /= p.W; const int h = (int)(t % p.H); const int n = (int)(t / p.H);
+        uint4 val = make_uint4(0u, 0u, 0u, 0u);
+        if (!(h & 1) && !(w & 1) && (h >> 1) < p.P && (w >> 1) < p.Q) val = src[(((long long)n * p.P + (h >> 1)) * p.Q + (w >> 1)) * G + g];
+        dst[v] = val;
+    }
+}
+void launch_zero_stuff(const UpProb* d, int nprob, long long max_vecs, cudaStream_t s) {
+    long long gx = (max_vecs + 255) / 256; if (gx > 148 * 16) gx = 148 * 16; if (gx < 1) gx = 1;
+    zero_stuff_kernel<<<dim3((unsigned)gx, nprob), 256, 0, s>>>(d);
 }
 
 // ------------------------------------------------------------------------------------------------ wgrad
@@ -394,18 +420,20 @@ struct TcGeom { int stages, chan_a, ncol, n_tile, kc, nchunks, Wp, box_w, box_h,
 // Decides whether (and how) the tensor-core kernel takes this problem.
 static bool tc_geometry(const ConvProb& p, int mode, TcGeom& g) {
     if (mode == CONV_WGRAD) return false;
-    if (p.stride != 1 || (p.ksz != 1 && p.ksz != 3)) return false;
+    // A stride-2 forward layer is computed at stride 1 and only the even positions are stored; stride-2 dgrad
+    // arrives here as a stride-1 problem on a zero-stuffed dy (see zero_stuff_kernel).
+    if ((p.ksz != 1 && p.ksz != 3) || p.stride < 1 || p.stride > 2 || (p.stride == 2 && mode != CONV_FWD)) return false;
     if (p.C % 16 || p.K % 16) return false;
     if (((uintptr_t)p.act | (uintptr_t)p.wgt | (uintptr_t)p.out | (uintptr_t)p.add) & 15) return false;
     g.chan_a = mode == CONV_FWD ? p.C : p.K;            // reduction channels
     g.ncol = mode == CONV_FWD ? p.K : p.C;              // output channels
-    g.flat = p.ksz == 1;
-    const int taps = p.ksz * p.ksz;
+    g.flat = p.ksz == 1 && p.stride == 1;
+    const int taps = p.ksz * p.ksz, pad2 = p.ksz - 1;
     if (g.flat) { g.n_img = 1; g.H = 1; g.W = p.N * p.H * p.W; g.Wp = g.W; g.box_w = 128; g.box_h = 1;
         g.tiles_per_img = (int)(((long long)g.W + 127) / 128); }
-    else { g.n_img = p.N; g.H = p.H; g.W = p.W; g.Wp = p.W + 2; if (g.Wp > 128) return false;
+    else { g.n_img = p.N; g.H = p.H; g.W = p.W; g.Wp = p.W + pad2; if (g.Wp > 128) return false;
         const int rows = (g.Wp - 1 + 127) / g.Wp + 1;   // rows 128 consecutive positions can touch
-        g.box_w = g.Wp; g.box_h = std::min(rows, p.H) + 2; if (g.box_h > 256) return false;
+        g.box_w = g.Wp; g.box_h = std::min(rows, p.H) + pad2; if (g.box_h > 256) return false;
         g.tiles_per_img = (p.H * g.Wp + 127) / 128; }
     g.n_tile = g.ncol; while (g.n_tile > 128) { if (g.n_tile % 2) return false; g.n_tile /= 2; }
     if (g.n_tile % 16) return false;
@@ -462,6 +490,7 @@ bool conv_tc_fill(const ConvProb& p, int mode, void* host_tc) {
     t.kc = g.kc; t.nchunks = g.nchunks; t.box_w = g.box_w; t.box_h = g.box_h; t.plane_bytes = g.plane_bytes;
     t.a_stage_bytes = g.a_stage; t.b_stage_bytes = g.b_stage; t.b_tap_bytes = g.b_tap; t.b_mn_major = mode == CONV_DGRAD ? 1 : 0;
     t.tmem_cols = g.tmem_cols; t.flat = g.flat; t.scale = p.scale; t.stages = g.stages;
+    t.os = (mode == CONV_FWD) ? p.stride : 1; t.P = p.P; t.Q = p.Q;
     memcpy(host_tc, &t, sizeof(t));
     return true;
 }
@@ -490,10 +519,10 @@ static bool wg_geometry(const ConvProb& p, int target_ctas, WgGeom& g) {
     if (p.K > 128 && p.K % 128) return false;
     if (((uintptr_t)p.act | (uintptr_t)p.wgt) & 15) return false;
     const int taps = p.ksz * p.ksz;
-    g.flat = p.ksz == 1;
+    g.flat = p.ksz == 1;                 // (a stride-2 1x1 layer arrives with stride 1 and a zero-stuffed dy: still flat)
     int rows = 1;
     if (g.flat) { g.n_img = 1; g.H = 1; g.W = p.N * p.H * p.W; g.Wp = g.W; g.box_w = 128; g.tiles_per_img = (int)(((long long)g.W + 127) / 128); }
-    else { g.n_img = p.N; g.H = p.H; g.W = p.W; g.Wp = p.W + 2; if (g.Wp > 128) return false;
+    else { g.n_img = p.N; g.H = p.H; g.W = p.W; g.Wp = p.W + (p.ksz - 1); if (g.Wp > 128) return false;
         // every one of the 128 positions of a stage enters the reduction, so all of them must hold data or the
         // zero fill of the TMA box, never stale shared memory: the boxes cover every row 128 positions can touch
         // (rows past the image come back as zeros), and the activation box has one row to spare for the two

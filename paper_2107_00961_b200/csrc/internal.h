@@ -60,6 +60,10 @@ inline void bn_chunking(BnProb& p, bool bf16) {
     p.rows_per_chunk = (int)rpc; p.chunks = (int)((m + rpc - 1) / rpc);
 }
 
+struct UpProb {           // zero stuffing of a stride-2 layer's dy: src [N,P,Q,K] -> dst [N,H,W,K] (bf16, K % 8 == 0)
+    const void* src; void* dst; int N, H, W, K, P, Q;
+};
+
 struct PoolProb {         // 3x3 stride-2 max-pool, pad 1: x [N,H,W,C] -> y [N,P,Q,C]
     const void* x; void* y; int* arg; const void* dy; void* dx;
     int N, H, W, C, P, Q;
@@ -110,6 +114,8 @@ void launch_maxpool_bwd(const PoolProb* d, int nprob, long long max_elems, bool 
 void launch_head_fwd(const HeadProb* d, int nprob, int maxB, int maxC, int max_classes, bool bf16, cudaStream_t s);
 void launch_head_bwd(const HeadProb* d, int nprob, int maxB, int maxC, int max_classes, long long max_elems,
                      bool bf16, cudaStream_t s);
+
+void launch_zero_stuff(const UpProb* d, int nprob, long long max_vecs, cudaStream_t s);   // conv_tc.cu
 
 // ---- launchers (kernels_bw.cu)
 void launch_sgd(const Segment* d, int nseg, long long nchunks, ParamArrays pa, float lr, float mu, float wd,

@@ -46,6 +46,21 @@ extern "C" int resist_conv2d(int32_t mode, int32_t dtype, int32_t backend, const
     p.tiles_m = (p.M + 63) / 64; p.tiles_n = (p.Ncol + 63) / 64; p.splits = 1;
     const int ktiles = (p.Kred + 15) / 16; p.ktiles_per_split = ktiles;
     int sm = 148; int dev = 0; cudaGetDevice(&dev); cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev);
+    // backward of a stride-2 layer on tensor cores: stride-1 problem on a zero-stuffed dy
+    char* up = nullptr;
+    if (dtype == RESIST_BF16 && backend == RESIST_CONV_AUTO && stride == 2 && mode != CONV_FWD && K % 8 == 0) {
+        ConvProb q = p; q.stride = 1; q.P = H; q.Q = W;
+        if (mode == CONV_DGRAD) q.M = (int)rows_in; else q.Kred = (int)rows_in;
+        size_t pb = 0;
+        if (mode == CONV_DGRAD ? conv_tc_supported(q, mode) : conv_wgrad_tc_supported(q, 2 * sm, &pb)) {
+            if (cudaMalloc(&up, (size_t)N * H * W * K * 2 + 256) != cudaSuccess) { g_layer_error = "cudaMalloc failed"; return RESIST_ENOMEM; }
+            UpProb u{mode == CONV_DGRAD ? p.act : p.wgt, up + 256, N, H, W, K, p.P, p.Q};
+            cudaMemcpyAsync(up, &u, sizeof(u), cudaMemcpyHostToDevice, st);
+            launch_zero_stuff((const UpProb*)up, 1, (long long)N * H * W * (K / 8), st);
+            if (mode == CONV_DGRAD) q.act = up + 256; else q.wgt = up + 256;
+            p = q;
+        }
+    }
     size_t wg_partial = 0;
     const bool tc = dtype == RESIST_BF16 && backend == RESIST_CONV_AUTO &&
                     (mode == CONV_WGRAD ? conv_wgrad_tc_supported(p, 2 * sm, &wg_partial) : conv_tc_supported(p, mode));
@@ -80,7 +95,7 @@ extern "C" int resist_conv2d(int32_t mode, int32_t dtype, int32_t backend, const
         e = cudaGetLastError();
     }
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
-    cudaFree(blob);
+    cudaFree(blob); cudaFree(up);
     if (e != cudaSuccess) { g_layer_error = cudaGetErrorString(e); return RESIST_ECUDA; }
     if (tc) { const int stv = conv_tc_read_status();
         if (stv) { g_layer_error = "a bounded device-side wait gave up (code " + std::to_string(stv) + ")"; return RESIST_ETIMEOUT; } }

@@ -64,6 +64,7 @@ struct Builder {
     std::vector<Op>* ops;
     // scratch shared by the operations of this sub-ResNet (they run one after another)
     double* bn_partial = nullptr; float* wgrad_partial = nullptr; size_t bn_partial_need = 0, wgrad_partial_need = 0;
+    char* up_buf = nullptr; size_t up_need = 0; const void* up_src = nullptr;      // zero-stuffed dy of the current stride-2 layer
     char* gbuf[6] = {}; bool gused[6] = {}; size_t gbig = 0;
     float* logits = nullptr;
     long long flops = 0; int n_tc = 0, n_cc = 0;
@@ -97,6 +98,25 @@ struct Builder {
         const int ktiles = (p.Kred + 15) / 16; p.ktiles_per_split = ktiles;
         flops += 2LL * rows_out * p.K * p.ksz * p.ksz * p.C;
         const bool tc_ok = ctx->opts.dtype == RESIST_BF16 && ctx->opts.conv_backend == RESIST_CONV_AUTO;
+        if (tc_ok && p.stride == 2 && mode != CONV_FWD && !patch && p.K % 8 == 0) {
+            // backward of a stride-2 layer: a stride-1 problem on dy zero-stuffed to the input resolution
+            ConvProb q = p; q.stride = 1; q.P = p.H; q.Q = p.W;
+            const size_t up_bytes = (size_t)N * p.H * p.W * p.K * 2;
+            if (mode == CONV_DGRAD) { q.act = up_buf; q.M = (int)rows_in; }
+            else { q.wgt = up_buf; q.Kred = (int)rows_in; }
+            size_t pb = 0;
+            const bool ok = mode == CONV_DGRAD ? conv_tc_supported(q, mode) : conv_wgrad_tc_supported(q, wgrad_target_ctas(ctx), &pb);
+            if (ok) {
+                up_need = std::max(up_need, up_bytes);
+                if (up_src != dy_or_null) {                  // first use of this dy: stuff it
+                    Op u{}; u.key = key; u.sub = sub; u.kind = OP_UPSAMPLE;
+                    u.up = UpProb{dy_or_null, up_buf, N, p.H, p.W, p.K, p.P, p.Q};
+                    ops->push_back(u); up_src = dy_or_null;
+                }
+                p = q;
+                if (mode == CONV_WGRAD) { wgrad_partial_need = std::max(wgrad_partial_need, pb); }
+            }
+        }
         if (mode == CONV_WGRAD) {
             size_t pb = 0;
             op.backend = (tc_ok && !patch && conv_wgrad_tc_supported(p, wgrad_target_ctas(ctx), &pb)) ? 1 : 0;
@@ -153,6 +173,7 @@ static size_t unroll_subnet(resist_ctx* ctx, Builder& bd, const std::vector<char
     // scratch first, so that its addresses do not depend on the network above it
     bd.bn_partial = (double*)bd.take(bd.bn_partial_need);
     bd.wgrad_partial = (float*)bd.take(bd.wgrad_partial_need);
+    bd.up_buf = (char*)bd.take(bd.up_need);
     if (!bd.eval) for (int i = 0; i < 6; ++i) bd.gbuf[i] = (char*)bd.take(bd.gbig);
 
     // ---- stem
@@ -224,6 +245,7 @@ static size_t unroll_subnet(resist_ctx* ctx, Builder& bd, const std::vector<char
         const long long key = BWD_BLOCK0 + 40LL * ((long long)order.size() - 1 - slot);
         const long long m_in = (long long)B * s.H * s.W, m_out = (long long)B * s.Ho * s.Wo;
         const char* dout = bd.gbuf[g_cur];
+        bd.up_src = nullptr;                                     // no zero-stuffed dy carries over from another block
         int g_sc = -1;
         if (K.has_projection) {
             bd.conv(key + 0, CONV_WGRAD, s.a1, r.proj, dout, nullptr, nullptr, B, s.H, s.W, 1.f);
@@ -283,16 +305,16 @@ static size_t unroll_subnet(resist_ctx* ctx, Builder& bd, const std::vector<char
 // ------------------------------------------------------------------------------------------------
 // Workspace: one slice per sub-ResNet, all slices the size of the largest.
 // ------------------------------------------------------------------------------------------------
-struct Needs { size_t bn_partial = 0, wgrad_partial = 0, gbig = 0, total = 0; };
+struct Needs { size_t bn_partial = 0, wgrad_partial = 0, gbig = 0, up = 0, total = 0; };
 
 static Needs measure_subnet(resist_ctx* ctx, int sub, int copy, const std::vector<char>& present, int B, bool eval, float inv_S) {
     std::vector<Op> scratch;
     Builder b1{ctx, B, sub, copy, eval, 0, nullptr}; b1.es = ctx->opts.dtype == RESIST_BF16 ? 2 : 4; b1.ops = &scratch;
     unroll_subnet(ctx, b1, present, inv_S);
-    Needs n; n.bn_partial = b1.bn_partial_need; n.wgrad_partial = b1.wgrad_partial_need; n.gbig = b1.gbig;
+    Needs n; n.bn_partial = b1.bn_partial_need; n.wgrad_partial = b1.wgrad_partial_need; n.gbig = b1.gbig; n.up = b1.up_need;
     scratch.clear();
     Builder b2{ctx, B, sub, copy, eval, 0, nullptr}; b2.es = b1.es; b2.ops = &scratch;
-    b2.bn_partial_need = n.bn_partial; b2.wgrad_partial_need = n.wgrad_partial; b2.gbig = n.gbig;
+    b2.bn_partial_need = n.bn_partial; b2.wgrad_partial_need = n.wgrad_partial; b2.gbig = n.gbig; b2.up_need = n.up;
     n.total = align_up(unroll_subnet(ctx, b2, present, inv_S), 256);
     return n;
 }
@@ -304,9 +326,13 @@ static std::vector<char> present_of(const resist_ctx* ctx, int sub) {
 }
 
 static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool single, cudaStream_t st) {
-    std::stable_sort(ops.begin(), ops.end(), [](const Op& a, const Op& b) { return a.key < b.key; });
+    // equal keys of different sub-ResNets become neighbours; a zero-stuffing op shares the key of the first
+    // convolution that reads its output and sorts in front of it
+    std::stable_sort(ops.begin(), ops.end(), [](const Op& a, const Op& b) {
+        if (a.key != b.key) return a.key < b.key;
+        return (a.kind == OP_UPSAMPLE) > (b.kind == OP_UPSAMPLE); });
     const double es = ctx->opts.dtype == RESIST_BF16 ? 2.0 : 4.0;
-    std::vector<ConvProb> conv; std::vector<BnProb> bn; std::vector<PoolProb> pool; std::vector<HeadProb> head;
+    std::vector<ConvProb> conv; std::vector<BnProb> bn; std::vector<PoolProb> pool; std::vector<HeadProb> head; std::vector<UpProb> up;
     const size_t tcb = conv_tc_prob_bytes(); std::vector<char> tc; int n_tc = 0;
     const size_t wtcb = conv_wgrad_tc_prob_bytes(); std::vector<char> wtc; int n_wtc = 0;
     struct HostSite { int arr; int idx; int field; int what; int sub; };
@@ -372,6 +398,13 @@ static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool s
                       else if (o.kind == OP_BN_BWD_REDUCE) L.bytes += 2 * es * e;
                       else L.bytes += es * e * (o.bn.add ? 4 : 3); }
                     break; }
+                case OP_UPSAMPLE: {
+                    if (k == i) L.first = (int)up.size();
+                    up.push_back(o.up);
+                    const double e = (double)o.up.N * o.up.K * 2.0;
+                    L.max_elems = std::max<long long>(L.max_elems, (long long)o.up.N * o.up.H * o.up.W * (o.up.K / 8));
+                    L.bytes += e * ((double)o.up.P * o.up.Q + (double)o.up.H * o.up.W);
+                    break; }
                 case OP_POOL_FWD: case OP_POOL_BWD: {
                     if (k == i) L.first = (int)pool.size();
                     pool.push_back(o.pool);
@@ -408,6 +441,7 @@ static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool s
     const size_t o_seg = off;  off += align_up(segs.size() * sizeof(Segment), 256);
     const size_t o_tc = off;   off += align_up(tc.size(), 256);
     const size_t o_wtc = off;  off += align_up(wtc.size(), 256);
+    const size_t o_up = off;   off += align_up(up.size() * sizeof(UpProb), 256);
     ctx_free(ctx, plan.d_blob);
     plan.d_blob = ctx_alloc(ctx, off + 256); plan.blob_bytes = off;
     if (!plan.d_blob) { ctx->err = "allocator returned NULL for the launch plan"; return RESIST_ENOMEM; }
@@ -435,6 +469,8 @@ static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool s
     plan.d_tc = base + o_tc; plan.tc_stride = tcb;
     if (!wtc.empty()) memcpy(host.data() + o_wtc, wtc.data(), wtc.size());
     plan.d_wtc = base + o_wtc; plan.wtc_stride = wtcb;
+    if (!up.empty()) memcpy(host.data() + o_up, up.data(), up.size() * sizeof(UpProb));
+    plan.d_up = (UpProb*)(base + o_up);
     cudaError_t e = cudaMemcpyAsync(plan.d_blob, host.data(), off, cudaMemcpyHostToDevice, st);
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
     if (e != cudaSuccess) { ctx->err = std::string("plan upload: ") + cudaGetErrorString(e); return RESIST_ECUDA; }
@@ -469,7 +505,7 @@ static int build_plan(resist_ctx* ctx, Plan& plan, int sub, int B, cudaStream_t 
     for (int s = s0; s < s1; ++s) {
         Builder bd{ctx, B, s, s, false, 0, (char*)ctx->d_ws + (size_t)s * ctx->ws_slice};
         bd.es = ctx->opts.dtype == RESIST_BF16 ? 2 : 4; bd.ops = &ops;
-        bd.bn_partial_need = needs[s].bn_partial; bd.wgrad_partial_need = needs[s].wgrad_partial; bd.gbig = needs[s].gbig;
+        bd.bn_partial_need = needs[s].bn_partial; bd.wgrad_partial_need = needs[s].wgrad_partial; bd.gbig = needs[s].gbig; bd.up_need = needs[s].up;
         const size_t used = unroll_subnet(ctx, bd, present_of(ctx, s), 1.f);
         if (used > ctx->ws_slice) { ctx->err = "internal: workspace slice too small"; return RESIST_EINVAL; }
         ctx->logits_dev[s] = bd.logits; ctx->logits_B[s] = B;
@@ -503,6 +539,7 @@ static int run_plan(resist_ctx* ctx, Plan& plan, const PatchArgs& pa, bool updat
             case OP_POOL_BWD: pk = PK_POOL_BWD; break;
             case OP_HEAD_FWD: pk = PK_HEAD_FWD; nk = 3; break;
             case OP_HEAD_BWD: pk = PK_HEAD_BWD; nk = 3; break;
+            case OP_UPSAMPLE: pk = PK_UPSAMPLE; break;
         }
         pf.begin(pk, nk, L.bytes, L.flops, st);
         switch (L.kind) {
@@ -521,6 +558,7 @@ static int run_plan(resist_ctx* ctx, Plan& plan, const PatchArgs& pa, bool updat
             case OP_POOL_BWD: launch_maxpool_bwd(plan.d_pool + L.first, L.count, L.max_elems, bf, st); ++n_launch; break;
             case OP_HEAD_FWD: launch_head_fwd(plan.d_head + L.first, L.count, L.max_b, L.max_c, L.max_classes, bf, st); n_launch += 3; break;
             case OP_HEAD_BWD: launch_head_bwd(plan.d_head + L.first, L.count, L.max_b, L.max_c, L.max_classes, L.max_elems, bf, st); n_launch += 3; break;
+            case OP_UPSAMPLE: launch_zero_stuff(plan.d_up + L.first, L.count, L.max_elems, st); ++n_launch; break;
         }
         pf.end(st);
     }
@@ -604,7 +642,7 @@ int resist_eval(resist_ctx* ctx, const void* images, const int32_t* labels, int3
         }
         std::vector<Op> ops;
         Builder bd{ctx, B, 0, copy, true, 0, (char*)ctx->d_eval_ws}; bd.es = ctx->opts.dtype == RESIST_BF16 ? 2 : 4; bd.ops = &ops;
-        bd.bn_partial_need = n.bn_partial; bd.wgrad_partial_need = n.wgrad_partial; bd.gbig = n.gbig;
+        bd.bn_partial_need = n.bn_partial; bd.wgrad_partial_need = n.wgrad_partial; bd.gbig = n.gbig; bd.up_need = n.up;
         unroll_subnet(ctx, bd, all, 1.f / (float)S);
         plan.sub = -2;
         rc = upload_plan(ctx, plan, ops, true, st);
