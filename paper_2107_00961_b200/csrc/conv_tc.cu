@@ -82,48 +82,37 @@ struct alignas(64) TcProb {
     int a_stage_bytes, b_stage_bytes, b_tap_bytes;
     int b_mn_major;                         // 0: forward (weights K-major); 1: dgrad (weights MN-major)
     int tmem_cols; int flat;                // flat = 1: 1x1 layer, tile = 128 consecutive pixels of the whole tensor
-    int stages;                             // depth of the activation ring (1..4)
-    int b_resident;                         // 1: the whole filter is fetched once per CTA and stays in shared memory
+    int stages;                             // pipeline depth: 1 when the reduction fits one stage, else 2
     int os, P, Q;                           // output stride: only positions (i,j) with i,j multiples of os are stored, as pixel (i/os, j/os) of a P x Q image
     float scale;
 };
 
 constexpr int TC_THREADS = 192;
-constexpr int TC_MAX_STAGES = 4;
+constexpr int TC_STAGES = 2;
 
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-
-// Persistent: a CTA walks the tiles blockIdx.x, blockIdx.x + gridDim.x, ... of its problem.  The activation
-// stages form a ring that runs ahead across tile boundaries, the accumulator is double-buffered in TMEM so the
-// epilogue of one tile overlaps the MMAs of the next, and when the whole filter fits (one channel chunk, one
-// N tile) the weights are fetched once per CTA and stay resident.
 __global__ void __launch_bounds__(TC_THREADS) conv_tc_kernel(const TcProb* __restrict__ probs) {
-    const TcProb* gp = probs + blockIdx.y;                        // the tensor maps are used from global memory
-    __shared__ __align__(64) uint32_t ps_words[sizeof(TcProb) / 4];
-    for (int w = threadIdx.x; w < (int)(sizeof(TcProb) / 4); w += TC_THREADS) ps_words[w] = reinterpret_cast<const uint32_t*>(gp)[w];
-    __syncthreads();
-    const TcProb& p = *reinterpret_cast<const TcProb*>(ps_words);
+    const TcProb& p = probs[blockIdx.y];
     const int tiles = p.n_img * p.tiles_per_img * p.tiles_n;
     if ((int)blockIdx.x >= tiles) return;
+    const int tn = blockIdx.x % p.tiles_n;
+    const int tm = blockIdx.x / p.tiles_n;
+    const int img = tm / p.tiles_per_img, t_in = tm % p.tiles_per_img;
+    const int pos0 = t_in * 128;                                  // first padded-flat position of this tile
+    const int row0 = p.flat ? 0 : pos0 / p.Wp;                    // first output row touched
+    const int a_off = p.flat ? 0 : pos0 - row0 * p.Wp;            // tile start inside the box, tap (0,0)
 
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 127) & ~(uintptr_t)127);
-    __shared__ __align__(8) uint64_t bars[2 * TC_MAX_STAGES + 5];
+    __shared__ __align__(8) uint64_t bars[2 * TC_STAGES + 1];
     __shared__ uint32_t tmem_base_s;
-    __shared__ volatile int abort_s;
-    const uint32_t bar_full = smem_u32(&bars[0]), bar_empty = smem_u32(&bars[TC_MAX_STAGES]), bar_b = smem_u32(&bars[2 * TC_MAX_STAGES]);
-    const uint32_t bar_tfull = smem_u32(&bars[2 * TC_MAX_STAGES + 1]), bar_tempty = smem_u32(&bars[2 * TC_MAX_STAGES + 3]);
+    __shared__ int abort_s;
+    const uint32_t bar_full = smem_u32(&bars[0]), bar_empty = smem_u32(&bars[TC_STAGES]), bar_acc = smem_u32(&bars[2 * TC_STAGES]);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int b_res_bytes = p.b_resident ? p.b_stage_bytes : 0;
-    const int stage_bytes = p.a_stage_bytes + (p.b_resident ? 0 : p.b_stage_bytes);
-    uint8_t* ring = smem + b_res_bytes;
+    const int stage_bytes = p.a_stage_bytes + p.b_stage_bytes;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < p.stages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
-        mbar_init(bar_b, 1);
-        for (int a = 0; a < 2; ++a) { mbar_init(bar_tfull + 8 * a, 1); mbar_init(bar_tempty + 8 * a, 4); }
+        for (int s = 0; s < TC_STAGES; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
+        mbar_init(bar_acc, 1);
         abort_s = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -139,28 +128,16 @@ __global__ void __launch_bounds__(TC_THREADS) conv_tc_kernel(const TcProb* __res
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer
         if (lane == 0) {
-            if (p.b_resident) {
-                mbar_expect_tx(bar_b, (uint32_t)(p.taps * p.b_tap_bytes));
-                tma_load_4d(smem_u32(smem), &gp->map_b, bar_b, 0, 0, 0, 0);
-            }
-            uint32_t it = 0;
-            for (int tile = blockIdx.x; tile < tiles && !abort_s; tile += gridDim.x) {
-                const int tn = tile % p.tiles_n, tm = tile / p.tiles_n;
-                const int img = tm / p.tiles_per_img, pos0 = (tm % p.tiles_per_img) * 128;
-                const int row0 = p.flat ? 0 : pos0 / p.Wp;
+            for (int c = 0; c < p.nchunks; ++c) {
+                const int s = c % p.stages, it = c / p.stages;
+                if (it > 0 && !mbar_wait(bar_empty + 8 * s, (it - 1) & 1)) { atomicExch(&abort_s, 1); atomicExch(p.status, 1); break; }
+                const uint32_t a_dst = smem_u32(smem + s * stage_bytes), b_dst = a_dst + p.a_stage_bytes;
+                mbar_expect_tx(bar_full + 8 * s, (uint32_t)((p.kc / 8) * p.box_w * p.box_h * 16 + p.taps * p.b_tap_bytes));
                 const int x0 = p.flat ? pos0 : -p.pad, y0 = p.flat ? 0 : row0 - p.pad;
-                for (int c = 0; c < p.nchunks; ++c, ++it) {
-                    const int s = it % p.stages; const uint32_t ph = (it / p.stages) & 1;
-                    if (!mbar_wait(bar_empty + 8 * s, ph ^ 1)) { abort_s = 1; atomicExch(p.status, 1); break; }
-                    const uint32_t a_dst = smem_u32(ring + s * stage_bytes), b_dst = a_dst + p.a_stage_bytes;
-                    mbar_expect_tx(bar_full + 8 * s, (uint32_t)((p.kc / 8) * p.box_w * p.box_h * 16 + (p.b_resident ? 0 : p.taps * p.b_tap_bytes)));
-                    for (int pl = 0; pl < p.kc / 8; ++pl)
-                        tma_load_4d(a_dst + pl * p.plane_bytes, &gp->map_a, bar_full + 8 * s, c * p.kc + pl * 8, x0, y0, img);
-                    if (!p.b_resident) {
-                        if (!p.b_mn_major) tma_load_4d(b_dst, &gp->map_b, bar_full + 8 * s, 0, tn * p.n_tile, c * (p.kc / 8), 0);
-                        else tma_load_4d(b_dst, &gp->map_b, bar_full + 8 * s, 0, c * p.kc, tn * (p.n_tile / 8), 0);
-                    }
-                }
+                for (int pl = 0; pl < p.kc / 8; ++pl)
+                    tma_load_4d(a_dst + pl * p.plane_bytes, &p.map_a, bar_full + 8 * s, c * p.kc + pl * 8, x0, y0, img);
+                if (!p.b_mn_major) tma_load_4d(b_dst, &p.map_b, bar_full + 8 * s, 0, tn * p.n_tile, c * (p.kc / 8), 0);
+                else tma_load_4d(b_dst, &p.map_b, bar_full + 8 * s, 0, c * p.kc, tn * (p.n_tile / 8), 0);
             }
         }
     } else if (warp == 1) {
@@ -171,68 +148,49 @@ __global__ void __launch_bounds__(TC_THREADS) conv_tc_kernel(const TcProb* __res
                                    ((uint32_t)(p.n_tile >> 3) << 17) | ((128u >> 4) << 24);
             const int ksz = p.taps == 9 ? 3 : 1;
             bool ok = true;
-            if (p.b_resident && !mbar_wait(bar_b, 0)) { abort_s = 1; atomicExch(p.status, 4); ok = false; }
-            uint32_t it = 0, tl = 0;
-            for (int tile = blockIdx.x; tile < tiles && ok && !abort_s; tile += gridDim.x, ++tl) {
-                const int pos0 = ((tile / p.tiles_n) % p.tiles_per_img) * 128;
-                const int a_off = p.flat ? 0 : pos0 % p.Wp;
-                const uint32_t acc = tl & 1, d_addr = tmem_d + acc * (uint32_t)p.n_tile;
-                if (!mbar_wait(bar_tempty + 8 * acc, ((tl >> 1) & 1) ^ 1)) { abort_s = 1; atomicExch(p.status, 5); ok = false; break; }
+            for (int c = 0; c < p.nchunks && ok; ++c) {
+                const int s = c % p.stages, it = c / p.stages;
+                if (!mbar_wait(bar_full + 8 * s, it & 1)) { atomicExch(&abort_s, 1); atomicExch(p.status, 2); ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                for (int c = 0; c < p.nchunks; ++c, ++it) {
-                    const int s = it % p.stages; const uint32_t ph = (it / p.stages) & 1;
-                    if (!mbar_wait(bar_full + 8 * s, ph)) { abort_s = 1; atomicExch(p.status, 2); ok = false; break; }
-                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    const uint32_t a_base = smem_u32(ring + s * stage_bytes);
-                    const uint32_t b_base = p.b_resident ? smem_u32(smem) : a_base + p.a_stage_bytes;
-                    for (int t = 0; t < p.taps; ++t) {
-                        const int r = t / ksz, q = t % ksz;
-                        const int shift = p.flip ? ((ksz - 1 - r) * p.Wp + (ksz - 1 - q)) : (r * p.Wp + q);
-                        for (int k16 = 0; k16 < p.kc / 16; ++k16) {
-                            const uint64_t ad = smem_desc(a_base + 2 * k16 * p.plane_bytes + (a_off + shift) * 16, p.plane_bytes, 128);
-                            uint64_t bd;
-                            if (!p.b_mn_major) bd = smem_desc(b_base + t * p.b_tap_bytes + 2 * k16 * p.n_tile * 16, p.n_tile * 16, 128);
-                            else bd = smem_desc(b_base + t * p.b_tap_bytes + k16 * 256, 128, p.kc * 16);
-                            umma_bf16(d_addr, ad, bd, idesc, (c | t | k16) ? 1u : 0u);
-                        }
+                const uint32_t a_base = smem_u32(smem + s * stage_bytes), b_base = a_base + p.a_stage_bytes;
+                for (int t = 0; t < p.taps; ++t) {
+                    const int r = t / ksz, q = t % ksz;
+                    const int shift = p.flip ? ((ksz - 1 - r) * p.Wp + (ksz - 1 - q)) : (r * p.Wp + q);
+                    for (int k16 = 0; k16 < p.kc / 16; ++k16) {
+                        const uint64_t ad = smem_desc(a_base + 2 * k16 * p.plane_bytes + (a_off + shift) * 16, p.plane_bytes, 128);
+                        uint64_t bd;
+                        if (!p.b_mn_major) bd = smem_desc(b_base + t * p.b_tap_bytes + 2 * k16 * p.n_tile * 16, p.n_tile * 16, 128);
+                        else bd = smem_desc(b_base + t * p.b_tap_bytes + k16 * 256, 128, p.kc * 16);
+                        umma_bf16(tmem_d, ad, bd, idesc, (c | t | k16) ? 1u : 0u);
                     }
-                    umma_commit(bar_empty + 8 * s);      // stage reusable once these MMAs have read it
                 }
-                if (ok) umma_commit(bar_tfull + 8 * acc);   // this accumulator is complete
+                umma_commit(bar_empty + 8 * s);          // stage reusable once these MMAs have read it
             }
+            if (ok) umma_commit(bar_acc);                // accumulator complete
         }
     } else {
         // ---------------------------------------------------------------- epilogue: 4 warps, one TMEM lane quadrant each
         const int quad = warp & 3;
         const int m = quad * 32 + lane;                  // row of the tile = TMEM lane
-        uint32_t tl = 0;
-        for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++tl) {
-            const int tn = tile % p.tiles_n, tm = tile / p.tiles_n;
-            const int img = tm / p.tiles_per_img, pos0 = (tm % p.tiles_per_img) * 128;
-            const uint32_t acc = tl & 1;
-            bool ok = mbar_wait(bar_tfull + 8 * acc, (tl >> 1) & 1);
-            ok = __all_sync(0xffffffffu, ok);            // tcgen05.ld below is warp-collective
-            if (!ok) { abort_s = 1; atomicExch(p.status, 3); break; }
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            // padded-flat position -> output pixel
-            long long pix = -1;
-            if (p.flat) { const long long g = (long long)pos0 + m; if (g < (long long)p.W) pix = g; }
-            else {
-                const int pos = pos0 + m, i = pos / p.Wp, j = pos - i * p.Wp;
-                if (i < p.H && j < p.W) {
-                    if (p.os == 1) pix = ((long long)img * p.H + i) * p.W + j;
-                    else if (i % p.os == 0 && j % p.os == 0) pix = ((long long)img * p.P + i / p.os) * p.Q + j / p.os;   // strided layer
-                }
+        bool ok = mbar_wait(bar_acc, 0);
+        ok = __all_sync(0xffffffffu, ok);                // tcgen05.ld below is warp-collective
+        if (!ok) { atomicExch(&abort_s, 1); atomicExch(p.status, 3); }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        // padded-flat position -> output pixel
+        long long pix = -1;
+        if (p.flat) { const long long g = (long long)pos0 + m; if (g < (long long)p.W) pix = g; }
+        else {
+            const int pos = pos0 + m, i = pos / p.Wp, j = pos - i * p.Wp;
+            if (i < p.H && j < p.W) {
+                if (p.os == 1) pix = ((long long)img * p.H + i) * p.W + j;
+                else if (i % p.os == 0 && j % p.os == 0) pix = ((long long)img * p.P + i / p.os) * p.Q + j / p.os;   // strided layer
             }
+        }
+        if (ok) {
             for (int c0 = 0; c0 < p.n_tile; c0 += 16) {
                 uint32_t v[16];
-                tmem_ld16(tmem_d + ((uint32_t)(quad * 32) << 16) + acc * (uint32_t)p.n_tile + (uint32_t)c0, v);
+                tmem_ld16(tmem_d + ((uint32_t)(quad * 32) << 16) + (uint32_t)c0, v);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                if (c0 + 16 >= p.n_tile) {               // last read of this accumulator: hand it back to the MMA warp
-                    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);
-                }
                 if (pix >= 0) {
                     const long long o = pix * p.ncol + tn * p.n_tile + c0;
                     float f[16];
@@ -457,7 +415,7 @@ static bool encode4(CUtensorMap* m, const void* base, const uint64_t dims[4], co
               CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-struct TcGeom { int b_resident, stages, chan_a, ncol, n_tile, kc, nchunks, Wp, box_w, box_h, plane_bytes, a_stage, b_stage, b_tap, tiles_per_img, n_img, H, W, flat, tmem_cols; size_t smem; };
+struct TcGeom { int stages, chan_a, ncol, n_tile, kc, nchunks, Wp, box_w, box_h, plane_bytes, a_stage, b_stage, b_tap, tiles_per_img, n_img, H, W, flat, tmem_cols; size_t smem; };
 
 // Decides whether (and how) the tensor-core kernel takes this problem.
 static bool tc_geometry(const ConvProb& p, int mode, TcGeom& g) {
@@ -489,15 +447,10 @@ static bool tc_geometry(const ConvProb& p, int mode, TcGeom& g) {
     g.plane_bytes = ((plane_px * 16 + 127) / 128) * 128;
     g.a_stage = (kc / 8) * g.plane_bytes;
     g.b_tap = g.n_tile * kc * 2; g.b_stage = ((taps * g.b_tap + 127) / 128) * 128;
-    g.b_resident = (g.nchunks == 1 && g.ncol == g.n_tile) ? 1 : 0;
-    const size_t fixed = g.b_resident ? g.b_stage : 0, per_stage = g.a_stage + (g.b_resident ? 0 : g.b_stage);
-    // a small footprint lets several CTAs share an SM; deep rings only when a stage is small
-    g.stages = TC_MAX_STAGES;
-    while (g.stages > 2 && fixed + (size_t)g.stages * per_stage > 64 * 1024) --g.stages;
-    while (g.stages > 1 && fixed + (size_t)g.stages * per_stage + 256 > 200 * 1024) --g.stages;
-    g.smem = fixed + (size_t)g.stages * per_stage + 256;
+    g.stages = g.nchunks > 1 ? TC_STAGES : 1;
+    g.smem = (size_t)g.stages * (g.a_stage + g.b_stage) + 256;
     if (g.smem > 200 * 1024) return false;
-    g.tmem_cols = 32; while (g.tmem_cols < 2 * g.n_tile) g.tmem_cols *= 2;
+    g.tmem_cols = 32; while (g.tmem_cols < g.n_tile) g.tmem_cols *= 2;
     return true;
 }
 
@@ -536,7 +489,7 @@ bool conv_tc_fill(const ConvProb& p, int mode, void* host_tc) {
     t.n_img = g.n_img; t.tiles_per_img = g.tiles_per_img; t.tiles_n = g.ncol / g.n_tile; t.ncol = g.ncol; t.n_tile = g.n_tile;
     t.kc = g.kc; t.nchunks = g.nchunks; t.box_w = g.box_w; t.box_h = g.box_h; t.plane_bytes = g.plane_bytes;
     t.a_stage_bytes = g.a_stage; t.b_stage_bytes = g.b_stage; t.b_tap_bytes = g.b_tap; t.b_mn_major = mode == CONV_DGRAD ? 1 : 0;
-    t.tmem_cols = g.tmem_cols; t.flat = g.flat; t.scale = p.scale; t.stages = g.stages; t.b_resident = g.b_resident;
+    t.tmem_cols = g.tmem_cols; t.flat = g.flat; t.scale = p.scale; t.stages = g.stages;
     t.os = (mode == CONV_FWD) ? p.stride : 1; t.P = p.P; t.Q = p.Q;
     memcpy(host_tc, &t, sizeof(t));
     return true;
@@ -544,8 +497,7 @@ bool conv_tc_fill(const ConvProb& p, int mode, void* host_tc) {
 size_t conv_tc_prob_bytes() { return sizeof(TcProb); }
 int conv_tc_tiles(const void* host_tc) { const TcProb* t = (const TcProb*)host_tc; return t->n_img * t->tiles_per_img * t->tiles_n; }
 size_t conv_tc_smem(const void* host_tc) {
-    const TcProb* t = (const TcProb*)host_tc;
-    return (size_t)(t->b_resident ? t->b_stage_bytes : 0) + (size_t)t->stages * (t->a_stage_bytes + (t->b_resident ? 0 : t->b_stage_bytes)) + 256;
+    const TcProb* t = (const TcProb*)host_tc; return (size_t)t->stages * (t->a_stage_bytes + t->b_stage_bytes) + 256;
 }
 
 void launch_conv_tc_probs(const void* d_tc, int nprob, int max_tiles, size_t max_smem, cudaStream_t s) {
@@ -554,11 +506,7 @@ void launch_conv_tc_probs(const void* d_tc, int nprob, int max_tiles, size_t max
         cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(200 * 1024 + 256));
         configured = 200 * 1024 + 256;
     }
-    // persistent CTAs: about three per SM over all problems of the launch, never more than the tiles of the largest
-    static int sms = 0;
-    if (!sms) { int dev = 0; cudaGetDevice(&dev); cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev); if (sms < 1) sms = 148; }
-    int gx = (3 * sms + nprob - 1) / nprob; if (gx > max_tiles) gx = max_tiles; if (gx < 1) gx = 1;
-    conv_tc_kernel<<<dim3(gx, nprob), TC_THREADS, max_smem, s>>>((const TcProb*)d_tc);
+    conv_tc_kernel<<<dim3(max_tiles, nprob), TC_THREADS, max_smem, s>>>((const TcProb*)d_tc);
 }
 
 // ---- wgrad host side

@@ -310,15 +310,19 @@ __global__ void __launch_bounds__(256) bn_reduce_kernel(const BnProb* __restrict
 
 template <class T, int MODE>
 __global__ void bn_finalize_kernel(const BnProb* __restrict__ probs) {
+    // one warp per channel: lane l adds chunks l, l+32, ... in order, then a fixed butterfly over the lanes
     const BnProb& p = probs[blockIdx.y];
-    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    const int lane = threadIdx.x & 31;
+    const int c = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (c >= p.C) return;
     if (p.eval) {
-        if (MODE == 0) { p.stat[c] = p.run_mean[c]; p.stat[p.C + c] = (float)(1.0 / sqrt((double)p.run_var[c] + (double)p.eps)); }
+        if (MODE == 0 && lane == 0) { p.stat[c] = p.run_mean[c]; p.stat[p.C + c] = (float)(1.0 / sqrt((double)p.run_var[c] + (double)p.eps)); }
         return;
     }
     double a0 = 0.0, a1 = 0.0;
-    for (int k = 0; k < p.chunks; ++k) { a0 += p.partial[((long long)k * 2 + 0) * p.C + c]; a1 += p.partial[((long long)k * 2 + 1) * p.C + c]; }
+    for (int k = lane; k < p.chunks; k += 32) { a0 += p.partial[((long long)k * 2 + 0) * p.C + c]; a1 += p.partial[((long long)k * 2 + 1) * p.C + c]; }
+    for (int d = 16; d; d >>= 1) { a0 += __shfl_xor_sync(0xffffffffu, a0, d); a1 += __shfl_xor_sync(0xffffffffu, a1, d); }
+    if (lane != 0) return;
     if (MODE == 0) {
         const double m = (double)p.m, dm = a0 / m;                 // sums are of x - x[0,c]
         double var = a1 / m - dm * dm; if (var < 0.0) var = 0.0;
@@ -370,8 +374,8 @@ static int ew_grid(long long n) { long long g = (n + 255) / 256; if (g > 148 * 1
 void launch_bn_stats(const BnProb* d, int nprob, int max_chunks, int max_c, bool bf16, cudaStream_t s) {
     if (bf16) bn_reduce_kernel<__nv_bfloat16, 0><<<dim3(max_chunks, nprob), 256, 0, s>>>(d);
     else bn_reduce_kernel<float, 0><<<dim3(max_chunks, nprob), 256, 0, s>>>(d);
-    if (bf16) bn_finalize_kernel<__nv_bfloat16, 0><<<dim3((max_c + 127) / 128, nprob), 128, 0, s>>>(d);
-    else bn_finalize_kernel<float, 0><<<dim3((max_c + 127) / 128, nprob), 128, 0, s>>>(d);
+    if (bf16) bn_finalize_kernel<__nv_bfloat16, 0><<<dim3((max_c + 7) / 8, nprob), 256, 0, s>>>(d);
+    else bn_finalize_kernel<float, 0><<<dim3((max_c + 7) / 8, nprob), 256, 0, s>>>(d);
 }
 void launch_bn_apply(const BnProb* d, int nprob, long long max_elems, bool bf16, cudaStream_t s) {
     if (bf16) bn_apply_kernel<__nv_bfloat16><<<dim3(ew_grid(max_elems), nprob), 256, 0, s>>>(d);
@@ -380,7 +384,7 @@ void launch_bn_apply(const BnProb* d, int nprob, long long max_elems, bool bf16,
 void launch_bn_bwd_reduce(const BnProb* d, int nprob, int max_chunks, int max_c, bool bf16, cudaStream_t s) {
     if (bf16) bn_reduce_kernel<__nv_bfloat16, 1><<<dim3(max_chunks, nprob), 256, 0, s>>>(d);
     else bn_reduce_kernel<float, 1><<<dim3(max_chunks, nprob), 256, 0, s>>>(d);
-    bn_finalize_kernel<float, 1><<<dim3((max_c + 127) / 128, nprob), 128, 0, s>>>(d);
+    bn_finalize_kernel<float, 1><<<dim3((max_c + 7) / 8, nprob), 256, 0, s>>>(d);
 }
 void launch_bn_bwd_apply(const BnProb* d, int nprob, long long max_elems, bool bf16, cudaStream_t s) {
     if (bf16) bn_bwd_apply_kernel<__nv_bfloat16><<<dim3(ew_grid(max_elems), nprob), 256, 0, s>>>(d);
