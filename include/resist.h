@@ -47,7 +47,7 @@ typedef enum {
 enum { RESIST_BASIC = 0, RESIST_BOTTLENECK = 1 };
 enum { RESIST_F32 = 0, RESIST_BF16 = 1 };
 enum { RESIST_MOMENTUM_RESTART = 0, RESIST_MOMENTUM_KEEP = 1 };
-enum { RESIST_CONV_AUTO = 0, RESIST_CONV_CUDA_CORES = 1 };
+enum { RESIST_CONV_AUTO = 0, RESIST_CONV_CUDA_CORES = 1, RESIST_CONV_TCGEN05 = 2, RESIST_CONV_WARP_MMA = 3 };
 #define RESIST_MAX_SUBNETS 32
 
 typedef struct resist_ctx resist_ctx;
@@ -84,7 +84,9 @@ typedef struct {
     float bn_momentum;       /* running = (1-m)*running + m*batch (variance unbiased) */
     int32_t min_depth;       /* >0: top sub-ResNets up to this many partitioned blocks (Sec. 2.6) */
     int32_t momentum_policy; /* RESIST_MOMENTUM_RESTART: zero the momentum at every partition */
-    int32_t conv_backend;    /* RESIST_CONV_AUTO: tensor cores where the shape allows; _CUDA_CORES: never */
+    int32_t conv_backend;    /* RESIST_CONV_AUTO: warp-level MMA for narrow layers (<= 64 channels), tcgen05 for wide ones,
+                                CUDA cores for the rest; _CUDA_CORES: never tensor cores; _TCGEN05 / _WARP_MMA: only that
+                                tensor-core family where the shape allows, CUDA cores elsewhere */
 } resist_opts;
 
 /* Device-memory source.  alloc returns a device pointer aligned to >= 256 bytes or NULL; release frees it.
@@ -160,8 +162,8 @@ int resist_get_step_info(resist_ctx* ctx, resist_step_info* out);
  *   mode 0 (forward): act = a, wgt = w, out = y = scale * conv(a, w) + add      (add: y-shaped or NULL)
  *   mode 1 (dgrad):   act = dy, wgt = w, out = da = conv^T(dy, w) + add         (add: a-shaped or NULL)
  *   mode 2 (wgrad):   act = a, wgt = dy, out = dw, fp32 [K,k,k,C]
- * backend: RESIST_CONV_AUTO or RESIST_CONV_CUDA_CORES; *used_backend (host, may be NULL) receives 1 when the
- * tensor-core kernel ran. */
+ * backend: one of RESIST_CONV_*; *used_backend (host, may be NULL) receives 0 (CUDA cores), 1 (tcgen05) or
+ * 2 (warp-level MMA). */
 int resist_conv2d(int32_t mode, int32_t dtype, int32_t backend, const void* act, const void* wgt, const void* add, void* out,
                   int32_t N, int32_t H, int32_t W, int32_t C, int32_t K, int32_t ksz, int32_t stride, float scale,
                   int32_t* used_backend, resist_stream stream);

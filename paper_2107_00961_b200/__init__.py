@@ -17,7 +17,7 @@ from . import build as _build
 
 RESIST_OK = 0
 F32, BF16 = 0, 1
-CONV_AUTO, CONV_CUDA_CORES = 0, 1
+CONV_AUTO, CONV_CUDA_CORES, CONV_TCGEN05, CONV_WARP_MMA = 0, 1, 2, 3
 MOMENTUM_RESTART, MOMENTUM_KEEP = 0, 1
 _STATUS = {0: "RESIST_OK", -1: "RESIST_EINVAL", -2: "RESIST_ESTATE", -3: "RESIST_ENOMEM", -4: "RESIST_ECUDA",
            -5: "RESIST_ETIMEOUT", -6: "RESIST_EUNSUPPORTED"}
@@ -133,7 +133,7 @@ def _dt(t: torch.Tensor) -> int:
 
 def resist_conv2d(mode: int, act: torch.Tensor, wgt: torch.Tensor, geom, add: Optional[torch.Tensor] = None,
                   scale: float = 1.0, backend: int = CONV_AUTO, stream=None):
-    """geom = (N, H, W, C, K, ksz, stride) of the forward convolution.  Returns (out, used_tensor_cores)."""
+    """geom = (N, H, W, C, K, ksz, stride) of the forward convolution.  Returns (out, family) with family 0 = CUDA cores, 1 = tcgen05, 2 = warp-level MMA."""
     N, H, W, Cc, K, ksz, stride = geom
     P, Q = _odim(H, ksz, stride), _odim(W, ksz, stride)
     if mode == 0:
@@ -146,7 +146,7 @@ def resist_conv2d(mode: int, act: torch.Tensor, wgt: torch.Tensor, geom, add: Op
     _layer_check(lib().resist_conv2d(mode, _dt(act), backend, act.data_ptr(), wgt.data_ptr(),
                                      add.data_ptr() if add is not None else None, out.data_ptr(), N, H, W, Cc, K, ksz,
                                      stride, scale, C.addressof(used), _stream_handle(stream)))
-    return out, bool(used.value)
+    return out, int(used.value)
 
 
 def resist_bn_relu_forward(x: torch.Tensor, gamma, beta, run_mean=None, run_var=None, eps=1e-5, momentum=0.1, stream=None):

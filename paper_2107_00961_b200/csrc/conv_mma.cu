@@ -1,0 +1,514 @@
+// Convolutions of NARROW layers (C and K multiples of 16, at most 64) on warp-level MMA (mma.sync m16n8k16, bf16
+// inputs, fp32 accumulation).
+//
+// Why not tcgen05 here: one tcgen05.mma with M = 128, K = 16 occupies the SM's tensor core for ~153 cycles whatever
+// N is (measured for N = 16 ... 256, every operand layout, one MMA at a time per SM), so a layer with 16 output
+// channels uses 1/16 of the array and is bound by that rate at a third of what HBM allows.  The warp-level MMA
+// has no such granularity (n = 8) and was measured at 550 TFLOP/s dense on this GPU, far more than these
+// HBM-bound layers need.  Wide layers (more than 64 channels) stay on tcgen05 (conv_tc.cu).
+//
+// Tiling: the whole batch is ONE tall zero-padded image.  With pad = k/2, image n occupies rows n*Hp .. n*Hp+H-1
+// (Hp = H + pad) of a map that is Wp = W + pad wide; row H of every image and column W of every row are zero and
+// serve as the padding of both neighbours, because positions are numbered row-major ("padded-flat", f = Y*Wp + X)
+// and a tap (r, s) reads position f + (r-pad)*Wp + (s-pad).  A tile is 128 or 256 consecutive positions; the window
+// of positions it needs (tile + halo of pad*Wp + pad on either side) is staged once in shared memory as
+// [position][channel] rows, padded by 16 bytes against bank conflicts, and the k*k taps read it at shifted row
+// offsets through ldmatrix.  Padding positions are computed like any other and dropped by the epilogue.
+#include <algorithm>
+#include <cstring>
+#include "internal.h"
+
+namespace resist {
+
+struct alignas(16) MmaProb {
+    const __nv_bfloat16* act;   // forward: a [n_img,H,W,ca]; dgrad: dy (stride 1, possibly zero-stuffed)
+    const __nv_bfloat16* wgt;   // [K][taps][C]
+    const __nv_bfloat16* add; __nv_bfloat16* out;
+    int ca, ncol;               // channels of act (reduction) and of out
+    int wC;                     // C of the weight tensor (its innermost extent)
+    int H, W, Hp, Wp;           // image extent; extent of one image in the tall padded map
+    unsigned inv_wp, inv_hp;    // floor(2^32 / d) + 1: __umulhi(f, inv) = f / d for every f the kernel meets
+    int total;                  // positions of the tall padded map, n_img * Hp * Wp
+    int tiles;                  // ceil(total / tile)
+    int os, P, Q;               // output stride (forward of a stride-2 layer stores even positions only, as a P x Q image)
+    int stages;                 // depth of the activation ring (2, 3 or 4)
+    int variant;                // which instantiation runs this problem (see mma_variant)
+    float scale;
+};
+
+__device__ __forceinline__ uint32_t s_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x2(uint32_t addr, uint32_t& r0, uint32_t& r1) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x2.shared.b16 {%0,%1}, [%2];" : "=r"(r0), "=r"(r1) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x2_t(uint32_t addr, uint32_t& r0, uint32_t& r1) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0,%1}, [%2];" : "=r"(r0), "=r"(r1) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void mma16816(float* c, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+constexpr int MMA_THREADS = 256;
+constexpr int MMA_SLOTS = 10;          // 16-byte pieces of the activation window a thread copies per tile (at most)
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");   // src_bytes 0: zeros
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// Column n of the MMA's B operand carries output channel chan_of_col(n): thread (g8, t4) of a warp then owns, over its
+// NB accumulator blocks, the 2*NB CONSECUTIVE channels t4*2*NB ... and stores them with 8- or 16-byte accesses.
+template <int NB> __host__ __device__ __forceinline__ int chan_of_col(int n) { return ((n & 7) >> 1) * (2 * NB) + 2 * (n >> 3) + (n & 1); }
+template <int NB> __host__ __device__ __forceinline__ int col_of_chan(int c) { return 8 * ((c % (2 * NB)) >> 1) + 2 * (c / (2 * NB)) + (c & 1); }
+
+// Persistent: a CTA keeps the whole filter in shared memory and walks the tiles blockIdx.x, blockIdx.x + gridDim.x, ...
+// of its problem.  The activation windows of the next tiles are in flight (cp.async, ring of p.stages) while the
+// warps run ldmatrix + mma.sync on the current one.
+// NB = output channels / 8 (2, 4, 6 or 8); MBW = 16-row blocks per warp (tile = 128 * MBW positions); KSZ = 1 or 3;
+// TRANS = false: forward (weights read as [n][k]); true: dgrad (weights read as [k][n] and transposed on load, taps flipped).
+template <int NB, int MBW, int KSZ, bool TRANS>
+__global__ void __launch_bounds__(MMA_THREADS) conv_mma_kernel(const MmaProb* __restrict__ probs) {
+    __shared__ MmaProb p;
+    if (threadIdx.x < sizeof(MmaProb) / 4) reinterpret_cast<uint32_t*>(&p)[threadIdx.x] = reinterpret_cast<const uint32_t*>(probs + blockIdx.y)[threadIdx.x];
+    __syncthreads();
+    constexpr int TILE = 128 * MBW, TAPS = KSZ * KSZ, PAD = KSZ / 2;
+    const int tiles = p.tiles;
+    if ((int)blockIdx.x >= tiles) return;
+    extern __shared__ __align__(16) uint8_t sm[];
+    const int ca = p.ca, apitch = ca * 2 + 16;                    // activation row pitch in bytes
+    constexpr int ncol = NB * 8;
+    const int wrows = TRANS ? ca : ncol;                          // rows of one tap of the staged filter
+    const int wcols = TRANS ? ncol : ca;                          // elements per row
+    const int wpitch = wcols * 2 + 16;
+    const int H = p.H, W = p.W, Hp = p.Hp, Wp = p.Wp, total = p.total, stages = p.stages, os = p.os;
+    const unsigned inv_wp = p.inv_wp, inv_hp = p.inv_hp;
+    const int halo = PAD * Wp + PAD, win_rows = TILE + 2 * halo;
+    const int stage_bytes = (win_rows * apitch + 127) & ~127;
+    uint8_t* s_w = sm + stages * stage_bytes;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const __nv_bfloat16* __restrict__ act = p.act;
+
+    // ---- the filter, once per CTA
+    if (!TRANS) {               // tap t, column n, 8-channel group g  <-  w[chan_of_col(n)][t][g*8..]
+        const int groups = ca / 8, n_chunks = TAPS * ncol * groups;
+        for (int id = tid; id < n_chunks; id += MMA_THREADS) {
+            const int g = id % groups, n = (id / groups) % ncol, t = id / (groups * ncol);
+            const uint4 v = __ldg(reinterpret_cast<const uint4*>(p.wgt + ((long long)chan_of_col<NB>(n) * TAPS + t) * p.wC + g * 8));
+            *reinterpret_cast<uint4*>(s_w + (t * wrows + n) * wpitch + g * 16) = v;
+        }
+    } else {                    // tap t, row k, column col_of_chan(c)  <-  w[k][t][c]
+        constexpr int groups = ncol / 8; const int n_chunks = TAPS * ca * groups;
+        for (int id = tid; id < n_chunks; id += MMA_THREADS) {
+            const int g = id % groups, k = (id / groups) % ca, t = id / (groups * ca);
+            const uint4 v = __ldg(reinterpret_cast<const uint4*>(p.wgt + ((long long)k * TAPS + t) * p.wC + g * 8));
+            const uint32_t w4[4] = {v.x, v.y, v.z, v.w};
+            uint8_t* row = s_w + (t * wrows + k) * wpitch;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) *reinterpret_cast<uint32_t*>(row + col_of_chan<NB>(g * 8 + 2 * e) * 2) = w4[e];   // channel pairs stay adjacent
+        }
+    }
+    // ---- what this thread copies for every tile: the same pieces of the window, fixed once (row | group << 16)
+    const int groups = ca / 8, nchunk = win_rows * groups;
+    int slot[MMA_SLOTS];
+#pragma unroll
+    for (int k = 0; k < MMA_SLOTS; ++k) {
+        const int id = tid + k * MMA_THREADS;
+        slot[k] = id < nchunk ? ((id / groups) | ((id % groups) << 16)) : -1;
+    }
+    auto issue = [&](int tile, int stage) {
+        const int f0 = tile * TILE - halo;                         // position of window row 0 (negative at the very start)
+        const uint32_t dst0 = s_u32(sm + stage * stage_bytes);
+#pragma unroll
+        for (int k = 0; k < MMA_SLOTS; ++k) {
+            if (slot[k] < 0) continue;
+            const int w = slot[k] & 0xFFFF, g = slot[k] >> 16;
+            const unsigned f = (unsigned)(f0 + w);
+            const unsigned Y = __umulhi(f, inv_wp), X = f - Y * Wp;
+            const unsigned n = __umulhi(Y, inv_hp), i = Y - n * Hp;
+            const bool ok = f < (unsigned)total && X < (unsigned)W && i < (unsigned)H;
+            const __nv_bfloat16* src = ok ? act + (((long long)n * H + i) * W + X) * ca + g * 8 : act;
+            cp_async16(dst0 + w * apitch + g * 16, src, ok ? 16u : 0u);
+        }
+    };
+
+    const uint32_t w_base = s_u32(s_w);
+    const int g8 = lane >> 2, t4 = lane & 3;
+    const uint32_t a_lane = (uint32_t)(warp * 16 * MBW + (lane & 15)) * apitch + (lane >> 4) * 16;
+    // B fragments of two 8-column blocks per ldmatrix.x4: lanes 0-7 / 8-15 address the two k halves of block j, lanes 16-31 those of block j+1
+    const uint32_t b_lane = TRANS ? (uint32_t)(((lane >> 3) & 1) * 8 + (lane & 7)) * wpitch + (lane >> 4) * 16
+                                  : (uint32_t)((lane >> 4) * 8 + (lane & 7)) * wpitch + ((lane >> 3) & 1) * 16;
+
+    // prologue: the first stages-1 tiles of this CTA
+    int nxt = blockIdx.x;
+    for (int st = 0; st < stages - 1; ++st) { if (nxt < tiles) issue(nxt, st); cp_async_commit(); nxt += gridDim.x; }
+    int stage = 0;
+    for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+        { const int ps = stage == 0 ? stages - 1 : stage - 1; if (nxt < tiles) issue(nxt, ps); cp_async_commit(); nxt += gridDim.x; }
+        if (stages == 2) cp_async_wait<1>(); else if (stages == 3) cp_async_wait<2>(); else cp_async_wait<3>();
+        __syncthreads();                                          // this tile's window (and, first time, the filter) is in shared memory
+
+        const uint32_t a_base = s_u32(sm + stage * stage_bytes) + a_lane;
+        float acc[MBW][NB][4];
+#pragma unroll
+        for (int mb = 0; mb < MBW; ++mb)
+#pragma unroll
+            for (int j = 0; j < NB; ++j) { acc[mb][j][0] = acc[mb][j][1] = acc[mb][j][2] = acc[mb][j][3] = 0.f; }
+#pragma unroll
+        for (int t = 0; t < TAPS; ++t) {
+            constexpr int K1 = KSZ - 1;
+            const int r = t / KSZ, q = t % KSZ;
+            const int shift = TRANS ? ((K1 - r) * Wp + (K1 - q)) : (r * Wp + q);
+            const uint32_t a_tap = a_base + (uint32_t)shift * apitch;
+            const uint32_t w_tap = w_base + (uint32_t)(t * wrows) * wpitch + b_lane;
+            for (int k0 = 0; k0 < ca; k0 += 16) {
+                uint32_t a[MBW][4];
+#pragma unroll
+                for (int mb = 0; mb < MBW; ++mb) ldsm_x4(a_tap + (uint32_t)(mb * 16) * apitch + k0 * 2, a[mb][0], a[mb][1], a[mb][2], a[mb][3]);
+#pragma unroll
+                for (int j = 0; j < NB; j += 2) {
+                    uint32_t b0, b1, b2, b3;
+                    if (!TRANS) ldsm_x4(w_tap + (uint32_t)(j * 8) * wpitch + k0 * 2, b0, b1, b2, b3);
+                    else ldsm_x4_t(w_tap + (uint32_t)k0 * wpitch + j * 16, b0, b1, b2, b3);
+#pragma unroll
+                    for (int mb = 0; mb < MBW; ++mb) {
+                        mma16816(acc[mb][j], a[mb][0], a[mb][1], a[mb][2], a[mb][3], b0, b1);
+                        mma16816(acc[mb][j + 1], a[mb][0], a[mb][1], a[mb][2], a[mb][3], b2, b3);
+                    }
+                }
+            }
+        }
+        // ---- epilogue: thread (g8, t4) holds rows g8 and g8+8 of each 16-row block, channels t4*2*NB ... t4*2*NB + 2*NB - 1
+        const float scale = p.scale;
+        const __nv_bfloat16* __restrict__ addp = p.add;
+#pragma unroll
+        for (int mb = 0; mb < MBW; ++mb)
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                const unsigned f = (unsigned)(tile * TILE + warp * 16 * MBW + mb * 16 + g8 + half * 8);
+                const unsigned Y = __umulhi(f, inv_wp), X = f - Y * Wp;
+                const unsigned n = __umulhi(Y, inv_hp), i = Y - n * Hp;
+                if (!(f < (unsigned)total && X < (unsigned)W && i < (unsigned)H)) continue;
+                long long pix;
+                if (os == 1) pix = ((long long)n * H + i) * W + X;
+                else { if ((i % os) | (X % os)) continue; pix = ((long long)n * p.P + i / os) * p.Q + X / os; }
+                const long long o = pix * ncol + t4 * (2 * NB);
+                uint32_t wv[NB];
+                if (addp) {
+                    if constexpr (NB % 4 == 0) {
+#pragma unroll
+                        for (int c4 = 0; c4 < NB / 4; ++c4) { const uint4 v = *reinterpret_cast<const uint4*>(addp + o + c4 * 8); wv[c4 * 4] = v.x; wv[c4 * 4 + 1] = v.y; wv[c4 * 4 + 2] = v.z; wv[c4 * 4 + 3] = v.w; }
+                    } else {
+#pragma unroll
+                        for (int c2 = 0; c2 < NB / 2; ++c2) { const uint2 v = *reinterpret_cast<const uint2*>(addp + o + c2 * 4); wv[c2 * 2] = v.x; wv[c2 * 2 + 1] = v.y; }
+                    }
+                }
+#pragma unroll
+                for (int j = 0; j < NB; ++j) {
+                    float v0 = acc[mb][j][half * 2] * scale, v1 = acc[mb][j][half * 2 + 1] * scale;
+                    if (addp) { v0 += __uint_as_float(wv[j] << 16); v1 += __uint_as_float(wv[j] & 0xFFFF0000u); }
+                    __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
+                    wv[j] = *reinterpret_cast<uint32_t*>(&h);
+                }
+                if constexpr (NB % 4 == 0) {
+#pragma unroll
+                    for (int c4 = 0; c4 < NB / 4; ++c4) *reinterpret_cast<uint4*>(p.out + o + c4 * 8) = make_uint4(wv[c4 * 4], wv[c4 * 4 + 1], wv[c4 * 4 + 2], wv[c4 * 4 + 3]);
+                } else {
+#pragma unroll
+                    for (int c2 = 0; c2 < NB / 2; ++c2) *reinterpret_cast<uint2*>(p.out + o + c2 * 4) = make_uint2(wv[c2 * 2], wv[c2 * 2 + 1]);
+                }
+            }
+        __syncthreads();                                          // every warp is done with this stage before it is refilled
+        stage = stage + 1 == stages ? 0 : stage + 1;
+    }
+    cp_async_wait<0>();
+}
+
+// ------------------------------------------------------------------------------------------------ host side
+struct MmaGeom { int ca, ncol, Hp, Wp, total, mbw, tiles, stages, variant; size_t smem; };
+
+// variant = (((stages * 4 + MBW) * 4 + ksz) * 2 + trans) * 16 + NB: everything a launch is specialised on
+static int mma_variant(int stages, int mbw, int ksz, int trans, int nb) { return (((stages * 4 + mbw) * 4 + ksz) * 2 + trans) * 16 + nb; }
+
+static bool mma_geometry(const ConvProb& p, int mode, MmaGeom& g) {
+    if (mode == CONV_WGRAD) return false;
+    if ((p.ksz != 1 && p.ksz != 3) || p.stride < 1 || p.stride > 2 || (p.stride == 2 && mode != CONV_FWD)) return false;
+    if (p.C % 16 || p.K % 16 || p.C > 64 || p.K > 64) return false;
+    if (((uintptr_t)p.act | (uintptr_t)p.wgt | (uintptr_t)p.out | (uintptr_t)p.add) & 15) return false;
+    g.ca = mode == CONV_FWD ? p.C : p.K; g.ncol = mode == CONV_FWD ? p.K : p.C;
+    const int pad = p.ksz / 2;
+    g.Hp = p.H + pad; g.Wp = p.W + pad;
+    if (g.Hp < 2 || g.Wp < 2 || g.Wp > 4096) return false;
+    const long long total = (long long)p.N * g.Hp * g.Wp;
+    const int halo = pad * g.Wp + pad;
+    if ((total + 512 + 2 * halo) * std::max(g.Hp, g.Wp) >= (1ll << 32) || total >= (1ll << 30)) return false;   // exact division by multiplication
+    g.total = (int)total;
+    const int apitch = g.ca * 2 + 16, groups = g.ca / 8;
+    const int wrows = mode == CONV_FWD ? g.ncol : g.ca, wcols = mode == CONV_FWD ? g.ca : g.ncol;
+    const size_t wbytes = (size_t)p.ksz * p.ksz * wrows * (wcols * 2 + 16);
+    // 256-position tiles when that still gives every SM work and the window fits the copy slots, else 128
+    g.mbw = total >= 256ll * 148 ? 2 : 1;
+    if (g.mbw == 2 && ((256 + 2 * halo) * groups > MMA_SLOTS * MMA_THREADS || g.ncol > 32)) g.mbw = 1;
+    const int tile = 128 * g.mbw, win_rows = tile + 2 * halo;
+    if (win_rows * groups > MMA_SLOTS * MMA_THREADS || win_rows > 65535) return false;
+    g.tiles = (int)((total + tile - 1) / tile);
+    const size_t stage = (size_t)((win_rows * apitch + 127) & ~127);
+    g.stages = 4; while (g.stages > 2 && g.stages * stage + wbytes + 64 > 100 * 1024) --g.stages;
+    g.smem = g.stages * stage + wbytes + 64;
+    g.variant = mma_variant(g.stages, g.mbw, p.ksz, mode == CONV_DGRAD ? 1 : 0, g.ncol / 8);
+    return g.smem <= 200 * 1024;
+}
+
+bool conv_mma_supported(const ConvProb& p, int mode) { MmaGeom g; return mma_geometry(p, mode, g); }
+int conv_mma_pick_variant(const ConvProb& p, int mode) { MmaGeom g; return mma_geometry(p, mode, g) ? g.variant : 0; }
+size_t conv_mma_prob_bytes() { return sizeof(MmaProb); }
+
+bool conv_mma_fill(const ConvProb& p, int mode, void* host) {
+    MmaGeom g; if (!mma_geometry(p, mode, g)) return false;
+    MmaProb t; memset(&t, 0, sizeof(t));
+    t.act = (const __nv_bfloat16*)p.act; t.wgt = (const __nv_bfloat16*)p.wgt; t.add = (const __nv_bfloat16*)p.add; t.out = (__nv_bfloat16*)p.out;
+    t.ca = g.ca; t.ncol = g.ncol; t.wC = p.C; t.H = p.H; t.W = p.W; t.Hp = g.Hp; t.Wp = g.Wp;
+    t.inv_wp = (unsigned)((1ull << 32) / (unsigned)g.Wp + 1); t.inv_hp = (unsigned)((1ull << 32) / (unsigned)g.Hp + 1);
+    t.total = g.total; t.tiles = g.tiles; t.os = mode == CONV_FWD ? p.stride : 1; t.P = p.P; t.Q = p.Q;
+    t.stages = g.stages; t.variant = g.variant; t.scale = p.scale;
+    memcpy(host, &t, sizeof(t));
+    return true;
+}
+int conv_mma_tiles(const void* h) { return ((const MmaProb*)h)->tiles; }
+int conv_mma_variant(const void* h) { return ((const MmaProb*)h)->variant; }
+size_t conv_mma_smem(const void* h) {
+    const MmaProb* t = (const MmaProb*)h;
+    const int v = t->variant, trans = (v >> 4) & 1, ksz = (v >> 5) & 3, mbw = (v >> 7) & 3;
+    const int pad = ksz / 2, halo = pad * t->Wp + pad, win_rows = 128 * mbw + 2 * halo, apitch = t->ca * 2 + 16;
+    const int wrows = trans ? t->ca : t->ncol, wcols = trans ? t->ncol : t->ca;
+    return (size_t)t->stages * ((win_rows * apitch + 127) & ~127) + (size_t)ksz * ksz * wrows * (wcols * 2 + 16) + 64;
+}
+
+template <int NB, int MBW, int KSZ, bool TRANS>
+static void launch_mma_inst(const void* d, dim3 grid, size_t smem, cudaStream_t s) {
+    static bool configured = false;
+    if (!configured) { cudaFuncSetAttribute(conv_mma_kernel<NB, MBW, KSZ, TRANS>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024); configured = true; }
+    conv_mma_kernel<NB, MBW, KSZ, TRANS><<<grid, MMA_THREADS, smem, s>>>((const MmaProb*)d);
+}
+template <int NB, int MBW>
+static void launch_mma_nb(const void* d, dim3 grid, size_t smem, int ksz, int trans, cudaStream_t s) {
+    if (ksz == 3) { if (trans) launch_mma_inst<NB, MBW, 3, true>(d, grid, smem, s); else launch_mma_inst<NB, MBW, 3, false>(d, grid, smem, s); }
+    else { if (trans) launch_mma_inst<NB, MBW, 1, true>(d, grid, smem, s); else launch_mma_inst<NB, MBW, 1, false>(d, grid, smem, s); }
+}
+// all problems of one launch share the variant
+void launch_conv_mma_probs(const void* d, int nprob, int max_tiles, size_t max_smem, int variant, cudaStream_t s) {
+    static int sms = 0;
+    if (!sms) { int dev = 0; cudaGetDevice(&dev); cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev); if (sms < 1) sms = 148; }
+    const int nb = variant & 15, trans = (variant >> 4) & 1, ksz = (variant >> 5) & 3, mbw = (variant >> 7) & 3;
+    // persistent CTAs: as many as fit on the chip at this shared-memory footprint (at most 4 per SM), over all problems
+    int per_sm = (int)((220 * 1024) / (max_smem + 1024)); if (per_sm > 4) per_sm = 4; if (per_sm < 1) per_sm = 1;
+    int gx = (per_sm * sms + nprob - 1) / nprob; if (gx > max_tiles) gx = max_tiles; if (gx < 1) gx = 1;
+    const dim3 grid(gx, nprob);
+    if (mbw == 2) {
+        if (nb == 2) launch_mma_nb<2, 2>(d, grid, max_smem, ksz, trans, s);
+        else if (nb == 4) launch_mma_nb<4, 2>(d, grid, max_smem, ksz, trans, s);
+    } else {
+        if (nb == 2) launch_mma_nb<2, 1>(d, grid, max_smem, ksz, trans, s);
+        else if (nb == 4) launch_mma_nb<4, 1>(d, grid, max_smem, ksz, trans, s);
+        else if (nb == 6) launch_mma_nb<6, 1>(d, grid, max_smem, ksz, trans, s);
+        else if (nb == 8) launch_mma_nb<8, 1>(d, grid, max_smem, ksz, trans, s);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------ wgrad
+// dw[k][t][c] = sum over positions of dy[pos][k] * a[pos + shift_t][c].  GEMM with M = output channels, N = (tap,
+// input channel), reduction over the padded-flat positions, 128 per staging step.  A CTA owns a group of taps and
+// a range of pixel tiles; each warp owns some 8-wide N blocks for ALL M blocks (so that one ldmatrix of the shifted
+// activations feeds MB MMAs) and keeps its accumulators in registers over the whole range; the CTA then writes an
+// fp32 partial and a second kernel adds the partials in a fixed order.
+struct alignas(16) MmaWgradProb {
+    const __nv_bfloat16* dy;    // [n_img,H,W,K]  (stride 1; a stride-2 layer passes the zero-stuffed dy)
+    const __nv_bfloat16* a;     // [n_img,H,W,C]
+    float* partial;             // [splits][taps][K][C]
+    float* out;                 // [K][taps][C]
+    int K, C, H, W, Wp, pad, ksz, taps, flat;
+    int n_img, tiles_per_img, pixel_tiles;
+    int box_w, box_h, act_rows;
+    int tap_groups, taps_per_group, splits, tiles_per_split;
+};
+
+template <int MB>   // MB = K / 16
+__global__ void __launch_bounds__(MMA_THREADS) conv_wgrad_mma_kernel(const MmaWgradProb* __restrict__ probs) {
+    constexpr int NBW = 16 / MB;                                  // N blocks a warp may own
+    __shared__ MmaWgradProb p;
+    if (threadIdx.x < sizeof(MmaWgradProb) / 4) reinterpret_cast<uint32_t*>(&p)[threadIdx.x] = reinterpret_cast<const uint32_t*>(probs + blockIdx.y)[threadIdx.x];
+    __syncthreads();
+    if ((int)blockIdx.x >= p.tap_groups * p.splits) return;
+    const int split = blockIdx.x % p.splits, tg = blockIdx.x / p.splits;
+    const int tap0 = tg * p.taps_per_group; int ntap = p.taps - tap0; if (ntap > p.taps_per_group) ntap = p.taps_per_group;
+    const int t_begin = split * p.tiles_per_split; int t_end = t_begin + p.tiles_per_split; if (t_end > p.pixel_tiles) t_end = p.pixel_tiles;
+    extern __shared__ __align__(16) uint8_t sm[];
+    const int K = p.K, C = p.C, dpitch = K * 2 + 16, apitch = C * 2 + 16;
+    uint8_t* s_dy = sm; uint8_t* s_a = sm + 128 * dpitch;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int nbc = C / 8, nblocks = ntap * nbc;                  // N blocks of this CTA: (tap, 8 channels)
+    float acc[NBW][MB][4];
+#pragma unroll
+    for (int b = 0; b < NBW; ++b)
+#pragma unroll
+        for (int m = 0; m < MB; ++m) { acc[b][m][0] = acc[b][m][1] = acc[b][m][2] = acc[b][m][3] = 0.f; }
+    const uint32_t dy_base = s_u32(s_dy), a_base = s_u32(s_a);
+    const int ksz = p.ksz;
+
+    for (int t = t_begin; t < t_end; ++t) {
+        const int img = t / p.tiles_per_img, pos0 = (t % p.tiles_per_img) * 128;
+        const int row0 = p.flat ? 0 : pos0 / p.Wp, a_off = p.flat ? 0 : pos0 - row0 * p.Wp;
+        __syncthreads();                                          // the previous tile has been consumed
+        {   // dy at the 128 positions; pad positions and rows past the image are zeros: they add nothing
+            const int groups = K / 8, total = 128 * groups;
+            for (int id = tid; id < total; id += MMA_THREADS) {
+                const int g = id % groups, m = id / groups;
+                uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                long long pix = -1;
+                if (p.flat) { const long long gp = (long long)pos0 + m; if (gp < (long long)p.W) pix = gp; }
+                else { const int pos = pos0 + m, i = pos / p.Wp, j = pos - i * p.Wp; if (i < p.H && j < p.W) pix = ((long long)img * p.H + i) * p.W + j; }
+                if (pix >= 0) v = __ldg(reinterpret_cast<const uint4*>(p.dy + pix * K + g * 8));
+                *reinterpret_cast<uint4*>(s_dy + m * dpitch + g * 16) = v;
+            }
+        }
+        {   // activation window with its halo
+            const int groups = C / 8, total = p.act_rows * groups, boxpx = p.box_w * p.box_h;
+            const int x0 = p.flat ? pos0 : -p.pad, y0 = p.flat ? 0 : row0 - p.pad;
+            for (int id = tid; id < total; id += MMA_THREADS) {
+                const int g = id % groups, px = id / groups;
+                uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                if (px < boxpx) {
+                    const int x = px % p.box_w, y = px / p.box_w, gy = y0 + y, gx = x0 + x;
+                    if (gy >= 0 && gy < p.H && gx >= 0 && gx < p.W)
+                        v = __ldg(reinterpret_cast<const uint4*>(p.a + (((long long)img * p.H + gy) * p.W + gx) * C + g * 8));
+                }
+                *reinterpret_cast<uint4*>(s_a + px * apitch + g * 16) = v;
+            }
+        }
+        __syncthreads();
+        for (int kk = 0; kk < 128; kk += 16) {
+            uint32_t af[MB][4];
+#pragma unroll
+            for (int m = 0; m < MB; ++m)       // A = dy^T: stored [pos][k], transposed on load
+                ldsm_x4_t(dy_base + (uint32_t)(kk + (lane & 7) + ((lane >> 4) & 1) * 8) * dpitch + (m * 16 + ((lane >> 3) & 1) * 8) * 2,
+                          af[m][0], af[m][1], af[m][2], af[m][3]);
+#pragma unroll
+            for (int b = 0; b < NBW; ++b) {
+                const int nb = warp + 8 * b;
+                if (nb < nblocks) {
+                    const int tt = nb / nbc, nj = nb % nbc, tp = tap0 + tt, r = tp / ksz, q = tp % ksz;
+                    uint32_t b0, b1;
+                    ldsm_x2_t(a_base + (uint32_t)(a_off + r * p.Wp + q + kk + (lane & 15)) * apitch + nj * 16, b0, b1);
+#pragma unroll
+                    for (int m = 0; m < MB; ++m) mma16816(acc[b][m], af[m][0], af[m][1], af[m][2], af[m][3], b0, b1);
+                }
+            }
+        }
+    }
+    // ---- partial sums: thread (g, t4) holds (m = 16*mi + g [+8], n = 8*nj + 2*t4 [+1])
+    const int g = lane >> 2, t4 = lane & 3;
+#pragma unroll
+    for (int b = 0; b < NBW; ++b) {
+        const int nb = warp + 8 * b;
+        if (nb >= nblocks) continue;
+        const int tt = nb / nbc, nj = nb % nbc;
+#pragma unroll
+        for (int m = 0; m < MB; ++m)
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                const int k = m * 16 + g + half * 8;
+                float* dst = p.partial + (((long long)split * p.taps + tap0 + tt) * K + k) * C + nj * 8 + t4 * 2;
+                *reinterpret_cast<float2*>(dst) = make_float2(acc[b][m][half * 2], acc[b][m][half * 2 + 1]);
+            }
+    }
+}
+
+// out[k][t][c] = sum over splits (ascending) of partial[split][t][k][c]
+__global__ void __launch_bounds__(256) wgrad_mma_reduce_kernel(const MmaWgradProb* __restrict__ probs) {
+    const MmaWgradProb& p = probs[blockIdx.y];
+    const long long n = (long long)p.taps * p.K * p.C;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+        const int c = (int)(i % p.C); const long long r = i / p.C; const int t = (int)(r % p.taps); const int k = (int)(r / p.taps);
+        const long long src = ((long long)t * p.K + k) * p.C + c;
+        float s = 0.f;
+        for (int sp = 0; sp < p.splits; ++sp) s += p.partial[(long long)sp * n + src];
+        p.out[i] = s;
+    }
+}
+
+struct MmaWgGeom { int flat, n_img, H, W, Wp, box_w, box_h, act_rows, tiles_per_img, pixel_tiles, tap_groups, taps_per_group, splits, tiles_per_split; size_t smem, partial_bytes; };
+
+static bool mma_wg_geometry(const ConvProb& p, int target_ctas, MmaWgGeom& g) {
+    if (p.stride != 1 || (p.ksz != 1 && p.ksz != 3)) return false;
+    if (p.C % 16 || p.K % 16 || p.C > 64 || p.K > 64) return false;
+    if (((uintptr_t)p.act | (uintptr_t)p.wgt) & 15) return false;
+    const int taps = p.ksz * p.ksz, pad2 = p.ksz - 1;
+    g.flat = p.ksz == 1;
+    if (g.flat) { g.n_img = 1; g.H = 1; g.W = p.N * p.H * p.W; g.Wp = g.W; g.box_w = 128; g.box_h = 1; g.tiles_per_img = (int)(((long long)g.W + 127) / 128); }
+    else { g.n_img = p.N; g.H = p.H; g.W = p.W; g.Wp = p.W + pad2; if (g.Wp > 128) return false;
+        const int rows = (g.Wp - 1 + 127) / g.Wp + 1;
+        g.box_w = g.Wp; g.box_h = rows + pad2; g.tiles_per_img = (p.H * g.Wp + 127) / 128; }
+    const int max_read = (g.flat ? 0 : g.Wp - 1) + pad2 * g.Wp + pad2 + 128;
+    g.act_rows = std::max(g.box_w * g.box_h, max_read);
+    g.pixel_tiles = g.n_img * g.tiles_per_img;
+    const int MB = p.K / 16, nbw = 16 / MB, nbc = p.C / 8;
+    g.taps_per_group = std::max(1, std::min(taps, (8 * nbw) / nbc));
+    g.tap_groups = (taps + g.taps_per_group - 1) / g.taps_per_group;
+    g.smem = (size_t)128 * (p.K * 2 + 16) + (size_t)g.act_rows * (p.C * 2 + 16) + 64;
+    if (g.smem > 200 * 1024) return false;
+    int want = std::max(1, target_ctas / g.tap_groups); if (want > g.pixel_tiles) want = g.pixel_tiles; if (want > 512) want = 512;
+    g.tiles_per_split = (g.pixel_tiles + want - 1) / want; g.splits = (g.pixel_tiles + g.tiles_per_split - 1) / g.tiles_per_split;
+    g.partial_bytes = (size_t)g.splits * taps * p.K * p.C * 4;
+    return true;
+}
+bool conv_wgrad_mma_supported(const ConvProb& p, int target_ctas, size_t* partial_bytes) {
+    MmaWgGeom g; if (!mma_wg_geometry(p, target_ctas, g)) return false;
+    if (partial_bytes) *partial_bytes = g.partial_bytes;
+    return true;
+}
+// p.act = a, p.wgt = dy, p.out = dw (fp32), p.partial = workspace
+bool conv_wgrad_mma_fill(const ConvProb& p, int target_ctas, void* host) {
+    MmaWgGeom g; if (!mma_wg_geometry(p, target_ctas, g)) return false;
+    MmaWgradProb t; memset(&t, 0, sizeof(t));
+    t.dy = (const __nv_bfloat16*)p.wgt; t.a = (const __nv_bfloat16*)p.act; t.partial = p.partial; t.out = (float*)p.out;
+    t.K = p.K; t.C = p.C; t.H = g.H; t.W = g.W; t.Wp = g.Wp; t.pad = p.ksz / 2; t.ksz = p.ksz; t.taps = p.ksz * p.ksz; t.flat = g.flat;
+    t.n_img = g.n_img; t.tiles_per_img = g.tiles_per_img; t.pixel_tiles = g.pixel_tiles; t.box_w = g.box_w; t.box_h = g.box_h; t.act_rows = g.act_rows;
+    t.tap_groups = g.tap_groups; t.taps_per_group = g.taps_per_group; t.splits = g.splits; t.tiles_per_split = g.tiles_per_split;
+    memcpy(host, &t, sizeof(t));
+    return true;
+}
+size_t conv_wgrad_mma_prob_bytes() { return sizeof(MmaWgradProb); }
+int conv_wgrad_mma_ctas(const void* h) { const MmaWgradProb* t = (const MmaWgradProb*)h; return t->tap_groups * t->splits; }
+size_t conv_wgrad_mma_smem(const void* h) { const MmaWgradProb* t = (const MmaWgradProb*)h; return (size_t)128 * (t->K * 2 + 16) + (size_t)t->act_rows * (t->C * 2 + 16) + 64; }
+long long conv_wgrad_mma_out_elems(const void* h) { const MmaWgradProb* t = (const MmaWgradProb*)h; return (long long)t->taps * t->K * t->C; }
+int conv_wgrad_mma_k(const void* h) { return ((const MmaWgradProb*)h)->K; }
+
+// all problems of one launch must have the same number of output channels K
+void launch_conv_wgrad_mma_probs(const void* d, int nprob, int max_ctas, size_t max_smem, long long max_out, int K, cudaStream_t s) {
+    static bool configured = false;
+    if (!configured) {
+        cudaFuncSetAttribute(conv_wgrad_mma_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        cudaFuncSetAttribute(conv_wgrad_mma_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        cudaFuncSetAttribute(conv_wgrad_mma_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        cudaFuncSetAttribute(conv_wgrad_mma_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        configured = true;
+    }
+    const dim3 grid(max_ctas, nprob);
+    switch (K / 16) {
+        case 1: conv_wgrad_mma_kernel<1><<<grid, MMA_THREADS, max_smem, s>>>((const MmaWgradProb*)d); break;
+        case 2: conv_wgrad_mma_kernel<2><<<grid, MMA_THREADS, max_smem, s>>>((const MmaWgradProb*)d); break;
+        case 3: conv_wgrad_mma_kernel<3><<<grid, MMA_THREADS, max_smem, s>>>((const MmaWgradProb*)d); break;
+        case 4: conv_wgrad_mma_kernel<4><<<grid, MMA_THREADS, max_smem, s>>>((const MmaWgradProb*)d); break;
+        default: return;
+    }
+    long long gx = (max_out + 255) / 256; if (gx > 592) gx = 592; if (gx < 1) gx = 1;
+    wgrad_mma_reduce_kernel<<<dim3((unsigned)gx, nprob), 256, 0, s>>>((const MmaWgradProb*)d);
+}
+
+}  // namespace resist

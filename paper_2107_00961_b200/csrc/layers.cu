@@ -20,6 +20,20 @@ int conv_wgrad_tc_ctas(const void* h);
 size_t conv_wgrad_tc_smem(const void* h);
 long long conv_wgrad_tc_out_elems(const void* h);
 void launch_conv_wgrad_tc_probs(const void* d_tc, int nprob, int max_ctas, size_t max_smem, long long max_out, cudaStream_t s);
+bool conv_mma_supported(const ConvProb& p, int mode);
+bool conv_mma_fill(const ConvProb& p, int mode, void* host);
+size_t conv_mma_prob_bytes();
+int conv_mma_tiles(const void* h);
+size_t conv_mma_smem(const void* h);
+void launch_conv_mma_probs(const void* d, int nprob, int max_tiles, size_t max_smem, int variant, cudaStream_t s);
+int conv_mma_pick_variant(const ConvProb& p, int mode);
+bool conv_wgrad_mma_supported(const ConvProb& p, int target_ctas, size_t* partial_bytes);
+bool conv_wgrad_mma_fill(const ConvProb& p, int target_ctas, void* host);
+size_t conv_wgrad_mma_prob_bytes();
+int conv_wgrad_mma_ctas(const void* h);
+size_t conv_wgrad_mma_smem(const void* h);
+long long conv_wgrad_mma_out_elems(const void* h);
+void launch_conv_wgrad_mma_probs(const void* d, int nprob, int max_ctas, size_t max_smem, long long max_out, int K, cudaStream_t s);
 }
 using namespace resist;
 
@@ -46,13 +60,27 @@ extern "C" int resist_conv2d(int32_t mode, int32_t dtype, int32_t backend, const
     p.tiles_m = (p.M + 63) / 64; p.tiles_n = (p.Ncol + 63) / 64; p.splits = 1;
     const int ktiles = (p.Kred + 15) / 16; p.ktiles_per_split = ktiles;
     int sm = 148; int dev = 0; cudaGetDevice(&dev); cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev);
+    // which kernel family: 0 CUDA cores, 1 tcgen05, 2 warp-level MMA
+    auto pick = [&](const ConvProb& q, size_t* pb) -> int {
+        if (dtype != RESIST_BF16 || backend == RESIST_CONV_CUDA_CORES) return 0;
+        const bool want_mma = backend == RESIST_CONV_AUTO || backend == RESIST_CONV_WARP_MMA;
+        const bool want_tc = backend == RESIST_CONV_AUTO || backend == RESIST_CONV_TCGEN05;
+        if (mode == CONV_WGRAD) {
+            if (want_mma && conv_wgrad_mma_supported(q, 2 * sm, pb)) return 2;
+            if (want_tc && conv_wgrad_tc_supported(q, 2 * sm, pb)) return 1;
+            return 0;
+        }
+        if (want_mma && conv_mma_supported(q, mode)) return 2;
+        if (want_tc && conv_tc_supported(q, mode)) return 1;
+        return 0;
+    };
     // backward of a stride-2 layer on tensor cores: stride-1 problem on a zero-stuffed dy
     char* up = nullptr;
-    if (dtype == RESIST_BF16 && backend == RESIST_CONV_AUTO && stride == 2 && mode != CONV_FWD && K % 8 == 0) {
+    if (stride == 2 && mode != CONV_FWD && K % 8 == 0) {
         ConvProb q = p; q.stride = 1; q.P = H; q.Q = W;
         if (mode == CONV_DGRAD) q.M = (int)rows_in; else q.Kred = (int)rows_in;
         size_t pb = 0;
-        if (mode == CONV_DGRAD ? conv_tc_supported(q, mode) : conv_wgrad_tc_supported(q, 2 * sm, &pb)) {
+        if (pick(q, &pb) != 0) {
             if (cudaMalloc(&up, (size_t)N * H * W * K * 2 + 256) != cudaSuccess) { g_layer_error = "cudaMalloc failed"; return RESIST_ENOMEM; }
             UpProb u{mode == CONV_DGRAD ? p.act : p.wgt, up + 256, N, H, W, K, p.P, p.Q};
             cudaMemcpyAsync(up, &u, sizeof(u), cudaMemcpyHostToDevice, st);
@@ -62,15 +90,14 @@ extern "C" int resist_conv2d(int32_t mode, int32_t dtype, int32_t backend, const
         }
     }
     size_t wg_partial = 0;
-    const bool tc = dtype == RESIST_BF16 && backend == RESIST_CONV_AUTO &&
-                    (mode == CONV_WGRAD ? conv_wgrad_tc_supported(p, 2 * sm, &wg_partial) : conv_tc_supported(p, mode));
-    if (used_backend) *used_backend = tc ? 1 : 0;
+    const int be = pick(p, &wg_partial);
+    if (used_backend) *used_backend = be;
     size_t scratch = 0;
-    std::vector<char> host_tc;
-    if (tc && mode == CONV_WGRAD) { host_tc.resize(conv_wgrad_tc_prob_bytes()); scratch = 1024 + wg_partial; }
-    else if (tc) { host_tc.resize(conv_tc_prob_bytes()); scratch = host_tc.size();
-        if (!conv_tc_fill(p, mode, host_tc.data())) { g_layer_error = "tensor map encoding failed"; return RESIST_ECUDA; } }
-    else if (mode == CONV_WGRAD) {
+    std::vector<char> hd;                                      // host copy of the kernel family's own descriptor
+    if (be == 1) hd.resize(mode == CONV_WGRAD ? conv_wgrad_tc_prob_bytes() : conv_tc_prob_bytes());
+    if (be == 2) hd.resize(mode == CONV_WGRAD ? conv_wgrad_mma_prob_bytes() : conv_mma_prob_bytes());
+    if (be && mode == CONV_WGRAD) scratch = 1024 + wg_partial; else if (be) scratch = 1024;
+    if (!be && mode == CONV_WGRAD) {
         const int tiles = p.tiles_m * p.tiles_n;
         int want = (2 * sm + tiles - 1) / tiles; want = std::max(1, std::min(std::min(want, 64), ktiles));
         p.ktiles_per_split = (ktiles + want - 1) / want; p.splits = (ktiles + p.ktiles_per_split - 1) / p.ktiles_per_split;
@@ -78,16 +105,20 @@ extern "C" int resist_conv2d(int32_t mode, int32_t dtype, int32_t backend, const
     }
     char* blob = nullptr;
     cudaError_t e = cudaMalloc(&blob, 1024 + scratch);
-    if (e != cudaSuccess) { g_layer_error = cudaGetErrorString(e); return RESIST_ENOMEM; }
-    if (!tc && p.splits > 1) p.partial = (float*)(blob + 1024);
-    if (tc && mode == CONV_WGRAD) { p.partial = (float*)(blob + 2048);
-        if (!conv_wgrad_tc_fill(p, 2 * sm, host_tc.data())) { cudaFree(blob); g_layer_error = "tensor map encoding failed"; return RESIST_ECUDA; } }
+    if (e != cudaSuccess) { cudaFree(up); g_layer_error = cudaGetErrorString(e); return RESIST_ENOMEM; }
+    if (!be && p.splits > 1) p.partial = (float*)(blob + 1024);
+    if (be && mode == CONV_WGRAD) p.partial = (float*)(blob + 2048);
+    bool filled = true;
+    if (be == 1) filled = mode == CONV_WGRAD ? conv_wgrad_tc_fill(p, 2 * sm, hd.data()) : conv_tc_fill(p, mode, hd.data());
+    if (be == 2) filled = mode == CONV_WGRAD ? conv_wgrad_mma_fill(p, 2 * sm, hd.data()) : conv_mma_fill(p, mode, hd.data());
+    if (!filled) { cudaFree(blob); cudaFree(up); g_layer_error = "descriptor set-up failed"; return RESIST_ECUDA; }
     e = cudaMemcpyAsync(blob, &p, sizeof(p), cudaMemcpyHostToDevice, st);
-    if (e == cudaSuccess && tc) e = cudaMemcpyAsync(blob + 1024, host_tc.data(), host_tc.size(), cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess && be) e = cudaMemcpyAsync(blob + 1024, hd.data(), hd.size(), cudaMemcpyHostToDevice, st);
     if (e == cudaSuccess) {
-        if (tc && mode == CONV_WGRAD) launch_conv_wgrad_tc_probs(blob + 1024, 1, conv_wgrad_tc_ctas(host_tc.data()), conv_wgrad_tc_smem(host_tc.data()),
-                                                                 conv_wgrad_tc_out_elems(host_tc.data()), st);
-        else if (tc) launch_conv_tc_probs(blob + 1024, 1, conv_tc_tiles(host_tc.data()), conv_tc_smem(host_tc.data()), st);
+        if (be == 1 && mode == CONV_WGRAD) launch_conv_wgrad_tc_probs(blob + 1024, 1, conv_wgrad_tc_ctas(hd.data()), conv_wgrad_tc_smem(hd.data()), conv_wgrad_tc_out_elems(hd.data()), st);
+        else if (be == 1) launch_conv_tc_probs(blob + 1024, 1, conv_tc_tiles(hd.data()), conv_tc_smem(hd.data()), st);
+        else if (be == 2 && mode == CONV_WGRAD) launch_conv_wgrad_mma_probs(blob + 1024, 1, conv_wgrad_mma_ctas(hd.data()), conv_wgrad_mma_smem(hd.data()), conv_wgrad_mma_out_elems(hd.data()), p.K, st);
+        else if (be == 2) launch_conv_mma_probs(blob + 1024, 1, conv_mma_tiles(hd.data()), conv_mma_smem(hd.data()), conv_mma_pick_variant(p, mode), st);
         else {
             launch_conv_ref((ConvProb*)blob, 1, p.tiles_m * p.tiles_n * p.splits, mode, dtype == RESIST_BF16, st);
             if (mode == CONV_WGRAD && p.splits > 1) launch_splitk_reduce((ConvProb*)blob, 1, p.M * p.Ncol, st);
@@ -97,7 +128,7 @@ extern "C" int resist_conv2d(int32_t mode, int32_t dtype, int32_t backend, const
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
     cudaFree(blob); cudaFree(up);
     if (e != cudaSuccess) { g_layer_error = cudaGetErrorString(e); return RESIST_ECUDA; }
-    if (tc) { const int stv = conv_tc_read_status();
+    if (be == 1) { const int stv = conv_tc_read_status();
         if (stv) { g_layer_error = "a bounded device-side wait gave up (code " + std::to_string(stv) + ")"; return RESIST_ETIMEOUT; } }
     return RESIST_OK;
 }

@@ -28,6 +28,35 @@ size_t conv_wgrad_tc_smem(const void* h);
 long long conv_wgrad_tc_out_elems(const void* h);
 void launch_conv_wgrad_tc_probs(const void* d_tc, int nprob, int max_ctas, size_t max_smem, long long max_out, cudaStream_t s);
 static int wgrad_target_ctas(const resist_ctx* ctx) { return std::max(8, 2 * ctx->sm_count / std::max(1, ctx->S)); }
+bool conv_mma_supported(const ConvProb& p, int mode);                                   // conv_mma.cu
+bool conv_mma_fill(const ConvProb& p, int mode, void* host);
+size_t conv_mma_prob_bytes();
+int conv_mma_tiles(const void* h);
+size_t conv_mma_smem(const void* h);
+void launch_conv_mma_probs(const void* d, int nprob, int max_tiles, size_t max_smem, int variant, cudaStream_t s);
+int conv_mma_pick_variant(const ConvProb& p, int mode);
+bool conv_wgrad_mma_supported(const ConvProb& p, int target_ctas, size_t* partial_bytes);
+bool conv_wgrad_mma_fill(const ConvProb& p, int target_ctas, void* host);
+size_t conv_wgrad_mma_prob_bytes();
+int conv_wgrad_mma_ctas(const void* h);
+size_t conv_wgrad_mma_smem(const void* h);
+long long conv_wgrad_mma_out_elems(const void* h);
+void launch_conv_wgrad_mma_probs(const void* d, int nprob, int max_ctas, size_t max_smem, long long max_out, int K, cudaStream_t s);
+
+// Which kernel family takes a bf16 convolution: 0 = CUDA cores, 1 = tcgen05, >= 200 = warp-level MMA (wgrad: 200 +
+// output channels; forward and dgrad: 1000 + the kernel variant, so that the value also separates launches by what
+// the kernel is specialised on).
+static int pick_backend(const ConvProb& p, int mode, int target_ctas, size_t* partial_bytes, int pref = RESIST_CONV_AUTO) {
+    const bool want_mma = pref == RESIST_CONV_AUTO || pref == RESIST_CONV_WARP_MMA, want_tc = pref == RESIST_CONV_AUTO || pref == RESIST_CONV_TCGEN05;
+    if (mode == CONV_WGRAD) {
+        if (pref == RESIST_CONV_WARP_MMA && conv_wgrad_mma_supported(p, target_ctas, partial_bytes)) return 200 + p.K;
+        if (want_tc && conv_wgrad_tc_supported(p, target_ctas, partial_bytes)) return 1;
+        return 0;
+    }
+    if (want_mma && conv_mma_supported(p, mode)) return 1000 + conv_mma_pick_variant(p, mode);
+    if (want_tc && conv_tc_supported(p, mode)) return 1;
+    return 0;
+}
 
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 static int out_dim(int h, int k, int stride) { return (h + 2 * ((k - 1) / 2) - k) / stride + 1; }
@@ -97,7 +126,8 @@ struct Builder {
         p.tiles_m = (p.M + 63) / 64; p.tiles_n = (p.Ncol + 63) / 64; p.splits = 1;
         const int ktiles = (p.Kred + 15) / 16; p.ktiles_per_split = ktiles;
         flops += 2LL * rows_out * p.K * p.ksz * p.ksz * p.C;
-        const bool tc_ok = ctx->opts.dtype == RESIST_BF16 && ctx->opts.conv_backend == RESIST_CONV_AUTO;
+        const bool tc_ok = ctx->opts.dtype == RESIST_BF16 && ctx->opts.conv_backend != RESIST_CONV_CUDA_CORES;
+        const int pref = ctx->opts.conv_backend;
         if (tc_ok && p.stride == 2 && mode != CONV_FWD && !patch && p.K % 8 == 0) {
             // backward of a stride-2 layer: a stride-1 problem on dy zero-stuffed to the input resolution
             ConvProb q = p; q.stride = 1; q.P = p.H; q.Q = p.W;
@@ -105,7 +135,7 @@ struct Builder {
             if (mode == CONV_DGRAD) { q.act = up_buf; q.M = (int)rows_in; }
             else { q.wgt = up_buf; q.Kred = (int)rows_in; }
             size_t pb = 0;
-            const bool ok = mode == CONV_DGRAD ? conv_tc_supported(q, mode) : conv_wgrad_tc_supported(q, wgrad_target_ctas(ctx), &pb);
+            const bool ok = pick_backend(q, mode, wgrad_target_ctas(ctx), &pb, pref) != 0;
             if (ok) {
                 up_need = std::max(up_need, up_bytes);
                 if (up_src != dy_or_null) {                  // first use of this dy: stuff it
@@ -119,9 +149,9 @@ struct Builder {
         }
         if (mode == CONV_WGRAD) {
             size_t pb = 0;
-            op.backend = (tc_ok && !patch && conv_wgrad_tc_supported(p, wgrad_target_ctas(ctx), &pb)) ? 1 : 0;
+            op.backend = (tc_ok && !patch) ? pick_backend(p, mode, wgrad_target_ctas(ctx), &pb, pref) : 0;
             if (op.backend) { wgrad_partial_need = std::max(wgrad_partial_need, pb); p.partial = wgrad_partial; }
-        } else op.backend = (tc_ok && conv_tc_supported(p, mode)) ? 1 : 0;
+        } else op.backend = tc_ok ? pick_backend(p, mode, 0, nullptr, pref) : 0;
         if (op.backend) ++n_tc; else ++n_cc;
         if (mode == CONV_WGRAD && !op.backend) {
             const int tiles = p.tiles_m * p.tiles_n;
@@ -330,11 +360,14 @@ static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool s
     // convolution that reads its output and sorts in front of it
     std::stable_sort(ops.begin(), ops.end(), [](const Op& a, const Op& b) {
         if (a.key != b.key) return a.key < b.key;
-        return (a.kind == OP_UPSAMPLE) > (b.kind == OP_UPSAMPLE); });
+        if ((a.kind == OP_UPSAMPLE) != (b.kind == OP_UPSAMPLE)) return a.kind == OP_UPSAMPLE;
+        return a.backend < b.backend; });
     const double es = ctx->opts.dtype == RESIST_BF16 ? 2.0 : 4.0;
     std::vector<ConvProb> conv; std::vector<BnProb> bn; std::vector<PoolProb> pool; std::vector<HeadProb> head; std::vector<UpProb> up;
     const size_t tcb = conv_tc_prob_bytes(); std::vector<char> tc; int n_tc = 0;
     const size_t wtcb = conv_wgrad_tc_prob_bytes(); std::vector<char> wtc; int n_wtc = 0;
+    const size_t mmb = conv_mma_prob_bytes(); std::vector<char> mm; int n_mm = 0;
+    const size_t wmmb = conv_wgrad_mma_prob_bytes(); std::vector<char> wmm; int n_wmm = 0;
     struct HostSite { int arr; int idx; int field; int what; int sub; };
     std::vector<HostSite> sites;
     plan.launches.clear();
@@ -346,6 +379,29 @@ static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool s
             const Op& o = ops[k]; const int slot = single ? 0 : o.sub;
             switch (o.kind) {
                 case OP_CONV_FWD: case OP_CONV_DGRAD: case OP_CONV_WGRAD: case OP_SPLITK: {
+                    if (o.backend >= 200 && o.kind != OP_SPLITK) {   // warp-level MMA kernels: their own descriptor arrays
+                        const ConvProb& p = o.conv;
+                        const double in_e = (double)p.N * p.H * p.W * p.C, out_e = (double)p.N * p.P * p.Q * p.K, w_e = (double)p.K * p.ksz * p.ksz * p.C;
+                        L.flops += 2.0 * out_e * p.ksz * p.ksz * p.C;
+                        if (o.kind == OP_CONV_WGRAD) {
+                            if (k == i) L.first = n_wmm;
+                            wmm.resize((size_t)(n_wmm + 1) * wmmb); char* h = wmm.data() + (size_t)n_wmm * wmmb;
+                            if (!conv_wgrad_mma_fill(o.conv, wgrad_target_ctas(ctx), h)) { ctx->err = "wgrad descriptor failed"; return RESIST_EINVAL; }
+                            L.gx = std::max(L.gx, conv_wgrad_mma_ctas(h));
+                            L.max_elems = std::max<long long>(L.max_elems, (long long)conv_wgrad_mma_smem(h));
+                            L.max_b = (int)std::max<long long>(L.max_b, conv_wgrad_mma_out_elems(h));
+                            ++n_wmm; L.bytes += es * (in_e + out_e) + 4.0 * w_e;
+                        } else {
+                            if (k == i) L.first = n_mm;
+                            mm.resize((size_t)(n_mm + 1) * mmb); char* h = mm.data() + (size_t)n_mm * mmb;
+                            const int mode = o.kind == OP_CONV_FWD ? CONV_FWD : CONV_DGRAD;
+                            if (!conv_mma_fill(o.conv, mode, h)) { ctx->err = "conv descriptor failed"; return RESIST_EINVAL; }
+                            L.gx = std::max(L.gx, conv_mma_tiles(h));
+                            L.max_elems = std::max<long long>(L.max_elems, (long long)conv_mma_smem(h));
+                            ++n_mm; L.bytes += es * (in_e + out_e + w_e + (p.add ? (o.kind == OP_CONV_FWD ? out_e : in_e) : 0.0));
+                        }
+                        break;
+                    }
                     if (o.backend && o.kind == OP_CONV_WGRAD) {  // tensor-core wgrad: its own descriptor array
                         if (k == i) L.first = n_wtc;
                         wtc.resize((size_t)(n_wtc + 1) * wtcb);
@@ -442,6 +498,8 @@ static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool s
     const size_t o_tc = off;   off += align_up(tc.size(), 256);
     const size_t o_wtc = off;  off += align_up(wtc.size(), 256);
     const size_t o_up = off;   off += align_up(up.size() * sizeof(UpProb), 256);
+    const size_t o_mm = off;   off += align_up(mm.size(), 256);
+    const size_t o_wmm = off;  off += align_up(wmm.size(), 256);
     ctx_free(ctx, plan.d_blob);
     plan.d_blob = ctx_alloc(ctx, off + 256); plan.blob_bytes = off;
     if (!plan.d_blob) { ctx->err = "allocator returned NULL for the launch plan"; return RESIST_ENOMEM; }
@@ -471,6 +529,9 @@ static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool s
     plan.d_wtc = base + o_wtc; plan.wtc_stride = wtcb;
     if (!up.empty()) memcpy(host.data() + o_up, up.data(), up.size() * sizeof(UpProb));
     plan.d_up = (UpProb*)(base + o_up);
+    if (!mm.empty()) memcpy(host.data() + o_mm, mm.data(), mm.size());
+    if (!wmm.empty()) memcpy(host.data() + o_wmm, wmm.data(), wmm.size());
+    plan.d_mm = base + o_mm; plan.mm_stride = mmb; plan.d_wmm = base + o_wmm; plan.wmm_stride = wmmb;
     cudaError_t e = cudaMemcpyAsync(plan.d_blob, host.data(), off, cudaMemcpyHostToDevice, st);
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
     if (e != cudaSuccess) { ctx->err = std::string("plan upload: ") + cudaGetErrorString(e); return RESIST_ECUDA; }
@@ -527,9 +588,9 @@ static int run_plan(resist_ctx* ctx, Plan& plan, const PatchArgs& pa, bool updat
     for (const Launch& L : plan.launches) {
         int pk = 0, nk = 1;
         switch (L.kind) {
-            case OP_CONV_FWD: pk = L.backend ? PK_CONV_FWD_TC : PK_CONV_FWD_CC; break;
-            case OP_CONV_DGRAD: pk = L.backend ? PK_CONV_DGRAD_TC : PK_CONV_DGRAD_CC; break;
-            case OP_CONV_WGRAD: pk = L.backend ? PK_CONV_WGRAD_TC : PK_CONV_WGRAD_CC; break;
+            case OP_CONV_FWD: pk = L.backend >= 200 ? PK_CONV_FWD_MMA : L.backend ? PK_CONV_FWD_TC : PK_CONV_FWD_CC; break;
+            case OP_CONV_DGRAD: pk = L.backend >= 200 ? PK_CONV_DGRAD_MMA : L.backend ? PK_CONV_DGRAD_TC : PK_CONV_DGRAD_CC; break;
+            case OP_CONV_WGRAD: pk = L.backend >= 200 ? PK_CONV_WGRAD_MMA : L.backend ? PK_CONV_WGRAD_TC : PK_CONV_WGRAD_CC; break;
             case OP_SPLITK: pk = PK_SPLITK; break;
             case OP_BN_STATS: pk = PK_BN_STATS; nk = 2; break;
             case OP_BN_APPLY: pk = PK_BN_APPLY; break;
@@ -545,7 +606,9 @@ static int run_plan(resist_ctx* ctx, Plan& plan, const PatchArgs& pa, bool updat
         switch (L.kind) {
             case OP_CONV_FWD: case OP_CONV_DGRAD: case OP_CONV_WGRAD: {
                 const int mode = L.kind == OP_CONV_FWD ? CONV_FWD : L.kind == OP_CONV_DGRAD ? CONV_DGRAD : CONV_WGRAD;
-                if (L.backend && mode == CONV_WGRAD) { launch_conv_wgrad_tc_probs((const char*)plan.d_wtc + (size_t)L.first * plan.wtc_stride, L.count, L.gx, (size_t)L.max_elems, L.max_b, st); ++n_launch; }
+                if (L.backend >= 200 && mode == CONV_WGRAD) { launch_conv_wgrad_mma_probs((const char*)plan.d_wmm + (size_t)L.first * plan.wmm_stride, L.count, L.gx, (size_t)L.max_elems, L.max_b, L.backend - 200, st); ++n_launch; }
+                else if (L.backend >= 200) launch_conv_mma_probs((const char*)plan.d_mm + (size_t)L.first * plan.mm_stride, L.count, L.gx, (size_t)L.max_elems, L.backend - 1000, st);
+                else if (L.backend && mode == CONV_WGRAD) { launch_conv_wgrad_tc_probs((const char*)plan.d_wtc + (size_t)L.first * plan.wtc_stride, L.count, L.gx, (size_t)L.max_elems, L.max_b, st); ++n_launch; }
                 else if (L.backend) launch_conv_tc_probs((const char*)plan.d_tc + (size_t)L.first * plan.tc_stride, L.count, L.gx, (size_t)L.max_elems, st);
                 else launch_conv_ref(plan.d_conv + L.first, L.count, L.gx, mode, bf, st);
                 ++n_launch; break; }

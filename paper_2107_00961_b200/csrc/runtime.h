@@ -40,7 +40,7 @@ struct Launch {
 enum ProfKind {
     PK_CONV_FWD_CC, PK_CONV_DGRAD_CC, PK_CONV_WGRAD_CC, PK_CONV_FWD_TC, PK_CONV_DGRAD_TC, PK_CONV_WGRAD_TC, PK_SPLITK,
     PK_BN_STATS, PK_BN_APPLY, PK_BN_BWD_REDUCE, PK_BN_BWD_APPLY, PK_POOL_FWD, PK_POOL_BWD, PK_HEAD_FWD, PK_HEAD_BWD,
-    PK_SGD, PK_PATCH, PK_SCATTER, PK_AGGREGATE, PK_UPSAMPLE, PK_COUNT
+    PK_SGD, PK_PATCH, PK_SCATTER, PK_AGGREGATE, PK_UPSAMPLE, PK_CONV_FWD_MMA, PK_CONV_DGRAD_MMA, PK_CONV_WGRAD_MMA, PK_COUNT
 };
 struct Profiler {
     bool on = false;
@@ -67,6 +67,7 @@ struct Plan {
     PatchSite* d_sites = nullptr; int nsites = 0;
     void* d_tc = nullptr; size_t tc_stride = 0;              // tensor-core convolution descriptors
     void* d_wtc = nullptr; size_t wtc_stride = 0;            // tensor-core wgrad descriptors
+    void* d_mm = nullptr; size_t mm_stride = 0; void* d_wmm = nullptr; size_t wmm_stride = 0;   // warp-level MMA descriptors
     Segment* d_sgd = nullptr; int n_sgd_seg = 0; long long sgd_chunks = 0; double sgd_params = 0;
     resist_step_info info{};
 };

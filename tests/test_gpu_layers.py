@@ -46,7 +46,8 @@ SHAPES = [
 
 
 @pytest.mark.parametrize("shape", SHAPES)
-@pytest.mark.parametrize("dtype,backend", [("f32", 1), ("bf16", 1), ("bf16", 0)])
+# backend: 0 automatic choice, 1 CUDA cores only, 2 tcgen05 where the shape allows, 3 warp-level MMA where it allows
+@pytest.mark.parametrize("dtype,backend", [("f32", 1), ("bf16", 1), ("bf16", 0), ("bf16", 2), ("bf16", 3)])
 def test_conv_modes(m, shape, dtype, backend):
     N, H, W, C, K, k, s = shape
     bf = dtype == "bf16"
@@ -75,6 +76,10 @@ def test_conv_modes(m, shape, dtype, backend):
     assert max_rel_err(dw.cpu().numpy(), oracle.conv_wgrad(dy, a, k, s)) < (2e-3 if bf else 1e-4)
     if backend == 1:
         assert not used           # RESIST_CONV_CUDA_CORES really keeps the tensor cores out
+    if backend == 2:
+        assert used in (0, 1)
+    if backend == 3:
+        assert used in (0, 2)
 
 
 @pytest.mark.parametrize("m_rows,C", [(4096, 16), (1000, 32), (517, 64), (300, 24), (64, 256), (50, 2048), (9000, 8)])
