@@ -322,149 +322,247 @@ void launch_conv_mma_probs(const void* d, int nprob, int max_tiles, size_t max_s
 }
 
 // ------------------------------------------------------------------------------------------------ wgrad
-// dw[k][t][c] = sum over positions of dy[pos][k] * a[pos + shift_t][c].  GEMM with M = output channels, N = (tap,
-// input channel), reduction over the padded-flat positions, 128 per staging step.  A CTA owns a group of taps and
-// a range of pixel tiles; each warp owns some 8-wide N blocks for ALL M blocks (so that one ldmatrix of the shifted
-// activations feeds MB MMAs) and keeps its accumulators in registers over the whole range; the CTA then writes an
-// fp32 partial and a second kernel adds the partials in a fixed order.
+// dw[k][t][c] = sum over positions f of dy[f][k] * a[f + shift_t][c], on the tall padded map of the forward kernel
+// (dy and a read as zero at its padding positions).  GEMM with M = output channels, N = (tap, input channel) and
+// the reduction over positions.
+//
+// Work is cut into GROUPS of G whole images (G * Hp * Wp positions) and each group into SUB-position pieces.  Because
+// a group starts on an image boundary, one table (position in the group's window -> pixel index, or -1 at padding)
+// built once per CTA serves every piece of every group: staging a piece is a table lookup and a cp.async per 16
+// bytes, with no index arithmetic.  A CTA walks pieces blockIdx-strided with a ring of stages in flight; its 8
+// warps form a WP x WN grid: a warp takes every WP-th 16-position step of a piece and, for ALL 16-row blocks of M,
+// PPW pairs of 8-column blocks of N, and keeps those accumulators in registers over the whole walk.  At the end the
+// WP partial sums are added in a fixed order through shared memory, the CTA writes one fp32 partial, and a second
+// kernel adds the partials of all CTAs in a fixed order.
 struct alignas(16) MmaWgradProb {
     const __nv_bfloat16* dy;    // [n_img,H,W,K]  (stride 1; a stride-2 layer passes the zero-stuffed dy)
     const __nv_bfloat16* a;     // [n_img,H,W,C]
     float* partial;             // [splits][taps][K][C]
     float* out;                 // [K][taps][C]
-    int K, C, H, W, Wp, pad, ksz, taps, flat;
-    int n_img, tiles_per_img, pixel_tiles;
-    int box_w, box_h, act_rows;
-    int tap_groups, taps_per_group, splits, tiles_per_split;
+    int K, C, H, W, Hp, Wp, ksz, taps;
+    int G, n_groups, gpos;      // images per group, groups, positions per group (G * Hp * Wp)
+    int sub, subs, units;       // positions per piece (multiple of 16 * WP), pieces per group, pieces in total
+    int table_rows;             // subs * sub + 2 * halo
+    int tap_groups, taps_per_group, splits;
+    int wn, stages, variant, smem_bytes;
+    unsigned inv_wp, inv_hp;
 };
 
-template <int MB>   // MB = K / 16
+template <int MB, int PPW>   // MB = K / 16; PPW = pairs of 8-column blocks a warp owns
 __global__ void __launch_bounds__(MMA_THREADS) conv_wgrad_mma_kernel(const MmaWgradProb* __restrict__ probs) {
-    constexpr int NBW = 16 / MB;                                  // N blocks a warp may own
     __shared__ MmaWgradProb p;
     if (threadIdx.x < sizeof(MmaWgradProb) / 4) reinterpret_cast<uint32_t*>(&p)[threadIdx.x] = reinterpret_cast<const uint32_t*>(probs + blockIdx.y)[threadIdx.x];
     __syncthreads();
     if ((int)blockIdx.x >= p.tap_groups * p.splits) return;
     const int split = blockIdx.x % p.splits, tg = blockIdx.x / p.splits;
     const int tap0 = tg * p.taps_per_group; int ntap = p.taps - tap0; if (ntap > p.taps_per_group) ntap = p.taps_per_group;
-    const int t_begin = split * p.tiles_per_split; int t_end = t_begin + p.tiles_per_split; if (t_end > p.pixel_tiles) t_end = p.pixel_tiles;
     extern __shared__ __align__(16) uint8_t sm[];
-    const int K = p.K, C = p.C, dpitch = K * 2 + 16, apitch = C * 2 + 16;
-    uint8_t* s_dy = sm; uint8_t* s_a = sm + 128 * dpitch;
+    const int K = p.K, C = p.C, dpitch = K * 2 + 16, apitch = C * 2 + 16, Wp = p.Wp, sub = p.sub, subs = p.subs, stages = p.stages;
+    const int pad = p.ksz / 2, halo = pad * Wp + pad, rows_a = sub + 2 * halo;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int nbc = C / 8, nblocks = ntap * nbc;                  // N blocks of this CTA: (tap, 8 channels)
-    float acc[NBW][MB][4];
-#pragma unroll
-    for (int b = 0; b < NBW; ++b)
-#pragma unroll
-        for (int m = 0; m < MB; ++m) { acc[b][m][0] = acc[b][m][1] = acc[b][m][2] = acc[b][m][3] = 0.f; }
-    const uint32_t dy_base = s_u32(s_dy), a_base = s_u32(s_a);
-    const int ksz = p.ksz;
+    const int WN = p.wn, WP = 8 / WN, warp_n = warp % WN, warp_p = warp / WN;
+    int* table = reinterpret_cast<int*>(sm);
+    const int table_bytes = (p.table_rows * 4 + 127) & ~127;
+    const int dy_bytes = (sub * dpitch + 127) & ~127, stage_bytes = dy_bytes + ((rows_a * apitch + 127) & ~127);
+    uint8_t* ring = sm + table_bytes;
 
-    for (int t = t_begin; t < t_end; ++t) {
-        const int img = t / p.tiles_per_img, pos0 = (t % p.tiles_per_img) * 128;
-        const int row0 = p.flat ? 0 : pos0 / p.Wp, a_off = p.flat ? 0 : pos0 - row0 * p.Wp;
-        __syncthreads();                                          // the previous tile has been consumed
-        {   // dy at the 128 positions; pad positions and rows past the image are zeros: they add nothing
-            const int groups = K / 8, total = 128 * groups;
-            for (int id = tid; id < total; id += MMA_THREADS) {
-                const int g = id % groups, m = id / groups;
-                uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                long long pix = -1;
-                if (p.flat) { const long long gp = (long long)pos0 + m; if (gp < (long long)p.W) pix = gp; }
-                else { const int pos = pos0 + m, i = pos / p.Wp, j = pos - i * p.Wp; if (i < p.H && j < p.W) pix = ((long long)img * p.H + i) * p.W + j; }
-                if (pix >= 0) v = __ldg(reinterpret_cast<const uint4*>(p.dy + pix * K + g * 8));
-                *reinterpret_cast<uint4*>(s_dy + m * dpitch + g * 16) = v;
+    // ---- window row w of a group (position f = w - halo of the group) -> pixel index inside the group, -1 at padding
+    for (int w = tid; w < p.table_rows; w += MMA_THREADS) {
+        const int f = w - halo;
+        int pix = -1;
+        if (f >= 0 && f < p.gpos) {
+            const unsigned Y = __umulhi((unsigned)f, p.inv_wp), X = (unsigned)f - Y * Wp;
+            const unsigned n = __umulhi(Y, p.inv_hp), i = Y - n * p.Hp;
+            if (X < (unsigned)p.W && i < (unsigned)p.H) pix = (int)((n * p.H + i) * p.W + X);
+        }
+        table[w] = pix;
+    }
+    // ---- this thread's part of every copy: one 8-channel piece of every (256 / pieces-per-row)-th row
+    const int ga = C / 8, gd = K / 8;
+    const int a_step = MMA_THREADS / ga, d_step = MMA_THREADS / gd;           // rows per sweep (threads past step * g idle)
+    const int a_row0 = tid / ga, a_g = tid % ga, d_row0 = tid / gd, d_g = tid % gd;
+    const bool a_on = tid < a_step * ga, d_on = tid < d_step * gd;
+    const long long img_a = (long long)p.H * p.W * C, img_d = (long long)p.H * p.W * K;
+    const __nv_bfloat16* __restrict__ a_ptr = p.a; const __nv_bfloat16* __restrict__ dy_ptr = p.dy;
+    auto issue = [&](int unit, int stage) {
+        const int grp = unit / subs, j = unit - grp * subs;
+        const __nv_bfloat16* ag = a_ptr + (long long)grp * p.G * img_a + a_g * 8;
+        const __nv_bfloat16* dg = dy_ptr + (long long)grp * p.G * img_d + d_g * 8;
+        const uint32_t st0 = s_u32(ring + stage * stage_bytes);
+        if (a_on) {
+            const int* t = table + j * sub + a_row0;
+            uint32_t dst = st0 + dy_bytes + a_g * 16 + a_row0 * apitch;
+            for (int row = a_row0; row < rows_a; row += a_step, t += a_step, dst += a_step * apitch) {
+                const int pix = *t;                                // padding: read nothing, write zeros
+                cp_async16(dst, ag + (long long)max(pix, 0) * C, pix >= 0 ? 16u : 0u);
             }
         }
-        {   // activation window with its halo
-            const int groups = C / 8, total = p.act_rows * groups, boxpx = p.box_w * p.box_h;
-            const int x0 = p.flat ? pos0 : -p.pad, y0 = p.flat ? 0 : row0 - p.pad;
-            for (int id = tid; id < total; id += MMA_THREADS) {
-                const int g = id % groups, px = id / groups;
-                uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                if (px < boxpx) {
-                    const int x = px % p.box_w, y = px / p.box_w, gy = y0 + y, gx = x0 + x;
-                    if (gy >= 0 && gy < p.H && gx >= 0 && gx < p.W)
-                        v = __ldg(reinterpret_cast<const uint4*>(p.a + (((long long)img * p.H + gy) * p.W + gx) * C + g * 8));
+        if (d_on) {
+            const int* t = table + j * sub + halo + d_row0;
+            uint32_t dst = st0 + d_g * 16 + d_row0 * dpitch;
+            for (int row = d_row0; row < sub; row += d_step, t += d_step, dst += d_step * dpitch) {
+                const int pix = *t;
+                cp_async16(dst, dg + (long long)max(pix, 0) * K, pix >= 0 ? 16u : 0u);
+            }
+        }
+    };
+
+    const uint32_t b_lane = (uint32_t)((lane & 7) + ((lane >> 3) & 1) * 8) * apitch + (lane >> 4) * 16;
+    // ---- the column pairs of this warp: byte offset of (tap shift, 16 channels) in the activation window.  A warp with
+    // fewer than PPW pairs repeats its first one (no branch in the inner loop) and drops those sums at the end.
+    const int cpairs = C / 16, NP = ntap * cpairs;
+    uint32_t b_off[PPW];
+#pragma unroll
+    for (int e = 0; e < PPW; ++e) {
+        int q = warp_n * PPW + e; if (q >= NP) q = 0;
+        const int tt = q / cpairs, cp = q - tt * cpairs, tap = tap0 + tt, r = tap / p.ksz, s = tap - r * p.ksz;
+        b_off[e] = (uint32_t)((r * Wp + s) * apitch + cp * 32) + b_lane;
+    }
+    float acc[PPW][2][MB][4];
+#pragma unroll
+    for (int e = 0; e < PPW; ++e)
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+#pragma unroll
+            for (int m = 0; m < MB; ++m) { acc[e][h][m][0] = acc[e][h][m][1] = acc[e][h][m][2] = acc[e][h][m][3] = 0.f; }
+    // A = dy^T (stored [position][k], transposed on load); B = activations (stored [position][c], transposed on load)
+    const uint32_t a_lane = (uint32_t)((lane & 7) + ((lane >> 4) & 1) * 8) * dpitch + ((lane >> 3) & 1) * 16;
+    const int ksteps = sub / 16;
+
+    __syncthreads();                                              // table complete
+    const int units = p.units;
+    int nxt = split;
+    for (int st = 0; st < stages - 1; ++st) { if (nxt < units) issue(nxt, st); cp_async_commit(); nxt += p.splits; }
+    int stage = 0;
+    for (int unit = split; unit < units; unit += p.splits) {
+        { const int ps = stage == 0 ? stages - 1 : stage - 1; if (nxt < units) issue(nxt, ps); cp_async_commit(); nxt += p.splits; }
+        if (stages == 2) cp_async_wait<1>(); else if (stages == 3) cp_async_wait<2>(); else cp_async_wait<3>();
+        __syncthreads();
+        const uint32_t st0 = s_u32(ring + stage * stage_bytes);
+        uint32_t dy_row = st0 + a_lane + (uint32_t)(warp_p * 16) * dpitch, b_row = st0 + dy_bytes + (uint32_t)(warp_p * 16) * apitch;
+        for (int ks = warp_p; ks < ksteps; ks += WP, dy_row += WP * 16 * dpitch, b_row += WP * 16 * apitch) {
+            uint32_t af[MB][4];
+#pragma unroll
+            for (int m = 0; m < MB; ++m) ldsm_x4_t(dy_row + m * 32, af[m][0], af[m][1], af[m][2], af[m][3]);
+#pragma unroll
+            for (int e = 0; e < PPW; ++e) {
+                uint32_t b0, b1, b2, b3;
+                ldsm_x4_t(b_row + b_off[e], b0, b1, b2, b3);
+#pragma unroll
+                for (int m = 0; m < MB; ++m) {
+                    mma16816(acc[e][0][m], af[m][0], af[m][1], af[m][2], af[m][3], b0, b1);
+                    mma16816(acc[e][1][m], af[m][0], af[m][1], af[m][2], af[m][3], b2, b3);
                 }
-                *reinterpret_cast<uint4*>(s_a + px * apitch + g * 16) = v;
             }
         }
         __syncthreads();
-        for (int kk = 0; kk < 128; kk += 16) {
-            uint32_t af[MB][4];
-#pragma unroll
-            for (int m = 0; m < MB; ++m)       // A = dy^T: stored [pos][k], transposed on load
-                ldsm_x4_t(dy_base + (uint32_t)(kk + (lane & 7) + ((lane >> 4) & 1) * 8) * dpitch + (m * 16 + ((lane >> 3) & 1) * 8) * 2,
-                          af[m][0], af[m][1], af[m][2], af[m][3]);
-#pragma unroll
-            for (int b = 0; b < NBW; ++b) {
-                const int nb = warp + 8 * b;
-                if (nb < nblocks) {
-                    const int tt = nb / nbc, nj = nb % nbc, tp = tap0 + tt, r = tp / ksz, q = tp % ksz;
-                    uint32_t b0, b1;
-                    ldsm_x2_t(a_base + (uint32_t)(a_off + r * p.Wp + q + kk + (lane & 15)) * apitch + nj * 16, b0, b1);
-#pragma unroll
-                    for (int m = 0; m < MB; ++m) mma16816(acc[b][m], af[m][0], af[m][1], af[m][2], af[m][3], b0, b1);
-                }
-            }
-        }
+        stage = stage + 1 == stages ? 0 : stage + 1;
     }
-    // ---- partial sums: thread (g, t4) holds (m = 16*mi + g [+8], n = 8*nj + 2*t4 [+1])
-    const int g = lane >> 2, t4 = lane & 3;
+    cp_async_wait<0>();
+    __syncthreads();
+    // ---- add the WP partial sums in a fixed order: red[warp_p][tap][k][c]; thread (g8, t4) holds rows g8, g8+8, columns 2*t4, +1
+    float* red = reinterpret_cast<float*>(sm);
+    const int per = ntap * K * C;
+    const int g8 = lane >> 2, t4 = lane & 3;
 #pragma unroll
-    for (int b = 0; b < NBW; ++b) {
-        const int nb = warp + 8 * b;
-        if (nb >= nblocks) continue;
-        const int tt = nb / nbc, nj = nb % nbc;
+    for (int e = 0; e < PPW; ++e) {
+        const int q = warp_n * PPW + e;
+        if (q >= NP) continue;
+        const int tt = q / cpairs, cp = q - tt * cpairs;
 #pragma unroll
-        for (int m = 0; m < MB; ++m)
+        for (int h = 0; h < 2; ++h)
 #pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                const int k = m * 16 + g + half * 8;
-                float* dst = p.partial + (((long long)split * p.taps + tap0 + tt) * K + k) * C + nj * 8 + t4 * 2;
-                *reinterpret_cast<float2*>(dst) = make_float2(acc[b][m][half * 2], acc[b][m][half * 2 + 1]);
-            }
+            for (int m = 0; m < MB; ++m)
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    const int k = m * 16 + g8 + half * 8, c = cp * 16 + h * 8 + t4 * 2;
+                    *reinterpret_cast<float2*>(red + (long long)warp_p * per + (tt * K + k) * C + c) = make_float2(acc[e][h][m][half * 2], acc[e][h][m][half * 2 + 1]);
+                }
+    }
+    __syncthreads();
+    float* dst = p.partial + ((long long)split * p.taps + tap0) * K * C;
+    for (int i = tid; i < per; i += MMA_THREADS) {
+        float s = red[i];
+        for (int w = 1; w < WP; ++w) s += red[(long long)w * per + i];
+        dst[i] = s;
     }
 }
 
-// out[k][t][c] = sum over splits (ascending) of partial[split][t][k][c]
+// out[k][t][c] = sum over splits of partial[split][t][k][c], in a fixed order: a block owns 32 consecutive elements,
+// warp w adds the splits w, w+8, ... (ascending), then the 8 sums are added in warp order.
 __global__ void __launch_bounds__(256) wgrad_mma_reduce_kernel(const MmaWgradProb* __restrict__ probs) {
     const MmaWgradProb& p = probs[blockIdx.y];
-    const long long n = (long long)p.taps * p.K * p.C;
-    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
-        const int c = (int)(i % p.C); const long long r = i / p.C; const int t = (int)(r % p.taps); const int k = (int)(r / p.taps);
-        const long long src = ((long long)t * p.K + k) * p.C + c;
+    const int n = p.taps * p.K * p.C, splits = p.splits, taps = p.taps, K = p.K, C = p.C;
+    const float* __restrict__ partial = p.partial;
+    __shared__ float red[8][32];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int base = blockIdx.x * 32; base < n; base += gridDim.x * 32) {
+        const int i = base + lane;                                // n is a multiple of 256
         float s = 0.f;
-        for (int sp = 0; sp < p.splits; ++sp) s += p.partial[(long long)sp * n + src];
-        p.out[i] = s;
+#pragma unroll 4
+        for (int sp = warp; sp < splits; sp += 8) s += partial[(long long)sp * n + i];
+        red[warp][lane] = s;
+        __syncthreads();
+        if (warp == 0) {
+            float t = red[0][lane];
+#pragma unroll
+            for (int w = 1; w < 8; ++w) t += red[w][lane];
+            const int c = i % C, r = i / C, k = r % K, tp = r / K;
+            p.out[((long long)k * taps + tp) * C + c] = t;
+        }
+        __syncthreads();
     }
 }
 
-struct MmaWgGeom { int flat, n_img, H, W, Wp, box_w, box_h, act_rows, tiles_per_img, pixel_tiles, tap_groups, taps_per_group, splits, tiles_per_split; size_t smem, partial_bytes; };
+struct MmaWgGeom { int Hp, Wp, G, n_groups, gpos, sub, subs, units, table_rows, tap_groups, taps_per_group, splits, wn, ppw, stages, variant; size_t smem, partial_bytes; };
 
 static bool mma_wg_geometry(const ConvProb& p, int target_ctas, MmaWgGeom& g) {
     if (p.stride != 1 || (p.ksz != 1 && p.ksz != 3)) return false;
-    if (p.C % 16 || p.K % 16 || p.C > 64 || p.K > 64) return false;
+    if (p.C % 16 || p.K % 16 || p.C > 64 || p.K > 64 || p.N < 1) return false;
     if (((uintptr_t)p.act | (uintptr_t)p.wgt) & 15) return false;
-    const int taps = p.ksz * p.ksz, pad2 = p.ksz - 1;
-    g.flat = p.ksz == 1;
-    if (g.flat) { g.n_img = 1; g.H = 1; g.W = p.N * p.H * p.W; g.Wp = g.W; g.box_w = 128; g.box_h = 1; g.tiles_per_img = (int)(((long long)g.W + 127) / 128); }
-    else { g.n_img = p.N; g.H = p.H; g.W = p.W; g.Wp = p.W + pad2; if (g.Wp > 128) return false;
-        const int rows = (g.Wp - 1 + 127) / g.Wp + 1;
-        g.box_w = g.Wp; g.box_h = rows + pad2; g.tiles_per_img = (p.H * g.Wp + 127) / 128; }
-    const int max_read = (g.flat ? 0 : g.Wp - 1) + pad2 * g.Wp + pad2 + 128;
-    g.act_rows = std::max(g.box_w * g.box_h, max_read);
-    g.pixel_tiles = g.n_img * g.tiles_per_img;
-    const int MB = p.K / 16, nbw = 16 / MB, nbc = p.C / 8;
-    g.taps_per_group = std::max(1, std::min(taps, (8 * nbw) / nbc));
+    const int taps = p.ksz * p.ksz, pad = p.ksz / 2, MB = p.K / 16, cpairs = p.C / 16;
+    g.Hp = p.H + pad; g.Wp = p.W + pad;
+    if (g.Hp < 2 || g.Wp < 2) return false;
+    const int ppi = g.Hp * g.Wp, halo = pad * g.Wp + pad;
+    // taps per CTA and the warp grid: the fewest column splits whose accumulators still fit the registers
+    static const int ppw_set[] = {1, 2, 3, 5, 9, 12};
+    g.wn = 0;
+    for (int tpg : {taps, 3, 1}) {
+        if (tpg > taps) continue;
+        for (int wn : {1, 2, 4, 8}) {
+            const int need = (tpg * cpairs + wn - 1) / wn;
+            int ppw = 0; for (int c : ppw_set) if (c >= need) { ppw = c; break; }
+            if (ppw && MB * ppw <= 12) { g.wn = wn; g.ppw = ppw; g.taps_per_group = tpg; break; }
+        }
+        if (g.wn) break;
+    }
+    if (!g.wn) return false;
     g.tap_groups = (taps + g.taps_per_group - 1) / g.taps_per_group;
-    g.smem = (size_t)128 * (p.K * 2 + 16) + (size_t)g.act_rows * (p.C * 2 + 16) + 64;
-    if (g.smem > 200 * 1024) return false;
-    int want = std::max(1, target_ctas / g.tap_groups); if (want > g.pixel_tiles) want = g.pixel_tiles; if (want > 512) want = 512;
-    g.tiles_per_split = (g.pixel_tiles + want - 1) / want; g.splits = (g.pixel_tiles + g.tiles_per_split - 1) / g.tiles_per_split;
+    const int quantum = 16 * (8 / g.wn), dpitch = p.K * 2 + 16, apitch = p.C * 2 + 16;
+    const size_t red_bytes = (size_t)(8 / g.wn) * g.taps_per_group * p.K * p.C * 4;
+    // images per group and positions per piece: little padding of the last piece, pieces not too small
+    double best = 1e30; g.sub = 0;
+    for (int G = 1; G <= std::min(p.N, 64); ++G) {
+        if (p.N % G) continue;
+        const int gpos = G * ppi;
+        if (gpos + 2 * halo + 512 > 8192) break;
+        for (int sub = quantum; sub <= 512; sub += quantum) {
+            const int subs = (gpos + sub - 1) / sub;
+            const size_t table = (size_t)(((subs * sub + 2 * halo) * 4 + 127) & ~127);
+            const size_t stage = (size_t)((sub * dpitch + 127) & ~127) + (size_t)(((sub + 2 * halo) * apitch + 127) & ~127);
+            int stages = 3; if (table + 3 * stage > 150 * 1024) stages = 2;
+            if (table + stages * stage + 64 > 200 * 1024) continue;
+            const double cost = (double)subs * sub / gpos * (1.0 + 48.0 / sub);
+            if (cost < best) { best = cost; g.G = G; g.gpos = gpos; g.sub = sub; g.subs = subs; g.stages = stages; g.smem = std::max(table + stages * stage, red_bytes) + 64; }
+        }
+    }
+    if (!g.sub || g.smem > 200 * 1024) return false;
+    g.n_groups = p.N / g.G; g.units = g.n_groups * g.subs; g.table_rows = g.subs * g.sub + 2 * halo;
+    const int per_sm = g.smem <= 100 * 1024 ? 2 : 1;
+    int want = std::max(1, target_ctas * per_sm / 2 / g.tap_groups); if (want > g.units) want = g.units; if (want > 512) want = 512;
+    g.splits = want;
     g.partial_bytes = (size_t)g.splits * taps * p.K * p.C * 4;
+    g.variant = MB + 8 * g.ppw;
     return true;
 }
 bool conv_wgrad_mma_supported(const ConvProb& p, int target_ctas, size_t* partial_bytes) {
@@ -472,42 +570,43 @@ bool conv_wgrad_mma_supported(const ConvProb& p, int target_ctas, size_t* partia
     if (partial_bytes) *partial_bytes = g.partial_bytes;
     return true;
 }
+int conv_wgrad_mma_pick_variant(const ConvProb& p, int target_ctas) { MmaWgGeom g; return mma_wg_geometry(p, target_ctas, g) ? g.variant : 0; }
 // p.act = a, p.wgt = dy, p.out = dw (fp32), p.partial = workspace
 bool conv_wgrad_mma_fill(const ConvProb& p, int target_ctas, void* host) {
     MmaWgGeom g; if (!mma_wg_geometry(p, target_ctas, g)) return false;
     MmaWgradProb t; memset(&t, 0, sizeof(t));
     t.dy = (const __nv_bfloat16*)p.wgt; t.a = (const __nv_bfloat16*)p.act; t.partial = p.partial; t.out = (float*)p.out;
-    t.K = p.K; t.C = p.C; t.H = g.H; t.W = g.W; t.Wp = g.Wp; t.pad = p.ksz / 2; t.ksz = p.ksz; t.taps = p.ksz * p.ksz; t.flat = g.flat;
-    t.n_img = g.n_img; t.tiles_per_img = g.tiles_per_img; t.pixel_tiles = g.pixel_tiles; t.box_w = g.box_w; t.box_h = g.box_h; t.act_rows = g.act_rows;
-    t.tap_groups = g.tap_groups; t.taps_per_group = g.taps_per_group; t.splits = g.splits; t.tiles_per_split = g.tiles_per_split;
+    t.K = p.K; t.C = p.C; t.H = p.H; t.W = p.W; t.Hp = g.Hp; t.Wp = g.Wp; t.ksz = p.ksz; t.taps = p.ksz * p.ksz;
+    t.G = g.G; t.n_groups = g.n_groups; t.gpos = g.gpos; t.sub = g.sub; t.subs = g.subs; t.units = g.units; t.table_rows = g.table_rows;
+    t.tap_groups = g.tap_groups; t.taps_per_group = g.taps_per_group; t.splits = g.splits; t.wn = g.wn; t.stages = g.stages; t.variant = g.variant;
+    t.inv_wp = (unsigned)((1ull << 32) / (unsigned)g.Wp + 1); t.inv_hp = (unsigned)((1ull << 32) / (unsigned)g.Hp + 1);
+    t.smem_bytes = (int)g.smem;
     memcpy(host, &t, sizeof(t));
     return true;
 }
 size_t conv_wgrad_mma_prob_bytes() { return sizeof(MmaWgradProb); }
 int conv_wgrad_mma_ctas(const void* h) { const MmaWgradProb* t = (const MmaWgradProb*)h; return t->tap_groups * t->splits; }
-size_t conv_wgrad_mma_smem(const void* h) { const MmaWgradProb* t = (const MmaWgradProb*)h; return (size_t)128 * (t->K * 2 + 16) + (size_t)t->act_rows * (t->C * 2 + 16) + 64; }
+size_t conv_wgrad_mma_smem(const void* h) { return (size_t)((const MmaWgradProb*)h)->smem_bytes; }
 long long conv_wgrad_mma_out_elems(const void* h) { const MmaWgradProb* t = (const MmaWgradProb*)h; return (long long)t->taps * t->K * t->C; }
-int conv_wgrad_mma_k(const void* h) { return ((const MmaWgradProb*)h)->K; }
 
-// all problems of one launch must have the same number of output channels K
-void launch_conv_wgrad_mma_probs(const void* d, int nprob, int max_ctas, size_t max_smem, long long max_out, int K, cudaStream_t s) {
+template <int MB, int PPW>
+static void launch_wg_inst(const void* d, dim3 grid, size_t smem, cudaStream_t s) {
     static bool configured = false;
-    if (!configured) {
-        cudaFuncSetAttribute(conv_wgrad_mma_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-        cudaFuncSetAttribute(conv_wgrad_mma_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-        cudaFuncSetAttribute(conv_wgrad_mma_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-        cudaFuncSetAttribute(conv_wgrad_mma_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-        configured = true;
-    }
+    if (!configured) { cudaFuncSetAttribute(conv_wgrad_mma_kernel<MB, PPW>, cudaFuncAttributeMaxDynamicSharedMemorySize, 202 * 1024); configured = true; }
+    conv_wgrad_mma_kernel<MB, PPW><<<grid, MMA_THREADS, smem, s>>>((const MmaWgradProb*)d);
+}
+// all problems of one launch share the variant (output channels / 16 + 8 * column pairs per warp)
+void launch_conv_wgrad_mma_probs(const void* d, int nprob, int max_ctas, size_t max_smem, long long max_out, int variant, cudaStream_t s) {
     const dim3 grid(max_ctas, nprob);
-    switch (K / 16) {
-        case 1: conv_wgrad_mma_kernel<1><<<grid, MMA_THREADS, max_smem, s>>>((const MmaWgradProb*)d); break;
-        case 2: conv_wgrad_mma_kernel<2><<<grid, MMA_THREADS, max_smem, s>>>((const MmaWgradProb*)d); break;
-        case 3: conv_wgrad_mma_kernel<3><<<grid, MMA_THREADS, max_smem, s>>>((const MmaWgradProb*)d); break;
-        case 4: conv_wgrad_mma_kernel<4><<<grid, MMA_THREADS, max_smem, s>>>((const MmaWgradProb*)d); break;
-        default: return;
-    }
-    long long gx = (max_out + 255) / 256; if (gx > 592) gx = 592; if (gx < 1) gx = 1;
+    const int mb = variant & 7, ppw = (variant >> 3) & 31;
+#define WG_CASE(M, P) if (mb == M && ppw == P) launch_wg_inst<M, P>(d, grid, max_smem, s); else
+    WG_CASE(1, 1) WG_CASE(1, 2) WG_CASE(1, 3) WG_CASE(1, 5) WG_CASE(1, 9) WG_CASE(1, 12)
+    WG_CASE(2, 1) WG_CASE(2, 2) WG_CASE(2, 3) WG_CASE(2, 5)
+    WG_CASE(3, 1) WG_CASE(3, 2) WG_CASE(3, 3)
+    WG_CASE(4, 1) WG_CASE(4, 2) WG_CASE(4, 3)
+    return;
+#undef WG_CASE
+    long long gx = (max_out + 31) / 32; if (gx > 1184) gx = 1184; if (gx < 1) gx = 1;
     wgrad_mma_reduce_kernel<<<dim3((unsigned)gx, nprob), 256, 0, s>>>((const MmaWgradProb*)d);
 }
 

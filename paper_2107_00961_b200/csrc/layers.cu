@@ -33,7 +33,8 @@ size_t conv_wgrad_mma_prob_bytes();
 int conv_wgrad_mma_ctas(const void* h);
 size_t conv_wgrad_mma_smem(const void* h);
 long long conv_wgrad_mma_out_elems(const void* h);
-void launch_conv_wgrad_mma_probs(const void* d, int nprob, int max_ctas, size_t max_smem, long long max_out, int K, cudaStream_t s);
+void launch_conv_wgrad_mma_probs(const void* d, int nprob, int max_ctas, size_t max_smem, long long max_out, int variant, cudaStream_t s);
+int conv_wgrad_mma_pick_variant(const ConvProb& p, int target_ctas);
 }
 using namespace resist;
 
@@ -117,7 +118,7 @@ extern "C" int resist_conv2d(int32_t mode, int32_t dtype, int32_t backend, const
     if (e == cudaSuccess) {
         if (be == 1 && mode == CONV_WGRAD) launch_conv_wgrad_tc_probs(blob + 1024, 1, conv_wgrad_tc_ctas(hd.data()), conv_wgrad_tc_smem(hd.data()), conv_wgrad_tc_out_elems(hd.data()), st);
         else if (be == 1) launch_conv_tc_probs(blob + 1024, 1, conv_tc_tiles(hd.data()), conv_tc_smem(hd.data()), st);
-        else if (be == 2 && mode == CONV_WGRAD) launch_conv_wgrad_mma_probs(blob + 1024, 1, conv_wgrad_mma_ctas(hd.data()), conv_wgrad_mma_smem(hd.data()), conv_wgrad_mma_out_elems(hd.data()), p.K, st);
+        else if (be == 2 && mode == CONV_WGRAD) launch_conv_wgrad_mma_probs(blob + 1024, 1, conv_wgrad_mma_ctas(hd.data()), conv_wgrad_mma_smem(hd.data()), conv_wgrad_mma_out_elems(hd.data()), conv_wgrad_mma_pick_variant(p, 2 * sm), st);
         else if (be == 2) launch_conv_mma_probs(blob + 1024, 1, conv_mma_tiles(hd.data()), conv_mma_smem(hd.data()), conv_mma_pick_variant(p, mode), st);
         else {
             launch_conv_ref((ConvProb*)blob, 1, p.tiles_m * p.tiles_n * p.splits, mode, dtype == RESIST_BF16, st);

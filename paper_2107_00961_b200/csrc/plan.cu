@@ -41,7 +41,8 @@ size_t conv_wgrad_mma_prob_bytes();
 int conv_wgrad_mma_ctas(const void* h);
 size_t conv_wgrad_mma_smem(const void* h);
 long long conv_wgrad_mma_out_elems(const void* h);
-void launch_conv_wgrad_mma_probs(const void* d, int nprob, int max_ctas, size_t max_smem, long long max_out, int K, cudaStream_t s);
+void launch_conv_wgrad_mma_probs(const void* d, int nprob, int max_ctas, size_t max_smem, long long max_out, int variant, cudaStream_t s);
+int conv_wgrad_mma_pick_variant(const ConvProb& p, int target_ctas);
 
 // Which kernel family takes a bf16 convolution: 0 = CUDA cores, 1 = tcgen05, >= 200 = warp-level MMA (wgrad: 200 +
 // output channels; forward and dgrad: 1000 + the kernel variant, so that the value also separates launches by what
@@ -49,7 +50,7 @@ void launch_conv_wgrad_mma_probs(const void* d, int nprob, int max_ctas, size_t 
 static int pick_backend(const ConvProb& p, int mode, int target_ctas, size_t* partial_bytes, int pref = RESIST_CONV_AUTO) {
     const bool want_mma = pref == RESIST_CONV_AUTO || pref == RESIST_CONV_WARP_MMA, want_tc = pref == RESIST_CONV_AUTO || pref == RESIST_CONV_TCGEN05;
     if (mode == CONV_WGRAD) {
-        if (pref == RESIST_CONV_WARP_MMA && conv_wgrad_mma_supported(p, target_ctas, partial_bytes)) return 200 + p.K;
+        if (want_mma && conv_wgrad_mma_supported(p, target_ctas, partial_bytes)) return 200 + conv_wgrad_mma_pick_variant(p, target_ctas);
         if (want_tc && conv_wgrad_tc_supported(p, target_ctas, partial_bytes)) return 1;
         return 0;
     }

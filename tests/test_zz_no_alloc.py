@@ -6,6 +6,8 @@ the library instead.  This file is named so that pytest collects it last: a run 
 has then already run every other test.  It calls the entry point twice in a row, on different data, because the
 second call finds the first call's leftovers in the shared array.
 """
+import gc
+
 import numpy as np
 import pytest
 import torch
@@ -39,10 +41,15 @@ def test_noalloc_matches_the_allocating_entry_point_twice_in_a_row(dtype):
         a_ref, stat_ref = m.resist_bn_relu_forward(x, g, b, rm, rv)
         a = torch.empty_like(x)
         stat = torch.zeros(4 * C, dtype=torch.float32, device="cuda")
-        before = torch.cuda.memory_allocated()
-        m.resist_bn_relu_forward_noalloc(x, g, b, a, stat, rm2, rv2)
-        torch.cuda.synchronize()
-        assert torch.cuda.memory_allocated() == before
+        gc.collect()                     # tensors of earlier tests that die in here would change the counter too
+        gc.disable()
+        try:
+            before = torch.cuda.memory_allocated()
+            m.resist_bn_relu_forward_noalloc(x, g, b, a, stat, rm2, rv2)
+            torch.cuda.synchronize()
+            assert torch.cuda.memory_allocated() == before
+        finally:
+            gc.enable()
         tol = 2e-2 if bf else 1e-4
         err = norm_max_abs if bf else max_rel_err
         assert err(a.float().cpu().numpy(), a_ref.float().cpu().numpy()) < tol
