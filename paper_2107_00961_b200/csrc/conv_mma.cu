@@ -1,19 +1,21 @@
 // Convolutions of NARROW layers (C and K multiples of 16, at most 64) on warp-level MMA (mma.sync m16n8k16, bf16
 // inputs, fp32 accumulation).
 //
-// Why not tcgen05 here: one tcgen05.mma with M = 128, K = 16 occupies the SM's tensor core for ~153 cycles whatever
-// N is (measured for N = 16 ... 256, every operand layout, one MMA at a time per SM), so a layer with 16 output
-// channels uses 1/16 of the array and is bound by that rate at a third of what HBM allows.  The warp-level MMA
-// has no such granularity (n = 8) and was measured at 550 TFLOP/s dense on this GPU, far more than these
-// HBM-bound layers need.  Wide layers (more than 64 channels) stay on tcgen05 (conv_tc.cu).
+// Why not tcgen05 here: the SM's tensor core takes about 40 cycles per tcgen05.mma with M = 128, K = 16 however
+// small N is (measured: 21 ns per MMA at N = 16 with two issuing threads, 41 ns with one), so a layer with 16
+// output channels uses 1/16 of the array and is bound by that rate below what HBM allows.  The warp-level MMA has
+// no such granularity (n = 8) and was measured at 550 TFLOP/s dense on this GPU, more than these HBM-bound layers
+// need.  Wide layers (more than 64 channels) stay on tcgen05 (conv_tc.cu).
 //
-// Tiling: the whole batch is ONE tall zero-padded image.  With pad = k/2, image n occupies rows n*Hp .. n*Hp+H-1
-// (Hp = H + pad) of a map that is Wp = W + pad wide; row H of every image and column W of every row are zero and
-// serve as the padding of both neighbours, because positions are numbered row-major ("padded-flat", f = Y*Wp + X)
-// and a tap (r, s) reads position f + (r-pad)*Wp + (s-pad).  A tile is 128 or 256 consecutive positions; the window
-// of positions it needs (tile + halo of pad*Wp + pad on either side) is staged once in shared memory as
-// [position][channel] rows, padded by 16 bytes against bank conflicts, and the k*k taps read it at shifted row
-// offsets through ldmatrix.  Padding positions are computed like any other and dropped by the epilogue.
+// Tiling: a GROUP of G whole images is one tall zero-padded map.  With pad = k/2, image n occupies rows
+// n*Hp .. n*Hp+H-1 (Hp = H + pad) of a map that is Wp = W + pad wide; row H of every image and column W of every
+// row are zero and serve as the padding of both neighbours, because positions are numbered row-major
+// ("padded-flat", f = Y*Wp + X) and a tap (r, s) reads position f + (r-pad)*Wp + (s-pad).  A group is cut into
+// pieces of SUB consecutive positions; the window a piece needs (piece + halo of pad*Wp + pad on either side) is
+// staged in shared memory as [position][channel] rows, padded by 16 bytes against bank conflicts, and the k*k
+// taps read it at shifted row offsets through ldmatrix.  Because a group starts on an image boundary, two small
+// tables built once per CTA (window row -> input pixel, position -> output pixel; -1 at padding) serve every
+// piece of every group: neither the copies nor the epilogue do any index arithmetic.
 #include <algorithm>
 #include <cstring>
 #include "internal.h"
@@ -28,13 +30,14 @@ struct alignas(16) MmaProb {
     int wC;                     // C of the weight tensor (its innermost extent)
     int H, W, Hp, Wp;           // image extent; extent of one image in the tall padded map
     unsigned inv_wp, inv_hp;    // floor(2^32 / d) + 1: __umulhi(f, inv) = f / d for every f the kernel meets
-    int total;                  // positions of the tall padded map, n_img * Hp * Wp
-    int tiles;                  // ceil(total / tile)
+    int G, gpos;                // images per group, positions per group (G * Hp * Wp)
+    int sub, subs, units;       // positions per piece (multiple of 16), pieces per group, pieces in total
     int os, P, Q;               // output stride (forward of a stride-2 layer stores even positions only, as a P x Q image)
     int stages;                 // depth of the activation ring (2, 3 or 4)
-    int variant;                // which instantiation runs this problem (see mma_variant)
+    int variant, smem_bytes;    // which instantiation runs this problem (see mma_variant); dynamic shared memory
     float scale;
 };
+
 
 __device__ __forceinline__ uint32_t s_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
@@ -55,7 +58,6 @@ __device__ __forceinline__ void mma16816(float* c, uint32_t a0, uint32_t a1, uin
 }
 
 constexpr int MMA_THREADS = 256;
-constexpr int MMA_SLOTS = 10;          // 16-byte pieces of the activation window a thread copies per tile (at most)
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");   // src_bytes 0: zeros
@@ -68,33 +70,56 @@ template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile(
 template <int NB> __host__ __device__ __forceinline__ int chan_of_col(int n) { return ((n & 7) >> 1) * (2 * NB) + 2 * (n >> 3) + (n & 1); }
 template <int NB> __host__ __device__ __forceinline__ int col_of_chan(int c) { return 8 * ((c % (2 * NB)) >> 1) + 2 * (c / (2 * NB)) + (c & 1); }
 
-// Persistent: a CTA keeps the whole filter in shared memory and walks the tiles blockIdx.x, blockIdx.x + gridDim.x, ...
-// of its problem.  The activation windows of the next tiles are in flight (cp.async, ring of p.stages) while the
-// warps run ldmatrix + mma.sync on the current one.
-// NB = output channels / 8 (2, 4, 6 or 8); MBW = 16-row blocks per warp (tile = 128 * MBW positions); KSZ = 1 or 3;
-// TRANS = false: forward (weights read as [n][k]); true: dgrad (weights read as [k][n] and transposed on load, taps flipped).
+
+// Persistent: a CTA keeps the whole filter in shared memory and walks the pieces blockIdx.x, blockIdx.x + gridDim.x,
+// ... of its problem.  The windows of the next pieces are in flight (cp.async, ring of p.stages) while the warps run
+// ldmatrix + mma.sync on the current one.  Warp w computes the 16-row blocks w, w + 8, ... of a piece.
+// NB = output channels / 8 (2, 4, 6 or 8); MBW = 16-row blocks per warp (a piece has at most 128 * MBW positions);
+// KSZ = 1 or 3; TRANS = false: forward (weights read as [n][k]); true: dgrad (weights read as [k][n] and transposed
+// on load, taps flipped).
 template <int NB, int MBW, int KSZ, bool TRANS>
 __global__ void __launch_bounds__(MMA_THREADS) conv_mma_kernel(const MmaProb* __restrict__ probs) {
     __shared__ MmaProb p;
     if (threadIdx.x < sizeof(MmaProb) / 4) reinterpret_cast<uint32_t*>(&p)[threadIdx.x] = reinterpret_cast<const uint32_t*>(probs + blockIdx.y)[threadIdx.x];
     __syncthreads();
-    constexpr int TILE = 128 * MBW, TAPS = KSZ * KSZ, PAD = KSZ / 2;
-    const int tiles = p.tiles;
-    if ((int)blockIdx.x >= tiles) return;
+    constexpr int TAPS = KSZ * KSZ, PAD = KSZ / 2, ncol = NB * 8;
+    const int units = p.units;
+    if ((int)blockIdx.x >= units) return;
     extern __shared__ __align__(16) uint8_t sm[];
     const int ca = p.ca, apitch = ca * 2 + 16;                    // activation row pitch in bytes
-    constexpr int ncol = NB * 8;
     const int wrows = TRANS ? ca : ncol;                          // rows of one tap of the staged filter
     const int wcols = TRANS ? ncol : ca;                          // elements per row
     const int wpitch = wcols * 2 + 16;
-    const int H = p.H, W = p.W, Hp = p.Hp, Wp = p.Wp, total = p.total, stages = p.stages, os = p.os;
-    const unsigned inv_wp = p.inv_wp, inv_hp = p.inv_hp;
-    const int halo = PAD * Wp + PAD, win_rows = TILE + 2 * halo;
+    const int Wp = p.Wp, sub = p.sub, subs = p.subs, stages = p.stages;
+    const int halo = PAD * Wp + PAD, win_rows = sub + 2 * halo, nblk = sub / 16;
+    const int it_rows = subs * sub + 2 * halo, ot_rows = subs * sub;
+    int* itable = reinterpret_cast<int*>(sm);
+    int* otable = itable + it_rows;
+    const int table_bytes = ((it_rows + ot_rows) * 4 + 127) & ~127;
     const int stage_bytes = (win_rows * apitch + 127) & ~127;
-    uint8_t* s_w = sm + stages * stage_bytes;
+    uint8_t* ring = sm + table_bytes;
+    uint8_t* s_w = ring + stages * stage_bytes;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const __nv_bfloat16* __restrict__ act = p.act;
+    const __nv_bfloat16* __restrict__ addp = p.add;
+    __nv_bfloat16* __restrict__ outp = p.out;
 
+    // ---- tables: window row w of a group (position f = w - halo) -> input pixel inside the group; position -> output pixel
+    for (int w = tid; w < it_rows; w += MMA_THREADS) {
+        const int f = w - halo;
+        int pix = -1, opix = -1;
+        if (f >= 0 && f < p.gpos) {
+            const unsigned Y = __umulhi((unsigned)f, p.inv_wp), X = (unsigned)f - Y * Wp;
+            const unsigned n = __umulhi(Y, p.inv_hp), i = Y - n * p.Hp;
+            if (X < (unsigned)p.W && i < (unsigned)p.H) {
+                pix = (int)((n * p.H + i) * p.W + X);
+                if (p.os == 1) opix = pix;
+                else if (!((i % p.os) | (X % p.os))) opix = (int)((n * p.P + i / p.os) * p.Q + X / p.os);
+            }
+        }
+        itable[w] = pix;
+        if (f >= 0 && f < ot_rows) otable[f] = opix;
+    }
     // ---- the filter, once per CTA
     if (!TRANS) {               // tap t, column n, 8-channel group g  <-  w[chan_of_col(n)][t][g*8..]
         const int groups = ca / 8, n_chunks = TAPS * ncol * groups;
@@ -114,47 +139,45 @@ __global__ void __launch_bounds__(MMA_THREADS) conv_mma_kernel(const MmaProb* __
             for (int e = 0; e < 4; ++e) *reinterpret_cast<uint32_t*>(row + col_of_chan<NB>(g * 8 + 2 * e) * 2) = w4[e];   // channel pairs stay adjacent
         }
     }
-    // ---- what this thread copies for every tile: the same pieces of the window, fixed once (row | group << 16)
-    const int groups = ca / 8, nchunk = win_rows * groups;
-    int slot[MMA_SLOTS];
-#pragma unroll
-    for (int k = 0; k < MMA_SLOTS; ++k) {
-        const int id = tid + k * MMA_THREADS;
-        slot[k] = id < nchunk ? ((id / groups) | ((id % groups) << 16)) : -1;
-    }
-    auto issue = [&](int tile, int stage) {
-        const int f0 = tile * TILE - halo;                         // position of window row 0 (negative at the very start)
-        const uint32_t dst0 = s_u32(sm + stage * stage_bytes);
-#pragma unroll
-        for (int k = 0; k < MMA_SLOTS; ++k) {
-            if (slot[k] < 0) continue;
-            const int w = slot[k] & 0xFFFF, g = slot[k] >> 16;
-            const unsigned f = (unsigned)(f0 + w);
-            const unsigned Y = __umulhi(f, inv_wp), X = f - Y * Wp;
-            const unsigned n = __umulhi(Y, inv_hp), i = Y - n * Hp;
-            const bool ok = f < (unsigned)total && X < (unsigned)W && i < (unsigned)H;
-            const __nv_bfloat16* src = ok ? act + (((long long)n * H + i) * W + X) * ca + g * 8 : act;
-            cp_async16(dst0 + w * apitch + g * 16, src, ok ? 16u : 0u);
+    // ---- this thread's part of every copy: one 8-channel piece of every (256 / pieces-per-row)-th window row
+    const int ga = ca / 8, a_step = MMA_THREADS / ga, a_row0 = tid / ga, a_g = tid % ga;
+    const bool a_on = tid < a_step * ga;
+    const long long grp_in = (long long)p.G * p.H * p.W * ca;                    // elements of a group of act
+    const long long grp_out = (long long)p.G * (p.os == 1 ? p.H * p.W : p.P * p.Q) * ncol;
+    auto issue = [&](int unit, int stage) {
+        const int grp = unit / subs, j = unit - grp * subs;
+        const __nv_bfloat16* ag = act + grp * grp_in + a_g * 8;
+        if (a_on) {
+            const int* t = itable + j * sub + a_row0;
+            uint32_t dst = s_u32(ring + stage * stage_bytes) + a_g * 16 + a_row0 * apitch;
+            for (int row = a_row0; row < win_rows; row += a_step, t += a_step, dst += a_step * apitch) {
+                const int pix = *t;                                // padding: read nothing, write zeros
+                cp_async16(dst, ag + (long long)max(pix, 0) * ca, pix >= 0 ? 16u : 0u);
+            }
         }
     };
 
     const uint32_t w_base = s_u32(s_w);
     const int g8 = lane >> 2, t4 = lane & 3;
-    const uint32_t a_lane = (uint32_t)(warp * 16 * MBW + (lane & 15)) * apitch + (lane >> 4) * 16;
+    // 16-row blocks of this warp; one past the piece repeats the last block (no branch in the inner loop) and is not stored
+    uint32_t a_blk[MBW];
+#pragma unroll
+    for (int mb = 0; mb < MBW; ++mb) a_blk[mb] = (uint32_t)(min(warp + 8 * mb, nblk - 1) * 16 + (lane & 15)) * apitch + (lane >> 4) * 16;
     // B fragments of two 8-column blocks per ldmatrix.x4: lanes 0-7 / 8-15 address the two k halves of block j, lanes 16-31 those of block j+1
     const uint32_t b_lane = TRANS ? (uint32_t)(((lane >> 3) & 1) * 8 + (lane & 7)) * wpitch + (lane >> 4) * 16
                                   : (uint32_t)((lane >> 4) * 8 + (lane & 7)) * wpitch + ((lane >> 3) & 1) * 16;
+    const float scale = p.scale;
 
-    // prologue: the first stages-1 tiles of this CTA
+    __syncthreads();                                              // tables complete
     int nxt = blockIdx.x;
-    for (int st = 0; st < stages - 1; ++st) { if (nxt < tiles) issue(nxt, st); cp_async_commit(); nxt += gridDim.x; }
+    for (int st = 0; st < stages - 1; ++st) { if (nxt < units) issue(nxt, st); cp_async_commit(); nxt += gridDim.x; }
     int stage = 0;
-    for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
-        { const int ps = stage == 0 ? stages - 1 : stage - 1; if (nxt < tiles) issue(nxt, ps); cp_async_commit(); nxt += gridDim.x; }
+    for (int unit = blockIdx.x; unit < units; unit += gridDim.x) {
+        { const int ps = stage == 0 ? stages - 1 : stage - 1; if (nxt < units) issue(nxt, ps); cp_async_commit(); nxt += gridDim.x; }
         if (stages == 2) cp_async_wait<1>(); else if (stages == 3) cp_async_wait<2>(); else cp_async_wait<3>();
-        __syncthreads();                                          // this tile's window (and, first time, the filter) is in shared memory
+        __syncthreads();                                          // this piece's window (and, first time, the filter) is in shared memory
 
-        const uint32_t a_base = s_u32(sm + stage * stage_bytes) + a_lane;
+        const uint32_t a_base = s_u32(ring + stage * stage_bytes);
         float acc[MBW][NB][4];
 #pragma unroll
         for (int mb = 0; mb < MBW; ++mb)
@@ -170,7 +193,7 @@ __global__ void __launch_bounds__(MMA_THREADS) conv_mma_kernel(const MmaProb* __
             for (int k0 = 0; k0 < ca; k0 += 16) {
                 uint32_t a[MBW][4];
 #pragma unroll
-                for (int mb = 0; mb < MBW; ++mb) ldsm_x4(a_tap + (uint32_t)(mb * 16) * apitch + k0 * 2, a[mb][0], a[mb][1], a[mb][2], a[mb][3]);
+                for (int mb = 0; mb < MBW; ++mb) ldsm_x4(a_tap + a_blk[mb] + k0 * 2, a[mb][0], a[mb][1], a[mb][2], a[mb][3]);
 #pragma unroll
                 for (int j = 0; j < NB; j += 2) {
                     uint32_t b0, b1, b2, b3;
@@ -185,20 +208,16 @@ __global__ void __launch_bounds__(MMA_THREADS) conv_mma_kernel(const MmaProb* __
             }
         }
         // ---- epilogue: thread (g8, t4) holds rows g8 and g8+8 of each 16-row block, channels t4*2*NB ... t4*2*NB + 2*NB - 1
-        const float scale = p.scale;
-        const __nv_bfloat16* __restrict__ addp = p.add;
+        const int grp = unit / subs, j0 = (unit - grp * subs) * sub;
+        const long long obase = grp * grp_out + t4 * (2 * NB);
 #pragma unroll
         for (int mb = 0; mb < MBW; ++mb)
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
-                const unsigned f = (unsigned)(tile * TILE + warp * 16 * MBW + mb * 16 + g8 + half * 8);
-                const unsigned Y = __umulhi(f, inv_wp), X = f - Y * Wp;
-                const unsigned n = __umulhi(Y, inv_hp), i = Y - n * Hp;
-                if (!(f < (unsigned)total && X < (unsigned)W && i < (unsigned)H)) continue;
-                long long pix;
-                if (os == 1) pix = ((long long)n * H + i) * W + X;
-                else { if ((i % os) | (X % os)) continue; pix = ((long long)n * p.P + i / os) * p.Q + X / os; }
-                const long long o = pix * ncol + t4 * (2 * NB);
+                const int blk = warp + 8 * mb;
+                const int opix = blk < nblk ? otable[j0 + blk * 16 + g8 + half * 8] : -1;
+                if (opix < 0) continue;
+                const long long o = obase + (long long)opix * ncol;
                 uint32_t wv[NB];
                 if (addp) {
                     if constexpr (NB % 4 == 0) {
@@ -218,10 +237,10 @@ __global__ void __launch_bounds__(MMA_THREADS) conv_mma_kernel(const MmaProb* __
                 }
                 if constexpr (NB % 4 == 0) {
 #pragma unroll
-                    for (int c4 = 0; c4 < NB / 4; ++c4) *reinterpret_cast<uint4*>(p.out + o + c4 * 8) = make_uint4(wv[c4 * 4], wv[c4 * 4 + 1], wv[c4 * 4 + 2], wv[c4 * 4 + 3]);
+                    for (int c4 = 0; c4 < NB / 4; ++c4) *reinterpret_cast<uint4*>(outp + o + c4 * 8) = make_uint4(wv[c4 * 4], wv[c4 * 4 + 1], wv[c4 * 4 + 2], wv[c4 * 4 + 3]);
                 } else {
 #pragma unroll
-                    for (int c2 = 0; c2 < NB / 2; ++c2) *reinterpret_cast<uint2*>(p.out + o + c2 * 4) = make_uint2(wv[c2 * 2], wv[c2 * 2 + 1]);
+                    for (int c2 = 0; c2 < NB / 2; ++c2) *reinterpret_cast<uint2*>(outp + o + c2 * 4) = make_uint2(wv[c2 * 2], wv[c2 * 2 + 1]);
                 }
             }
         __syncthreads();                                          // every warp is done with this stage before it is refilled
@@ -231,38 +250,49 @@ __global__ void __launch_bounds__(MMA_THREADS) conv_mma_kernel(const MmaProb* __
 }
 
 // ------------------------------------------------------------------------------------------------ host side
-struct MmaGeom { int ca, ncol, Hp, Wp, total, mbw, tiles, stages, variant; size_t smem; };
+struct MmaGeom { int ca, ncol, Hp, Wp, G, gpos, sub, subs, units, mbw, stages, variant; size_t smem; };
 
-// variant = (((stages * 4 + MBW) * 4 + ksz) * 2 + trans) * 16 + NB: everything a launch is specialised on
-static int mma_variant(int stages, int mbw, int ksz, int trans, int nb) { return (((stages * 4 + mbw) * 4 + ksz) * 2 + trans) * 16 + nb; }
+// variant = ((MBW * 4 + ksz) * 2 + trans) * 16 + NB: everything a launch is specialised on
+static int mma_variant(int mbw, int ksz, int trans, int nb) { return ((mbw * 4 + ksz) * 2 + trans) * 16 + nb; }
 
 static bool mma_geometry(const ConvProb& p, int mode, MmaGeom& g) {
     if (mode == CONV_WGRAD) return false;
     if ((p.ksz != 1 && p.ksz != 3) || p.stride < 1 || p.stride > 2 || (p.stride == 2 && mode != CONV_FWD)) return false;
-    if (p.C % 16 || p.K % 16 || p.C > 64 || p.K > 64) return false;
+    if (p.C % 16 || p.K % 16 || p.C > 64 || p.K > 64 || p.N < 1) return false;
     if (((uintptr_t)p.act | (uintptr_t)p.wgt | (uintptr_t)p.out | (uintptr_t)p.add) & 15) return false;
     g.ca = mode == CONV_FWD ? p.C : p.K; g.ncol = mode == CONV_FWD ? p.K : p.C;
     const int pad = p.ksz / 2;
     g.Hp = p.H + pad; g.Wp = p.W + pad;
-    if (g.Hp < 2 || g.Wp < 2 || g.Wp > 4096) return false;
-    const long long total = (long long)p.N * g.Hp * g.Wp;
-    const int halo = pad * g.Wp + pad;
-    if ((total + 512 + 2 * halo) * std::max(g.Hp, g.Wp) >= (1ll << 32) || total >= (1ll << 30)) return false;   // exact division by multiplication
-    g.total = (int)total;
-    const int apitch = g.ca * 2 + 16, groups = g.ca / 8;
+    if (g.Hp < 2 || g.Wp < 2) return false;
+    const int ppi = g.Hp * g.Wp, halo = pad * g.Wp + pad;
+    const int apitch = g.ca * 2 + 16;
     const int wrows = mode == CONV_FWD ? g.ncol : g.ca, wcols = mode == CONV_FWD ? g.ca : g.ncol;
     const size_t wbytes = (size_t)p.ksz * p.ksz * wrows * (wcols * 2 + 16);
-    // 256-position tiles when that still gives every SM work and the window fits the copy slots, else 128
-    g.mbw = total >= 256ll * 148 ? 2 : 1;
-    if (g.mbw == 2 && ((256 + 2 * halo) * groups > MMA_SLOTS * MMA_THREADS || g.ncol > 32)) g.mbw = 1;
-    const int tile = 128 * g.mbw, win_rows = tile + 2 * halo;
-    if (win_rows * groups > MMA_SLOTS * MMA_THREADS || win_rows > 65535) return false;
-    g.tiles = (int)((total + tile - 1) / tile);
-    const size_t stage = (size_t)((win_rows * apitch + 127) & ~127);
-    g.stages = 4; while (g.stages > 2 && g.stages * stage + wbytes + 64 > 100 * 1024) --g.stages;
-    g.smem = g.stages * stage + wbytes + 64;
-    g.variant = mma_variant(g.stages, g.mbw, p.ksz, mode == CONV_DGRAD ? 1 : 0, g.ncol / 8);
-    return g.smem <= 200 * 1024;
+    const int max_mbw = g.ncol <= 32 ? 3 : 2;                     // accumulators: MBW * (ncol / 8) * 4 registers
+    // images per group and positions per piece: little padding of the last piece, all warps busy, pieces not too
+    // small, enough pieces to go round
+    double best = 1e30; g.sub = 0;
+    for (int G = 1; G <= std::min(p.N, 64); ++G) {
+        if (p.N % G) continue;
+        const int gpos = G * ppi;
+        if (gpos > 3000 && g.sub) break;
+        if (gpos > 7000) break;
+        for (int sub = 64; sub <= 128 * max_mbw; sub += 16) {
+            const int subs = (gpos + sub - 1) / sub, nblk = sub / 16, mbw = (nblk + 7) / 8;
+            const size_t table = (size_t)(((2 * subs * sub + 2 * halo) * 4 + 127) & ~127);
+            const size_t stage = (size_t)(((sub + 2 * halo) * apitch + 127) & ~127);
+            int stages = 4; while (stages > 2 && table + stages * stage + wbytes + 64 > 100 * 1024) --stages;
+            if (table + stages * stage + wbytes + 64 > 200 * 1024) continue;
+            const long long units = (long long)(p.N / G) * subs;
+            double cost = (double)subs * sub / gpos * (1.0 + 48.0 / sub) * (8.0 * mbw / nblk);
+            if (units < 64) cost *= 1.0 + 0.5 * (64 - units) / 64.0;
+            if (cost < best) { best = cost; g.G = G; g.gpos = gpos; g.sub = sub; g.subs = subs; g.units = (int)units; g.mbw = mbw; g.stages = stages;
+                               g.smem = table + stages * stage + wbytes + 64; }
+        }
+    }
+    if (!g.sub) return false;
+    g.variant = mma_variant(g.mbw, p.ksz, mode == CONV_DGRAD ? 1 : 0, g.ncol / 8);
+    return true;
 }
 
 bool conv_mma_supported(const ConvProb& p, int mode) { MmaGeom g; return mma_geometry(p, mode, g); }
@@ -275,25 +305,20 @@ bool conv_mma_fill(const ConvProb& p, int mode, void* host) {
     t.act = (const __nv_bfloat16*)p.act; t.wgt = (const __nv_bfloat16*)p.wgt; t.add = (const __nv_bfloat16*)p.add; t.out = (__nv_bfloat16*)p.out;
     t.ca = g.ca; t.ncol = g.ncol; t.wC = p.C; t.H = p.H; t.W = p.W; t.Hp = g.Hp; t.Wp = g.Wp;
     t.inv_wp = (unsigned)((1ull << 32) / (unsigned)g.Wp + 1); t.inv_hp = (unsigned)((1ull << 32) / (unsigned)g.Hp + 1);
-    t.total = g.total; t.tiles = g.tiles; t.os = mode == CONV_FWD ? p.stride : 1; t.P = p.P; t.Q = p.Q;
-    t.stages = g.stages; t.variant = g.variant; t.scale = p.scale;
+    t.G = g.G; t.gpos = g.gpos; t.sub = g.sub; t.subs = g.subs; t.units = g.units;
+    t.os = mode == CONV_FWD ? p.stride : 1; t.P = p.P; t.Q = p.Q;
+    t.stages = g.stages; t.variant = g.variant; t.smem_bytes = (int)g.smem; t.scale = p.scale;
     memcpy(host, &t, sizeof(t));
     return true;
 }
-int conv_mma_tiles(const void* h) { return ((const MmaProb*)h)->tiles; }
+int conv_mma_tiles(const void* h) { return ((const MmaProb*)h)->units; }
 int conv_mma_variant(const void* h) { return ((const MmaProb*)h)->variant; }
-size_t conv_mma_smem(const void* h) {
-    const MmaProb* t = (const MmaProb*)h;
-    const int v = t->variant, trans = (v >> 4) & 1, ksz = (v >> 5) & 3, mbw = (v >> 7) & 3;
-    const int pad = ksz / 2, halo = pad * t->Wp + pad, win_rows = 128 * mbw + 2 * halo, apitch = t->ca * 2 + 16;
-    const int wrows = trans ? t->ca : t->ncol, wcols = trans ? t->ncol : t->ca;
-    return (size_t)t->stages * ((win_rows * apitch + 127) & ~127) + (size_t)ksz * ksz * wrows * (wcols * 2 + 16) + 64;
-}
+size_t conv_mma_smem(const void* h) { return (size_t)((const MmaProb*)h)->smem_bytes; }
 
 template <int NB, int MBW, int KSZ, bool TRANS>
 static void launch_mma_inst(const void* d, dim3 grid, size_t smem, cudaStream_t s) {
     static bool configured = false;
-    if (!configured) { cudaFuncSetAttribute(conv_mma_kernel<NB, MBW, KSZ, TRANS>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024); configured = true; }
+    if (!configured) { cudaFuncSetAttribute(conv_mma_kernel<NB, MBW, KSZ, TRANS>, cudaFuncAttributeMaxDynamicSharedMemorySize, 202 * 1024); configured = true; }
     conv_mma_kernel<NB, MBW, KSZ, TRANS><<<grid, MMA_THREADS, smem, s>>>((const MmaProb*)d);
 }
 template <int NB, int MBW>
@@ -306,19 +331,15 @@ void launch_conv_mma_probs(const void* d, int nprob, int max_tiles, size_t max_s
     static int sms = 0;
     if (!sms) { int dev = 0; cudaGetDevice(&dev); cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev); if (sms < 1) sms = 148; }
     const int nb = variant & 15, trans = (variant >> 4) & 1, ksz = (variant >> 5) & 3, mbw = (variant >> 7) & 3;
-    // persistent CTAs: as many as fit on the chip at this shared-memory footprint (at most 4 per SM), over all problems
-    int per_sm = (int)((220 * 1024) / (max_smem + 1024)); if (per_sm > 4) per_sm = 4; if (per_sm < 1) per_sm = 1;
+    // persistent CTAs: as many as fit on the chip at this shared-memory footprint (at most 3 per SM), over all problems
+    int per_sm = (int)((225 * 1024) / (max_smem + 1024)); if (per_sm > 3) per_sm = 3; if (per_sm < 1) per_sm = 1;
     int gx = (per_sm * sms + nprob - 1) / nprob; if (gx > max_tiles) gx = max_tiles; if (gx < 1) gx = 1;
     const dim3 grid(gx, nprob);
-    if (mbw == 2) {
-        if (nb == 2) launch_mma_nb<2, 2>(d, grid, max_smem, ksz, trans, s);
-        else if (nb == 4) launch_mma_nb<4, 2>(d, grid, max_smem, ksz, trans, s);
-    } else {
-        if (nb == 2) launch_mma_nb<2, 1>(d, grid, max_smem, ksz, trans, s);
-        else if (nb == 4) launch_mma_nb<4, 1>(d, grid, max_smem, ksz, trans, s);
-        else if (nb == 6) launch_mma_nb<6, 1>(d, grid, max_smem, ksz, trans, s);
-        else if (nb == 8) launch_mma_nb<8, 1>(d, grid, max_smem, ksz, trans, s);
-    }
+#define MMA_CASE(N_, M_) if (nb == N_ && mbw == M_) launch_mma_nb<N_, M_>(d, grid, max_smem, ksz, trans, s); else
+    MMA_CASE(2, 1) MMA_CASE(2, 2) MMA_CASE(2, 3) MMA_CASE(4, 1) MMA_CASE(4, 2) MMA_CASE(4, 3)
+    MMA_CASE(6, 1) MMA_CASE(6, 2) MMA_CASE(8, 1) MMA_CASE(8, 2)
+    return;
+#undef MMA_CASE
 }
 
 // ------------------------------------------------------------------------------------------------ wgrad
@@ -346,6 +367,7 @@ struct alignas(16) MmaWgradProb {
     int tap_groups, taps_per_group, splits;
     int wn, stages, variant, smem_bytes;
     unsigned inv_wp, inv_hp;
+    int out_ld, out_cols;       // 1x1 problems only: row stride and valid columns of out (an im2col'ed stem); else C, C
 };
 
 template <int MB, int PPW>   // MB = K / 16; PPW = pairs of 8-column blocks a warp owns
@@ -508,7 +530,7 @@ __global__ void __launch_bounds__(256) wgrad_mma_reduce_kernel(const MmaWgradPro
 #pragma unroll
             for (int w = 1; w < 8; ++w) t += red[w][lane];
             const int c = i % C, r = i / C, k = r % K, tp = r / K;
-            p.out[((long long)k * taps + tp) * C + c] = t;
+            if (c < p.out_cols) p.out[((long long)k * taps + tp) * p.out_ld + c] = t;
         }
         __syncthreads();
     }
@@ -581,6 +603,8 @@ bool conv_wgrad_mma_fill(const ConvProb& p, int target_ctas, void* host) {
     t.tap_groups = g.tap_groups; t.taps_per_group = g.taps_per_group; t.splits = g.splits; t.wn = g.wn; t.stages = g.stages; t.variant = g.variant;
     t.inv_wp = (unsigned)((1ull << 32) / (unsigned)g.Wp + 1); t.inv_hp = (unsigned)((1ull << 32) / (unsigned)g.Hp + 1);
     t.smem_bytes = (int)g.smem;
+    t.out_ld = p.C; t.out_cols = p.C;
+    if (p.wg_ld > 0 && p.ksz == 1) { t.out_ld = p.wg_ld; t.out_cols = p.wg_cols; }
     memcpy(host, &t, sizeof(t));
     return true;
 }

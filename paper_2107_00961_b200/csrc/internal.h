@@ -23,6 +23,7 @@ struct ConvProb {
     int M, Ncol, Kred;    // GEMM extents of this mode
     int tiles_m, tiles_n, splits, ktiles_per_split;
     float scale;          // result = scale*acc + add
+    int wg_ld, wg_cols;   // wgrad of a 1x1 problem on an im2col'ed input: row stride and valid columns of dw (0: K x C dense)
     int pad_;
 };
 
@@ -59,6 +60,13 @@ inline void bn_chunking(BnProb& p, bool bf16) {
     const long long lim = (m + 1023) / 1024; if (rpc < lim) rpc = lim;
     p.rows_per_chunk = (int)rpc; p.chunks = (int)((m + rpc - 1) / rpc);
 }
+
+// im2col of a few-channel input (C * ksz * ksz <= 32): dst [N*P*Q][32] (bf16, columns (r, s, c), zero beyond), and the
+// layer's weights packed alike: w32 [K][32].
+struct ColProb {
+    const void* src; void* dst; const void* w; void* w32;
+    int N, H, W, C, ksz, stride, pad, P, Q, K, kk, pad_;
+};
 
 struct UpProb {           // zero stuffing of a stride-2 layer's dy: src [N,P,Q,K] -> dst [N,H,W,K] (bf16, K % 8 == 0)
     const void* src; void* dst; int N, H, W, K, P, Q;
@@ -115,6 +123,7 @@ void launch_head_fwd(const HeadProb* d, int nprob, int maxB, int maxC, int max_c
 void launch_head_bwd(const HeadProb* d, int nprob, int maxB, int maxC, int max_classes, long long max_elems,
                      bool bf16, cudaStream_t s);
 
+void launch_im2col(const ColProb* d, int nprob, long long max_rows, cudaStream_t s);      // kernels_ref.cu
 void launch_zero_stuff(const UpProb* d, int nprob, long long max_vecs, cudaStream_t s);   // conv_tc.cu
 
 // ---- launchers (kernels_bw.cu)

@@ -539,4 +539,41 @@ void launch_head_bwd(const HeadProb* d, int nprob, int maxB, int maxC, int max_c
     else avgpool_bwd_kernel<float><<<dim3(ew_grid(max_elems), nprob), 256, 0, s>>>(d);
 }
 
+
+// ------------------------------------------------------------------------------------------------ im2col (few-channel stem)
+// One thread per (output position, 8-column group).  The first K*4 threads also pack the weights.
+__global__ void __launch_bounds__(256) im2col_kernel(const ColProb* __restrict__ probs) {
+    const ColProb& p = probs[blockIdx.y];
+    const __nv_bfloat16* __restrict__ src = (const __nv_bfloat16*)p.src;
+    const long long rows = (long long)p.N * p.P * p.Q, total = rows * 4;
+    for (long long id = blockIdx.x * (long long)blockDim.x + threadIdx.x; id < total; id += (long long)gridDim.x * blockDim.x) {
+        const int g = (int)(id & 3); const long long row = id >> 2;
+        const int q = (int)(row % p.Q); const long long t = row / p.Q; const int pr = (int)(t % p.P); const int n = (int)(t / p.P);
+        __align__(16) __nv_bfloat16 v[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const int j = g * 8 + e;
+            float x = 0.f;
+            if (j < p.kk) {
+                const int c = j % p.C, rs = j / p.C, s = rs % p.ksz, r = rs / p.ksz;
+                const int y = pr * p.stride - p.pad + r, xx = q * p.stride - p.pad + s;
+                if (y >= 0 && y < p.H && xx >= 0 && xx < p.W) x = __bfloat162float(src[(((long long)n * p.H + y) * p.W + xx) * p.C + c]);
+            }
+            v[e] = __float2bfloat16(x);
+        }
+        *reinterpret_cast<uint4*>((__nv_bfloat16*)p.dst + row * 32 + g * 8) = *reinterpret_cast<const uint4*>(v);
+        if (id < (long long)p.K * 4) {                             // weights: w[k][kk] -> w32[k][32]
+            const int kx = (int)(id >> 2);
+            __align__(16) __nv_bfloat16 wv[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) { const int j = g * 8 + e; wv[e] = j < p.kk ? ((const __nv_bfloat16*)p.w)[(long long)kx * p.kk + j] : __float2bfloat16(0.f); }
+            *reinterpret_cast<uint4*>((__nv_bfloat16*)p.w32 + kx * 32 + g * 8) = *reinterpret_cast<const uint4*>(wv);
+        }
+    }
+}
+void launch_im2col(const ColProb* d, int nprob, long long max_rows, cudaStream_t s) {
+    long long gx = (max_rows * 4 + 255) / 256; if (gx > 148 * 16) gx = 148 * 16; if (gx < 1) gx = 1;
+    im2col_kernel<<<dim3((unsigned)gx, nprob), 256, 0, s>>>(d);
+}
+
 }  // namespace resist

@@ -95,6 +95,7 @@ struct Builder {
     // scratch shared by the operations of this sub-ResNet (they run one after another)
     double* bn_partial = nullptr; float* wgrad_partial = nullptr; size_t bn_partial_need = 0, wgrad_partial_need = 0;
     char* up_buf = nullptr; size_t up_need = 0; const void* up_src = nullptr;      // zero-stuffed dy of the current stride-2 layer
+    char* col_buf = nullptr; char* col_w = nullptr;                                 // im2col of the input images and the stem's weights packed alike
     char* gbuf[6] = {}; bool gused[6] = {}; size_t gbig = 0;
     float* logits = nullptr;
     long long flops = 0; int n_tc = 0, n_cc = 0;
@@ -167,6 +168,38 @@ struct Builder {
         if (mode == CONV_WGRAD && p.splits > 1) { Op r = op; r.key = key + 1; r.kind = OP_SPLITK; r.patch_images = 0; ops->push_back(r); }
     }
 
+    // A stem with few input channels (C * k * k <= 32, bf16): the images are expanded once per step to rows of 32
+    // columns, and forward and wgrad become 1x1 problems with 32 input channels on the warp-MMA kernels.
+    bool stem_as_im2col(const ConvRef& cr) const {
+        return ctx->opts.dtype == RESIST_BF16 && ctx->opts.conv_backend != RESIST_CONV_CUDA_CORES && ctx->opts.conv_backend != RESIST_CONV_TCGEN05 &&
+               cr.cin * cr.k * cr.k <= 32 && cr.cout % 16 == 0 && cr.cout <= 64;
+    }
+    void stem_im2col(long long key, const ConvRef& cr, int N, int H, int Wd) {
+        const int P = out_dim(H, cr.k, cr.stride), Q = out_dim(Wd, cr.k, cr.stride);
+        col_buf = (char*)take((size_t)N * P * Q * 64); col_w = (char*)take((size_t)cr.cout * 64);
+        Op u{}; u.key = key; u.sub = sub; u.kind = OP_IM2COL;
+        u.col = ColProb{nullptr, col_buf, CW(cr.w), col_w, N, H, Wd, cr.cin, cr.k, cr.stride, (cr.k - 1) / 2, P, Q, cr.cout, cr.cin * cr.k * cr.k, 0};
+        ops->push_back(u);
+    }
+    // the stem as a 1x1 problem on the im2col'ed images: forward (out = y) or wgrad (dy given; dw goes to the stem's gradient)
+    void stem_conv(long long key, int mode, const ConvRef& cr, const void* dy, void* out, int N, int H, int Wd) {
+        const int P = out_dim(H, cr.k, cr.stride), Q = out_dim(Wd, cr.k, cr.stride);
+        Op op{}; op.key = key; op.sub = sub; op.kind = mode == CONV_FWD ? OP_CONV_FWD : OP_CONV_WGRAD;
+        ConvProb& p = op.conv;
+        p.N = N; p.H = P; p.W = Q; p.C = 32; p.K = cr.cout; p.ksz = 1; p.stride = 1; p.pad = 0; p.P = P; p.Q = Q; p.scale = 1.f;
+        const long long rows = (long long)N * P * Q;
+        p.act = col_buf;
+        if (mode == CONV_FWD) { p.wgt = col_w; p.out = out; p.M = (int)rows; p.Ncol = p.K; p.Kred = 32; }
+        else { p.wgt = dy; p.out = G() + cr.w; p.M = p.K; p.Ncol = 32; p.Kred = (int)rows; p.wg_ld = cr.cin * cr.k * cr.k; p.wg_cols = p.wg_ld; }
+        p.tiles_m = (p.M + 63) / 64; p.tiles_n = (p.Ncol + 63) / 64; p.splits = 1; p.ktiles_per_split = (p.Kred + 15) / 16;
+        flops += 2LL * rows * p.K * cr.k * cr.k * cr.cin;
+        size_t pb = 0;
+        op.backend = pick_backend(p, mode, wgrad_target_ctas(ctx), &pb, RESIST_CONV_WARP_MMA);
+        if (mode == CONV_WGRAD) { wgrad_partial_need = std::max(wgrad_partial_need, pb); p.partial = wgrad_partial; }
+        ++n_tc;
+        ops->push_back(op);
+    }
+
     // forward BN+ReLU: statistics (or running statistics in evaluation) then apply
     float* bn_fwd(long long key, const void* x, void* a, const BNRef& r, long long m) {
         float* stat = (float*)take((size_t)4 * r.c * 4);
@@ -211,7 +244,9 @@ static size_t unroll_subnet(resist_ctx* ctx, Builder& bd, const std::vector<char
     const int Hs = out_dim(A.in_h, A.stem_k, A.stem_stride), Ws = out_dim(A.in_w, A.stem_k, A.stem_stride);
     const long long m_stem = (long long)B * Hs * Ws;
     void* stem_y = bd.act(m_stem * A.stem_cout); void* stem_a = nullptr; void* stem_p = nullptr; int* stem_arg = nullptr; float* stem_stat = nullptr;
-    bd.conv(0, CONV_FWD, nullptr, L.stem, nullptr, nullptr, stem_y, B, A.in_h, A.in_w, 1.f, true);
+    const bool stem_col = bd.stem_as_im2col(L.stem);
+    if (stem_col) { bd.stem_im2col(0, L.stem, B, A.in_h, A.in_w); bd.stem_conv(0, CONV_FWD, L.stem, nullptr, stem_y, B, A.in_h, A.in_w); }
+    else bd.conv(0, CONV_FWD, nullptr, L.stem, nullptr, nullptr, stem_y, B, A.in_h, A.in_w, 1.f, true);
     void* cur = stem_y; int cH = Hs, cW = Ws, cC = A.stem_cout;
     if (A.stem_bn_relu) { stem_a = bd.act(m_stem * cC); stem_stat = bd.bn_fwd(1, stem_y, stem_a, L.stem_bn, m_stem); cur = stem_a; }
     if (A.stem_maxpool) {
@@ -329,7 +364,8 @@ static size_t unroll_subnet(resist_ctx* ctx, Builder& bd, const std::vector<char
         bd.ops->push_back(op); bd.grel(g_cur); g_cur = g;
     }
     if (A.stem_bn_relu) { const int g = bd.gtake(); bd.bn_bwd(BWD_END + 1, stem_y, bd.gbuf[g_cur], bd.gbuf[g], nullptr, L.stem_bn, stem_stat, m_stem); bd.grel(g_cur); g_cur = g; }
-    bd.conv(BWD_END + 3, CONV_WGRAD, nullptr, L.stem, bd.gbuf[g_cur], nullptr, nullptr, B, A.in_h, A.in_w, 1.f, true);
+    if (stem_col) bd.stem_conv(BWD_END + 3, CONV_WGRAD, L.stem, bd.gbuf[g_cur], nullptr, B, A.in_h, A.in_w);
+    else bd.conv(BWD_END + 3, CONV_WGRAD, nullptr, L.stem, bd.gbuf[g_cur], nullptr, nullptr, B, A.in_h, A.in_w, 1.f, true);
     return bd.off;
 }
 
@@ -357,14 +393,15 @@ static std::vector<char> present_of(const resist_ctx* ctx, int sub) {
 }
 
 static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool single, cudaStream_t st) {
-    // equal keys of different sub-ResNets become neighbours; a zero-stuffing op shares the key of the first
+    // equal keys of different sub-ResNets become neighbours; a zero-stuffing or im2col op shares the key of the first
     // convolution that reads its output and sorts in front of it
     std::stable_sort(ops.begin(), ops.end(), [](const Op& a, const Op& b) {
         if (a.key != b.key) return a.key < b.key;
-        if ((a.kind == OP_UPSAMPLE) != (b.kind == OP_UPSAMPLE)) return a.kind == OP_UPSAMPLE;
+        const bool pa = a.kind == OP_UPSAMPLE || a.kind == OP_IM2COL, pb = b.kind == OP_UPSAMPLE || b.kind == OP_IM2COL;
+        if (pa != pb) return pa;
         return a.backend < b.backend; });
     const double es = ctx->opts.dtype == RESIST_BF16 ? 2.0 : 4.0;
-    std::vector<ConvProb> conv; std::vector<BnProb> bn; std::vector<PoolProb> pool; std::vector<HeadProb> head; std::vector<UpProb> up;
+    std::vector<ConvProb> conv; std::vector<BnProb> bn; std::vector<PoolProb> pool; std::vector<HeadProb> head; std::vector<UpProb> up; std::vector<ColProb> col;
     const size_t tcb = conv_tc_prob_bytes(); std::vector<char> tc; int n_tc = 0;
     const size_t wtcb = conv_wgrad_tc_prob_bytes(); std::vector<char> wtc; int n_wtc = 0;
     const size_t mmb = conv_mma_prob_bytes(); std::vector<char> mm; int n_mm = 0;
@@ -455,6 +492,14 @@ static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool s
                       else if (o.kind == OP_BN_BWD_REDUCE) L.bytes += 2 * es * e;
                       else L.bytes += es * e * (o.bn.add ? 4 : 3); }
                     break; }
+                case OP_IM2COL: {
+                    if (k == i) L.first = (int)col.size();
+                    sites.push_back({2, (int)col.size(), 0, 0, slot});
+                    col.push_back(o.col);
+                    const double rows = (double)o.col.N * o.col.P * o.col.Q;
+                    L.max_elems = std::max<long long>(L.max_elems, (long long)rows);
+                    L.bytes += 64.0 * rows + 2.0 * o.col.N * o.col.H * o.col.W * o.col.C;
+                    break; }
                 case OP_UPSAMPLE: {
                     if (k == i) L.first = (int)up.size();
                     up.push_back(o.up);
@@ -500,17 +545,20 @@ static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool s
     const size_t o_wtc = off;  off += align_up(wtc.size(), 256);
     const size_t o_up = off;   off += align_up(up.size() * sizeof(UpProb), 256);
     const size_t o_mm = off;   off += align_up(mm.size(), 256);
+    const size_t o_col = off;  off += align_up(col.size() * sizeof(ColProb), 256);
     const size_t o_wmm = off;  off += align_up(wmm.size(), 256);
     ctx_free(ctx, plan.d_blob);
     plan.d_blob = ctx_alloc(ctx, off + 256); plan.blob_bytes = off;
     if (!plan.d_blob) { ctx->err = "allocator returned NULL for the launch plan"; return RESIST_ENOMEM; }
     char* base = (char*)plan.d_blob;
     plan.d_conv = (ConvProb*)(base + o_conv); plan.d_bn = (BnProb*)(base + o_bn); plan.d_pool = (PoolProb*)(base + o_pool);
+    plan.d_col = (ColProb*)(base + o_col);
     plan.d_head = (HeadProb*)(base + o_head); plan.d_sites = (PatchSite*)(base + o_site); plan.d_sgd = (Segment*)(base + o_seg);
     std::vector<PatchSite> dsites;
     for (const HostSite& h : sites) {
         PatchSite s{}; s.what = h.what; s.sub = h.sub;
         if (h.arr == 0) s.where = (void**)&plan.d_conv[h.idx].act;
+        else if (h.arr == 2) s.where = (void**)&plan.d_col[h.idx].src;
         else if (h.field == 0) s.where = (void**)&plan.d_head[h.idx].labels;
         else if (h.field == 1) s.where = (void**)&plan.d_head[h.idx].loss_user;
         else if (h.field == 2) s.where = (void**)&plan.d_head[h.idx].logits_user;
@@ -529,6 +577,7 @@ static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool s
     if (!wtc.empty()) memcpy(host.data() + o_wtc, wtc.data(), wtc.size());
     plan.d_wtc = base + o_wtc; plan.wtc_stride = wtcb;
     if (!up.empty()) memcpy(host.data() + o_up, up.data(), up.size() * sizeof(UpProb));
+    if (!col.empty()) memcpy(host.data() + o_col, col.data(), col.size() * sizeof(ColProb));
     plan.d_up = (UpProb*)(base + o_up);
     if (!mm.empty()) memcpy(host.data() + o_mm, mm.data(), mm.size());
     if (!wmm.empty()) memcpy(host.data() + o_wmm, wmm.data(), wmm.size());
@@ -602,6 +651,7 @@ static int run_plan(resist_ctx* ctx, Plan& plan, const PatchArgs& pa, bool updat
             case OP_HEAD_FWD: pk = PK_HEAD_FWD; nk = 3; break;
             case OP_HEAD_BWD: pk = PK_HEAD_BWD; nk = 3; break;
             case OP_UPSAMPLE: pk = PK_UPSAMPLE; break;
+            case OP_IM2COL: pk = PK_IM2COL; break;
         }
         pf.begin(pk, nk, L.bytes, L.flops, st);
         switch (L.kind) {
@@ -623,6 +673,7 @@ static int run_plan(resist_ctx* ctx, Plan& plan, const PatchArgs& pa, bool updat
             case OP_HEAD_FWD: launch_head_fwd(plan.d_head + L.first, L.count, L.max_b, L.max_c, L.max_classes, bf, st); n_launch += 3; break;
             case OP_HEAD_BWD: launch_head_bwd(plan.d_head + L.first, L.count, L.max_b, L.max_c, L.max_classes, L.max_elems, bf, st); n_launch += 3; break;
             case OP_UPSAMPLE: launch_zero_stuff(plan.d_up + L.first, L.count, L.max_elems, st); ++n_launch; break;
+            case OP_IM2COL: launch_im2col(plan.d_col + L.first, L.count, L.max_elems, st); ++n_launch; break;
         }
         pf.end(st);
     }

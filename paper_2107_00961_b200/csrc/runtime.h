@@ -18,13 +18,13 @@ Layout make_layout(const resist_arch& a, const std::vector<resist_block>& blocks
 
 enum OpKind {
     OP_CONV_FWD, OP_CONV_DGRAD, OP_CONV_WGRAD, OP_SPLITK, OP_BN_STATS, OP_BN_APPLY, OP_BN_BWD_REDUCE, OP_BN_BWD_APPLY,
-    OP_POOL_FWD, OP_POOL_BWD, OP_HEAD_FWD, OP_HEAD_BWD, OP_UPSAMPLE
+    OP_POOL_FWD, OP_POOL_BWD, OP_HEAD_FWD, OP_HEAD_BWD, OP_UPSAMPLE, OP_IM2COL
 };
 
 // One operation of one sub-ResNet, keyed so that equal keys of different sub-ResNets share a launch.
 struct Op {
     long long key; OpKind kind; int sub;
-    ConvProb conv; BnProb bn; PoolProb pool; HeadProb head; UpProb up;
+    ConvProb conv; BnProb bn; PoolProb pool; HeadProb head; UpProb up; ColProb col;
     int backend;          // convolutions: 0 = CUDA cores, 1 = tensor cores
     int patch_images;     // conv.act must be replaced by the caller's image pointer
 };
@@ -40,7 +40,7 @@ struct Launch {
 enum ProfKind {
     PK_CONV_FWD_CC, PK_CONV_DGRAD_CC, PK_CONV_WGRAD_CC, PK_CONV_FWD_TC, PK_CONV_DGRAD_TC, PK_CONV_WGRAD_TC, PK_SPLITK,
     PK_BN_STATS, PK_BN_APPLY, PK_BN_BWD_REDUCE, PK_BN_BWD_APPLY, PK_POOL_FWD, PK_POOL_BWD, PK_HEAD_FWD, PK_HEAD_BWD,
-    PK_SGD, PK_PATCH, PK_SCATTER, PK_AGGREGATE, PK_UPSAMPLE, PK_CONV_FWD_MMA, PK_CONV_DGRAD_MMA, PK_CONV_WGRAD_MMA, PK_COUNT
+    PK_SGD, PK_PATCH, PK_SCATTER, PK_AGGREGATE, PK_UPSAMPLE, PK_CONV_FWD_MMA, PK_CONV_DGRAD_MMA, PK_CONV_WGRAD_MMA, PK_IM2COL, PK_COUNT
 };
 struct Profiler {
     bool on = false;
@@ -63,7 +63,7 @@ struct Plan {
     bool valid = false; int B = 0; unsigned long long generation = 0; int sub = -1;   // sub = -1: all sub-ResNets grouped
     std::vector<Launch> launches;
     void* d_blob = nullptr; size_t blob_bytes = 0;            // descriptor arrays in one device allocation
-    ConvProb* d_conv = nullptr; BnProb* d_bn = nullptr; PoolProb* d_pool = nullptr; HeadProb* d_head = nullptr; UpProb* d_up = nullptr;
+    ConvProb* d_conv = nullptr; BnProb* d_bn = nullptr; PoolProb* d_pool = nullptr; HeadProb* d_head = nullptr; UpProb* d_up = nullptr; ColProb* d_col = nullptr;
     PatchSite* d_sites = nullptr; int nsites = 0;
     void* d_tc = nullptr; size_t tc_stride = 0;              // tensor-core convolution descriptors
     void* d_wtc = nullptr; size_t wtc_stride = 0;            // tensor-core wgrad descriptors
