@@ -635,7 +635,28 @@ static int run_plan(resist_ctx* ctx, Plan& plan, const PatchArgs& pa, bool updat
     long long n_launch = 0;
     Profiler& pf = ctx->prof;
     if (plan.nsites) { pf.begin(PK_PATCH, 1, 0, 0, st); patch_kernel<<<(plan.nsites + 63) / 64, 64, 0, st>>>(plan.d_sites, plan.nsites, pa); pf.end(st); ++n_launch; }
+    // A layer's weight gradient and data gradient both read dy and are independent of each other: the weight gradients
+    // (and their partial-sum reductions) go to a second stream, one after another, while the main stream carries on
+    // with the data gradient and the BN reduction that follows it.  Everything else may write a buffer that a weight
+    // gradient still reads (gradient buffers are recycled), so the main stream first waits for the second.  Per-kernel
+    // profiling keeps everything on one stream.
+    const bool overlap = !pf.on && update;
+    if (overlap && !ctx->side_stream) {
+        if (cudaStreamCreateWithFlags(&ctx->side_stream, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&ctx->ev_side_done, cudaEventDisableTiming) != cudaSuccess) { ctx->err = "cannot create the second stream"; return RESIST_ECUDA; }
+    }
+    bool side_pending = false;
+    const cudaStream_t main_st = st;
     for (const Launch& L : plan.launches) {
+        const bool on_side = overlap && (L.kind == OP_CONV_WGRAD || (L.kind == OP_SPLITK && side_pending));
+        if (on_side) {
+            cudaEventRecord(ctx->ev_fork, main_st); cudaStreamWaitEvent(ctx->side_stream, ctx->ev_fork, 0);
+            st = ctx->side_stream;
+        } else {
+            st = main_st;
+            if (side_pending && L.kind != OP_CONV_DGRAD && L.kind != OP_BN_BWD_REDUCE) { cudaStreamWaitEvent(main_st, ctx->ev_side_done, 0); side_pending = false; }
+        }
         int pk = 0, nk = 1;
         switch (L.kind) {
             case OP_CONV_FWD: pk = L.backend >= 200 ? PK_CONV_FWD_MMA : L.backend ? PK_CONV_FWD_TC : PK_CONV_FWD_CC; break;
@@ -676,7 +697,10 @@ static int run_plan(resist_ctx* ctx, Plan& plan, const PatchArgs& pa, bool updat
             case OP_IM2COL: launch_im2col(plan.d_col + L.first, L.count, L.max_elems, st); ++n_launch; break;
         }
         pf.end(st);
+        if (on_side) { cudaEventRecord(ctx->ev_side_done, ctx->side_stream); side_pending = true; }
     }
+    st = main_st;
+    if (side_pending) cudaStreamWaitEvent(main_st, ctx->ev_side_done, 0);
     if (update && plan.sgd_chunks) {
         pf.begin(PK_SGD, 1, (bf ? 22.0 : 20.0) * plan.sgd_params, 0, st);
         launch_sgd(plan.d_sgd, plan.n_sgd_seg, plan.sgd_chunks, ctx->pa, lr, ctx->opts.momentum, ctx->opts.weight_decay, bf, st);

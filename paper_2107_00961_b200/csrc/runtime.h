@@ -97,5 +97,7 @@ struct resist_ctx {
     resist_step_info info{};
     resist::Profiler prof;
     int sm_count = 148;
+    // weight gradients run beside the data gradient of the same layer on a second stream (created on first use)
+    cudaStream_t side_stream = nullptr; cudaEvent_t ev_fork = nullptr, ev_side_done = nullptr;
     std::string err;
 };
