@@ -47,7 +47,7 @@ struct BnProb {
 };
 
 // How the rows of a BN problem are cut into chunks (one CTA each) and whether the vector path applies.
-inline void bn_chunking(BnProb& p, bool bf16) {
+inline void bn_chunking(BnProb& p, bool bf16, int target_chunks = 0) {
     const int C = p.C; const long long m = p.m;
     const int G = C / 8;
     const bool pow2 = G > 0 && (G & (G - 1)) == 0;
@@ -58,6 +58,10 @@ inline void bn_chunking(BnProb& p, bool bf16) {
     if (p.vec) { const int R = 256 / G; rpc = (long long)R * 16; }
     else { const int nl = C < 256 ? C : 256, R = 256 / nl; rpc = (long long)R * 32; }
     const long long lim = (m + 1023) / 1024; if (rpc < lim) rpc = lim;
+    if (p.vec && target_chunks > 0 && (m + rpc - 1) / rpc < target_chunks) {      // more, smaller chunks (whole sweeps of the CTA's rows)
+        const int R = 256 / G;
+        rpc = ((m + target_chunks - 1) / target_chunks + R - 1) / R * R; if (rpc < R) rpc = R;
+    }
     p.rows_per_chunk = (int)rpc; p.chunks = (int)((m + rpc - 1) / rpc);
 }
 
@@ -123,6 +127,8 @@ void launch_head_fwd(const HeadProb* d, int nprob, int maxB, int maxC, int max_c
 void launch_head_bwd(const HeadProb* d, int nprob, int maxB, int maxC, int max_classes, long long max_elems,
                      bool bf16, cudaStream_t s);
 
+// statistics, finalisation and apply of BN+ReLU in one cooperative launch (bf16 vector path, training mode); false if the grid cannot be co-resident
+bool launch_bn_fused(const BnProb* d, int nprob, int max_chunks, int backward, cudaStream_t s);   // kernels_ref.cu
 void launch_im2col(const ColProb* d, int nprob, long long max_rows, cudaStream_t s);      // kernels_ref.cu
 void launch_zero_stuff(const UpProb* d, int nprob, long long max_vecs, cudaStream_t s);   // conv_tc.cu
 

@@ -2,8 +2,10 @@
 // fp32 arithmetic.  It is the whole path of the fp32 mode, and in bf16 mode it runs whatever the
 // tensor-core kernels do not take (3-channel stems, odd shapes) and the small head/loss kernels.
 // All reductions have a fixed order: results are reproducible run to run.
+#include <cooperative_groups.h>
 #include "internal.h"
 
+namespace cg = cooperative_groups;
 namespace resist {
 
 template <class T> __device__ __forceinline__ float ldf(const void* p, long long i);
@@ -227,8 +229,8 @@ __device__ void bn_reduce_vec(const BnProb& p) {
     }
 }
 
-template <int MODE>   // 0: forward apply; 1: backward apply
-__device__ void bn_apply_vec(const BnProb& p) {
+template <int MODE>   // 0: forward apply; 1: backward apply.  stat: [4][C] as BnProb::stat, in global or shared memory
+__device__ void bn_apply_vec(const BnProb& p, const float* __restrict__ stat) {
     const int C = p.C, G = C >> 3;
     const long long nv = p.m * G;
     const float inv_m = 1.f / (float)p.m;
@@ -240,8 +242,8 @@ __device__ void bn_apply_vec(const BnProb& p) {
     for (long long v = blockIdx.x * (long long)blockDim.x + threadIdx.x; v < nv; v += stride) {
         const int c0 = (int)(v & (long long)(G - 1)) * 8;          // G is a power of two
         float x[8], o[8]; unpack8(xv[v], x);
-        const float4 m0 = *reinterpret_cast<const float4*>(p.stat + c0), m1 = *reinterpret_cast<const float4*>(p.stat + c0 + 4);
-        const float4 i0 = *reinterpret_cast<const float4*>(p.stat + C + c0), i1 = *reinterpret_cast<const float4*>(p.stat + C + c0 + 4);
+        const float4 m0 = *reinterpret_cast<const float4*>(stat + c0), m1 = *reinterpret_cast<const float4*>(stat + c0 + 4);
+        const float4 i0 = *reinterpret_cast<const float4*>(stat + C + c0), i1 = *reinterpret_cast<const float4*>(stat + C + c0 + 4);
         const float4 g0 = *reinterpret_cast<const float4*>(p.gamma + c0), g1 = *reinterpret_cast<const float4*>(p.gamma + c0 + 4);
         const float4 b0 = *reinterpret_cast<const float4*>(p.beta + c0), b1 = *reinterpret_cast<const float4*>(p.beta + c0 + 4);
         const float mean[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w}, istd[8] = {i0.x, i0.y, i0.z, i0.w, i1.x, i1.y, i1.z, i1.w};
@@ -251,8 +253,8 @@ __device__ void bn_apply_vec(const BnProb& p) {
             for (int j = 0; j < 8; ++j) { const float z = (x[j] - mean[j]) * istd[j] * ga[j] + be[j]; o[j] = z > 0.f ? z : 0.f; }
         } else {
             float d[8]; unpack8(dv[v], d);
-            const float4 s0 = *reinterpret_cast<const float4*>(p.stat + 2 * C + c0), s1 = *reinterpret_cast<const float4*>(p.stat + 2 * C + c0 + 4);
-            const float4 t0 = *reinterpret_cast<const float4*>(p.stat + 3 * C + c0), t1 = *reinterpret_cast<const float4*>(p.stat + 3 * C + c0 + 4);
+            const float4 s0 = *reinterpret_cast<const float4*>(stat + 2 * C + c0), s1 = *reinterpret_cast<const float4*>(stat + 2 * C + c0 + 4);
+            const float4 t0 = *reinterpret_cast<const float4*>(stat + 3 * C + c0), t1 = *reinterpret_cast<const float4*>(stat + 3 * C + c0 + 4);
             const float sb[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w}, sg[8] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
@@ -343,7 +345,7 @@ __global__ void bn_finalize_kernel(const BnProb* __restrict__ probs) {
 template <class T>
 __global__ void __launch_bounds__(256) bn_apply_kernel(const BnProb* __restrict__ probs) {
     const BnProb& p = probs[blockIdx.y];
-    if (p.vec) { bn_apply_vec<0>(p); return; }
+    if (p.vec) { bn_apply_vec<0>(p, p.stat); return; }
     const long long n = p.m * p.C;
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
         const int c = (int)(i % p.C);
@@ -355,7 +357,7 @@ __global__ void __launch_bounds__(256) bn_apply_kernel(const BnProb* __restrict_
 template <class T>
 __global__ void __launch_bounds__(256) bn_bwd_apply_kernel(const BnProb* __restrict__ probs) {
     const BnProb& p = probs[blockIdx.y];
-    if (p.vec) { bn_apply_vec<1>(p); return; }
+    if (p.vec) { bn_apply_vec<1>(p, p.stat); return; }
     const long long n = p.m * p.C;
     const float inv_m = 1.f / (float)p.m;
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
@@ -367,6 +369,66 @@ __global__ void __launch_bounds__(256) bn_bwd_apply_kernel(const BnProb* __restr
         if (p.add) v += ldf<T>(p.add, i);
         stf<T>(p.dx, i, v);
     }
+}
+
+
+// ------------------------------------------------------------------------------------------------ fused BN+ReLU (cooperative)
+// One launch per BN layer and direction: partial sums per chunk, a grid-wide barrier, then EVERY CTA adds the
+// partials of its problem in the same fixed order (so all CTAs hold identical statistics without a second barrier;
+// CTA 0 of the problem also stores them) and takes its share of the elementwise pass, whose re-read of x comes
+// from L2.  bf16 vector path, training mode only.
+template <int MODE>
+__global__ void __launch_bounds__(256) bn_fused_kernel(const BnProb* __restrict__ probs) {
+    const BnProb& p = probs[blockIdx.y];
+    __shared__ __align__(16) float s_stat[4 * 512];               // callers keep C <= 512
+    if ((int)blockIdx.x < p.chunks) bn_reduce_vec<MODE>(p);
+    __threadfence();
+    cg::this_grid().sync();
+    const int C = p.C, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int c = warp; c < C; c += 8) {
+        // lane l adds chunks l, l+32, ... in order, then a fixed butterfly over the lanes
+        double a0 = 0.0, a1 = 0.0;
+        for (int k = lane; k < p.chunks; k += 32) { a0 += __ldcg(p.partial + ((long long)k * 2 + 0) * C + c); a1 += __ldcg(p.partial + ((long long)k * 2 + 1) * C + c); }
+        for (int d = 16; d; d >>= 1) { a0 += __shfl_xor_sync(0xffffffffu, a0, d); a1 += __shfl_xor_sync(0xffffffffu, a1, d); }
+        if (lane != 0) continue;
+        if (MODE == 0) {
+            const double m = (double)p.m, dm = a0 / m;             // sums are of x - x[0,c]
+            double var = a1 / m - dm * dm; if (var < 0.0) var = 0.0;
+            const double mean = dm + (double)__bfloat162float(((const __nv_bfloat16*)p.x)[c]);
+            const float fm = (float)mean, fi = (float)(1.0 / sqrt(var + (double)p.eps));
+            s_stat[c] = fm; s_stat[C + c] = fi;
+            if (blockIdx.x == 0) {
+                p.stat[c] = fm; p.stat[C + c] = fi;
+                if (p.run_mean) {
+                    const double unb = p.m > 1 ? var * m / (m - 1.0) : var, mo = (double)p.momentum;
+                    p.run_mean[c] = (float)((1.0 - mo) * (double)p.run_mean[c] + mo * mean);
+                    p.run_var[c] = (float)((1.0 - mo) * (double)p.run_var[c] + mo * unb);
+                }
+            }
+        } else {
+            s_stat[c] = p.stat[c]; s_stat[C + c] = p.stat[C + c];
+            s_stat[2 * C + c] = (float)a0; s_stat[3 * C + c] = (float)a1;
+            if (blockIdx.x == 0) { p.stat[2 * C + c] = (float)a0; p.stat[3 * C + c] = (float)a1; p.dbeta[c] = (float)a0; p.dgamma[c] = (float)a1; }
+        }
+    }
+    __syncthreads();
+    bn_apply_vec<MODE>(p, s_stat);
+}
+
+bool launch_bn_fused(const BnProb* d, int nprob, int max_chunks, int backward, cudaStream_t s) {
+    static int cap[2] = {0, 0};                                    // co-resident CTAs of each kernel on this device
+    if (!cap[backward]) {
+        int dev = 0, sms = 0, per = 0; cudaGetDevice(&dev); cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (backward) cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per, bn_fused_kernel<1>, 256, 0);
+        else cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per, bn_fused_kernel<0>, 256, 0);
+        cap[backward] = per * sms > 0 ? per * sms : -1;
+    }
+    if ((long long)max_chunks * nprob > cap[backward]) return false;
+    void* args[] = {(void*)&d};
+    const dim3 grid(max_chunks, nprob), block(256);
+    const cudaError_t e = backward ? cudaLaunchCooperativeKernel((void*)bn_fused_kernel<1>, grid, block, args, 0, s)
+                                   : cudaLaunchCooperativeKernel((void*)bn_fused_kernel<0>, grid, block, args, 0, s);
+    return e == cudaSuccess;
 }
 
 static int ew_grid(long long n) { long long g = (n + 255) / 256; if (g > 148 * 16) g = 148 * 16; if (g < 1) g = 1; return (int)g; }

@@ -102,8 +102,11 @@ struct Builder {
 
     void* take(size_t bytes) { off = align_up(off, 256); void* p = base ? base + off : nullptr; off += bytes; return p; }
     void* act(long long elems) { size_t b = (size_t)elems * es; if (b > gbig) gbig = b; return take(b); }
-    int gtake() { for (int i = 0; i < 6; ++i) if (!gused[i]) { gused[i] = true; return i; } return -1; }
-    void grel(int i) { if (i >= 0) gused[i] = false; }
+    // gradient buffers are handed out oldest-released first: a weight gradient that still reads a released buffer on
+    // the second stream then has several layers' time before the buffer is written again
+    int gstamp[6] = {}; int gclock = 0;
+    int gtake() { int best = -1; for (int i = 0; i < 6; ++i) if (!gused[i] && (best < 0 || gstamp[i] < gstamp[best])) best = i; if (best >= 0) gused[best] = true; return best; }
+    void grel(int i) { if (i >= 0) { gused[i] = false; gstamp[i] = ++gclock; } }
 
     float* W() const { return ctx->pa.w + (long long)copy * ctx->pa.n; }
     float* G() const { return ctx->pa.g + (long long)copy * ctx->pa.n; }
@@ -200,6 +203,8 @@ struct Builder {
         ops->push_back(op);
     }
 
+    // chunks per BN problem that give the fused (cooperative) kernels about two CTAs per SM over all sub-ResNets
+    int fused_chunks() const { return std::max(8, 2 * ctx->sm_count / std::max(1, ctx->S)); }
     // forward BN+ReLU: statistics (or running statistics in evaluation) then apply
     float* bn_fwd(long long key, const void* x, void* a, const BNRef& r, long long m) {
         float* stat = (float*)take((size_t)4 * r.c * 4);
@@ -208,9 +213,10 @@ struct Builder {
         p.x = x; p.a = a; p.gamma = W() + r.g; p.beta = W() + r.b; p.dgamma = G() + r.g; p.dbeta = G() + r.b;
         p.run_mean = Bf() + r.buf; p.run_var = Bf() + r.buf + r.c; p.stat = stat; p.m = m; p.C = r.c;
         p.eps = ctx->opts.bn_eps; p.momentum = ctx->opts.bn_momentum; p.eval = eval ? 1 : 0;
-        bn_chunking(p, ctx->opts.dtype == RESIST_BF16);
+        bn_chunking(p, ctx->opts.dtype == RESIST_BF16, fused_chunks());
         bn_partial_need = std::max(bn_partial_need, (size_t)p.chunks * 2 * r.c * 8);
         p.partial = bn_partial;
+        if (p.vec && !eval && r.c <= 512) { op.kind = OP_BN_FWD_FUSED; ops->push_back(op); return stat; }   // one cooperative launch
         ops->push_back(op);
         op.key = key + 1; op.kind = OP_BN_APPLY; ops->push_back(op);
         return stat;
@@ -220,8 +226,10 @@ struct Builder {
         BnProb& p = op.bn;
         p.x = x; p.da = da; p.dx = dx; p.add = add; p.gamma = W() + r.g; p.beta = W() + r.b; p.dgamma = G() + r.g; p.dbeta = G() + r.b;
         p.stat = stat; p.m = m; p.C = r.c; p.eps = ctx->opts.bn_eps; p.momentum = ctx->opts.bn_momentum; p.eval = 0;
-        bn_chunking(p, ctx->opts.dtype == RESIST_BF16);
+        bn_chunking(p, ctx->opts.dtype == RESIST_BF16, fused_chunks());
+        bn_partial_need = std::max(bn_partial_need, (size_t)p.chunks * 2 * r.c * 8);
         p.partial = bn_partial;
+        if (p.vec && r.c <= 512) { op.kind = OP_BN_BWD_FUSED; ops->push_back(op); return; }
         ops->push_back(op);
         op.key = key + 1; op.kind = OP_BN_BWD_APPLY; ops->push_back(op);
     }
@@ -409,6 +417,7 @@ static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool s
     struct HostSite { int arr; int idx; int field; int what; int sub; };
     std::vector<HostSite> sites;
     plan.launches.clear();
+    std::vector<const void*> inflight;                         // tensors read by the weight gradients not yet joined
     for (size_t i = 0; i < ops.size();) {
         size_t j = i;
         while (j < ops.size() && ops[j].key == ops[i].key && ops[j].kind == ops[i].kind && ops[j].backend == ops[i].backend) ++j;
@@ -481,7 +490,7 @@ static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool s
                         if (o.kind == OP_CONV_WGRAD) L.bytes += es * (in_e + out_e) + 4.0 * w_e;
                         else L.bytes += es * (in_e + out_e + w_e + (p.add ? (o.kind == OP_CONV_FWD ? out_e : in_e) : 0.0)); }
                     break; }
-                case OP_BN_STATS: case OP_BN_APPLY: case OP_BN_BWD_REDUCE: case OP_BN_BWD_APPLY: {
+                case OP_BN_STATS: case OP_BN_APPLY: case OP_BN_BWD_REDUCE: case OP_BN_BWD_APPLY: case OP_BN_FWD_FUSED: case OP_BN_BWD_FUSED: {
                     if (k == i) L.first = (int)bn.size();
                     bn.push_back(o.bn);
                     L.gx = std::max(L.gx, o.bn.chunks); L.max_c = std::max(L.max_c, o.bn.C);
@@ -490,6 +499,8 @@ static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool s
                       if (o.kind == OP_BN_STATS) L.bytes += o.bn.eval ? 0.0 : es * e;
                       else if (o.kind == OP_BN_APPLY) L.bytes += 2 * es * e;
                       else if (o.kind == OP_BN_BWD_REDUCE) L.bytes += 2 * es * e;
+                      else if (o.kind == OP_BN_FWD_FUSED) L.bytes += 2 * es * e;          // x once from HBM (the second read is an L2 hit), a once
+                      else if (o.kind == OP_BN_BWD_FUSED) L.bytes += es * e * (o.bn.add ? 4 : 3);
                       else L.bytes += es * e * (o.bn.add ? 4 : 3); }
                     break; }
                 case OP_IM2COL: {
@@ -525,6 +536,28 @@ static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool s
                     L.max_elems = std::max<long long>(L.max_elems, (long long)p.B * p.HW * p.C);
                     L.bytes += es * (double)p.B * p.HW * p.C + 4.0 * p.classes * p.C;
                     break; }
+            }
+        }
+        // what a weight gradient in flight on the second stream reads, and whether this launch writes any of it
+        {
+            std::vector<const void*> wr; bool always = false;
+            for (size_t k = i; k < j; ++k) {
+                const Op& o = ops[k];
+                switch (o.kind) {
+                    case OP_CONV_FWD: case OP_CONV_DGRAD: wr.push_back(o.conv.out); break;
+                    case OP_CONV_WGRAD: case OP_SPLITK: break;
+                    case OP_BN_STATS: case OP_BN_BWD_REDUCE: break;
+                    case OP_BN_APPLY: case OP_BN_FWD_FUSED: wr.push_back(o.bn.a); break;
+                    case OP_BN_BWD_APPLY: case OP_BN_BWD_FUSED: wr.push_back(o.bn.dx); break;
+                    default: always = true; break;
+                }
+            }
+            L.join_before = false;
+            if (L.kind == OP_CONV_WGRAD) { for (size_t k = i; k < j; ++k) { inflight.push_back(ops[k].conv.act); inflight.push_back(ops[k].conv.wgt); } }
+            else if (L.kind != OP_SPLITK && !inflight.empty()) {
+                bool hit = always;
+                for (const void* w : wr) for (const void* r : inflight) if (w == r) hit = true;
+                if (hit) { L.join_before = true; inflight.clear(); }
             }
         }
         plan.launches.push_back(L);
@@ -637,9 +670,9 @@ static int run_plan(resist_ctx* ctx, Plan& plan, const PatchArgs& pa, bool updat
     if (plan.nsites) { pf.begin(PK_PATCH, 1, 0, 0, st); patch_kernel<<<(plan.nsites + 63) / 64, 64, 0, st>>>(plan.d_sites, plan.nsites, pa); pf.end(st); ++n_launch; }
     // A layer's weight gradient and data gradient both read dy and are independent of each other: the weight gradients
     // (and their partial-sum reductions) go to a second stream, one after another, while the main stream carries on
-    // with the data gradient and the BN reduction that follows it.  Everything else may write a buffer that a weight
-    // gradient still reads (gradient buffers are recycled), so the main stream first waits for the second.  Per-kernel
-    // profiling keeps everything on one stream.
+    // down the network.  Gradient buffers are recycled, so a launch that writes a buffer which a weight gradient in
+    // flight still reads first waits for the second stream (join_before, worked out when the plan was built).
+    // Per-kernel profiling keeps everything on one stream.
     const bool overlap = !pf.on && update;
     if (overlap && !ctx->side_stream) {
         if (cudaStreamCreateWithFlags(&ctx->side_stream, cudaStreamNonBlocking) != cudaSuccess ||
@@ -655,7 +688,7 @@ static int run_plan(resist_ctx* ctx, Plan& plan, const PatchArgs& pa, bool updat
             st = ctx->side_stream;
         } else {
             st = main_st;
-            if (side_pending && L.kind != OP_CONV_DGRAD && L.kind != OP_BN_BWD_REDUCE) { cudaStreamWaitEvent(main_st, ctx->ev_side_done, 0); side_pending = false; }
+            if (side_pending && L.join_before) { cudaStreamWaitEvent(main_st, ctx->ev_side_done, 0); side_pending = false; }
         }
         int pk = 0, nk = 1;
         switch (L.kind) {
@@ -673,6 +706,8 @@ static int run_plan(resist_ctx* ctx, Plan& plan, const PatchArgs& pa, bool updat
             case OP_HEAD_BWD: pk = PK_HEAD_BWD; nk = 3; break;
             case OP_UPSAMPLE: pk = PK_UPSAMPLE; break;
             case OP_IM2COL: pk = PK_IM2COL; break;
+            case OP_BN_FWD_FUSED: pk = PK_BN_FWD_FUSED; break;
+            case OP_BN_BWD_FUSED: pk = PK_BN_BWD_FUSED; break;
         }
         pf.begin(pk, nk, L.bytes, L.flops, st);
         switch (L.kind) {
@@ -695,6 +730,14 @@ static int run_plan(resist_ctx* ctx, Plan& plan, const PatchArgs& pa, bool updat
             case OP_HEAD_BWD: launch_head_bwd(plan.d_head + L.first, L.count, L.max_b, L.max_c, L.max_classes, L.max_elems, bf, st); n_launch += 3; break;
             case OP_UPSAMPLE: launch_zero_stuff(plan.d_up + L.first, L.count, L.max_elems, st); ++n_launch; break;
             case OP_IM2COL: launch_im2col(plan.d_col + L.first, L.count, L.max_elems, st); ++n_launch; break;
+            case OP_BN_FWD_FUSED:
+                if (launch_bn_fused(plan.d_bn + L.first, L.count, L.gx, 0, st)) ++n_launch;
+                else { launch_bn_stats(plan.d_bn + L.first, L.count, L.gx, L.max_c, bf, st); launch_bn_apply(plan.d_bn + L.first, L.count, L.max_elems, bf, st); n_launch += 3; }
+                break;
+            case OP_BN_BWD_FUSED:
+                if (launch_bn_fused(plan.d_bn + L.first, L.count, L.gx, 1, st)) ++n_launch;
+                else { launch_bn_bwd_reduce(plan.d_bn + L.first, L.count, L.gx, L.max_c, bf, st); launch_bn_bwd_apply(plan.d_bn + L.first, L.count, L.max_elems, bf, st); n_launch += 3; }
+                break;
         }
         pf.end(st);
         if (on_side) { cudaEventRecord(ctx->ev_side_done, ctx->side_stream); side_pending = true; }

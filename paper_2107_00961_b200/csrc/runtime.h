@@ -18,7 +18,7 @@ Layout make_layout(const resist_arch& a, const std::vector<resist_block>& blocks
 
 enum OpKind {
     OP_CONV_FWD, OP_CONV_DGRAD, OP_CONV_WGRAD, OP_SPLITK, OP_BN_STATS, OP_BN_APPLY, OP_BN_BWD_REDUCE, OP_BN_BWD_APPLY,
-    OP_POOL_FWD, OP_POOL_BWD, OP_HEAD_FWD, OP_HEAD_BWD, OP_UPSAMPLE, OP_IM2COL
+    OP_POOL_FWD, OP_POOL_BWD, OP_HEAD_FWD, OP_HEAD_BWD, OP_UPSAMPLE, OP_IM2COL, OP_BN_FWD_FUSED, OP_BN_BWD_FUSED
 };
 
 // One operation of one sub-ResNet, keyed so that equal keys of different sub-ResNets share a launch.
@@ -35,12 +35,13 @@ struct Launch {
     OpKind kind; int backend; int first, count;               // range in the typed device array
     int gx; long long max_elems; int max_b, max_c, max_classes;
     double bytes, flops;                                      // algorithmic work of this launch
+    bool join_before;                                         // the main stream first waits for the weight gradients in flight
 };
 
 enum ProfKind {
     PK_CONV_FWD_CC, PK_CONV_DGRAD_CC, PK_CONV_WGRAD_CC, PK_CONV_FWD_TC, PK_CONV_DGRAD_TC, PK_CONV_WGRAD_TC, PK_SPLITK,
     PK_BN_STATS, PK_BN_APPLY, PK_BN_BWD_REDUCE, PK_BN_BWD_APPLY, PK_POOL_FWD, PK_POOL_BWD, PK_HEAD_FWD, PK_HEAD_BWD,
-    PK_SGD, PK_PATCH, PK_SCATTER, PK_AGGREGATE, PK_UPSAMPLE, PK_CONV_FWD_MMA, PK_CONV_DGRAD_MMA, PK_CONV_WGRAD_MMA, PK_IM2COL, PK_COUNT
+    PK_SGD, PK_PATCH, PK_SCATTER, PK_AGGREGATE, PK_UPSAMPLE, PK_CONV_FWD_MMA, PK_CONV_DGRAD_MMA, PK_CONV_WGRAD_MMA, PK_IM2COL, PK_BN_FWD_FUSED, PK_BN_BWD_FUSED, PK_COUNT
 };
 struct Profiler {
     bool on = false;
