@@ -384,13 +384,24 @@ __global__ void __launch_bounds__(256) bn_fused_kernel(const BnProb* __restrict_
     if ((int)blockIdx.x < p.chunks) bn_reduce_vec<MODE>(p);
     __threadfence();
     cg::this_grid().sync();
-    const int C = p.C, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    for (int c = warp; c < C; c += 8) {
-        // lane l adds chunks l, l+32, ... in order, then a fixed butterfly over the lanes
+    // every CTA adds the partial sums of all chunks in the same fixed order: thread (c, q) adds chunks q, q+Q, ...
+    // (independent loads), then thread c adds the Q sums in order
+    const int C = p.C;
+    __shared__ double s_red[2][256];
+    for (int cb = 0; cb < C; cb += 256) {
+        const int nl = C - cb < 256 ? C - cb : 256, Q = 256 / nl;
+        const int c = cb + (int)threadIdx.x % nl, q = (int)threadIdx.x / nl;
         double a0 = 0.0, a1 = 0.0;
-        for (int k = lane; k < p.chunks; k += 32) { a0 += __ldcg(p.partial + ((long long)k * 2 + 0) * C + c); a1 += __ldcg(p.partial + ((long long)k * 2 + 1) * C + c); }
-        for (int d = 16; d; d >>= 1) { a0 += __shfl_xor_sync(0xffffffffu, a0, d); a1 += __shfl_xor_sync(0xffffffffu, a1, d); }
-        if (lane != 0) continue;
+        if (q < Q) {
+#pragma unroll 4
+            for (int k = q; k < p.chunks; k += Q) { a0 += __ldcg(p.partial + ((long long)k * 2 + 0) * C + c); a1 += __ldcg(p.partial + ((long long)k * 2 + 1) * C + c); }
+        }
+        __syncthreads();
+        s_red[0][threadIdx.x] = a0; s_red[1][threadIdx.x] = a1;
+        __syncthreads();
+        if (q != 0) continue;
+        a0 = 0.0; a1 = 0.0;
+        for (int k = 0; k < Q; ++k) { a0 += s_red[0][k * nl + (c - cb)]; a1 += s_red[1][k * nl + (c - cb)]; }
         if (MODE == 0) {
             const double m = (double)p.m, dm = a0 / m;             // sums are of x - x[0,c]
             double var = a1 / m - dm * dm; if (var < 0.0) var = 0.0;
