@@ -34,6 +34,7 @@ struct alignas(16) MmaProb {
     int sub, subs, units;       // positions per piece (multiple of 16), pieces per group, pieces in total
     int os, P, Q;               // output stride (forward of a stride-2 layer stores even positions only, as a P x Q image)
     int stages;                 // depth of the activation ring (2, 3 or 4)
+    int nsplit;                 // 1, or 2: a CTA computes one half of the output channels (its half of the filter resident)
     int variant, smem_bytes;    // which instantiation runs this problem (see mma_variant); dynamic shared memory
     float scale;
 };
@@ -82,9 +83,11 @@ __global__ void __launch_bounds__(MMA_THREADS) conv_mma_kernel(const MmaProb* __
     __shared__ MmaProb p;
     if (threadIdx.x < sizeof(MmaProb) / 4) reinterpret_cast<uint32_t*>(&p)[threadIdx.x] = reinterpret_cast<const uint32_t*>(probs + blockIdx.y)[threadIdx.x];
     __syncthreads();
-    constexpr int TAPS = KSZ * KSZ, PAD = KSZ / 2, ncol = NB * 8;
-    const int units = p.units;
-    if ((int)blockIdx.x >= units) return;
+    constexpr int TAPS = KSZ * KSZ, PAD = KSZ / 2, ncol = NB * 8;   // ncol: output channels of THIS CTA
+    const int units = p.units, nsplit = p.nsplit;
+    const int ncol_all = ncol * nsplit, n_off = ((int)blockIdx.x % nsplit) * ncol;
+    const int cta = blockIdx.x / nsplit, ncta = gridDim.x / nsplit;   // the launcher makes gridDim.x a multiple of nsplit
+    if (cta >= units) return;
     extern __shared__ __align__(16) uint8_t sm[];
     const int ca = p.ca, apitch = ca * 2 + 16;                    // activation row pitch in bytes
     const int wrows = TRANS ? ca : ncol;                          // rows of one tap of the staged filter
@@ -93,9 +96,9 @@ __global__ void __launch_bounds__(MMA_THREADS) conv_mma_kernel(const MmaProb* __
     const int Wp = p.Wp, sub = p.sub, subs = p.subs, stages = p.stages;
     const int halo = PAD * Wp + PAD, win_rows = sub + 2 * halo, nblk = sub / 16;
     const int it_rows = subs * sub + 2 * halo, ot_rows = subs * sub;
-    int* itable = reinterpret_cast<int*>(sm);
-    int* otable = itable + it_rows;
-    const int table_bytes = ((it_rows + ot_rows) * 4 + 127) & ~127;
+    short* itable = reinterpret_cast<short*>(sm);               // a group has fewer than 32768 pixels
+    short* otable = itable + it_rows;
+    const int table_bytes = ((it_rows + ot_rows) * 2 + 127) & ~127;
     const int stage_bytes = (win_rows * apitch + 127) & ~127;
     uint8_t* ring = sm + table_bytes;
     uint8_t* s_w = ring + stages * stage_bytes;
@@ -117,22 +120,22 @@ __global__ void __launch_bounds__(MMA_THREADS) conv_mma_kernel(const MmaProb* __
                 else if (!((i % p.os) | (X % p.os))) opix = (int)((n * p.P + i / p.os) * p.Q + X / p.os);
             }
         }
-        itable[w] = pix;
-        if (f >= 0 && f < ot_rows) otable[f] = opix;
+        itable[w] = (short)pix;
+        if (f >= 0 && f < ot_rows) otable[f] = (short)opix;
     }
     // ---- the filter, once per CTA
     if (!TRANS) {               // tap t, column n, 8-channel group g  <-  w[chan_of_col(n)][t][g*8..]
         const int groups = ca / 8, n_chunks = TAPS * ncol * groups;
         for (int id = tid; id < n_chunks; id += MMA_THREADS) {
             const int g = id % groups, n = (id / groups) % ncol, t = id / (groups * ncol);
-            const uint4 v = __ldg(reinterpret_cast<const uint4*>(p.wgt + ((long long)chan_of_col<NB>(n) * TAPS + t) * p.wC + g * 8));
+            const uint4 v = __ldg(reinterpret_cast<const uint4*>(p.wgt + ((long long)(n_off + chan_of_col<NB>(n)) * TAPS + t) * p.wC + g * 8));
             *reinterpret_cast<uint4*>(s_w + (t * wrows + n) * wpitch + g * 16) = v;
         }
     } else {                    // tap t, row k, column col_of_chan(c)  <-  w[k][t][c]
         constexpr int groups = ncol / 8; const int n_chunks = TAPS * ca * groups;
         for (int id = tid; id < n_chunks; id += MMA_THREADS) {
             const int g = id % groups, k = (id / groups) % ca, t = id / (groups * ca);
-            const uint4 v = __ldg(reinterpret_cast<const uint4*>(p.wgt + ((long long)k * TAPS + t) * p.wC + g * 8));
+            const uint4 v = __ldg(reinterpret_cast<const uint4*>(p.wgt + ((long long)k * TAPS + t) * p.wC + n_off + g * 8));
             const uint32_t w4[4] = {v.x, v.y, v.z, v.w};
             uint8_t* row = s_w + (t * wrows + k) * wpitch;
 #pragma unroll
@@ -143,12 +146,12 @@ __global__ void __launch_bounds__(MMA_THREADS) conv_mma_kernel(const MmaProb* __
     const int ga = ca / 8, a_step = MMA_THREADS / ga, a_row0 = tid / ga, a_g = tid % ga;
     const bool a_on = tid < a_step * ga;
     const long long grp_in = (long long)p.G * p.H * p.W * ca;                    // elements of a group of act
-    const long long grp_out = (long long)p.G * (p.os == 1 ? p.H * p.W : p.P * p.Q) * ncol;
+    const long long grp_out = (long long)p.G * (p.os == 1 ? p.H * p.W : p.P * p.Q) * ncol_all;
     auto issue = [&](int unit, int stage) {
         const int grp = unit / subs, j = unit - grp * subs;
         const __nv_bfloat16* ag = act + grp * grp_in + a_g * 8;
         if (a_on) {
-            const int* t = itable + j * sub + a_row0;
+            const short* t = itable + j * sub + a_row0;
             uint32_t dst = s_u32(ring + stage * stage_bytes) + a_g * 16 + a_row0 * apitch;
             for (int row = a_row0; row < win_rows; row += a_step, t += a_step, dst += a_step * apitch) {
                 const int pix = *t;                                // padding: read nothing, write zeros
@@ -169,11 +172,11 @@ __global__ void __launch_bounds__(MMA_THREADS) conv_mma_kernel(const MmaProb* __
     const float scale = p.scale;
 
     __syncthreads();                                              // tables complete
-    int nxt = blockIdx.x;
-    for (int st = 0; st < stages - 1; ++st) { if (nxt < units) issue(nxt, st); cp_async_commit(); nxt += gridDim.x; }
+    int nxt = cta;
+    for (int st = 0; st < stages - 1; ++st) { if (nxt < units) issue(nxt, st); cp_async_commit(); nxt += ncta; }
     int stage = 0;
-    for (int unit = blockIdx.x; unit < units; unit += gridDim.x) {
-        { const int ps = stage == 0 ? stages - 1 : stage - 1; if (nxt < units) issue(nxt, ps); cp_async_commit(); nxt += gridDim.x; }
+    for (int unit = cta; unit < units; unit += ncta) {
+        { const int ps = stage == 0 ? stages - 1 : stage - 1; if (nxt < units) issue(nxt, ps); cp_async_commit(); nxt += ncta; }
         if (stages == 2) cp_async_wait<1>(); else if (stages == 3) cp_async_wait<2>(); else cp_async_wait<3>();
         __syncthreads();                                          // this piece's window (and, first time, the filter) is in shared memory
 
@@ -209,7 +212,7 @@ __global__ void __launch_bounds__(MMA_THREADS) conv_mma_kernel(const MmaProb* __
         }
         // ---- epilogue: thread (g8, t4) holds rows g8 and g8+8 of each 16-row block, channels t4*2*NB ... t4*2*NB + 2*NB - 1
         const int grp = unit / subs, j0 = (unit - grp * subs) * sub;
-        const long long obase = grp * grp_out + t4 * (2 * NB);
+        const long long obase = grp * grp_out + n_off + t4 * (2 * NB);
 #pragma unroll
         for (int mb = 0; mb < MBW; ++mb)
 #pragma unroll
@@ -217,7 +220,7 @@ __global__ void __launch_bounds__(MMA_THREADS) conv_mma_kernel(const MmaProb* __
                 const int blk = warp + 8 * mb;
                 const int opix = blk < nblk ? otable[j0 + blk * 16 + g8 + half * 8] : -1;
                 if (opix < 0) continue;
-                const long long o = obase + (long long)opix * ncol;
+                const long long o = obase + (long long)opix * ncol_all;
                 uint32_t wv[NB];
                 if (addp) {
                     if constexpr (NB % 4 == 0) {
@@ -250,7 +253,7 @@ __global__ void __launch_bounds__(MMA_THREADS) conv_mma_kernel(const MmaProb* __
 }
 
 // ------------------------------------------------------------------------------------------------ host side
-struct MmaGeom { int ca, ncol, Hp, Wp, G, gpos, sub, subs, units, mbw, stages, variant; size_t smem; };
+struct MmaGeom { int ca, ncol, Hp, Wp, G, gpos, sub, subs, units, mbw, stages, nsplit, variant; size_t smem; };
 
 // variant = ((MBW * 4 + ksz) * 2 + trans) * 16 + NB: everything a launch is specialised on
 static int mma_variant(int mbw, int ksz, int trans, int nb) { return ((mbw * 4 + ksz) * 2 + trans) * 16 + nb; }
@@ -267,8 +270,13 @@ static bool mma_geometry(const ConvProb& p, int mode, MmaGeom& g) {
     const int ppi = g.Hp * g.Wp, halo = pad * g.Wp + pad;
     const int apitch = g.ca * 2 + 16;
     const int wrows = mode == CONV_FWD ? g.ncol : g.ca, wcols = mode == CONV_FWD ? g.ca : g.ncol;
-    const size_t wbytes = (size_t)p.ksz * p.ksz * wrows * (wcols * 2 + 16);
-    const int max_mbw = g.ncol <= 32 ? 3 : 2;                     // accumulators: MBW * (ncol / 8) * 4 registers
+    // 64 output channels: two CTAs share a piece, each with half of the filter resident (twice the CTAs per SM)
+    g.nsplit = g.ncol == 64 && p.ksz == 3 ? 2 : 1;
+    const int ncta_col = g.ncol / g.nsplit;
+    const int wrows_c = mode == CONV_FWD ? ncta_col : g.ca, wcols_c = mode == CONV_FWD ? g.ca : ncta_col;
+    const size_t wbytes = (size_t)p.ksz * p.ksz * wrows_c * (wcols_c * 2 + 16);
+    (void)wrows; (void)wcols;
+    const int max_mbw = ncta_col <= 32 ? 3 : 2;                   // accumulators: MBW * (channels / 8) * 4 registers
     // images per group and positions per piece: little padding of the last piece, all warps busy, pieces not too
     // small, enough pieces to go round
     double best = 1e30; g.sub = 0;
@@ -279,7 +287,8 @@ static bool mma_geometry(const ConvProb& p, int mode, MmaGeom& g) {
         if (gpos > 7000) break;
         for (int sub = 64; sub <= 128 * max_mbw; sub += 16) {
             const int subs = (gpos + sub - 1) / sub, nblk = sub / 16, mbw = (nblk + 7) / 8;
-            const size_t table = (size_t)(((2 * subs * sub + 2 * halo) * 4 + 127) & ~127);
+            if (gpos >= 32768 || (long long)G * p.H * p.W >= 32768) continue;
+            const size_t table = (size_t)(((2 * subs * sub + 2 * halo) * 2 + 127) & ~127);
             const size_t stage = (size_t)(((sub + 2 * halo) * apitch + 127) & ~127);
             int stages = 4; while (stages > 2 && table + stages * stage + wbytes + 64 > 100 * 1024) --stages;
             if (table + stages * stage + wbytes + 64 > 200 * 1024) continue;
@@ -291,7 +300,7 @@ static bool mma_geometry(const ConvProb& p, int mode, MmaGeom& g) {
         }
     }
     if (!g.sub) return false;
-    g.variant = mma_variant(g.mbw, p.ksz, mode == CONV_DGRAD ? 1 : 0, g.ncol / 8);
+    g.variant = mma_variant(g.mbw, p.ksz, mode == CONV_DGRAD ? 1 : 0, ncta_col / 8);
     return true;
 }
 
@@ -307,11 +316,11 @@ bool conv_mma_fill(const ConvProb& p, int mode, void* host) {
     t.inv_wp = (unsigned)((1ull << 32) / (unsigned)g.Wp + 1); t.inv_hp = (unsigned)((1ull << 32) / (unsigned)g.Hp + 1);
     t.G = g.G; t.gpos = g.gpos; t.sub = g.sub; t.subs = g.subs; t.units = g.units;
     t.os = mode == CONV_FWD ? p.stride : 1; t.P = p.P; t.Q = p.Q;
-    t.stages = g.stages; t.variant = g.variant; t.smem_bytes = (int)g.smem; t.scale = p.scale;
+    t.stages = g.stages; t.nsplit = g.nsplit; t.variant = g.variant; t.smem_bytes = (int)g.smem; t.scale = p.scale;
     memcpy(host, &t, sizeof(t));
     return true;
 }
-int conv_mma_tiles(const void* h) { return ((const MmaProb*)h)->units; }
+int conv_mma_tiles(const void* h) { return ((const MmaProb*)h)->units * ((const MmaProb*)h)->nsplit; }
 int conv_mma_variant(const void* h) { return ((const MmaProb*)h)->variant; }
 size_t conv_mma_smem(const void* h) { return (size_t)((const MmaProb*)h)->smem_bytes; }
 
@@ -332,8 +341,9 @@ void launch_conv_mma_probs(const void* d, int nprob, int max_tiles, size_t max_s
     if (!sms) { int dev = 0; cudaGetDevice(&dev); cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev); if (sms < 1) sms = 148; }
     const int nb = variant & 15, trans = (variant >> 4) & 1, ksz = (variant >> 5) & 3, mbw = (variant >> 7) & 3;
     // persistent CTAs: as many as fit on the chip at this shared-memory footprint (at most 3 per SM), over all problems
-    int per_sm = (int)((225 * 1024) / (max_smem + 1024)); if (per_sm > 3) per_sm = 3; if (per_sm < 1) per_sm = 1;
-    int gx = (per_sm * sms + nprob - 1) / nprob; if (gx > max_tiles) gx = max_tiles; if (gx < 1) gx = 1;
+    int per_sm = (int)((227 * 1024) / (max_smem + 1024)); if (per_sm > 3) per_sm = 3; if (per_sm < 1) per_sm = 1;
+    int gx = (per_sm * sms + nprob - 1) / nprob; if (gx > max_tiles) gx = max_tiles; if (gx < 2) gx = 2;
+    gx &= ~1;                                                      // even: a CTA pair shares a piece when the channels are split
     const dim3 grid(gx, nprob);
 #define MMA_CASE(N_, M_) if (nb == N_ && mbw == M_) launch_mma_nb<N_, M_>(d, grid, max_smem, ksz, trans, s); else
     MMA_CASE(2, 1) MMA_CASE(2, 2) MMA_CASE(2, 3) MMA_CASE(4, 1) MMA_CASE(4, 2) MMA_CASE(4, 3)
