@@ -64,6 +64,18 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");   // src_bytes 0: zeros
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+// Programmatic dependent launch: a kernel launched with the attribute may start while the kernel before it in the
+// stream is still running; it must not touch anything that kernel writes before pdl_wait() returns (which is when that
+// kernel has finished and its writes are visible).  pdl_trigger() lets the NEXT kernel of the stream start early.
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+template <class K, class A>
+static void launch_pdl(K kernel, dim3 grid, size_t smem, cudaStream_t s, bool pdl, A arg) {
+    cudaLaunchConfig_t cfg = {}; cfg.gridDim = grid; cfg.blockDim = dim3(256); cfg.dynamicSmemBytes = smem; cfg.stream = s;
+    cudaLaunchAttribute at[1]; at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization; at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at; cfg.numAttrs = pdl ? 1 : 0;
+    cudaLaunchKernelEx(&cfg, kernel, arg);
+}
 template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 // Column n of the MMA's B operand carries output channel chan_of_col(n): thread (g8, t4) of a warp then owns, over its
@@ -83,6 +95,7 @@ __global__ void __launch_bounds__(MMA_THREADS) conv_mma_kernel(const MmaProb* __
     __shared__ MmaProb p;
     if (threadIdx.x < sizeof(MmaProb) / 4) reinterpret_cast<uint32_t*>(&p)[threadIdx.x] = reinterpret_cast<const uint32_t*>(probs + blockIdx.y)[threadIdx.x];
     __syncthreads();
+    pdl_trigger();
     constexpr int TAPS = KSZ * KSZ, PAD = KSZ / 2, ncol = NB * 8;   // ncol: output channels of THIS CTA
     const int units = p.units, nsplit = p.nsplit;
     const int ncol_all = ncol * nsplit, n_off = ((int)blockIdx.x % nsplit) * ncol;
@@ -172,6 +185,7 @@ __global__ void __launch_bounds__(MMA_THREADS) conv_mma_kernel(const MmaProb* __
     const float scale = p.scale;
 
     __syncthreads();                                              // tables complete
+    pdl_wait();                                                   // from here on: tensors the previous kernel may have written
     int nxt = cta;
     for (int st = 0; st < stages - 1; ++st) { if (nxt < units) issue(nxt, st); cp_async_commit(); nxt += ncta; }
     int stage = 0;
@@ -325,18 +339,19 @@ int conv_mma_variant(const void* h) { return ((const MmaProb*)h)->variant; }
 size_t conv_mma_smem(const void* h) { return (size_t)((const MmaProb*)h)->smem_bytes; }
 
 template <int NB, int MBW, int KSZ, bool TRANS>
-static void launch_mma_inst(const void* d, dim3 grid, size_t smem, cudaStream_t s) {
+static void launch_mma_inst(const void* d, dim3 grid, size_t smem, bool pdl, cudaStream_t s) {
     static bool configured = false;
     if (!configured) { cudaFuncSetAttribute(conv_mma_kernel<NB, MBW, KSZ, TRANS>, cudaFuncAttributeMaxDynamicSharedMemorySize, 202 * 1024); configured = true; }
-    conv_mma_kernel<NB, MBW, KSZ, TRANS><<<grid, MMA_THREADS, smem, s>>>((const MmaProb*)d);
+    launch_pdl(conv_mma_kernel<NB, MBW, KSZ, TRANS>, grid, smem, s, pdl, (const MmaProb*)d);
 }
 template <int NB, int MBW>
-static void launch_mma_nb(const void* d, dim3 grid, size_t smem, int ksz, int trans, cudaStream_t s) {
-    if (ksz == 3) { if (trans) launch_mma_inst<NB, MBW, 3, true>(d, grid, smem, s); else launch_mma_inst<NB, MBW, 3, false>(d, grid, smem, s); }
-    else { if (trans) launch_mma_inst<NB, MBW, 1, true>(d, grid, smem, s); else launch_mma_inst<NB, MBW, 1, false>(d, grid, smem, s); }
+static void launch_mma_nb(const void* d, dim3 grid, size_t smem, int ksz, int trans, bool pdl, cudaStream_t s) {
+    if (ksz == 3) { if (trans) launch_mma_inst<NB, MBW, 3, true>(d, grid, smem, pdl, s); else launch_mma_inst<NB, MBW, 3, false>(d, grid, smem, pdl, s); }
+    else { if (trans) launch_mma_inst<NB, MBW, 1, true>(d, grid, smem, pdl, s); else launch_mma_inst<NB, MBW, 1, false>(d, grid, smem, pdl, s); }
 }
 // all problems of one launch share the variant
-void launch_conv_mma_probs(const void* d, int nprob, int max_tiles, size_t max_smem, int variant, cudaStream_t s) {
+// pdl: the kernel may start before the previous kernel of the stream has finished (that kernel must not write the weights)
+void launch_conv_mma_probs(const void* d, int nprob, int max_tiles, size_t max_smem, int variant, cudaStream_t s, bool pdl) {
     static int sms = 0;
     if (!sms) { int dev = 0; cudaGetDevice(&dev); cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev); if (sms < 1) sms = 148; }
     const int nb = variant & 15, trans = (variant >> 4) & 1, ksz = (variant >> 5) & 3, mbw = (variant >> 7) & 3;
@@ -345,7 +360,7 @@ void launch_conv_mma_probs(const void* d, int nprob, int max_tiles, size_t max_s
     int gx = (per_sm * sms + nprob - 1) / nprob; if (gx > max_tiles) gx = max_tiles; if (gx < 2) gx = 2;
     gx &= ~1;                                                      // even: a CTA pair shares a piece when the channels are split
     const dim3 grid(gx, nprob);
-#define MMA_CASE(N_, M_) if (nb == N_ && mbw == M_) launch_mma_nb<N_, M_>(d, grid, max_smem, ksz, trans, s); else
+#define MMA_CASE(N_, M_) if (nb == N_ && mbw == M_) launch_mma_nb<N_, M_>(d, grid, max_smem, ksz, trans, pdl, s); else
     MMA_CASE(2, 1) MMA_CASE(2, 2) MMA_CASE(2, 3) MMA_CASE(4, 1) MMA_CASE(4, 2) MMA_CASE(4, 3)
     MMA_CASE(6, 1) MMA_CASE(6, 2) MMA_CASE(8, 1) MMA_CASE(8, 2)
     return;
@@ -385,6 +400,7 @@ __global__ void __launch_bounds__(MMA_THREADS) conv_wgrad_mma_kernel(const MmaWg
     __shared__ MmaWgradProb p;
     if (threadIdx.x < sizeof(MmaWgradProb) / 4) reinterpret_cast<uint32_t*>(&p)[threadIdx.x] = reinterpret_cast<const uint32_t*>(probs + blockIdx.y)[threadIdx.x];
     __syncthreads();
+    pdl_trigger();
     if ((int)blockIdx.x >= p.tap_groups * p.splits) return;
     const int split = blockIdx.x % p.splits, tg = blockIdx.x / p.splits;
     const int tap0 = tg * p.taps_per_group; int ntap = p.taps - tap0; if (ntap > p.taps_per_group) ntap = p.taps_per_group;
@@ -462,6 +478,7 @@ __global__ void __launch_bounds__(MMA_THREADS) conv_wgrad_mma_kernel(const MmaWg
     const int ksteps = sub / 16;
 
     __syncthreads();                                              // table complete
+    pdl_wait();                                                   // from here on: tensors the previous kernel may have written
     const int units = p.units;
     int nxt = split;
     for (int st = 0; st < stages - 1; ++st) { if (nxt < units) issue(nxt, st); cp_async_commit(); nxt += p.splits; }
@@ -523,6 +540,7 @@ __global__ void __launch_bounds__(MMA_THREADS) conv_wgrad_mma_kernel(const MmaWg
 // out[k][t][c] = sum over splits of partial[split][t][k][c], in a fixed order: a block owns 32 consecutive elements,
 // warp w adds the splits w, w+8, ... (ascending), then the 8 sums are added in warp order.
 __global__ void __launch_bounds__(256) wgrad_mma_reduce_kernel(const MmaWgradProb* __restrict__ probs) {
+    pdl_trigger();
     const MmaWgradProb& p = probs[blockIdx.y];
     const int n = p.taps * p.K * p.C, splits = p.splits, taps = p.taps, K = p.K, C = p.C;
     const float* __restrict__ partial = p.partial;
@@ -624,16 +642,16 @@ size_t conv_wgrad_mma_smem(const void* h) { return (size_t)((const MmaWgradProb*
 long long conv_wgrad_mma_out_elems(const void* h) { const MmaWgradProb* t = (const MmaWgradProb*)h; return (long long)t->taps * t->K * t->C; }
 
 template <int MB, int PPW>
-static void launch_wg_inst(const void* d, dim3 grid, size_t smem, cudaStream_t s) {
+static void launch_wg_inst(const void* d, dim3 grid, size_t smem, bool pdl, cudaStream_t s) {
     static bool configured = false;
     if (!configured) { cudaFuncSetAttribute(conv_wgrad_mma_kernel<MB, PPW>, cudaFuncAttributeMaxDynamicSharedMemorySize, 202 * 1024); configured = true; }
-    conv_wgrad_mma_kernel<MB, PPW><<<grid, MMA_THREADS, smem, s>>>((const MmaWgradProb*)d);
+    launch_pdl(conv_wgrad_mma_kernel<MB, PPW>, grid, smem, s, pdl, (const MmaWgradProb*)d);
 }
 // all problems of one launch share the variant (output channels / 16 + 8 * column pairs per warp)
-void launch_conv_wgrad_mma_probs(const void* d, int nprob, int max_ctas, size_t max_smem, long long max_out, int variant, cudaStream_t s) {
+void launch_conv_wgrad_mma_probs(const void* d, int nprob, int max_ctas, size_t max_smem, long long max_out, int variant, cudaStream_t s, bool pdl) {
     const dim3 grid(max_ctas, nprob);
     const int mb = variant & 7, ppw = (variant >> 3) & 31;
-#define WG_CASE(M, P) if (mb == M && ppw == P) launch_wg_inst<M, P>(d, grid, max_smem, s); else
+#define WG_CASE(M, P) if (mb == M && ppw == P) launch_wg_inst<M, P>(d, grid, max_smem, pdl, s); else
     WG_CASE(1, 1) WG_CASE(1, 2) WG_CASE(1, 3) WG_CASE(1, 5) WG_CASE(1, 9) WG_CASE(1, 12)
     WG_CASE(2, 1) WG_CASE(2, 2) WG_CASE(2, 3) WG_CASE(2, 5)
     WG_CASE(3, 1) WG_CASE(3, 2) WG_CASE(3, 3)

@@ -379,6 +379,7 @@ __global__ void __launch_bounds__(256) bn_bwd_apply_kernel(const BnProb* __restr
 // from L2.  bf16 vector path, training mode only.
 template <int MODE>
 __global__ void __launch_bounds__(256) bn_fused_kernel(const BnProb* __restrict__ probs) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // a convolution launched behind this kernel may start its prologue
     const BnProb& p = probs[blockIdx.y];
     __shared__ __align__(16) float s_stat[4 * 512];               // callers keep C <= 512
     if ((int)blockIdx.x < p.chunks) bn_reduce_vec<MODE>(p);

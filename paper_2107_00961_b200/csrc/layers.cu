@@ -25,7 +25,7 @@ bool conv_mma_fill(const ConvProb& p, int mode, void* host);
 size_t conv_mma_prob_bytes();
 int conv_mma_tiles(const void* h);
 size_t conv_mma_smem(const void* h);
-void launch_conv_mma_probs(const void* d, int nprob, int max_tiles, size_t max_smem, int variant, cudaStream_t s);
+void launch_conv_mma_probs(const void* d, int nprob, int max_tiles, size_t max_smem, int variant, cudaStream_t s, bool pdl = false);
 int conv_mma_pick_variant(const ConvProb& p, int mode);
 bool conv_wgrad_mma_supported(const ConvProb& p, int target_ctas, size_t* partial_bytes);
 bool conv_wgrad_mma_fill(const ConvProb& p, int target_ctas, void* host);
@@ -33,7 +33,7 @@ size_t conv_wgrad_mma_prob_bytes();
 int conv_wgrad_mma_ctas(const void* h);
 size_t conv_wgrad_mma_smem(const void* h);
 long long conv_wgrad_mma_out_elems(const void* h);
-void launch_conv_wgrad_mma_probs(const void* d, int nprob, int max_ctas, size_t max_smem, long long max_out, int variant, cudaStream_t s);
+void launch_conv_wgrad_mma_probs(const void* d, int nprob, int max_ctas, size_t max_smem, long long max_out, int variant, cudaStream_t s, bool pdl = false);
 int conv_wgrad_mma_pick_variant(const ConvProb& p, int target_ctas);
 }
 using namespace resist;

@@ -33,7 +33,7 @@ bool conv_mma_fill(const ConvProb& p, int mode, void* host);
 size_t conv_mma_prob_bytes();
 int conv_mma_tiles(const void* h);
 size_t conv_mma_smem(const void* h);
-void launch_conv_mma_probs(const void* d, int nprob, int max_tiles, size_t max_smem, int variant, cudaStream_t s);
+void launch_conv_mma_probs(const void* d, int nprob, int max_tiles, size_t max_smem, int variant, cudaStream_t s, bool pdl = false);
 int conv_mma_pick_variant(const ConvProb& p, int mode);
 bool conv_wgrad_mma_supported(const ConvProb& p, int target_ctas, size_t* partial_bytes);
 bool conv_wgrad_mma_fill(const ConvProb& p, int target_ctas, void* host);
@@ -41,7 +41,7 @@ size_t conv_wgrad_mma_prob_bytes();
 int conv_wgrad_mma_ctas(const void* h);
 size_t conv_wgrad_mma_smem(const void* h);
 long long conv_wgrad_mma_out_elems(const void* h);
-void launch_conv_wgrad_mma_probs(const void* d, int nprob, int max_ctas, size_t max_smem, long long max_out, int variant, cudaStream_t s);
+void launch_conv_wgrad_mma_probs(const void* d, int nprob, int max_ctas, size_t max_smem, long long max_out, int variant, cudaStream_t s, bool pdl = false);
 int conv_wgrad_mma_pick_variant(const ConvProb& p, int target_ctas);
 
 // Which kernel family takes a bf16 convolution: 0 = CUDA cores, 1 = tcgen05, >= 200 = warp-level MMA (wgrad: 200 +
@@ -681,7 +681,10 @@ static int run_plan(resist_ctx* ctx, Plan& plan, const PatchArgs& pa, bool updat
     }
     bool side_pending = false;
     const cudaStream_t main_st = st;
+    OpKind prev_kind = OP_HEAD_FWD;
     for (const Launch& L : plan.launches) {
+        // early start of a warp-MMA convolution: not behind the im2col pass that writes the stem's packed weights, not while profiling
+        const bool pdl_ok = !pf.on && prev_kind != OP_IM2COL; prev_kind = L.kind;
         const bool on_side = overlap && (L.kind == OP_CONV_WGRAD || (L.kind == OP_SPLITK && side_pending));
         if (on_side) {
             cudaEventRecord(ctx->ev_fork, main_st); cudaStreamWaitEvent(ctx->side_stream, ctx->ev_fork, 0);
@@ -713,8 +716,8 @@ static int run_plan(resist_ctx* ctx, Plan& plan, const PatchArgs& pa, bool updat
         switch (L.kind) {
             case OP_CONV_FWD: case OP_CONV_DGRAD: case OP_CONV_WGRAD: {
                 const int mode = L.kind == OP_CONV_FWD ? CONV_FWD : L.kind == OP_CONV_DGRAD ? CONV_DGRAD : CONV_WGRAD;
-                if (L.backend >= 200 && mode == CONV_WGRAD) { launch_conv_wgrad_mma_probs((const char*)plan.d_wmm + (size_t)L.first * plan.wmm_stride, L.count, L.gx, (size_t)L.max_elems, L.max_b, L.backend - 200, st); ++n_launch; }
-                else if (L.backend >= 200) launch_conv_mma_probs((const char*)plan.d_mm + (size_t)L.first * plan.mm_stride, L.count, L.gx, (size_t)L.max_elems, L.backend - 1000, st);
+                if (L.backend >= 200 && mode == CONV_WGRAD) { launch_conv_wgrad_mma_probs((const char*)plan.d_wmm + (size_t)L.first * plan.wmm_stride, L.count, L.gx, (size_t)L.max_elems, L.max_b, L.backend - 200, st, pdl_ok); ++n_launch; }
+                else if (L.backend >= 200) launch_conv_mma_probs((const char*)plan.d_mm + (size_t)L.first * plan.mm_stride, L.count, L.gx, (size_t)L.max_elems, L.backend - 1000, st, pdl_ok);
                 else if (L.backend && mode == CONV_WGRAD) { launch_conv_wgrad_tc_probs((const char*)plan.d_wtc + (size_t)L.first * plan.wtc_stride, L.count, L.gx, (size_t)L.max_elems, L.max_b, st); ++n_launch; }
                 else if (L.backend) launch_conv_tc_probs((const char*)plan.d_tc + (size_t)L.first * plan.tc_stride, L.count, L.gx, (size_t)L.max_elems, st);
                 else launch_conv_ref(plan.d_conv + L.first, L.count, L.gx, mode, bf, st);
