@@ -47,7 +47,8 @@ typedef enum {
 enum { RESIST_BASIC = 0, RESIST_BOTTLENECK = 1 };
 enum { RESIST_F32 = 0, RESIST_BF16 = 1 };
 enum { RESIST_MOMENTUM_RESTART = 0, RESIST_MOMENTUM_KEEP = 1 };
-enum { RESIST_CONV_AUTO = 0, RESIST_CONV_CUDA_CORES = 1, RESIST_CONV_TCGEN05 = 2, RESIST_CONV_WARP_MMA = 3 };
+enum { RESIST_CONV_AUTO = 0, RESIST_CONV_CUDA_CORES = 1, RESIST_CONV_TCGEN05 = 2, RESIST_CONV_WARP_MMA = 3,
+       RESIST_CONV_WARP_MMA_UNFUSED = 4 };
 #define RESIST_MAX_SUBNETS 32
 
 typedef struct resist_ctx resist_ctx;
@@ -86,7 +87,9 @@ typedef struct {
     int32_t momentum_policy; /* RESIST_MOMENTUM_RESTART: zero the momentum at every partition */
     int32_t conv_backend;    /* RESIST_CONV_AUTO: warp-level MMA for narrow layers (<= 64 channels), tcgen05 for wide ones,
                                 CUDA cores for the rest; _CUDA_CORES: never tensor cores; _TCGEN05 / _WARP_MMA: only that
-                                tensor-core family where the shape allows, CUDA cores elsewhere */
+                                tensor-core family where the shape allows, CUDA cores elsewhere.  With _AUTO and _WARP_MMA
+                                the BN+ReLU (forward or backward) that consumes a warp-MMA convolution's output runs inside
+                                that convolution's launch; _WARP_MMA_UNFUSED keeps BN in launches of its own */
 } resist_opts;
 
 /* Device-memory source.  alloc returns a device pointer aligned to >= 256 bytes or NULL; release frees it.

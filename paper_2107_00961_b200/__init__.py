@@ -17,7 +17,7 @@ from . import build as _build
 
 RESIST_OK = 0
 F32, BF16 = 0, 1
-CONV_AUTO, CONV_CUDA_CORES, CONV_TCGEN05, CONV_WARP_MMA = 0, 1, 2, 3
+CONV_AUTO, CONV_CUDA_CORES, CONV_TCGEN05, CONV_WARP_MMA, CONV_WARP_MMA_UNFUSED = 0, 1, 2, 3, 4
 MOMENTUM_RESTART, MOMENTUM_KEEP = 0, 1
 _STATUS = {0: "RESIST_OK", -1: "RESIST_EINVAL", -2: "RESIST_ESTATE", -3: "RESIST_ENOMEM", -4: "RESIST_ECUDA",
            -5: "RESIST_ETIMEOUT", -6: "RESIST_EUNSUPPORTED"}

@@ -16,9 +16,19 @@
 // taps read it at shifted row offsets through ldmatrix.  Because a group starts on an image boundary, two small
 // tables built once per CTA (window row -> input pixel, position -> output pixel; -1 at padding) serve every
 // piece of every group: neither the copies nor the epilogue do any index arithmetic.
+//
+// Fused BatchNorm (bn.fuse != 0): at this problem size a layer is a few microseconds of work and a training step is a
+// chain of dependent launches, so the BN+ReLU that consumes a convolution's output runs in the SAME launch.  The
+// epilogue adds up the per-channel sums the BN needs (forward: x, x^2 of the stored bf16 output; backward: dz, dz*xhat
+// with dz = da * [relu input > 0]) per CTA in a fixed order, the CTAs meet at a grid-wide barrier (cooperative launch),
+// every CTA adds the per-CTA partial sums of its problem in the same fixed order, and the grid makes the elementwise
+// pass over the tensor it has just written (an L2 hit).
 #include <algorithm>
 #include <cstring>
+#include <cooperative_groups.h>
 #include "internal.h"
+
+namespace cg = cooperative_groups;
 
 namespace resist {
 
@@ -37,7 +47,21 @@ struct alignas(16) MmaProb {
     int nsplit;                 // 1, or 2: a CTA computes one half of the output channels (its half of the filter resident)
     int variant, smem_bytes;    // which instantiation runs this problem (see mma_variant); dynamic shared memory
     float scale;
+    int fuse;                   // 0: convolution only; 1: + BN+ReLU forward of out; 2: + BN+ReLU backward with out as da
+    BnProb bn;                  // fuse 1: x = out, a; fuse 2: x, da = out, dx, add.  partial: [CTAs of the problem][2][C] doubles
 };
+
+__device__ __forceinline__ void bf8_unpack(const uint4& v, float* f) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { f[2 * i] = __uint_as_float(w[i] << 16); f[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u); }
+}
+__device__ __forceinline__ uint4 bf8_pack(const float* f) {
+    uint32_t w[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]); w[i] = *reinterpret_cast<uint32_t*>(&h); }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+}
 
 
 __device__ __forceinline__ uint32_t s_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -100,8 +124,12 @@ __global__ void __launch_bounds__(MMA_THREADS) conv_mma_kernel(const MmaProb* __
     const int units = p.units, nsplit = p.nsplit;
     const int ncol_all = ncol * nsplit, n_off = ((int)blockIdx.x % nsplit) * ncol;
     const int cta = blockIdx.x / nsplit, ncta = gridDim.x / nsplit;   // the launcher makes gridDim.x a multiple of nsplit
-    if (cta >= units) return;
+    constexpr bool FUSABLE = NB <= 4;                             // wider CTAs would pay for the sums with registers: the host never asks
+    const int fuse = FUSABLE ? p.fuse : 0;
+    if (cta >= units && !fuse) return;                            // fused: every CTA must reach the grid barrier
     extern __shared__ __align__(16) uint8_t sm[];
+    __shared__ float s_red[8][2][NB * 8];                         // per-warp sums of the fused BN, over the CTA's whole walk
+    __shared__ float s_bn[4][NB * 8];                             // fuse 2: mean, 1/std, gamma, beta of this CTA's channels
     const int ca = p.ca, apitch = ca * 2 + 16;                    // activation row pitch in bytes
     const int wrows = TRANS ? ca : ncol;                          // rows of one tap of the staged filter
     const int wcols = TRANS ? ncol : ca;                          // elements per row
@@ -183,9 +211,15 @@ __global__ void __launch_bounds__(MMA_THREADS) conv_mma_kernel(const MmaProb* __
     const uint32_t b_lane = TRANS ? (uint32_t)(((lane >> 3) & 1) * 8 + (lane & 7)) * wpitch + (lane >> 4) * 16
                                   : (uint32_t)((lane >> 4) * 8 + (lane & 7)) * wpitch + ((lane >> 3) & 1) * 16;
     const float scale = p.scale;
+    if (fuse) for (int i = tid; i < 8 * 2 * ncol; i += MMA_THREADS) (&s_red[0][0][0])[i] = 0.f;
 
     __syncthreads();                                              // tables complete
     pdl_wait();                                                   // from here on: tensors the previous kernel may have written
+    const __nv_bfloat16* __restrict__ bnx = reinterpret_cast<const __nv_bfloat16*>(p.bn.x);
+    if (fuse == 2 && tid < ncol) {
+        const int c = n_off + tid;
+        s_bn[0][tid] = p.bn.stat[c]; s_bn[1][tid] = p.bn.stat[p.bn.C + c]; s_bn[2][tid] = p.bn.gamma[c]; s_bn[3][tid] = p.bn.beta[c];
+    }
     int nxt = cta;
     for (int st = 0; st < stages - 1; ++st) { if (nxt < units) issue(nxt, st); cp_async_commit(); nxt += ncta; }
     int stage = 0;
@@ -227,6 +261,9 @@ __global__ void __launch_bounds__(MMA_THREADS) conv_mma_kernel(const MmaProb* __
         // ---- epilogue: thread (g8, t4) holds rows g8 and g8+8 of each 16-row block, channels t4*2*NB ... t4*2*NB + 2*NB - 1
         const int grp = unit / subs, j0 = (unit - grp * subs) * sub;
         const long long obase = grp * grp_out + n_off + t4 * (2 * NB);
+        float ps[2 * NB], pq[2 * NB];                             // fused BN: this thread's sums over the piece
+#pragma unroll
+        for (int i = 0; i < 2 * NB; ++i) { ps[i] = 0.f; pq[i] = 0.f; }
 #pragma unroll
         for (int mb = 0; mb < MBW; ++mb)
 #pragma unroll
@@ -252,6 +289,34 @@ __global__ void __launch_bounds__(MMA_THREADS) conv_mma_kernel(const MmaProb* __
                     __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
                     wv[j] = *reinterpret_cast<uint32_t*>(&h);
                 }
+                if (fuse == 1) {                                  // sums of the STORED values: x, x^2
+#pragma unroll
+                    for (int j = 0; j < NB; ++j) {
+                        const float r0 = __uint_as_float(wv[j] << 16), r1 = __uint_as_float(wv[j] & 0xFFFF0000u);
+                        ps[2 * j] += r0; pq[2 * j] += r0 * r0; ps[2 * j + 1] += r1; pq[2 * j + 1] += r1 * r1;
+                    }
+                } else if (fuse == 2) {                           // sums of dz = da * [relu input > 0] and dz * xhat
+                    uint32_t xv[NB];
+                    if constexpr (NB % 4 == 0) {
+#pragma unroll
+                        for (int c4 = 0; c4 < NB / 4; ++c4) { const uint4 v = *reinterpret_cast<const uint4*>(bnx + o + c4 * 8); xv[c4 * 4] = v.x; xv[c4 * 4 + 1] = v.y; xv[c4 * 4 + 2] = v.z; xv[c4 * 4 + 3] = v.w; }
+                    } else {
+#pragma unroll
+                        for (int c2 = 0; c2 < NB / 2; ++c2) { const uint2 v = *reinterpret_cast<const uint2*>(bnx + o + c2 * 4); xv[c2 * 2] = v.x; xv[c2 * 2 + 1] = v.y; }
+                    }
+#pragma unroll
+                    for (int j = 0; j < NB; ++j) {
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            const int c = t4 * (2 * NB) + 2 * j + e;
+                            const float x = e ? __uint_as_float(xv[j] & 0xFFFF0000u) : __uint_as_float(xv[j] << 16);
+                            const float d = e ? __uint_as_float(wv[j] & 0xFFFF0000u) : __uint_as_float(wv[j] << 16);
+                            const float xh = (x - s_bn[0][c]) * s_bn[1][c];
+                            const float dz = (xh * s_bn[2][c] + s_bn[3][c] > 0.f) ? d : 0.f;
+                            ps[2 * j + e] += dz; pq[2 * j + e] += dz * xh;
+                        }
+                    }
+                }
                 if constexpr (NB % 4 == 0) {
 #pragma unroll
                     for (int c4 = 0; c4 < NB / 4; ++c4) *reinterpret_cast<uint4*>(outp + o + c4 * 8) = make_uint4(wv[c4 * 4], wv[c4 * 4 + 1], wv[c4 * 4 + 2], wv[c4 * 4 + 3]);
@@ -260,16 +325,110 @@ __global__ void __launch_bounds__(MMA_THREADS) conv_mma_kernel(const MmaProb* __
                     for (int c2 = 0; c2 < NB / 2; ++c2) *reinterpret_cast<uint2*>(outp + o + c2 * 4) = make_uint2(wv[c2 * 2], wv[c2 * 2 + 1]);
                 }
             }
+        if (fuse) {                                               // the 8 lanes that own the same channels, fixed butterfly; lane g8 = 0 keeps the warp's running sum
+#pragma unroll
+            for (int i = 0; i < 2 * NB; ++i) {
+#pragma unroll
+                for (int off = 4; off < 32; off <<= 1) { ps[i] += __shfl_xor_sync(0xffffffffu, ps[i], off); pq[i] += __shfl_xor_sync(0xffffffffu, pq[i], off); }
+            }
+            if (g8 == 0) {
+#pragma unroll
+                for (int i = 0; i < 2 * NB; ++i) { s_red[warp][0][t4 * (2 * NB) + i] += ps[i]; s_red[warp][1][t4 * (2 * NB) + i] += pq[i]; }
+            }
+        }
         __syncthreads();                                          // every warp is done with this stage before it is refilled
         stage = stage + 1 == stages ? 0 : stage + 1;
     }
     cp_async_wait<0>();
+    if (!fuse) return;
+
+    // ---- fused BN: this CTA's sums (warps added in order, in double) -> partial[cta][2][C]; grid barrier; statistics; elementwise pass
+    const BnProb& bn = p.bn;
+    const int C = bn.C;                                           // = ncol_all
+    __syncthreads();
+    if (cta < units && tid < 2 * ncol) {
+        const int k = tid / ncol, c = tid - k * ncol;
+        double a = 0.0;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) a += (double)s_red[w][k][c];
+        bn.partial[((long long)cta * 2 + k) * C + n_off + c] = a;
+    }
+    __threadfence();
+    cg::this_grid().sync();
+    float* s_stat = reinterpret_cast<float*>(sm);                 // [6][C]: mean, 1/std, sum dz, sum dz*xhat, gamma, beta (the tables are no longer needed)
+    double* s_dred = reinterpret_cast<double*>(sm + 6 * 64 * 4);  // [2][256]
+    {
+        const int rows = min(ncta, units), Q = MMA_THREADS / C, c = tid % C, q = tid / C;   // C is 16, 32 or 64
+        double a0 = 0.0, a1 = 0.0;
+#pragma unroll 4
+        for (int k = q; k < rows; k += Q) { a0 += __ldcg(bn.partial + ((long long)k * 2 + 0) * C + c); a1 += __ldcg(bn.partial + ((long long)k * 2 + 1) * C + c); }
+        s_dred[tid] = a0; s_dred[256 + tid] = a1;
+        __syncthreads();
+        if (q == 0) {
+            a0 = 0.0; a1 = 0.0;
+            for (int k = 0; k < Q; ++k) { a0 += s_dred[k * C + c]; a1 += s_dred[256 + k * C + c]; }
+            if (fuse == 1) {
+                const double m = (double)bn.m, mean = a0 / m;
+                double var = a1 / m - mean * mean; if (var < 0.0) var = 0.0;
+                const float fm = (float)mean, fi = (float)(1.0 / sqrt(var + (double)bn.eps));
+                s_stat[c] = fm; s_stat[C + c] = fi;
+                if (blockIdx.x == 0) {
+                    bn.stat[c] = fm; bn.stat[C + c] = fi;
+                    if (bn.run_mean) {
+                        const double unb = bn.m > 1 ? var * m / (m - 1.0) : var, mo = (double)bn.momentum;
+                        bn.run_mean[c] = (float)((1.0 - mo) * (double)bn.run_mean[c] + mo * mean);
+                        bn.run_var[c] = (float)((1.0 - mo) * (double)bn.run_var[c] + mo * unb);
+                    }
+                }
+            } else {
+                s_stat[c] = bn.stat[c]; s_stat[C + c] = bn.stat[C + c];
+                s_stat[2 * C + c] = (float)a0; s_stat[3 * C + c] = (float)a1;
+                if (blockIdx.x == 0) { bn.stat[2 * C + c] = (float)a0; bn.stat[3 * C + c] = (float)a1; bn.dbeta[c] = (float)a0; bn.dgamma[c] = (float)a1; }
+            }
+        }
+        __syncthreads();
+    }
+    // elementwise pass, 8 channels per access; the per-channel constants are read from shared memory where they are used
+    // (kept in registers they would raise the register count of the whole kernel)
+    {
+        if (tid < C) { s_stat[4 * C + tid] = bn.gamma[tid]; s_stat[5 * C + tid] = bn.beta[tid]; }
+        __syncthreads();
+        const int G = C >> 3;
+        const long long nv = bn.m * G, stride = (long long)gridDim.x * MMA_THREADS;
+        const float inv_m = 1.f / (float)bn.m;
+        const uint4* xv = reinterpret_cast<const uint4*>(bn.x);
+        const uint4* dv = reinterpret_cast<const uint4*>(bn.da);
+        const uint4* av = reinterpret_cast<const uint4*>(bn.add);
+        uint4* ov = reinterpret_cast<uint4*>(fuse == 1 ? bn.a : bn.dx);
+        for (long long v = (long long)blockIdx.x * MMA_THREADS + tid; v < nv; v += stride) {
+            const float* st = s_stat + ((int)v & (G - 1)) * 8;
+            float x[8], o[8]; bf8_unpack(__ldcg(xv + v), x);
+            if (fuse == 1) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) { const float z = (x[j] - st[j]) * st[C + j] * st[4 * C + j] + st[5 * C + j]; o[j] = z > 0.f ? z : 0.f; }
+            } else {
+                float d[8]; bf8_unpack(__ldcg(dv + v), d);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const float istd = st[C + j], ga = st[4 * C + j];
+                    const float xh = (x[j] - st[j]) * istd;
+                    const float dz = (xh * ga + st[5 * C + j] > 0.f) ? d[j] : 0.f;
+                    o[j] = ga * istd * (dz - st[2 * C + j] * inv_m - xh * st[3 * C + j] * inv_m);
+                }
+                if (av) { float ad[8]; bf8_unpack(__ldcg(av + v), ad);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) o[j] += ad[j]; }
+            }
+            ov[v] = bf8_pack(o);
+        }
+    }
 }
 
 // ------------------------------------------------------------------------------------------------ host side
 struct MmaGeom { int ca, ncol, Hp, Wp, G, gpos, sub, subs, units, mbw, stages, nsplit, variant; size_t smem; };
 
-// variant = ((MBW * 4 + ksz) * 2 + trans) * 16 + NB: everything a launch is specialised on
+// variant = ((MBW * 4 + ksz) * 2 + trans) * 16 + NB: everything a launch is specialised on; + MMA_VARIANT_FUSED: with BN
+constexpr int MMA_VARIANT_FUSED = 512;
 static int mma_variant(int mbw, int ksz, int trans, int nb) { return ((mbw * 4 + ksz) * 2 + trans) * 16 + nb; }
 
 static bool mma_geometry(const ConvProb& p, int mode, MmaGeom& g) {
@@ -322,7 +481,14 @@ bool conv_mma_supported(const ConvProb& p, int mode) { MmaGeom g; return mma_geo
 int conv_mma_pick_variant(const ConvProb& p, int mode) { MmaGeom g; return mma_geometry(p, mode, g) ? g.variant : 0; }
 size_t conv_mma_prob_bytes() { return sizeof(MmaProb); }
 
-bool conv_mma_fill(const ConvProb& p, int mode, void* host) {
+// bn != nullptr: the BN+ReLU that consumes the output runs in the same launch (forward of mode CONV_FWD, backward of
+// CONV_DGRAD); bn->partial must hold conv_mma_bn_partial_bytes(C) bytes
+size_t conv_mma_bn_partial_bytes(int C, int sms) { return (size_t)3 * sms * 2 * C * sizeof(double); }
+bool conv_mma_can_fuse_bn(const ConvProb& p, int mode, int C) {
+    MmaGeom g; if (!mma_geometry(p, mode, g)) return false;
+    return (C == 16 || C == 32 || C == 64) && C == g.ncol && g.ncol / g.nsplit <= 32;
+}
+bool conv_mma_fill(const ConvProb& p, int mode, void* host, const BnProb* bn) {
     MmaGeom g; if (!mma_geometry(p, mode, g)) return false;
     MmaProb t; memset(&t, 0, sizeof(t));
     t.act = (const __nv_bfloat16*)p.act; t.wgt = (const __nv_bfloat16*)p.wgt; t.add = (const __nv_bfloat16*)p.add; t.out = (__nv_bfloat16*)p.out;
@@ -331,6 +497,11 @@ bool conv_mma_fill(const ConvProb& p, int mode, void* host) {
     t.G = g.G; t.gpos = g.gpos; t.sub = g.sub; t.subs = g.subs; t.units = g.units;
     t.os = mode == CONV_FWD ? p.stride : 1; t.P = p.P; t.Q = p.Q;
     t.stages = g.stages; t.nsplit = g.nsplit; t.variant = g.variant; t.smem_bytes = (int)g.smem; t.scale = p.scale;
+    if (bn) {
+        if (!conv_mma_can_fuse_bn(p, mode, bn->C)) return false;
+        t.fuse = mode == CONV_FWD ? 1 : 2; t.bn = *bn; t.variant |= MMA_VARIANT_FUSED;
+        if (t.smem_bytes < 8192) t.smem_bytes = 8192;             // the BN phase reuses the start of the dynamic shared memory (5.5 KB)
+    }
     memcpy(host, &t, sizeof(t));
     return true;
 }
@@ -338,33 +509,57 @@ int conv_mma_tiles(const void* h) { return ((const MmaProb*)h)->units * ((const 
 int conv_mma_variant(const void* h) { return ((const MmaProb*)h)->variant; }
 size_t conv_mma_smem(const void* h) { return (size_t)((const MmaProb*)h)->smem_bytes; }
 
+struct MmaLaunch { const void* d; int nprob, max_tiles; size_t smem; bool pdl, coop; cudaStream_t s; bool ok; };
+
+// Persistent CTAs: as many as are co-resident at this shared-memory footprint (at most 3 per SM), over all problems.
+// A fused launch is cooperative (grid barrier): its grid never exceeds what is co-resident.
 template <int NB, int MBW, int KSZ, bool TRANS>
-static void launch_mma_inst(const void* d, dim3 grid, size_t smem, bool pdl, cudaStream_t s) {
-    static bool configured = false;
-    if (!configured) { cudaFuncSetAttribute(conv_mma_kernel<NB, MBW, KSZ, TRANS>, cudaFuncAttributeMaxDynamicSharedMemorySize, 202 * 1024); configured = true; }
-    launch_pdl(conv_mma_kernel<NB, MBW, KSZ, TRANS>, grid, smem, s, pdl, (const MmaProb*)d);
+static void launch_mma_inst(MmaLaunch& a) {
+    static bool configured = false; static int sms = 0; static signed char occ[256] = {};
+    static int coop_pdl = 1;                                      // 1: cooperative + programmatic launch together until the driver refuses it
+    auto kernel = conv_mma_kernel<NB, MBW, KSZ, TRANS>;
+    if (!configured) {
+        cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 202 * 1024);
+        int dev = 0; cudaGetDevice(&dev); cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev); if (sms < 1) sms = 148;
+        configured = true;
+    }
+    const int slot = (int)std::min<size_t>(a.smem / 1024, 255);
+    if (!occ[slot]) { int n = 0; cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, MMA_THREADS, (a.smem / 1024 + 1) * 1024); occ[slot] = (signed char)std::max(1, std::min(n, 3)); }
+    const int cap = occ[slot] * sms;
+    int gx = a.coop ? cap / a.nprob : (cap + a.nprob - 1) / a.nprob;
+    if (gx > a.max_tiles) gx = a.max_tiles;
+    gx &= ~1;                                                     // even: a CTA pair shares a piece when the channels are split
+    if (gx < 2) gx = 2;
+    if (a.coop && gx * a.nprob > cap) { a.ok = false; return; }
+    cudaLaunchConfig_t cfg = {}; cfg.gridDim = dim3(gx, a.nprob); cfg.blockDim = dim3(MMA_THREADS); cfg.dynamicSmemBytes = a.smem; cfg.stream = a.s;
+    cudaLaunchAttribute at[2]; int n = 0;
+    if (a.coop) { at[n].id = cudaLaunchAttributeCooperative; at[n].val.cooperative = 1; ++n; }
+    if (a.pdl && (!a.coop || coop_pdl)) { at[n].id = cudaLaunchAttributeProgrammaticStreamSerialization; at[n].val.programmaticStreamSerializationAllowed = 1; ++n; }
+    cfg.attrs = at; cfg.numAttrs = n;
+    const MmaProb* d = (const MmaProb*)a.d;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, d);
+    if (e != cudaSuccess && a.coop && n == 2) {                   // the combination is refused: cooperative alone from now on
+        cudaGetLastError(); coop_pdl = 0; cfg.numAttrs = 1;
+        e = cudaLaunchKernelEx(&cfg, kernel, d);
+    }
+    a.ok = e == cudaSuccess;
 }
 template <int NB, int MBW>
-static void launch_mma_nb(const void* d, dim3 grid, size_t smem, int ksz, int trans, bool pdl, cudaStream_t s) {
-    if (ksz == 3) { if (trans) launch_mma_inst<NB, MBW, 3, true>(d, grid, smem, pdl, s); else launch_mma_inst<NB, MBW, 3, false>(d, grid, smem, pdl, s); }
-    else { if (trans) launch_mma_inst<NB, MBW, 1, true>(d, grid, smem, pdl, s); else launch_mma_inst<NB, MBW, 1, false>(d, grid, smem, pdl, s); }
+static void launch_mma_nb(MmaLaunch& a, int ksz, int trans) {
+    if (ksz == 3) { if (trans) launch_mma_inst<NB, MBW, 3, true>(a); else launch_mma_inst<NB, MBW, 3, false>(a); }
+    else { if (trans) launch_mma_inst<NB, MBW, 1, true>(a); else launch_mma_inst<NB, MBW, 1, false>(a); }
 }
 // all problems of one launch share the variant
 // pdl: the kernel may start before the previous kernel of the stream has finished (that kernel must not write the weights)
-void launch_conv_mma_probs(const void* d, int nprob, int max_tiles, size_t max_smem, int variant, cudaStream_t s, bool pdl) {
-    static int sms = 0;
-    if (!sms) { int dev = 0; cudaGetDevice(&dev); cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev); if (sms < 1) sms = 148; }
+bool launch_conv_mma_probs(const void* d, int nprob, int max_tiles, size_t max_smem, int variant, cudaStream_t s, bool pdl) {
     const int nb = variant & 15, trans = (variant >> 4) & 1, ksz = (variant >> 5) & 3, mbw = (variant >> 7) & 3;
-    // persistent CTAs: as many as fit on the chip at this shared-memory footprint (at most 3 per SM), over all problems
-    int per_sm = (int)((227 * 1024) / (max_smem + 1024)); if (per_sm > 3) per_sm = 3; if (per_sm < 1) per_sm = 1;
-    int gx = (per_sm * sms + nprob - 1) / nprob; if (gx > max_tiles) gx = max_tiles; if (gx < 2) gx = 2;
-    gx &= ~1;                                                      // even: a CTA pair shares a piece when the channels are split
-    const dim3 grid(gx, nprob);
-#define MMA_CASE(N_, M_) if (nb == N_ && mbw == M_) launch_mma_nb<N_, M_>(d, grid, max_smem, ksz, trans, pdl, s); else
+    MmaLaunch a{d, nprob, max_tiles, max_smem, pdl, (variant & MMA_VARIANT_FUSED) != 0, s, false};
+#define MMA_CASE(N_, M_) if (nb == N_ && mbw == M_) launch_mma_nb<N_, M_>(a, ksz, trans); else
     MMA_CASE(2, 1) MMA_CASE(2, 2) MMA_CASE(2, 3) MMA_CASE(4, 1) MMA_CASE(4, 2) MMA_CASE(4, 3)
     MMA_CASE(6, 1) MMA_CASE(6, 2) MMA_CASE(8, 1) MMA_CASE(8, 2)
-    return;
+    return false;
 #undef MMA_CASE
+    return a.ok;
 }
 
 // ------------------------------------------------------------------------------------------------ wgrad

@@ -21,11 +21,11 @@ size_t conv_wgrad_tc_smem(const void* h);
 long long conv_wgrad_tc_out_elems(const void* h);
 void launch_conv_wgrad_tc_probs(const void* d_tc, int nprob, int max_ctas, size_t max_smem, long long max_out, cudaStream_t s);
 bool conv_mma_supported(const ConvProb& p, int mode);
-bool conv_mma_fill(const ConvProb& p, int mode, void* host);
+bool conv_mma_fill(const ConvProb& p, int mode, void* host, const BnProb* bn = nullptr);
 size_t conv_mma_prob_bytes();
 int conv_mma_tiles(const void* h);
 size_t conv_mma_smem(const void* h);
-void launch_conv_mma_probs(const void* d, int nprob, int max_tiles, size_t max_smem, int variant, cudaStream_t s, bool pdl = false);
+bool launch_conv_mma_probs(const void* d, int nprob, int max_tiles, size_t max_smem, int variant, cudaStream_t s, bool pdl = false);
 int conv_mma_pick_variant(const ConvProb& p, int mode);
 bool conv_wgrad_mma_supported(const ConvProb& p, int target_ctas, size_t* partial_bytes);
 bool conv_wgrad_mma_fill(const ConvProb& p, int target_ctas, void* host);

@@ -29,11 +29,14 @@ long long conv_wgrad_tc_out_elems(const void* h);
 void launch_conv_wgrad_tc_probs(const void* d_tc, int nprob, int max_ctas, size_t max_smem, long long max_out, cudaStream_t s);
 static int wgrad_target_ctas(const resist_ctx* ctx) { return std::max(8, 2 * ctx->sm_count / std::max(1, ctx->S)); }
 bool conv_mma_supported(const ConvProb& p, int mode);                                   // conv_mma.cu
-bool conv_mma_fill(const ConvProb& p, int mode, void* host);
+bool conv_mma_fill(const ConvProb& p, int mode, void* host, const BnProb* bn = nullptr);
+bool conv_mma_can_fuse_bn(const ConvProb& p, int mode, int C);
+size_t conv_mma_bn_partial_bytes(int C, int sms);
 size_t conv_mma_prob_bytes();
 int conv_mma_tiles(const void* h);
 size_t conv_mma_smem(const void* h);
-void launch_conv_mma_probs(const void* d, int nprob, int max_tiles, size_t max_smem, int variant, cudaStream_t s, bool pdl = false);
+bool launch_conv_mma_probs(const void* d, int nprob, int max_tiles, size_t max_smem, int variant, cudaStream_t s, bool pdl = false);
+constexpr int MMA_BACKEND_FUSED = 512;                       // added to a warp-MMA forward/dgrad backend value: the consuming BN runs in the same launch
 int conv_mma_pick_variant(const ConvProb& p, int mode);
 bool conv_wgrad_mma_supported(const ConvProb& p, int target_ctas, size_t* partial_bytes);
 bool conv_wgrad_mma_fill(const ConvProb& p, int target_ctas, void* host);
@@ -48,7 +51,7 @@ int conv_wgrad_mma_pick_variant(const ConvProb& p, int target_ctas);
 // output channels; forward and dgrad: 1000 + the kernel variant, so that the value also separates launches by what
 // the kernel is specialised on).
 static int pick_backend(const ConvProb& p, int mode, int target_ctas, size_t* partial_bytes, int pref = RESIST_CONV_AUTO) {
-    const bool want_mma = pref == RESIST_CONV_AUTO || pref == RESIST_CONV_WARP_MMA, want_tc = pref == RESIST_CONV_AUTO || pref == RESIST_CONV_TCGEN05;
+    const bool want_mma = pref == RESIST_CONV_AUTO || pref == RESIST_CONV_WARP_MMA || pref == RESIST_CONV_WARP_MMA_UNFUSED, want_tc = pref == RESIST_CONV_AUTO || pref == RESIST_CONV_TCGEN05;
     if (mode == CONV_WGRAD) {
         if (want_mma && conv_wgrad_mma_supported(p, target_ctas, partial_bytes)) return 200 + conv_wgrad_mma_pick_variant(p, target_ctas);
         if (want_tc && conv_wgrad_tc_supported(p, target_ctas, partial_bytes)) return 1;
@@ -99,6 +102,15 @@ struct Builder {
     char* gbuf[6] = {}; bool gused[6] = {}; size_t gbig = 0;
     float* logits = nullptr;
     long long flops = 0; int n_tc = 0, n_cc = 0;
+    // The BN+ReLU that consumes a warp-MMA convolution's output joins that convolution's launch (forward: the BN of the
+    // output; backward: the BN backward whose da the data gradient produces).  Index of the candidate in *ops, or -1.
+    int last_fwd_conv = -1, last_dgrad = -1;
+    bool fusable(int idx, const void* tensor, const BnProb& p) const {
+        if (idx < 0 || eval || ctx->opts.dtype != RESIST_BF16 || (ctx->opts.conv_backend != RESIST_CONV_AUTO && ctx->opts.conv_backend != RESIST_CONV_WARP_MMA)) return false;
+        const Op& o = (*ops)[idx];
+        const int cout = o.kind == OP_CONV_FWD ? o.conv.K : o.conv.C;
+        return o.backend >= 1000 && o.conv.out == tensor && p.vec && p.C == cout && conv_mma_can_fuse_bn(o.conv, o.kind == OP_CONV_FWD ? CONV_FWD : CONV_DGRAD, p.C);
+    }
 
     void* take(size_t bytes) { off = align_up(off, 256); void* p = base ? base + off : nullptr; off += bytes; return p; }
     void* act(long long elems) { size_t b = (size_t)elems * es; if (b > gbig) gbig = b; return take(b); }
@@ -168,7 +180,16 @@ struct Builder {
             }
         }
         ops->push_back(op);
+        if (mode == CONV_FWD) last_fwd_conv = op.backend >= 1000 ? (int)ops->size() - 1 : -1;
+        if (mode == CONV_DGRAD) last_dgrad = op.backend >= 1000 ? (int)ops->size() - 1 : -1;
         if (mode == CONV_WGRAD && p.splits > 1) { Op r = op; r.key = key + 1; r.kind = OP_SPLITK; r.patch_images = 0; ops->push_back(r); }
+    }
+    // the BN joins the launch of the convolution at *ops[idx]
+    void fuse_into(int idx, const BnProb& p, int which) {
+        Op& o = (*ops)[idx];
+        o.fuse = which; o.bn = p; o.backend += MMA_BACKEND_FUSED;
+        bn_partial_need = std::max(bn_partial_need, conv_mma_bn_partial_bytes(p.C, ctx->sm_count));
+        o.bn.partial = bn_partial;
     }
 
     // A stem with few input channels (C * k * k <= 32, bf16): the images are expanded once per step to rows of 32
@@ -201,6 +222,7 @@ struct Builder {
         if (mode == CONV_WGRAD) { wgrad_partial_need = std::max(wgrad_partial_need, pb); p.partial = wgrad_partial; }
         ++n_tc;
         ops->push_back(op);
+        if (mode == CONV_FWD) last_fwd_conv = op.backend >= 1000 ? (int)ops->size() - 1 : -1;
     }
 
     // chunks per BN problem that give the fused (cooperative) kernels about two CTAs per SM over all sub-ResNets
@@ -216,6 +238,8 @@ struct Builder {
         bn_chunking(p, ctx->opts.dtype == RESIST_BF16, fused_chunks());
         bn_partial_need = std::max(bn_partial_need, (size_t)p.chunks * 2 * r.c * 8);
         p.partial = bn_partial;
+        const int producer = last_fwd_conv; last_fwd_conv = -1;
+        if (fusable(producer, x, p)) { fuse_into(producer, p, 1); return stat; }                            // inside the producing convolution's launch
         if (p.vec && !eval && r.c <= 512) { op.kind = OP_BN_FWD_FUSED; ops->push_back(op); return stat; }   // one cooperative launch
         ops->push_back(op);
         op.key = key + 1; op.kind = OP_BN_APPLY; ops->push_back(op);
@@ -229,6 +253,8 @@ struct Builder {
         bn_chunking(p, ctx->opts.dtype == RESIST_BF16, fused_chunks());
         bn_partial_need = std::max(bn_partial_need, (size_t)p.chunks * 2 * r.c * 8);
         p.partial = bn_partial;
+        const int producer = last_dgrad; last_dgrad = -1;
+        if (fusable(producer, da, p)) { fuse_into(producer, p, 2); return; }
         if (p.vec && r.c <= 512) { op.kind = OP_BN_BWD_FUSED; ops->push_back(op); return; }
         ops->push_back(op);
         op.key = key + 1; op.kind = OP_BN_BWD_APPLY; ops->push_back(op);
@@ -262,7 +288,7 @@ static size_t unroll_subnet(resist_ctx* ctx, Builder& bd, const std::vector<char
         stem_p = bd.act((long long)B * Hp * Wp * cC); stem_arg = (int*)bd.take((size_t)B * Hp * Wp * cC * 4);
         Op op{}; op.key = 3; op.sub = bd.sub; op.kind = OP_POOL_FWD;
         op.pool = PoolProb{cur, stem_p, stem_arg, nullptr, nullptr, B, cH, cW, cC, Hp, Wp};
-        bd.ops->push_back(op);
+        bd.ops->push_back(op); bd.last_fwd_conv = -1;
         cur = stem_p; cH = Hp; cW = Wp;
     }
 
@@ -369,7 +395,7 @@ static size_t unroll_subnet(resist_ctx* ctx, Builder& bd, const std::vector<char
         Op op{}; op.key = BWD_END; op.sub = bd.sub; op.kind = OP_POOL_BWD;
         op.pool = PoolProb{stem_a ? stem_a : stem_y, nullptr, stem_arg, bd.gbuf[g_cur], bd.gbuf[g], B, Hs, Ws, A.stem_cout, cH, cW};
         op.pool.P = out_dim(Hs, 3, 2); op.pool.Q = out_dim(Ws, 3, 2);
-        bd.ops->push_back(op); bd.grel(g_cur); g_cur = g;
+        bd.ops->push_back(op); bd.grel(g_cur); g_cur = g; bd.last_dgrad = -1;
     }
     if (A.stem_bn_relu) { const int g = bd.gtake(); bd.bn_bwd(BWD_END + 1, stem_y, bd.gbuf[g_cur], bd.gbuf[g], nullptr, L.stem_bn, stem_stat, m_stem); bd.grel(g_cur); g_cur = g; }
     if (stem_col) bd.stem_conv(BWD_END + 3, CONV_WGRAD, L.stem, bd.gbuf[g_cur], nullptr, B, A.in_h, A.in_w);
@@ -442,10 +468,13 @@ static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool s
                             if (k == i) L.first = n_mm;
                             mm.resize((size_t)(n_mm + 1) * mmb); char* h = mm.data() + (size_t)n_mm * mmb;
                             const int mode = o.kind == OP_CONV_FWD ? CONV_FWD : CONV_DGRAD;
-                            if (!conv_mma_fill(o.conv, mode, h)) { ctx->err = "conv descriptor failed"; return RESIST_EINVAL; }
+                            if (!conv_mma_fill(o.conv, mode, h, o.fuse ? &o.bn : nullptr)) { ctx->err = "conv descriptor failed"; return RESIST_EINVAL; }
                             L.gx = std::max(L.gx, conv_mma_tiles(h));
                             L.max_elems = std::max<long long>(L.max_elems, (long long)conv_mma_smem(h));
                             ++n_mm; L.bytes += es * (in_e + out_e + w_e + (p.add ? (o.kind == OP_CONV_FWD ? out_e : in_e) : 0.0));
+                            // fused BN: forward writes a (its read of the output just written is an L2 hit); backward reads x (+ the skip gradient) and writes dx
+                            if (o.fuse == 1) L.bytes += es * out_e;
+                            if (o.fuse == 2) L.bytes += es * in_e * (o.bn.add ? 3 : 2);
                         }
                         break;
                     }
@@ -544,7 +573,9 @@ static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool s
             for (size_t k = i; k < j; ++k) {
                 const Op& o = ops[k];
                 switch (o.kind) {
-                    case OP_CONV_FWD: case OP_CONV_DGRAD: wr.push_back(o.conv.out); break;
+                    case OP_CONV_FWD: case OP_CONV_DGRAD: wr.push_back(o.conv.out);
+                        if (o.fuse == 1) wr.push_back(o.bn.a); else if (o.fuse == 2) wr.push_back(o.bn.dx);
+                        break;
                     case OP_CONV_WGRAD: case OP_SPLITK: break;
                     case OP_BN_STATS: case OP_BN_BWD_REDUCE: break;
                     case OP_BN_APPLY: case OP_BN_FWD_FUSED: wr.push_back(o.bn.a); break;
@@ -695,8 +726,8 @@ static int run_plan(resist_ctx* ctx, Plan& plan, const PatchArgs& pa, bool updat
         }
         int pk = 0, nk = 1;
         switch (L.kind) {
-            case OP_CONV_FWD: pk = L.backend >= 200 ? PK_CONV_FWD_MMA : L.backend ? PK_CONV_FWD_TC : PK_CONV_FWD_CC; break;
-            case OP_CONV_DGRAD: pk = L.backend >= 200 ? PK_CONV_DGRAD_MMA : L.backend ? PK_CONV_DGRAD_TC : PK_CONV_DGRAD_CC; break;
+            case OP_CONV_FWD: pk = L.backend >= 1000 + MMA_BACKEND_FUSED ? PK_CONV_FWD_MMA_BN : L.backend >= 200 ? PK_CONV_FWD_MMA : L.backend ? PK_CONV_FWD_TC : PK_CONV_FWD_CC; break;
+            case OP_CONV_DGRAD: pk = L.backend >= 1000 + MMA_BACKEND_FUSED ? PK_CONV_DGRAD_MMA_BN : L.backend >= 200 ? PK_CONV_DGRAD_MMA : L.backend ? PK_CONV_DGRAD_TC : PK_CONV_DGRAD_CC; break;
             case OP_CONV_WGRAD: pk = L.backend >= 200 ? PK_CONV_WGRAD_MMA : L.backend ? PK_CONV_WGRAD_TC : PK_CONV_WGRAD_CC; break;
             case OP_SPLITK: pk = PK_SPLITK; break;
             case OP_BN_STATS: pk = PK_BN_STATS; nk = 2; break;
@@ -717,7 +748,10 @@ static int run_plan(resist_ctx* ctx, Plan& plan, const PatchArgs& pa, bool updat
             case OP_CONV_FWD: case OP_CONV_DGRAD: case OP_CONV_WGRAD: {
                 const int mode = L.kind == OP_CONV_FWD ? CONV_FWD : L.kind == OP_CONV_DGRAD ? CONV_DGRAD : CONV_WGRAD;
                 if (L.backend >= 200 && mode == CONV_WGRAD) { launch_conv_wgrad_mma_probs((const char*)plan.d_wmm + (size_t)L.first * plan.wmm_stride, L.count, L.gx, (size_t)L.max_elems, L.max_b, L.backend - 200, st, pdl_ok); ++n_launch; }
-                else if (L.backend >= 200) launch_conv_mma_probs((const char*)plan.d_mm + (size_t)L.first * plan.mm_stride, L.count, L.gx, (size_t)L.max_elems, L.backend - 1000, st, pdl_ok);
+                else if (L.backend >= 200) {
+                    if (!launch_conv_mma_probs((const char*)plan.d_mm + (size_t)L.first * plan.mm_stride, L.count, L.gx, (size_t)L.max_elems, L.backend - 1000, st, pdl_ok)) {
+                        ctx->err = "warp-MMA convolution launch failed"; cudaGetLastError(); return RESIST_ECUDA; }
+                }
                 else if (L.backend && mode == CONV_WGRAD) { launch_conv_wgrad_tc_probs((const char*)plan.d_wtc + (size_t)L.first * plan.wtc_stride, L.count, L.gx, (size_t)L.max_elems, L.max_b, st); ++n_launch; }
                 else if (L.backend) launch_conv_tc_probs((const char*)plan.d_tc + (size_t)L.first * plan.tc_stride, L.count, L.gx, (size_t)L.max_elems, st);
                 else launch_conv_ref(plan.d_conv + L.first, L.count, L.gx, mode, bf, st);

@@ -27,6 +27,7 @@ struct Op {
     ConvProb conv; BnProb bn; PoolProb pool; HeadProb head; UpProb up; ColProb col;
     int backend;          // convolutions: 0 = CUDA cores, 1 = tensor cores
     int patch_images;     // conv.act must be replaced by the caller's image pointer
+    int fuse;             // warp-MMA convolutions: 1 = `bn` is the BN+ReLU forward of the output, 2 = the BN+ReLU backward whose da is the output; it runs in the same launch
 };
 
 struct PatchSite { void** where; int what; int sub; };        // what: 0 images, 1 labels, 2 loss_out, 3 logits_out, 4 correct
@@ -41,7 +42,7 @@ struct Launch {
 enum ProfKind {
     PK_CONV_FWD_CC, PK_CONV_DGRAD_CC, PK_CONV_WGRAD_CC, PK_CONV_FWD_TC, PK_CONV_DGRAD_TC, PK_CONV_WGRAD_TC, PK_SPLITK,
     PK_BN_STATS, PK_BN_APPLY, PK_BN_BWD_REDUCE, PK_BN_BWD_APPLY, PK_POOL_FWD, PK_POOL_BWD, PK_HEAD_FWD, PK_HEAD_BWD,
-    PK_SGD, PK_PATCH, PK_SCATTER, PK_AGGREGATE, PK_UPSAMPLE, PK_CONV_FWD_MMA, PK_CONV_DGRAD_MMA, PK_CONV_WGRAD_MMA, PK_IM2COL, PK_BN_FWD_FUSED, PK_BN_BWD_FUSED, PK_COUNT
+    PK_SGD, PK_PATCH, PK_SCATTER, PK_AGGREGATE, PK_UPSAMPLE, PK_CONV_FWD_MMA, PK_CONV_DGRAD_MMA, PK_CONV_WGRAD_MMA, PK_IM2COL, PK_BN_FWD_FUSED, PK_BN_BWD_FUSED, PK_CONV_FWD_MMA_BN, PK_CONV_DGRAD_MMA_BN, PK_COUNT
 };
 struct Profiler {
     bool on = false;

@@ -116,7 +116,7 @@ def check_bf16(out, arch, tol=2e-2, grads=True):
 #   * whole-step gradients are checked for direction against the oracle run with the same storage rounding
 #     (quant=1): even there one rounding tie broken the other way by the summation order flips a mask and
 #     moves a small tensor by 10 % (seen on the tiny net at batch 8).
-@pytest.mark.parametrize("backend", [1, 0, 2])
+@pytest.mark.parametrize("backend", [1, 0, 2, 4])
 def test_tiny_bf16_step(lib_mod, backend):
     c = synth.config(1)
     out = run_protocol_both(c.arch, 2, 8, 1, 5, "bf16", 0, True, lib_mod, conv_backend=backend)
@@ -129,7 +129,7 @@ def test_tiny_bf16_step(lib_mod, backend):
             assert g @ h / (np.linalg.norm(g) * np.linalg.norm(h)) > 0.97, s
 
 
-@pytest.mark.parametrize("backend", [1, 0, 2])
+@pytest.mark.parametrize("backend", [1, 0, 2, 4])
 def test_resnet110_bf16_reduced_batch(lib_mod, backend):
     # configuration 2's network and S at batch 8 (the oracle finishes in seconds); one local step
     c = synth.config(2)
