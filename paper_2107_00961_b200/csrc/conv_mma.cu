@@ -113,8 +113,9 @@ template <int NB> __host__ __device__ __forceinline__ int col_of_chan(int c) { r
 // ldmatrix + mma.sync on the current one.  Warp w computes the 16-row blocks w, w + 8, ... of a piece.
 // NB = output channels / 8 (2, 4, 6 or 8); MBW = 16-row blocks per warp (a piece has at most 128 * MBW positions);
 // KSZ = 1 or 3; TRANS = false: forward (weights read as [n][k]); true: dgrad (weights read as [k][n] and transposed
-// on load, taps flipped).
-template <int NB, int MBW, int KSZ, bool TRANS>
+// on load, taps flipped).  CA = channels of the staged activations when the instance is specialised on them (all pitches
+// and the reduction loop are then compile-time), 0 = read from the problem.
+template <int NB, int MBW, int KSZ, bool TRANS, int CA>
 __global__ void __launch_bounds__(MMA_THREADS) conv_mma_kernel(const MmaProb* __restrict__ probs) {
     __shared__ MmaProb p;
     if (threadIdx.x < sizeof(MmaProb) / 4) reinterpret_cast<uint32_t*>(&p)[threadIdx.x] = reinterpret_cast<const uint32_t*>(probs + blockIdx.y)[threadIdx.x];
@@ -130,7 +131,7 @@ __global__ void __launch_bounds__(MMA_THREADS) conv_mma_kernel(const MmaProb* __
     extern __shared__ __align__(16) uint8_t sm[];
     __shared__ float s_red[8][2][NB * 8];                         // per-warp sums of the fused BN, over the CTA's whole walk
     __shared__ float s_bn[4][NB * 8];                             // fuse 2: mean, 1/std, gamma, beta of this CTA's channels
-    const int ca = p.ca, apitch = ca * 2 + 16;                    // activation row pitch in bytes
+    const int ca = CA ? CA : p.ca, apitch = ca * 2 + 16;          // activation row pitch in bytes
     const int wrows = TRANS ? ca : ncol;                          // rows of one tap of the staged filter
     const int wcols = TRANS ? ncol : ca;                          // elements per row
     const int wpitch = wcols * 2 + 16;
@@ -167,20 +168,42 @@ __global__ void __launch_bounds__(MMA_THREADS) conv_mma_kernel(const MmaProb* __
     // ---- the filter, once per CTA
     if (!TRANS) {               // tap t, column n, 8-channel group g  <-  w[chan_of_col(n)][t][g*8..]
         const int groups = ca / 8, n_chunks = TAPS * ncol * groups;
-        for (int id = tid; id < n_chunks; id += MMA_THREADS) {
-            const int g = id % groups, n = (id / groups) % ncol, t = id / (groups * ncol);
-            const uint4 v = __ldg(reinterpret_cast<const uint4*>(p.wgt + ((long long)(n_off + chan_of_col<NB>(n)) * TAPS + t) * p.wC + g * 8));
-            *reinterpret_cast<uint4*>(s_w + (t * wrows + n) * wpitch + g * 16) = v;
+        for (int id0 = tid; id0 < n_chunks; id0 += 4 * MMA_THREADS) {       // four loads in flight per thread
+            uint4 v[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int id = min(id0 + u * MMA_THREADS, n_chunks - 1);
+                const int g = id % groups, n = (id / groups) % ncol, t = id / (groups * ncol);
+                v[u] = __ldg(reinterpret_cast<const uint4*>(p.wgt + ((long long)(n_off + chan_of_col<NB>(n)) * TAPS + t) * p.wC + g * 8));
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int id = id0 + u * MMA_THREADS;
+                if (id < n_chunks) { const int g = id % groups, n = (id / groups) % ncol, t = id / (groups * ncol);
+                    *reinterpret_cast<uint4*>(s_w + (t * wrows + n) * wpitch + g * 16) = v[u]; }
+            }
         }
     } else {                    // tap t, row k, column col_of_chan(c)  <-  w[k][t][c]
         constexpr int groups = ncol / 8; const int n_chunks = TAPS * ca * groups;
-        for (int id = tid; id < n_chunks; id += MMA_THREADS) {
-            const int g = id % groups, k = (id / groups) % ca, t = id / (groups * ca);
-            const uint4 v = __ldg(reinterpret_cast<const uint4*>(p.wgt + ((long long)k * TAPS + t) * p.wC + n_off + g * 8));
-            const uint32_t w4[4] = {v.x, v.y, v.z, v.w};
-            uint8_t* row = s_w + (t * wrows + k) * wpitch;
+        for (int id0 = tid; id0 < n_chunks; id0 += 4 * MMA_THREADS) {       // four loads in flight per thread
+            uint4 v[4];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) *reinterpret_cast<uint32_t*>(row + col_of_chan<NB>(g * 8 + 2 * e) * 2) = w4[e];   // channel pairs stay adjacent
+            for (int u = 0; u < 4; ++u) {
+                const int id = min(id0 + u * MMA_THREADS, n_chunks - 1);
+                const int g = id % groups, k = (id / groups) % ca, t = id / (groups * ca);
+                v[u] = __ldg(reinterpret_cast<const uint4*>(p.wgt + ((long long)k * TAPS + t) * p.wC + n_off + g * 8));
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int id = id0 + u * MMA_THREADS;
+                if (id < n_chunks) {
+                    const int g = id % groups, k = (id / groups) % ca, t = id / (groups * ca);
+                    const uint32_t w4[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+                    uint8_t* row = s_w + (t * wrows + k) * wpitch;
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) *reinterpret_cast<uint32_t*>(row + col_of_chan<NB>(g * 8 + 2 * e) * 2) = w4[e];   // channel pairs stay adjacent
+                }
+            }
         }
     }
     // ---- this thread's part of every copy: one 8-channel piece of every (256 / pieces-per-row)-th window row
@@ -241,6 +264,7 @@ __global__ void __launch_bounds__(MMA_THREADS) conv_mma_kernel(const MmaProb* __
             const int shift = TRANS ? ((K1 - r) * Wp + (K1 - q)) : (r * Wp + q);
             const uint32_t a_tap = a_base + (uint32_t)shift * apitch;
             const uint32_t w_tap = w_base + (uint32_t)(t * wrows) * wpitch + b_lane;
+#pragma unroll
             for (int k0 = 0; k0 < ca; k0 += 16) {
                 uint32_t a[MBW][4];
 #pragma unroll
@@ -258,9 +282,22 @@ __global__ void __launch_bounds__(MMA_THREADS) conv_mma_kernel(const MmaProb* __
                 }
             }
         }
-        // ---- epilogue: thread (g8, t4) holds rows g8 and g8+8 of each 16-row block, channels t4*2*NB ... t4*2*NB + 2*NB - 1
+        // ---- epilogue: thread (g8, t4) holds rows g8 and g8+8 of each 16-row block, channels t4*2*NB ... t4*2*NB + 2*NB - 1.
+        // No branch around the loads: a row at a padding position reads pixel 0 and is neither stored nor counted, so the
+        // loads of all rows can be in flight together.
         const int grp = unit / subs, j0 = (unit - grp * subs) * sub;
         const long long obase = grp * grp_out + n_off + t4 * (2 * NB);
+        const __nv_bfloat16* __restrict__ add_g = addp + obase;
+        const __nv_bfloat16* __restrict__ bnx_g = bnx + obase;
+        __nv_bfloat16* __restrict__ out_g = outp + obase;
+        int opx[MBW][2];
+#pragma unroll
+        for (int mb = 0; mb < MBW; ++mb) {
+            const int blk = min(warp + 8 * mb, nblk - 1);
+            const bool real = warp + 8 * mb < nblk;
+#pragma unroll
+            for (int half = 0; half < 2; ++half) { const int v = otable[j0 + blk * 16 + g8 + half * 8]; opx[mb][half] = real ? v : -1; }
+        }
         float ps[2 * NB], pq[2 * NB];                             // fused BN: this thread's sums over the piece
 #pragma unroll
         for (int i = 0; i < 2 * NB; ++i) { ps[i] = 0.f; pq[i] = 0.f; }
@@ -268,18 +305,26 @@ __global__ void __launch_bounds__(MMA_THREADS) conv_mma_kernel(const MmaProb* __
         for (int mb = 0; mb < MBW; ++mb)
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
-                const int blk = warp + 8 * mb;
-                const int opix = blk < nblk ? otable[j0 + blk * 16 + g8 + half * 8] : -1;
-                if (opix < 0) continue;
-                const long long o = obase + (long long)opix * ncol_all;
-                uint32_t wv[NB];
+                const int opix = opx[mb][half];
+                const bool valid = opix >= 0;
+                const int o = max(opix, 0) * ncol_all;            // a tensor of one problem has fewer than 2^31 elements
+                uint32_t wv[NB], xv[NB];
                 if (addp) {
                     if constexpr (NB % 4 == 0) {
 #pragma unroll
-                        for (int c4 = 0; c4 < NB / 4; ++c4) { const uint4 v = *reinterpret_cast<const uint4*>(addp + o + c4 * 8); wv[c4 * 4] = v.x; wv[c4 * 4 + 1] = v.y; wv[c4 * 4 + 2] = v.z; wv[c4 * 4 + 3] = v.w; }
+                        for (int c4 = 0; c4 < NB / 4; ++c4) { const uint4 v = *reinterpret_cast<const uint4*>(add_g + o + c4 * 8); wv[c4 * 4] = v.x; wv[c4 * 4 + 1] = v.y; wv[c4 * 4 + 2] = v.z; wv[c4 * 4 + 3] = v.w; }
                     } else {
 #pragma unroll
-                        for (int c2 = 0; c2 < NB / 2; ++c2) { const uint2 v = *reinterpret_cast<const uint2*>(addp + o + c2 * 4); wv[c2 * 2] = v.x; wv[c2 * 2 + 1] = v.y; }
+                        for (int c2 = 0; c2 < NB / 2; ++c2) { const uint2 v = *reinterpret_cast<const uint2*>(add_g + o + c2 * 4); wv[c2 * 2] = v.x; wv[c2 * 2 + 1] = v.y; }
+                    }
+                }
+                if (fuse == 2) {
+                    if constexpr (NB % 4 == 0) {
+#pragma unroll
+                        for (int c4 = 0; c4 < NB / 4; ++c4) { const uint4 v = *reinterpret_cast<const uint4*>(bnx_g + o + c4 * 8); xv[c4 * 4] = v.x; xv[c4 * 4 + 1] = v.y; xv[c4 * 4 + 2] = v.z; xv[c4 * 4 + 3] = v.w; }
+                    } else {
+#pragma unroll
+                        for (int c2 = 0; c2 < NB / 2; ++c2) { const uint2 v = *reinterpret_cast<const uint2*>(bnx_g + o + c2 * 4); xv[c2 * 2] = v.x; xv[c2 * 2 + 1] = v.y; }
                     }
                 }
 #pragma unroll
@@ -292,37 +337,29 @@ __global__ void __launch_bounds__(MMA_THREADS) conv_mma_kernel(const MmaProb* __
                 if (fuse == 1) {                                  // sums of the STORED values: x, x^2
 #pragma unroll
                     for (int j = 0; j < NB; ++j) {
-                        const float r0 = __uint_as_float(wv[j] << 16), r1 = __uint_as_float(wv[j] & 0xFFFF0000u);
+                        const float r0 = valid ? __uint_as_float(wv[j] << 16) : 0.f, r1 = valid ? __uint_as_float(wv[j] & 0xFFFF0000u) : 0.f;
                         ps[2 * j] += r0; pq[2 * j] += r0 * r0; ps[2 * j + 1] += r1; pq[2 * j + 1] += r1 * r1;
                     }
                 } else if (fuse == 2) {                           // sums of dz = da * [relu input > 0] and dz * xhat
-                    uint32_t xv[NB];
-                    if constexpr (NB % 4 == 0) {
-#pragma unroll
-                        for (int c4 = 0; c4 < NB / 4; ++c4) { const uint4 v = *reinterpret_cast<const uint4*>(bnx + o + c4 * 8); xv[c4 * 4] = v.x; xv[c4 * 4 + 1] = v.y; xv[c4 * 4 + 2] = v.z; xv[c4 * 4 + 3] = v.w; }
-                    } else {
-#pragma unroll
-                        for (int c2 = 0; c2 < NB / 2; ++c2) { const uint2 v = *reinterpret_cast<const uint2*>(bnx + o + c2 * 4); xv[c2 * 2] = v.x; xv[c2 * 2 + 1] = v.y; }
-                    }
 #pragma unroll
                     for (int j = 0; j < NB; ++j) {
-#pragma unroll
-                        for (int e = 0; e < 2; ++e) {
-                            const int c = t4 * (2 * NB) + 2 * j + e;
-                            const float x = e ? __uint_as_float(xv[j] & 0xFFFF0000u) : __uint_as_float(xv[j] << 16);
-                            const float d = e ? __uint_as_float(wv[j] & 0xFFFF0000u) : __uint_as_float(wv[j] << 16);
-                            const float xh = (x - s_bn[0][c]) * s_bn[1][c];
-                            const float dz = (xh * s_bn[2][c] + s_bn[3][c] > 0.f) ? d : 0.f;
-                            ps[2 * j + e] += dz; pq[2 * j + e] += dz * xh;
-                        }
+                        const int c = t4 * (2 * NB) + 2 * j;
+                        const float2 mean = *reinterpret_cast<const float2*>(&s_bn[0][c]), istd = *reinterpret_cast<const float2*>(&s_bn[1][c]);
+                        const float2 ga = *reinterpret_cast<const float2*>(&s_bn[2][c]), be = *reinterpret_cast<const float2*>(&s_bn[3][c]);
+                        const float xh0 = (__uint_as_float(xv[j] << 16) - mean.x) * istd.x, xh1 = (__uint_as_float(xv[j] & 0xFFFF0000u) - mean.y) * istd.y;
+                        const float dz0 = (valid && xh0 * ga.x + be.x > 0.f) ? __uint_as_float(wv[j] << 16) : 0.f;
+                        const float dz1 = (valid && xh1 * ga.y + be.y > 0.f) ? __uint_as_float(wv[j] & 0xFFFF0000u) : 0.f;
+                        ps[2 * j] += dz0; pq[2 * j] += dz0 * xh0; ps[2 * j + 1] += dz1; pq[2 * j + 1] += dz1 * xh1;
                     }
                 }
-                if constexpr (NB % 4 == 0) {
+                if (valid) {
+                    if constexpr (NB % 4 == 0) {
 #pragma unroll
-                    for (int c4 = 0; c4 < NB / 4; ++c4) *reinterpret_cast<uint4*>(outp + o + c4 * 8) = make_uint4(wv[c4 * 4], wv[c4 * 4 + 1], wv[c4 * 4 + 2], wv[c4 * 4 + 3]);
-                } else {
+                        for (int c4 = 0; c4 < NB / 4; ++c4) *reinterpret_cast<uint4*>(out_g + o + c4 * 8) = make_uint4(wv[c4 * 4], wv[c4 * 4 + 1], wv[c4 * 4 + 2], wv[c4 * 4 + 3]);
+                    } else {
 #pragma unroll
-                    for (int c2 = 0; c2 < NB / 2; ++c2) *reinterpret_cast<uint2*>(outp + o + c2 * 4) = make_uint2(wv[c2 * 2], wv[c2 * 2 + 1]);
+                        for (int c2 = 0; c2 < NB / 2; ++c2) *reinterpret_cast<uint2*>(out_g + o + c2 * 4) = make_uint2(wv[c2 * 2], wv[c2 * 2 + 1]);
+                    }
                 }
             }
         if (fuse) {                                               // the 8 lanes that own the same channels, fixed butterfly; lane g8 = 0 keeps the warp's running sum
@@ -360,8 +397,19 @@ __global__ void __launch_bounds__(MMA_THREADS) conv_mma_kernel(const MmaProb* __
     {
         const int rows = min(ncta, units), Q = MMA_THREADS / C, c = tid % C, q = tid / C;   // C is 16, 32 or 64
         double a0 = 0.0, a1 = 0.0;
-#pragma unroll 4
-        for (int k = q; k < rows; k += Q) { a0 += __ldcg(bn.partial + ((long long)k * 2 + 0) * C + c); a1 += __ldcg(bn.partial + ((long long)k * 2 + 1) * C + c); }
+        {   // 8 rows (16 loads) in flight per thread: the loop is bound by L2 latency, not by its few kilobytes
+            const double* pp = bn.partial + (long long)q * 2 * C + c;
+            const long long step = (long long)Q * 2 * C;
+            int k = q;
+            for (; k + 7 * Q < rows; k += 8 * Q, pp += 8 * step) {
+                double v0[8], v1[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) { v0[u] = __ldcg(pp + u * step); v1[u] = __ldcg(pp + u * step + C); }
+#pragma unroll
+                for (int u = 0; u < 8; ++u) { a0 += v0[u]; a1 += v1[u]; }
+            }
+            for (; k < rows; k += Q, pp += step) { a0 += __ldcg(pp); a1 += __ldcg(pp + C); }
+        }
         s_dred[tid] = a0; s_dred[256 + tid] = a1;
         __syncthreads();
         if (q == 0) {
@@ -429,6 +477,8 @@ struct MmaGeom { int ca, ncol, Hp, Wp, G, gpos, sub, subs, units, mbw, stages, n
 
 // variant = ((MBW * 4 + ksz) * 2 + trans) * 16 + NB: everything a launch is specialised on; + MMA_VARIANT_FUSED: with BN
 constexpr int MMA_VARIANT_FUSED = 512;
+// + (1, 2, 3) << 10: a 3x3 instance specialised on 16, 32 or 64 staged channels (CTAs of 16 or 32 output channels)
+static int mma_ca_code(int ksz, int nb, int ca) { return ksz == 3 && (nb == 2 || nb == 4) ? (ca == 16 ? 1 : ca == 32 ? 2 : ca == 64 ? 3 : 0) : 0; }
 static int mma_variant(int mbw, int ksz, int trans, int nb) { return ((mbw * 4 + ksz) * 2 + trans) * 16 + nb; }
 
 static bool mma_geometry(const ConvProb& p, int mode, MmaGeom& g) {
@@ -463,7 +513,9 @@ static bool mma_geometry(const ConvProb& p, int mode, MmaGeom& g) {
             if (gpos >= 32768 || (long long)G * p.H * p.W >= 32768) continue;
             const size_t table = (size_t)(((2 * subs * sub + 2 * halo) * 2 + 127) & ~127);
             const size_t stage = (size_t)(((sub + 2 * halo) * apitch + 127) & ~127);
-            int stages = 4; while (stages > 2 && table + stages * stage + wbytes + 64 > 100 * 1024) --stages;
+            // 16-channel CTAs need few registers: three of them share an SM when each stays below 72 KB
+            const size_t budget = (ncta_col <= 16 && table + 2 * stage + wbytes + 64 <= 72 * 1024) ? 72 * 1024 : 100 * 1024;
+            int stages = 4; while (stages > 2 && table + stages * stage + wbytes + 64 > budget) --stages;
             if (table + stages * stage + wbytes + 64 > 200 * 1024) continue;
             const long long units = (long long)(p.N / G) * subs;
             double cost = (double)subs * sub / gpos * (1.0 + 48.0 / sub) * (8.0 * mbw / nblk);
@@ -473,7 +525,7 @@ static bool mma_geometry(const ConvProb& p, int mode, MmaGeom& g) {
         }
     }
     if (!g.sub) return false;
-    g.variant = mma_variant(g.mbw, p.ksz, mode == CONV_DGRAD ? 1 : 0, ncta_col / 8);
+    g.variant = mma_variant(g.mbw, p.ksz, mode == CONV_DGRAD ? 1 : 0, ncta_col / 8) | (mma_ca_code(p.ksz, ncta_col / 8, g.ca) << 10);
     return true;
 }
 
@@ -513,11 +565,11 @@ struct MmaLaunch { const void* d; int nprob, max_tiles; size_t smem; bool pdl, c
 
 // Persistent CTAs: as many as are co-resident at this shared-memory footprint (at most 3 per SM), over all problems.
 // A fused launch is cooperative (grid barrier): its grid never exceeds what is co-resident.
-template <int NB, int MBW, int KSZ, bool TRANS>
+template <int NB, int MBW, int KSZ, bool TRANS, int CA = 0>
 static void launch_mma_inst(MmaLaunch& a) {
     static bool configured = false; static int sms = 0; static signed char occ[256] = {};
     static int coop_pdl = 1;                                      // 1: cooperative + programmatic launch together until the driver refuses it
-    auto kernel = conv_mma_kernel<NB, MBW, KSZ, TRANS>;
+    auto kernel = conv_mma_kernel<NB, MBW, KSZ, TRANS, CA>;
     if (!configured) {
         cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 202 * 1024);
         int dev = 0; cudaGetDevice(&dev); cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev); if (sms < 1) sms = 148;
@@ -545,6 +597,11 @@ static void launch_mma_inst(MmaLaunch& a) {
     a.ok = e == cudaSuccess;
 }
 template <int NB, int MBW>
+static void launch_mma_ca(MmaLaunch& a, int trans, int cac) {      // 3x3 instances specialised on the staged channels
+    if (trans) { if (cac == 1) launch_mma_inst<NB, MBW, 3, true, 16>(a); else if (cac == 2) launch_mma_inst<NB, MBW, 3, true, 32>(a); else launch_mma_inst<NB, MBW, 3, true, 64>(a); }
+    else { if (cac == 1) launch_mma_inst<NB, MBW, 3, false, 16>(a); else if (cac == 2) launch_mma_inst<NB, MBW, 3, false, 32>(a); else launch_mma_inst<NB, MBW, 3, false, 64>(a); }
+}
+template <int NB, int MBW>
 static void launch_mma_nb(MmaLaunch& a, int ksz, int trans) {
     if (ksz == 3) { if (trans) launch_mma_inst<NB, MBW, 3, true>(a); else launch_mma_inst<NB, MBW, 3, false>(a); }
     else { if (trans) launch_mma_inst<NB, MBW, 1, true>(a); else launch_mma_inst<NB, MBW, 1, false>(a); }
@@ -554,6 +611,12 @@ static void launch_mma_nb(MmaLaunch& a, int ksz, int trans) {
 bool launch_conv_mma_probs(const void* d, int nprob, int max_tiles, size_t max_smem, int variant, cudaStream_t s, bool pdl) {
     const int nb = variant & 15, trans = (variant >> 4) & 1, ksz = (variant >> 5) & 3, mbw = (variant >> 7) & 3;
     MmaLaunch a{d, nprob, max_tiles, max_smem, pdl, (variant & MMA_VARIANT_FUSED) != 0, s, false};
+    const int cac = (variant >> 10) & 3;
+    if (cac && ksz == 3 && (nb == 2 || nb == 4) && mbw >= 1 && mbw <= 3) {
+        if (nb == 2) { if (mbw == 1) launch_mma_ca<2, 1>(a, trans, cac); else if (mbw == 2) launch_mma_ca<2, 2>(a, trans, cac); else launch_mma_ca<2, 3>(a, trans, cac); }
+        else { if (mbw == 1) launch_mma_ca<4, 1>(a, trans, cac); else if (mbw == 2) launch_mma_ca<4, 2>(a, trans, cac); else launch_mma_ca<4, 3>(a, trans, cac); }
+        return a.ok;
+    }
 #define MMA_CASE(N_, M_) if (nb == N_ && mbw == M_) launch_mma_nb<N_, M_>(a, ksz, trans); else
     MMA_CASE(2, 1) MMA_CASE(2, 2) MMA_CASE(2, 3) MMA_CASE(4, 1) MMA_CASE(4, 2) MMA_CASE(4, 3)
     MMA_CASE(6, 1) MMA_CASE(6, 2) MMA_CASE(8, 1) MMA_CASE(8, 2)

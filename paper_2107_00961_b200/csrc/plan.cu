@@ -27,7 +27,9 @@ int conv_wgrad_tc_ctas(const void* h);
 size_t conv_wgrad_tc_smem(const void* h);
 long long conv_wgrad_tc_out_elems(const void* h);
 void launch_conv_wgrad_tc_probs(const void* d_tc, int nprob, int max_ctas, size_t max_smem, long long max_out, cudaStream_t s);
-static int wgrad_target_ctas(const resist_ctx* ctx) { return std::max(8, 2 * ctx->sm_count / std::max(1, ctx->S)); }
+// CTAs per weight-gradient problem so that a launch of nprob problems fills the GPU; the partial-sum workspace is sized for
+// a problem launched alone (nprob = 1, the default)
+static int wgrad_target_ctas(const resist_ctx* ctx, int nprob = 1) { return std::max(8, 2 * ctx->sm_count / std::max(1, nprob)); }
 bool conv_mma_supported(const ConvProb& p, int mode);                                   // conv_mma.cu
 bool conv_mma_fill(const ConvProb& p, int mode, void* host, const BnProb* bn = nullptr);
 bool conv_mma_can_fuse_bn(const ConvProb& p, int mode, int C);
@@ -459,7 +461,7 @@ static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool s
                         if (o.kind == OP_CONV_WGRAD) {
                             if (k == i) L.first = n_wmm;
                             wmm.resize((size_t)(n_wmm + 1) * wmmb); char* h = wmm.data() + (size_t)n_wmm * wmmb;
-                            if (!conv_wgrad_mma_fill(o.conv, wgrad_target_ctas(ctx), h)) { ctx->err = "wgrad descriptor failed"; return RESIST_EINVAL; }
+                            if (!conv_wgrad_mma_fill(o.conv, wgrad_target_ctas(ctx, (int)(j - i)), h)) { ctx->err = "wgrad descriptor failed"; return RESIST_EINVAL; }
                             L.gx = std::max(L.gx, conv_wgrad_mma_ctas(h));
                             L.max_elems = std::max<long long>(L.max_elems, (long long)conv_wgrad_mma_smem(h));
                             L.max_b = (int)std::max<long long>(L.max_b, conv_wgrad_mma_out_elems(h));
@@ -482,7 +484,7 @@ static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool s
                         if (k == i) L.first = n_wtc;
                         wtc.resize((size_t)(n_wtc + 1) * wtcb);
                         char* h = wtc.data() + (size_t)n_wtc * wtcb;
-                        if (!conv_wgrad_tc_fill(o.conv, wgrad_target_ctas(ctx), h)) { ctx->err = "tensor map encoding failed"; return RESIST_ECUDA; }
+                        if (!conv_wgrad_tc_fill(o.conv, wgrad_target_ctas(ctx, (int)(j - i)), h)) { ctx->err = "tensor map encoding failed"; return RESIST_ECUDA; }
                         L.gx = std::max(L.gx, conv_wgrad_tc_ctas(h));
                         L.max_elems = std::max<long long>(L.max_elems, (long long)conv_wgrad_tc_smem(h));
                         L.max_b = (int)std::max<long long>(L.max_b, conv_wgrad_tc_out_elems(h));
@@ -726,8 +728,8 @@ static int run_plan(resist_ctx* ctx, Plan& plan, const PatchArgs& pa, bool updat
         }
         int pk = 0, nk = 1;
         switch (L.kind) {
-            case OP_CONV_FWD: pk = L.backend >= 1000 + MMA_BACKEND_FUSED ? PK_CONV_FWD_MMA_BN : L.backend >= 200 ? PK_CONV_FWD_MMA : L.backend ? PK_CONV_FWD_TC : PK_CONV_FWD_CC; break;
-            case OP_CONV_DGRAD: pk = L.backend >= 1000 + MMA_BACKEND_FUSED ? PK_CONV_DGRAD_MMA_BN : L.backend >= 200 ? PK_CONV_DGRAD_MMA : L.backend ? PK_CONV_DGRAD_TC : PK_CONV_DGRAD_CC; break;
+            case OP_CONV_FWD: pk = (L.backend >= 1000 && ((L.backend - 1000) & MMA_BACKEND_FUSED)) ? PK_CONV_FWD_MMA_BN : L.backend >= 200 ? PK_CONV_FWD_MMA : L.backend ? PK_CONV_FWD_TC : PK_CONV_FWD_CC; break;
+            case OP_CONV_DGRAD: pk = (L.backend >= 1000 && ((L.backend - 1000) & MMA_BACKEND_FUSED)) ? PK_CONV_DGRAD_MMA_BN : L.backend >= 200 ? PK_CONV_DGRAD_MMA : L.backend ? PK_CONV_DGRAD_TC : PK_CONV_DGRAD_CC; break;
             case OP_CONV_WGRAD: pk = L.backend >= 200 ? PK_CONV_WGRAD_MMA : L.backend ? PK_CONV_WGRAD_TC : PK_CONV_WGRAD_CC; break;
             case OP_SPLITK: pk = PK_SPLITK; break;
             case OP_BN_STATS: pk = PK_BN_STATS; nk = 2; break;
