@@ -43,6 +43,7 @@ struct alignas(16) MmaProb {
     int G, gpos;                // images per group, positions per group (G * Hp * Wp)
     int sub, subs, units;       // positions per piece (multiple of 16), pieces per group, pieces in total
     int os, P, Q;               // output stride (forward of a stride-2 layer stores even positions only, as a P x Q image)
+    int is, iP, iQ;             // input stride: 2 = act is stored compact [n_img,iP,iQ,ca] and read as if zero-stuffed to H x W
     int stages;                 // depth of the activation ring (2, 3 or 4)
     int nsplit;                 // 1, or 2: a CTA computes one half of the output channels (its half of the filter resident)
     int variant, smem_bytes;    // which instantiation runs this problem (see mma_variant); dynamic shared memory
@@ -157,8 +158,9 @@ __global__ void __launch_bounds__(MMA_THREADS) conv_mma_kernel(const MmaProb* __
             const unsigned Y = __umulhi((unsigned)f, p.inv_wp), X = (unsigned)f - Y * Wp;
             const unsigned n = __umulhi(Y, p.inv_hp), i = Y - n * p.Hp;
             if (X < (unsigned)p.W && i < (unsigned)p.H) {
-                pix = (int)((n * p.H + i) * p.W + X);
-                if (p.os == 1) opix = pix;
+                if (p.is == 2) pix = ((i | X) & 1u) ? -1 : (int)((n * p.iP + (i >> 1)) * p.iQ + (X >> 1));   // zero-stuffed: only even positions exist
+                else pix = (int)((n * p.H + i) * p.W + X);
+                if (p.os == 1) opix = (int)((n * p.H + i) * p.W + X);
                 else if (!((i % p.os) | (X % p.os))) opix = (int)((n * p.P + i / p.os) * p.Q + X / p.os);
             }
         }
@@ -209,7 +211,7 @@ __global__ void __launch_bounds__(MMA_THREADS) conv_mma_kernel(const MmaProb* __
     // ---- this thread's part of every copy: one 8-channel piece of every (256 / pieces-per-row)-th window row
     const int ga = ca / 8, a_step = MMA_THREADS / ga, a_row0 = tid / ga, a_g = tid % ga;
     const bool a_on = tid < a_step * ga;
-    const long long grp_in = (long long)p.G * p.H * p.W * ca;                    // elements of a group of act
+    const long long grp_in = (long long)p.G * (p.is == 2 ? p.iP * p.iQ : p.H * p.W) * ca;   // elements of a group of act
     const long long grp_out = (long long)p.G * (p.os == 1 ? p.H * p.W : p.P * p.Q) * ncol_all;
     auto issue = [&](int unit, int stage) {
         const int grp = unit / subs, j = unit - grp * subs;
@@ -548,6 +550,7 @@ bool conv_mma_fill(const ConvProb& p, int mode, void* host, const BnProb* bn) {
     t.inv_wp = (unsigned)((1ull << 32) / (unsigned)g.Wp + 1); t.inv_hp = (unsigned)((1ull << 32) / (unsigned)g.Hp + 1);
     t.G = g.G; t.gpos = g.gpos; t.sub = g.sub; t.subs = g.subs; t.units = g.units;
     t.os = mode == CONV_FWD ? p.stride : 1; t.P = p.P; t.Q = p.Q;
+    t.is = (mode == CONV_DGRAD && p.dy_sub == 2) ? 2 : 1; t.iP = p.dy_P; t.iQ = p.dy_Q;
     t.stages = g.stages; t.nsplit = g.nsplit; t.variant = g.variant; t.smem_bytes = (int)g.smem; t.scale = p.scale;
     if (bn) {
         if (!conv_mma_can_fuse_bn(p, mode, bn->C)) return false;
@@ -651,6 +654,7 @@ struct alignas(16) MmaWgradProb {
     int wn, stages, variant, smem_bytes;
     unsigned inv_wp, inv_hp;
     int out_ld, out_cols;       // 1x1 problems only: row stride and valid columns of out (an im2col'ed stem); else C, C
+    int ds, dP, dQ;             // 2 = dy is stored compact [n_img,dP,dQ,K] and read as if zero-stuffed to H x W (a second table maps its rows)
 };
 
 template <int MB, int PPW>   // MB = K / 16; PPW = pairs of 8-column blocks a warp owns
@@ -683,12 +687,28 @@ __global__ void __launch_bounds__(MMA_THREADS) conv_wgrad_mma_kernel(const MmaWg
         }
         table[w] = pix;
     }
+    // zero-stuffed dy: position f of a group -> pixel of the compact dy (even positions), -1 elsewhere
+    const bool stuffed = p.ds == 2;
+    int* dtable = reinterpret_cast<int*>(sm + table_bytes);
+    const int dtable_bytes = stuffed ? ((subs * sub * 4 + 127) & ~127) : 0;
+    if (stuffed) {
+        for (int f = tid; f < subs * sub; f += MMA_THREADS) {
+            int pix = -1;
+            if (f < p.gpos) {
+                const unsigned Y = __umulhi((unsigned)f, p.inv_wp), X = (unsigned)f - Y * Wp;
+                const unsigned n = __umulhi(Y, p.inv_hp), i = Y - n * p.Hp;
+                if (X < (unsigned)p.W && i < (unsigned)p.H && !((i | X) & 1u)) pix = (int)((n * p.dP + (i >> 1)) * p.dQ + (X >> 1));
+            }
+            dtable[f] = pix;
+        }
+    }
+    ring += dtable_bytes;
     // ---- this thread's part of every copy: one 8-channel piece of every (256 / pieces-per-row)-th row
     const int ga = C / 8, gd = K / 8;
     const int a_step = MMA_THREADS / ga, d_step = MMA_THREADS / gd;           // rows per sweep (threads past step * g idle)
     const int a_row0 = tid / ga, a_g = tid % ga, d_row0 = tid / gd, d_g = tid % gd;
     const bool a_on = tid < a_step * ga, d_on = tid < d_step * gd;
-    const long long img_a = (long long)p.H * p.W * C, img_d = (long long)p.H * p.W * K;
+    const long long img_a = (long long)p.H * p.W * C, img_d = (stuffed ? (long long)p.dP * p.dQ : (long long)p.H * p.W) * K;
     const __nv_bfloat16* __restrict__ a_ptr = p.a; const __nv_bfloat16* __restrict__ dy_ptr = p.dy;
     auto issue = [&](int unit, int stage) {
         const int grp = unit / subs, j = unit - grp * subs;
@@ -704,7 +724,7 @@ __global__ void __launch_bounds__(MMA_THREADS) conv_wgrad_mma_kernel(const MmaWg
             }
         }
         if (d_on) {
-            const int* t = table + j * sub + halo + d_row0;
+            const int* t = stuffed ? dtable + j * sub + d_row0 : table + j * sub + halo + d_row0;
             uint32_t dst = st0 + d_g * 16 + d_row0 * dpitch;
             for (int row = d_row0; row < sub; row += d_step, t += d_step, dst += d_step * dpitch) {
                 const int pix = *t;
@@ -856,7 +876,7 @@ static bool mma_wg_geometry(const ConvProb& p, int target_ctas, MmaWgGeom& g) {
         if (gpos + 2 * halo + 512 > 8192) break;
         for (int sub = quantum; sub <= 512; sub += quantum) {
             const int subs = (gpos + sub - 1) / sub;
-            const size_t table = (size_t)(((subs * sub + 2 * halo) * 4 + 127) & ~127);
+            const size_t table = (size_t)(((subs * sub + 2 * halo) * 4 + 127) & ~127) + (p.dy_sub == 2 ? (size_t)((subs * sub * 4 + 127) & ~127) : 0);
             const size_t stage = (size_t)((sub * dpitch + 127) & ~127) + (size_t)(((sub + 2 * halo) * apitch + 127) & ~127);
             int stages = 3; if (table + 3 * stage > 150 * 1024) stages = 2;
             if (table + stages * stage + 64 > 200 * 1024) continue;
@@ -890,6 +910,7 @@ bool conv_wgrad_mma_fill(const ConvProb& p, int target_ctas, void* host) {
     t.inv_wp = (unsigned)((1ull << 32) / (unsigned)g.Wp + 1); t.inv_hp = (unsigned)((1ull << 32) / (unsigned)g.Hp + 1);
     t.smem_bytes = (int)g.smem;
     t.out_ld = p.C; t.out_cols = p.C;
+    t.ds = p.dy_sub == 2 ? 2 : 1; t.dP = p.dy_P; t.dQ = p.dy_Q;
     if (p.wg_ld > 0 && p.ksz == 1) { t.out_ld = p.wg_ld; t.out_cols = p.wg_cols; }
     memcpy(host, &t, sizeof(t));
     return true;

@@ -24,6 +24,8 @@ struct ConvProb {
     int tiles_m, tiles_n, splits, ktiles_per_split;
     float scale;          // result = scale*acc + add
     int wg_ld, wg_cols;   // wgrad of a 1x1 problem on an im2col'ed input: row stride and valid columns of dw (0: K x C dense)
+    int dy_sub;           // backward of a stride-2 layer as a stride-1 problem: 2 = dy is stored compact [N,dy_P,dy_Q,K] and read as if
+    int dy_P, dy_Q;       //   zero-stuffed to H x W (only even positions exist); 0 or 1 = dy is stored at the problem's resolution
     int pad_;
 };
 

@@ -516,7 +516,15 @@ __global__ void avgpool_kernel(const HeadProb* __restrict__ probs) {
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
         const int c = i % p.C, b = i / p.C;
         float s = 0.f;
-        for (int k = 0; k < p.HW; ++k) s += ldf<T>(p.a, ((long long)b * p.HW + k) * p.C + c);
+        int k = 0;
+        for (; k + 8 <= p.HW; k += 8) {                          // eight loads in flight, added in order
+            float v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) v[u] = ldf<T>(p.a, ((long long)b * p.HW + k + u) * p.C + c);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) s += v[u];
+        }
+        for (; k < p.HW; ++k) s += ldf<T>(p.a, ((long long)b * p.HW + k) * p.C + c);
         p.pooled[i] = s / (float)p.HW;
     }
 }
@@ -534,11 +542,11 @@ __global__ void head_logits_kernel(const HeadProb* __restrict__ probs) {
     }
 }
 // one CTA per problem; one warp per sample, samples strided over the warps; fixed-order loss sum
-__global__ void __launch_bounds__(256) loss_kernel(const HeadProb* __restrict__ probs) {
+__global__ void __launch_bounds__(1024) loss_kernel(const HeadProb* __restrict__ probs) {
     const HeadProb& p = probs[blockIdx.x];
     __shared__ float sl[1024]; __shared__ int sc[1024];
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-    for (int b = warp; b < p.B; b += 8) {
+    for (int b = warp; b < p.B; b += (int)(blockDim.x >> 5)) {
         const float* lg = p.logits + (long long)b * p.classes;
         float mx = -INFINITY; int arg = 0x7fffffff;
         for (int k = lane; k < p.classes; k += 32) { float v = lg[k]; if (v > mx) { mx = v; arg = k; } }
@@ -566,17 +574,19 @@ __global__ void __launch_bounds__(256) loss_kernel(const HeadProb* __restrict__ 
         if (p.correct) *p.correct = c;
     }
 }
+// one warp per output element: lane l adds samples l, l+32, ... in order, then a fixed butterfly over the lanes
 __global__ void head_bwd_w_kernel(const HeadProb* __restrict__ probs) {
     const HeadProb& p = probs[blockIdx.y];
-    const int n = p.classes * p.C;
-    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n + p.classes; i += gridDim.x * blockDim.x) {
+    const int n = p.classes * p.C, lane = threadIdx.x & 31;
+    const int nw = gridDim.x * (blockDim.x >> 5);
+    for (int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); i < n + p.classes; i += nw) {
         float s = 0.f;
         if (i < n) { const int c = i % p.C, k = i / p.C;
-            for (int b = 0; b < p.B; ++b) s = fmaf(p.dlogits[(long long)b * p.classes + k], p.pooled[(long long)b * p.C + c], s);
-            p.dw[i] = s;
+            for (int b = lane; b < p.B; b += 32) s = fmaf(p.dlogits[(long long)b * p.classes + k], p.pooled[(long long)b * p.C + c], s);
         } else { const int k = i - n;
-            for (int b = 0; b < p.B; ++b) s += p.dlogits[(long long)b * p.classes + k];
-            p.db[k] = s; }
+            for (int b = lane; b < p.B; b += 32) s += p.dlogits[(long long)b * p.classes + k]; }
+        for (int d = 16; d; d >>= 1) s += __shfl_xor_sync(0xffffffffu, s, d);
+        if (lane == 0) { if (i < n) p.dw[i] = s; else p.db[i - n] = s; }
     }
 }
 __global__ void head_bwd_x_kernel(const HeadProb* __restrict__ probs) {
@@ -593,6 +603,16 @@ template <class T>
 __global__ void avgpool_bwd_kernel(const HeadProb* __restrict__ probs) {
     const HeadProb& p = probs[blockIdx.y];
     const long long n = (long long)p.B * p.HW * p.C;
+    if (sizeof(T) == 2 && p.C % 8 == 0 && (((uintptr_t)p.da | (uintptr_t)p.dpooled) & 15) == 0) {   // 8 channels per thread
+        const int G = p.C / 8; const long long nv = n / 8;
+        for (long long v = blockIdx.x * (long long)blockDim.x + threadIdx.x; v < nv; v += (long long)gridDim.x * blockDim.x) {
+            const int g = (int)(v % G); const long long b = v / ((long long)p.HW * G);
+            const float4 f0 = *reinterpret_cast<const float4*>(p.dpooled + b * p.C + g * 8), f1 = *reinterpret_cast<const float4*>(p.dpooled + b * p.C + g * 8 + 4);
+            const float f[8] = {f0.x, f0.y, f0.z, f0.w, f1.x, f1.y, f1.z, f1.w};
+            reinterpret_cast<uint4*>(p.da)[v] = pack8(f);
+        }
+        return;
+    }
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
         const int c = (int)(i % p.C); const long long b = i / ((long long)p.HW * p.C);
         stf<T>(p.da, i, p.dpooled[b * p.C + c]);
@@ -603,11 +623,11 @@ void launch_head_fwd(const HeadProb* d, int nprob, int maxB, int maxC, int max_c
     if (bf16) avgpool_kernel<__nv_bfloat16><<<dim3(ew_grid((long long)maxB * maxC), nprob), 256, 0, s>>>(d);
     else avgpool_kernel<float><<<dim3(ew_grid((long long)maxB * maxC), nprob), 256, 0, s>>>(d);
     head_logits_kernel<<<dim3(ew_grid((long long)maxB * max_classes * 32), nprob), 256, 0, s>>>(d);
-    loss_kernel<<<nprob, 256, 0, s>>>(d);
+    loss_kernel<<<nprob, 1024, 0, s>>>(d);
 }
 void launch_head_bwd(const HeadProb* d, int nprob, int maxB, int maxC, int max_classes, long long max_elems,
                      bool bf16, cudaStream_t s) {
-    head_bwd_w_kernel<<<dim3(ew_grid((long long)max_classes * (maxC + 1)), nprob), 256, 0, s>>>(d);
+    head_bwd_w_kernel<<<dim3(ew_grid((long long)max_classes * (maxC + 1) * 32), nprob), 256, 0, s>>>(d);
     head_bwd_x_kernel<<<dim3(ew_grid((long long)maxB * maxC), nprob), 256, 0, s>>>(d);
     if (bf16) avgpool_bwd_kernel<__nv_bfloat16><<<dim3(ew_grid(max_elems), nprob), 256, 0, s>>>(d);
     else avgpool_bwd_kernel<float><<<dim3(ew_grid(max_elems), nprob), 256, 0, s>>>(d);
@@ -620,22 +640,30 @@ __global__ void __launch_bounds__(256) im2col_kernel(const ColProb* __restrict__
     const ColProb& p = probs[blockIdx.y];
     const __nv_bfloat16* __restrict__ src = (const __nv_bfloat16*)p.src;
     const long long rows = (long long)p.N * p.P * p.Q, total = rows * 4;
+    // column j of a row = tap (r, s), channel c: the three are looked up, not divided out, for every element
+    __shared__ int s_r[32], s_s[32], s_off[32];
+    if (threadIdx.x < 32) {
+        const int j = threadIdx.x;
+        if (j < p.kk) { const int c = j % p.C, rs = j / p.C, ss = rs % p.ksz, r = rs / p.ksz; s_r[j] = r - p.pad; s_s[j] = ss - p.pad; s_off[j] = ((r - p.pad) * p.W + (ss - p.pad)) * p.C + c; }
+        else { s_r[j] = -(1 << 20); s_s[j] = 0; s_off[j] = 0; }   // beyond the taps: never inside the image
+    }
+    __syncthreads();
+    const unsigned short* __restrict__ src16 = reinterpret_cast<const unsigned short*>(src);
     for (long long id = blockIdx.x * (long long)blockDim.x + threadIdx.x; id < total; id += (long long)gridDim.x * blockDim.x) {
         const int g = (int)(id & 3); const long long row = id >> 2;
         const int q = (int)(row % p.Q); const long long t = row / p.Q; const int pr = (int)(t % p.P); const int n = (int)(t / p.P);
-        __align__(16) __nv_bfloat16 v[8];
+        const int y0 = pr * p.stride, x0 = q * p.stride;
+        const long long base = (((long long)n * p.H + y0) * p.W + x0) * p.C;
+        unsigned short h[8];
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
             const int j = g * 8 + e;
-            float x = 0.f;
-            if (j < p.kk) {
-                const int c = j % p.C, rs = j / p.C, s = rs % p.ksz, r = rs / p.ksz;
-                const int y = pr * p.stride - p.pad + r, xx = q * p.stride - p.pad + s;
-                if (y >= 0 && y < p.H && xx >= 0 && xx < p.W) x = __bfloat162float(src[(((long long)n * p.H + y) * p.W + xx) * p.C + c]);
-            }
-            v[e] = __float2bfloat16(x);
+            const int y = y0 + s_r[j], xx = x0 + s_s[j];
+            const bool in = y >= 0 && y < p.H && xx >= 0 && xx < p.W;
+            h[e] = in ? src16[base + s_off[j]] : (unsigned short)0;
         }
-        *reinterpret_cast<uint4*>((__nv_bfloat16*)p.dst + row * 32 + g * 8) = *reinterpret_cast<const uint4*>(v);
+        *reinterpret_cast<uint4*>((__nv_bfloat16*)p.dst + row * 32 + g * 8) =
+            make_uint4(h[0] | ((unsigned)h[1] << 16), h[2] | ((unsigned)h[3] << 16), h[4] | ((unsigned)h[5] << 16), h[6] | ((unsigned)h[7] << 16));
         if (id < (long long)p.K * 4) {                             // weights: w[k][kk] -> w32[k][32]
             const int kx = (int)(id >> 2);
             __align__(16) __nv_bfloat16 wv[8];

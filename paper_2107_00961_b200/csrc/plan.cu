@@ -154,6 +154,13 @@ struct Builder {
             if (mode == CONV_DGRAD) { q.act = up_buf; q.M = (int)rows_in; }
             else { q.wgt = up_buf; q.Kred = (int)rows_in; }
             size_t pb = 0;
+            // warp-MMA kernels read the compact dy through their pixel tables (odd positions are zero): nothing is materialised
+            ConvProb q2 = q; q2.dy_sub = 2; q2.dy_P = p.P; q2.dy_Q = p.Q;
+            if (mode == CONV_DGRAD) q2.act = dy_or_null; else q2.wgt = dy_or_null;
+            if (pick_backend(q2, mode, wgrad_target_ctas(ctx), &pb, pref) >= 200) {
+                p = q2;
+                if (mode == CONV_WGRAD) wgrad_partial_need = std::max(wgrad_partial_need, pb);
+            } else {
             const bool ok = pick_backend(q, mode, wgrad_target_ctas(ctx), &pb, pref) != 0;
             if (ok) {
                 up_need = std::max(up_need, up_bytes);
@@ -164,6 +171,7 @@ struct Builder {
                 }
                 p = q;
                 if (mode == CONV_WGRAD) { wgrad_partial_need = std::max(wgrad_partial_need, pb); }
+            }
             }
         }
         if (mode == CONV_WGRAD) {
@@ -456,7 +464,8 @@ static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool s
                 case OP_CONV_FWD: case OP_CONV_DGRAD: case OP_CONV_WGRAD: case OP_SPLITK: {
                     if (o.backend >= 200 && o.kind != OP_SPLITK) {   // warp-level MMA kernels: their own descriptor arrays
                         const ConvProb& p = o.conv;
-                        const double in_e = (double)p.N * p.H * p.W * p.C, out_e = (double)p.N * p.P * p.Q * p.K, w_e = (double)p.K * p.ksz * p.ksz * p.C;
+                        // algorithmic work of the layer itself: a stride-2 layer's dy has dy_P x dy_Q positions, whatever resolution the kernel walks
+                        const double in_e = (double)p.N * p.H * p.W * p.C, out_e = (double)p.N * (p.dy_sub == 2 ? (double)p.dy_P * p.dy_Q : (double)p.P * p.Q) * p.K, w_e = (double)p.K * p.ksz * p.ksz * p.C;
                         L.flops += 2.0 * out_e * p.ksz * p.ksz * p.C;
                         if (o.kind == OP_CONV_WGRAD) {
                             if (k == i) L.first = n_wmm;
