@@ -117,7 +117,8 @@ template <int NB> __host__ __device__ __forceinline__ int col_of_chan(int c) { r
 // on load, taps flipped).  CA = channels of the staged activations when the instance is specialised on them (all pitches
 // and the reduction loop are then compile-time), 0 = read from the problem.
 template <int NB, int MBW, int KSZ, bool TRANS, int CA>
-__global__ void __launch_bounds__(MMA_THREADS) conv_mma_kernel(const MmaProb* __restrict__ probs) {
+__global__ void __launch_bounds__(MMA_THREADS, (NB == 2 && CA != 0) ? 3 : 2) conv_mma_kernel(   // registers for three (16-channel CTAs) or two CTAs per SM
+const MmaProb* __restrict__ probs) {
     __shared__ MmaProb p;
     if (threadIdx.x < sizeof(MmaProb) / 4) reinterpret_cast<uint32_t*>(&p)[threadIdx.x] = reinterpret_cast<const uint32_t*>(probs + blockIdx.y)[threadIdx.x];
     __syncthreads();

@@ -101,7 +101,8 @@ struct Builder {
     double* bn_partial = nullptr; float* wgrad_partial = nullptr; size_t bn_partial_need = 0, wgrad_partial_need = 0;
     char* up_buf = nullptr; size_t up_need = 0; const void* up_src = nullptr;      // zero-stuffed dy of the current stride-2 layer
     char* col_buf = nullptr; char* col_w = nullptr;                                 // im2col of the input images and the stem's weights packed alike
-    char* gbuf[6] = {}; bool gused[6] = {}; size_t gbig = 0;
+    static constexpr int NGBUF = 12;           // rotating gradient buffers: the more, the further the main stream runs ahead of the weight gradients
+    char* gbuf[NGBUF] = {}; bool gused[NGBUF] = {}; size_t gbig = 0;
     float* logits = nullptr;
     long long flops = 0; int n_tc = 0, n_cc = 0;
     // The BN+ReLU that consumes a warp-MMA convolution's output joins that convolution's launch (forward: the BN of the
@@ -118,8 +119,8 @@ struct Builder {
     void* act(long long elems) { size_t b = (size_t)elems * es; if (b > gbig) gbig = b; return take(b); }
     // gradient buffers are handed out oldest-released first: a weight gradient that still reads a released buffer on
     // the second stream then has several layers' time before the buffer is written again
-    int gstamp[6] = {}; int gclock = 0;
-    int gtake() { int best = -1; for (int i = 0; i < 6; ++i) if (!gused[i] && (best < 0 || gstamp[i] < gstamp[best])) best = i; if (best >= 0) gused[best] = true; return best; }
+    int gstamp[NGBUF] = {}; int gclock = 0;
+    int gtake() { int best = -1; for (int i = 0; i < NGBUF; ++i) if (!gused[i] && (best < 0 || gstamp[i] < gstamp[best])) best = i; if (best >= 0) gused[best] = true; return best; }
     void grel(int i) { if (i >= 0) { gused[i] = false; gstamp[i] = ++gclock; } }
 
     float* W() const { return ctx->pa.w + (long long)copy * ctx->pa.n; }
@@ -282,7 +283,7 @@ static size_t unroll_subnet(resist_ctx* ctx, Builder& bd, const std::vector<char
     bd.bn_partial = (double*)bd.take(bd.bn_partial_need);
     bd.wgrad_partial = (float*)bd.take(bd.wgrad_partial_need);
     bd.up_buf = (char*)bd.take(bd.up_need);
-    if (!bd.eval) for (int i = 0; i < 6; ++i) bd.gbuf[i] = (char*)bd.take(bd.gbig);
+    if (!bd.eval) for (int i = 0; i < Builder::NGBUF; ++i) bd.gbuf[i] = (char*)bd.take(bd.gbig);
 
     // ---- stem
     const int Hs = out_dim(A.in_h, A.stem_k, A.stem_stride), Ws = out_dim(A.in_w, A.stem_k, A.stem_stride);
@@ -709,13 +710,21 @@ static int run_plan(resist_ctx* ctx, Plan& plan, const PatchArgs& pa, bool updat
     const bool bf = ctx->opts.dtype == RESIST_BF16;
     long long n_launch = 0;
     Profiler& pf = ctx->prof;
+    const cudaStream_t caller_st = st;
+    const bool overlap = !pf.on && update;
+    if (overlap && !ctx->main_stream) {
+        int lo = 0, hi = 0; cudaDeviceGetStreamPriorityRange(&lo, &hi);      // hi: numerically lowest = greatest priority
+        if (cudaStreamCreateWithPriority(&ctx->main_stream, cudaStreamNonBlocking, hi) != cudaSuccess ||
+            cudaEventCreateWithFlags(&ctx->ev_enter, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&ctx->ev_leave, cudaEventDisableTiming) != cudaSuccess) { ctx->err = "cannot create the main stream"; return RESIST_ECUDA; }
+    }
+    if (overlap) { cudaEventRecord(ctx->ev_enter, caller_st); cudaStreamWaitEvent(ctx->main_stream, ctx->ev_enter, 0); st = ctx->main_stream; }
     if (plan.nsites) { pf.begin(PK_PATCH, 1, 0, 0, st); patch_kernel<<<(plan.nsites + 63) / 64, 64, 0, st>>>(plan.d_sites, plan.nsites, pa); pf.end(st); ++n_launch; }
     // A layer's weight gradient and data gradient both read dy and are independent of each other: the weight gradients
     // (and their partial-sum reductions) go to a second stream, one after another, while the main stream carries on
     // down the network.  Gradient buffers are recycled, so a launch that writes a buffer which a weight gradient in
     // flight still reads first waits for the second stream (join_before, worked out when the plan was built).
     // Per-kernel profiling keeps everything on one stream.
-    const bool overlap = !pf.on && update;
     if (overlap && !ctx->side_stream) {
         if (cudaStreamCreateWithFlags(&ctx->side_stream, cudaStreamNonBlocking) != cudaSuccess ||
             cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
@@ -798,6 +807,7 @@ static int run_plan(resist_ctx* ctx, Plan& plan, const PatchArgs& pa, bool updat
         pf.end(st);
         ++n_launch;
     }
+    if (overlap) { cudaEventRecord(ctx->ev_leave, st); cudaStreamWaitEvent(caller_st, ctx->ev_leave, 0); }
     pf.collect(st);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { ctx->err = std::string("launch failed: ") + cudaGetErrorString(e); return RESIST_ECUDA; }

@@ -215,6 +215,7 @@ int resist_destroy(resist_ctx* ctx) {
     ctx_free(ctx, ctx->d_param_blob); ctx_free(ctx, ctx->pa.global); ctx_free(ctx, ctx->d_ws); ctx_free(ctx, ctx->d_eval_ws);
     ctx_free(ctx, ctx->d_seg);
     if (ctx->side_stream) { cudaStreamDestroy(ctx->side_stream); cudaEventDestroy(ctx->ev_fork); cudaEventDestroy(ctx->ev_side_done); }
+    if (ctx->main_stream) { cudaStreamDestroy(ctx->main_stream); cudaEventDestroy(ctx->ev_enter); cudaEventDestroy(ctx->ev_leave); }
     delete ctx;
     return RESIST_OK;
 }

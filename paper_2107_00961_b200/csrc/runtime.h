@@ -101,5 +101,8 @@ struct resist_ctx {
     int sm_count = 148;
     // weight gradients run beside the data gradient of the same layer on a second stream (created on first use)
     cudaStream_t side_stream = nullptr; cudaEvent_t ev_fork = nullptr, ev_side_done = nullptr;
+    // while they overlap, the main chain of the step runs on a stream of the library's own with the highest priority
+    // (forked from and joined to the caller's stream), so that its CTAs are placed before those of the weight gradients
+    cudaStream_t main_stream = nullptr; cudaEvent_t ev_enter = nullptr, ev_leave = nullptr;
     std::string err;
 };

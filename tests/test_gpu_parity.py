@@ -145,6 +145,58 @@ def test_resnet110_bf16_reduced_batch(lib_mod, backend):
             assert not g[rr[b, 0]:rr[b, 1]].any()
 
 
+def test_resnet110_bf16_full_size_grouped_step(lib_mod):
+    """Configuration 2 at its full size and in the launch configuration bench.py times (S = 4 sub-ResNets of
+    ResNet-110, batch 128 each, one grouped bf16 step).  The oracle computes one sub-ResNet in full (a quarter of a
+    minute); the others are checked through properties that hold at any size."""
+    c = synth.config(2)
+    a = c.arch.to_int32()
+    S, B = c.S, c.batch
+    p0, buf0 = synth.perturbed_params(c.arch, 41)
+    ctx = lib_mod.Context(a, dtype=lib_mod.BF16, momentum=c.momentum)
+    ctx.set_params(p0, buf0)
+    mask = ctx.partition(c.round_seed(0), S)
+    np.testing.assert_array_equal(mask, oracle.partition(a, c.round_seed(0), S))
+    xs, ys = zip(*[synth.batch(c, 0, 0, s, as_bf16=True) for s in range(S)])
+    dx = [to_dev(x, torch.bfloat16) for x in xs]
+    dy = [to_dev(y, None) for y in ys]
+    loss = torch.zeros(S, dtype=torch.float32, device="cuda")
+    ctx.local_step_grouped(dx, dy, c.lr, loss)
+    torch.cuda.synchronize()
+    info = ctx.step_info()
+    assert info["cuda_core_convs"] == 0 and info["tensor_core_convs"] > 0
+    loss = loss.cpu().numpy()
+    rr = oracle.block_ranges(a)
+    for s in range(S):
+        g = ctx.get_grads(s)
+        assert np.isfinite(loss[s]) and np.isfinite(g).all()
+        assert abs(loss[s] - np.log(10.0)) < 2.0                                   # an untrained 10-class net
+        for b, m in enumerate(mask):
+            if not (m >> s & 1):
+                assert not g[rr[b, 0]:rr[b, 1]].any()                              # absent blocks: exactly zero
+        lg = ctx.get_logits(s, B)
+        mx = lg.max(axis=1, keepdims=True)                                         # the loss is the mean cross-entropy of the logits
+        ce = (mx[:, 0] + np.log(np.exp(lg - mx).sum(axis=1)) - lg[np.arange(B), ys[s]]).mean()
+        assert abs(ce - loss[s]) < 1e-4 * max(1.0, abs(ce))
+    # sub-ResNet 0 against the oracle: plain fp32 for logits and loss, same storage rounding for the gradient direction
+    import threading
+    s, res = 0, {}
+
+    def run_oracle(quant):
+        par, mom, buf = p0.copy(), np.zeros_like(p0), buf0.copy()
+        res[quant] = oracle.step(a, oracle.present_of(mask, s), par, mom, buf, xs[s], ys[s], lr=c.lr, mu=c.momentum, quant=quant)
+
+    th = [threading.Thread(target=run_oracle, args=(q,)) for q in (0, 1)]     # the C oracle runs outside the interpreter lock
+    for t in th:
+        t.start()
+    for t in th:
+        t.join()
+    assert norm_max_abs(ctx.get_logits(s, B), res[0]["logits"]) < 2e-2
+    assert abs(loss[s] - res[0]["loss"]) < 2e-2 * max(1.0, abs(res[0]["loss"]))
+    g, h = ctx.get_grads(s).astype(np.float64), res[1]["grads"].astype(np.float64)
+    assert g @ h / (np.linalg.norm(g) * np.linalg.norm(h)) > 0.85
+
+
 def test_eval_matches_oracle(lib_mod):
     for arch in (synth.tiny_arch(), small_bottleneck_arch()):
         a = arch.to_int32()
