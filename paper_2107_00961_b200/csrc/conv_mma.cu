@@ -214,6 +214,8 @@ const MmaProb* __restrict__ probs) {
     const bool a_on = tid < a_step * ga;
     const long long grp_in = (long long)p.G * (p.is == 2 ? p.iP * p.iQ : p.H * p.W) * ca;   // elements of a group of act
     const long long grp_out = (long long)p.G * (p.os == 1 ? p.H * p.W : p.P * p.Q) * ncol_all;
+    const __nv_bfloat16* pf_add = addp;
+    const __nv_bfloat16* pf_x = fuse == 2 ? reinterpret_cast<const __nv_bfloat16*>(p.bn.x) : nullptr;
     auto issue = [&](int unit, int stage) {
         const int grp = unit / subs, j = unit - grp * subs;
         const __nv_bfloat16* ag = act + grp * grp_in + a_g * 8;
@@ -223,6 +225,19 @@ const MmaProb* __restrict__ probs) {
             for (int row = a_row0; row < win_rows; row += a_step, t += a_step, dst += a_step * apitch) {
                 const int pix = *t;                                // padding: read nothing, write zeros
                 cp_async16(dst, ag + (long long)max(pix, 0) * ca, pix >= 0 ? 16u : 0u);
+            }
+        }
+        // what the epilogue of that piece will read besides its accumulators (the residual; the BN input of a fused
+        // backward) was written long ago and is no longer in L2: ask for its 128-byte lines now
+        if (pf_add != nullptr || pf_x != nullptr) {
+            const short* ot = otable + j * sub;
+            for (int r = tid; r < sub; r += MMA_THREADS) {
+                const int op = ot[r];
+                const long long e = grp * grp_out + (long long)op * ncol_all;
+                if (op >= 0 && (e & 63) == 0) {
+                    if (pf_add != nullptr) asm volatile("prefetch.global.L2 [%0];" ::"l"(pf_add + e));
+                    if (pf_x != nullptr) asm volatile("prefetch.global.L2 [%0];" ::"l"(pf_x + e));
+                }
             }
         }
     };
