@@ -33,6 +33,7 @@ sys.path.insert(0, ROOT)
 import synth  # noqa: E402
 
 LOCAL_STEPS = 50
+NCU_DRAM_BYTES_PER_LAUNCH = {"conv_dgrad_mma_bn": 15.80e6, "conv_fwd_mma_bn": 9.86e6}
 POOL = 16            # distinct batches per sub-ResNet, cycled
 
 
@@ -209,7 +210,11 @@ def run_ours(args):
         roof.update(bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s")
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof["peak_source"] = peaks["source"]
-    roof["traffic"] = None
+    # DRAM bytes (read + written) per launch of that kernel family from the ncu capture summarised under profiles/
+    # (mean over the launches of one step); None for a family the capture does not cover
+    roof["traffic"] = NCU_DRAM_BYTES_PER_LAUNCH.get(top_name)
+    roof["traffic_unit"] = "bytes per launch (ncu dram__bytes_read.sum + dram__bytes_write.sum, mean over one step's launches)"
+    roof["algorithmic_bytes_per_launch"] = top["bytes"] / top["operations"]
     roof["arithmetic_intensity"] = ai
     conv_ms = sum(v["ms"] for k, v in prof.items() if k.startswith("conv_") or k == "wgrad_splitk_reduce")
     conv_flops = sum(v["flops"] for k, v in prof.items() if k.startswith("conv_"))
