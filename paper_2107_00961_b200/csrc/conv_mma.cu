@@ -45,7 +45,7 @@ struct alignas(16) MmaProb {
     int os, P, Q;               // output stride (forward of a stride-2 layer stores even positions only, as a P x Q image)
     int is, iP, iQ;             // input stride: 2 = act is stored compact [n_img,iP,iQ,ca] and read as if zero-stuffed to H x W
     int stages;                 // depth of the activation ring (2, 3 or 4)
-    int nsplit;                 // 1, or 2: a CTA computes one half of the output channels (its half of the filter resident)
+    int nsplit;                 // 1, 2 or 4: a CTA computes that fraction of the output channels (its part of the filter resident)
     int variant, smem_bytes;    // which instantiation runs this problem (see mma_variant); dynamic shared memory
     float scale;
     int fuse;                   // 0: convolution only; 1: + BN+ReLU forward of out; 2: + BN+ReLU backward with out as da
@@ -511,7 +511,8 @@ static bool mma_geometry(const ConvProb& p, int mode, MmaGeom& g) {
     const int ppi = g.Hp * g.Wp, halo = pad * g.Wp + pad;
     const int apitch = g.ca * 2 + 16;
     const int wrows = mode == CONV_FWD ? g.ncol : g.ca, wcols = mode == CONV_FWD ? g.ca : g.ncol;
-    // 64 output channels: two CTAs share a piece, each with half of the filter resident (twice the CTAs per SM)
+    // 64 output channels: two CTAs share a piece, each with half of the filter resident (twice the CTAs per SM).  (A split
+    // in four on the 8x8 stage, with three 16-channel CTAs per SM, was measured: no faster, the window is staged four times.)
     g.nsplit = g.ncol == 64 && p.ksz == 3 ? 2 : 1;
     const int ncta_col = g.ncol / g.nsplit;
     const int wrows_c = mode == CONV_FWD ? ncta_col : g.ca, wcols_c = mode == CONV_FWD ? g.ca : ncta_col;
@@ -599,8 +600,8 @@ static void launch_mma_inst(MmaLaunch& a) {
     const int cap = occ[slot] * sms;
     int gx = a.coop ? cap / a.nprob : (cap + a.nprob - 1) / a.nprob;
     if (gx > a.max_tiles) gx = a.max_tiles;
-    gx &= ~1;                                                     // even: a CTA pair shares a piece when the channels are split
-    if (gx < 2) gx = 2;
+    if (gx >= 4) gx &= ~3; else gx &= ~1;                         // a multiple of the channel split (1, 2 or 4): the CTAs of a piece are neighbours
+    if (gx < 4) gx = 4;
     if (a.coop && gx * a.nprob > cap) { a.ok = false; return; }
     cudaLaunchConfig_t cfg = {}; cfg.gridDim = dim3(gx, a.nprob); cfg.blockDim = dim3(MMA_THREADS); cfg.dynamicSmemBytes = a.smem; cfg.stream = a.s;
     cudaLaunchAttribute at[2]; int n = 0;
@@ -835,6 +836,7 @@ __global__ void __launch_bounds__(MMA_THREADS) conv_wgrad_mma_kernel(const MmaWg
 // warp w adds the splits w, w+8, ... (ascending), then the 8 sums are added in warp order.
 __global__ void __launch_bounds__(256) wgrad_mma_reduce_kernel(const MmaWgradProb* __restrict__ probs) {
     pdl_trigger();
+    pdl_wait();                                                   // launched programmatically behind the kernel that writes the partial sums
     const MmaWgradProb& p = probs[blockIdx.y];
     const int n = p.taps * p.K * p.C, splits = p.splits, taps = p.taps, K = p.K, C = p.C;
     const float* __restrict__ partial = p.partial;
@@ -954,7 +956,7 @@ void launch_conv_wgrad_mma_probs(const void* d, int nprob, int max_ctas, size_t 
     return;
 #undef WG_CASE
     long long gx = (max_out + 31) / 32; if (gx > 1184) gx = 1184; if (gx < 1) gx = 1;
-    wgrad_mma_reduce_kernel<<<dim3((unsigned)gx, nprob), 256, 0, s>>>((const MmaWgradProb*)d);
+    launch_pdl(wgrad_mma_reduce_kernel, dim3((unsigned)gx, nprob), 0, s, true, (const MmaWgradProb*)d);
 }
 
 }  // namespace resist
