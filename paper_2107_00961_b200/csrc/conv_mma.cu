@@ -45,7 +45,7 @@ struct alignas(16) MmaProb {
     int os, P, Q;               // output stride (forward of a stride-2 layer stores even positions only, as a P x Q image)
     int is, iP, iQ;             // input stride: 2 = act is stored compact [n_img,iP,iQ,ca] and read as if zero-stuffed to H x W
     int stages;                 // depth of the activation ring (2, 3 or 4)
-    int nsplit;                 // 1, 2 or 4: a CTA computes that fraction of the output channels (its part of the filter resident)
+    int nsplit;                 // 1, or 2: a CTA computes one half of the output channels (its half of the filter resident)
     int variant, smem_bytes;    // which instantiation runs this problem (see mma_variant); dynamic shared memory
     float scale;
     int fuse;                   // 0: convolution only; 1: + BN+ReLU forward of out; 2: + BN+ReLU backward with out as da
@@ -600,8 +600,8 @@ static void launch_mma_inst(MmaLaunch& a) {
     const int cap = occ[slot] * sms;
     int gx = a.coop ? cap / a.nprob : (cap + a.nprob - 1) / a.nprob;
     if (gx > a.max_tiles) gx = a.max_tiles;
-    if (gx >= 4) gx &= ~3; else gx &= ~1;                         // a multiple of the channel split (1, 2 or 4): the CTAs of a piece are neighbours
-    if (gx < 4) gx = 4;
+    gx &= ~1;                                                     // even: a CTA pair shares a piece when the channels are split
+    if (gx < 2) gx = 2;
     if (a.coop && gx * a.nprob > cap) { a.ok = false; return; }
     cudaLaunchConfig_t cfg = {}; cfg.gridDim = dim3(gx, a.nprob); cfg.blockDim = dim3(MMA_THREADS); cfg.dynamicSmemBytes = a.smem; cfg.stream = a.s;
     cudaLaunchAttribute at[2]; int n = 0;
@@ -825,10 +825,10 @@ __global__ void __launch_bounds__(MMA_THREADS) conv_wgrad_mma_kernel(const MmaWg
     }
     __syncthreads();
     float* dst = p.partial + ((long long)split * p.taps + tap0) * K * C;
-    for (int i = tid; i < per; i += MMA_THREADS) {
-        float s = red[i];
-        for (int w = 1; w < WP; ++w) s += red[(long long)w * per + i];
-        dst[i] = s;
+    for (int i = tid * 4; i < per; i += MMA_THREADS * 4) {           // per is a multiple of 256; four sums per thread and access
+        float4 s = *reinterpret_cast<const float4*>(red + i);
+        for (int w = 1; w < WP; ++w) { const float4 v = *reinterpret_cast<const float4*>(red + (long long)w * per + i); s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w; }
+        *reinterpret_cast<float4*>(dst + i) = s;
     }
 }
 
@@ -845,7 +845,7 @@ __global__ void __launch_bounds__(256) wgrad_mma_reduce_kernel(const MmaWgradPro
     for (int base = blockIdx.x * 32; base < n; base += gridDim.x * 32) {
         const int i = base + lane;                                // n is a multiple of 256
         float s = 0.f;
-#pragma unroll 4
+#pragma unroll 8
         for (int sp = warp; sp < splits; sp += 8) s += partial[(long long)sp * n + i];
         red[warp][lane] = s;
         __syncthreads();
