@@ -11,7 +11,9 @@ Inputs are synthetic (Gaussian pixels, uniform labels), generated before the tim
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
 
 `value` is measured with the inputs resident in HBM; `e2e` repeats the same steps through the same public calls
-with the inputs in pinned host memory (copied in every step, the losses copied out every step).
+with the inputs in pinned host memory: every step's inputs are copied to the device inside the timed region (on a copy
+stream, into one of two staging sets, so that the copy for the next step runs beside the current step) and every
+step's losses are copied back to pinned host memory.
 With --gpus N > 1 (under torchrun) every rank runs an independent replica on its own GPU and the values add up:
 the path has no exchange between GPUs.
 """
@@ -123,11 +125,18 @@ def run_ours(args):
     d_y = [[torch.from_numpy(y).to(dev) for y in by] for by in ys]
     h_x = [[torch.from_numpy(synth.bf16_bits(x).view(np.int16)).view(torch.bfloat16).pin_memory() for x in bx] for bx in xs]
     h_y = [[torch.from_numpy(y).pin_memory() for y in by] for by in ys]
-    stage_x = [torch.empty_like(d_x[0][s]) for s in range(S)]
-    stage_y = [torch.empty_like(d_y[0][s]) for s in range(S)]
+    # end-to-end pass: two sets of device staging buffers; the copy of step i+1's inputs (pinned host memory -> device, on a
+    # copy stream) runs while step i computes, and every step's losses are copied to their own slot of a pinned host ring
+    stage_x = [[torch.empty_like(d_x[0][s]) for s in range(S)] for _ in range(2)]
+    stage_y = [[torch.empty_like(d_y[0][s]) for s in range(S)] for _ in range(2)]
     loss = torch.zeros(S, dtype=torch.float32, device=dev)
-    h_loss = torch.zeros(S, dtype=torch.float32).pin_memory()
+    h_loss = torch.zeros(max(K, W) + 1, S, dtype=torch.float32).pin_memory()
     stream = torch.cuda.current_stream()
+    copy_stream = torch.cuda.Stream(device=dev)
+    ev_copied = [torch.cuda.Event() for _ in range(2)]
+    ev_free = [torch.cuda.Event() for _ in range(2)]
+    for e in ev_free:
+        e.record(stream)
     state = {"step": 0, "round": 0, "launches": 0}
 
     def new_round():
@@ -137,12 +146,17 @@ def run_ours(args):
     def one_step(e2e: bool):
         i = state["step"] % POOL
         if e2e:
-            for s in range(S):
-                stage_x[s].copy_(h_x[i][s], non_blocking=True)
-                stage_y[s].copy_(h_y[i][s], non_blocking=True)
-            ctx.local_step_grouped(stage_x, stage_y, cfg.lr, loss)
-            h_loss.copy_(loss, non_blocking=True)
-            stream.synchronize()              # the caller reads the loss every step
+            b = state["step"] % 2
+            copy_stream.wait_event(ev_free[b])                    # the step that last used this staging set has finished
+            with torch.cuda.stream(copy_stream):
+                for s in range(S):
+                    stage_x[b][s].copy_(h_x[i][s], non_blocking=True)
+                    stage_y[b][s].copy_(h_y[i][s], non_blocking=True)
+                ev_copied[b].record(copy_stream)
+            stream.wait_event(ev_copied[b])
+            ctx.local_step_grouped(stage_x[b], stage_y[b], cfg.lr, loss)
+            h_loss[state["step"] % h_loss.shape[0]].copy_(loss, non_blocking=True)   # this step's losses, read by the host after the run
+            ev_free[b].record(stream)
         else:
             ctx.local_step_grouped(d_x[i], d_y[i], cfg.lr, loss)
         state["step"] += 1
@@ -184,6 +198,7 @@ def run_ours(args):
     clocks = sampler.stop()
     info = ctx.step_info()
     ms_e2e, _ = timed(True)
+    assert bool(torch.isfinite(h_loss[:min(K, h_loss.shape[0])]).all()), "the end-to-end pass produced a non-finite loss"
 
     # per-kernel pass: the same steps with every launch bracketed by CUDA events on the library's stream
     peaks = measured_peaks()
