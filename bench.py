@@ -164,7 +164,7 @@ def run_ours(args):
         if state["step"] % LOCAL_STEPS == 0:
             ctx.aggregate()
             new_round()
-            state["launches"] += 4            # aggregate (parameters, buffers) + scatter (parameters, buffers)
+            state["launches"] += 3            # aggregate (one launch) + scatter (parameters, buffers)
 
     def barrier():
         if world > 1:
@@ -325,15 +325,62 @@ def run_reference(args):
         "e2e": {"value": v, "unit": "images/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
 
 
+def run_reassembly(args):
+    """Secondary measurement (not the headline line): the synchronisation step alone on the ResNet-101 parameter set
+    (44.5 M fp32 parameters, bf16 shadow, momentum), S in {2, 4, 8}: `steps` calls of resist_aggregate and of
+    resist_partition each, per-kernel CUDA-event times from the library, bandwidth against the measured HBM peak.
+    The working copies hold the scattered global values (bandwidth does not depend on the values)."""
+    import torch
+    import paper_2107_00961_b200 as lib
+    torch.cuda.set_device(0)
+    cfg = synth.config(5)
+    peaks = measured_peaks()
+    ctx = lib.Context(cfg.arch.to_int32(), dtype=lib.BF16, momentum=0.9, seed=cfg.init_seed, device="cuda:0")
+    K, W = args.steps, args.warmup
+    out = {"metric": "reassembly and repartition bandwidth", "unit": "GB/s", "n_gpus": 1, "steps": K, "warmup": W, "dtype": "f32",
+           "data": "synthetic", "config": {"workload": "configs[4]: reassembly / repartition stress on the ResNet-101 parameter set, S in {2,4,8}"},
+           "peak_GBps": peaks["hbm_gbs"], "peak_source": peaks["source"], "by_S": {}}
+    for S in (2, 4, 8):
+        for i in range(W):
+            ctx.partition(cfg.round_seed(100 * S + i), S)
+            ctx.aggregate()
+        torch.cuda.synchronize()
+        ctx.set_profiling(True)
+        ctx.get_profile()
+        t0 = time.perf_counter()
+        for i in range(K):
+            ctx.partition(cfg.round_seed(1000 * S + i), S)
+        torch.cuda.synchronize()
+        t1 = time.perf_counter()
+        for i in range(K):
+            ctx.aggregate()
+        torch.cuda.synchronize()
+        t2 = time.perf_counter()
+        prof = ctx.get_profile()
+        ctx.set_profiling(False)
+        rec = {"partition_call_us": (t1 - t0) / K * 1e6, "aggregate_call_us": (t2 - t1) / K * 1e6}
+        for name in ("scatter", "aggregate"):
+            v = prof[name]
+            gbps = v["bytes"] / max(v["ms"], 1e-9) / 1e6
+            rec[name] = {"us_per_call": v["ms"] / v["operations"] * 1e3, "MB_per_call": v["bytes"] / v["operations"] / 1e6, "GBps": gbps,
+                         "frac_of_hbm_peak": gbps / peaks["hbm_gbs"]}
+        out["by_S"][str(S)] = rec
+    print(json.dumps(out))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="train", choices=["train", "reassembly"],
+                    help="train (default): the headline line; reassembly: the synchronisation kernels alone")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
-    if args.impl == "reference":
+    if args.workload == "reassembly":
+        run_reassembly(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

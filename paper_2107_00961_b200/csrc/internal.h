@@ -140,7 +140,7 @@ void launch_sgd(const Segment* d, int nseg, long long nchunks, ParamArrays pa, f
 void launch_scatter(const Segment* d, int nseg, long long nchunks, ParamArrays pa, bool zero_momentum, bool shadow,
                     cudaStream_t s);
 void launch_scatter_buffers(const Segment* d, int nseg, long long nchunks, ParamArrays pa, cudaStream_t s);
-void launch_aggregate(const Segment* d, int nseg, long long nchunks, const float* sub, long long stride,
-                      float* global, int S, cudaStream_t s);
+struct AggArrays { const float* sub_p; const float* sub_b; long long stride_p, stride_b; float* global_p; float* global_b; };   // _p parameters, _b BN running statistics
+void launch_aggregate(const Segment* d, int nseg, long long nchunks, const AggArrays& arr, int S, cudaStream_t s);
 
 }  // namespace resist

@@ -103,33 +103,57 @@ __device__ __forceinline__ float mean_of_owners(const float* __restrict__ sub, l
     return __fadd_rn(first, __fdiv_rn(acc, (float)cnt));
 }
 
-__global__ void __launch_bounds__(256) aggregate_kernel(const Segment* __restrict__ segs, int nseg,
-                                                        const float* __restrict__ sub, long long stride,
-                                                        float* __restrict__ global, int S) {
+// Segment::sub selects the array pair: 0 = parameters, 1 = BN running statistics (one launch serves both).
+__global__ void __launch_bounds__(256, 4) aggregate_kernel(const Segment* __restrict__ segs, int nseg, AggArrays arr, int S) {
     const Segment& sg = find_segment(segs, nseg, blockIdx.x);
     const Range r = chunk_range(sg, blockIdx.x);
-    const unsigned mask = sg.mask;
+    const int which = sg.sub != 0;
+    const float* __restrict__ sub = which ? arr.sub_b : arr.sub_p; const long long stride = which ? arr.stride_b : arr.stride_p;
+    float* __restrict__ global = which ? arr.global_b : arr.global_p;
+    const unsigned mask = sg.mask & (S >= 32 ? 0xffffffffu : ((1u << S) - 1u));   // owners are sub-ResNets 0 .. S-1
     int done = 0;
     if (((r.base | stride) & 3) == 0) {
         const int nq = r.len >> 2;
         const int cnt = __popc(mask);
-        for (int q = threadIdx.x; q < nq; q += 256) {
-            const long long i = r.base + 4LL * q;
-            float4 first = make_float4(0.f, 0.f, 0.f, 0.f), acc = first; int seen = 0;
-            for (int s = 0; s < S; ++s)
-                if (mask >> s & 1u) {
-                    const float4 x = *reinterpret_cast<const float4*>(sub + (long long)s * stride + i);
-                    if (seen == 0) first = x;
-                    else { acc.x = __fadd_rn(acc.x, __fsub_rn(x.x, first.x)); acc.y = __fadd_rn(acc.y, __fsub_rn(x.y, first.y));
-                           acc.z = __fadd_rn(acc.z, __fsub_rn(x.z, first.z)); acc.w = __fadd_rn(acc.w, __fsub_rn(x.w, first.w)); }
-                    ++seen;
+        // Four 16-byte groups per thread at a time, and for each owner (ascending; the mask is the segment's, so the loop is
+        // uniform over the CTA) their four loads in flight together: the kernel is bound by how many bytes it keeps in flight.
+        // The arithmetic per element is the scalar routine's: first + (sum over the other owners of (w_s - first)) / count.
+        for (int q0 = threadIdx.x; q0 < nq && cnt > 0; q0 += 4 * 256) {
+            float4 first[4], acc[4];
+            unsigned m = mask;
+            const int s0 = __ffs(m) - 1; m &= m - 1;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int q = q0 + u * 256;
+                first[u] = q < nq ? *reinterpret_cast<const float4*>(sub + (long long)s0 * stride + r.base + 4LL * q) : make_float4(0.f, 0.f, 0.f, 0.f);
+                acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            while (m) {
+                const int sidx = __ffs(m) - 1; m &= m - 1;
+                float4 x[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int q = q0 + u * 256;
+                    x[u] = q < nq ? *reinterpret_cast<const float4*>(sub + (long long)sidx * stride + r.base + 4LL * q) : first[u];
                 }
-            if (cnt == 0) continue;
-            float4 out = first;
-            if (cnt > 1) { const float c = (float)cnt;
-                out.x = __fadd_rn(first.x, __fdiv_rn(acc.x, c)); out.y = __fadd_rn(first.y, __fdiv_rn(acc.y, c));
-                out.z = __fadd_rn(first.z, __fdiv_rn(acc.z, c)); out.w = __fadd_rn(first.w, __fdiv_rn(acc.w, c)); }
-            *reinterpret_cast<float4*>(global + i) = out;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    acc[u].x = __fadd_rn(acc[u].x, __fsub_rn(x[u].x, first[u].x)); acc[u].y = __fadd_rn(acc[u].y, __fsub_rn(x[u].y, first[u].y));
+                    acc[u].z = __fadd_rn(acc[u].z, __fsub_rn(x[u].z, first[u].z)); acc[u].w = __fadd_rn(acc[u].w, __fsub_rn(x[u].w, first[u].w));
+                }
+            }
+            const float c = (float)cnt;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int q = q0 + u * 256;
+                if (q >= nq) continue;
+                float4 out = first[u];
+                if (cnt > 1) {
+                    out.x = __fadd_rn(first[u].x, __fdiv_rn(acc[u].x, c)); out.y = __fadd_rn(first[u].y, __fdiv_rn(acc[u].y, c));
+                    out.z = __fadd_rn(first[u].z, __fdiv_rn(acc[u].z, c)); out.w = __fadd_rn(first[u].w, __fdiv_rn(acc[u].w, c));
+                }
+                *reinterpret_cast<float4*>(global + r.base + 4LL * q) = out;
+            }
         }
         done = nq << 2;
     }
@@ -158,10 +182,9 @@ void launch_scatter_buffers(const Segment* d, int nseg, long long nchunks, Param
     if (nchunks <= 0) return;
     scatter_buffers_kernel<<<(unsigned)nchunks, 256, 0, s>>>(d, nseg, pa);
 }
-void launch_aggregate(const Segment* d, int nseg, long long nchunks, const float* sub, long long stride,
-                      float* global, int S, cudaStream_t s) {
+void launch_aggregate(const Segment* d, int nseg, long long nchunks, const AggArrays& arr, int S, cudaStream_t s) {
     if (nchunks <= 0) return;
-    aggregate_kernel<<<(unsigned)nchunks, 256, 0, s>>>(d, nseg, sub, stride, global, S);
+    aggregate_kernel<<<(unsigned)nchunks, 256, 0, s>>>(d, nseg, arr, S);
 }
 
 }  // namespace resist

@@ -356,7 +356,7 @@ int resist_aggregate(resist_ctx* ctx, resist_stream stream) {
     auto build = [&](bool buffers, std::vector<Segment>& out, long long& ch) {
         const long long total = buffers ? L.n_buffers : L.n_params;
         long long run = 0; uint32_t run_mask = all;
-        auto flush = [&](long long end) { if (end > run) { Segment s{run, end - run, ch, run_mask, 0}; ch += (s.len + SEG_CHUNK - 1) / SEG_CHUNK; out.push_back(s); } run = end; };
+        auto flush = [&](long long end) { if (end > run) { Segment s{run, end - run, ch, run_mask, buffers ? 1 : 0}; ch += (s.len + SEG_CHUNK - 1) / SEG_CHUNK; out.push_back(s); } run = end; };
         for (size_t b = 0; b < L.blk.size(); ++b) {
             const long long bb = buffers ? L.blk[b].buf_begin : L.blk[b].begin, be = buffers ? L.blk[b].buf_end : L.blk[b].end;
             if (ctx->mask[b] == run_mask) continue;           // extends the current run (block ranges are contiguous)
@@ -366,17 +366,16 @@ int resist_aggregate(resist_ctx* ctx, resist_stream stream) {
         if (!L.blk.empty() && run_mask != all) { flush(buffers ? L.blk.back().buf_end : L.blk.back().end); run_mask = all; }
         flush(total);
     };
-    build(false, segs, chunks); build(true, bsegs, bchunks);
-    int rc = ensure_seg_table(ctx, (int)(segs.size() + bsegs.size()));
+    build(false, segs, chunks); bchunks = chunks; build(true, bsegs, bchunks);   // one table, one launch: the statistics' chunks follow the parameters'
+    segs.insert(segs.end(), bsegs.begin(), bsegs.end());
+    int rc = ensure_seg_table(ctx, (int)segs.size());
     if (rc) return rc;
     CK(cudaMemcpyAsync(ctx->d_seg, segs.data(), segs.size() * sizeof(Segment), cudaMemcpyHostToDevice, st));
-    CK(cudaMemcpyAsync(ctx->d_seg + segs.size(), bsegs.data(), bsegs.size() * sizeof(Segment), cudaMemcpyHostToDevice, st));
     double rd = 0, wr = 0;
     for (const Segment& g : segs) { rd += (double)g.len * __builtin_popcount(g.mask); wr += (double)g.len; }
-    for (const Segment& g : bsegs) { rd += (double)g.len * __builtin_popcount(g.mask); wr += (double)g.len; }
-    ctx->prof.begin(PK_AGGREGATE, 2, 4.0 * (rd + wr), 0, st);
-    launch_aggregate(ctx->d_seg, (int)segs.size(), chunks, ctx->pa.w, ctx->pa.n, ctx->pa.global, S, st);
-    launch_aggregate(ctx->d_seg + segs.size(), (int)bsegs.size(), bchunks, ctx->pa.buf, ctx->pa.nbuf, ctx->pa.global_buf, S, st);
+    ctx->prof.begin(PK_AGGREGATE, 1, 4.0 * (rd + wr), 0, st);
+    const AggArrays arr{ctx->pa.w, ctx->pa.buf, ctx->pa.n, ctx->pa.nbuf, ctx->pa.global, ctx->pa.global_buf};
+    launch_aggregate(ctx->d_seg, (int)segs.size(), bchunks, arr, S, st);
     ctx->prof.end(st); ctx->prof.collect(st);
     CK(cudaGetLastError());
     CK(cudaStreamSynchronize(st));
