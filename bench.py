@@ -365,6 +365,28 @@ def run_reassembly(args):
             rec[name] = {"us_per_call": v["ms"] / v["operations"] * 1e3, "MB_per_call": v["bytes"] / v["operations"] / 1e6, "GBps": gbps,
                          "frac_of_hbm_peak": gbps / peaks["hbm_gbs"]}
         out["by_S"][str(S)] = rec
+    ctx.close()
+    # the fused SGD-momentum update at a parameter count where bandwidth, not launch latency, is the time: a wide CIFAR
+    # bottleneck net (the widths of configs[2] at reduced depth, 14 M parameters), S = 4, batch 2, grouped steps
+    arch = synth.wide_cifar_arch(policy="stage_first_shared", depths=(2, 2, 2, 2))
+    ctx = lib.Context(arch.to_int32(), dtype=lib.BF16, momentum=0.9, seed=1, device="cuda:0")
+    S, B = 4, 2
+    ctx.partition(11, S)
+    xs = [torch.from_numpy(synth.round_to_bf16(synth.standard_normal(s, B * 32 * 32 * 3).astype(np.float32).reshape(B, 32, 32, 3))).cuda().to(torch.bfloat16)
+          for s in range(S)]
+    ys = [torch.zeros(B, dtype=torch.int32, device="cuda") for _ in range(S)]
+    loss = torch.zeros(S, dtype=torch.float32, device="cuda")
+    for _ in range(W):
+        ctx.local_step_grouped(xs, ys, 0.1, loss)
+    torch.cuda.synchronize()
+    ctx.set_profiling(True)
+    ctx.get_profile()
+    for _ in range(min(K, 20)):
+        ctx.local_step_grouped(xs, ys, 0.1, loss)
+    v = ctx.get_profile()["sgd_momentum"]
+    gbps = v["bytes"] / max(v["ms"], 1e-9) / 1e6
+    out["sgd_momentum"] = {"params_per_subnet_held": v["bytes"] / v["operations"] / 22.0 / S, "us_per_call": v["ms"] / v["operations"] * 1e3,
+                           "MB_per_call": v["bytes"] / v["operations"] / 1e6, "GBps": gbps, "frac_of_hbm_peak": gbps / peaks["hbm_gbs"]}
     print(json.dumps(out))
 
 

@@ -168,6 +168,21 @@ def test_bottleneck_bf16_mixed_kernel_families(lib_mod, backend):
         print("worst gradient tensor against the same-rounding oracle:", name, v)
 
 
+def test_wide_bottleneck_bf16_all_widths_of_configuration_3(lib_mod):
+    """The widths of configuration 3 (bottlenecks of 64..512 channels expanding to 256..2048, 32x32 inputs, 100 classes)
+    at reduced depth and batch: every convolution on a tensor-core path, logits and loss against the oracle with the same
+    storage rounding (2e-2) and against plain fp32 (4e-2, see the note in the full-size test), gradient direction."""
+    arch = synth.wide_cifar_arch(policy="stage_first_shared", depths=(2, 2, 2, 2))
+    out = run_protocol_both(arch, 2, 4, 1, 7, "bf16", 1, True, lib_mod)
+    assert out["info"]["cuda_core_convs"] == 0 and out["info"]["tensor_core_convs"] > 0
+    check_bf16(out, arch, grads=False)
+    for s, r in enumerate(out["steps"][0]["subs"]):
+        g, h = r["grads_gpu"].astype(np.float64), r["grads_cpu"].astype(np.float64)
+        assert g @ h / (np.linalg.norm(g) * np.linalg.norm(h)) > 0.9, s
+    out = run_protocol_both(arch, 2, 4, 1, 7, "bf16", 0, True, lib_mod)
+    check_bf16(out, arch, tol=4e-2, grads=False)
+
+
 def test_resnet110_bf16_full_size_grouped_step(lib_mod):
     """Configuration 2 at its full size and in the launch configuration bench.py times (S = 4 sub-ResNets of
     ResNet-110, batch 128 each, one grouped bf16 step).  The oracle computes one sub-ResNet in full (a quarter of a
