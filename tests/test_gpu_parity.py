@@ -183,6 +183,21 @@ def test_wide_bottleneck_bf16_all_widths_of_configuration_3(lib_mod):
     check_bf16(out, arch, tol=4e-2, grads=False)
 
 
+def test_imagenet_stem_bottleneck_bf16(lib_mod):
+    """The layer types of configurations 4 and 5 in bf16: 7x7 stride-2 stem (CUDA cores: 3 input channels), stem BN+ReLU,
+    3x3 stride-2 max-pool forward and backward, bottlenecks of 64..512 output channels.  Against the oracle with the same
+    storage rounding; the comparison with plain fp32 arithmetic is the fp32 test of this family (a max-pool over
+    bf16-rounded values picks other winners than one over fp32 values, so the two runs differ by 5e-2 whoever computes)."""
+    arch = synth.Arch(48, 48, 3, 10, 7, 2, 16, 1, 1,
+                      synth._stack(synth.BOTTLENECK, 16, (1, 2, 3, 1), (64, 128, 256, 512), (16, 32, 64, 128), "paper_section3"))
+    out = run_protocol_both(arch, 2, 4, 1, 9, "bf16", 1, True, lib_mod)
+    check_bf16(out, arch, grads=False)
+    assert out["info"]["tensor_core_convs"] > 100 and out["info"]["cuda_core_convs"] <= 4     # only the stems (2 sub-ResNets x forward, wgrad)
+    for s, r in enumerate(out["steps"][0]["subs"]):
+        g, h = r["grads_gpu"].astype(np.float64), r["grads_cpu"].astype(np.float64)
+        assert g @ h / (np.linalg.norm(g) * np.linalg.norm(h)) > 0.9, s
+
+
 def test_resnet110_bf16_full_size_grouped_step(lib_mod):
     """Configuration 2 at its full size and in the launch configuration bench.py times (S = 4 sub-ResNets of
     ResNet-110, batch 128 each, one grouped bf16 step).  The oracle computes one sub-ResNet in full (a quarter of a
