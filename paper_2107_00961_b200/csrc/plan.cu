@@ -306,9 +306,30 @@ static size_t unroll_subnet(resist_ctx* ctx, Builder& bd, const std::vector<char
     // ---- blocks
     std::vector<BlockMem> bm(nb); std::vector<int> order;
     for (int b = 0; b < nb; ++b) if (present[b]) order.push_back(b);
+    // Launch slots are aligned by stage: the i-th present block of stage t gets slot base(t) + i, where base(t) adds up, over
+    // the earlier stages, the largest number of blocks any sub-ResNet of this round holds there.  Sub-ResNets then share a
+    // launch only with blocks of the same stage (same shapes, same kernel variant), instead of splitting a slot's launch
+    // whenever their block counts per stage differ.
+    std::vector<int> aslot(order.size(), 0); int n_aslots = 0;
+    {
+        int n_stage = 0; for (int b = 0; b < nb; ++b) n_stage = std::max(n_stage, ctx->blocks[b].stage + 1);
+        std::vector<int> stage_max(std::max(n_stage, 1), 0), cnt(std::max(n_stage, 1), 0);
+        for (int b = 0; b < nb; ++b) if (present[b]) ++cnt[std::max(0, ctx->blocks[b].stage)];
+        stage_max = cnt;
+        for (int s2 = 0; s2 < ctx->S && (int)ctx->mask.size() == nb; ++s2) {
+            std::fill(cnt.begin(), cnt.end(), 0);
+            for (int b = 0; b < nb; ++b) if (ctx->mask[b] >> s2 & 1u) ++cnt[std::max(0, ctx->blocks[b].stage)];
+            for (size_t t = 0; t < cnt.size(); ++t) stage_max[t] = std::max(stage_max[t], cnt[t]);
+        }
+        std::vector<int> base(stage_max.size() + 1, 0);
+        for (size_t t = 0; t < stage_max.size(); ++t) base[t + 1] = base[t] + stage_max[t];
+        n_aslots = base.back();
+        std::fill(cnt.begin(), cnt.end(), 0);
+        for (size_t i = 0; i < order.size(); ++i) { const int t = std::max(0, ctx->blocks[order[i]].stage); aslot[i] = base[t] + cnt[t]++; }
+    }
     for (size_t slot = 0; slot < order.size(); ++slot) {
         const int b = order[slot]; const resist_block& K = ctx->blocks[b]; const BlockRef& r = L.blk[b]; BlockMem& s = bm[b];
-        const long long key = KEY_BLOCK0 + 20LL * (long long)slot;
+        const long long key = KEY_BLOCK0 + 20LL * (long long)aslot[slot];
         s.H = cH; s.W = cW; s.Ho = out_dim(cH, 3, K.stride); s.Wo = out_dim(cW, 3, K.stride);
         const long long m_in = (long long)B * s.H * s.W, m_out = (long long)B * s.Ho * s.Wo;
         const float scale = (bd.eval && K.partitionable) ? inv_S : 1.f;
@@ -353,7 +374,7 @@ static size_t unroll_subnet(resist_ctx* ctx, Builder& bd, const std::vector<char
     { int g = bd.gtake(); bd.bn_bwd(BWD0 + 1, xF, bd.gbuf[g_cur], bd.gbuf[g], nullptr, L.final_bn, statF, mF); bd.grel(g_cur); g_cur = g; }
     for (int slot = (int)order.size() - 1; slot >= 0; --slot) {
         const int b = order[slot]; const resist_block& K = ctx->blocks[b]; const BlockRef& r = L.blk[b]; BlockMem& s = bm[b];
-        const long long key = BWD_BLOCK0 + 40LL * ((long long)order.size() - 1 - slot);
+        const long long key = BWD_BLOCK0 + 40LL * ((long long)n_aslots - 1 - aslot[slot]);
         const long long m_in = (long long)B * s.H * s.W, m_out = (long long)B * s.Ho * s.Wo;
         const char* dout = bd.gbuf[g_cur];
         bd.up_src = nullptr;                                     // no zero-stuffed dy carries over from another block
