@@ -35,7 +35,7 @@ sys.path.insert(0, ROOT)
 import synth  # noqa: E402
 
 LOCAL_STEPS = 50
-NCU_DRAM_BYTES_PER_LAUNCH = {"conv_dgrad_mma_bn": 15.80e6, "conv_fwd_mma_bn": 9.86e6}
+NCU_DRAM_BYTES_PER_LAUNCH = {"conv_dgrad_mma_bn": 17.56e6, "conv_fwd_mma_bn": 10.50e6}
 POOL = 16            # distinct batches per sub-ResNet, cycled
 
 
