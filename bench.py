@@ -34,9 +34,16 @@ sys.path.insert(0, ROOT)
 
 import synth  # noqa: E402
 
-LOCAL_STEPS = 50
+# workload name -> (synth configuration number, description, distinct batches per sub-ResNet that are cycled)
+WORKLOADS = {
+    "wide": (3, "configs[2]: wide CIFAR-shaped bottleneck ResNet [3,4,23,3] (64..512 x4), 32x32x3, 100 classes, S=8 sub-ResNets, "
+                "batch 128 per sub-ResNet, bf16 + fp32 master, 50 local steps per round", 8),
+    "resnet110": (2, "configs[1]: CIFAR-shaped ResNet-110, S=4 sub-ResNets, batch 128 per sub-ResNet, bf16 + fp32 master, "
+                     "50 local steps per round", 16),
+    "imagenet": (4, "configs[3]: ImageNet-shaped ResNet-101, 224x224x3, 1000 classes, S=4 sub-ResNets, batch 64 per sub-ResNet, "
+                    "bf16 + fp32 master, 20 local steps per round", 3),
+}
 NCU_DRAM_BYTES_PER_LAUNCH = {"conv_dgrad_mma_bn": 17.56e6, "conv_fwd_mma_bn": 10.50e6}
-POOL = 16            # distinct batches per sub-ResNet, cycled
 
 
 def measured_peaks():
@@ -125,8 +132,10 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
     torch.cuda.set_device(local)
     dev = torch.device(f"cuda:{local}")
-    cfg = synth.config(2)
+    cfg = synth.config(WORKLOADS[args.workload][0])
     S, B, K, W = cfg.S, cfg.batch, args.steps, args.warmup
+    LOCAL_STEPS = cfg.local_steps
+    POOL = WORKLOADS[args.workload][2]
 
     ctx = lib.Context(cfg.arch.to_int32(), dtype=lib.BF16, momentum=cfg.momentum, seed=cfg.init_seed, device=str(dev))
     p0, b0 = synth.init_params(cfg.arch, cfg.init_seed)
@@ -251,13 +260,12 @@ def run_ours(args):
         "metric": "sub-ResNet train images/s", "value": images / (ms * 1e-3), "unit": "images/s", "n_gpus": world, "steps": K,
         "warmup": W, "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
-        "config": {"workload": "configs[1]: CIFAR-shaped ResNet-110, S=4 sub-ResNets, batch 128 per sub-ResNet, bf16 + fp32 master, "
-                               "50 local steps per round with aggregate + repartition between rounds",
+        "config": {"workload": WORKLOADS[args.workload][1],
                    "S": S, "batch_per_subnet": B, "local_steps": LOCAL_STEPS, "multi_gpu": "independent replicas" if world > 1 else "single GPU",
                    "l2": "working set per step (saved activations, %.0f MB) exceeds the 126 MB L2; no flush" % (info["workspace_bytes"] / 1e6)},
         "clocks": clocks,
         "e2e": {"value": images / (ms_e2e * 1e-3), "unit": "images/s", "ms_per_step": ms_e2e / K,
-                "h2d_bytes_per_step": int(S * (B * 32 * 32 * 3 * 2 + B * 4)), "d2h_bytes_per_step": int(S * 4)},
+                "h2d_bytes_per_step": int(S * (B * cfg.arch.in_h * cfg.arch.in_w * cfg.arch.in_c * 2 + B * 4)), "d2h_bytes_per_step": int(S * 4)},
         "gpu_launches": int(launches),
         "conv": {"TFLOPs": conv_flops / max(conv_ms, 1e-9) / 1e9, "frac_of_bf16_peak": conv_flops / max(conv_ms, 1e-9) / 1e9 / peaks["bf16_tflops"],
                  "tensor_core_convs": info["tensor_core_convs"], "cuda_core_convs": info["cuda_core_convs"],
@@ -265,7 +273,8 @@ def run_ours(args):
         "roofline": roof, "kernels": kernels,
     }
     if rank == 0:
-        out["cpu_baseline"] = cpu_baseline(cfg, budget_s=20.0)
+        if not args.skip_cpu_baseline:
+            out["cpu_baseline"] = cpu_baseline(cfg, budget_s=20.0)
         print(json.dumps(out))
     if world > 1:
         dist.barrier()
@@ -405,8 +414,10 @@ def main():
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="train", choices=["train", "reassembly"],
-                    help="train (default): the headline line; reassembly: the synchronisation kernels alone")
+    ap.add_argument("--workload", default="wide", choices=["wide", "resnet110", "imagenet", "reassembly"],
+                    help="wide (default): the headline line; resnet110, imagenet: the other training configurations; "
+                         "reassembly: the synchronisation kernels alone")
+    ap.add_argument("--skip-cpu-baseline", action="store_true", help="leave the oracle's timing out of the line (quick kernel work)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.workload == "reassembly":
