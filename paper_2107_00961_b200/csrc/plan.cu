@@ -19,6 +19,7 @@ bool conv_tc_fill(const ConvProb& p, int mode, void* host_tc);
 size_t conv_tc_prob_bytes();
 int conv_tc_tiles(const void* host_tc);
 size_t conv_tc_smem(const void* host_tc);
+size_t conv_tc_merge(size_t a, size_t b);
 void launch_conv_tc_probs(const void* d_tc, int nprob, int max_tiles, size_t max_smem, cudaStream_t s);
 bool conv_wgrad_tc_supported(const ConvProb& p, int target_ctas, size_t* partial_bytes);
 bool conv_wgrad_tc_fill(const ConvProb& p, int target_ctas, void* host_tc);
@@ -531,7 +532,7 @@ static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool s
                         const int mode = o.kind == OP_CONV_FWD ? CONV_FWD : o.kind == OP_CONV_DGRAD ? CONV_DGRAD : CONV_WGRAD;
                         if (!conv_tc_fill(o.conv, mode, tc.data() + (size_t)n_tc * tcb)) { ctx->err = "tensor map encoding failed"; return RESIST_ECUDA; }
                         L.gx = std::max(L.gx, conv_tc_tiles(tc.data() + (size_t)n_tc * tcb));
-                        L.max_elems = std::max<long long>(L.max_elems, (long long)conv_tc_smem(tc.data() + (size_t)n_tc * tcb));
+                        L.max_elems = (long long)conv_tc_merge((size_t)L.max_elems, conv_tc_smem(tc.data() + (size_t)n_tc * tcb));
                         ++n_tc;
                         const ConvProb& p = o.conv;
                         const double in_e = (double)p.N * p.H * p.W * p.C, out_e = (double)p.N * p.P * p.Q * p.K, w_e = (double)p.K * p.ksz * p.ksz * p.C;
