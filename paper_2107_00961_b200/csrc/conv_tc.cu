@@ -91,49 +91,83 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* v) {
                  : "r"(taddr));
 }
 __device__ __forceinline__ int floor_div(int a, int b) { int q = a / b; if ((a % b != 0) && ((a < 0) != (b < 0))) --q; return q; }
+__device__ __forceinline__ void tma_store_2d(const void* tmap, uint32_t src, int c0, int c1) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(tmap), "r"(src), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void bar_sync_epi() { asm volatile("bar.sync 1, 128;" ::: "memory"); }   // the four epilogue warps
+__device__ __forceinline__ bool bar_and_epi(bool v) {             // barrier of the four epilogue warps that also ANDs a flag
+    uint32_t r;
+    asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.u32 p, %1, 0;\n\tbar.red.and.pred q, 1, 128, p;\n\tselp.u32 %0, 1, 0, q;\n\t}" : "=r"(r) : "r"((uint32_t)v) : "memory");
+    return r != 0;
+}
+__device__ __forceinline__ uint4 lds128(uint32_t a) { uint4 v; asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a)); return v; }
+__device__ __forceinline__ void sts128(uint32_t a, uint4 v) { asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory"); }
+__device__ __forceinline__ uint32_t lds32(uint32_t a) { uint32_t v; asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(a)); return v; }
 
 constexpr int TC_THREADS = 192;
 constexpr int TC_MAX_STAGES = 6;
 constexpr int TILE_M = 128;
+constexpr int SLAB_BYTES = TILE_M * 128;      // 128 rows x 64 channels of bf16
 
-// One forward / dgrad problem.  The two tensor maps come first so that each is 64-byte aligned.
+struct TapRef { int wtap; int shift; };       // weight tap index (r*ksz + s); row shift of the operand inside the window
+
+// One forward / dgrad problem.  The tensor maps come first so that each is 64-byte aligned.
+//
+// Positions and windows.  The positions of a problem are either the pixels of the output in order ("dense": 1x1 layers) or a
+// tall map of Hp x Wp positions per image with `pad` zero rows before each image and `pad` zero columns after each row (3x3
+// layers).  A tile is 128 consecutive positions [p0, p0 + 128).  Its operand for one tap group is a window of positions
+// [p0 - hb, ...) fetched once per 64-channel slab; tap t of the group reads the window from row (p0 - hb - window start) +
+// taps[t].shift on.  Window position (image, yy, xx) holds activation pixel ((yy - pad) * es + gys, xx * es + gxs) of that
+// image, zero outside it: es = 2 with one group per input parity phase makes a stride-2 layer exact work (forward), and four
+// problems, one per output phase, do the same for a stride-2 dgrad.
 struct alignas(64) TcProb {
-    CUtensorMap map_a;        // activations (forward: a; dgrad: dy): flat (channel, pixel); tall (channel, x, y, image)
+    CUtensorMap map_a;        // activations (forward: a; dgrad: dy): (channel, pixel) or (channel, x, y, image), possibly element-strided
     CUtensorMap map_b;        // weights [K][taps][C] viewed as (C, tap, K)
+    CUtensorMap map_out;      // dense problems: the output as (channel, pixel), box 64 x 128
+    CUtensorMap map_add;      // dense problems with a residual: the residual likewise
     const __nv_bfloat16* add; __nv_bfloat16* out;
+    float* stat_tiles;        // [tiles_m][2][ncol]: column sums and sums of squares of the stored tile, or nullptr
     int* status;
-    int flat, taps, ksz, flip;               // flip: dgrad reads weight tap taps-1-t for window tap t
-    int H, W, Wp, Hp, n_img;
-    int R, box_pos, nbox, halo;              // window = nbox boxes of R tall rows (box_pos positions each); halo = Wp + 1 or 0
-    int a_box_bytes;
+    int a_flat;               // 1: a window is one box of 128 pixels of the (channel, pixel) map
+    int dense;                // 1: position index == output pixel index
+    int add_mode;             // 0 none; 1 fetched by TMA into the staging tile (dense); 2 global loads at the output pixel; 3 global loads from a compact tensor that applies at even (y, x) only
+    int ngroups; int gbeg[5]; int gxs[4], gys[4];
+    TapRef taps[9];
+    int es, pad;
+    int Hp, Wp, n_img;
+    int R, box_pos, nbox, hb, a_box_bytes;
     int tiles_m, tiles_n, n_tile, ncol;      // output tile grid; MMA N; channels of the output tensor
     int red, slabs;                          // reduction channels, 64-channel slabs
     int b_mn_major;                          // 0: forward (weights K-major); 1: dgrad (weights MN-major)
     int b_bytes;                             // bytes of one weight tile (one slab, one tap)
-    long long total_pos;                     // positions walked (flat: pixels; tall: n_img * Hp * Wp)
+    int out_slabs;                           // 64-column slabs of the output tile
+    int total_pos;
     float scale;
-    int os, P, Q;                            // output stride: only positions (y, x) with y, x multiples of os are stored, as pixel (y/os, x/os) of a P x Q image
+    int OH, OW, os, oy, ox;                  // position (image, yy, xx) -> output pixel ((yy - pad) * os + oy, xx * os + ox) of an OH x OW image
 };
 
-struct TcLaunch { int nprob, na, nb, a_stage, b_stage, tmem_cols, acc_stride; };
+struct TcLaunch { int nprob, na, nb, a_stage, b_stage, tmem_cols, acc_stride, n_stg, stg_bytes; };
 
 __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const TcProb* __restrict__ probs, const TcLaunch L) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    __shared__ __align__(8) uint64_t bars[4 * TC_MAX_STAGES + 4];
+    __shared__ __align__(8) uint64_t bars[4 * TC_MAX_STAGES + 8];
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
+    __shared__ int pix_s[TILE_M];
+    __shared__ float stat_s[4][2][256];
     const uint32_t a_full = smem_u32(&bars[0]), a_empty = smem_u32(&bars[TC_MAX_STAGES]);
     const uint32_t b_full = smem_u32(&bars[2 * TC_MAX_STAGES]), b_empty = smem_u32(&bars[3 * TC_MAX_STAGES]);
     const uint32_t acc_full = smem_u32(&bars[4 * TC_MAX_STAGES]), acc_empty = smem_u32(&bars[4 * TC_MAX_STAGES + 2]);
-    const uint32_t a_ring = smem_u32(smem), b_ring = a_ring + (uint32_t)(L.na * L.a_stage);
+    const uint32_t add_full = smem_u32(&bars[4 * TC_MAX_STAGES + 4]), stg_free = smem_u32(&bars[4 * TC_MAX_STAGES + 6]);
+    const uint32_t a_ring = smem_u32(smem), b_ring = a_ring + (uint32_t)(L.na * L.a_stage), stg_base = b_ring + (uint32_t)(L.nb * L.b_stage);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < TC_MAX_STAGES; ++s) {
             mbar_init(a_full + 8 * s, 1); mbar_init(a_empty + 8 * s, 1); mbar_init(b_full + 8 * s, 1); mbar_init(b_empty + 8 * s, 1);
         }
-        for (int s = 0; s < 2; ++s) { mbar_init(acc_full + 8 * s, 1); mbar_init(acc_empty + 8 * s, 4); }
+        for (int s = 0; s < 2; ++s) { mbar_init(acc_full + 8 * s, 1); mbar_init(acc_empty + 8 * s, 4); mbar_init(add_full + 8 * s, 1); mbar_init(stg_free + 8 * s, 1); }
         abort_s = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -152,36 +186,47 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const TcProb* __
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer
         if (lane == 0) {
-            uint32_t a_cnt = 0, b_cnt = 0; bool ok = true;
-            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+            uint32_t a_cnt = 0, b_cnt = 0, seq = 0, add_use[2] = {0u, 0u}; bool ok = true;
+            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++seq) {
                 int pi = 0, loc = t;
                 while (loc >= probs[pi].tiles_m * probs[pi].tiles_n) { loc -= probs[pi].tiles_m * probs[pi].tiles_n; ++pi; }
                 const TcProb& p = probs[pi];
                 const int tn = loc % p.tiles_n, tm = loc / p.tiles_n;
-                const int bx0 = p.flat ? 0 : floor_div(tm * TILE_M - p.halo, p.box_pos);
+                if (p.add_mode == 1) {
+                    // the residual tile goes straight into the staging tile the epilogue will finish in place
+                    const uint32_t sb = L.n_stg == 2 ? (seq & 1u) : 0u, uses = L.n_stg == 2 ? (seq >> 1) : seq;
+                    if (!mbar_wait(stg_free + 8 * sb, (uses & 1u) ^ 1u, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(p.status, 7); ok = false; break; }
+                    mbar_expect_tx(add_full + 8 * sb, (uint32_t)(p.out_slabs * SLAB_BYTES));
+                    for (int j = 0; j < p.out_slabs; ++j)
+                        tma_load_2d(stg_base + sb * (uint32_t)L.stg_bytes + (uint32_t)(j * SLAB_BYTES), &p.map_add, add_full + 8 * sb, tn * p.n_tile + j * 64, tm * TILE_M);
+                    ++add_use[sb];
+                }
+                const int bx0 = p.a_flat ? 0 : floor_div(tm * TILE_M - p.hb, p.box_pos);
                 for (int sl = 0; sl < p.slabs && ok; ++sl) {
-                    {
-                        const int s = (int)(a_cnt % (uint32_t)L.na); const uint32_t ph = (a_cnt / (uint32_t)L.na) & 1u;
-                        if (!mbar_wait(a_empty + 8 * s, ph ^ 1u, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(p.status, 1); ok = false; break; }
-                        const uint32_t dst = a_ring + (uint32_t)(s * L.a_stage);
-                        mbar_expect_tx(a_full + 8 * s, (uint32_t)(p.nbox * p.a_box_bytes));
-                        if (p.flat) tma_load_2d(dst, &p.map_a, a_full + 8 * s, sl * 64, tm * TILE_M);
-                        else for (int i = 0; i < p.nbox; ++i) {
-                            const int trow = (bx0 + i) * p.R, img = floor_div(trow, p.Hp), y0 = trow - img * p.Hp - 1;
-                            tma_load_4d(dst + (uint32_t)(i * p.a_box_bytes), &p.map_a, a_full + 8 * s, sl * 64, 0, y0, img);
+                    for (int g = 0; g < p.ngroups && ok; ++g) {
+                        {
+                            const int s = (int)(a_cnt % (uint32_t)L.na); const uint32_t ph = (a_cnt / (uint32_t)L.na) & 1u;
+                            if (!mbar_wait(a_empty + 8 * s, ph ^ 1u, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(p.status, 1); ok = false; break; }
+                            const uint32_t dst = a_ring + (uint32_t)(s * L.a_stage);
+                            mbar_expect_tx(a_full + 8 * s, (uint32_t)(p.nbox * p.a_box_bytes));
+                            if (p.a_flat) tma_load_2d(dst, &p.map_a, a_full + 8 * s, sl * 64, tm * TILE_M);
+                            else for (int i = 0; i < p.nbox; ++i) {
+                                const int trow = (bx0 + i) * p.R, img = floor_div(trow, p.Hp), yy0 = trow - img * p.Hp;
+                                tma_load_4d(dst + (uint32_t)(i * p.a_box_bytes), &p.map_a, a_full + 8 * s, sl * 64, p.gxs[g], (yy0 - p.pad) * p.es + p.gys[g], img);
+                            }
+                            ++a_cnt;
                         }
-                        ++a_cnt;
-                    }
-                    for (int tap = 0; tap < p.taps; ++tap) {
-                        const int s = (int)(b_cnt % (uint32_t)L.nb); const uint32_t ph = (b_cnt / (uint32_t)L.nb) & 1u;
-                        if (!mbar_wait(b_empty + 8 * s, ph ^ 1u, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(p.status, 2); ok = false; break; }
-                        const uint32_t dst = b_ring + (uint32_t)(s * L.b_stage);
-                        const int wtap = p.flip ? p.taps - 1 - tap : tap;
-                        mbar_expect_tx(b_full + 8 * s, (uint32_t)p.b_bytes);
-                        if (!p.b_mn_major) tma_load_3d(dst, &p.map_b, b_full + 8 * s, sl * 64, wtap, tn * p.n_tile);
-                        else for (int j = 0; j * 64 < p.n_tile; ++j)
-                            tma_load_3d(dst + (uint32_t)(j * 8192), &p.map_b, b_full + 8 * s, tn * p.n_tile + j * 64, wtap, sl * 64);
-                        ++b_cnt;
+                        for (int tap = p.gbeg[g]; tap < p.gbeg[g + 1]; ++tap) {
+                            const int s = (int)(b_cnt % (uint32_t)L.nb); const uint32_t ph = (b_cnt / (uint32_t)L.nb) & 1u;
+                            if (!mbar_wait(b_empty + 8 * s, ph ^ 1u, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(p.status, 2); ok = false; break; }
+                            const uint32_t dst = b_ring + (uint32_t)(s * L.b_stage);
+                            const int wtap = p.taps[tap].wtap;
+                            mbar_expect_tx(b_full + 8 * s, (uint32_t)p.b_bytes);
+                            if (!p.b_mn_major) tma_load_3d(dst, &p.map_b, b_full + 8 * s, sl * 64, wtap, tn * p.n_tile);
+                            else for (int j = 0; j * 64 < p.n_tile; ++j)
+                                tma_load_3d(dst + (uint32_t)(j * 8192), &p.map_b, b_full + 8 * s, tn * p.n_tile + j * 64, wtap, sl * 64);
+                            ++b_cnt;
+                        }
                     }
                 }
             }
@@ -191,6 +236,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const TcProb* __
                     for (int i = 0; i < 4096 && !mbar_try(a_full + 8 * (c % L.na), (c / L.na) & 1u); ++i) __nanosleep(64);
                 for (uint32_t c = b_cnt > (uint32_t)L.nb ? b_cnt - L.nb : 0; c < b_cnt; ++c)
                     for (int i = 0; i < 4096 && !mbar_try(b_full + 8 * (c % L.nb), (c / L.nb) & 1u); ++i) __nanosleep(64);
+                for (uint32_t sb = 0; sb < 2; ++sb)
+                    if (add_use[sb]) for (int i = 0; i < 4096 && !mbar_try(add_full + 8 * sb, (add_use[sb] - 1u) & 1u); ++i) __nanosleep(64);
             }
         }
     } else if (warp == 1) {
@@ -202,8 +249,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const TcProb* __
                 while (loc >= probs[pi].tiles_m * probs[pi].tiles_n) { loc -= probs[pi].tiles_m * probs[pi].tiles_n; ++pi; }
                 const TcProb& p = probs[pi];
                 const int tm = loc / p.tiles_n;
-                const int bx0 = p.flat ? 0 : floor_div(tm * TILE_M - p.halo, p.box_pos);
-                const int a_off = p.flat ? 0 : tm * TILE_M - p.halo - bx0 * p.box_pos;
+                const int bx0 = p.a_flat ? 0 : floor_div(tm * TILE_M - p.hb, p.box_pos);
+                const int a_off = p.a_flat ? 0 : tm * TILE_M - p.hb - bx0 * p.box_pos;
                 const uint32_t buf = acc_cnt & 1u, aph = (acc_cnt >> 1) & 1u;
                 if (!mbar_wait(acc_empty + 8 * buf, aph ^ 1u, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(p.status, 3); ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -213,30 +260,31 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const TcProb* __
                                        ((uint32_t)(p.n_tile >> 3) << 17) | ((128u >> 4) << 24);
                 uint32_t acc = 0;
                 for (int sl = 0; sl < p.slabs && ok; ++sl) {
-                    const int sa = (int)(a_cnt % (uint32_t)L.na); const uint32_t pha = (a_cnt / (uint32_t)L.na) & 1u;
-                    if (!mbar_wait(a_full + 8 * sa, pha, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(p.status, 4); ok = false; break; }
-                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    const uint32_t a_base = a_ring + (uint32_t)(sa * L.a_stage) + (uint32_t)a_off * 128u;
                     const int ksteps = (min(64, p.red - sl * 64) + 15) >> 4;
-                    for (int tap = 0; tap < p.taps; ++tap) {
-                        const int sb = (int)(b_cnt % (uint32_t)L.nb); const uint32_t phb = (b_cnt / (uint32_t)L.nb) & 1u;
-                        if (!mbar_wait(b_full + 8 * sb, phb, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(p.status, 5); ok = false; break; }
+                    for (int g = 0; g < p.ngroups && ok; ++g) {
+                        const int sa = (int)(a_cnt % (uint32_t)L.na); const uint32_t pha = (a_cnt / (uint32_t)L.na) & 1u;
+                        if (!mbar_wait(a_full + 8 * sa, pha, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(p.status, 4); ok = false; break; }
                         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                        const int r = tap / p.ksz, q = tap - r * p.ksz;
-                        const uint32_t a_tap = a_base + (uint32_t)(r * p.Wp + q) * 128u;
-                        const uint32_t b_base = b_ring + (uint32_t)(sb * L.b_stage);
-                        for (int k16 = 0; k16 < ksteps; ++k16) {
-                            const uint64_t ad = desc_sw128(a_tap + (uint32_t)k16 * 32u, 16, 1024);
-                            const uint64_t bd = p.b_mn_major ? desc_sw128(b_base + (uint32_t)k16 * 2048u, 8192, 1024)
-                                                             : desc_sw128(b_base + (uint32_t)k16 * 32u, 16, 1024);
-                            umma_bf16(d_tmem, ad, bd, idesc, acc);
-                            acc = 1;
+                        const uint32_t a_base = a_ring + (uint32_t)(sa * L.a_stage) + (uint32_t)a_off * 128u;
+                        for (int tap = p.gbeg[g]; tap < p.gbeg[g + 1]; ++tap) {
+                            const int sb = (int)(b_cnt % (uint32_t)L.nb); const uint32_t phb = (b_cnt / (uint32_t)L.nb) & 1u;
+                            if (!mbar_wait(b_full + 8 * sb, phb, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(p.status, 5); ok = false; break; }
+                            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                            const uint32_t a_tap = a_base + (uint32_t)p.taps[tap].shift * 128u;
+                            const uint32_t b_base = b_ring + (uint32_t)(sb * L.b_stage);
+                            for (int k16 = 0; k16 < ksteps; ++k16) {
+                                const uint64_t ad = desc_sw128(a_tap + (uint32_t)k16 * 32u, 16, 1024);
+                                const uint64_t bd = p.b_mn_major ? desc_sw128(b_base + (uint32_t)k16 * 2048u, 8192, 1024)
+                                                                 : desc_sw128(b_base + (uint32_t)k16 * 32u, 16, 1024);
+                                umma_bf16(d_tmem, ad, bd, idesc, acc);
+                                acc = 1;
+                            }
+                            umma_commit(b_empty + 8 * sb);       // weight tile reusable once these MMAs have read it
+                            ++b_cnt;
                         }
-                        umma_commit(b_empty + 8 * sb);           // weight tile reusable once these MMAs have read it
-                        ++b_cnt;
+                        umma_commit(a_empty + 8 * sa);
+                        ++a_cnt;
                     }
-                    umma_commit(a_empty + 8 * sa);
-                    ++a_cnt;
                 }
                 if (ok) umma_commit(acc_full + 8 * buf);         // accumulator complete
             }
@@ -245,67 +293,130 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const TcProb* __
         // ---------------------------------------------------------------- epilogue: 4 warps, one TMEM lane quadrant each
         const int quad = warp & 3;
         const int m = quad * 32 + lane;                          // row of the tile = TMEM lane
-        uint32_t acc_cnt = 0; bool ok = true;
+        const int et = threadIdx.x - 64;                         // 0..127 among the epilogue threads
+        const bool leader = et == 0;
+        uint32_t acc_cnt = 0, add_use[2] = {0u, 0u}; bool ok = true;
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++acc_cnt) {
             int pi = 0, loc = t;
             while (loc >= probs[pi].tiles_m * probs[pi].tiles_n) { loc -= probs[pi].tiles_m * probs[pi].tiles_n; ++pi; }
             const TcProb& p = probs[pi];
             const int tn = loc % p.tiles_n, tm = loc / p.tiles_n;
             const uint32_t buf = acc_cnt & 1u, aph = (acc_cnt >> 1) & 1u;
+            const uint32_t sb = L.n_stg == 2 ? (acc_cnt & 1u) : 0u;
+            const uint32_t stg = stg_base + sb * (uint32_t)L.stg_bytes;
+            // the staging tile is free again: the leader has waited for the reads of the bulk store it issued from it, and
+            // every warp has finished its share of the last copy-out
+            bar_sync_epi();
             ok = mbar_wait(acc_full + 8 * buf, aph, &abort_s);
-            ok = __all_sync(0xffffffffu, ok);                    // tcgen05.ld below is warp-collective
+            if (ok && p.add_mode == 1) { ok = mbar_wait(add_full + 8 * sb, add_use[sb] & 1u, &abort_s); ++add_use[sb]; }
+            ok = bar_and_epi(ok);                                // one decision for the four warps: they share the barriers below
             if (!ok) { atomicExch(&abort_s, 1); atomicExch(p.status, 6); break; }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            // position -> output pixel
-            long long pix = -1;
-            const long long pos = (long long)tm * TILE_M + m;
-            if (p.flat) { if (pos < p.total_pos) pix = pos; }
-            else if (pos < p.total_pos) {
-                const int trow = (int)(pos / p.Wp), x = (int)(pos - (long long)trow * p.Wp);
-                const int img = trow / p.Hp, y = trow - img * p.Hp - 1;
-                if (x < p.W && y >= 0) {
-                    if (p.os == 1) pix = ((long long)img * p.H + y) * p.W + x;
-                    else if (y % p.os == 0 && x % p.os == 0) pix = ((long long)img * p.P + y / p.os) * p.Q + x / p.os;   // strided layer
-                }
+            // position -> output pixel (and the residual's pixel)
+            const int pos = tm * TILE_M + m;
+            bool valid = pos < p.total_pos;
+            long long pix = pos, addpix = -1;
+            if (valid && (!p.dense || p.add_mode == 3)) {
+                const int trow = pos / p.Wp, xx = pos - trow * p.Wp, img = trow / p.Hp, yy = trow - img * p.Hp;
+                const int y = (yy - p.pad) * p.os + p.oy, x = xx * p.os + p.ox;
+                valid = yy >= p.pad && xx < p.Wp - p.pad && y < p.OH && x < p.OW;
+                pix = ((long long)img * p.OH + y) * p.OW + x;
+                if (p.add_mode == 3 && !((y | x) & 1)) addpix = ((long long)img * ((p.OH + 1) >> 1) + (y >> 1)) * ((p.OW + 1) >> 1) + (x >> 1);
             }
+            if (p.add_mode == 2) addpix = pix;
+            if (!p.dense) pix_s[m] = valid ? (int)pix : -1;
             const uint32_t t_row = tmem_base + buf * (uint32_t)L.acc_stride + ((uint32_t)(quad * 32) << 16);
             const int col0 = tn * p.n_tile;
+            const uint32_t s_row = stg + (uint32_t)m * 128u;
+            const bool gadd = p.add_mode >= 2 && valid && addpix >= 0;
             for (int c0 = 0; c0 < p.n_tile; c0 += 32) {
                 uint32_t v[32];
                 tmem_ld32(t_row + (uint32_t)c0, v);
+                uint4 ga[4];
+                if (gadd) {
+#pragma unroll
+                    for (int g = 0; g < 4; ++g)
+                        ga[g] = (c0 + g * 8 < p.n_tile && col0 + c0 + g * 8 < p.ncol) ? __ldg(reinterpret_cast<const uint4*>(p.add + addpix * p.ncol + col0 + c0 + g * 8)) : make_uint4(0u, 0u, 0u, 0u);
+                }
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                if (pix >= 0) {
 #pragma unroll
-                    for (int g = 0; g < 4; ++g) {
-                        const int c = c0 + g * 8;
-                        if (c < p.n_tile && col0 + c < p.ncol) {
-                            const long long o = pix * p.ncol + col0 + c;
-                            float f[8];
+                for (int g = 0; g < 4; ++g) {
+                    const int c = c0 + g * 8;
+                    if (c < p.n_tile) {
+                        const uint32_t sa = s_row + (uint32_t)(c >> 6) * SLAB_BYTES + ((uint32_t)(((c >> 3) & 7) ^ (m & 7)) << 4);
+                        float f[8];
 #pragma unroll
-                            for (int k = 0; k < 8; ++k) f[k] = __uint_as_float(v[g * 8 + k]) * p.scale;
-                            if (p.add) {
-                                const uint4 a0 = *reinterpret_cast<const uint4*>(p.add + o);
-                                const uint32_t aw[4] = {a0.x, a0.y, a0.z, a0.w};
+                        for (int k = 0; k < 8; ++k) f[k] = valid ? __uint_as_float(v[g * 8 + k]) * p.scale : 0.f;
+                        if (p.add_mode == 1 || gadd) {
+                            const uint4 a0 = p.add_mode == 1 ? lds128(sa) : ga[g];
+                            const uint32_t aw[4] = {a0.x, a0.y, a0.z, a0.w};
+                            if (valid) {
 #pragma unroll
                                 for (int k = 0; k < 4; ++k) {
                                     f[2 * k] += __uint_as_float(aw[k] << 16);
                                     f[2 * k + 1] += __uint_as_float(aw[k] & 0xFFFF0000u);
                                 }
                             }
-                            uint32_t w[4];
-#pragma unroll
-                            for (int k = 0; k < 4; ++k) {
-                                __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * k], f[2 * k + 1]);
-                                w[k] = *reinterpret_cast<uint32_t*>(&h);
-                            }
-                            *reinterpret_cast<uint4*>(p.out + o) = make_uint4(w[0], w[1], w[2], w[3]);
                         }
+                        uint32_t w[4];
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * k], f[2 * k + 1]);
+                            w[k] = *reinterpret_cast<uint32_t*>(&h);
+                        }
+                        sts128(sa, make_uint4(w[0], w[1], w[2], w[3]));
                     }
                 }
             }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // the bulk store reads what this thread wrote
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
             if (lane == 0) mbar_arrive(acc_empty + 8 * buf);     // this warp has read its quadrant of the accumulator
+            bar_sync_epi();                                      // the staging tile is complete
+            if (p.dense && leader) {
+                for (int j = 0; j < p.out_slabs; ++j) tma_store_2d(&p.map_out, stg + (uint32_t)(j * SLAB_BYTES), col0 + j * 64, tm * TILE_M);
+                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            }
+            if (p.stat_tiles) {
+                // column sums of the stored (rounded) values: every warp over its own 32 rows, lane = two neighbouring columns;
+                // the four warps' sums are then added in a fixed order
+                for (int j = 0; j < p.out_slabs; ++j) {
+                    float s0 = 0.f, s1 = 0.f, q0 = 0.f, q1 = 0.f;
+#pragma unroll 8
+                    for (int r = 0; r < 32; ++r) {
+                        const int row = quad * 32 + r;
+                        const uint32_t u = lds32(stg + (uint32_t)(j * SLAB_BYTES) + (uint32_t)row * 128u + ((uint32_t)((lane >> 2) ^ (row & 7)) << 4) + ((uint32_t)(lane & 3) << 2));
+                        const float lo = __uint_as_float(u << 16), hi = __uint_as_float(u & 0xFFFF0000u);
+                        s0 += lo; q0 += lo * lo; s1 += hi; q1 += hi * hi;
+                    }
+                    stat_s[quad][0][j * 64 + 2 * lane] = s0; stat_s[quad][0][j * 64 + 2 * lane + 1] = s1;
+                    stat_s[quad][1][j * 64 + 2 * lane] = q0; stat_s[quad][1][j * 64 + 2 * lane + 1] = q1;
+                }
+                bar_sync_epi();
+                for (int c = et; c < p.n_tile; c += 128) {
+                    if (col0 + c < p.ncol) {
+                        const float su = ((stat_s[0][0][c] + stat_s[1][0][c]) + stat_s[2][0][c]) + stat_s[3][0][c];
+                        const float sq = ((stat_s[0][1][c] + stat_s[1][1][c]) + stat_s[2][1][c]) + stat_s[3][1][c];
+                        p.stat_tiles[((long long)tm * 2 + 0) * p.ncol + col0 + c] = su;
+                        p.stat_tiles[((long long)tm * 2 + 1) * p.ncol + col0 + c] = sq;
+                    }
+                }
+            }
+            if (!p.dense) {
+                // copy-out of a tall tile: 16-byte chunks, eight consecutive lanes per 128-byte run of one output pixel
+                const int n_chunks = p.out_slabs * TILE_M * 8;
+                for (int idx = et; idx < n_chunks; idx += 128) {
+                    const int ch = idx & 7, row = (idx >> 3) & (TILE_M - 1), j = idx >> 10;
+                    const int c = j * 64 + ch * 8, px = pix_s[row];
+                    if (px >= 0 && c < p.n_tile && col0 + c < p.ncol)
+                        *reinterpret_cast<uint4*>(p.out + (long long)px * p.ncol + col0 + c) =
+                            lds128(stg + (uint32_t)(j * SLAB_BYTES) + (uint32_t)row * 128u + ((uint32_t)(ch ^ (row & 7)) << 4));
+                }
+            }
+            if (leader) {
+                if (p.dense) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                mbar_arrive(stg_free + 8 * sb);
+            }
         }
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -340,22 +451,25 @@ void launch_zero_stuff(const UpProb* d, int nprob, long long max_vecs, cudaStrea
 
 // ------------------------------------------------------------------------------------------------ wgrad
 // dw[k][r][s][c] = sum over output positions of dy[pos][k] * a[pos + shift(r,s)][c].  The reduction runs over the
-// positions of the forward kernel (flat pixels, or the tall zero-padded map, where dy reads as zero at the padding
+// positions of the forward problem (pixels in order, or the tall zero-padded map, where dy reads as zero at the padding
 // positions and adds nothing), 128 per pipeline stage: D[cout (128 lanes), cin] per tap, A = dy^T and B = shifted a,
-// both MN-major straight from their 128-byte rows.  A CTA accumulates a range of position chunks for a group of taps
-// and writes an fp32 partial (or, alone on its tile, the result); a second kernel adds the partials in a fixed order.
+// both MN-major straight from their 128-byte rows.  A CTA accumulates a range of position chunks for one group of taps
+// (taps that read the same window: up to three taps of a stride-1 layer, the taps of one input parity phase of a stride-2
+// layer) and writes an fp32 partial, or, alone on its tile, the result; a second kernel adds the partials in a fixed order.
 struct alignas(64) TcWgradProb {
-    CUtensorMap map_dy;       // flat (channel k, pixel); tall (channel k, x, y, image)
-    CUtensorMap map_a;        // likewise for a
+    CUtensorMap map_dy;       // (channel k, pixel) or (channel k, x, y, image)
+    CUtensorMap map_a;        // likewise for a, possibly element-strided
     float* partial;           // [splits][taps][cout][cin]
     float* out;               // [cout][taps][cin]
     int* status;
-    int flat, taps, ksz;
-    int H, W, Wp, Hp, n_img;
-    int R, box_pos, nbox_dy, nbox_a, halo, box_bytes;
+    int dy_flat, a_flat, taps;
+    int es, pad, Hp, Wp, n_img;
+    int R, box_pos, nbox_dy, nbox_a, hb, dy_box_bytes, a_box_bytes;
     int chunks;                                   // position chunks of 128 in total
     int cout, cin, m_tiles, n_tile, n_tiles, a_slabs;
-    int tap_groups, taps_per_group, splits, chunks_per_split;
+    int tap_groups; int gbeg[10]; int gxs[9], gys[9];
+    TapRef tap[9];                                // wtap = index of the tap in dw; shift = row shift inside the a window
+    int splits, chunks_per_split;
     int dy_slab_bytes, a_slab_bytes;              // one 64-channel slab of a stage
     int stage_bytes, stages, tmem_cols;
 };
@@ -370,8 +484,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_wgrad_tc_kernel(const TcWg
     const int tn = id % p.n_tiles; const int tm = id / p.n_tiles;
     const int c_begin = split * p.chunks_per_split;
     const int c_end = min(c_begin + p.chunks_per_split, p.chunks);
-    const int tap0 = tg * p.taps_per_group;
-    const int ntap = min(p.taps - tap0, p.taps_per_group);
+    const int tap0 = p.gbeg[tg], ntap = p.gbeg[tg + 1] - tap0;
     const int nc = c_end - c_begin;
 
     extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -406,21 +519,26 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_wgrad_tc_kernel(const TcWg
                 if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(p.status, 11); ok = false; break; }
                 const int pos0 = (c_begin + i) * TILE_M;
                 const uint32_t dy_dst = ring + (uint32_t)(s * p.stage_bytes), a_dst = dy_dst + 2u * (uint32_t)p.dy_slab_bytes;
-                mbar_expect_tx(bar_full + 8 * s, (uint32_t)((2 * p.nbox_dy + p.a_slabs * p.nbox_a) * p.box_bytes));
-                if (p.flat) {
+                mbar_expect_tx(bar_full + 8 * s, (uint32_t)(2 * p.nbox_dy * p.dy_box_bytes + p.a_slabs * p.nbox_a * p.a_box_bytes));
+                if (p.dy_flat) {
                     for (int j = 0; j < 2; ++j) tma_load_2d(dy_dst + (uint32_t)(j * p.dy_slab_bytes), &p.map_dy, bar_full + 8 * s, tm * 128 + j * 64, pos0);
+                } else {
+                    const int bd0 = pos0 / p.box_pos;
+                    for (int b = 0; b < p.nbox_dy; ++b) {
+                        const int trow = (bd0 + b) * p.R, img = trow / p.Hp, yy0 = trow - img * p.Hp;
+                        for (int j = 0; j < 2; ++j)
+                            tma_load_4d(dy_dst + (uint32_t)(j * p.dy_slab_bytes + b * p.dy_box_bytes), &p.map_dy, bar_full + 8 * s, tm * 128 + j * 64, 0, yy0 - p.pad, img);
+                    }
+                }
+                if (p.a_flat) {
                     for (int j = 0; j < p.a_slabs; ++j) tma_load_2d(a_dst + (uint32_t)(j * p.a_slab_bytes), &p.map_a, bar_full + 8 * s, tn * p.n_tile + j * 64, pos0);
                 } else {
-                    const int bd0 = pos0 / p.box_pos, ba0 = floor_div(pos0 - p.halo, p.box_pos);
-                    for (int b = 0; b < p.nbox_dy; ++b) {
-                        const int trow = (bd0 + b) * p.R, img = trow / p.Hp, y0 = trow - img * p.Hp - 1;
-                        for (int j = 0; j < 2; ++j)
-                            tma_load_4d(dy_dst + (uint32_t)(j * p.dy_slab_bytes + b * p.box_bytes), &p.map_dy, bar_full + 8 * s, tm * 128 + j * 64, 0, y0, img);
-                    }
+                    const int ba0 = floor_div(pos0 - p.hb, p.box_pos);
                     for (int b = 0; b < p.nbox_a; ++b) {
-                        const int trow = (ba0 + b) * p.R, img = floor_div(trow, p.Hp), y0 = trow - img * p.Hp - 1;
+                        const int trow = (ba0 + b) * p.R, img = floor_div(trow, p.Hp), yy0 = trow - img * p.Hp;
                         for (int j = 0; j < p.a_slabs; ++j)
-                            tma_load_4d(a_dst + (uint32_t)(j * p.a_slab_bytes + b * p.box_bytes), &p.map_a, bar_full + 8 * s, tn * p.n_tile + j * 64, 0, y0, img);
+                            tma_load_4d(a_dst + (uint32_t)(j * p.a_slab_bytes + b * p.a_box_bytes), &p.map_a, bar_full + 8 * s, tn * p.n_tile + j * 64,
+                                        p.gxs[tg], (yy0 - p.pad) * p.es + p.gys[tg], img);
                     }
                 }
             }
@@ -438,13 +556,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_wgrad_tc_kernel(const TcWg
                 if (!mbar_wait(bar_full + 8 * s, ph, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(p.status, 12); ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const int pos0 = (c_begin + i) * TILE_M;
-                int dy_off = 0, a_off = 0;
-                if (!p.flat) { dy_off = pos0 - (pos0 / p.box_pos) * p.box_pos; a_off = pos0 - p.halo - floor_div(pos0 - p.halo, p.box_pos) * p.box_pos; }
+                const int dy_off = p.dy_flat ? 0 : pos0 - (pos0 / p.box_pos) * p.box_pos;
+                const int a_off = p.a_flat ? 0 : pos0 - p.hb - floor_div(pos0 - p.hb, p.box_pos) * p.box_pos;
                 const uint32_t dy_base = ring + (uint32_t)(s * p.stage_bytes) + (uint32_t)dy_off * 128u;
                 const uint32_t a_base = ring + (uint32_t)(s * p.stage_bytes) + 2u * (uint32_t)p.dy_slab_bytes + (uint32_t)a_off * 128u;
                 for (int tt = 0; tt < ntap; ++tt) {
-                    const int t = tap0 + tt, r = t / p.ksz, q = t - r * p.ksz;
-                    const uint32_t a_tap = a_base + (uint32_t)(r * p.Wp + q) * 128u;
+                    const uint32_t a_tap = a_base + (uint32_t)p.tap[tap0 + tt].shift * 128u;
                     for (int k16 = 0; k16 < 8; ++k16) {
                         const uint64_t ad = desc_sw128(dy_base + (uint32_t)k16 * 2048u, (uint32_t)p.dy_slab_bytes, 1024);
                         const uint64_t bd = desc_sw128(a_tap + (uint32_t)k16 * 2048u, (uint32_t)p.a_slab_bytes, 1024);
@@ -464,8 +581,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_wgrad_tc_kernel(const TcWg
         const int k = tm * 128 + m;
         if (ok && quad * 32 < p.cout - tm * 128) {            // warp-uniform: this lane quadrant holds real output channels
             for (int tt = 0; tt < ntap; ++tt) {
-                float* dst = p.splits > 1 ? p.partial + (((long long)split * p.taps + tap0 + tt) * p.cout + k) * p.cin + tn * p.n_tile
-                                          : p.out + ((long long)k * p.taps + tap0 + tt) * p.cin + tn * p.n_tile;
+                const int wt = p.tap[tap0 + tt].wtap;
+                float* dst = p.splits > 1 ? p.partial + (((long long)split * p.taps + wt) * p.cout + k) * p.cin + tn * p.n_tile
+                                          : p.out + ((long long)k * p.taps + wt) * p.cin + tn * p.n_tile;
                 for (int c0 = 0; c0 < p.n_tile; c0 += 32) {
                     uint32_t v[32];
                     if (nc > 0) { tmem_ld32(tmem_d + ((uint32_t)(quad * 32) << 16) + (uint32_t)(tt * p.n_tile + c0), v);
@@ -503,6 +621,33 @@ __global__ void __launch_bounds__(256) wgrad_tc_reduce_kernel(const TcWgradProb*
     }
 }
 
+// ------------------------------------------------------------------------------------------------ BN statistics from the tiles' sums
+// The forward kernel leaves, per 128-position tile, the column sums and sums of squares of the values it stored.  One warp
+// per channel adds them in a fixed order in double and turns them into mean, 1/sqrt(var + eps) and the running statistics.
+__global__ void __launch_bounds__(256) bn_finalize_tiles_kernel(const BnProb* __restrict__ probs) {
+    const BnProb& p = probs[blockIdx.y];
+    const int lane = threadIdx.x & 31;
+    const int c = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (c >= p.C) return;
+    const float* tiles = reinterpret_cast<const float*>(p.partial);
+    double a0 = 0.0, a1 = 0.0;
+    for (int k = lane; k < p.chunks; k += 32) { a0 += (double)tiles[((long long)k * 2 + 0) * p.C + c]; a1 += (double)tiles[((long long)k * 2 + 1) * p.C + c]; }
+    for (int d = 16; d; d >>= 1) { a0 += __shfl_xor_sync(0xffffffffu, a0, d); a1 += __shfl_xor_sync(0xffffffffu, a1, d); }
+    if (lane != 0) return;
+    const double m = (double)p.m, mean = a0 / m;
+    double var = a1 / m - mean * mean; if (var < 0.0) var = 0.0;
+    p.stat[c] = (float)mean;
+    p.stat[p.C + c] = (float)(1.0 / sqrt(var + (double)p.eps));
+    if (p.run_mean) {
+        const double unb = p.m > 1 ? var * m / (m - 1.0) : var, mo = (double)p.momentum;
+        p.run_mean[c] = (float)((1.0 - mo) * (double)p.run_mean[c] + mo * mean);
+        p.run_var[c] = (float)((1.0 - mo) * (double)p.run_var[c] + mo * unb);
+    }
+}
+void launch_bn_finalize_tiles(const BnProb* d, int nprob, int max_c, cudaStream_t s) {
+    bn_finalize_tiles_kernel<<<dim3((max_c + 7) / 8, nprob), 256, 0, s>>>(d);
+}
+
 // ------------------------------------------------------------------------------------------------ host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
@@ -517,65 +662,76 @@ static EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// bf16 tensor map of `rank` dimensions (innermost first), 128-byte swizzle, zero fill out of bounds
-static bool encode_map(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes, const uint32_t* box) {
+// bf16 tensor map of `rank` dimensions (innermost first), 128-byte swizzle, zero fill out of bounds; estr = traversal strides
+static bool encode_map(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes, const uint32_t* box,
+                       const uint32_t* estr = nullptr) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     cuuint64_t d[5]; cuuint64_t st[4]; cuuint32_t b[5]; cuuint32_t es[5];
-    for (int i = 0; i < rank; ++i) { d[i] = dims[i]; b[i] = box[i]; es[i] = 1; if (i + 1 < rank) st[i] = strides_bytes[i]; }
+    for (int i = 0; i < rank; ++i) { d[i] = dims[i]; b[i] = box[i]; es[i] = estr ? estr[i] : 1; if (i + 1 < rank) st[i] = strides_bytes[i]; }
     return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), d, st, b, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
-// activations [n_img][H][W][chan] as the tall map's source (channel, x, y, image), or flat (channel, pixel)
-static bool encode_act(CUtensorMap* m, const void* base, int chan, bool flat, long long pixels, int n_img, int H, int W, int Wp, int R) {
-    if (flat) {
-        const uint64_t dims[2] = {(uint64_t)chan, (uint64_t)pixels}; const uint64_t st[1] = {(uint64_t)chan * 2}; const uint32_t box[2] = {64, 128};
-        return encode_map(m, base, 2, dims, st, box);
-    }
+// [pixels][chan] as (channel, pixel), box 64 x 128
+static bool encode_flat(CUtensorMap* m, const void* base, int chan, long long pixels) {
+    const uint64_t dims[2] = {(uint64_t)chan, (uint64_t)pixels}; const uint64_t st[1] = {(uint64_t)chan * 2}; const uint32_t box[2] = {64, 128};
+    return encode_map(m, base, 2, dims, st, box);
+}
+// [n_img][H][W][chan] as (channel, x, y, image): a box is R rows of Wp window positions, every es-th pixel in x and y
+static bool encode_tall(CUtensorMap* m, const void* base, int chan, int n_img, int H, int W, int Wp, int R, int es) {
     const uint64_t dims[4] = {(uint64_t)chan, (uint64_t)W, (uint64_t)H, (uint64_t)n_img};
     const uint64_t st[3] = {(uint64_t)chan * 2, (uint64_t)chan * 2 * W, (uint64_t)chan * 2 * W * H};
-    const uint32_t box[4] = {64, (uint32_t)Wp, (uint32_t)R, 1};
-    return encode_map(m, base, 4, dims, st, box);
+    const uint32_t box[4] = {64, (uint32_t)(Wp * es), (uint32_t)(R * es), 1};
+    const uint32_t estr[4] = {1, (uint32_t)es, (uint32_t)es, 1};
+    return encode_map(m, base, 4, dims, st, box, estr);
 }
 
-// rows of the tall map fetched by one box: the largest divisor of Hp whose box holds at most 64 positions
-static int box_rows(int Hp, int Wp) { int best = 1; for (int r = 1; r <= Hp; ++r) if (Hp % r == 0 && r * Wp <= 64) best = r; return best; }
+// rows of the tall map fetched by one box: the largest divisor of Hp whose box holds at most 64 positions (and fits a TMA box)
+static int box_rows(int Hp, int Wp, int es) { int best = 1; for (int r = 1; r <= Hp; ++r) if (Hp % r == 0 && r * Wp <= 64 && r * es <= 256) best = r; return best; }
 
-struct TcGeom { int flat, chan_a, ncol, n_tile, tiles_n, tiles_m, slabs, Wp, Hp, R, box_pos, nbox, halo, a_box_bytes, a_stage, b_bytes, b_stage, n_img, H, W;
-                long long total_pos; };
+// The tall map of a grid of Hg x Wg positions per image
+struct Tall { int Hp, Wp, R, box_pos, box_bytes; };
+static bool tall_of(int Hg, int Wg, int pad, int es, Tall& t) {
+    t.Hp = Hg + pad; t.Wp = Wg + pad;
+    if (t.Wp * es > 256) return false;
+    t.R = box_rows(t.Hp, t.Wp, es); t.box_pos = t.R * t.Wp; t.box_bytes = t.box_pos * 128;
+    return true;
+}
+static int boxes_for(int span, int box_pos) { return (span + 2 * (box_pos - 1)) / box_pos; }   // boxes that cover `span` positions from any start
 
-// Decides whether (and how) the tensor-core kernel takes this problem.
-static bool tc_geometry(const ConvProb& p, int mode, TcGeom& g) {
-    if (mode == CONV_WGRAD) return false;
-    // A stride-2 forward layer is computed at stride 1 and only the even positions are stored; stride-2 dgrad
-    // arrives here as a stride-1 problem on a zero-stuffed dy (see zero_stuff_kernel).
-    if ((p.ksz != 1 && p.ksz != 3) || p.stride < 1 || p.stride > 2 || (p.stride == 2 && mode != CONV_FWD)) return false;
+// The taps of output phase (u, v) of a stride-2 3x3 dgrad (u, v = parity of the input row and column), or of input phase (u, v)
+// of a stride-2 3x3 forward / wgrad: tap (r, s) belongs to the phase with (r - 1) = u, (s - 1) = v modulo 2.
+static int phase_taps(int u, int v, int rs[4][2]) {
+    int n = 0;
+    for (int r = 0; r < 3; ++r) for (int s = 0; s < 3; ++s)
+        if ((((r - 1) % 2) + 2) % 2 == u && (((s - 1) % 2) + 2) % 2 == v) { rs[n][0] = r; rs[n][1] = s; ++n; }
+    return n;
+}
+
+static bool tc_shape_ok(const ConvProb& p) {
+    if ((p.ksz != 1 && p.ksz != 3) || p.stride < 1 || p.stride > 2) return false;
     if (p.C % 8 || p.K % 8) return false;
-    if (((uintptr_t)p.act | (uintptr_t)p.wgt | (uintptr_t)p.out | (uintptr_t)p.add) & 15) return false;
-    g.chan_a = mode == CONV_FWD ? p.C : p.K;            // reduction channels
-    g.ncol = mode == CONV_FWD ? p.K : p.C;              // output channels
-    g.flat = p.ksz == 1 && p.stride == 1;
-    g.n_img = p.N; g.H = p.H; g.W = p.W;
-    if (g.flat) { g.total_pos = (long long)p.N * p.H * p.W; g.Wp = 0; g.Hp = 0; g.R = 0; g.box_pos = 128; g.nbox = 1; g.halo = 0; g.a_box_bytes = 128 * 128; }
-    else {
-        g.Wp = p.W + 1; g.Hp = p.H + 1; if (g.Wp > 256) return false;
-        g.total_pos = (long long)p.N * g.Hp * g.Wp;
-        g.R = box_rows(g.Hp, g.Wp); g.box_pos = g.R * g.Wp; g.halo = p.ksz == 3 ? g.Wp + 1 : 0;
-        g.nbox = (TILE_M + 2 * g.halo + g.box_pos - 1 + g.box_pos - 1) / g.box_pos;
-        g.a_box_bytes = g.box_pos * 128;
-    }
-    if (g.total_pos > (1ll << 30)) return false;
-    g.tiles_m = (int)((g.total_pos + TILE_M - 1) / TILE_M);
-    g.tiles_n = (g.ncol + 255) / 256;
-    g.n_tile = (((g.ncol + g.tiles_n - 1) / g.tiles_n) + 15) / 16 * 16;
-    g.slabs = (g.chan_a + 63) / 64;
-    g.a_stage = (g.nbox * g.a_box_bytes + 1023) / 1024 * 1024;
-    g.b_bytes = mode == CONV_FWD ? g.n_tile * 128 : ((g.n_tile + 63) / 64) * 8192;
-    g.b_stage = (g.b_bytes + 1023) / 1024 * 1024;
+    if ((long long)p.N * (p.H + 1) * (p.W + 1) > (1ll << 30)) return false;
     return true;
 }
 
-bool conv_tc_supported(const ConvProb& p, int mode) { TcGeom g; return encode_fn() != nullptr && tc_geometry(p, mode, g); }
+// Number of TcProb descriptors a forward / dgrad problem needs (0: not supported): one, or one per output phase of a stride-2 3x3 dgrad.
+int conv_tc_count(const ConvProb& p, int mode) {
+    if (mode == CONV_WGRAD || !encode_fn() || !tc_shape_ok(p)) return 0;
+    if (((uintptr_t)p.act | (uintptr_t)p.wgt | (uintptr_t)p.out | (uintptr_t)p.add) & 15) return 0;
+    Tall t;
+    if (p.ksz == 3 && !tall_of(p.stride == 2 ? p.P : p.H, p.stride == 2 ? p.Q : p.W, 1, mode == CONV_FWD ? p.stride : 1, t)) return 0;
+    if (p.ksz == 1 && p.stride == 2 && mode == CONV_FWD && !tall_of(p.P, p.Q, 0, 2, t)) return 0;
+    return (mode == CONV_DGRAD && p.ksz == 3 && p.stride == 2) ? 4 : 1;
+}
+bool conv_tc_supported(const ConvProb& p, int mode) { return conv_tc_count(p, mode) > 0; }
+// 128-position tiles of a forward problem (the rows of ConvProb::stat_tiles)
+int conv_tc_stat_tiles(const ConvProb& p) {
+    long long pos;
+    if (p.ksz == 1) pos = (long long)p.N * p.P * p.Q;
+    else pos = (long long)p.N * (p.P + 1) * (p.Q + 1);
+    return (int)((pos + TILE_M - 1) / TILE_M);
+}
 
 static int* g_status = nullptr;      // one status word per process, zeroed at creation
 int* conv_tc_status_word() {
@@ -589,47 +745,116 @@ int conv_tc_read_status() {
     return v;
 }
 
-// Fills a host-side TcProb for this problem.  Returns false when the problem is not supported.
-bool conv_tc_fill(const ConvProb& p, int mode, void* host_tc) {
-    TcGeom g; if (!tc_geometry(p, mode, g)) return false;
-    TcProb t; memset(&t, 0, sizeof(t));
+// Fills conv_tc_count() host-side TcProbs for this problem.  Returns the number written (0: not supported or encoding failed).
+int conv_tc_fill(const ConvProb& p, int mode, void* host_tc) {
+    const int count = conv_tc_count(p, mode);
+    if (!count) return 0;
     const int taps = p.ksz * p.ksz;
-    if (!encode_act(&t.map_a, p.act, g.chan_a, g.flat != 0, g.total_pos, g.n_img, g.H, g.W, g.Wp, g.R)) return false;
-    // weights [K][taps][C] viewed as (C, tap, K).  Forward: a tile is n_tile output channels (rows) x 64 input channels.
-    // dgrad: a block is 64 reduction channels k (rows) x 64 output columns c.
-    { const uint64_t dims[3] = {(uint64_t)p.C, (uint64_t)taps, (uint64_t)p.K};
-      const uint64_t st[2] = {(uint64_t)p.C * 2, (uint64_t)taps * p.C * 2};
-      const uint32_t box[3] = {64, 1, mode == CONV_FWD ? (uint32_t)g.n_tile : 64u};
-      if (!encode_map(&t.map_b, p.wgt, 3, dims, st, box)) return false; }
-    t.add = (const __nv_bfloat16*)p.add; t.out = (__nv_bfloat16*)p.out; t.status = conv_tc_status_word();
-    t.flat = g.flat; t.taps = taps; t.ksz = p.ksz; t.flip = mode == CONV_DGRAD ? 1 : 0;
-    t.H = g.H; t.W = g.W; t.Wp = g.Wp; t.Hp = g.Hp; t.n_img = g.n_img;
-    t.R = g.R; t.box_pos = g.box_pos; t.nbox = g.nbox; t.halo = g.halo; t.a_box_bytes = g.a_box_bytes;
-    t.tiles_m = g.tiles_m; t.tiles_n = g.tiles_n; t.n_tile = g.n_tile; t.ncol = g.ncol;
-    t.red = g.chan_a; t.slabs = g.slabs; t.b_mn_major = mode == CONV_DGRAD ? 1 : 0; t.b_bytes = g.b_bytes;
-    t.total_pos = g.total_pos; t.scale = p.scale;
-    t.os = (mode == CONV_FWD) ? p.stride : 1; t.P = p.P; t.Q = p.Q;
-    memcpy(host_tc, &t, sizeof(t));
-    return true;
+    const int chan_a = mode == CONV_FWD ? p.C : p.K, ncol = mode == CONV_FWD ? p.K : p.C;
+    for (int ph = 0; ph < count; ++ph) {
+        TcProb t; memset(&t, 0, sizeof(t));
+        t.add = (const __nv_bfloat16*)p.add; t.out = (__nv_bfloat16*)p.out; t.status = conv_tc_status_word();
+        t.stat_tiles = mode == CONV_FWD ? p.stat_tiles : nullptr;
+        t.n_img = p.N; t.ncol = ncol; t.red = chan_a; t.slabs = (chan_a + 63) / 64; t.scale = p.scale;
+        t.b_mn_major = mode == CONV_DGRAD ? 1 : 0;
+        t.es = 1; t.pad = 0; t.os = 1; t.oy = 0; t.ox = 0; t.ngroups = 1; t.gbeg[0] = 0;
+        const void* act = p.act;
+        long long out_pixels = 0;
+        if (p.ksz == 1 && (p.stride == 1 || mode == CONV_DGRAD)) {
+            // plain GEMM over the pixels of the operand: forward at stride 1, dgrad at either stride (stride 2: over the P x Q pixels of dy)
+            const int Hg = mode == CONV_DGRAD ? p.P : p.H, Wg = mode == CONV_DGRAD ? p.Q : p.W;
+            t.a_flat = 1; t.Hp = Hg; t.Wp = Wg; t.R = 0; t.box_pos = TILE_M; t.nbox = 1; t.hb = 0; t.a_box_bytes = SLAB_BYTES;
+            t.total_pos = p.N * Hg * Wg;
+            t.taps[0] = TapRef{0, 0}; t.gbeg[1] = 1;
+            if (!encode_flat(&t.map_a, act, chan_a, t.total_pos)) return 0;
+            if (p.stride == 2 && !p.out_compact) { t.dense = 0; t.OH = p.H; t.OW = p.W; t.os = 2; out_pixels = (long long)p.N * p.H * p.W; }   // scattered to the even positions
+            else { t.dense = 1; t.OH = Hg; t.OW = Wg; out_pixels = t.total_pos; }
+        } else if (p.ksz == 1) {
+            // forward of a stride-2 1x1 layer: the positions are the output pixels, the window gathers every second input pixel
+            Tall g; if (!tall_of(p.P, p.Q, 0, 2, g)) return 0;
+            t.a_flat = 0; t.dense = 1; t.es = 2; t.Hp = g.Hp; t.Wp = g.Wp; t.R = g.R; t.box_pos = g.box_pos; t.a_box_bytes = g.box_bytes; t.hb = 0;
+            t.nbox = boxes_for(TILE_M, g.box_pos); t.total_pos = p.N * g.Hp * g.Wp; t.OH = p.P; t.OW = p.Q; out_pixels = t.total_pos;
+            t.taps[0] = TapRef{0, 0}; t.gbeg[1] = 1;
+            if (!encode_tall(&t.map_a, act, chan_a, p.N, p.H, p.W, g.Wp, g.R, 2)) return 0;
+        } else if (p.stride == 1) {
+            // 3x3 at stride 1: one window, nine taps; dgrad walks the taps mirrored
+            Tall g; if (!tall_of(p.H, p.W, 1, 1, g)) return 0;
+            t.a_flat = 0; t.dense = 0; t.pad = 1; t.Hp = g.Hp; t.Wp = g.Wp; t.R = g.R; t.box_pos = g.box_pos; t.a_box_bytes = g.box_bytes; t.hb = g.Wp + 1;
+            t.nbox = boxes_for(TILE_M + 2 * t.hb, g.box_pos); t.total_pos = p.N * g.Hp * g.Wp; t.OH = p.H; t.OW = p.W; out_pixels = (long long)p.N * p.H * p.W;
+            for (int w = 0; w < 9; ++w) t.taps[w] = TapRef{mode == CONV_DGRAD ? 8 - w : w, (w / 3) * g.Wp + (w % 3)};
+            t.gbeg[1] = 9;
+            if (!encode_tall(&t.map_a, act, chan_a, p.N, p.H, p.W, g.Wp, g.R, 1)) return 0;
+        } else if (mode == CONV_FWD) {
+            // 3x3 at stride 2, forward: positions over the P x Q outputs, one window per input parity phase (element-strided fetch)
+            Tall g; if (!tall_of(p.P, p.Q, 1, 2, g)) return 0;
+            t.a_flat = 0; t.dense = 0; t.pad = 1; t.es = 2; t.Hp = g.Hp; t.Wp = g.Wp; t.R = g.R; t.box_pos = g.box_pos; t.a_box_bytes = g.box_bytes; t.hb = g.Wp + 1;
+            t.nbox = boxes_for(TILE_M + t.hb, g.box_pos); t.total_pos = p.N * g.Hp * g.Wp; t.OH = p.P; t.OW = p.Q; out_pixels = (long long)p.N * p.P * p.Q;
+            int n = 0; t.ngroups = 0;
+            for (int u = 0; u < 2; ++u) for (int v = 0; v < 2; ++v) {
+                int rs[4][2]; const int k = phase_taps(u, v, rs);
+                t.gxs[t.ngroups] = v; t.gys[t.ngroups] = u;
+                for (int i = 0; i < k; ++i) {
+                    const int di = rs[i][0] == 0 ? -1 : 0, dj = rs[i][1] == 0 ? -1 : 0;    // tap 0 reads the previous phase row / column
+                    t.taps[n++] = TapRef{rs[i][0] * 3 + rs[i][1], t.hb + di * g.Wp + dj};
+                }
+                t.gbeg[++t.ngroups] = n;
+            }
+            if (!encode_tall(&t.map_a, act, chan_a, p.N, p.H, p.W, g.Wp, g.R, 2)) return 0;
+        } else {
+            // 3x3 at stride 2, dgrad: one problem per output parity phase (u, v), positions over the P x Q grid of dy; input row 2i + u
+            // takes dy row i + (u + 1 - r) / 2 through tap r
+            const int u = ph >> 1, v = ph & 1;
+            Tall g; if (!tall_of(p.P, p.Q, 1, 1, g)) return 0;
+            t.a_flat = 0; t.dense = 0; t.pad = 1; t.Hp = g.Hp; t.Wp = g.Wp; t.R = g.R; t.box_pos = g.box_pos; t.a_box_bytes = g.box_bytes; t.hb = 0;
+            t.nbox = boxes_for(TILE_M + g.Wp + 1, g.box_pos); t.total_pos = p.N * g.Hp * g.Wp;
+            t.OH = p.H; t.OW = p.W; t.os = 2; t.oy = u; t.ox = v; out_pixels = (long long)p.N * p.H * p.W;
+            int rs[4][2]; const int k = phase_taps(u, v, rs);
+            for (int i = 0; i < k; ++i) t.taps[i] = TapRef{rs[i][0] * 3 + rs[i][1], ((u + 1 - rs[i][0]) / 2) * g.Wp + (v + 1 - rs[i][1]) / 2};
+            t.gbeg[1] = k;
+            if (!encode_tall(&t.map_a, act, chan_a, p.N, p.P, p.Q, g.Wp, g.R, 1)) return 0;
+        }
+        // residual
+        t.add_mode = !p.add ? 0 : p.add_sub == 2 ? 3 : t.dense ? 1 : 2;
+        // output tiles: up to 256 columns (128 with a prefetched residual: two staging tiles), a multiple of 64 when there are several
+        const int n_cap = t.add_mode == 1 ? 128 : 256;
+        t.tiles_n = (ncol + n_cap - 1) / n_cap;
+        t.n_tile = (ncol + t.tiles_n - 1) / t.tiles_n;
+        t.n_tile = t.tiles_n > 1 ? (t.n_tile + 63) / 64 * 64 : (t.n_tile + 15) / 16 * 16;
+        t.tiles_n = (ncol + t.n_tile - 1) / t.n_tile;
+        t.out_slabs = (t.n_tile + 63) / 64;
+        t.tiles_m = (t.total_pos + TILE_M - 1) / TILE_M;
+        t.b_bytes = mode == CONV_FWD ? t.n_tile * 128 : ((t.n_tile + 63) / 64) * 8192;
+        // weights [K][taps][C] viewed as (C, tap, K).  Forward: a tile is n_tile output channels (rows) x 64 input channels.
+        // dgrad: a block is 64 reduction channels k (rows) x 64 output columns c.
+        { const uint64_t dims[3] = {(uint64_t)p.C, (uint64_t)taps, (uint64_t)p.K};
+          const uint64_t st[2] = {(uint64_t)p.C * 2, (uint64_t)taps * p.C * 2};
+          const uint32_t box[3] = {64, 1, mode == CONV_FWD ? (uint32_t)t.n_tile : 64u};
+          if (!encode_map(&t.map_b, p.wgt, 3, dims, st, box)) return 0; }
+        if (t.dense) {
+            if (!encode_flat(&t.map_out, p.out, ncol, out_pixels)) return 0;
+            if (t.add_mode == 1 && !encode_flat(&t.map_add, p.add, ncol, out_pixels)) return 0;
+        }
+        memcpy((char*)host_tc + (size_t)ph * sizeof(TcProb), &t, sizeof(t));
+    }
+    return count;
 }
 size_t conv_tc_prob_bytes() { return sizeof(TcProb); }
 int conv_tc_tiles(const void* host_tc) { const TcProb* t = (const TcProb*)host_tc; return t->tiles_m * t->tiles_n; }
-// packs what a launch has to know about its largest problem into one number: window bytes, weight-tile bytes, MMA N
+// packs what a launch has to know about its largest problem into one number: window KB, weight-tile KB, staging tiles, MMA N
 size_t conv_tc_smem(const void* host_tc) {
     const TcProb* t = (const TcProb*)host_tc;
     const size_t a_stage = ((size_t)t->nbox * t->a_box_bytes + 1023) / 1024, b_stage = ((size_t)t->b_bytes + 1023) / 1024;
-    return (a_stage << 40) | (b_stage << 20) | (size_t)t->n_tile;
+    return (a_stage << 48) | (b_stage << 32) | ((size_t)(t->add_mode == 1 ? 2 : 1) << 24) | (size_t)t->n_tile;
 }
-
 // field-wise maximum of two packed values
 size_t conv_tc_merge(size_t a, size_t b) {
-    const size_t m20 = 0xFFFFF;
-    return (std::max(a >> 40, b >> 40) << 40) | (std::max((a >> 20) & m20, (b >> 20) & m20) << 20) | std::max(a & m20, b & m20);
+    return (std::max(a >> 48, b >> 48) << 48) | (std::max((a >> 32) & 0xFFFF, (b >> 32) & 0xFFFF) << 32) |
+           (std::max((a >> 24) & 0xFF, (b >> 24) & 0xFF) << 24) | std::max(a & 0xFFFFFF, b & 0xFFFFFF);
 }
 
 constexpr size_t TC_SMEM_BUDGET = 200 * 1024;
 
-// total_tiles: tiles of all problems of the launch; packed: the largest conv_tc_smem() value of its problems (fields are maxima)
+// total_tiles: an upper bound of the tiles of all problems of the launch (max_tiles * nprob); packed: conv_tc_merge over its problems
 void launch_conv_tc_probs(const void* d_tc, int nprob, int max_tiles, size_t packed, cudaStream_t s) {
     static bool configured = false; static int sms = 0;
     if (!configured) {
@@ -639,67 +864,94 @@ void launch_conv_tc_probs(const void* d_tc, int nprob, int max_tiles, size_t pac
     }
     TcLaunch L{};
     L.nprob = nprob;
-    L.a_stage = (int)(packed >> 40) * 1024; L.b_stage = (int)((packed >> 20) & 0xFFFFF) * 1024;
-    const int n_tile = (int)(packed & 0xFFFFF);
+    L.a_stage = (int)(packed >> 48) * 1024; L.b_stage = (int)((packed >> 32) & 0xFFFF) * 1024;
+    L.n_stg = (int)((packed >> 24) & 0xFF);
+    const int n_tile = (int)(packed & 0xFFFFFF);
+    L.stg_bytes = ((n_tile + 63) / 64) * SLAB_BYTES;
+    const size_t rings = TC_SMEM_BUDGET - (size_t)L.n_stg * L.stg_bytes;
     // ring depths: up to 4 windows and up to 6 weight tiles within the budget, at least 2 of each
     L.na = 2; L.nb = 2;
     while (true) {
         bool grown = false;
-        if (L.nb < TC_MAX_STAGES && (size_t)L.na * L.a_stage + (size_t)(L.nb + 1) * L.b_stage <= TC_SMEM_BUDGET) { ++L.nb; grown = true; }
-        if (L.na < 4 && (size_t)(L.na + 1) * L.a_stage + (size_t)L.nb * L.b_stage <= TC_SMEM_BUDGET) { ++L.na; grown = true; }
+        if (L.nb < TC_MAX_STAGES && (size_t)L.na * L.a_stage + (size_t)(L.nb + 1) * L.b_stage <= rings) { ++L.nb; grown = true; }
+        if (L.na < 4 && (size_t)(L.na + 1) * L.a_stage + (size_t)L.nb * L.b_stage <= rings) { ++L.na; grown = true; }
         if (!grown) break;
     }
     L.acc_stride = (n_tile + 31) / 32 * 32;
     L.tmem_cols = 32; while (L.tmem_cols < 2 * L.acc_stride) L.tmem_cols *= 2;
     // at least 120 KB of shared memory so that two CTAs that allocate tensor memory never share an SM
-    const size_t smem = std::max((size_t)L.na * L.a_stage + (size_t)L.nb * L.b_stage, (size_t)120 * 1024) + 1024;
-    const int total = max_tiles * nprob;
-    const int grid = std::max(1, std::min(total, sms));
+    const size_t smem = std::max((size_t)L.na * L.a_stage + (size_t)L.nb * L.b_stage + (size_t)L.n_stg * L.stg_bytes, (size_t)120 * 1024) + 1024;
+    const long long total = (long long)max_tiles * nprob;
+    const int grid = (int)std::max(1ll, std::min(total, (long long)sms));
     conv_tc_kernel<<<grid, TC_THREADS, smem, s>>>((const TcProb*)d_tc, L);
 }
 
 // ---- wgrad host side
-struct WgGeom { int flat, n_img, H, W, Wp, Hp, R, box_pos, nbox_dy, nbox_a, halo, box_bytes, chunks, m_tiles, n_tile, n_tiles, a_slabs, tap_groups, taps_per_group,
-                splits, chunks_per_split, dy_slab, a_slab, stage_bytes, stages, tmem_cols; size_t smem, partial_bytes; };
+struct WgGeom { TcWgradProb t; size_t smem, partial_bytes; };
 
-static bool wg_geometry(const ConvProb& p, int target_ctas, WgGeom& g) {
-    if (p.stride != 1 || (p.ksz != 1 && p.ksz != 3)) return false;
-    if (p.C % 8 || p.K % 8) return false;
+static bool wg_geometry(const ConvProb& p, int target_ctas, WgGeom& w) {
+    if (!tc_shape_ok(p)) return false;
     if (((uintptr_t)p.act | (uintptr_t)p.wgt) & 15) return false;
+    TcWgradProb& t = w.t; memset(&t, 0, sizeof(t));
     const int taps = p.ksz * p.ksz;
-    g.flat = p.ksz == 1;                 // (a stride-2 1x1 layer arrives with stride 1 and a zero-stuffed dy: still flat)
-    g.n_img = p.N; g.H = p.H; g.W = p.W;
+    t.taps = taps; t.n_img = p.N; t.cout = p.K; t.cin = p.C; t.es = 1; t.pad = 0;
     long long total_pos;
-    if (g.flat) { total_pos = (long long)p.N * p.H * p.W; g.Wp = 0; g.Hp = 0; g.R = 0; g.box_pos = 128; g.nbox_dy = 1; g.nbox_a = 1; g.halo = 0; g.box_bytes = 128 * 128; }
-    else {
-        g.Wp = p.W + 1; g.Hp = p.H + 1; if (g.Wp > 256) return false;
+    if (p.ksz == 1 && p.stride == 1) {
+        t.dy_flat = 1; t.a_flat = 1; t.Hp = p.H; t.Wp = p.W; t.box_pos = TILE_M; t.nbox_dy = 1; t.nbox_a = 1; t.hb = 0;
+        t.dy_box_bytes = SLAB_BYTES; t.a_box_bytes = SLAB_BYTES; total_pos = (long long)p.N * p.H * p.W;
+        t.tap_groups = 1; t.gbeg[1] = 1; t.tap[0] = TapRef{0, 0};
+    } else if (p.ksz == 1) {
+        // stride-2 1x1: the positions are the P x Q pixels of dy in order; a is gathered at every second pixel
+        Tall g; if (!tall_of(p.P, p.Q, 0, 2, g)) return false;
+        t.dy_flat = 1; t.a_flat = 0; t.es = 2; t.Hp = g.Hp; t.Wp = g.Wp; t.R = g.R; t.box_pos = g.box_pos; t.hb = 0;
+        t.nbox_dy = 1; t.dy_box_bytes = SLAB_BYTES; t.nbox_a = boxes_for(TILE_M, g.box_pos); t.a_box_bytes = g.box_bytes;
         total_pos = (long long)p.N * g.Hp * g.Wp;
-        g.R = box_rows(g.Hp, g.Wp); g.box_pos = g.R * g.Wp; g.halo = g.Wp + 1; g.box_bytes = g.box_pos * 128;
-        g.nbox_dy = (TILE_M + g.box_pos - 1 + g.box_pos - 1) / g.box_pos;
-        g.nbox_a = (TILE_M + 2 * g.halo + g.box_pos - 1 + g.box_pos - 1) / g.box_pos;
+        t.tap_groups = 1; t.gbeg[1] = 1; t.tap[0] = TapRef{0, 0};
+    } else if (p.stride == 1) {
+        Tall g; if (!tall_of(p.H, p.W, 1, 1, g)) return false;
+        t.dy_flat = 0; t.a_flat = 0; t.pad = 1; t.Hp = g.Hp; t.Wp = g.Wp; t.R = g.R; t.box_pos = g.box_pos; t.hb = g.Wp + 1;
+        t.nbox_dy = boxes_for(TILE_M, g.box_pos); t.nbox_a = boxes_for(TILE_M + 2 * t.hb, g.box_pos); t.dy_box_bytes = g.box_bytes; t.a_box_bytes = g.box_bytes;
+        total_pos = (long long)p.N * g.Hp * g.Wp;
+        for (int i = 0; i < 9; ++i) t.tap[i] = TapRef{i, (i / 3) * g.Wp + (i % 3)};
+        t.tap_groups = 0;                                // groups of up to three taps: set below, once the column tile is known
+    } else {
+        Tall g; if (!tall_of(p.P, p.Q, 1, 2, g)) return false;
+        Tall gd; if (!tall_of(p.P, p.Q, 1, 1, gd)) return false;
+        if (gd.R != g.R) { g.R = gd.R = 1; g.box_pos = gd.box_pos = g.Wp; g.box_bytes = gd.box_bytes = g.Wp * 128; }   // both operands use the same boxes of rows
+        t.dy_flat = 0; t.a_flat = 0; t.pad = 1; t.es = 2; t.Hp = g.Hp; t.Wp = g.Wp; t.R = g.R; t.box_pos = g.box_pos; t.hb = g.Wp + 1;
+        t.nbox_dy = boxes_for(TILE_M, g.box_pos); t.nbox_a = boxes_for(TILE_M + t.hb, g.box_pos); t.dy_box_bytes = g.box_bytes; t.a_box_bytes = g.box_bytes;
+        total_pos = (long long)p.N * g.Hp * g.Wp;
+        int n = 0; t.tap_groups = 0;
+        for (int u = 0; u < 2; ++u) for (int v = 0; v < 2; ++v) {
+            int rs[4][2]; const int k = phase_taps(u, v, rs);
+            t.gxs[t.tap_groups] = v; t.gys[t.tap_groups] = u;
+            for (int i = 0; i < k; ++i) t.tap[n++] = TapRef{rs[i][0] * 3 + rs[i][1], t.hb + (rs[i][0] == 0 ? -1 : 0) * g.Wp + (rs[i][1] == 0 ? -1 : 0)};
+            t.gbeg[++t.tap_groups] = n;
+        }
     }
-    if (total_pos > (1ll << 30)) return false;
-    g.chunks = (int)((total_pos + TILE_M - 1) / TILE_M);
-    g.m_tiles = (p.K + 127) / 128;
-    // columns of one CTA: the input channels in tiles of at most 256 (1x1) or 128 (3x3, three taps per CTA), tap groups within 512 columns of tensor memory
+    t.chunks = (int)((total_pos + TILE_M - 1) / TILE_M);
+    t.m_tiles = (p.K + 127) / 128;
+    // columns of one CTA: the input channels in tiles of at most 256 (1x1) or 128 (3x3: up to four taps in 512 columns of tensor memory)
     const int n_cap = taps == 1 ? 256 : 128;
-    g.n_tiles = (p.C + n_cap - 1) / n_cap;
-    g.n_tile = (((p.C + g.n_tiles - 1) / g.n_tiles) + 15) / 16 * 16;
-    g.a_slabs = (g.n_tile + 63) / 64;
-    g.taps_per_group = taps == 1 ? 1 : std::min(3, 512 / g.n_tile);
-    g.tap_groups = (taps + g.taps_per_group - 1) / g.taps_per_group;
-    g.tmem_cols = 32; while (g.tmem_cols < g.taps_per_group * g.n_tile) g.tmem_cols *= 2;
-    if (g.tmem_cols > 512) return false;
-    g.dy_slab = (g.nbox_dy * g.box_bytes + 1023) / 1024 * 1024;
-    g.a_slab = (g.nbox_a * g.box_bytes + 1023) / 1024 * 1024;
-    g.stage_bytes = 2 * g.dy_slab + g.a_slabs * g.a_slab;
-    g.stages = TC_MAX_STAGES; while (g.stages > 1 && (size_t)g.stages * g.stage_bytes > TC_SMEM_BUDGET) --g.stages;
-    if ((size_t)g.stages * g.stage_bytes > TC_SMEM_BUDGET) return false;
-    g.smem = std::max((size_t)g.stages * g.stage_bytes, (size_t)120 * 1024) + 1024;
-    const int fixed = g.m_tiles * g.n_tiles * g.tap_groups;
-    int want = std::max(1, target_ctas / fixed); if (want > g.chunks) want = g.chunks; if (want > 256) want = 256;
-    g.chunks_per_split = (g.chunks + want - 1) / want; g.splits = (g.chunks + g.chunks_per_split - 1) / g.chunks_per_split;
-    g.partial_bytes = g.splits > 1 ? (size_t)g.splits * taps * p.K * p.C * 4 : 0;
+    t.n_tiles = (p.C + n_cap - 1) / n_cap;
+    t.n_tile = (p.C + t.n_tiles - 1) / t.n_tiles;
+    t.n_tile = t.n_tiles > 1 ? (t.n_tile + 63) / 64 * 64 : (t.n_tile + 15) / 16 * 16;
+    t.n_tiles = (p.C + t.n_tile - 1) / t.n_tile;
+    t.a_slabs = (t.n_tile + 63) / 64;
+    if (taps == 9 && p.stride == 1) { for (int g = 0; g < 3; ++g) { t.gbeg[g + 1] = 3 * (g + 1); t.gxs[g] = 0; t.gys[g] = 0; } t.tap_groups = 3; }
+    int max_group = 0; for (int g = 0; g < t.tap_groups; ++g) max_group = std::max(max_group, t.gbeg[g + 1] - t.gbeg[g]);
+    t.tmem_cols = 32; while (t.tmem_cols < max_group * t.n_tile) t.tmem_cols *= 2;
+    if (t.tmem_cols > 512) return false;
+    t.dy_slab_bytes = (t.nbox_dy * t.dy_box_bytes + 1023) / 1024 * 1024;
+    t.a_slab_bytes = (t.nbox_a * t.a_box_bytes + 1023) / 1024 * 1024;
+    t.stage_bytes = 2 * t.dy_slab_bytes + t.a_slabs * t.a_slab_bytes;
+    t.stages = TC_MAX_STAGES; while (t.stages > 1 && (size_t)t.stages * t.stage_bytes > TC_SMEM_BUDGET) --t.stages;
+    if ((size_t)t.stages * t.stage_bytes > TC_SMEM_BUDGET) return false;
+    w.smem = std::max((size_t)t.stages * t.stage_bytes, (size_t)120 * 1024) + 1024;
+    const int fixed = t.m_tiles * t.n_tiles * t.tap_groups;
+    int want = std::max(1, target_ctas / fixed); if (want > t.chunks) want = t.chunks; if (want > 256) want = 256;
+    t.chunks_per_split = (t.chunks + want - 1) / want; t.splits = (t.chunks + t.chunks_per_split - 1) / t.chunks_per_split;
+    w.partial_bytes = t.splits > 1 ? (size_t)t.splits * taps * p.K * p.C * 4 : 0;
     return true;
 }
 
@@ -712,17 +964,12 @@ bool conv_wgrad_tc_supported(const ConvProb& p, int target_ctas, size_t* partial
 // p.act = a, p.wgt = dy, p.out = dw (fp32), p.partial = workspace of at least partial_bytes
 bool conv_wgrad_tc_fill(const ConvProb& p, int target_ctas, void* host_tc) {
     WgGeom g; if (!wg_geometry(p, target_ctas, g)) return false;
-    TcWgradProb t; memset(&t, 0, sizeof(t));
-    const long long pixels = (long long)p.N * p.H * p.W;
-    if (!encode_act(&t.map_dy, p.wgt, p.K, g.flat != 0, pixels, g.n_img, g.H, g.W, g.Wp, g.R)) return false;
-    if (!encode_act(&t.map_a, p.act, p.C, g.flat != 0, pixels, g.n_img, g.H, g.W, g.Wp, g.R)) return false;
+    TcWgradProb& t = g.t;
+    if (t.dy_flat) { if (!encode_flat(&t.map_dy, p.wgt, p.K, (long long)p.N * p.P * p.Q)) return false; }
+    else if (!encode_tall(&t.map_dy, p.wgt, p.K, p.N, p.P, p.Q, t.Wp, t.R, 1)) return false;
+    if (t.a_flat) { if (!encode_flat(&t.map_a, p.act, p.C, (long long)p.N * p.H * p.W)) return false; }
+    else if (!encode_tall(&t.map_a, p.act, p.C, p.N, p.H, p.W, t.Wp, t.R, t.es)) return false;
     t.partial = p.partial; t.out = (float*)p.out; t.status = conv_tc_status_word();
-    t.flat = g.flat; t.taps = p.ksz * p.ksz; t.ksz = p.ksz;
-    t.H = g.H; t.W = g.W; t.Wp = g.Wp; t.Hp = g.Hp; t.n_img = g.n_img;
-    t.R = g.R; t.box_pos = g.box_pos; t.nbox_dy = g.nbox_dy; t.nbox_a = g.nbox_a; t.halo = g.halo; t.box_bytes = g.box_bytes;
-    t.chunks = g.chunks; t.cout = p.K; t.cin = p.C; t.m_tiles = g.m_tiles; t.n_tile = g.n_tile; t.n_tiles = g.n_tiles; t.a_slabs = g.a_slabs;
-    t.tap_groups = g.tap_groups; t.taps_per_group = g.taps_per_group; t.splits = g.splits; t.chunks_per_split = g.chunks_per_split;
-    t.dy_slab_bytes = g.dy_slab; t.a_slab_bytes = g.a_slab; t.stage_bytes = g.stage_bytes; t.stages = g.stages; t.tmem_cols = g.tmem_cols;
     memcpy(host_tc, &t, sizeof(t));
     return true;
 }

@@ -18,7 +18,6 @@ struct ConvProb {
     const void* add;      // optional tensor added to the result (shape of out), or nullptr
     void* out;            // fwd: y (T);        dgrad: da (T);        wgrad: dw (fp32, [K][ksz][ksz][C])
     float* partial;       // wgrad split-K workspace [splits][K*ksz*ksz*C], or nullptr
-    double* stat_partial; // fwd (tensor-core path): per-tile column sums for the next BN, or nullptr
     int N, H, W, C, K, ksz, stride, pad, P, Q;
     int M, Ncol, Kred;    // GEMM extents of this mode
     int tiles_m, tiles_n, splits, ktiles_per_split;
@@ -26,7 +25,9 @@ struct ConvProb {
     int wg_ld, wg_cols;   // wgrad of a 1x1 problem on an im2col'ed input: row stride and valid columns of dw (0: K x C dense)
     int dy_sub;           // backward of a stride-2 layer as a stride-1 problem: 2 = dy is stored compact [N,dy_P,dy_Q,K] and read as if
     int dy_P, dy_Q;       //   zero-stuffed to H x W (only even positions exist); 0 or 1 = dy is stored at the problem's resolution
-    int pad_;
+    int out_compact;      // dgrad of a stride-2 1x1 layer on tcgen05: out is [N,P,Q,C], the gradient at the even input positions (all others are zero)
+    int add_sub;          // 2: `add` is such a compact tensor [N,(H+1)/2,(W+1)/2,Ncol] and is added at the even positions of the H x W result only
+    float* stat_tiles;    // forward on tcgen05: per 128-position tile, the column sums and sums of squares of the stored output [tiles][2][K], or nullptr
 };
 
 // One batch-normalisation + ReLU problem over x [m, C] (forward or backward).

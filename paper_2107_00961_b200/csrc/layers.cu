@@ -7,7 +7,9 @@
 
 namespace resist {
 bool conv_tc_supported(const ConvProb& p, int mode);
-bool conv_tc_fill(const ConvProb& p, int mode, void* host_tc);
+int conv_tc_fill(const ConvProb& p, int mode, void* host_tc);
+int conv_tc_count(const ConvProb& p, int mode);
+size_t conv_tc_merge(size_t a, size_t b);
 size_t conv_tc_prob_bytes();
 int conv_tc_tiles(const void* host_tc);
 size_t conv_tc_smem(const void* host_tc);
@@ -75,13 +77,14 @@ extern "C" int resist_conv2d(int32_t mode, int32_t dtype, int32_t backend, const
         if (want_tc && conv_tc_supported(q, mode)) return 1;
         return 0;
     };
-    // backward of a stride-2 layer on tensor cores: stride-1 problem on a zero-stuffed dy
+    // backward of a stride-2 layer on the warp-MMA kernels: stride-1 problem on a zero-stuffed dy (the tcgen05 kernels take the
+    // stride-2 problem as it is)
     char* up = nullptr;
     if (stride == 2 && mode != CONV_FWD && K % 8 == 0) {
         ConvProb q = p; q.stride = 1; q.P = H; q.Q = W;
         if (mode == CONV_DGRAD) q.M = (int)rows_in; else q.Kred = (int)rows_in;
         size_t pb = 0;
-        if (pick(q, &pb) != 0) {
+        if (pick(q, &pb) == 2) {
             if (cudaMalloc(&up, (size_t)N * H * W * K * 2 + 256) != cudaSuccess) { g_layer_error = "cudaMalloc failed"; return RESIST_ENOMEM; }
             UpProb u{mode == CONV_DGRAD ? p.act : p.wgt, up + 256, N, H, W, K, p.P, p.Q};
             cudaMemcpyAsync(up, &u, sizeof(u), cudaMemcpyHostToDevice, st);
@@ -95,9 +98,11 @@ extern "C" int resist_conv2d(int32_t mode, int32_t dtype, int32_t backend, const
     if (used_backend) *used_backend = be;
     size_t scratch = 0;
     std::vector<char> hd;                                      // host copy of the kernel family's own descriptor
-    if (be == 1) hd.resize(mode == CONV_WGRAD ? conv_wgrad_tc_prob_bytes() : conv_tc_prob_bytes());
+    int n_tc = 1;
+    if (be == 1) { n_tc = mode == CONV_WGRAD ? 1 : conv_tc_count(p, mode); hd.resize(mode == CONV_WGRAD ? conv_wgrad_tc_prob_bytes() : (size_t)n_tc * conv_tc_prob_bytes()); }
     if (be == 2) hd.resize(mode == CONV_WGRAD ? conv_wgrad_mma_prob_bytes() : conv_mma_prob_bytes());
-    if (be && mode == CONV_WGRAD) scratch = 1024 + wg_partial; else if (be) scratch = 1024;
+    const size_t hd_room = (hd.size() + 255) / 256 * 256;
+    if (be && mode == CONV_WGRAD) scratch = hd_room + wg_partial; else if (be) scratch = hd_room;
     if (!be && mode == CONV_WGRAD) {
         const int tiles = p.tiles_m * p.tiles_n;
         int want = (2 * sm + tiles - 1) / tiles; want = std::max(1, std::min(std::min(want, 64), ktiles));
@@ -108,16 +113,26 @@ extern "C" int resist_conv2d(int32_t mode, int32_t dtype, int32_t backend, const
     cudaError_t e = cudaMalloc(&blob, 1024 + scratch);
     if (e != cudaSuccess) { cudaFree(up); g_layer_error = cudaGetErrorString(e); return RESIST_ENOMEM; }
     if (!be && p.splits > 1) p.partial = (float*)(blob + 1024);
-    if (be && mode == CONV_WGRAD) p.partial = (float*)(blob + 2048);
+    if (be && mode == CONV_WGRAD) p.partial = (float*)(blob + 1024 + hd_room);
     bool filled = true;
-    if (be == 1) filled = mode == CONV_WGRAD ? conv_wgrad_tc_fill(p, 2 * sm, hd.data()) : conv_tc_fill(p, mode, hd.data());
+    if (be == 1) filled = mode == CONV_WGRAD ? conv_wgrad_tc_fill(p, 2 * sm, hd.data()) : conv_tc_fill(p, mode, hd.data()) == n_tc;
+    // dgrad of a stride-2 1x1 layer on tcgen05 stores the even positions only: the rest of the gradient is zero
+    // (with a residual the rest is the residual itself)
+    if (be == 1 && mode == CONV_DGRAD && ksz == 1 && stride == 2) {
+        if (add) cudaMemcpyAsync(out, add, (size_t)rows_in * C * 2, cudaMemcpyDeviceToDevice, st);
+        else cudaMemsetAsync(out, 0, (size_t)rows_in * C * 2, st);
+    }
     if (be == 2) filled = mode == CONV_WGRAD ? conv_wgrad_mma_fill(p, 2 * sm, hd.data()) : conv_mma_fill(p, mode, hd.data());
     if (!filled) { cudaFree(blob); cudaFree(up); g_layer_error = "descriptor set-up failed"; return RESIST_ECUDA; }
     e = cudaMemcpyAsync(blob, &p, sizeof(p), cudaMemcpyHostToDevice, st);
     if (e == cudaSuccess && be) e = cudaMemcpyAsync(blob + 1024, hd.data(), hd.size(), cudaMemcpyHostToDevice, st);
     if (e == cudaSuccess) {
         if (be == 1 && mode == CONV_WGRAD) launch_conv_wgrad_tc_probs(blob + 1024, 1, conv_wgrad_tc_ctas(hd.data()), conv_wgrad_tc_smem(hd.data()), conv_wgrad_tc_out_elems(hd.data()), st);
-        else if (be == 1) launch_conv_tc_probs(blob + 1024, 1, conv_tc_tiles(hd.data()), conv_tc_smem(hd.data()), st);
+        else if (be == 1) {
+            int tiles = 0; size_t packed = 0;
+            for (int i = 0; i < n_tc; ++i) { const char* h = hd.data() + (size_t)i * conv_tc_prob_bytes(); tiles = std::max(tiles, conv_tc_tiles(h)); packed = conv_tc_merge(packed, conv_tc_smem(h)); }
+            launch_conv_tc_probs(blob + 1024, n_tc, tiles, packed, st);
+        }
         else if (be == 2 && mode == CONV_WGRAD) launch_conv_wgrad_mma_probs(blob + 1024, 1, conv_wgrad_mma_ctas(hd.data()), conv_wgrad_mma_smem(hd.data()), conv_wgrad_mma_out_elems(hd.data()), conv_wgrad_mma_pick_variant(p, 2 * sm), st);
         else if (be == 2) launch_conv_mma_probs(blob + 1024, 1, conv_mma_tiles(hd.data()), conv_mma_smem(hd.data()), conv_mma_pick_variant(p, mode), st);
         else {

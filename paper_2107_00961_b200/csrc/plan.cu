@@ -15,7 +15,10 @@ void held_segments(const resist_ctx* ctx, int sub, uint32_t bit, bool buffers, s
 int ensure_param_arrays(resist_ctx* ctx, int S);
 int ensure_seg_table(resist_ctx* ctx, int n);
 bool conv_tc_supported(const ConvProb& p, int mode);                                   // conv_tc.cu
-bool conv_tc_fill(const ConvProb& p, int mode, void* host_tc);
+int conv_tc_fill(const ConvProb& p, int mode, void* host_tc);
+int conv_tc_count(const ConvProb& p, int mode);
+int conv_tc_stat_tiles(const ConvProb& p);
+void launch_bn_finalize_tiles(const BnProb* d, int nprob, int max_c, cudaStream_t s);
 size_t conv_tc_prob_bytes();
 int conv_tc_tiles(const void* host_tc);
 size_t conv_tc_smem(const void* host_tc);
@@ -109,6 +112,7 @@ struct Builder {
     // The BN+ReLU that consumes a warp-MMA convolution's output joins that convolution's launch (forward: the BN of the
     // output; backward: the BN backward whose da the data gradient produces).  Index of the candidate in *ops, or -1.
     int last_fwd_conv = -1, last_dgrad = -1;
+    int last_tc_fwd = -1;     // the last forward convolution if it runs on tcgen05: its epilogue can leave the sums the BN of its output needs
     bool fusable(int idx, const void* tensor, const BnProb& p) const {
         if (idx < 0 || eval || ctx->opts.dtype != RESIST_BF16 || (ctx->opts.conv_backend != RESIST_CONV_AUTO && ctx->opts.conv_backend != RESIST_CONV_WARP_MMA)) return false;
         const Op& o = (*ops)[idx];
@@ -132,14 +136,16 @@ struct Builder {
         return W() + o;
     }
 
-    void conv(long long key, int mode, const void* a, const ConvRef& cr, const void* dy_or_null, const void* add, void* out,
-              int N, int H, int Wd, float scale, bool patch = false) {
+    // add_compact: `add` holds the gradient at the even positions only ([N,(H+1)/2,(W+1)/2,C], what a stride-2 projection's dgrad on
+    // tcgen05 leaves).  Returns whether THIS convolution's output is such a compact tensor.
+    bool conv(long long key, int mode, const void* a, const ConvRef& cr, const void* dy_or_null, const void* add, void* out,
+              int N, int H, int Wd, float scale, bool patch = false, bool add_compact = false) {
         Op op{}; op.key = key; op.sub = sub; op.patch_images = patch ? 1 : 0;
         op.kind = mode == CONV_FWD ? OP_CONV_FWD : mode == CONV_DGRAD ? OP_CONV_DGRAD : OP_CONV_WGRAD;
         ConvProb& p = op.conv;
         p.N = N; p.H = H; p.W = Wd; p.C = cr.cin; p.K = cr.cout; p.ksz = cr.k; p.stride = cr.stride; p.pad = (cr.k - 1) / 2;
         p.P = out_dim(H, cr.k, cr.stride); p.Q = out_dim(Wd, cr.k, cr.stride);
-        p.scale = scale; p.add = add; p.out = out; p.partial = nullptr; p.stat_partial = nullptr;
+        p.scale = scale; p.add = add; p.out = out; p.partial = nullptr;
         const long long rows_out = (long long)N * p.P * p.Q, rows_in = (long long)N * H * Wd;
         if (mode == CONV_FWD) { p.act = a; p.wgt = CW(cr.w); p.M = (int)rows_out; p.Ncol = p.K; p.Kred = p.ksz * p.ksz * p.C; }
         else if (mode == CONV_DGRAD) { p.act = dy_or_null; p.wgt = CW(cr.w); p.M = (int)rows_in; p.Ncol = p.C; p.Kred = p.ksz * p.ksz * p.K; }
@@ -150,30 +156,14 @@ struct Builder {
         const bool tc_ok = ctx->opts.dtype == RESIST_BF16 && ctx->opts.conv_backend != RESIST_CONV_CUDA_CORES;
         const int pref = ctx->opts.conv_backend;
         if (tc_ok && p.stride == 2 && mode != CONV_FWD && !patch && p.K % 8 == 0) {
-            // backward of a stride-2 layer: a stride-1 problem on dy zero-stuffed to the input resolution
-            ConvProb q = p; q.stride = 1; q.P = p.H; q.Q = p.W;
-            const size_t up_bytes = (size_t)N * p.H * p.W * p.K * 2;
-            if (mode == CONV_DGRAD) { q.act = up_buf; q.M = (int)rows_in; }
-            else { q.wgt = up_buf; q.Kred = (int)rows_in; }
+            // backward of a stride-2 layer on the warp-MMA kernels: a stride-1 problem that reads the compact dy through its pixel
+            // tables (odd positions are zero); the tcgen05 kernels take the stride-2 problem as it is
+            ConvProb q = p; q.stride = 1; q.P = p.H; q.Q = p.W; q.dy_sub = 2; q.dy_P = p.P; q.dy_Q = p.Q;
+            if (mode == CONV_DGRAD) q.M = (int)rows_in; else q.Kred = (int)rows_in;
             size_t pb = 0;
-            // warp-MMA kernels read the compact dy through their pixel tables (odd positions are zero): nothing is materialised
-            ConvProb q2 = q; q2.dy_sub = 2; q2.dy_P = p.P; q2.dy_Q = p.Q;
-            if (mode == CONV_DGRAD) q2.act = dy_or_null; else q2.wgt = dy_or_null;
-            if (pick_backend(q2, mode, wgrad_target_ctas(ctx), &pb, pref) >= 200) {
-                p = q2;
-                if (mode == CONV_WGRAD) wgrad_partial_need = std::max(wgrad_partial_need, pb);
-            } else {
-            const bool ok = pick_backend(q, mode, wgrad_target_ctas(ctx), &pb, pref) != 0;
-            if (ok) {
-                up_need = std::max(up_need, up_bytes);
-                if (up_src != dy_or_null) {                  // first use of this dy: stuff it
-                    Op u{}; u.key = key; u.sub = sub; u.kind = OP_UPSAMPLE;
-                    u.up = UpProb{dy_or_null, up_buf, N, p.H, p.W, p.K, p.P, p.Q};
-                    ops->push_back(u); up_src = dy_or_null;
-                }
+            if (pick_backend(q, mode, wgrad_target_ctas(ctx), &pb, pref) >= 200) {
                 p = q;
-                if (mode == CONV_WGRAD) { wgrad_partial_need = std::max(wgrad_partial_need, pb); }
-            }
+                if (mode == CONV_WGRAD) wgrad_partial_need = std::max(wgrad_partial_need, pb);
             }
         }
         if (mode == CONV_WGRAD) {
@@ -182,6 +172,17 @@ struct Builder {
             if (op.backend) { wgrad_partial_need = std::max(wgrad_partial_need, pb); p.partial = wgrad_partial; }
         } else op.backend = tc_ok ? pick_backend(p, mode, 0, nullptr, pref) : 0;
         if (op.backend) ++n_tc; else ++n_cc;
+        const bool out_compact = mode == CONV_DGRAD && op.backend == 1 && p.ksz == 1 && p.stride == 2;
+        if (out_compact) p.out_compact = 1;
+        if (add && add_compact) {
+            if (op.backend == 1 && mode == CONV_DGRAD) p.add_sub = 2;            // added at the even positions in the epilogue
+            else {                                                               // spread out to the full resolution first
+                up_need = std::max(up_need, (size_t)rows_in * p.C * 2);
+                Op u{}; u.key = key; u.sub = sub; u.kind = OP_UPSAMPLE;
+                u.up = UpProb{add, up_buf, N, H, Wd, p.C, (H + 1) / 2, (Wd + 1) / 2};
+                ops->push_back(u); p.add = up_buf;
+            }
+        }
         if (mode == CONV_WGRAD && !op.backend) {
             const int tiles = p.tiles_m * p.tiles_n;
             int want = (2 * ctx->sm_count + tiles - 1) / tiles; if (want > 64) want = 64; if (want > ktiles) want = ktiles; if (want < 1) want = 1;
@@ -192,9 +193,10 @@ struct Builder {
             }
         }
         ops->push_back(op);
-        if (mode == CONV_FWD) last_fwd_conv = op.backend >= 1000 ? (int)ops->size() - 1 : -1;
+        if (mode == CONV_FWD) { last_fwd_conv = op.backend >= 1000 ? (int)ops->size() - 1 : -1; last_tc_fwd = op.backend == 1 ? (int)ops->size() - 1 : -1; }
         if (mode == CONV_DGRAD) last_dgrad = op.backend >= 1000 ? (int)ops->size() - 1 : -1;
         if (mode == CONV_WGRAD && p.splits > 1) { Op r = op; r.key = key + 1; r.kind = OP_SPLITK; r.patch_images = 0; ops->push_back(r); }
+        return out_compact;
     }
     // the BN joins the launch of the convolution at *ops[idx]
     void fuse_into(int idx, const BnProb& p, int which) {
@@ -251,7 +253,18 @@ struct Builder {
         bn_partial_need = std::max(bn_partial_need, (size_t)p.chunks * 2 * r.c * 8);
         p.partial = bn_partial;
         const int producer = last_fwd_conv; last_fwd_conv = -1;
+        const int tc_producer = last_tc_fwd; last_tc_fwd = -1;
         if (fusable(producer, x, p)) { fuse_into(producer, p, 1); return stat; }                            // inside the producing convolution's launch
+        if (!eval && p.vec && tc_producer >= 0 && (*ops)[tc_producer].conv.out == x && (*ops)[tc_producer].conv.K == r.c) {
+            // the tcgen05 convolution that produces x leaves per-tile column sums: a small launch turns them into statistics, then one elementwise pass
+            ConvProb& c = (*ops)[tc_producer].conv;
+            const int tiles = conv_tc_stat_tiles(c);
+            bn_partial_need = std::max(bn_partial_need, (size_t)tiles * 2 * r.c * 4);
+            c.stat_tiles = (float*)bn_partial; p.partial = bn_partial; p.chunks = tiles;
+            op.kind = OP_BN_TILE_STATS; ops->push_back(op);
+            op.key = key + 1; op.kind = OP_BN_APPLY; ops->push_back(op);
+            return stat;
+        }
         if (p.vec && !eval && r.c <= 512) { op.kind = OP_BN_FWD_FUSED; ops->push_back(op); return stat; }   // one cooperative launch
         ops->push_back(op);
         op.key = key + 1; op.kind = OP_BN_APPLY; ops->push_back(op);
@@ -300,7 +313,7 @@ static size_t unroll_subnet(resist_ctx* ctx, Builder& bd, const std::vector<char
         stem_p = bd.act((long long)B * Hp * Wp * cC); stem_arg = (int*)bd.take((size_t)B * Hp * Wp * cC * 4);
         Op op{}; op.key = 3; op.sub = bd.sub; op.kind = OP_POOL_FWD;
         op.pool = PoolProb{cur, stem_p, stem_arg, nullptr, nullptr, B, cH, cW, cC, Hp, Wp};
-        bd.ops->push_back(op); bd.last_fwd_conv = -1;
+        bd.ops->push_back(op); bd.last_fwd_conv = -1; bd.last_tc_fwd = -1;
         cur = stem_p; cH = Hp; cW = Wp;
     }
 
@@ -379,11 +392,11 @@ static size_t unroll_subnet(resist_ctx* ctx, Builder& bd, const std::vector<char
         const long long m_in = (long long)B * s.H * s.W, m_out = (long long)B * s.Ho * s.Wo;
         const char* dout = bd.gbuf[g_cur];
         bd.up_src = nullptr;                                     // no zero-stuffed dy carries over from another block
-        int g_sc = -1;
+        int g_sc = -1; bool sc_compact = false;
         if (K.has_projection) {
             bd.conv(key + 0, CONV_WGRAD, s.a1, r.proj, dout, nullptr, nullptr, B, s.H, s.W, 1.f);
             g_sc = bd.gtake();
-            bd.conv(key + 2, CONV_DGRAD, nullptr, r.proj, dout, nullptr, bd.gbuf[g_sc], B, s.H, s.W, 1.f);
+            sc_compact = bd.conv(key + 2, CONV_DGRAD, nullptr, r.proj, dout, nullptr, bd.gbuf[g_sc], B, s.H, s.W, 1.f);
         }
         int g_da1 = -1;
         if (K.kind == RESIST_BASIC) {
@@ -395,7 +408,7 @@ static size_t unroll_subnet(resist_ctx* ctx, Builder& bd, const std::vector<char
             bd.grel(g_da2);
             bd.conv(key + 8, CONV_WGRAD, s.a1, r.conv[0], bd.gbuf[g_dy1], nullptr, nullptr, B, s.H, s.W, 1.f);
             g_da1 = bd.gtake();
-            bd.conv(key + 10, CONV_DGRAD, nullptr, r.conv[0], bd.gbuf[g_dy1], g_sc >= 0 ? bd.gbuf[g_sc] : nullptr, bd.gbuf[g_da1], B, s.H, s.W, 1.f);
+            bd.conv(key + 10, CONV_DGRAD, nullptr, r.conv[0], bd.gbuf[g_dy1], g_sc >= 0 ? bd.gbuf[g_sc] : nullptr, bd.gbuf[g_da1], B, s.H, s.W, 1.f, false, sc_compact);
             bd.grel(g_dy1);
         } else {
             const int g_da3 = bd.gtake();
@@ -413,7 +426,7 @@ static size_t unroll_subnet(resist_ctx* ctx, Builder& bd, const std::vector<char
             bd.grel(g_da2);
             bd.conv(key + 13, CONV_WGRAD, s.a1, r.conv[0], bd.gbuf[g_dy1], nullptr, nullptr, B, s.H, s.W, 1.f);
             g_da1 = bd.gtake();
-            bd.conv(key + 15, CONV_DGRAD, nullptr, r.conv[0], bd.gbuf[g_dy1], g_sc >= 0 ? bd.gbuf[g_sc] : nullptr, bd.gbuf[g_da1], B, s.H, s.W, 1.f);
+            bd.conv(key + 15, CONV_DGRAD, nullptr, r.conv[0], bd.gbuf[g_dy1], g_sc >= 0 ? bd.gbuf[g_sc] : nullptr, bd.gbuf[g_da1], B, s.H, s.W, 1.f, false, sc_compact);
             bd.grel(g_dy1);
         }
         bd.grel(g_sc);
@@ -481,6 +494,12 @@ static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool s
         size_t j = i;
         while (j < ops.size() && ops[j].key == ops[i].key && ops[j].kind == ops[i].kind && ops[j].backend == ops[i].backend) ++j;
         Launch L{}; L.kind = ops[i].kind; L.backend = ops[i].backend; L.count = (int)(j - i);
+        if (ops[i].kind == OP_CONV_FWD || ops[i].kind == OP_CONV_DGRAD || ops[i].kind == OP_CONV_WGRAD) {
+            const ConvProb& c = ops[i].conv;
+            snprintf(L.label, sizeof(L.label), "%dx%d C%d K%d HW%d s%d%s x%d", c.ksz, c.ksz, c.C, c.K, c.H, c.stride, c.dy_sub == 2 ? "*" : "", L.count);
+        } else if (ops[i].kind != OP_HEAD_FWD && ops[i].kind != OP_HEAD_BWD && ops[i].kind != OP_POOL_FWD && ops[i].kind != OP_POOL_BWD &&
+                   ops[i].kind != OP_UPSAMPLE && ops[i].kind != OP_IM2COL && ops[i].kind != OP_SPLITK)
+            snprintf(L.label, sizeof(L.label), "bn m%lld C%d x%d", ops[i].bn.m, ops[i].bn.C, L.count);
         for (size_t k = i; k < j; ++k) {
             const Op& o = ops[k]; const int slot = single ? 0 : o.sub;
             switch (o.kind) {
@@ -526,14 +545,17 @@ static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool s
                         L.flops += 2.0 * out_e * p.ksz * p.ksz * p.C; L.bytes += es * (in_e + out_e) + 4.0 * w_e;
                         break;
                     }
-                    if (o.backend && o.kind != OP_SPLITK) {      // tensor-core problem: its own descriptor array
+                    if (o.backend && o.kind != OP_SPLITK) {      // tensor-core problem: its own descriptor array (one descriptor, or one per output phase)
                         if (k == i) L.first = n_tc;
-                        tc.resize((size_t)(n_tc + 1) * tcb);
                         const int mode = o.kind == OP_CONV_FWD ? CONV_FWD : o.kind == OP_CONV_DGRAD ? CONV_DGRAD : CONV_WGRAD;
-                        if (!conv_tc_fill(o.conv, mode, tc.data() + (size_t)n_tc * tcb)) { ctx->err = "tensor map encoding failed"; return RESIST_ECUDA; }
-                        L.gx = std::max(L.gx, conv_tc_tiles(tc.data() + (size_t)n_tc * tcb));
-                        L.max_elems = (long long)conv_tc_merge((size_t)L.max_elems, conv_tc_smem(tc.data() + (size_t)n_tc * tcb));
-                        ++n_tc;
+                        const int nd = conv_tc_count(o.conv, mode);
+                        tc.resize((size_t)(n_tc + std::max(nd, 1)) * tcb);
+                        if (!nd || conv_tc_fill(o.conv, mode, tc.data() + (size_t)n_tc * tcb) != nd) { ctx->err = "tensor map encoding failed"; return RESIST_ECUDA; }
+                        for (int d = 0; d < nd; ++d) {
+                            L.gx = std::max(L.gx, conv_tc_tiles(tc.data() + (size_t)(n_tc + d) * tcb));
+                            L.max_elems = (long long)conv_tc_merge((size_t)L.max_elems, conv_tc_smem(tc.data() + (size_t)(n_tc + d) * tcb));
+                        }
+                        n_tc += nd; L.ndesc += nd;
                         const ConvProb& p = o.conv;
                         const double in_e = (double)p.N * p.H * p.W * p.C, out_e = (double)p.N * p.P * p.Q * p.K, w_e = (double)p.K * p.ksz * p.ksz * p.C;
                         L.flops += 2.0 * out_e * p.ksz * p.ksz * p.C;
@@ -553,13 +575,14 @@ static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool s
                         if (o.kind == OP_CONV_WGRAD) L.bytes += es * (in_e + out_e) + 4.0 * w_e;
                         else L.bytes += es * (in_e + out_e + w_e + (p.add ? (o.kind == OP_CONV_FWD ? out_e : in_e) : 0.0)); }
                     break; }
-                case OP_BN_STATS: case OP_BN_APPLY: case OP_BN_BWD_REDUCE: case OP_BN_BWD_APPLY: case OP_BN_FWD_FUSED: case OP_BN_BWD_FUSED: {
+                case OP_BN_STATS: case OP_BN_APPLY: case OP_BN_BWD_REDUCE: case OP_BN_BWD_APPLY: case OP_BN_FWD_FUSED: case OP_BN_BWD_FUSED: case OP_BN_TILE_STATS: {
                     if (k == i) L.first = (int)bn.size();
                     bn.push_back(o.bn);
                     L.gx = std::max(L.gx, o.bn.chunks); L.max_c = std::max(L.max_c, o.bn.C);
                     L.max_elems = std::max<long long>(L.max_elems, o.bn.m * o.bn.C);
                     { const double e = (double)o.bn.m * o.bn.C;
-                      if (o.kind == OP_BN_STATS) L.bytes += o.bn.eval ? 0.0 : es * e;
+                      if (o.kind == OP_BN_TILE_STATS) L.bytes += 8.0 * o.bn.chunks * o.bn.C;
+                      else if (o.kind == OP_BN_STATS) L.bytes += o.bn.eval ? 0.0 : es * e;
                       else if (o.kind == OP_BN_APPLY) L.bytes += 2 * es * e;
                       else if (o.kind == OP_BN_BWD_REDUCE) L.bytes += 2 * es * e;
                       else if (o.kind == OP_BN_FWD_FUSED) L.bytes += 2 * es * e;          // x once from HBM (the second read is an L2 hit), a once
@@ -611,7 +634,7 @@ static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool s
                         if (o.fuse == 1) wr.push_back(o.bn.a); else if (o.fuse == 2) wr.push_back(o.bn.dx);
                         break;
                     case OP_CONV_WGRAD: case OP_SPLITK: break;
-                    case OP_BN_STATS: case OP_BN_BWD_REDUCE: break;
+                    case OP_BN_STATS: case OP_BN_BWD_REDUCE: case OP_BN_TILE_STATS: break;
                     case OP_BN_APPLY: case OP_BN_FWD_FUSED: wr.push_back(o.bn.a); break;
                     case OP_BN_BWD_APPLY: case OP_BN_BWD_FUSED: wr.push_back(o.bn.dx); break;
                     default: always = true; break;
@@ -783,9 +806,10 @@ static int run_plan(resist_ctx* ctx, Plan& plan, const PatchArgs& pa, bool updat
             case OP_UPSAMPLE: pk = PK_UPSAMPLE; break;
             case OP_IM2COL: pk = PK_IM2COL; break;
             case OP_BN_FWD_FUSED: pk = PK_BN_FWD_FUSED; break;
+            case OP_BN_TILE_STATS: pk = PK_BN_TILE_STATS; break;
             case OP_BN_BWD_FUSED: pk = PK_BN_BWD_FUSED; break;
         }
-        pf.begin(pk, nk, L.bytes, L.flops, st);
+        pf.begin(pk, nk, L.bytes, L.flops, st, L.label);
         switch (L.kind) {
             case OP_CONV_FWD: case OP_CONV_DGRAD: case OP_CONV_WGRAD: {
                 const int mode = L.kind == OP_CONV_FWD ? CONV_FWD : L.kind == OP_CONV_DGRAD ? CONV_DGRAD : CONV_WGRAD;
@@ -795,7 +819,7 @@ static int run_plan(resist_ctx* ctx, Plan& plan, const PatchArgs& pa, bool updat
                         ctx->err = "warp-MMA convolution launch failed"; cudaGetLastError(); return RESIST_ECUDA; }
                 }
                 else if (L.backend && mode == CONV_WGRAD) { launch_conv_wgrad_tc_probs((const char*)plan.d_wtc + (size_t)L.first * plan.wtc_stride, L.count, L.gx, (size_t)L.max_elems, L.max_b, st); ++n_launch; }
-                else if (L.backend) launch_conv_tc_probs((const char*)plan.d_tc + (size_t)L.first * plan.tc_stride, L.count, L.gx, (size_t)L.max_elems, st);
+                else if (L.backend) launch_conv_tc_probs((const char*)plan.d_tc + (size_t)L.first * plan.tc_stride, L.ndesc, L.gx, (size_t)L.max_elems, st);
                 else launch_conv_ref(plan.d_conv + L.first, L.count, L.gx, mode, bf, st);
                 ++n_launch; break; }
             case OP_SPLITK: launch_splitk_reduce(plan.d_conv + L.first, L.count, (int)L.max_elems, st); ++n_launch; break;
@@ -809,6 +833,7 @@ static int run_plan(resist_ctx* ctx, Plan& plan, const PatchArgs& pa, bool updat
             case OP_HEAD_BWD: launch_head_bwd(plan.d_head + L.first, L.count, L.max_b, L.max_c, L.max_classes, L.max_elems, bf, st); n_launch += 3; break;
             case OP_UPSAMPLE: launch_zero_stuff(plan.d_up + L.first, L.count, L.max_elems, st); ++n_launch; break;
             case OP_IM2COL: launch_im2col(plan.d_col + L.first, L.count, L.max_elems, st); ++n_launch; break;
+            case OP_BN_TILE_STATS: launch_bn_finalize_tiles(plan.d_bn + L.first, L.count, L.max_c, st); ++n_launch; break;
             case OP_BN_FWD_FUSED:
                 if (launch_bn_fused(plan.d_bn + L.first, L.count, L.gx, 0, st)) ++n_launch;
                 else { launch_bn_stats(plan.d_bn + L.first, L.count, L.gx, L.max_c, bf, st); launch_bn_apply(plan.d_bn + L.first, L.count, L.max_elems, bf, st); n_launch += 3; }

@@ -277,11 +277,13 @@ int resist_get_step_info(resist_ctx* ctx, resist_step_info* out) {
 static const char* const PK_NAMES[PK_COUNT] = {
     "conv_fwd_cuda_core", "conv_dgrad_cuda_core", "conv_wgrad_cuda_core", "conv_fwd_tcgen05", "conv_dgrad_tcgen05",
     "conv_wgrad_tcgen05", "wgrad_splitk_reduce", "bn_stats", "bn_apply_relu", "bn_bwd_reduce", "bn_bwd_apply", "maxpool_fwd",
-    "maxpool_bwd", "head_fwd", "head_bwd", "sgd_momentum", "patch_pointers", "scatter", "aggregate", "zero_stuff_dy", "conv_fwd_mma", "conv_dgrad_mma", "conv_wgrad_mma", "im2col_stem", "bn_relu_fwd_fused", "bn_relu_bwd_fused", "conv_fwd_mma_bn", "conv_dgrad_mma_bn"};
+    "maxpool_bwd", "head_fwd", "head_bwd", "sgd_momentum", "patch_pointers", "scatter", "aggregate", "zero_stuff_dy", "conv_fwd_mma", "conv_dgrad_mma", "conv_wgrad_mma", "im2col_stem", "bn_relu_fwd_fused", "bn_relu_bwd_fused", "conv_fwd_mma_bn", "conv_dgrad_mma_bn", "bn_stats_from_tiles"};
 
 int resist_set_profiling(resist_ctx* ctx, int32_t on) {
     if (!ctx) return RESIST_EINVAL;
     ctx->prof.on = on != 0;
+    // RESIST_LAUNCH_TRACE=<file>: while profiling, every bracketed launch also appends "family-index, shape label, ms, bytes, flops"
+    if (on && !ctx->prof.trace) { const char* f = getenv("RESIST_LAUNCH_TRACE"); if (f && *f) ctx->prof.trace = fopen(f, "a"); }
     return RESIST_OK;
 }
 

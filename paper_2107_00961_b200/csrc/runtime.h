@@ -1,5 +1,6 @@
 // Host runtime of the ResIST library: context, parameter layout, per-round schedule and launch plans.
 #pragma once
+#include <cstdio>
 #include <string>
 #include <vector>
 #include "../../include/resist.h"
@@ -18,7 +19,7 @@ Layout make_layout(const resist_arch& a, const std::vector<resist_block>& blocks
 
 enum OpKind {
     OP_CONV_FWD, OP_CONV_DGRAD, OP_CONV_WGRAD, OP_SPLITK, OP_BN_STATS, OP_BN_APPLY, OP_BN_BWD_REDUCE, OP_BN_BWD_APPLY,
-    OP_POOL_FWD, OP_POOL_BWD, OP_HEAD_FWD, OP_HEAD_BWD, OP_UPSAMPLE, OP_IM2COL, OP_BN_FWD_FUSED, OP_BN_BWD_FUSED
+    OP_POOL_FWD, OP_POOL_BWD, OP_HEAD_FWD, OP_HEAD_BWD, OP_UPSAMPLE, OP_IM2COL, OP_BN_FWD_FUSED, OP_BN_BWD_FUSED, OP_BN_TILE_STATS
 };
 
 // One operation of one sub-ResNet, keyed so that equal keys of different sub-ResNets share a launch.
@@ -34,30 +35,35 @@ struct PatchSite { void** where; int what; int sub; };        // what: 0 images,
 
 struct Launch {
     OpKind kind; int backend; int first, count;               // range in the typed device array
+    int ndesc;                                                // tcgen05 forward / dgrad: descriptors of the launch (a stride-2 dgrad has one per output phase)
     int gx; long long max_elems; int max_b, max_c, max_classes;
     double bytes, flops;                                      // algorithmic work of this launch
     bool join_before;                                         // the main stream first waits for the weight gradients in flight
+    char label[40];                                           // shape of the launch's first problem, for the per-launch trace
 };
 
 enum ProfKind {
     PK_CONV_FWD_CC, PK_CONV_DGRAD_CC, PK_CONV_WGRAD_CC, PK_CONV_FWD_TC, PK_CONV_DGRAD_TC, PK_CONV_WGRAD_TC, PK_SPLITK,
     PK_BN_STATS, PK_BN_APPLY, PK_BN_BWD_REDUCE, PK_BN_BWD_APPLY, PK_POOL_FWD, PK_POOL_BWD, PK_HEAD_FWD, PK_HEAD_BWD,
-    PK_SGD, PK_PATCH, PK_SCATTER, PK_AGGREGATE, PK_UPSAMPLE, PK_CONV_FWD_MMA, PK_CONV_DGRAD_MMA, PK_CONV_WGRAD_MMA, PK_IM2COL, PK_BN_FWD_FUSED, PK_BN_BWD_FUSED, PK_CONV_FWD_MMA_BN, PK_CONV_DGRAD_MMA_BN, PK_COUNT
+    PK_SGD, PK_PATCH, PK_SCATTER, PK_AGGREGATE, PK_UPSAMPLE, PK_CONV_FWD_MMA, PK_CONV_DGRAD_MMA, PK_CONV_WGRAD_MMA, PK_IM2COL, PK_BN_FWD_FUSED, PK_BN_BWD_FUSED, PK_CONV_FWD_MMA_BN, PK_CONV_DGRAD_MMA_BN, PK_BN_TILE_STATS, PK_COUNT
 };
 struct Profiler {
     bool on = false;
     std::vector<cudaEvent_t> pool; size_t used = 0;
-    struct Pending { int kind; int launches; double bytes, flops; cudaEvent_t e0, e1; };
+    struct Pending { int kind; int launches; double bytes, flops; cudaEvent_t e0, e1; const char* label; };
+    FILE* trace = nullptr;                                    // RESIST_LAUNCH_TRACE=<file>: one line per bracketed launch (label, ms, bytes, flops)
     std::vector<Pending> pending;
     long long launches[PK_COUNT] = {}, ops[PK_COUNT] = {}; double ms[PK_COUNT] = {}, bytes[PK_COUNT] = {}, flops[PK_COUNT] = {};
     cudaEvent_t ev() { if (used == pool.size()) { cudaEvent_t e; cudaEventCreate(&e); pool.push_back(e); } return pool[used++]; }
-    void begin(int kind, int launches_, double b, double f, cudaStream_t st) {
-        if (!on) return; Pending p{kind, launches_, b, f, ev(), ev()}; cudaEventRecord(p.e0, st); pending.push_back(p); }
+    void begin(int kind, int launches_, double b, double f, cudaStream_t st, const char* label = "") {
+        if (!on) return; Pending p{kind, launches_, b, f, ev(), ev(), label}; cudaEventRecord(p.e0, st); pending.push_back(p); }
     void end(cudaStream_t st) { if (!on) return; cudaEventRecord(pending.back().e1, st); }
     void collect(cudaStream_t st) {
         if (!on) return; cudaStreamSynchronize(st);
         for (auto& p : pending) { float t = 0.f; cudaEventElapsedTime(&t, p.e0, p.e1);
-            ms[p.kind] += t; launches[p.kind] += p.launches; ops[p.kind] += 1; bytes[p.kind] += p.bytes; flops[p.kind] += p.flops; }
+            ms[p.kind] += t; launches[p.kind] += p.launches; ops[p.kind] += 1; bytes[p.kind] += p.bytes; flops[p.kind] += p.flops;
+            if (trace) fprintf(trace, "%d\t%s\t%.6f\t%.0f\t%.0f\n", p.kind, p.label, t, p.bytes, p.flops); }
+        if (trace) fflush(trace);
         pending.clear(); used = 0; }
 };
 

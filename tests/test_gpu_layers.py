@@ -42,6 +42,9 @@ SHAPES = [
     (3, 8, 8, 256, 256, 3, 1), (4, 32, 32, 3, 16, 3, 1), (2, 36, 36, 3, 64, 7, 2),
     (3, 10, 6, 24, 40, 3, 1), (5, 7, 7, 72, 40, 3, 2), (2, 14, 14, 64, 64, 3, 1), (1, 28, 28, 128, 128, 3, 1),
     (3, 13, 9, 40, 24, 1, 1),
+    # wide layers of the bottleneck nets: several 64-channel slabs, several column tiles, 4x4 maps, strided projections
+    (2, 4, 4, 512, 512, 3, 1), (2, 16, 16, 256, 512, 1, 2), (2, 8, 8, 1024, 256, 1, 1), (2, 8, 8, 256, 1024, 1, 1),
+    (2, 8, 8, 256, 256, 3, 2), (3, 6, 10, 136, 72, 3, 1), (2, 9, 7, 64, 128, 1, 2),
 ]
 
 
