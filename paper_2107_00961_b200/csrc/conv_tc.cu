@@ -105,26 +105,21 @@ __device__ __forceinline__ void sts128(uint32_t a, uint4 v) { asm volatile("st.s
 __device__ __forceinline__ uint32_t lds32(uint32_t a) { uint32_t v; asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(a)); return v; }
 
 constexpr int TC_THREADS = 192;
-constexpr int TC_MAX_STAGES = 6;
+constexpr int TC_MAX_STAGES = 12;
 constexpr int TILE_M = 128;
 constexpr int SLAB_BYTES = TILE_M * 128;      // 128 rows x 64 channels of bf16
 
 struct TapRef { int wtap; int shift; };       // weight tap index (r*ksz + s); row shift of the operand inside the window
-
 // One forward / dgrad problem.  The tensor maps come first so that each is 64-byte aligned.
 //
 // Positions and windows.  The positions of a problem are either the pixels of the output in order ("dense": 1x1 layers) or a
 // tall map of Hp x Wp positions per image with `pad` zero rows before each image and `pad` zero columns after each row (3x3
 // layers).  A tile is 128 consecutive positions [p0, p0 + 128).  Its operand for one tap group is a window of positions
 // [p0 - hb, ...) fetched once per 64-channel slab; tap t of the group reads the window from row (p0 - hb - window start) +
-// taps[t].shift on.  Window position (image, yy, xx) holds activation pixel ((yy - pad) * es + gys, xx * es + gxs) of that
+// shift[t] on.  Window position (image, yy, xx) holds activation pixel ((yy - pad) * es + gys, xx * es + gxs) of that
 // image, zero outside it: es = 2 with one group per input parity phase makes a stride-2 layer exact work (forward), and four
 // problems, one per output phase, do the same for a stride-2 dgrad.
-struct alignas(64) TcProb {
-    CUtensorMap map_a;        // activations (forward: a; dgrad: dy): (channel, pixel) or (channel, x, y, image), possibly element-strided
-    CUtensorMap map_b;        // weights [K][taps][C] viewed as (C, tap, K)
-    CUtensorMap map_out;      // dense problems: the output as (channel, pixel), box 64 x 128
-    CUtensorMap map_add;      // dense problems with a residual: the residual likewise
+struct TcHot {                // everything the kernel's loops read: each role keeps a copy in shared memory
     const __nv_bfloat16* add; __nv_bfloat16* out;
     float* stat_tiles;        // [tiles_m][2][ncol]: column sums and sums of squares of the stored tile, or nullptr
     int* status;
@@ -132,7 +127,7 @@ struct alignas(64) TcProb {
     int dense;                // 1: position index == output pixel index
     int add_mode;             // 0 none; 1 fetched by TMA into the staging tile (dense); 2 global loads at the output pixel; 3 global loads from a compact tensor that applies at even (y, x) only
     int ngroups; int gbeg[5]; int gxs[4], gys[4];
-    TapRef taps[9];
+    int wtap[9], shift[9];    // per tap: weight tap index (r*ksz + s); row shift of the operand inside the window
     int es, pad;
     int Hp, Wp, n_img;
     int R, box_pos, nbox, hb, a_box_bytes;
@@ -145,21 +140,37 @@ struct alignas(64) TcProb {
     float scale;
     int OH, OW, os, oy, ox;                  // position (image, yy, xx) -> output pixel ((yy - pad) * os + oy, xx * os + ox) of an OH x OW image
 };
+struct alignas(64) TcProb {
+    CUtensorMap map_a;        // activations (forward: a; dgrad: dy): (channel, pixel) or (channel, x, y, image), possibly element-strided
+    CUtensorMap map_b;        // weights [K][taps][C] viewed as (C, tap, K)
+    CUtensorMap map_out;      // dense problems: the output as (channel, pixel), box 64 x 128
+    CUtensorMap map_add;      // dense problems with a residual: the residual likewise
+    TcHot h;
+};
+static_assert(sizeof(TcHot) % 4 == 0, "copied word by word");
 
 struct TcLaunch { int nprob, na, nb, a_stage, b_stage, tmem_cols, acc_stride, n_stg, stg_bytes; };
+constexpr int TC_MAX_PROBS = 128;             // descriptors per launch (sub-ResNets x output phases)
+
+__device__ __forceinline__ void copy_hot(TcHot* dst, const TcHot* src, int tid, int nthreads) {
+    const uint32_t* s4 = reinterpret_cast<const uint32_t*>(src); uint32_t* d4 = reinterpret_cast<uint32_t*>(dst);
+    for (int i = tid; i < (int)(sizeof(TcHot) / 4); i += nthreads) d4[i] = __ldg(s4 + i);
+}
 
 __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const TcProb* __restrict__ probs, const TcLaunch L) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    __shared__ __align__(8) uint64_t bars[4 * TC_MAX_STAGES + 8];
+    __shared__ __align__(8) uint64_t bars[4 * TC_MAX_STAGES + 12];
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
     __shared__ int pix_s[TILE_M];
     __shared__ float stat_s[4][2][256];
+    __shared__ int tile_end_s[TC_MAX_PROBS];                      // running sum of the problems' tile counts
+    __shared__ TcHot hot_s[3];                                    // the current problem of the producer, the MMA issuer, the epilogue
     const uint32_t a_full = smem_u32(&bars[0]), a_empty = smem_u32(&bars[TC_MAX_STAGES]);
     const uint32_t b_full = smem_u32(&bars[2 * TC_MAX_STAGES]), b_empty = smem_u32(&bars[3 * TC_MAX_STAGES]);
     const uint32_t acc_full = smem_u32(&bars[4 * TC_MAX_STAGES]), acc_empty = smem_u32(&bars[4 * TC_MAX_STAGES + 2]);
-    const uint32_t add_full = smem_u32(&bars[4 * TC_MAX_STAGES + 4]), stg_free = smem_u32(&bars[4 * TC_MAX_STAGES + 6]);
+    const uint32_t add_full = smem_u32(&bars[4 * TC_MAX_STAGES + 4]), stg_free = smem_u32(&bars[4 * TC_MAX_STAGES + 8]);
     const uint32_t a_ring = smem_u32(smem), b_ring = a_ring + (uint32_t)(L.na * L.a_stage), stg_base = b_ring + (uint32_t)(L.nb * L.b_stage);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -167,8 +178,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const TcProb* __
         for (int s = 0; s < TC_MAX_STAGES; ++s) {
             mbar_init(a_full + 8 * s, 1); mbar_init(a_empty + 8 * s, 1); mbar_init(b_full + 8 * s, 1); mbar_init(b_empty + 8 * s, 1);
         }
-        for (int s = 0; s < 2; ++s) { mbar_init(acc_full + 8 * s, 1); mbar_init(acc_empty + 8 * s, 4); mbar_init(add_full + 8 * s, 1); mbar_init(stg_free + 8 * s, 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(acc_full + 8 * s, 1); mbar_init(acc_empty + 8 * s, 4); }
+        for (int s = 0; s < 4; ++s) { mbar_init(add_full + 8 * s, 1); mbar_init(stg_free + 8 * s, 1); }
         abort_s = 0;
+        int run = 0;
+        for (int i = 0; i < L.nprob; ++i) { run += probs[i].h.tiles_m * probs[i].h.tiles_n; tile_end_s[i] = run; }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -179,53 +193,58 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const TcProb* __
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = tmem_base_s;
-
-    int total_tiles = 0;
-    for (int i = 0; i < L.nprob; ++i) total_tiles += probs[i].tiles_m * probs[i].tiles_n;
+    const int total_tiles = tile_end_s[L.nprob - 1];
 
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer
         if (lane == 0) {
-            uint32_t a_cnt = 0, b_cnt = 0, seq = 0, add_use[2] = {0u, 0u}; bool ok = true;
+            uint32_t a_cnt = 0, b_cnt = 0, seq = 0, add_use[4] = {0u, 0u, 0u, 0u}; bool ok = true;
+            int cur = -1; TcHot& h = hot_s[0];
+            int sa = 0, sb_ = 0; uint32_t pha = 0, phb = 0;       // ring positions and phases
             for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++seq) {
-                int pi = 0, loc = t;
-                while (loc >= probs[pi].tiles_m * probs[pi].tiles_n) { loc -= probs[pi].tiles_m * probs[pi].tiles_n; ++pi; }
-                const TcProb& p = probs[pi];
-                const int tn = loc % p.tiles_n, tm = loc / p.tiles_n;
-                if (p.add_mode == 1) {
+                int pi = 0; while (t >= tile_end_s[pi]) ++pi;
+                if (pi != cur) { copy_hot(&h, &probs[pi].h, 0, 1); cur = pi; }
+                const TcProb* pp = probs + pi;
+                const int loc = t - (pi ? tile_end_s[pi - 1] : 0);
+                const int tiles_n = h.tiles_n, n_tile = h.n_tile, slabs = h.slabs, ngroups = h.ngroups, a_flat = h.a_flat, nbox = h.nbox,
+                          a_box_bytes = h.a_box_bytes, R = h.R, Hp = h.Hp, pad = h.pad, es = h.es, b_bytes = h.b_bytes, mn = h.b_mn_major;
+                const int tn = loc % tiles_n, tm = loc / tiles_n;
+                if (h.add_mode == 1) {
                     // the residual tile goes straight into the staging tile the epilogue will finish in place
-                    const uint32_t sb = L.n_stg == 2 ? (seq & 1u) : 0u, uses = L.n_stg == 2 ? (seq >> 1) : seq;
-                    if (!mbar_wait(stg_free + 8 * sb, (uses & 1u) ^ 1u, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(p.status, 7); ok = false; break; }
-                    mbar_expect_tx(add_full + 8 * sb, (uint32_t)(p.out_slabs * SLAB_BYTES));
-                    for (int j = 0; j < p.out_slabs; ++j)
-                        tma_load_2d(stg_base + sb * (uint32_t)L.stg_bytes + (uint32_t)(j * SLAB_BYTES), &p.map_add, add_full + 8 * sb, tn * p.n_tile + j * 64, tm * TILE_M);
+                    const uint32_t sb = seq % (uint32_t)L.n_stg, uses = seq / (uint32_t)L.n_stg;
+                    if (!mbar_wait(stg_free + 8 * sb, (uses & 1u) ^ 1u, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(h.status, 7); ok = false; break; }
+                    mbar_expect_tx(add_full + 8 * sb, (uint32_t)(h.out_slabs * SLAB_BYTES));
+                    for (int j = 0; j < h.out_slabs; ++j)
+                        tma_load_2d(stg_base + sb * (uint32_t)L.stg_bytes + (uint32_t)(j * SLAB_BYTES), &pp->map_add, add_full + 8 * sb, tn * n_tile + j * 64, tm * TILE_M);
                     ++add_use[sb];
                 }
-                const int bx0 = p.a_flat ? 0 : floor_div(tm * TILE_M - p.hb, p.box_pos);
-                for (int sl = 0; sl < p.slabs && ok; ++sl) {
-                    for (int g = 0; g < p.ngroups && ok; ++g) {
+                const int bx0 = a_flat ? 0 : floor_div(tm * TILE_M - h.hb, h.box_pos);
+                for (int sl = 0; sl < slabs && ok; ++sl) {
+                    for (int g = 0; g < ngroups && ok; ++g) {
                         {
-                            const int s = (int)(a_cnt % (uint32_t)L.na); const uint32_t ph = (a_cnt / (uint32_t)L.na) & 1u;
-                            if (!mbar_wait(a_empty + 8 * s, ph ^ 1u, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(p.status, 1); ok = false; break; }
-                            const uint32_t dst = a_ring + (uint32_t)(s * L.a_stage);
-                            mbar_expect_tx(a_full + 8 * s, (uint32_t)(p.nbox * p.a_box_bytes));
-                            if (p.a_flat) tma_load_2d(dst, &p.map_a, a_full + 8 * s, sl * 64, tm * TILE_M);
-                            else for (int i = 0; i < p.nbox; ++i) {
-                                const int trow = (bx0 + i) * p.R, img = floor_div(trow, p.Hp), yy0 = trow - img * p.Hp;
-                                tma_load_4d(dst + (uint32_t)(i * p.a_box_bytes), &p.map_a, a_full + 8 * s, sl * 64, p.gxs[g], (yy0 - p.pad) * p.es + p.gys[g], img);
+                            if (!mbar_wait(a_empty + 8 * sa, pha ^ 1u, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(h.status, 1); ok = false; break; }
+                            const uint32_t dst = a_ring + (uint32_t)(sa * L.a_stage);
+                            mbar_expect_tx(a_full + 8 * sa, (uint32_t)(nbox * a_box_bytes));
+                            if (a_flat) tma_load_2d(dst, &pp->map_a, a_full + 8 * sa, sl * 64, tm * TILE_M);
+                            else {
+                                const int gx = h.gxs[g], gy = h.gys[g];
+                                for (int i = 0; i < nbox; ++i) {
+                                    const int trow = (bx0 + i) * R, img = floor_div(trow, Hp), yy0 = trow - img * Hp;
+                                    tma_load_4d(dst + (uint32_t)(i * a_box_bytes), &pp->map_a, a_full + 8 * sa, sl * 64, gx, (yy0 - pad) * es + gy, img);
+                                }
                             }
-                            ++a_cnt;
+                            ++a_cnt; if (++sa == L.na) { sa = 0; pha ^= 1u; }
                         }
-                        for (int tap = p.gbeg[g]; tap < p.gbeg[g + 1]; ++tap) {
-                            const int s = (int)(b_cnt % (uint32_t)L.nb); const uint32_t ph = (b_cnt / (uint32_t)L.nb) & 1u;
-                            if (!mbar_wait(b_empty + 8 * s, ph ^ 1u, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(p.status, 2); ok = false; break; }
-                            const uint32_t dst = b_ring + (uint32_t)(s * L.b_stage);
-                            const int wtap = p.taps[tap].wtap;
-                            mbar_expect_tx(b_full + 8 * s, (uint32_t)p.b_bytes);
-                            if (!p.b_mn_major) tma_load_3d(dst, &p.map_b, b_full + 8 * s, sl * 64, wtap, tn * p.n_tile);
-                            else for (int j = 0; j * 64 < p.n_tile; ++j)
-                                tma_load_3d(dst + (uint32_t)(j * 8192), &p.map_b, b_full + 8 * s, tn * p.n_tile + j * 64, wtap, sl * 64);
-                            ++b_cnt;
+                        const int t_end = h.gbeg[g + 1];
+                        for (int tap = h.gbeg[g]; tap < t_end; ++tap) {
+                            if (!mbar_wait(b_empty + 8 * sb_, phb ^ 1u, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(h.status, 2); ok = false; break; }
+                            const uint32_t dst = b_ring + (uint32_t)(sb_ * L.b_stage);
+                            const int wtap = h.wtap[tap];
+                            mbar_expect_tx(b_full + 8 * sb_, (uint32_t)b_bytes);
+                            if (!mn) tma_load_3d(dst, &pp->map_b, b_full + 8 * sb_, sl * 64, wtap, tn * n_tile);
+                            else for (int j = 0; j * 64 < n_tile; ++j)
+                                tma_load_3d(dst + (uint32_t)(j * 8192), &pp->map_b, b_full + 8 * sb_, tn * n_tile + j * 64, wtap, sl * 64);
+                            ++b_cnt; if (++sb_ == L.nb) { sb_ = 0; phb ^= 1u; }
                         }
                     }
                 }
@@ -236,54 +255,57 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const TcProb* __
                     for (int i = 0; i < 4096 && !mbar_try(a_full + 8 * (c % L.na), (c / L.na) & 1u); ++i) __nanosleep(64);
                 for (uint32_t c = b_cnt > (uint32_t)L.nb ? b_cnt - L.nb : 0; c < b_cnt; ++c)
                     for (int i = 0; i < 4096 && !mbar_try(b_full + 8 * (c % L.nb), (c / L.nb) & 1u); ++i) __nanosleep(64);
-                for (uint32_t sb = 0; sb < 2; ++sb)
+                for (uint32_t sb = 0; sb < 4; ++sb)
                     if (add_use[sb]) for (int i = 0; i < 4096 && !mbar_try(add_full + 8 * sb, (add_use[sb] - 1u) & 1u); ++i) __nanosleep(64);
             }
         }
     } else if (warp == 1) {
         // ---------------------------------------------------------------- MMA issuer
         if (lane == 0) {
-            uint32_t a_cnt = 0, b_cnt = 0, acc_cnt = 0; bool ok = true;
+            uint32_t acc_cnt = 0; bool ok = true;
+            int cur = -1; TcHot& h = hot_s[1];
+            int sa = 0, sb = 0; uint32_t pha = 0, phb = 0;
+            // the constant part of a 128-byte-swizzle descriptor: stride between 8-row groups 1024 bytes, version, swizzle mode
+            const uint64_t desc_k = desc_sw128(0, 16, 1024), desc_mn = desc_sw128(0, 8192, 1024);
             for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++acc_cnt) {
-                int pi = 0, loc = t;
-                while (loc >= probs[pi].tiles_m * probs[pi].tiles_n) { loc -= probs[pi].tiles_m * probs[pi].tiles_n; ++pi; }
-                const TcProb& p = probs[pi];
-                const int tm = loc / p.tiles_n;
-                const int bx0 = p.a_flat ? 0 : floor_div(tm * TILE_M - p.hb, p.box_pos);
-                const int a_off = p.a_flat ? 0 : tm * TILE_M - p.hb - bx0 * p.box_pos;
+                int pi = 0; while (t >= tile_end_s[pi]) ++pi;
+                if (pi != cur) { copy_hot(&h, &probs[pi].h, 0, 1); cur = pi; }
+                const int loc = t - (pi ? tile_end_s[pi - 1] : 0);
+                const int slabs = h.slabs, ngroups = h.ngroups, red = h.red, mn = h.b_mn_major;
+                const int tm = loc / h.tiles_n;
+                const int bx0 = h.a_flat ? 0 : floor_div(tm * TILE_M - h.hb, h.box_pos);
+                const int a_off = h.a_flat ? 0 : tm * TILE_M - h.hb - bx0 * h.box_pos;
                 const uint32_t buf = acc_cnt & 1u, aph = (acc_cnt >> 1) & 1u;
-                if (!mbar_wait(acc_empty + 8 * buf, aph ^ 1u, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(p.status, 3); ok = false; break; }
+                if (!mbar_wait(acc_empty + 8 * buf, aph ^ 1u, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(h.status, 3); ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t d_tmem = tmem_base + buf * (uint32_t)L.acc_stride;
                 // instruction descriptor: fp32 accumulate, bf16 x bf16, A K-major, B K-major or MN-major, N, M = 128
-                const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)p.b_mn_major << 16) |
-                                       ((uint32_t)(p.n_tile >> 3) << 17) | ((128u >> 4) << 24);
+                const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)mn << 16) |
+                                       ((uint32_t)(h.n_tile >> 3) << 17) | ((128u >> 4) << 24);
+                const uint64_t b_const = mn ? desc_mn : desc_k;
+                const uint32_t b_step = mn ? 128u : 2u;           // one K = 16 step: 16 rows of 128 bytes (MN-major) or 32 bytes along the row (K-major), in 16-byte units
                 uint32_t acc = 0;
-                for (int sl = 0; sl < p.slabs && ok; ++sl) {
-                    const int ksteps = (min(64, p.red - sl * 64) + 15) >> 4;
-                    for (int g = 0; g < p.ngroups && ok; ++g) {
-                        const int sa = (int)(a_cnt % (uint32_t)L.na); const uint32_t pha = (a_cnt / (uint32_t)L.na) & 1u;
-                        if (!mbar_wait(a_full + 8 * sa, pha, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(p.status, 4); ok = false; break; }
+                for (int sl = 0; sl < slabs && ok; ++sl) {
+                    const int ksteps = (min(64, red - sl * 64) + 15) >> 4;
+                    for (int g = 0; g < ngroups && ok; ++g) {
+                        if (!mbar_wait(a_full + 8 * sa, pha, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(h.status, 4); ok = false; break; }
                         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                        const uint32_t a_base = a_ring + (uint32_t)(sa * L.a_stage) + (uint32_t)a_off * 128u;
-                        for (int tap = p.gbeg[g]; tap < p.gbeg[g + 1]; ++tap) {
-                            const int sb = (int)(b_cnt % (uint32_t)L.nb); const uint32_t phb = (b_cnt / (uint32_t)L.nb) & 1u;
-                            if (!mbar_wait(b_full + 8 * sb, phb, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(p.status, 5); ok = false; break; }
+                        const uint32_t a_rows16 = ((a_ring + (uint32_t)(sa * L.a_stage)) >> 4) + (uint32_t)a_off * 8u;   // start address in 16-byte units
+                        const int t_end = h.gbeg[g + 1];
+                        for (int tap = h.gbeg[g]; tap < t_end; ++tap) {
+                            const uint32_t a16 = a_rows16 + (uint32_t)h.shift[tap] * 8u;
+                            if (!mbar_wait(b_full + 8 * sb, phb, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(h.status, 5); ok = false; break; }
                             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                            const uint32_t a_tap = a_base + (uint32_t)p.taps[tap].shift * 128u;
-                            const uint32_t b_base = b_ring + (uint32_t)(sb * L.b_stage);
+                            const uint32_t b16 = (b_ring + (uint32_t)(sb * L.b_stage)) >> 4;
                             for (int k16 = 0; k16 < ksteps; ++k16) {
-                                const uint64_t ad = desc_sw128(a_tap + (uint32_t)k16 * 32u, 16, 1024);
-                                const uint64_t bd = p.b_mn_major ? desc_sw128(b_base + (uint32_t)k16 * 2048u, 8192, 1024)
-                                                                 : desc_sw128(b_base + (uint32_t)k16 * 32u, 16, 1024);
-                                umma_bf16(d_tmem, ad, bd, idesc, acc);
+                                umma_bf16(d_tmem, desc_k | (uint64_t)((a16 + 2u * (uint32_t)k16) & 0x3FFFu), b_const | (uint64_t)((b16 + b_step * (uint32_t)k16) & 0x3FFFu), idesc, acc);
                                 acc = 1;
                             }
                             umma_commit(b_empty + 8 * sb);       // weight tile reusable once these MMAs have read it
-                            ++b_cnt;
+                            if (++sb == L.nb) { sb = 0; phb ^= 1u; }
                         }
                         umma_commit(a_empty + 8 * sa);
-                        ++a_cnt;
+                        if (++sa == L.na) { sa = 0; pha ^= 1u; }
                     }
                 }
                 if (ok) umma_commit(acc_full + 8 * buf);         // accumulator complete
@@ -295,60 +317,66 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const TcProb* __
         const int m = quad * 32 + lane;                          // row of the tile = TMEM lane
         const int et = threadIdx.x - 64;                         // 0..127 among the epilogue threads
         const bool leader = et == 0;
-        uint32_t acc_cnt = 0, add_use[2] = {0u, 0u}; bool ok = true;
+        uint32_t acc_cnt = 0, add_use[4] = {0u, 0u, 0u, 0u}; bool ok = true;
+        int cur = -1; const TcHot& h = hot_s[2];
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++acc_cnt) {
-            int pi = 0, loc = t;
-            while (loc >= probs[pi].tiles_m * probs[pi].tiles_n) { loc -= probs[pi].tiles_m * probs[pi].tiles_n; ++pi; }
-            const TcProb& p = probs[pi];
-            const int tn = loc % p.tiles_n, tm = loc / p.tiles_n;
+            int pi = 0; while (t >= tile_end_s[pi]) ++pi;
+            const TcProb* pp = probs + pi;
+            const int loc = t - (pi ? tile_end_s[pi - 1] : 0);
             const uint32_t buf = acc_cnt & 1u, aph = (acc_cnt >> 1) & 1u;
-            const uint32_t sb = L.n_stg == 2 ? (acc_cnt & 1u) : 0u;
+            const uint32_t sb = acc_cnt % (uint32_t)L.n_stg;
             const uint32_t stg = stg_base + sb * (uint32_t)L.stg_bytes;
             // the staging tile is free again: the leader has waited for the reads of the bulk store it issued from it, and
             // every warp has finished its share of the last copy-out
             bar_sync_epi();
+            if (pi != cur) { copy_hot(&hot_s[2], &probs[pi].h, et, 128); cur = pi; bar_sync_epi(); }
+            const int tiles_n = h.tiles_n, n_tile = h.n_tile, ncol = h.ncol, add_mode = h.add_mode, dense = h.dense, out_slabs = h.out_slabs;
+            const float scale = h.scale;
+            const __nv_bfloat16* addp = h.add; __nv_bfloat16* outp = h.out; float* stat_tiles = h.stat_tiles;
+            const int tn = loc % tiles_n, tm = loc / tiles_n;
             ok = mbar_wait(acc_full + 8 * buf, aph, &abort_s);
-            if (ok && p.add_mode == 1) { ok = mbar_wait(add_full + 8 * sb, add_use[sb] & 1u, &abort_s); ++add_use[sb]; }
+            if (ok && add_mode == 1) { ok = mbar_wait(add_full + 8 * sb, add_use[sb] & 1u, &abort_s); ++add_use[sb]; }
             ok = bar_and_epi(ok);                                // one decision for the four warps: they share the barriers below
-            if (!ok) { atomicExch(&abort_s, 1); atomicExch(p.status, 6); break; }
+            if (!ok) { atomicExch(&abort_s, 1); atomicExch(h.status, 6); break; }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             // position -> output pixel (and the residual's pixel)
             const int pos = tm * TILE_M + m;
-            bool valid = pos < p.total_pos;
+            bool valid = pos < h.total_pos;
             long long pix = pos, addpix = -1;
-            if (valid && (!p.dense || p.add_mode == 3)) {
-                const int trow = pos / p.Wp, xx = pos - trow * p.Wp, img = trow / p.Hp, yy = trow - img * p.Hp;
-                const int y = (yy - p.pad) * p.os + p.oy, x = xx * p.os + p.ox;
-                valid = yy >= p.pad && xx < p.Wp - p.pad && y < p.OH && x < p.OW;
-                pix = ((long long)img * p.OH + y) * p.OW + x;
-                if (p.add_mode == 3 && !((y | x) & 1)) addpix = ((long long)img * ((p.OH + 1) >> 1) + (y >> 1)) * ((p.OW + 1) >> 1) + (x >> 1);
+            if (valid && (!dense || add_mode == 3)) {
+                const int Wp = h.Wp, Hp = h.Hp, pad = h.pad, os = h.os, OH = h.OH, OW = h.OW;
+                const int trow = pos / Wp, xx = pos - trow * Wp, img = trow / Hp, yy = trow - img * Hp;
+                const int y = (yy - pad) * os + h.oy, x = xx * os + h.ox;
+                valid = yy >= pad && xx < Wp - pad && y < OH && x < OW;
+                pix = ((long long)img * OH + y) * OW + x;
+                if (add_mode == 3 && !((y | x) & 1)) addpix = ((long long)img * ((OH + 1) >> 1) + (y >> 1)) * ((OW + 1) >> 1) + (x >> 1);
             }
-            if (p.add_mode == 2) addpix = pix;
-            if (!p.dense) pix_s[m] = valid ? (int)pix : -1;
+            if (add_mode == 2) addpix = pix;
+            if (!dense) pix_s[m] = valid ? (int)pix : -1;
             const uint32_t t_row = tmem_base + buf * (uint32_t)L.acc_stride + ((uint32_t)(quad * 32) << 16);
-            const int col0 = tn * p.n_tile;
+            const int col0 = tn * n_tile;
             const uint32_t s_row = stg + (uint32_t)m * 128u;
-            const bool gadd = p.add_mode >= 2 && valid && addpix >= 0;
-            for (int c0 = 0; c0 < p.n_tile; c0 += 32) {
+            const bool gadd = add_mode >= 2 && valid && addpix >= 0;
+            for (int c0 = 0; c0 < n_tile; c0 += 32) {
                 uint32_t v[32];
                 tmem_ld32(t_row + (uint32_t)c0, v);
                 uint4 ga[4];
                 if (gadd) {
 #pragma unroll
                     for (int g = 0; g < 4; ++g)
-                        ga[g] = (c0 + g * 8 < p.n_tile && col0 + c0 + g * 8 < p.ncol) ? __ldg(reinterpret_cast<const uint4*>(p.add + addpix * p.ncol + col0 + c0 + g * 8)) : make_uint4(0u, 0u, 0u, 0u);
+                        ga[g] = (c0 + g * 8 < n_tile && col0 + c0 + g * 8 < ncol) ? __ldg(reinterpret_cast<const uint4*>(addp + addpix * ncol + col0 + c0 + g * 8)) : make_uint4(0u, 0u, 0u, 0u);
                 }
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
                 for (int g = 0; g < 4; ++g) {
                     const int c = c0 + g * 8;
-                    if (c < p.n_tile) {
+                    if (c < n_tile) {
                         const uint32_t sa = s_row + (uint32_t)(c >> 6) * SLAB_BYTES + ((uint32_t)(((c >> 3) & 7) ^ (m & 7)) << 4);
                         float f[8];
 #pragma unroll
-                        for (int k = 0; k < 8; ++k) f[k] = valid ? __uint_as_float(v[g * 8 + k]) * p.scale : 0.f;
-                        if (p.add_mode == 1 || gadd) {
-                            const uint4 a0 = p.add_mode == 1 ? lds128(sa) : ga[g];
+                        for (int k = 0; k < 8; ++k) f[k] = valid ? __uint_as_float(v[g * 8 + k]) * scale : 0.f;
+                        if (add_mode == 1 || gadd) {
+                            const uint4 a0 = add_mode == 1 ? lds128(sa) : ga[g];
                             const uint32_t aw[4] = {a0.x, a0.y, a0.z, a0.w};
                             if (valid) {
 #pragma unroll
@@ -361,8 +389,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const TcProb* __
                         uint32_t w[4];
 #pragma unroll
                         for (int k = 0; k < 4; ++k) {
-                            __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * k], f[2 * k + 1]);
-                            w[k] = *reinterpret_cast<uint32_t*>(&h);
+                            __nv_bfloat162 hh = __floats2bfloat162_rn(f[2 * k], f[2 * k + 1]);
+                            w[k] = *reinterpret_cast<uint32_t*>(&hh);
                         }
                         sts128(sa, make_uint4(w[0], w[1], w[2], w[3]));
                     }
@@ -373,14 +401,14 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const TcProb* __
             __syncwarp();
             if (lane == 0) mbar_arrive(acc_empty + 8 * buf);     // this warp has read its quadrant of the accumulator
             bar_sync_epi();                                      // the staging tile is complete
-            if (p.dense && leader) {
-                for (int j = 0; j < p.out_slabs; ++j) tma_store_2d(&p.map_out, stg + (uint32_t)(j * SLAB_BYTES), col0 + j * 64, tm * TILE_M);
+            if (dense && leader) {
+                for (int j = 0; j < out_slabs; ++j) tma_store_2d(&pp->map_out, stg + (uint32_t)(j * SLAB_BYTES), col0 + j * 64, tm * TILE_M);
                 asm volatile("cp.async.bulk.commit_group;" ::: "memory");
             }
-            if (p.stat_tiles) {
+            if (stat_tiles) {
                 // column sums of the stored (rounded) values: every warp over its own 32 rows, lane = two neighbouring columns;
                 // the four warps' sums are then added in a fixed order
-                for (int j = 0; j < p.out_slabs; ++j) {
+                for (int j = 0; j < out_slabs; ++j) {
                     float s0 = 0.f, s1 = 0.f, q0 = 0.f, q1 = 0.f;
 #pragma unroll 8
                     for (int r = 0; r < 32; ++r) {
@@ -393,28 +421,28 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const TcProb* __
                     stat_s[quad][1][j * 64 + 2 * lane] = q0; stat_s[quad][1][j * 64 + 2 * lane + 1] = q1;
                 }
                 bar_sync_epi();
-                for (int c = et; c < p.n_tile; c += 128) {
-                    if (col0 + c < p.ncol) {
+                for (int c = et; c < n_tile; c += 128) {
+                    if (col0 + c < ncol) {
                         const float su = ((stat_s[0][0][c] + stat_s[1][0][c]) + stat_s[2][0][c]) + stat_s[3][0][c];
                         const float sq = ((stat_s[0][1][c] + stat_s[1][1][c]) + stat_s[2][1][c]) + stat_s[3][1][c];
-                        p.stat_tiles[((long long)tm * 2 + 0) * p.ncol + col0 + c] = su;
-                        p.stat_tiles[((long long)tm * 2 + 1) * p.ncol + col0 + c] = sq;
+                        stat_tiles[((long long)tm * 2 + 0) * ncol + col0 + c] = su;
+                        stat_tiles[((long long)tm * 2 + 1) * ncol + col0 + c] = sq;
                     }
                 }
             }
-            if (!p.dense) {
+            if (!dense) {
                 // copy-out of a tall tile: 16-byte chunks, eight consecutive lanes per 128-byte run of one output pixel
-                const int n_chunks = p.out_slabs * TILE_M * 8;
+                const int n_chunks = out_slabs * TILE_M * 8;
                 for (int idx = et; idx < n_chunks; idx += 128) {
                     const int ch = idx & 7, row = (idx >> 3) & (TILE_M - 1), j = idx >> 10;
                     const int c = j * 64 + ch * 8, px = pix_s[row];
-                    if (px >= 0 && c < p.n_tile && col0 + c < p.ncol)
-                        *reinterpret_cast<uint4*>(p.out + (long long)px * p.ncol + col0 + c) =
+                    if (px >= 0 && c < n_tile && col0 + c < ncol)
+                        *reinterpret_cast<uint4*>(outp + (long long)px * ncol + col0 + c) =
                             lds128(stg + (uint32_t)(j * SLAB_BYTES) + (uint32_t)row * 128u + ((uint32_t)(ch ^ (row & 7)) << 4));
                 }
             }
             if (leader) {
-                if (p.dense) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                if (dense) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
                 mbar_arrive(stg_free + 8 * sb);
             }
         }
@@ -478,13 +506,19 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_wgrad_tc_kernel(const TcWg
     const TcWgradProb& p = probs[blockIdx.y];
     const int ctas = p.m_tiles * p.n_tiles * p.tap_groups * p.splits;
     if ((int)blockIdx.x >= ctas) return;
+    // everything the loops read, in registers (the descriptor lives in global memory)
+    const int splits = p.splits, tap_groups = p.tap_groups, n_tiles = p.n_tiles, chunks = p.chunks, chunks_per_split = p.chunks_per_split;
+    const int stages = p.stages, stage_bytes = p.stage_bytes, dy_slab_bytes = p.dy_slab_bytes, a_slab_bytes = p.a_slab_bytes, a_slabs = p.a_slabs;
+    const int n_tile = p.n_tile, dy_flat = p.dy_flat, a_flat = p.a_flat, box_pos = p.box_pos, hb = p.hb, R = p.R, Hp = p.Hp, pad = p.pad, es = p.es;
+    const int nbox_dy = p.nbox_dy, nbox_a = p.nbox_a, dy_box_bytes = p.dy_box_bytes, a_box_bytes = p.a_box_bytes, tmem_cols = p.tmem_cols;
     int id = blockIdx.x;
-    const int split = id % p.splits; id /= p.splits;
-    const int tg = id % p.tap_groups; id /= p.tap_groups;
-    const int tn = id % p.n_tiles; const int tm = id / p.n_tiles;
-    const int c_begin = split * p.chunks_per_split;
-    const int c_end = min(c_begin + p.chunks_per_split, p.chunks);
+    const int split = id % splits; id /= splits;
+    const int tg = id % tap_groups; id /= tap_groups;
+    const int tn = id % n_tiles; const int tm = id / n_tiles;
+    const int c_begin = split * chunks_per_split;
+    const int c_end = min(c_begin + chunks_per_split, chunks);
     const int tap0 = p.gbeg[tg], ntap = p.gbeg[tg + 1] - tap0;
+    const int gx = p.gxs[tg], gy = p.gys[tg];
     const int nc = c_end - c_begin;
 
     extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -492,6 +526,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_wgrad_tc_kernel(const TcWg
     __shared__ __align__(8) uint64_t bars[2 * TC_MAX_STAGES + 1];
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
+    __shared__ int shift8_s[4], wtap_s[4];                       // the group's taps: row shift in 16-byte units, index in dw
     const uint32_t bar_full = smem_u32(&bars[0]), bar_empty = smem_u32(&bars[TC_MAX_STAGES]), bar_acc = smem_u32(&bars[2 * TC_MAX_STAGES]);
     const uint32_t ring = smem_u32(smem);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -500,10 +535,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_wgrad_tc_kernel(const TcWg
         for (int s = 0; s < TC_MAX_STAGES; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
         mbar_init(bar_acc, 1);
         abort_s = 0;
+        for (int i = 0; i < ntap; ++i) { shift8_s[i] = p.tap[tap0 + i].shift * 8; wtap_s[i] = p.tap[tap0 + i].wtap; }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(p.tmem_cols) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(tmem_cols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -513,86 +549,89 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_wgrad_tc_kernel(const TcWg
 
     if (warp == 0) {
         if (lane == 0) {
-            int i = 0; bool ok = true;
+            int i = 0; bool ok = true; int s = 0; uint32_t ph = 0;
+            const uint32_t tx = (uint32_t)(2 * nbox_dy * dy_box_bytes + a_slabs * nbox_a * a_box_bytes);
             for (; i < nc; ++i) {
-                const int s = i % p.stages; const uint32_t ph = (uint32_t)(i / p.stages) & 1u;
                 if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(p.status, 11); ok = false; break; }
                 const int pos0 = (c_begin + i) * TILE_M;
-                const uint32_t dy_dst = ring + (uint32_t)(s * p.stage_bytes), a_dst = dy_dst + 2u * (uint32_t)p.dy_slab_bytes;
-                mbar_expect_tx(bar_full + 8 * s, (uint32_t)(2 * p.nbox_dy * p.dy_box_bytes + p.a_slabs * p.nbox_a * p.a_box_bytes));
-                if (p.dy_flat) {
-                    for (int j = 0; j < 2; ++j) tma_load_2d(dy_dst + (uint32_t)(j * p.dy_slab_bytes), &p.map_dy, bar_full + 8 * s, tm * 128 + j * 64, pos0);
+                const uint32_t dy_dst = ring + (uint32_t)(s * stage_bytes), a_dst = dy_dst + 2u * (uint32_t)dy_slab_bytes;
+                mbar_expect_tx(bar_full + 8 * s, tx);
+                if (dy_flat) {
+                    for (int j = 0; j < 2; ++j) tma_load_2d(dy_dst + (uint32_t)(j * dy_slab_bytes), &p.map_dy, bar_full + 8 * s, tm * 128 + j * 64, pos0);
                 } else {
-                    const int bd0 = pos0 / p.box_pos;
-                    for (int b = 0; b < p.nbox_dy; ++b) {
-                        const int trow = (bd0 + b) * p.R, img = trow / p.Hp, yy0 = trow - img * p.Hp;
+                    const int bd0 = pos0 / box_pos;
+                    for (int b = 0; b < nbox_dy; ++b) {
+                        const int trow = (bd0 + b) * R, img = trow / Hp, yy0 = trow - img * Hp;
                         for (int j = 0; j < 2; ++j)
-                            tma_load_4d(dy_dst + (uint32_t)(j * p.dy_slab_bytes + b * p.dy_box_bytes), &p.map_dy, bar_full + 8 * s, tm * 128 + j * 64, 0, yy0 - p.pad, img);
+                            tma_load_4d(dy_dst + (uint32_t)(j * dy_slab_bytes + b * dy_box_bytes), &p.map_dy, bar_full + 8 * s, tm * 128 + j * 64, 0, yy0 - pad, img);
                     }
                 }
-                if (p.a_flat) {
-                    for (int j = 0; j < p.a_slabs; ++j) tma_load_2d(a_dst + (uint32_t)(j * p.a_slab_bytes), &p.map_a, bar_full + 8 * s, tn * p.n_tile + j * 64, pos0);
+                if (a_flat) {
+                    for (int j = 0; j < a_slabs; ++j) tma_load_2d(a_dst + (uint32_t)(j * a_slab_bytes), &p.map_a, bar_full + 8 * s, tn * n_tile + j * 64, pos0);
                 } else {
-                    const int ba0 = floor_div(pos0 - p.hb, p.box_pos);
-                    for (int b = 0; b < p.nbox_a; ++b) {
-                        const int trow = (ba0 + b) * p.R, img = floor_div(trow, p.Hp), yy0 = trow - img * p.Hp;
-                        for (int j = 0; j < p.a_slabs; ++j)
-                            tma_load_4d(a_dst + (uint32_t)(j * p.a_slab_bytes + b * p.a_box_bytes), &p.map_a, bar_full + 8 * s, tn * p.n_tile + j * 64,
-                                        p.gxs[tg], (yy0 - p.pad) * p.es + p.gys[tg], img);
+                    const int ba0 = floor_div(pos0 - hb, box_pos);
+                    for (int b = 0; b < nbox_a; ++b) {
+                        const int trow = (ba0 + b) * R, img = floor_div(trow, Hp), yy0 = trow - img * Hp;
+                        for (int j = 0; j < a_slabs; ++j)
+                            tma_load_4d(a_dst + (uint32_t)(j * a_slab_bytes + b * a_box_bytes), &p.map_a, bar_full + 8 * s, tn * n_tile + j * 64,
+                                        gx, (yy0 - pad) * es + gy, img);
                     }
                 }
+                if (++s == stages) { s = 0; ph ^= 1u; }
             }
             if (!ok)
-                for (int c = max(0, i - p.stages); c < i; ++c)
-                    for (int w = 0; w < 4096 && !mbar_try(bar_full + 8 * (c % p.stages), (uint32_t)(c / p.stages) & 1u); ++w) __nanosleep(64);
+                for (int c = max(0, i - stages); c < i; ++c)
+                    for (int w = 0; w < 4096 && !mbar_try(bar_full + 8 * (c % stages), (uint32_t)(c / stages) & 1u); ++w) __nanosleep(64);
         }
     } else if (warp == 1) {
         if (lane == 0) {
             // fp32 accumulate, bf16 x bf16, A and B MN-major, N = n_tile, M = 128
-            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) | ((uint32_t)(p.n_tile >> 3) << 17) | ((128u >> 4) << 24);
-            bool ok = true;
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) | ((uint32_t)(n_tile >> 3) << 17) | ((128u >> 4) << 24);
+            const uint64_t dy_const = desc_sw128(0, (uint32_t)dy_slab_bytes, 1024), a_const = desc_sw128(0, (uint32_t)a_slab_bytes, 1024);
+            bool ok = true; int s = 0; uint32_t ph = 0;
             for (int i = 0; i < nc && ok; ++i) {
-                const int s = i % p.stages; const uint32_t ph = (uint32_t)(i / p.stages) & 1u;
                 if (!mbar_wait(bar_full + 8 * s, ph, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(p.status, 12); ok = false; break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const int pos0 = (c_begin + i) * TILE_M;
-                const int dy_off = p.dy_flat ? 0 : pos0 - (pos0 / p.box_pos) * p.box_pos;
-                const int a_off = p.a_flat ? 0 : pos0 - p.hb - floor_div(pos0 - p.hb, p.box_pos) * p.box_pos;
-                const uint32_t dy_base = ring + (uint32_t)(s * p.stage_bytes) + (uint32_t)dy_off * 128u;
-                const uint32_t a_base = ring + (uint32_t)(s * p.stage_bytes) + 2u * (uint32_t)p.dy_slab_bytes + (uint32_t)a_off * 128u;
+                const int dy_off = dy_flat ? 0 : pos0 - (pos0 / box_pos) * box_pos;
+                const int a_off = a_flat ? 0 : pos0 - hb - floor_div(pos0 - hb, box_pos) * box_pos;
+                const uint32_t dy16 = ((ring + (uint32_t)(s * stage_bytes)) >> 4) + (uint32_t)dy_off * 8u;       // start addresses in 16-byte units
+                const uint32_t a16 = ((ring + (uint32_t)(s * stage_bytes) + 2u * (uint32_t)dy_slab_bytes) >> 4) + (uint32_t)a_off * 8u;
                 for (int tt = 0; tt < ntap; ++tt) {
-                    const uint32_t a_tap = a_base + (uint32_t)p.tap[tap0 + tt].shift * 128u;
-                    for (int k16 = 0; k16 < 8; ++k16) {
-                        const uint64_t ad = desc_sw128(dy_base + (uint32_t)k16 * 2048u, (uint32_t)p.dy_slab_bytes, 1024);
-                        const uint64_t bd = desc_sw128(a_tap + (uint32_t)k16 * 2048u, (uint32_t)p.a_slab_bytes, 1024);
-                        umma_bf16(tmem_d + (uint32_t)(tt * p.n_tile), ad, bd, idesc, (i | k16) ? 1u : 0u);
-                    }
+                    const uint32_t at16 = a16 + (uint32_t)shift8_s[tt];
+                    const uint32_t d_t = tmem_d + (uint32_t)(tt * n_tile);
+#pragma unroll
+                    for (int k16 = 0; k16 < 8; ++k16)          // 16 positions = 16 rows of 128 bytes per step
+                        umma_bf16(d_t, dy_const | (uint64_t)((dy16 + 128u * (uint32_t)k16) & 0x3FFFu), a_const | (uint64_t)((at16 + 128u * (uint32_t)k16) & 0x3FFFu), idesc, (i | k16) ? 1u : 0u);
                 }
                 umma_commit(bar_empty + 8 * s);
+                if (++s == stages) { s = 0; ph ^= 1u; }
             }
             if (ok) umma_commit(bar_acc);
         }
     } else {
         const int quad = warp & 3, m = quad * 32 + lane;
+        const int cout = p.cout, cin = p.cin, taps = p.taps;
+        float* const partial = p.partial; float* const outp = p.out;
         bool ok = nc > 0 ? mbar_wait(bar_acc, 0, &abort_s) : true;
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) { atomicExch(&abort_s, 1); atomicExch(p.status, 13); }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const int k = tm * 128 + m;
-        if (ok && quad * 32 < p.cout - tm * 128) {            // warp-uniform: this lane quadrant holds real output channels
+        if (ok && quad * 32 < cout - tm * 128) {              // warp-uniform: this lane quadrant holds real output channels
             for (int tt = 0; tt < ntap; ++tt) {
-                const int wt = p.tap[tap0 + tt].wtap;
-                float* dst = p.splits > 1 ? p.partial + (((long long)split * p.taps + wt) * p.cout + k) * p.cin + tn * p.n_tile
-                                          : p.out + ((long long)k * p.taps + wt) * p.cin + tn * p.n_tile;
-                for (int c0 = 0; c0 < p.n_tile; c0 += 32) {
+                const int wt = wtap_s[tt];
+                float* dst = splits > 1 ? partial + (((long long)split * taps + wt) * cout + k) * cin + tn * n_tile
+                                        : outp + ((long long)k * taps + wt) * cin + tn * n_tile;
+                for (int c0 = 0; c0 < n_tile; c0 += 32) {
                     uint32_t v[32];
-                    if (nc > 0) { tmem_ld32(tmem_d + ((uint32_t)(quad * 32) << 16) + (uint32_t)(tt * p.n_tile + c0), v);
+                    if (nc > 0) { tmem_ld32(tmem_d + ((uint32_t)(quad * 32) << 16) + (uint32_t)(tt * n_tile + c0), v);
                         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
                     else { for (int j = 0; j < 32; ++j) v[j] = 0u; }
-                    if (k < p.cout) {
+                    if (k < cout) {
 #pragma unroll
                         for (int j = 0; j < 32; j += 4)
-                            if (c0 + j < p.n_tile && tn * p.n_tile + c0 + j < p.cin)
+                            if (c0 + j < n_tile && tn * n_tile + c0 + j < cin)
                                 *reinterpret_cast<uint4*>(dst + c0 + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
                     }
                 }
@@ -603,7 +642,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_wgrad_tc_kernel(const TcWg
     __syncthreads();
     if (warp == 1) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(p.tmem_cols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(tmem_cols) : "memory");
     }
 }
 
@@ -677,24 +716,36 @@ static bool encode_flat(CUtensorMap* m, const void* base, int chan, long long pi
     const uint64_t dims[2] = {(uint64_t)chan, (uint64_t)pixels}; const uint64_t st[1] = {(uint64_t)chan * 2}; const uint32_t box[2] = {64, 128};
     return encode_map(m, base, 2, dims, st, box);
 }
-// [n_img][H][W][chan] as (channel, x, y, image): a box is R rows of Wp window positions, every es-th pixel in x and y
-static bool encode_tall(CUtensorMap* m, const void* base, int chan, int n_img, int H, int W, int Wp, int R, int es) {
+// [n_img][H][W][chan] as (channel, x, y, image): a box is box_h rows of Wp window positions of box_n images, every es-th pixel in x and y
+static bool encode_tall(CUtensorMap* m, const void* base, int chan, int n_img, int H, int W, int Wp, int box_h, int box_n, int es) {
     const uint64_t dims[4] = {(uint64_t)chan, (uint64_t)W, (uint64_t)H, (uint64_t)n_img};
     const uint64_t st[3] = {(uint64_t)chan * 2, (uint64_t)chan * 2 * W, (uint64_t)chan * 2 * W * H};
-    const uint32_t box[4] = {64, (uint32_t)(Wp * es), (uint32_t)(R * es), 1};
+    const uint32_t box[4] = {64, (uint32_t)(Wp * es), (uint32_t)(box_h * es), (uint32_t)box_n};
     const uint32_t estr[4] = {1, (uint32_t)es, (uint32_t)es, 1};
     return encode_map(m, base, 4, dims, st, box, estr);
 }
 
-// rows of the tall map fetched by one box: the largest divisor of Hp whose box holds at most 64 positions (and fits a TMA box)
-static int box_rows(int Hp, int Wp, int es) { int best = 1; for (int r = 1; r <= Hp; ++r) if (Hp % r == 0 && r * Wp <= 64 && r * es <= 256) best = r; return best; }
-
-// The tall map of a grid of Hg x Wg positions per image
-struct Tall { int Hp, Wp, R, box_pos, box_bytes; };
+// The tall map of a grid of Hg x Wg positions per image: Wp = Wg + pad positions per row, Hp rows per image (Hg + pad, rounded up
+// to a multiple of the rows of a box: the extra rows read as zero like the padding).  A box is R consecutive tall rows: part of
+// one image (R divides Hp), or box_n whole images.  Larger boxes mean fewer TMA issues per window but more rows fetched around it;
+// the choice: at most 96 positions per box, at most 6.5 % of extra rows, then the largest box.
+struct Tall { int Hp, Wp, R, box_pos, box_bytes, box_h, box_n; };
 static bool tall_of(int Hg, int Wg, int pad, int es, Tall& t) {
-    t.Hp = Hg + pad; t.Wp = Wg + pad;
+    t.Wp = Wg + pad;
+    const int H0 = Hg + pad;
     if (t.Wp * es > 256) return false;
-    t.R = box_rows(t.Hp, t.Wp, es); t.box_pos = t.R * t.Wp; t.box_bytes = t.box_pos * 128;
+    int best_r = 1, best_hp = H0;
+    for (int r = 1; r <= H0; ++r) {
+        const int hp = (H0 + r - 1) / r * r;
+        if (r * t.Wp > 96 || r * es > 256 || (hp - H0) * 200 > 13 * H0 || (pad == 0 && hp != H0)) continue;   // pad = 0: positions are the pixels in order, no extra rows
+        if (r * t.Wp > best_r * t.Wp) { best_r = r; best_hp = hp; }
+    }
+    t.Hp = best_hp; t.R = best_r; t.box_h = best_r; t.box_n = 1;
+    if (best_r == best_hp) {                      // whole images: several per box when they are small
+        int ni = 96 / (t.Hp * t.Wp); if (ni < 1) ni = 1; if (ni > 8) ni = 8;
+        t.box_n = ni; t.R = t.Hp * ni;
+    }
+    t.box_pos = t.R * t.Wp; t.box_bytes = t.box_pos * 128;
     return true;
 }
 static int boxes_for(int span, int box_pos) { return (span + 2 * (box_pos - 1)) / box_pos; }   // boxes that cover `span` positions from any start
@@ -727,9 +778,9 @@ int conv_tc_count(const ConvProb& p, int mode) {
 bool conv_tc_supported(const ConvProb& p, int mode) { return conv_tc_count(p, mode) > 0; }
 // 128-position tiles of a forward problem (the rows of ConvProb::stat_tiles)
 int conv_tc_stat_tiles(const ConvProb& p) {
-    long long pos;
-    if (p.ksz == 1) pos = (long long)p.N * p.P * p.Q;
-    else pos = (long long)p.N * (p.P + 1) * (p.Q + 1);
+    long long pos = (long long)p.N * p.P * p.Q;
+    if (p.ksz == 1 && p.stride == 2) { Tall g; tall_of(p.P, p.Q, 0, 2, g); pos = (long long)p.N * g.Hp * g.Wp; }
+    if (p.ksz != 1) { Tall g; tall_of(p.P, p.Q, 1, p.stride, g); pos = (long long)p.N * g.Hp * g.Wp; }
     return (int)((pos + TILE_M - 1) / TILE_M);
 }
 
@@ -752,7 +803,7 @@ int conv_tc_fill(const ConvProb& p, int mode, void* host_tc) {
     const int taps = p.ksz * p.ksz;
     const int chan_a = mode == CONV_FWD ? p.C : p.K, ncol = mode == CONV_FWD ? p.K : p.C;
     for (int ph = 0; ph < count; ++ph) {
-        TcProb t; memset(&t, 0, sizeof(t));
+        TcProb tp; memset(&tp, 0, sizeof(tp)); TcHot& t = tp.h;
         t.add = (const __nv_bfloat16*)p.add; t.out = (__nv_bfloat16*)p.out; t.status = conv_tc_status_word();
         t.stat_tiles = mode == CONV_FWD ? p.stat_tiles : nullptr;
         t.n_img = p.N; t.ncol = ncol; t.red = chan_a; t.slabs = (chan_a + 63) / 64; t.scale = p.scale;
@@ -765,8 +816,8 @@ int conv_tc_fill(const ConvProb& p, int mode, void* host_tc) {
             const int Hg = mode == CONV_DGRAD ? p.P : p.H, Wg = mode == CONV_DGRAD ? p.Q : p.W;
             t.a_flat = 1; t.Hp = Hg; t.Wp = Wg; t.R = 0; t.box_pos = TILE_M; t.nbox = 1; t.hb = 0; t.a_box_bytes = SLAB_BYTES;
             t.total_pos = p.N * Hg * Wg;
-            t.taps[0] = TapRef{0, 0}; t.gbeg[1] = 1;
-            if (!encode_flat(&t.map_a, act, chan_a, t.total_pos)) return 0;
+            { const int ti_ = 0; t.wtap[ti_] = 0; t.shift[ti_] = 0; } t.gbeg[1] = 1;
+            if (!encode_flat(&tp.map_a, act, chan_a, t.total_pos)) return 0;
             if (p.stride == 2 && !p.out_compact) { t.dense = 0; t.OH = p.H; t.OW = p.W; t.os = 2; out_pixels = (long long)p.N * p.H * p.W; }   // scattered to the even positions
             else { t.dense = 1; t.OH = Hg; t.OW = Wg; out_pixels = t.total_pos; }
         } else if (p.ksz == 1) {
@@ -774,16 +825,16 @@ int conv_tc_fill(const ConvProb& p, int mode, void* host_tc) {
             Tall g; if (!tall_of(p.P, p.Q, 0, 2, g)) return 0;
             t.a_flat = 0; t.dense = 1; t.es = 2; t.Hp = g.Hp; t.Wp = g.Wp; t.R = g.R; t.box_pos = g.box_pos; t.a_box_bytes = g.box_bytes; t.hb = 0;
             t.nbox = boxes_for(TILE_M, g.box_pos); t.total_pos = p.N * g.Hp * g.Wp; t.OH = p.P; t.OW = p.Q; out_pixels = t.total_pos;
-            t.taps[0] = TapRef{0, 0}; t.gbeg[1] = 1;
-            if (!encode_tall(&t.map_a, act, chan_a, p.N, p.H, p.W, g.Wp, g.R, 2)) return 0;
+            { const int ti_ = 0; t.wtap[ti_] = 0; t.shift[ti_] = 0; } t.gbeg[1] = 1;
+            if (!encode_tall(&tp.map_a, act, chan_a, p.N, p.H, p.W, g.Wp, g.box_h, g.box_n, 2)) return 0;
         } else if (p.stride == 1) {
             // 3x3 at stride 1: one window, nine taps; dgrad walks the taps mirrored
             Tall g; if (!tall_of(p.H, p.W, 1, 1, g)) return 0;
             t.a_flat = 0; t.dense = 0; t.pad = 1; t.Hp = g.Hp; t.Wp = g.Wp; t.R = g.R; t.box_pos = g.box_pos; t.a_box_bytes = g.box_bytes; t.hb = g.Wp + 1;
             t.nbox = boxes_for(TILE_M + 2 * t.hb, g.box_pos); t.total_pos = p.N * g.Hp * g.Wp; t.OH = p.H; t.OW = p.W; out_pixels = (long long)p.N * p.H * p.W;
-            for (int w = 0; w < 9; ++w) t.taps[w] = TapRef{mode == CONV_DGRAD ? 8 - w : w, (w / 3) * g.Wp + (w % 3)};
+            for (int w = 0; w < 9; ++w) { const int ti_ = w; t.wtap[ti_] = mode == CONV_DGRAD ? 8 - w : w; t.shift[ti_] = (w / 3) * g.Wp + (w % 3); }
             t.gbeg[1] = 9;
-            if (!encode_tall(&t.map_a, act, chan_a, p.N, p.H, p.W, g.Wp, g.R, 1)) return 0;
+            if (!encode_tall(&tp.map_a, act, chan_a, p.N, p.H, p.W, g.Wp, g.box_h, g.box_n, 1)) return 0;
         } else if (mode == CONV_FWD) {
             // 3x3 at stride 2, forward: positions over the P x Q outputs, one window per input parity phase (element-strided fetch)
             Tall g; if (!tall_of(p.P, p.Q, 1, 2, g)) return 0;
@@ -795,11 +846,11 @@ int conv_tc_fill(const ConvProb& p, int mode, void* host_tc) {
                 t.gxs[t.ngroups] = v; t.gys[t.ngroups] = u;
                 for (int i = 0; i < k; ++i) {
                     const int di = rs[i][0] == 0 ? -1 : 0, dj = rs[i][1] == 0 ? -1 : 0;    // tap 0 reads the previous phase row / column
-                    t.taps[n++] = TapRef{rs[i][0] * 3 + rs[i][1], t.hb + di * g.Wp + dj};
+                    { const int ti_ = n++; t.wtap[ti_] = rs[i][0] * 3 + rs[i][1]; t.shift[ti_] = t.hb + di * g.Wp + dj; }
                 }
                 t.gbeg[++t.ngroups] = n;
             }
-            if (!encode_tall(&t.map_a, act, chan_a, p.N, p.H, p.W, g.Wp, g.R, 2)) return 0;
+            if (!encode_tall(&tp.map_a, act, chan_a, p.N, p.H, p.W, g.Wp, g.box_h, g.box_n, 2)) return 0;
         } else {
             // 3x3 at stride 2, dgrad: one problem per output parity phase (u, v), positions over the P x Q grid of dy; input row 2i + u
             // takes dy row i + (u + 1 - r) / 2 through tap r
@@ -809,9 +860,9 @@ int conv_tc_fill(const ConvProb& p, int mode, void* host_tc) {
             t.nbox = boxes_for(TILE_M + g.Wp + 1, g.box_pos); t.total_pos = p.N * g.Hp * g.Wp;
             t.OH = p.H; t.OW = p.W; t.os = 2; t.oy = u; t.ox = v; out_pixels = (long long)p.N * p.H * p.W;
             int rs[4][2]; const int k = phase_taps(u, v, rs);
-            for (int i = 0; i < k; ++i) t.taps[i] = TapRef{rs[i][0] * 3 + rs[i][1], ((u + 1 - rs[i][0]) / 2) * g.Wp + (v + 1 - rs[i][1]) / 2};
+            for (int i = 0; i < k; ++i) { const int ti_ = i; t.wtap[ti_] = rs[i][0] * 3 + rs[i][1]; t.shift[ti_] = ((u + 1 - rs[i][0]) / 2) * g.Wp + (v + 1 - rs[i][1]) / 2; }
             t.gbeg[1] = k;
-            if (!encode_tall(&t.map_a, act, chan_a, p.N, p.P, p.Q, g.Wp, g.R, 1)) return 0;
+            if (!encode_tall(&tp.map_a, act, chan_a, p.N, p.P, p.Q, g.Wp, g.box_h, g.box_n, 1)) return 0;
         }
         // residual
         t.add_mode = !p.add ? 0 : p.add_sub == 2 ? 3 : t.dense ? 1 : 2;
@@ -829,20 +880,20 @@ int conv_tc_fill(const ConvProb& p, int mode, void* host_tc) {
         { const uint64_t dims[3] = {(uint64_t)p.C, (uint64_t)taps, (uint64_t)p.K};
           const uint64_t st[2] = {(uint64_t)p.C * 2, (uint64_t)taps * p.C * 2};
           const uint32_t box[3] = {64, 1, mode == CONV_FWD ? (uint32_t)t.n_tile : 64u};
-          if (!encode_map(&t.map_b, p.wgt, 3, dims, st, box)) return 0; }
+          if (!encode_map(&tp.map_b, p.wgt, 3, dims, st, box)) return 0; }
         if (t.dense) {
-            if (!encode_flat(&t.map_out, p.out, ncol, out_pixels)) return 0;
-            if (t.add_mode == 1 && !encode_flat(&t.map_add, p.add, ncol, out_pixels)) return 0;
+            if (!encode_flat(&tp.map_out, p.out, ncol, out_pixels)) return 0;
+            if (t.add_mode == 1 && !encode_flat(&tp.map_add, p.add, ncol, out_pixels)) return 0;
         }
-        memcpy((char*)host_tc + (size_t)ph * sizeof(TcProb), &t, sizeof(t));
+        memcpy((char*)host_tc + (size_t)ph * sizeof(TcProb), &tp, sizeof(tp));
     }
     return count;
 }
 size_t conv_tc_prob_bytes() { return sizeof(TcProb); }
-int conv_tc_tiles(const void* host_tc) { const TcProb* t = (const TcProb*)host_tc; return t->tiles_m * t->tiles_n; }
+int conv_tc_tiles(const void* host_tc) { const TcHot* t = &((const TcProb*)host_tc)->h; return t->tiles_m * t->tiles_n; }
 // packs what a launch has to know about its largest problem into one number: window KB, weight-tile KB, staging tiles, MMA N
 size_t conv_tc_smem(const void* host_tc) {
-    const TcProb* t = (const TcProb*)host_tc;
+    const TcHot* t = &((const TcProb*)host_tc)->h;
     const size_t a_stage = ((size_t)t->nbox * t->a_box_bytes + 1023) / 1024, b_stage = ((size_t)t->b_bytes + 1023) / 1024;
     return (a_stage << 48) | (b_stage << 32) | ((size_t)(t->add_mode == 1 ? 2 : 1) << 24) | (size_t)t->n_tile;
 }
@@ -852,7 +903,7 @@ size_t conv_tc_merge(size_t a, size_t b) {
            (std::max((a >> 24) & 0xFF, (b >> 24) & 0xFF) << 24) | std::max(a & 0xFFFFFF, b & 0xFFFFFF);
 }
 
-constexpr size_t TC_SMEM_BUDGET = 200 * 1024;
+constexpr size_t TC_SMEM_BUDGET = 212 * 1024;
 
 // total_tiles: an upper bound of the tiles of all problems of the launch (max_tiles * nprob); packed: conv_tc_merge over its problems
 void launch_conv_tc_probs(const void* d_tc, int nprob, int max_tiles, size_t packed, cudaStream_t s) {
@@ -868,15 +919,15 @@ void launch_conv_tc_probs(const void* d_tc, int nprob, int max_tiles, size_t pac
     L.n_stg = (int)((packed >> 24) & 0xFF);
     const int n_tile = (int)(packed & 0xFFFFFF);
     L.stg_bytes = ((n_tile + 63) / 64) * SLAB_BYTES;
+    // Shared memory: with a prefetched residual three staging tiles (two residual tiles in flight behind the one the epilogue works
+    // on), else one; three weight tiles; the rest goes to the ring of activation windows: an HBM-bound layer runs at the bytes it
+    // keeps in flight
+    if (L.n_stg > 1) L.n_stg = 3;
+    while (L.n_stg > 1 && (size_t)L.n_stg * L.stg_bytes + 2 * (size_t)(L.a_stage + L.b_stage) > TC_SMEM_BUDGET) --L.n_stg;
     const size_t rings = TC_SMEM_BUDGET - (size_t)L.n_stg * L.stg_bytes;
-    // ring depths: up to 4 windows and up to 6 weight tiles within the budget, at least 2 of each
-    L.na = 2; L.nb = 2;
-    while (true) {
-        bool grown = false;
-        if (L.nb < TC_MAX_STAGES && (size_t)L.na * L.a_stage + (size_t)(L.nb + 1) * L.b_stage <= rings) { ++L.nb; grown = true; }
-        if (L.na < 4 && (size_t)(L.na + 1) * L.a_stage + (size_t)L.nb * L.b_stage <= rings) { ++L.na; grown = true; }
-        if (!grown) break;
-    }
+    L.nb = 3; while (L.nb > 2 && (size_t)L.nb * L.b_stage + 2 * (size_t)L.a_stage > rings) --L.nb;
+    L.na = 2; while (L.na < TC_MAX_STAGES && (size_t)(L.na + 1) * L.a_stage + (size_t)L.nb * L.b_stage <= rings) ++L.na;
+    while (L.nb < 6 && (size_t)L.na * L.a_stage + (size_t)(L.nb + 1) * L.b_stage <= rings) ++L.nb;
     L.acc_stride = (n_tile + 31) / 32 * 32;
     L.tmem_cols = 32; while (L.tmem_cols < 2 * L.acc_stride) L.tmem_cols *= 2;
     // at least 120 KB of shared memory so that two CTAs that allocate tensor memory never share an SM
@@ -887,7 +938,7 @@ void launch_conv_tc_probs(const void* d_tc, int nprob, int max_tiles, size_t pac
 }
 
 // ---- wgrad host side
-struct WgGeom { TcWgradProb t; size_t smem, partial_bytes; };
+struct WgGeom { TcWgradProb t; size_t smem, partial_bytes; int box_h, box_n; };
 
 static bool wg_geometry(const ConvProb& p, int target_ctas, WgGeom& w) {
     if (!tc_shape_ok(p)) return false;
@@ -903,12 +954,14 @@ static bool wg_geometry(const ConvProb& p, int target_ctas, WgGeom& w) {
     } else if (p.ksz == 1) {
         // stride-2 1x1: the positions are the P x Q pixels of dy in order; a is gathered at every second pixel
         Tall g; if (!tall_of(p.P, p.Q, 0, 2, g)) return false;
+        w.box_h = g.box_h; w.box_n = g.box_n;
         t.dy_flat = 1; t.a_flat = 0; t.es = 2; t.Hp = g.Hp; t.Wp = g.Wp; t.R = g.R; t.box_pos = g.box_pos; t.hb = 0;
         t.nbox_dy = 1; t.dy_box_bytes = SLAB_BYTES; t.nbox_a = boxes_for(TILE_M, g.box_pos); t.a_box_bytes = g.box_bytes;
         total_pos = (long long)p.N * g.Hp * g.Wp;
         t.tap_groups = 1; t.gbeg[1] = 1; t.tap[0] = TapRef{0, 0};
     } else if (p.stride == 1) {
         Tall g; if (!tall_of(p.H, p.W, 1, 1, g)) return false;
+        w.box_h = g.box_h; w.box_n = g.box_n;
         t.dy_flat = 0; t.a_flat = 0; t.pad = 1; t.Hp = g.Hp; t.Wp = g.Wp; t.R = g.R; t.box_pos = g.box_pos; t.hb = g.Wp + 1;
         t.nbox_dy = boxes_for(TILE_M, g.box_pos); t.nbox_a = boxes_for(TILE_M + 2 * t.hb, g.box_pos); t.dy_box_bytes = g.box_bytes; t.a_box_bytes = g.box_bytes;
         total_pos = (long long)p.N * g.Hp * g.Wp;
@@ -917,7 +970,8 @@ static bool wg_geometry(const ConvProb& p, int target_ctas, WgGeom& w) {
     } else {
         Tall g; if (!tall_of(p.P, p.Q, 1, 2, g)) return false;
         Tall gd; if (!tall_of(p.P, p.Q, 1, 1, gd)) return false;
-        if (gd.R != g.R) { g.R = gd.R = 1; g.box_pos = gd.box_pos = g.Wp; g.box_bytes = gd.box_bytes = g.Wp * 128; }   // both operands use the same boxes of rows
+        if (gd.R != g.R || gd.Hp != g.Hp) return false;          // both operands walk the same boxes of rows
+        w.box_h = g.box_h; w.box_n = g.box_n;
         t.dy_flat = 0; t.a_flat = 0; t.pad = 1; t.es = 2; t.Hp = g.Hp; t.Wp = g.Wp; t.R = g.R; t.box_pos = g.box_pos; t.hb = g.Wp + 1;
         t.nbox_dy = boxes_for(TILE_M, g.box_pos); t.nbox_a = boxes_for(TILE_M + t.hb, g.box_pos); t.dy_box_bytes = g.box_bytes; t.a_box_bytes = g.box_bytes;
         total_pos = (long long)p.N * g.Hp * g.Wp;
@@ -966,9 +1020,9 @@ bool conv_wgrad_tc_fill(const ConvProb& p, int target_ctas, void* host_tc) {
     WgGeom g; if (!wg_geometry(p, target_ctas, g)) return false;
     TcWgradProb& t = g.t;
     if (t.dy_flat) { if (!encode_flat(&t.map_dy, p.wgt, p.K, (long long)p.N * p.P * p.Q)) return false; }
-    else if (!encode_tall(&t.map_dy, p.wgt, p.K, p.N, p.P, p.Q, t.Wp, t.R, 1)) return false;
+    else if (!encode_tall(&t.map_dy, p.wgt, p.K, p.N, p.P, p.Q, t.Wp, g.box_h, g.box_n, 1)) return false;
     if (t.a_flat) { if (!encode_flat(&t.map_a, p.act, p.C, (long long)p.N * p.H * p.W)) return false; }
-    else if (!encode_tall(&t.map_a, p.act, p.C, p.N, p.H, p.W, t.Wp, t.R, t.es)) return false;
+    else if (!encode_tall(&t.map_a, p.act, p.C, p.N, p.H, p.W, t.Wp, g.box_h, g.box_n, t.es)) return false;
     t.partial = p.partial; t.out = (float*)p.out; t.status = conv_tc_status_word();
     memcpy(host_tc, &t, sizeof(t));
     return true;
