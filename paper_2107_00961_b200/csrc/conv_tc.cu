@@ -94,20 +94,27 @@ __device__ __forceinline__ int floor_div(int a, int b) { int q = a / b; if ((a %
 __device__ __forceinline__ void tma_store_2d(const void* tmap, uint32_t src, int c0, int c1) {
     asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(tmap), "r"(src), "r"(c0), "r"(c1) : "memory");
 }
-__device__ __forceinline__ void bar_sync_epi() { asm volatile("bar.sync 1, 128;" ::: "memory"); }   // the four epilogue warps
-__device__ __forceinline__ bool bar_and_epi(bool v) {             // barrier of the four epilogue warps that also ANDs a flag
+__device__ __forceinline__ void bar_sync_epi(int id) { asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory"); }   // the four warps of one epilogue group
+__device__ __forceinline__ bool bar_and_epi(int id, bool v) {     // barrier of the four warps of an epilogue group that also ANDs a flag
     uint32_t r;
-    asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.u32 p, %1, 0;\n\tbar.red.and.pred q, 1, 128, p;\n\tselp.u32 %0, 1, 0, q;\n\t}" : "=r"(r) : "r"((uint32_t)v) : "memory");
+    asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.u32 p, %2, 0;\n\tbar.red.and.pred q, %1, 128, p;\n\tselp.u32 %0, 1, 0, q;\n\t}" : "=r"(r) : "r"(id), "r"((uint32_t)v) : "memory");
     return r != 0;
+}
+__device__ __forceinline__ void bulk_wait_read(int pending) {     // at most `pending` of this thread's latest bulk stores may still be reading shared memory
+    if (pending <= 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+    else if (pending == 1) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+    else asm volatile("cp.async.bulk.wait_group.read 2;" ::: "memory");
 }
 __device__ __forceinline__ uint4 lds128(uint32_t a) { uint4 v; asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a)); return v; }
 __device__ __forceinline__ void sts128(uint32_t a, uint4 v) { asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory"); }
 __device__ __forceinline__ uint32_t lds32(uint32_t a) { uint32_t v; asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(a)); return v; }
 
-constexpr int TC_THREADS = 192;
+constexpr int TC_THREADS = 192;              // wgrad kernel: producer warp, MMA warp, four epilogue warps
+constexpr int TC_CONV_THREADS = 320;         // forward / dgrad kernel: producer warp, MMA warp, two groups of four epilogue warps
 constexpr int TC_MAX_STAGES = 12;
 constexpr int TILE_M = 128;
 constexpr int SLAB_BYTES = TILE_M * 128;      // 128 rows x 64 channels of bf16
+constexpr size_t TC_RESIDENT_BUDGET = 96 * 1024;   // weights of one column tile that may stay in shared memory
 
 struct TapRef { int wtap; int shift; };       // weight tap index (r*ksz + s); row shift of the operand inside the window
 // One forward / dgrad problem.  The tensor maps come first so that each is 64-byte aligned.
@@ -135,6 +142,7 @@ struct TcHot {                // everything the kernel's loops read: each role k
     int red, slabs;                          // reduction channels, 64-channel slabs
     int b_mn_major;                          // 0: forward (weights K-major); 1: dgrad (weights MN-major)
     int b_bytes;                             // bytes of one weight tile (one slab, one tap)
+    int b_total;                             // bytes of all weight tiles of one column tile, each rounded up to 1 KB
     int out_slabs;                           // 64-column slabs of the output tile
     int total_pos;
     float scale;
@@ -149,7 +157,8 @@ struct alignas(64) TcProb {
 };
 static_assert(sizeof(TcHot) % 4 == 0, "copied word by word");
 
-struct TcLaunch { int nprob, na, nb, a_stage, b_stage, tmem_cols, acc_stride, n_stg, stg_bytes; };
+struct TcLaunch { int nprob, na, nb, a_stage, b_stage, tmem_cols, acc_stride, n_stg, stg_bytes, b_res, b_region, groups, pg, prefetch; };   // b_res: the weights of a (problem, column tile) stay in shared memory; b_region: bytes of the weight ring or of the resident weights;
+// groups: epilogue groups (they take alternate tiles); pg: staging tiles per group (n_stg = groups * pg); prefetch: some problem's residual is fetched by TMA
 constexpr int TC_MAX_PROBS = 128;             // descriptors per launch (sub-ResNets x output phases)
 
 __device__ __forceinline__ void copy_hot(TcHot* dst, const TcHot* src, int tid, int nthreads) {
@@ -157,21 +166,22 @@ __device__ __forceinline__ void copy_hot(TcHot* dst, const TcHot* src, int tid, 
     for (int i = tid; i < (int)(sizeof(TcHot) / 4); i += nthreads) d4[i] = __ldg(s4 + i);
 }
 
-__global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const TcProb* __restrict__ probs, const TcLaunch L) {
+__global__ void __launch_bounds__(TC_CONV_THREADS, 1) conv_tc_kernel(const TcProb* __restrict__ probs, const TcLaunch L) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    __shared__ __align__(8) uint64_t bars[4 * TC_MAX_STAGES + 12];
+    __shared__ __align__(8) uint64_t bars[4 * TC_MAX_STAGES + 14];
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
-    __shared__ int pix_s[TILE_M];
-    __shared__ float stat_s[4][2][256];
+    __shared__ int pix_s2[2][TILE_M];
+    __shared__ float stat_s2[2][4][2][256];
     __shared__ int tile_end_s[TC_MAX_PROBS];                      // running sum of the problems' tile counts
-    __shared__ TcHot hot_s[3];                                    // the current problem of the producer, the MMA issuer, the epilogue
+    __shared__ TcHot hot_s[4];                                    // the current problem of the producer, the MMA issuer, the two epilogue groups
     const uint32_t a_full = smem_u32(&bars[0]), a_empty = smem_u32(&bars[TC_MAX_STAGES]);
     const uint32_t b_full = smem_u32(&bars[2 * TC_MAX_STAGES]), b_empty = smem_u32(&bars[3 * TC_MAX_STAGES]);
     const uint32_t acc_full = smem_u32(&bars[4 * TC_MAX_STAGES]), acc_empty = smem_u32(&bars[4 * TC_MAX_STAGES + 2]);
     const uint32_t add_full = smem_u32(&bars[4 * TC_MAX_STAGES + 4]), stg_free = smem_u32(&bars[4 * TC_MAX_STAGES + 8]);
-    const uint32_t a_ring = smem_u32(smem), b_ring = a_ring + (uint32_t)(L.na * L.a_stage), stg_base = b_ring + (uint32_t)(L.nb * L.b_stage);
+    const uint32_t bres_full = smem_u32(&bars[4 * TC_MAX_STAGES + 12]), bres_empty = smem_u32(&bars[4 * TC_MAX_STAGES + 13]);
+    const uint32_t a_ring = smem_u32(smem), b_ring = a_ring + (uint32_t)(L.na * L.a_stage), stg_base = b_ring + (uint32_t)L.b_region;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
@@ -180,6 +190,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const TcProb* __
         }
         for (int s = 0; s < 2; ++s) { mbar_init(acc_full + 8 * s, 1); mbar_init(acc_empty + 8 * s, 4); }
         for (int s = 0; s < 4; ++s) { mbar_init(add_full + 8 * s, 1); mbar_init(stg_free + 8 * s, 1); }
+        mbar_init(bres_full, 1); mbar_init(bres_empty, 1);
         abort_s = 0;
         int run = 0;
         for (int i = 0; i < L.nprob; ++i) { run += probs[i].h.tiles_m * probs[i].h.tiles_n; tile_end_s[i] = run; }
@@ -193,7 +204,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const TcProb* __
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = tmem_base_s;
-    const int total_tiles = tile_end_s[L.nprob - 1];
+    // The tiles of all problems, column tile innermost, are dealt round-robin: the CTAs that run side by side work on neighbouring
+    // tiles, share activation windows and weight tiles in L2 and read HBM as one moving front.  (Contiguous runs per CTA, with the
+    // column tile outermost, were measured too: no faster, and slower for the layers whose weights stream.)
+    const int t_begin = (int)blockIdx.x, t_stop = tile_end_s[L.nprob - 1], t_step = (int)gridDim.x;
 
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer
@@ -201,17 +215,34 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const TcProb* __
             uint32_t a_cnt = 0, b_cnt = 0, seq = 0, add_use[4] = {0u, 0u, 0u, 0u}; bool ok = true;
             int cur = -1; TcHot& h = hot_s[0];
             int sa = 0, sb_ = 0; uint32_t pha = 0, phb = 0;       // ring positions and phases
-            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++seq) {
+            int cur_unit = -1; uint32_t unit_cnt = 0;
+            for (int t = t_begin; t < t_stop && ok; t += t_step, ++seq) {
                 int pi = 0; while (t >= tile_end_s[pi]) ++pi;
                 if (pi != cur) { copy_hot(&h, &probs[pi].h, 0, 1); cur = pi; }
                 const TcProb* pp = probs + pi;
                 const int loc = t - (pi ? tile_end_s[pi - 1] : 0);
-                const int tiles_n = h.tiles_n, n_tile = h.n_tile, slabs = h.slabs, ngroups = h.ngroups, a_flat = h.a_flat, nbox = h.nbox,
+                const int n_tile = h.n_tile, slabs = h.slabs, ngroups = h.ngroups, a_flat = h.a_flat, nbox = h.nbox,
                           a_box_bytes = h.a_box_bytes, R = h.R, Hp = h.Hp, pad = h.pad, es = h.es, b_bytes = h.b_bytes, mn = h.b_mn_major;
-                const int tn = loc % tiles_n, tm = loc / tiles_n;
+                const int tiles_n = h.tiles_n, tn = loc % tiles_n, tm = loc / tiles_n;
+                if (L.b_res && (pi << 8 | tn) != cur_unit) {
+                    // new (problem, column tile): all its weight tiles go to the resident region, once the MMAs of the last one have read theirs
+                    if (!mbar_wait(bres_empty, (unit_cnt & 1u) ^ 1u, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(h.status, 8); ok = false; break; }
+                    const int ntaps = h.gbeg[ngroups];
+                    mbar_expect_tx(bres_full, (uint32_t)(slabs * ntaps * b_bytes));
+                    for (int sl = 0; sl < slabs; ++sl)
+                        for (int tap = 0; tap < ntaps; ++tap) {
+                            const uint32_t dst = b_ring + (uint32_t)((sl * ntaps + tap) * ((b_bytes + 1023) & ~1023));
+                            const int wtap = h.wtap[tap];
+                            if (!mn) tma_load_3d(dst, &pp->map_b, bres_full, sl * 64, wtap, tn * n_tile);
+                            else for (int j = 0; j * 64 < n_tile; ++j)
+                                tma_load_3d(dst + (uint32_t)(j * 8192), &pp->map_b, bres_full, tn * n_tile + j * 64, wtap, sl * 64);
+                        }
+                    ++unit_cnt; cur_unit = pi << 8 | tn;
+                }
                 if (h.add_mode == 1) {
                     // the residual tile goes straight into the staging tile the epilogue will finish in place
-                    const uint32_t sb = seq % (uint32_t)L.n_stg, uses = seq / (uint32_t)L.n_stg;
+                    const uint32_t grp = L.groups == 2 ? (seq & 1u) : 0u, kk = L.groups == 2 ? (seq >> 1) : seq;
+                    const uint32_t sb = grp * (uint32_t)L.pg + kk % (uint32_t)L.pg, uses = kk / (uint32_t)L.pg;
                     if (!mbar_wait(stg_free + 8 * sb, (uses & 1u) ^ 1u, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(h.status, 7); ok = false; break; }
                     mbar_expect_tx(add_full + 8 * sb, (uint32_t)(h.out_slabs * SLAB_BYTES));
                     for (int j = 0; j < h.out_slabs; ++j)
@@ -235,7 +266,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const TcProb* __
                             }
                             ++a_cnt; if (++sa == L.na) { sa = 0; pha ^= 1u; }
                         }
-                        const int t_end = h.gbeg[g + 1];
+                        const int t_end = L.b_res ? 0 : h.gbeg[g + 1];
                         for (int tap = h.gbeg[g]; tap < t_end; ++tap) {
                             if (!mbar_wait(b_empty + 8 * sb_, phb ^ 1u, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(h.status, 2); ok = false; break; }
                             const uint32_t dst = b_ring + (uint32_t)(sb_ * L.b_stage);
@@ -265,14 +296,21 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const TcProb* __
             uint32_t acc_cnt = 0; bool ok = true;
             int cur = -1; TcHot& h = hot_s[1];
             int sa = 0, sb = 0; uint32_t pha = 0, phb = 0;
+            int cur_unit = -1; uint32_t unit_cnt = 0;
             // the constant part of a 128-byte-swizzle descriptor: stride between 8-row groups 1024 bytes, version, swizzle mode
             const uint64_t desc_k = desc_sw128(0, 16, 1024), desc_mn = desc_sw128(0, 8192, 1024);
-            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++acc_cnt) {
+            for (int t = t_begin; t < t_stop && ok; t += t_step, ++acc_cnt) {
                 int pi = 0; while (t >= tile_end_s[pi]) ++pi;
                 if (pi != cur) { copy_hot(&h, &probs[pi].h, 0, 1); cur = pi; }
                 const int loc = t - (pi ? tile_end_s[pi - 1] : 0);
                 const int slabs = h.slabs, ngroups = h.ngroups, red = h.red, mn = h.b_mn_major;
-                const int tm = loc / h.tiles_n;
+                const int tiles_n = h.tiles_n, tn = loc % tiles_n, tm = loc / tiles_n;
+                const int ntaps = h.gbeg[ngroups], b_stride = (h.b_bytes + 1023) & ~1023;
+                if (L.b_res && (pi << 8 | tn) != cur_unit) {
+                    if (!mbar_wait(bres_full, unit_cnt & 1u, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(h.status, 9); ok = false; break; }
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    ++unit_cnt; cur_unit = pi << 8 | tn;
+                }
                 const int bx0 = h.a_flat ? 0 : floor_div(tm * TILE_M - h.hb, h.box_pos);
                 const int a_off = h.a_flat ? 0 : tm * TILE_M - h.hb - bx0 * h.box_pos;
                 const uint32_t buf = acc_cnt & 1u, aph = (acc_cnt >> 1) & 1u;
@@ -294,49 +332,72 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const TcProb* __
                         const int t_end = h.gbeg[g + 1];
                         for (int tap = h.gbeg[g]; tap < t_end; ++tap) {
                             const uint32_t a16 = a_rows16 + (uint32_t)h.shift[tap] * 8u;
-                            if (!mbar_wait(b_full + 8 * sb, phb, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(h.status, 5); ok = false; break; }
-                            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                            const uint32_t b16 = (b_ring + (uint32_t)(sb * L.b_stage)) >> 4;
+                            uint32_t b16;
+                            if (L.b_res) b16 = (b_ring + (uint32_t)((sl * ntaps + tap) * b_stride)) >> 4;
+                            else {
+                                if (!mbar_wait(b_full + 8 * sb, phb, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(h.status, 5); ok = false; break; }
+                                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                                b16 = (b_ring + (uint32_t)(sb * L.b_stage)) >> 4;
+                            }
                             for (int k16 = 0; k16 < ksteps; ++k16) {
                                 umma_bf16(d_tmem, desc_k | (uint64_t)((a16 + 2u * (uint32_t)k16) & 0x3FFFu), b_const | (uint64_t)((b16 + b_step * (uint32_t)k16) & 0x3FFFu), idesc, acc);
                                 acc = 1;
                             }
-                            umma_commit(b_empty + 8 * sb);       // weight tile reusable once these MMAs have read it
-                            if (++sb == L.nb) { sb = 0; phb ^= 1u; }
+                            if (!L.b_res) {
+                                umma_commit(b_empty + 8 * sb);   // weight tile reusable once these MMAs have read it
+                                if (++sb == L.nb) { sb = 0; phb ^= 1u; }
+                            }
                         }
                         umma_commit(a_empty + 8 * sa);
                         if (++sa == L.na) { sa = 0; pha ^= 1u; }
                     }
                 }
                 if (ok) umma_commit(acc_full + 8 * buf);         // accumulator complete
+                if (ok && L.b_res) {
+                    // last tile of this (problem, column tile) for this CTA: the resident weights may be replaced once these MMAs are done
+                    bool last = t + t_step >= t_stop;
+                    if (!last) { const int t2 = t + t_step; int pn = pi; while (t2 >= tile_end_s[pn]) ++pn; const int l2 = t2 - (pn ? tile_end_s[pn - 1] : 0);
+                        last = pn != pi || l2 % tiles_n != tn; }
+                    if (last) umma_commit(bres_empty);
+                }
             }
         }
     } else {
-        // ---------------------------------------------------------------- epilogue: 4 warps, one TMEM lane quadrant each
+        // ---------------------------------------------------------------- epilogue: two groups of 4 warps (one TMEM lane quadrant each);
+        // group g takes the tiles whose accumulator is buffer g, so two epilogues run side by side
+        const int grp = (warp - 2) >> 2, bid = 1 + grp;
         const int quad = warp & 3;
         const int m = quad * 32 + lane;                          // row of the tile = TMEM lane
-        const int et = threadIdx.x - 64;                         // 0..127 among the epilogue threads
+        const int et = threadIdx.x - 64 - grp * 128;             // 0..127 among the group's threads
         const bool leader = et == 0;
-        uint32_t acc_cnt = 0, add_use[4] = {0u, 0u, 0u, 0u}; bool ok = true;
-        int cur = -1; const TcHot& h = hot_s[2];
-        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++acc_cnt) {
+        int* const pix_s = pix_s2[grp];
+        float (*const stat_s)[2][256] = stat_s2[grp];
+        uint32_t add_use[4] = {0u, 0u, 0u, 0u}; bool ok = true;
+        int cur = -1; const TcHot& h = hot_s[2 + grp];
+        for (int t = t_begin + grp * t_step; grp < L.groups && t < t_stop && ok; t += L.groups * t_step) {
+            const uint32_t acc_cnt = (uint32_t)((t - t_begin) / t_step), kk = acc_cnt / (uint32_t)L.groups;     // tile number of the CTA, of the group
             int pi = 0; while (t >= tile_end_s[pi]) ++pi;
             const TcProb* pp = probs + pi;
             const int loc = t - (pi ? tile_end_s[pi - 1] : 0);
             const uint32_t buf = acc_cnt & 1u, aph = (acc_cnt >> 1) & 1u;
-            const uint32_t sb = acc_cnt % (uint32_t)L.n_stg;
+            const uint32_t sb = (uint32_t)(grp * L.pg) + kk % (uint32_t)L.pg;
             const uint32_t stg = stg_base + sb * (uint32_t)L.stg_bytes;
-            // the staging tile is free again: the leader has waited for the reads of the bulk store it issued from it, and
-            // every warp has finished its share of the last copy-out
-            bar_sync_epi();
-            if (pi != cur) { copy_hot(&hot_s[2], &probs[pi].h, et, 128); cur = pi; bar_sync_epi(); }
-            const int tiles_n = h.tiles_n, n_tile = h.n_tile, ncol = h.ncol, add_mode = h.add_mode, dense = h.dense, out_slabs = h.out_slabs;
+            if (leader) {
+                // the staging tile of this tile (and, with a prefetched residual, the next tile's, which the producer is waiting to
+                // fill) must have been read by the bulk store issued from it
+                bulk_wait_read(L.prefetch ? L.pg - 2 : L.pg - 1);
+                if (L.prefetch && kk + 1 >= (uint32_t)L.pg) mbar_arrive(stg_free + 8 * ((uint32_t)(grp * L.pg) + (kk + 1) % (uint32_t)L.pg));
+            }
+            // ... and every warp must have finished its share of the last copy-out
+            bar_sync_epi(bid);
+            if (pi != cur) { copy_hot(&hot_s[2 + grp], &probs[pi].h, et, 128); cur = pi; bar_sync_epi(bid); }
+            const int n_tile = h.n_tile, ncol = h.ncol, add_mode = h.add_mode, dense = h.dense, out_slabs = h.out_slabs;
             const float scale = h.scale;
             const __nv_bfloat16* addp = h.add; __nv_bfloat16* outp = h.out; float* stat_tiles = h.stat_tiles;
-            const int tn = loc % tiles_n, tm = loc / tiles_n;
+            const int tiles_n = h.tiles_n, tn = loc % tiles_n, tm = loc / tiles_n;
             ok = mbar_wait(acc_full + 8 * buf, aph, &abort_s);
             if (ok && add_mode == 1) { ok = mbar_wait(add_full + 8 * sb, add_use[sb] & 1u, &abort_s); ++add_use[sb]; }
-            ok = bar_and_epi(ok);                                // one decision for the four warps: they share the barriers below
+            ok = bar_and_epi(bid, ok);                           // one decision for the four warps: they share the barriers below
             if (!ok) { atomicExch(&abort_s, 1); atomicExch(h.status, 6); break; }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             // position -> output pixel (and the residual's pixel)
@@ -400,7 +461,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const TcProb* __
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
             if (lane == 0) mbar_arrive(acc_empty + 8 * buf);     // this warp has read its quadrant of the accumulator
-            bar_sync_epi();                                      // the staging tile is complete
+            bar_sync_epi(bid);                                   // the staging tile is complete
             if (dense && leader) {
                 for (int j = 0; j < out_slabs; ++j) tma_store_2d(&pp->map_out, stg + (uint32_t)(j * SLAB_BYTES), col0 + j * 64, tm * TILE_M);
                 asm volatile("cp.async.bulk.commit_group;" ::: "memory");
@@ -420,7 +481,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const TcProb* __
                     stat_s[quad][0][j * 64 + 2 * lane] = s0; stat_s[quad][0][j * 64 + 2 * lane + 1] = s1;
                     stat_s[quad][1][j * 64 + 2 * lane] = q0; stat_s[quad][1][j * 64 + 2 * lane + 1] = q1;
                 }
-                bar_sync_epi();
+                bar_sync_epi(bid);
                 for (int c = et; c < n_tile; c += 128) {
                     if (col0 + c < ncol) {
                         const float su = ((stat_s[0][0][c] + stat_s[1][0][c]) + stat_s[2][0][c]) + stat_s[3][0][c];
@@ -441,11 +502,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_tc_kernel(const TcProb* __
                             lds128(stg + (uint32_t)(j * SLAB_BYTES) + (uint32_t)row * 128u + ((uint32_t)(ch ^ (row & 7)) << 4));
                 }
             }
-            if (leader) {
-                if (dense) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-                mbar_arrive(stg_free + 8 * sb);
-            }
         }
+        if (leader) bulk_wait_read(0);                           // shared memory stays until the last bulk stores have read it
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
@@ -866,15 +924,19 @@ int conv_tc_fill(const ConvProb& p, int mode, void* host_tc) {
         }
         // residual
         t.add_mode = !p.add ? 0 : p.add_sub == 2 ? 3 : t.dense ? 1 : 2;
-        // output tiles: up to 256 columns (128 with a prefetched residual: two staging tiles), a multiple of 64 when there are several
+        // output tiles: up to 256 columns (128 with a prefetched residual: several staging tiles), a multiple of 64 when there are several
         const int n_cap = t.add_mode == 1 ? 128 : 256;
+        const int ntaps = t.gbeg[t.ngroups];
+        auto b_tile = [&](int nt) { return mode == CONV_FWD ? nt * 128 : ((nt + 63) / 64) * 8192; };
+        auto b_total = [&](int nt) { return (size_t)t.slabs * ntaps * ((b_tile(nt) + 1023) / 1024 * 1024); };
         t.tiles_n = (ncol + n_cap - 1) / n_cap;
         t.n_tile = (ncol + t.tiles_n - 1) / t.tiles_n;
         t.n_tile = t.tiles_n > 1 ? (t.n_tile + 63) / 64 * 64 : (t.n_tile + 15) / 16 * 16;
         t.tiles_n = (ncol + t.n_tile - 1) / t.n_tile;
         t.out_slabs = (t.n_tile + 63) / 64;
         t.tiles_m = (t.total_pos + TILE_M - 1) / TILE_M;
-        t.b_bytes = mode == CONV_FWD ? t.n_tile * 128 : ((t.n_tile + 63) / 64) * 8192;
+        t.b_bytes = b_tile(t.n_tile);
+        t.b_total = (int)b_total(t.n_tile);
         // weights [K][taps][C] viewed as (C, tap, K).  Forward: a tile is n_tile output channels (rows) x 64 input channels.
         // dgrad: a block is 64 reduction channels k (rows) x 64 output columns c.
         { const uint64_t dims[3] = {(uint64_t)p.C, (uint64_t)taps, (uint64_t)p.K};
@@ -891,19 +953,20 @@ int conv_tc_fill(const ConvProb& p, int mode, void* host_tc) {
 }
 size_t conv_tc_prob_bytes() { return sizeof(TcProb); }
 int conv_tc_tiles(const void* host_tc) { const TcHot* t = &((const TcProb*)host_tc)->h; return t->tiles_m * t->tiles_n; }
-// packs what a launch has to know about its largest problem into one number: window KB, weight-tile KB, staging tiles, MMA N
+// packs what a launch has to know about its largest problem into one number: window KB (12 bits), weight-tile KB (12), staging
+// tiles (4), KB of all weight tiles of a column tile (16), MMA N (20)
 size_t conv_tc_smem(const void* host_tc) {
     const TcHot* t = &((const TcProb*)host_tc)->h;
     const size_t a_stage = ((size_t)t->nbox * t->a_box_bytes + 1023) / 1024, b_stage = ((size_t)t->b_bytes + 1023) / 1024;
-    return (a_stage << 48) | (b_stage << 32) | ((size_t)(t->add_mode == 1 ? 2 : 1) << 24) | (size_t)t->n_tile;
+    return (a_stage << 52) | (b_stage << 40) | ((size_t)(t->add_mode == 1 ? 2 : 1) << 36) | ((size_t)std::min(t->b_total / 1024, 0xFFFF) << 20) | (size_t)t->n_tile;
 }
 // field-wise maximum of two packed values
 size_t conv_tc_merge(size_t a, size_t b) {
-    return (std::max(a >> 48, b >> 48) << 48) | (std::max((a >> 32) & 0xFFFF, (b >> 32) & 0xFFFF) << 32) |
-           (std::max((a >> 24) & 0xFF, (b >> 24) & 0xFF) << 24) | std::max(a & 0xFFFFFF, b & 0xFFFFFF);
+    return (std::max(a >> 52, b >> 52) << 52) | (std::max((a >> 40) & 0xFFF, (b >> 40) & 0xFFF) << 40) | (std::max((a >> 36) & 0xF, (b >> 36) & 0xF) << 36) |
+           (std::max((a >> 20) & 0xFFFF, (b >> 20) & 0xFFFF) << 20) | std::max(a & 0xFFFFF, b & 0xFFFFF);
 }
 
-constexpr size_t TC_SMEM_BUDGET = 212 * 1024;
+constexpr size_t TC_SMEM_BUDGET = 204 * 1024;
 
 // total_tiles: an upper bound of the tiles of all problems of the launch (max_tiles * nprob); packed: conv_tc_merge over its problems
 void launch_conv_tc_probs(const void* d_tc, int nprob, int max_tiles, size_t packed, cudaStream_t s) {
@@ -915,26 +978,42 @@ void launch_conv_tc_probs(const void* d_tc, int nprob, int max_tiles, size_t pac
     }
     TcLaunch L{};
     L.nprob = nprob;
-    L.a_stage = (int)(packed >> 48) * 1024; L.b_stage = (int)((packed >> 32) & 0xFFFF) * 1024;
-    L.n_stg = (int)((packed >> 24) & 0xFF);
-    const int n_tile = (int)(packed & 0xFFFFFF);
+    L.a_stage = (int)(packed >> 52) * 1024; L.b_stage = (int)((packed >> 40) & 0xFFF) * 1024;
+    L.prefetch = ((packed >> 36) & 0xF) > 1 ? 1 : 0;
+    const size_t b_total = ((packed >> 20) & 0xFFFF) * 1024;
+    const int n_tile = (int)(packed & 0xFFFFF);
     L.stg_bytes = ((n_tile + 63) / 64) * SLAB_BYTES;
-    // Shared memory: with a prefetched residual three staging tiles (two residual tiles in flight behind the one the epilogue works
-    // on), else one; three weight tiles; the rest goes to the ring of activation windows: an HBM-bound layer runs at the bytes it
-    // keeps in flight
-    if (L.n_stg > 1) L.n_stg = 3;
-    while (L.n_stg > 1 && (size_t)L.n_stg * L.stg_bytes + 2 * (size_t)(L.a_stage + L.b_stage) > TC_SMEM_BUDGET) --L.n_stg;
+    // Shared memory.  Staging tiles: two epilogue groups where they fit (they take alternate tiles, so two epilogues run side by
+    // side), each with two tiles when the residual is prefetched into them by TMA, else one; a single group (three tiles behind a
+    // prefetched residual) otherwise.  Weights: resident when all tiles of a column tile are small, else a ring of three tiles.  The
+    // rest goes to the ring of activation windows: an HBM-bound layer runs at the bytes it keeps in flight.
+    L.b_res = b_total <= TC_RESIDENT_BUDGET ? 1 : 0;
+    const size_t kgroups = L.b_stage ? b_total / (size_t)L.b_stage : 1;
+    const size_t b_min = L.b_res ? b_total : 2 * (size_t)L.b_stage;
+    L.groups = 2; L.pg = L.prefetch ? 2 : 1;
+    if (kgroups > 8) L.groups = 1;                             // long reductions: the epilogue is a small share, the smem goes to the rings
+    if (L.groups == 1 || (size_t)L.groups * L.pg * L.stg_bytes + 3 * (size_t)L.a_stage + b_min > TC_SMEM_BUDGET) {
+        L.groups = 1; L.pg = L.prefetch ? 3 : 1;
+        while (L.pg > (L.prefetch ? 2 : 1) && (size_t)L.pg * L.stg_bytes + 2 * (size_t)L.a_stage + b_min > TC_SMEM_BUDGET) --L.pg;
+    }
+    L.n_stg = L.groups * L.pg;
     const size_t rings = TC_SMEM_BUDGET - (size_t)L.n_stg * L.stg_bytes;
-    L.nb = 3; while (L.nb > 2 && (size_t)L.nb * L.b_stage + 2 * (size_t)L.a_stage > rings) --L.nb;
-    L.na = 2; while (L.na < TC_MAX_STAGES && (size_t)(L.na + 1) * L.a_stage + (size_t)L.nb * L.b_stage <= rings) ++L.na;
-    while (L.nb < 6 && (size_t)L.na * L.a_stage + (size_t)(L.nb + 1) * L.b_stage <= rings) ++L.nb;
+    if (L.b_res) {
+        L.nb = 0; L.b_region = (int)b_total;
+        L.na = 2; while (L.na < TC_MAX_STAGES && (size_t)(L.na + 1) * L.a_stage + b_total <= rings) ++L.na;
+    } else {
+        L.nb = 3; while (L.nb > 2 && (size_t)L.nb * L.b_stage + 2 * (size_t)L.a_stage > rings) --L.nb;
+        L.na = 2; while (L.na < TC_MAX_STAGES && (size_t)(L.na + 1) * L.a_stage + (size_t)L.nb * L.b_stage <= rings) ++L.na;
+        while (L.nb < 6 && (size_t)L.na * L.a_stage + (size_t)(L.nb + 1) * L.b_stage <= rings) ++L.nb;
+        L.b_region = L.nb * L.b_stage;
+    }
     L.acc_stride = (n_tile + 31) / 32 * 32;
     L.tmem_cols = 32; while (L.tmem_cols < 2 * L.acc_stride) L.tmem_cols *= 2;
     // at least 120 KB of shared memory so that two CTAs that allocate tensor memory never share an SM
-    const size_t smem = std::max((size_t)L.na * L.a_stage + (size_t)L.nb * L.b_stage + (size_t)L.n_stg * L.stg_bytes, (size_t)120 * 1024) + 1024;
+    const size_t smem = std::max((size_t)L.na * L.a_stage + (size_t)L.b_region + (size_t)L.n_stg * L.stg_bytes, (size_t)120 * 1024) + 1024;
     const long long total = (long long)max_tiles * nprob;
     const int grid = (int)std::max(1ll, std::min(total, (long long)sms));
-    conv_tc_kernel<<<grid, TC_THREADS, smem, s>>>((const TcProb*)d_tc, L);
+    conv_tc_kernel<<<grid, TC_CONV_THREADS, smem, s>>>((const TcProb*)d_tc, L);
 }
 
 // ---- wgrad host side

@@ -2,6 +2,7 @@
 // fp32 arithmetic.  It is the whole path of the fp32 mode, and in bf16 mode it runs whatever the
 // tensor-core kernels do not take (3-channel stems, odd shapes) and the small head/loss kernels.
 // All reductions have a fixed order: results are reproducible run to run.
+#include <algorithm>
 #include <cooperative_groups.h>
 #include "internal.h"
 
@@ -229,6 +230,67 @@ __device__ void bn_reduce_vec(const BnProb& p) {
     }
 }
 
+// Streaming form of the elementwise pass (bf16 vector path): a thread keeps ONE group of 8 channels for all its rows, so the
+// per-channel constants are loaded once into registers and the loop is loads, arithmetic and a store; a CTA takes at least 16 passes
+// of 256 / G rows (32768 elements), four rows of loads in flight per thread.  MODE 0: a = relu(bn(x)); MODE 1: dx (+ add).
+template <int MODE>
+__device__ void bn_stream_vec(const BnProb& p) {
+    const int C = p.C, G = C >> 3, R = 256 / G;
+    const int g = threadIdx.x % G, r = threadIdx.x / G;
+    // the grid's CTAs share the rows evenly, in whole passes of 4 * R rows (at least 16 passes of R rows each)
+    long long rows_per_cta = (p.m + gridDim.x - 1) / gridDim.x;
+    rows_per_cta = (rows_per_cta + 4 * R - 1) / (4 * R) * (4 * R); if (rows_per_cta < 16 * R) rows_per_cta = 16 * R;
+    const long long r0 = (long long)blockIdx.x * rows_per_cta;
+    if (r0 >= p.m) return;
+    const long long r1 = r0 + rows_per_cta < p.m ? r0 + rows_per_cta : p.m;
+    float mean[8], istd[8], ga[8], be[8], sb[8], sg[8];
+    const float inv_m = 1.f / (float)p.m;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const int c = g * 8 + j;
+        mean[j] = p.stat[c]; istd[j] = p.stat[C + c]; ga[j] = p.gamma[c]; be[j] = p.beta[c];
+        if (MODE == 1) { sb[j] = p.stat[2 * C + c] * inv_m; sg[j] = p.stat[3 * C + c] * inv_m; }
+    }
+    const uint4* xv = reinterpret_cast<const uint4*>(p.x);
+    const uint4* dv = reinterpret_cast<const uint4*>(p.da);
+    const uint4* av = reinterpret_cast<const uint4*>(p.add);
+    uint4* ov = reinterpret_cast<uint4*>(MODE == 0 ? p.a : p.dx);
+    for (long long row = r0 + r; row < r1; row += 4 * R) {
+        uint4 xs[4], ds[4], as[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const long long rr = row + (long long)u * R;
+            if (rr < r1) {
+                xs[u] = __ldg(xv + rr * G + g);
+                if (MODE == 1) { ds[u] = __ldg(dv + rr * G + g); if (av) as[u] = __ldg(av + rr * G + g); }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const long long rr = row + (long long)u * R;
+            if (rr < r1) {
+                float x[8], o[8]; unpack8(xs[u], x);
+                if (MODE == 0) {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) { const float z = (x[j] - mean[j]) * istd[j] * ga[j] + be[j]; o[j] = z > 0.f ? z : 0.f; }
+                } else {
+                    float d[8]; unpack8(ds[u], d);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const float xh = (x[j] - mean[j]) * istd[j];
+                        const float dz = (xh * ga[j] + be[j] > 0.f) ? d[j] : 0.f;
+                        o[j] = ga[j] * istd[j] * (dz - sb[j] - xh * sg[j]);
+                    }
+                    if (av) { float ad[8]; unpack8(as[u], ad);
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) o[j] += ad[j]; }
+                }
+                ov[rr * G + g] = pack8(o);
+            }
+        }
+    }
+}
+
 template <int MODE>   // 0: forward apply; 1: backward apply.  stat: [4][C] as BnProb::stat, in global or shared memory
 __device__ void bn_apply_vec(const BnProb& p, const float* __restrict__ stat) {
     const int C = p.C, G = C >> 3;
@@ -345,7 +407,7 @@ __global__ void bn_finalize_kernel(const BnProb* __restrict__ probs) {
 template <class T>
 __global__ void __launch_bounds__(256) bn_apply_kernel(const BnProb* __restrict__ probs) {
     const BnProb& p = probs[blockIdx.y];
-    if (p.vec) { bn_apply_vec<0>(p, p.stat); return; }
+    if (p.vec) { bn_stream_vec<0>(p); return; }
     const long long n = p.m * p.C;
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
         const int c = (int)(i % p.C);
@@ -357,7 +419,7 @@ __global__ void __launch_bounds__(256) bn_apply_kernel(const BnProb* __restrict_
 template <class T>
 __global__ void __launch_bounds__(256) bn_bwd_apply_kernel(const BnProb* __restrict__ probs) {
     const BnProb& p = probs[blockIdx.y];
-    if (p.vec) { bn_apply_vec<1>(p, p.stat); return; }
+    if (p.vec) { bn_stream_vec<1>(p); return; }
     const long long n = p.m * p.C;
     const float inv_m = 1.f / (float)p.m;
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
@@ -451,8 +513,10 @@ void launch_bn_stats(const BnProb* d, int nprob, int max_chunks, int max_c, bool
     if (bf16) bn_finalize_kernel<__nv_bfloat16, 0><<<dim3((max_c + 7) / 8, nprob), 256, 0, s>>>(d);
     else bn_finalize_kernel<float, 0><<<dim3((max_c + 7) / 8, nprob), 256, 0, s>>>(d);
 }
+// the vector path takes at least 32768 elements per CTA (see bn_stream_vec), and about 16 CTAs per SM over the launch
+static int stream_grid(long long n, int nprob) { long long g = (n + 32767) / 32768; const long long cap = std::max(1, 148 * 16 / std::max(1, nprob)); if (g > cap) g = cap; if (g < 1) g = 1; return (int)g; }
 void launch_bn_apply(const BnProb* d, int nprob, long long max_elems, bool bf16, cudaStream_t s) {
-    if (bf16) bn_apply_kernel<__nv_bfloat16><<<dim3(ew_grid(max_elems), nprob), 256, 0, s>>>(d);
+    if (bf16) bn_apply_kernel<__nv_bfloat16><<<dim3(stream_grid(max_elems, nprob), nprob), 256, 0, s>>>(d);
     else bn_apply_kernel<float><<<dim3(ew_grid(max_elems), nprob), 256, 0, s>>>(d);
 }
 void launch_bn_bwd_reduce(const BnProb* d, int nprob, int max_chunks, int max_c, bool bf16, cudaStream_t s) {
@@ -461,7 +525,7 @@ void launch_bn_bwd_reduce(const BnProb* d, int nprob, int max_chunks, int max_c,
     bn_finalize_kernel<float, 1><<<dim3((max_c + 7) / 8, nprob), 256, 0, s>>>(d);
 }
 void launch_bn_bwd_apply(const BnProb* d, int nprob, long long max_elems, bool bf16, cudaStream_t s) {
-    if (bf16) bn_bwd_apply_kernel<__nv_bfloat16><<<dim3(ew_grid(max_elems), nprob), 256, 0, s>>>(d);
+    if (bf16) bn_bwd_apply_kernel<__nv_bfloat16><<<dim3(stream_grid(max_elems, nprob), nprob), 256, 0, s>>>(d);
     else bn_bwd_apply_kernel<float><<<dim3(ew_grid(max_elems), nprob), 256, 0, s>>>(d);
 }
 
@@ -574,19 +638,20 @@ __global__ void __launch_bounds__(1024) loss_kernel(const HeadProb* __restrict__
         if (p.correct) *p.correct = c;
     }
 }
-// one warp per output element: lane l adds samples l, l+32, ... in order, then a fixed butterfly over the lanes
+// one thread per element of dw (neighbouring threads = neighbouring input channels: the loads of `pooled` are coalesced and the
+// dlogits value is the same for a whole warp); samples added in order.  The last `classes` threads make the bias gradient.
 __global__ void head_bwd_w_kernel(const HeadProb* __restrict__ probs) {
     const HeadProb& p = probs[blockIdx.y];
-    const int n = p.classes * p.C, lane = threadIdx.x & 31;
-    const int nw = gridDim.x * (blockDim.x >> 5);
-    for (int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); i < n + p.classes; i += nw) {
+    const int n = p.classes * p.C;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n + p.classes; i += gridDim.x * blockDim.x) {
         float s = 0.f;
         if (i < n) { const int c = i % p.C, k = i / p.C;
-            for (int b = lane; b < p.B; b += 32) s = fmaf(p.dlogits[(long long)b * p.classes + k], p.pooled[(long long)b * p.C + c], s);
+#pragma unroll 4
+            for (int b = 0; b < p.B; ++b) s = fmaf(p.dlogits[(long long)b * p.classes + k], p.pooled[(long long)b * p.C + c], s);
+            p.dw[i] = s;
         } else { const int k = i - n;
-            for (int b = lane; b < p.B; b += 32) s += p.dlogits[(long long)b * p.classes + k]; }
-        for (int d = 16; d; d >>= 1) s += __shfl_xor_sync(0xffffffffu, s, d);
-        if (lane == 0) { if (i < n) p.dw[i] = s; else p.db[i - n] = s; }
+            for (int b = 0; b < p.B; ++b) s += p.dlogits[(long long)b * p.classes + k];
+            p.db[k] = s; }
     }
 }
 __global__ void head_bwd_x_kernel(const HeadProb* __restrict__ probs) {
@@ -627,7 +692,7 @@ void launch_head_fwd(const HeadProb* d, int nprob, int maxB, int maxC, int max_c
 }
 void launch_head_bwd(const HeadProb* d, int nprob, int maxB, int maxC, int max_classes, long long max_elems,
                      bool bf16, cudaStream_t s) {
-    head_bwd_w_kernel<<<dim3(ew_grid((long long)max_classes * (maxC + 1) * 32), nprob), 256, 0, s>>>(d);
+    head_bwd_w_kernel<<<dim3(ew_grid((long long)max_classes * (maxC + 1)), nprob), 256, 0, s>>>(d);
     head_bwd_x_kernel<<<dim3(ew_grid((long long)maxB * maxC), nprob), 256, 0, s>>>(d);
     if (bf16) avgpool_bwd_kernel<__nv_bfloat16><<<dim3(ew_grid(max_elems), nprob), 256, 0, s>>>(d);
     else avgpool_bwd_kernel<float><<<dim3(ew_grid(max_elems), nprob), 256, 0, s>>>(d);

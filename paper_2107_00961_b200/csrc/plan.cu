@@ -275,6 +275,8 @@ struct Builder {
         BnProb& p = op.bn;
         p.x = x; p.da = da; p.dx = dx; p.add = add; p.gamma = W() + r.g; p.beta = W() + r.b; p.dgamma = G() + r.g; p.dbeta = G() + r.b;
         p.stat = stat; p.m = m; p.C = r.c; p.eps = ctx->opts.bn_eps; p.momentum = ctx->opts.bn_momentum; p.eval = 0;
+        // (measured on 8 x 67 MB tensors, far beyond L2: the single cooperative launch, 794 us, still beats a reduction with many small
+        // chunks followed by a streaming elementwise pass, 308 + 539 us; both move the same six passes over HBM)
         bn_chunking(p, ctx->opts.dtype == RESIST_BF16, fused_chunks());
         bn_partial_need = std::max(bn_partial_need, (size_t)p.chunks * 2 * r.c * 8);
         p.partial = bn_partial;
