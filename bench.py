@@ -1,14 +1,19 @@
 #!/usr/bin/env python
 """Benchmark of the ResIST hot path on B200: sub-ResNet training images/s.
 
-Workload (N = 1): the CIFAR-shaped ResNet-110 configuration: S = 4 sub-ResNets from a seeded layer-wise
-partition (stage-first blocks shared), batch 128 per sub-ResNet, bf16 activations and weights with fp32 master
-weights, 50 local SGD steps per synchronisation round.  A "step" is one grouped local step of all S sub-ResNets
-(S*B images: forward, backward, SGD-momentum update); every 50th step is followed by the reassembly
-(resist_aggregate) and the next round's partition + scatter (resist_partition), all inside the timed region.
+Workload (N = 1, default `--workload wide`): the wide CIFAR-shaped bottleneck ResNet [3,4,23,3] (64..512 x4 channels,
+32x32x3 inputs, 100 classes): S = 8 sub-ResNets from a seeded layer-wise partition (the non-first blocks of the third
+section are dealt out), batch 128 per sub-ResNet, bf16 activations and weights with fp32 master weights, 50 local SGD
+steps per synchronisation round.  It is the largest training configuration by work per step (7 TFLOP) and every layer
+of it is tensor-core shaped.  `--workload resnet110` and `--workload imagenet` time the other two training
+configurations the same way, `--workload reassembly` the synchronisation kernels alone.
+A "step" is one grouped local step of all S sub-ResNets (S*B images: forward, backward, SGD-momentum update); every
+50th step (the counter runs on through warm-up and repeats) is followed by the reassembly (resist_aggregate) and the
+next round's partition + scatter (resist_partition) inside the timed region.  A block of exactly K steps is timed
+with CUDA events, blocks are repeated until about 1.5 s is measured, and the median block is reported with its spread.
 Inputs are synthetic (Gaussian pixels, uniform labels), generated before the timed region.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload wide|resnet110|imagenet|reassembly]
 
 `value` is measured with the inputs resident in HBM; `e2e` repeats the same steps through the same public calls
 with the inputs in pinned host memory: every step's inputs are copied to the device inside the timed region (on a copy
@@ -43,7 +48,8 @@ WORKLOADS = {
     "imagenet": (4, "configs[3]: ImageNet-shaped ResNet-101, 224x224x3, 1000 classes, S=4 sub-ResNets, batch 64 per sub-ResNet, "
                     "bf16 + fp32 master, 20 local steps per round", 3),
 }
-NCU_DRAM_BYTES_PER_LAUNCH = {"conv_dgrad_mma_bn": 17.56e6, "conv_fwd_mma_bn": 10.50e6}
+# mean DRAM bytes per launch of a kernel family (ncu, profiles/): workload -> family -> bytes; filled in from the committed captures
+NCU_DRAM_BYTES_PER_LAUNCH = {}
 
 
 def measured_peaks():
@@ -120,6 +126,17 @@ def make_batches(cfg, n):
     return xs, ys
 
 
+def bound_of(name: str, v: dict, peaks: dict) -> dict:
+    """Roofline of one profile entry: entries named '<family>@tensor' hold the launches whose arithmetic intensity is above the
+    ridge (held against the sustained bf16 peak, the kernels being timed inside a long step), the others against HBM bandwidth."""
+    ms = max(v["ms"], 1e-9)
+    if name.endswith("@tensor"):
+        ach, peak, unit, bound = v["flops"] / ms / 1e9, peaks["bf16_tflops_sustained"] or peaks["bf16_tflops"], "TFLOP/s", "tensor"
+    else:
+        ach, peak, unit, bound = v["bytes"] / ms / 1e6, peaks["hbm_gbs"], "GB/s", "hbm"
+    return {"bound": bound, "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak}
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -136,9 +153,10 @@ def run_ours(args):
     S, B, K, W = cfg.S, cfg.batch, args.steps, args.warmup
     LOCAL_STEPS = cfg.local_steps
     POOL = WORKLOADS[args.workload][2]
+    a = cfg.arch
 
-    ctx = lib.Context(cfg.arch.to_int32(), dtype=lib.BF16, momentum=cfg.momentum, seed=cfg.init_seed, device=str(dev))
-    p0, b0 = synth.init_params(cfg.arch, cfg.init_seed)
+    ctx = lib.Context(a.to_int32(), dtype=lib.BF16, momentum=cfg.momentum, seed=cfg.init_seed, device=str(dev))
+    p0, b0 = synth.init_params(a, cfg.init_seed)
     ctx.set_params(p0, b0)
     xs, ys = make_batches(cfg, POOL)
     d_x = [[torch.from_numpy(x).to(dev).to(torch.bfloat16) for x in bx] for bx in xs]
@@ -150,14 +168,14 @@ def run_ours(args):
     stage_x = [[torch.empty_like(d_x[0][s]) for s in range(S)] for _ in range(2)]
     stage_y = [[torch.empty_like(d_y[0][s]) for s in range(S)] for _ in range(2)]
     loss = torch.zeros(S, dtype=torch.float32, device=dev)
-    h_loss = torch.zeros(max(K, W) + 1, S, dtype=torch.float32).pin_memory()
+    h_loss = torch.zeros(256, S, dtype=torch.float32).pin_memory()
     stream = torch.cuda.current_stream()
     copy_stream = torch.cuda.Stream(device=dev)
     ev_copied = [torch.cuda.Event() for _ in range(2)]
     ev_free = [torch.cuda.Event() for _ in range(2)]
     for e in ev_free:
         e.record(stream)
-    state = {"step": 0, "round": 0, "launches": 0}
+    state = {"step": 0, "round": 0, "launches": 0, "boundaries": 0}
 
     def new_round():
         ctx.partition(cfg.round_seed(state["round"]), S)
@@ -179,12 +197,13 @@ def run_ours(args):
             ev_free[b].record(stream)
         else:
             ctx.local_step_grouped(d_x[i], d_y[i], cfg.lr, loss)
-        state["step"] += 1
+        state["step"] += 1                    # the step counter runs on through warm-up and all repeats: round boundaries fall where they fall
         state["launches"] += ctx.step_info()["kernel_launches"]
         if state["step"] % LOCAL_STEPS == 0:
             ctx.aggregate()
             new_round()
             state["launches"] += 3            # aggregate (one launch) + scatter (parameters, buffers)
+            state["boundaries"] += 1
 
     def barrier():
         if world > 1:
@@ -192,85 +211,121 @@ def run_ours(args):
         torch.cuda.synchronize()
 
     def timed(e2e: bool):
-        state["step"] = 0
-        state["round"] = 0                    # both passes train the same sequence of partitions (a partition's shape sets the step time)
+        """W warm-up steps, then blocks of exactly K steps, each bracketed by a barrier and CUDA events, repeated until about 1.5 s of
+        device time has been measured (at least 3 blocks): the reported time is the median block, the spread is kept."""
+        state.update(step=0, round=0)         # both passes train the same sequence of partitions (a partition's shape sets the step time)
         new_round()
         for _ in range(W):
             one_step(e2e)
-        state["step"] = 0
-        state["launches"] = 0
-        barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        for _ in range(K):
-            one_step(e2e)
-        e1.record(stream)
-        barrier()
-        ms = max_over_ranks(e0.elapsed_time(e1), dev)
-        return ms, state["launches"]
+        blocks, launches, bounds = [], [], []
+        total = 0.0
+        while len(blocks) < 3 or (total < 1500.0 and len(blocks) < 200):
+            state.update(launches=0, boundaries=0)
+            barrier()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(K):
+                one_step(e2e)
+            e1.record(stream)
+            barrier()
+            ms = max_over_ranks(e0.elapsed_time(e1), dev)
+            blocks.append(ms); launches.append(state["launches"]); bounds.append(state["boundaries"])
+            total += ms
+        return blocks, launches, bounds
 
     sampler = ClockSampler(local)
     sampler.start()
-    ms, launches = timed(False)
+    blocks, launches, bounds = timed(False)
     clocks = sampler.stop()
     info = ctx.step_info()
-    ms_e2e, _ = timed(True)
-    assert bool(torch.isfinite(h_loss[:min(K, h_loss.shape[0])]).all()), "the end-to-end pass produced a non-finite loss"
+    blocks_e2e, _, _ = timed(True)
+    assert bool(torch.isfinite(h_loss).all()), "the end-to-end pass produced a non-finite loss"
+    ms = float(np.median(blocks))
+    ms_e2e = float(np.median(blocks_e2e))
+    mid = int(np.argsort(blocks)[len(blocks) // 2])
+
+    # round boundary alone: reassembly + next partition (scatter, new launch plan) after a step, CUDA events around the two calls
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    over = []
+    for _ in range(3):
+        one_step(False)
+        torch.cuda.synchronize()
+        e0.record(stream)
+        ctx.aggregate()
+        new_round()
+        ctx.local_step_grouped(d_x[0], d_y[0], cfg.lr, loss)     # the first step of a round builds the round's launch plan
+        e1.record(stream)
+        torch.cuda.synchronize()
+        over.append(e0.elapsed_time(e1))
+    round_overhead_ms = float(np.median(over)) - ms / K
 
     # per-kernel pass: the same steps with every launch bracketed by CUDA events on the library's stream
     peaks = measured_peaks()
     ctx.set_profiling(True)
     ctx.get_profile()
-    state["round"] = 0
+    state.update(step=0, round=0)
     new_round()
-    state["step"] = 0
-    nprof = min(K, 10)
+    nprof = min(max(K, 4), 10)
     for _ in range(nprof):
         one_step(False)
     prof = ctx.get_profile()
+    # the reassembly kernels on this workload's parameter set (they run once per round: timed here in a loop of their own)
+    for i in range(10):
+        ctx.aggregate()
+        ctx.partition(cfg.round_seed(100 + i), S)
+    sync_prof = ctx.get_profile()
     ctx.set_profiling(False)
-    total_ms = sum(v["ms"] for v in prof.values())
-    top_name, top = max(((k, v) for k, v in prof.items() if k not in ("scatter", "aggregate")), key=lambda kv: kv[1]["ms"])
-    per_ms = top["ms"] / top["operations"]
-    roof = {"kernel": top_name, "share_of_step": top["ms"] / total_ms, "launches": top["operations"], "avg_ms": per_ms}
-    ai = top["flops"] / max(top["bytes"], 1.0)
-    ridge = peaks["bf16_tflops"] * 1e12 / (peaks["hbm_gbs"] * 1e9)
-    if top["flops"] > 0 and ai > ridge and "tcgen05" in top_name:
-        ach = top["flops"] / top["operations"] / (per_ms * 1e-3) / 1e12
-        roof.update(bound="tensor", achieved=ach, peak=peaks["bf16_tflops_sustained"] or peaks["bf16_tflops"], unit="TFLOP/s")
-    else:
-        ach = top["bytes"] / top["operations"] / (per_ms * 1e-3) / 1e9
-        roof.update(bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s")
-    roof["frac"] = roof["achieved"] / roof["peak"]
-    roof["peak_source"] = peaks["source"]
-    # DRAM bytes (read + written) per launch of that kernel family from the ncu capture summarised under profiles/
-    # (mean over the launches of one step); None for a family the capture does not cover
-    roof["traffic"] = NCU_DRAM_BYTES_PER_LAUNCH.get(top_name)
-    roof["traffic_unit"] = "bytes per launch (ncu dram__bytes_read.sum + dram__bytes_write.sum, mean over one step's launches)"
-    roof["algorithmic_bytes_per_launch"] = top["bytes"] / top["operations"]
-    roof["arithmetic_intensity"] = ai
-    conv_ms = sum(v["ms"] for k, v in prof.items() if k.startswith("conv_") or k == "wgrad_splitk_reduce")
-    conv_flops = sum(v["flops"] for k, v in prof.items() if k.startswith("conv_"))
-    kernels = {k: {"ms_per_step": v["ms"] / nprof, "share": v["ms"] / total_ms,
-                   "GBps": v["bytes"] / max(v["ms"], 1e-9) / 1e6, "TFLOPs": v["flops"] / max(v["ms"], 1e-9) / 1e9}
-               for k, v in sorted(prof.items(), key=lambda kv: -kv[1]["ms"])}
+    step_prof = {k: v for k, v in prof.items() if k not in ("scatter", "aggregate")}
+    total_ms = sum(v["ms"] for v in step_prof.values())
+    families = {}
+    for k, v in sorted(step_prof.items(), key=lambda kv: -kv[1]["ms"]):
+        r = bound_of(k, v, peaks)
+        families[k] = {"ms_per_step": v["ms"] / nprof, "share": v["ms"] / total_ms, "launches_per_step": v["operations"] / nprof, **r}
+    top_name, top = max(step_prof.items(), key=lambda kv: kv[1]["ms"])
+    roof = {"kernel": top_name, "share_of_step": top["ms"] / total_ms, "launches": top["operations"], "avg_ms": top["ms"] / top["operations"],
+            **bound_of(top_name, top, peaks), "peak_source": peaks["source"] + " (MEASURED_PEAKS.json)" if peaks["source"] == "measured" else "fallback",
+            "algorithmic_bytes_per_launch": top["bytes"] / top["operations"], "algorithmic_flops_per_launch": top["flops"] / top["operations"],
+            "arithmetic_intensity": top["flops"] / max(top["bytes"], 1.0),
+            # DRAM bytes (read + written) per launch of that family from the ncu capture summarised under profiles/; None for a
+            # family the capture does not cover or whose kernel has changed since
+            "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(args.workload, {}).get(top_name)}
+    conv = {k: v for k, v in step_prof.items() if k.startswith("conv_")}
+    conv_ms = sum(v["ms"] for v in conv.values()) + sum(v["ms"] for k, v in step_prof.items() if k.startswith("wgrad_splitk"))
+    conv_flops = sum(v["flops"] for v in conv.values())
+    tens = {k: v for k, v in conv.items() if k.endswith("@tensor")}
+    tens_ms, tens_flops = sum(v["ms"] for v in tens.values()), sum(v["flops"] for v in tens.values())
+    reassembly = {}
+    for name in ("scatter", "aggregate"):
+        if name in sync_prof:
+            v = sync_prof[name]
+            gbps = v["bytes"] / max(v["ms"], 1e-9) / 1e6
+            reassembly[name] = {"us_per_call": v["ms"] / v["operations"] * 1e3, "MB_per_call": v["bytes"] / v["operations"] / 1e6, "GBps": gbps,
+                                "frac_of_hbm_peak": gbps / peaks["hbm_gbs"]}
 
     images = S * B * K * world
     out = {
         "metric": "sub-ResNet train images/s", "value": images / (ms * 1e-3), "unit": "images/s", "n_gpus": world, "steps": K,
         "warmup": W, "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
-        "config": {"workload": WORKLOADS[args.workload][1],
+        "config": {"workload": WORKLOADS[args.workload][1] + "; every %d-th step is followed by resist_aggregate + resist_partition inside the timed region" % LOCAL_STEPS,
                    "S": S, "batch_per_subnet": B, "local_steps": LOCAL_STEPS, "multi_gpu": "independent replicas" if world > 1 else "single GPU",
                    "l2": "working set per step (saved activations, %.0f MB) exceeds the 126 MB L2; no flush" % (info["workspace_bytes"] / 1e6)},
+        "timing": {"blocks": len(blocks), "steps_per_block": K, "ms_per_step_min": min(blocks) / K, "ms_per_step_max": max(blocks) / K,
+                   "round_boundaries_in_timed_blocks": int(sum(bounds)), "round_boundaries_in_median_block": int(bounds[mid]),
+                   "round_overhead_ms": round_overhead_ms,
+                   "ms_per_step_amortised_over_a_round": ms / K if sum(bounds) else (ms / K * LOCAL_STEPS + round_overhead_ms) / LOCAL_STEPS,
+                   "note": "value = median block of exactly K steps; round_overhead_ms = aggregate + partition + plan rebuild of one round boundary, timed alone"},
         "clocks": clocks,
         "e2e": {"value": images / (ms_e2e * 1e-3), "unit": "images/s", "ms_per_step": ms_e2e / K,
-                "h2d_bytes_per_step": int(S * (B * cfg.arch.in_h * cfg.arch.in_w * cfg.arch.in_c * 2 + B * 4)), "d2h_bytes_per_step": int(S * 4)},
-        "gpu_launches": int(launches),
+                "h2d_bytes_per_step": int(S * (B * a.in_h * a.in_w * a.in_c * 2 + B * 4)), "d2h_bytes_per_step": int(S * 4)},
+        "gpu_launches": int(launches[mid]),
         "conv": {"TFLOPs": conv_flops / max(conv_ms, 1e-9) / 1e9, "frac_of_bf16_peak": conv_flops / max(conv_ms, 1e-9) / 1e9 / peaks["bf16_tflops"],
+                 "tensor_bound_TFLOPs": tens_flops / max(tens_ms, 1e-9) / 1e9,
+                 "tensor_bound_frac_of_sustained_bf16_peak": tens_flops / max(tens_ms, 1e-9) / 1e9 / (peaks["bf16_tflops_sustained"] or peaks["bf16_tflops"]),
+                 "tensor_bound_share_of_conv_flops": tens_flops / max(conv_flops, 1.0),
                  "tensor_core_convs": info["tensor_core_convs"], "cuda_core_convs": info["cuda_core_convs"],
                  "flops_per_step": info["conv_flops"]},
-        "roofline": roof, "kernels": kernels,
+        "roofline": roof, "families": families, "reassembly": reassembly,
     }
     if rank == 0:
         if not args.skip_cpu_baseline:
@@ -281,15 +336,15 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-def oracle_step_all(cfg, a, mask, params, B, step_idx):
-    """One oracle local step of every sub-ResNet at batch B, one thread per sub-ResNet.  Returns seconds."""
+def oracle_step_all(cfg, a, mask, params, B, step_idx, subs=None):
+    """One oracle local step of the sub-ResNets in `subs` (default all) at batch B, one thread per sub-ResNet.  Returns seconds."""
     import oracle
-    S = cfg.S
-    data = [synth.batch(cfg, 0, step_idx, s, B=B, as_bf16=True) for s in range(S)]
-    moms = [np.zeros_like(params[s]) for s in range(S)]
+    subs = list(range(cfg.S)) if subs is None else subs
+    data = {s: synth.batch(cfg, 0, step_idx, s, B=B, as_bf16=True) for s in subs}
+    moms = {s: np.zeros_like(params[s]) for s in subs}
     t0 = time.perf_counter()
     th = [threading.Thread(target=oracle.step, args=(a, oracle.present_of(mask, s), params[s], moms[s], None, data[s][0], data[s][1]),
-                           kwargs=dict(lr=cfg.lr, mu=cfg.momentum, quant=0)) for s in range(S)]
+                           kwargs=dict(lr=cfg.lr, mu=cfg.momentum, quant=0)) for s in subs]
     for t in th:
         t.start()
     for t in th:
@@ -297,18 +352,25 @@ def oracle_step_all(cfg, a, mask, params, B, step_idx):
     return time.perf_counter() - t0
 
 
+def cpu_sample(cfg):
+    """Sub-ResNets per oracle step: as many as the host has cores, at most S (one thread each)."""
+    return list(range(min(cfg.S, max(1, os.cpu_count() or 1))))
+
+
 def cpu_baseline(cfg, budget_s: float):
-    """The oracle as it stands, on the host cores: one local step of all S sub-ResNets at a reduced batch."""
+    """The oracle as it stands, on the host cores: one local step at a reduced batch, one thread per sub-ResNet."""
     import oracle
     a = cfg.arch.to_int32()
     mask = oracle.partition(a, cfg.round_seed(0), cfg.S)
     p0, _ = synth.init_params(cfg.arch, cfg.init_seed)
     params = [p0.copy() for _ in range(cfg.S)]
-    t2 = oracle_step_all(cfg, a, mask, params, 2, 0)
-    B = int(max(2, min(cfg.batch, 2 * budget_s / max(t2, 1e-3))))
-    t = oracle_step_all(cfg, a, mask, params, B, 1)
-    return {"value": cfg.S * B / t, "unit": "images/s", "cores": cfg.S, "kind": "oracle",
-            "sample": f"one local step of all S={cfg.S} sub-ResNets of the same network at batch {B} per sub-ResNet "
+    subs = cpu_sample(cfg)
+    B, t = 2, oracle_step_all(cfg, a, mask, params, 2, 0, subs)
+    if t < budget_s / 4:                                         # cheap network: a larger batch within the budget
+        B = int(max(2, min(cfg.batch, 2 * budget_s / max(t, 1e-3))))
+        t = oracle_step_all(cfg, a, mask, params, B, 1, subs)
+    return {"value": len(subs) * B / t, "unit": "images/s", "cores": len(subs), "kind": "oracle",
+            "sample": f"one local step of {len(subs)} of the S={cfg.S} sub-ResNets of the same network at batch {B} per sub-ResNet "
                       f"({t:.1f} s, one thread per sub-ResNet, {os.cpu_count()} host cores present)"}
 
 
@@ -317,29 +379,32 @@ def run_reference(args):
     if rank != 0:
         return
     import oracle
-    cfg = synth.config(2)
+    cfg = synth.config(WORKLOADS[args.workload][0])
     a = cfg.arch.to_int32()
     mask = oracle.partition(a, cfg.round_seed(0), cfg.S)
     p0, _ = synth.init_params(cfg.arch, cfg.init_seed)
     params = [p0.copy() for _ in range(cfg.S)]
     K, W = args.steps, args.warmup
-    t2 = oracle_step_all(cfg, a, mask, params, 2, 0)
+    subs = cpu_sample(cfg)
+    t2 = oracle_step_all(cfg, a, mask, params, 2, 0, subs)
     per_step = 150.0 / max(K + W, 1)                       # the whole run should end within a few minutes
     B = int(max(2, min(cfg.batch, 2 * per_step / max(t2, 1e-3))))
+    if t2 > per_step and len(subs) > 1:                    # still too long at batch 2: fewer sub-ResNets per step
+        subs = subs[:max(1, int(len(subs) * per_step / t2))]
     for i in range(W):
-        oracle_step_all(cfg, a, mask, params, B, i)
+        oracle_step_all(cfg, a, mask, params, B, i, subs)
     t = 0.0
     for i in range(K):
-        t += oracle_step_all(cfg, a, mask, params, B, W + i)
-    v = cfg.S * B * K / t
-    sample = f"each step = one local step of all S={cfg.S} sub-ResNets at batch {B} per sub-ResNet (full workload: 128)"
+        t += oracle_step_all(cfg, a, mask, params, B, W + i, subs)
+    v = len(subs) * B * K / t
+    sample = (f"each step = one local step of {len(subs)} of the S={cfg.S} sub-ResNets at batch {B} per sub-ResNet "
+              f"(full workload: all {cfg.S} at batch {cfg.batch})")
     print(json.dumps({
         "impl": "reference", "metric": "sub-ResNet train images/s", "value": v, "unit": "images/s", "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
         "steps": K, "warmup": W, "ms_per_step": 1e3 * t / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
-        "config": {"workload": "configs[1]: CIFAR-shaped ResNet-110, S=4 sub-ResNets; CPU oracle on a bounded sample", "S": cfg.S,
-                   "batch_per_subnet": B},
-        "cpu_baseline": {"value": v, "unit": "images/s", "cores": cfg.S, "kind": "oracle", "sample": sample},
+        "config": {"workload": WORKLOADS[args.workload][1] + "; CPU oracle on a bounded sample", "S": cfg.S, "batch_per_subnet": B},
+        "cpu_baseline": {"value": v, "unit": "images/s", "cores": len(subs), "kind": "oracle", "sample": sample},
         "e2e": {"value": v, "unit": "images/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
 
 
@@ -411,7 +476,7 @@ def run_reassembly(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="wide", choices=["wide", "resnet110", "imagenet", "reassembly"],

@@ -205,7 +205,10 @@ const char* resist_noalloc_last_error(void);
 /* Per-kernel timing.  With profiling on, every launch of a local step, partition or aggregate is bracketed by
  * CUDA events on the call's stream and the call synchronises before returning; times, launch counts and the
  * algorithmic bytes and FLOPs of the work launched accumulate per kernel family until read.
- * resist_get_profile copies up to `cap` entries to host memory, returns the number of families in *n (may
+ * A family's launches are reported in two entries: those whose algorithmic work has an arithmetic intensity above
+ * 250 FLOP per byte (where the bf16 tensor peak of a B200 meets its HBM bandwidth) under "<name>@tensor", the
+ * others under "<name>": the first are held against the tensor peak, the second against HBM bandwidth.
+ * resist_get_profile copies up to `cap` entries to host memory, returns the number of entries in *n (may
  * exceed cap) and clears the counters. */
 typedef struct {
     char name[32];

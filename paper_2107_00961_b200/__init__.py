@@ -332,11 +332,11 @@ class Context:
 
     def get_profile(self) -> dict:
         """{family: dict(launches, operations, ms, bytes, flops)} since the last read; clears the counters."""
-        arr = (_ProfileEntry * 32)()
+        arr = (_ProfileEntry * 96)()
         n = C.c_int32(0)
-        self._check(self._lib.resist_get_profile(self._ctx, C.addressof(arr), 32, C.addressof(n)))
+        self._check(self._lib.resist_get_profile(self._ctx, C.addressof(arr), 96, C.addressof(n)))
         return {arr[i].name.decode(): {"launches": arr[i].launches, "operations": arr[i].operations, "ms": arr[i].ms,
-                                       "bytes": arr[i].bytes, "flops": arr[i].flops} for i in range(min(n.value, 32))}
+                                       "bytes": arr[i].bytes, "flops": arr[i].flops} for i in range(min(n.value, 96))}
 
     def step_info(self) -> dict:
         s = _StepInfo()

@@ -291,14 +291,16 @@ int resist_get_profile(resist_ctx* ctx, resist_profile_entry* out, int32_t cap, 
     if (!ctx || !n) return RESIST_EINVAL;
     Profiler& pf = ctx->prof;
     int k = 0;
-    for (int i = 0; i < PK_COUNT; ++i) {
-        if (!pf.ops[i]) continue;
-        if (out && k < cap) { resist_profile_entry& e = out[k]; memset(&e, 0, sizeof(e)); strncpy(e.name, PK_NAMES[i], sizeof(e.name) - 1);
-            e.launches = pf.launches[i]; e.operations = pf.ops[i]; e.ms = pf.ms[i]; e.bytes = pf.bytes[i]; e.flops = pf.flops[i]; }
-        ++k;
-    }
+    for (int i = 0; i < PK_COUNT; ++i)
+        for (int b = 0; b < 2; ++b) {
+            if (!pf.ops[i][b]) continue;
+            if (out && k < cap) { resist_profile_entry& e = out[k]; memset(&e, 0, sizeof(e));
+                snprintf(e.name, sizeof(e.name), "%s%s", PK_NAMES[i], b ? "@tensor" : "");
+                e.launches = pf.launches[i][b]; e.operations = pf.ops[i][b]; e.ms = pf.ms[i][b]; e.bytes = pf.bytes[i][b]; e.flops = pf.flops[i][b]; }
+            ++k;
+        }
     *n = k;
-    for (int i = 0; i < PK_COUNT; ++i) { pf.launches[i] = pf.ops[i] = 0; pf.ms[i] = pf.bytes[i] = pf.flops[i] = 0; }
+    for (int i = 0; i < PK_COUNT; ++i) for (int b = 0; b < 2; ++b) { pf.launches[i][b] = pf.ops[i][b] = 0; pf.ms[i][b] = pf.bytes[i][b] = pf.flops[i][b] = 0; }
     return RESIST_OK;
 }
 

@@ -47,13 +47,16 @@ enum ProfKind {
     PK_BN_STATS, PK_BN_APPLY, PK_BN_BWD_REDUCE, PK_BN_BWD_APPLY, PK_POOL_FWD, PK_POOL_BWD, PK_HEAD_FWD, PK_HEAD_BWD,
     PK_SGD, PK_PATCH, PK_SCATTER, PK_AGGREGATE, PK_UPSAMPLE, PK_CONV_FWD_MMA, PK_CONV_DGRAD_MMA, PK_CONV_WGRAD_MMA, PK_IM2COL, PK_BN_FWD_FUSED, PK_BN_BWD_FUSED, PK_CONV_FWD_MMA_BN, PK_CONV_DGRAD_MMA_BN, PK_BN_TILE_STATS, PK_COUNT
 };
+constexpr double PROFILE_RIDGE = 250.0;          // FLOP per byte at which a B200's bf16 tensor peak meets its HBM bandwidth (about 1.63e15 / 6.5e12)
 struct Profiler {
     bool on = false;
     std::vector<cudaEvent_t> pool; size_t used = 0;
     struct Pending { int kind; int launches; double bytes, flops; cudaEvent_t e0, e1; const char* label; };
     FILE* trace = nullptr;                                    // RESIST_LAUNCH_TRACE=<file>: one line per bracketed launch (label, ms, bytes, flops)
     std::vector<Pending> pending;
-    long long launches[PK_COUNT] = {}, ops[PK_COUNT] = {}; double ms[PK_COUNT] = {}, bytes[PK_COUNT] = {}, flops[PK_COUNT] = {};
+    // per family, split by what bounds the launch: [0] = HBM (arithmetic intensity of the launch's algorithmic work at or below
+    // PROFILE_RIDGE FLOP per byte), [1] = tensor cores (above it)
+    long long launches[PK_COUNT][2] = {}, ops[PK_COUNT][2] = {}; double ms[PK_COUNT][2] = {}, bytes[PK_COUNT][2] = {}, flops[PK_COUNT][2] = {};
     cudaEvent_t ev() { if (used == pool.size()) { cudaEvent_t e; cudaEventCreate(&e); pool.push_back(e); } return pool[used++]; }
     void begin(int kind, int launches_, double b, double f, cudaStream_t st, const char* label = "") {
         if (!on) return; Pending p{kind, launches_, b, f, ev(), ev(), label}; cudaEventRecord(p.e0, st); pending.push_back(p); }
@@ -61,7 +64,8 @@ struct Profiler {
     void collect(cudaStream_t st) {
         if (!on) return; cudaStreamSynchronize(st);
         for (auto& p : pending) { float t = 0.f; cudaEventElapsedTime(&t, p.e0, p.e1);
-            ms[p.kind] += t; launches[p.kind] += p.launches; ops[p.kind] += 1; bytes[p.kind] += p.bytes; flops[p.kind] += p.flops;
+            const int b = p.flops > PROFILE_RIDGE * p.bytes ? 1 : 0;
+            ms[p.kind][b] += t; launches[p.kind][b] += p.launches; ops[p.kind][b] += 1; bytes[p.kind][b] += p.bytes; flops[p.kind][b] += p.flops;
             if (trace) fprintf(trace, "%d\t%s\t%.6f\t%.0f\t%.0f\n", p.kind, p.label, t, p.bytes, p.flops); }
         if (trace) fflush(trace);
         pending.clear(); used = 0; }
