@@ -144,6 +144,9 @@ int resist_get_params(resist_ctx* ctx, int32_t subnet /* -1 = global */, float* 
 int resist_set_params(resist_ctx* ctx, const float* host_params, const float* host_buffers);   /* global */
 int resist_get_grads(resist_ctx* ctx, int32_t subnet, float* host_grads);    /* last step's dL/dW; absent blocks 0 */
 int resist_get_logits(resist_ctx* ctx, int32_t subnet, float* host_logits);  /* last step's [B][classes] */
+/* bf16 mode: the convolutions' copy of sub-ResNet `subnet`'s parameters (bf16 bit patterns, flat order): after every
+ * update it is the fp32 working copy rounded to nearest even (Algorithm 1's W_s, as the tensor cores read it). */
+int resist_get_shadow(resist_ctx* ctx, int32_t subnet, uint16_t* host_bf16);
 
 /* Work counters of the last local step call (grouped or single). */
 typedef struct {
@@ -180,6 +183,20 @@ int resist_bn_relu_forward(int32_t dtype, const void* x, const float* gamma, con
 int resist_bn_relu_backward(int32_t dtype, const void* x, const void* da, const float* gamma, const float* beta, float* stat,
                             const void* add, void* dx, float* dgamma, float* dbeta, int64_t m, int32_t C,
                             resist_stream stream);
+/* A convolution together with the BN+ReLU that consumes its output (Sec. 2.1: every convolution of a pre-activation
+ * block feeds a BN -> ReLU), launched the way the local step launches the pair, bf16 only:
+ *   mode 0: y = scale * conv(a, w) + add  [out];  a_out = relu(bn(y)) with batch statistics  [bn_out]; stat as in
+ *           resist_bn_relu_forward; run_mean / run_var updated when non-NULL.  x, bn_add, dgamma, dbeta unused.
+ *   mode 1: da = conv^T(dy, w) + add  [out];  dx = backward of the BN+ReLU with input x (a-shaped) and output gradient da,
+ *           plus bn_add when non-NULL  [bn_out]; dgamma, dbeta; stat must hold that BN's mean and 1/sqrt(var+eps).
+ * Layers of up to 64 channels run the BN inside the warp-MMA convolution's launch; wider ones take the statistics from
+ * the per-tile sums of the tcgen05 convolution's epilogue (forward) or run the BN launch behind the dgrad.
+ * *used_backend: 1 tcgen05, 2 warp-level MMA.  RESIST_EUNSUPPORTED when no tensor-core family takes the pair. */
+int resist_conv2d_bn_relu(int32_t mode, int32_t backend, const void* act, const void* wgt, const void* add, void* out,
+                          int32_t N, int32_t H, int32_t W, int32_t C, int32_t K, int32_t ksz, int32_t stride, float scale,
+                          const void* x, const float* gamma, const float* beta, float* stat, float* run_mean, float* run_var,
+                          const void* bn_add, void* bn_out, float* dgamma, float* dbeta, float eps, float momentum,
+                          int32_t* used_backend, resist_stream stream);
 const char* resist_layer_last_error(void);
 
 /* resist_bn_relu_forward for callers that cannot allocate device memory (the paper has no counterpart: this is a

@@ -84,12 +84,14 @@ def lib():
         L.resist_set_params.argtypes = [P, P, P]
         L.resist_get_grads.argtypes = [P, I, P]
         L.resist_get_logits.argtypes = [P, I, P]
+        L.resist_get_shadow.argtypes = [P, I, P]
         L.resist_get_step_info.argtypes = [P, C.POINTER(_StepInfo)]
         L.resist_splitmix64.argtypes = [U64, C.c_int64, P]
         L.resist_splitmix64.restype = None
         L.resist_set_profiling.argtypes = [P, I]
         L.resist_get_profile.argtypes = [P, P, I, P]
         L.resist_conv2d.argtypes = [I, I, I, P, P, P, P, I, I, I, I, I, I, I, F, P, P]
+        L.resist_conv2d_bn_relu.argtypes = [I, I, P, P, P, P, I, I, I, I, I, I, I, F, P, P, P, P, P, P, P, P, P, P, F, F, P, P]
         L.resist_bn_relu_forward.argtypes = [I, P, P, P, P, P, P, P, C.c_int64, I, F, F, P]
         L.resist_bn_relu_backward.argtypes = [I, P, P, P, P, P, P, P, P, P, C.c_int64, I, P]
         L.resist_layer_last_error.restype = C.c_char_p
@@ -103,8 +105,8 @@ def lib():
 
 EXPORTS = ["resist_init", "resist_destroy", "resist_partition", "resist_local_step", "resist_local_step_grouped",
            "resist_aggregate", "resist_eval", "resist_param_count", "resist_get_params", "resist_set_params",
-           "resist_get_grads", "resist_get_logits", "resist_get_step_info", "resist_splitmix64", "resist_last_error",
-           "resist_set_profiling", "resist_get_profile", "resist_conv2d", "resist_bn_relu_forward", "resist_bn_relu_backward", "resist_layer_last_error",
+           "resist_get_grads", "resist_get_logits", "resist_get_shadow", "resist_get_step_info", "resist_splitmix64", "resist_last_error",
+           "resist_set_profiling", "resist_get_profile", "resist_conv2d", "resist_conv2d_bn_relu", "resist_bn_relu_forward", "resist_bn_relu_backward", "resist_layer_last_error",
            "resist_bn_relu_forward_noalloc", "resist_noalloc_last_error"]
 
 
@@ -147,6 +149,32 @@ def resist_conv2d(mode: int, act: torch.Tensor, wgt: torch.Tensor, geom, add: Op
                                      add.data_ptr() if add is not None else None, out.data_ptr(), N, H, W, Cc, K, ksz,
                                      stride, scale, C.addressof(used), _stream_handle(stream)))
     return out, int(used.value)
+
+
+def resist_conv2d_bn_relu(mode: int, act: torch.Tensor, wgt: torch.Tensor, geom, gamma, beta, stat=None, x=None, add=None, bn_add=None,
+                          run_mean=None, run_var=None, scale: float = 1.0, eps=1e-5, momentum=0.1, backend: int = CONV_AUTO, stream=None):
+    """The convolution and the BN+ReLU that consumes its output, as one call (see resist.h).  mode 0 returns (y, a, stat, family);
+    mode 1 returns (da, dx, dgamma, dbeta, family)."""
+    N, H, W, Cc, K, ksz, stride = geom
+    P, Q = _odim(H, ksz, stride), _odim(W, ksz, stride)
+    dev = act.device
+    ptr = lambda t: t.data_ptr() if t is not None else None
+    used = C.c_int32(0)
+    if mode == 0:
+        out = torch.empty(N, P, Q, K, dtype=act.dtype, device=dev)
+        stat = torch.zeros(4 * K, dtype=torch.float32, device=dev)
+        dg = db = None
+    else:
+        out = torch.empty(N, H, W, Cc, dtype=act.dtype, device=dev)
+        dg, db = torch.zeros(Cc, dtype=torch.float32, device=dev), torch.zeros(Cc, dtype=torch.float32, device=dev)
+    bn_out = torch.empty_like(out)
+    _layer_check(lib().resist_conv2d_bn_relu(mode, backend, act.data_ptr(), wgt.data_ptr(), ptr(add), out.data_ptr(), N, H, W, Cc, K, ksz, stride,
+                                             scale, ptr(x), gamma.data_ptr(), beta.data_ptr(), stat.data_ptr(), ptr(run_mean), ptr(run_var),
+                                             ptr(bn_add), bn_out.data_ptr(), ptr(dg), ptr(db), eps, momentum, C.addressof(used),
+                                             _stream_handle(stream)))
+    if mode == 0:
+        return out, bn_out, stat, int(used.value)
+    return out, bn_out, dg, db, int(used.value)
 
 
 def resist_bn_relu_forward(x: torch.Tensor, gamma, beta, run_mean=None, run_var=None, eps=1e-5, momentum=0.1, stream=None):
@@ -325,6 +353,12 @@ class Context:
     def get_logits(self, subnet: int, B: int) -> np.ndarray:
         out = np.empty((B, self.classes), dtype=np.float32)
         self._check(self._lib.resist_get_logits(self._ctx, subnet, out.ctypes.data))
+        return out
+
+    def get_shadow(self, subnet: int) -> np.ndarray:
+        """bf16 bit patterns (uint16) of the convolutions' copy of a sub-ResNet's parameters, flat order."""
+        out = np.empty(self.n_params, dtype=np.uint16)
+        self._check(self._lib.resist_get_shadow(self._ctx, subnet, out.ctypes.data))
         return out
 
     def set_profiling(self, on: bool):

@@ -199,3 +199,88 @@ extern "C" int resist_bn_relu_backward(int32_t dtype, const void* x, const void*
     if (e != cudaSuccess) { g_layer_error = cudaGetErrorString(e); return RESIST_ECUDA; }
     return RESIST_OK;
 }
+
+namespace resist {
+bool conv_mma_can_fuse_bn(const ConvProb& p, int mode, int C);
+size_t conv_mma_bn_partial_bytes(int C, int sms);
+int conv_tc_stat_tiles(const ConvProb& p);
+void launch_bn_finalize_tiles(const BnProb* d, int nprob, int max_c, cudaStream_t s);
+}
+
+// A convolution together with the BN+ReLU that consumes its output, launched the way the local step launches the pair (bf16):
+//   mode 0: y = scale * conv(a, w) + add;  a_out = relu(bn(y)) with batch statistics (stat, running statistics updated)
+//   mode 1: da = conv^T(dy, w) + add;      dx = BN+ReLU backward of the BN with input x and output gradient da (+ bn_add), dgamma, dbeta
+// Warp-MMA family (narrow layers): the BN runs inside the convolution's launch.  tcgen05 family: forward statistics come from the
+// per-tile sums of the convolution's epilogue (a finalize launch, then the elementwise pass); backward is the cooperative BN launch
+// behind the dgrad.  *used_backend: 1 tcgen05, 2 warp-level MMA.
+extern "C" int resist_conv2d_bn_relu(int32_t mode, int32_t backend, const void* act, const void* wgt, const void* add, void* out,
+                                     int32_t N, int32_t H, int32_t W, int32_t C, int32_t K, int32_t ksz, int32_t stride, float scale,
+                                     const void* x, const float* gamma, const float* beta, float* stat, float* run_mean, float* run_var,
+                                     const void* bn_add, void* bn_out, float* dgamma, float* dbeta, float eps, float momentum,
+                                     int32_t* used_backend, resist_stream stream) {
+    if (!act || !wgt || !out || !gamma || !beta || !stat || !bn_out || mode < 0 || mode > 1 || N < 1 || H < 1 || W < 1 || C < 1 || K < 1 ||
+        (ksz != 1 && ksz != 3) || stride < 1 || stride > 2) { g_layer_error = "bad argument"; return RESIST_EINVAL; }
+    if (mode == 1 && (!x || !dgamma || !dbeta)) { g_layer_error = "backward needs x, dgamma, dbeta"; return RESIST_EINVAL; }
+    cudaStream_t st = (cudaStream_t)stream;
+    ConvProb p{};
+    p.N = N; p.H = H; p.W = W; p.C = C; p.K = K; p.ksz = ksz; p.stride = stride; p.pad = (ksz - 1) / 2;
+    p.P = out_dim(H, ksz, stride); p.Q = out_dim(W, ksz, stride); p.scale = scale; p.add = add; p.out = out; p.act = act; p.wgt = wgt;
+    const long long rows_out = (long long)N * p.P * p.Q, rows_in = (long long)N * H * W;
+    if (mode == CONV_FWD) { p.M = (int)rows_out; p.Ncol = K; p.Kred = ksz * ksz * C; } else { p.M = (int)rows_in; p.Ncol = C; p.Kred = ksz * ksz * K; }
+    int sm = 148; int dev = 0; cudaGetDevice(&dev); cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev);
+    BnProb bn{};
+    bn.gamma = gamma; bn.beta = beta; bn.stat = stat; bn.run_mean = run_mean; bn.run_var = run_var; bn.eps = eps; bn.momentum = momentum;
+    bn.dgamma = dgamma; bn.dbeta = dbeta;
+    if (mode == CONV_FWD) { bn.x = out; bn.a = bn_out; bn.m = rows_out; bn.C = K; }
+    else { bn.x = x; bn.da = out; bn.dx = bn_out; bn.add = bn_add; bn.m = rows_in; bn.C = C; }
+    bn_chunking(bn, true, std::max(8, 2 * sm));
+    if (!bn.vec) { g_layer_error = "the BN does not take the bf16 vector path (channels a power of two times 8, 16-byte aligned tensors)"; return RESIST_EUNSUPPORTED; }
+    const bool want_mma = backend == RESIST_CONV_AUTO || backend == RESIST_CONV_WARP_MMA, want_tc = backend == RESIST_CONV_AUTO || backend == RESIST_CONV_TCGEN05;
+    ConvProb q = p;                                           // the warp-MMA kernels take a stride-2 dgrad as a stride-1 problem that reads dy through its tables
+    if (mode == CONV_DGRAD && stride == 2) { q.stride = 1; q.P = H; q.Q = W; q.dy_sub = 2; q.dy_P = p.P; q.dy_Q = p.Q; }
+    int be = 0;
+    if (want_mma && conv_mma_supported(q, mode) && conv_mma_can_fuse_bn(q, mode, bn.C)) be = 2;
+    else if (want_tc && conv_tc_supported(p, mode) && !(mode == CONV_DGRAD && ksz == 1 && stride == 2)) be = 1;
+    if (used_backend) *used_backend = be;
+    if (!be) { g_layer_error = "no tensor-core family takes this convolution with its BN"; return RESIST_EUNSUPPORTED; }
+    const int tiles = be == 1 && mode == CONV_FWD ? conv_tc_stat_tiles(p) : 0;
+    const size_t partial_bytes = be == 2 ? conv_mma_bn_partial_bytes(bn.C, sm) : std::max((size_t)bn.chunks * 2 * bn.C * 8, (size_t)tiles * 2 * bn.C * 4);
+    const int n_tc = be == 1 ? conv_tc_count(p, mode) : 1;
+    std::vector<char> hd(be == 1 ? (size_t)n_tc * conv_tc_prob_bytes() : conv_mma_prob_bytes());
+    const size_t hd_room = (hd.size() + 255) / 256 * 256;
+    char* blob = nullptr;
+    cudaError_t e = cudaMalloc(&blob, 1024 + hd_room + partial_bytes + 256);
+    if (e != cudaSuccess) { g_layer_error = cudaGetErrorString(e); return RESIST_ENOMEM; }
+    bn.partial = (double*)(blob + 1024 + hd_room);
+    bool ok = true;
+    if (be == 2) ok = conv_mma_fill(q, mode, hd.data(), &bn);
+    else {
+        if (mode == CONV_FWD) { p.stat_tiles = (float*)bn.partial; bn.chunks = tiles; }
+        ok = conv_tc_fill(p, mode, hd.data()) == n_tc;
+    }
+    if (!ok) { cudaFree(blob); g_layer_error = "descriptor set-up failed"; return RESIST_ECUDA; }
+    e = cudaMemcpyAsync(blob, &bn, sizeof(bn), cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(blob + 1024, hd.data(), hd.size(), cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) {
+        if (be == 2) {
+            if (!launch_conv_mma_probs(blob + 1024, 1, conv_mma_tiles(hd.data()), conv_mma_smem(hd.data()), conv_mma_pick_variant(q, mode) + 512, st)) {
+                cudaGetLastError(); cudaFree(blob); g_layer_error = "the fused launch was refused (cooperative grid too large?)"; return RESIST_ECUDA; }
+        } else {
+            int t = 0; size_t packed = 0;
+            for (int i = 0; i < n_tc; ++i) { const char* h = hd.data() + (size_t)i * conv_tc_prob_bytes(); t = std::max(t, conv_tc_tiles(h)); packed = conv_tc_merge(packed, conv_tc_smem(h)); }
+            launch_conv_tc_probs(blob + 1024, n_tc, t, packed, st);
+            if (mode == CONV_FWD) { launch_bn_finalize_tiles((BnProb*)blob, 1, bn.C, st); launch_bn_apply((BnProb*)blob, 1, bn.m * bn.C, true, st); }
+            else if (!(bn.C <= 512 && launch_bn_fused((BnProb*)blob, 1, bn.chunks, 1, st))) {
+                cudaGetLastError();
+                launch_bn_bwd_reduce((BnProb*)blob, 1, bn.chunks, bn.C, true, st); launch_bn_bwd_apply((BnProb*)blob, 1, bn.m * bn.C, true, st);
+            }
+        }
+        e = cudaGetLastError();
+    }
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    cudaFree(blob);
+    if (e != cudaSuccess) { g_layer_error = cudaGetErrorString(e); return RESIST_ECUDA; }
+    if (be == 1) { const int stv = conv_tc_read_status();
+        if (stv) { g_layer_error = "a bounded device-side wait gave up (code " + std::to_string(stv) + ")"; return RESIST_ETIMEOUT; } }
+    return RESIST_OK;
+}

@@ -259,6 +259,15 @@ int resist_get_grads(resist_ctx* ctx, int32_t subnet, float* host_grads) {
     return device_status(ctx);
 }
 
+int resist_get_shadow(resist_ctx* ctx, int32_t subnet, uint16_t* host_bf16) {
+    if (!ctx || !host_bf16) return RESIST_EINVAL;
+    if (subnet < 0 || subnet >= ctx->S) { ctx->err = "subnet out of range"; return RESIST_EINVAL; }
+    if (ctx->opts.dtype != RESIST_BF16 || !ctx->pa.wb) { ctx->err = "no bf16 copy in fp32 mode"; return RESIST_EUNSUPPORTED; }
+    CK(cudaDeviceSynchronize());
+    CK(cudaMemcpy(host_bf16, ctx->pa.wb + (long long)subnet * ctx->pa.n, (size_t)ctx->L.n_params * 2, cudaMemcpyDeviceToHost));
+    return RESIST_OK;
+}
+
 int resist_get_logits(resist_ctx* ctx, int32_t subnet, float* host_logits) {
     if (!ctx || !host_logits) return RESIST_EINVAL;
     if (subnet < 0 || subnet >= ctx->S) { ctx->err = "subnet out of range"; return RESIST_EINVAL; }

@@ -57,7 +57,7 @@ def run_protocol_both(arch, S, B, steps, seed, dtype, quant, grouped, lib_mod, p
     mask_gpu = ctx.partition(policy_seed, S)
     mask_cpu = oracle.partition(a, policy_seed, S)
     tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
-    out = {"mask_gpu": mask_gpu, "mask_cpu": mask_cpu, "steps": []}
+    out = {"mask_gpu": mask_gpu, "mask_cpu": mask_cpu, "steps": [], "arch": arch}
     subs = [p0.copy() for _ in range(S)]
     moms = [np.zeros_like(p0) for _ in range(S)]
     bufs = [buf0.copy() for _ in range(S)]

@@ -90,7 +90,21 @@ def test_fp32_ragged_sizes_span_tiles(lib_mod):
     check_fp32(out, arch)
 
 
-def check_bf16(out, arch, tol=2e-2, grads=True):
+def buffers_worst(arch, got, ref, skip_blocks=()):
+    """Worst normalised max-abs error over the BN layers' running statistics (mean | var per BN, in layout order)."""
+    worst, o = 0.0, 0
+    for t in synth.param_layout(arch)[0]:
+        if t.kind == "gamma":
+            n = 2 * t.size
+            if t.block not in skip_blocks:
+                worst = max(worst, norm_max_abs(got[o:o + n], ref[o:o + n]))
+            o += n
+    return worst
+
+
+def check_bf16(out, arch, tol=2e-2, grads=False, params_tol=None, bufs_tol=None):
+    """logits and loss at `tol`; grads=True: every gradient tensor at `tol` too; params_tol / bufs_tol: every updated parameter
+    tensor / every BN's running statistics of the blocks the sub-ResNet holds, normalised max-abs."""
     np.testing.assert_array_equal(out["mask_gpu"], out["mask_cpu"])
     for rec in out["steps"]:
         for s, r in enumerate(rec["subs"]):
@@ -99,10 +113,28 @@ def check_bf16(out, arch, tol=2e-2, grads=True):
             if grads:
                 v, name = per_tensor(arch, r["grads_gpu"], r["grads_cpu"], norm_max_abs)
                 assert v < tol, ("grads", name, v)
+            if params_tol is not None:
                 v, name = per_tensor(arch, r["params_gpu"], r["params_cpu"], norm_max_abs, skip_blocks=absent(out, s))
-                assert v < tol, ("params", name, v)
+                assert v < params_tol, ("params", name, v)
+            if bufs_tol is not None:
+                v = buffers_worst(arch, r["bufs_gpu"], r["bufs_cpu"], skip_blocks=absent(out, s))
+                assert v < bufs_tol, ("running statistics", v)
     np.testing.assert_array_equal(out["global_gpu"], out["global_from_gpu_subs"])
     np.testing.assert_array_equal(out["global_buf_gpu"], out["global_buf_from_gpu_subs"])
+
+
+def check_shadow(out, S):
+    """The convolutions' bf16 copy of every held parameter is the fp32 working copy rounded to nearest even, bit for bit."""
+    ctx = out["ctx"]
+    ts = synth.param_layout(out["arch"])[0]
+    for s in range(S):
+        w, _ = ctx.get_params(s)
+        sh = ctx.get_shadow(s)
+        hold = absent(out, s)
+        for t in ts:
+            if t.block in hold:
+                continue
+            np.testing.assert_array_equal(sh[t.offset:t.offset + t.size], synth.bf16_bits(w[t.offset:t.offset + t.size]), err_msg=t.name)
 
 
 # A note on what a whole-step bf16 comparison can show.  Rounding an activation to bf16 moves it by up to
@@ -121,12 +153,32 @@ def test_tiny_bf16_step(lib_mod, backend):
     c = synth.config(1)
     out = run_protocol_both(c.arch, 2, 8, 1, 5, "bf16", 0, True, lib_mod, conv_backend=backend)
     check_bf16(out, c.arch, grads=False)
+    # configs[0]'s network, one step, against the oracle with the same storage rounding: every gradient tensor and every updated
+    # parameter tensor within 2e-2 normalised max-abs (observed 3e-3 and 1e-4), running statistics within 1e-3
+    out = run_protocol_both(c.arch, 2, 8, 1, 5, "bf16", 1, True, lib_mod, conv_backend=backend)
+    check_bf16(out, c.arch, grads=True, params_tol=2e-2, bufs_tol=1e-3)
     for B, seed, grouped in ((8, 5, True), (32, 6, False)):
         out = run_protocol_both(c.arch, 2, B, 1, seed, "bf16", 1, grouped, lib_mod, conv_backend=backend)
         check_bf16(out, c.arch, grads=False)
         for s, r in enumerate(out["steps"][0]["subs"]):
             g, h = r["grads_gpu"].astype(np.float64), r["grads_cpu"].astype(np.float64)
             assert g @ h / (np.linalg.norm(g) * np.linalg.norm(h)) > 0.97, s
+
+
+@pytest.mark.parametrize("arch_name", ["tiny", "resnet110"])
+def test_bf16_second_step_reads_the_refreshed_weight_copy(lib_mod, arch_name):
+    """Two local steps in bf16: the second step's convolutions read the bf16 copy that the first step's update wrote.  After each
+    protocol the copy must be the fp32 working copy rounded to nearest even, bit for bit, and the second step's logits must still
+    follow the oracle (a stale copy would repeat the first step's forward pass: the logits of step 2 would equal those of step 1's
+    weights, far outside the bound)."""
+    arch = synth.config(1).arch if arch_name == "tiny" else synth.config(2).arch
+    S = 2 if arch_name == "tiny" else 4
+    out = run_protocol_both(arch, S, 8, 2, 5 if arch_name == "tiny" else 31, "bf16", 1, True, lib_mod)
+    check_shadow(out, S)
+    for s, r in enumerate(out["steps"][1]["subs"]):
+        assert norm_max_abs(r["logits_gpu"], r["logits_cpu"]) < 6e-2, s        # observed 1.4e-2 (tiny), 3.4e-2 (ResNet-110): two chaotic steps
+        stale = out["steps"][0]["subs"][s]["logits_gpu"]
+        assert norm_max_abs(r["logits_gpu"], r["logits_cpu"]) < 0.5 * norm_max_abs(stale, r["logits_cpu"]) or norm_max_abs(stale, r["logits_cpu"]) < 6e-2
 
 
 @pytest.mark.parametrize("backend", [1, 0, 2, 4])
@@ -136,7 +188,10 @@ def test_resnet110_bf16_reduced_batch(lib_mod, backend):
     out = run_protocol_both(c.arch, c.S, 8, 1, 31, "bf16", 0, True, lib_mod, policy_seed=c.round_seed(0), conv_backend=backend)
     check_bf16(out, c.arch, grads=False)
     out = run_protocol_both(c.arch, c.S, 8, 1, 31, "bf16", 1, True, lib_mod, policy_seed=c.round_seed(0), conv_backend=backend)
-    check_bf16(out, c.arch, grads=False)
+    # every updated parameter tensor within 4e-2 of its largest entry (observed 1.4-1.8e-2: at batch 8 the ReLU masks of the two
+    # sides differ in a few places, see the note above), running statistics of every BN within 1e-2 (observed 3e-3)
+    check_bf16(out, c.arch, grads=False, params_tol=4e-2, bufs_tol=1e-2)
+    check_shadow(out, c.S)
     for s, r in enumerate(out["steps"][0]["subs"]):
         g, h = r["grads_gpu"].astype(np.float64), r["grads_cpu"].astype(np.float64)
         assert g @ h / (np.linalg.norm(g) * np.linalg.norm(h)) > 0.85, s          # same direction
@@ -164,8 +219,11 @@ def test_bottleneck_bf16_mixed_kernel_families(lib_mod, backend):
     for s, r in enumerate(out["steps"][0]["subs"]):
         g, h = r["grads_gpu"].astype(np.float64), r["grads_cpu"].astype(np.float64)
         assert g @ h / (np.linalg.norm(g) * np.linalg.norm(h)) > 0.9, s
+        # worst gradient tensor against the same-rounding oracle: a handful of flipped ReLU masks at batch 8 move a small BN
+        # tensor by up to its own size; what is held is that no tensor is off by more (a wrong kernel gives 1.4 and more: unrelated values)
         v, name = per_tensor(arch, r["grads_gpu"], r["grads_cpu"], norm_max_abs)
-        print("worst gradient tensor against the same-rounding oracle:", name, v)
+        assert v < 1.0, (name, v)
+    check_bf16(out, arch, grads=False, params_tol=8e-2, bufs_tol=2e-2)
 
 
 def test_wide_bottleneck_bf16_all_widths_of_configuration_3(lib_mod):
@@ -175,7 +233,8 @@ def test_wide_bottleneck_bf16_all_widths_of_configuration_3(lib_mod):
     arch = synth.wide_cifar_arch(policy="stage_first_shared", depths=(2, 2, 2, 2))
     out = run_protocol_both(arch, 2, 4, 1, 7, "bf16", 1, True, lib_mod)
     assert out["info"]["cuda_core_convs"] == 0 and out["info"]["tensor_core_convs"] > 0
-    check_bf16(out, arch, grads=False)
+    check_bf16(out, arch, grads=False, params_tol=8e-2, bufs_tol=2e-2)          # observed 3.5e-2 and 4e-3 at batch 4
+    check_shadow(out, 2)
     for s, r in enumerate(out["steps"][0]["subs"]):
         g, h = r["grads_gpu"].astype(np.float64), r["grads_cpu"].astype(np.float64)
         assert g @ h / (np.linalg.norm(g) * np.linalg.norm(h)) > 0.9, s
