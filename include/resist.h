@@ -16,7 +16,8 @@
  *    memory only through the resist_allocator given at init (or cudaMalloc when that is NULL).
  *  - Work is enqueued on the given stream; calls that return host data synchronise that stream.
  *  - State machine: init -> partition -> (local_step)* -> aggregate -> partition ...; a call out of
- *    order returns RESIST_ESTATE.
+ *    order (a local step before the first partition, or after aggregate without a new partition)
+ *    returns RESIST_ESTATE.
  *
  * Flat parameter order (all fp32 on the boundary): stem conv; stem BN gamma, beta (if any); per block in
  * network order: basic = bn1 g,b | conv1 3x3 | bn2 g,b | conv2 3x3 | projection 1x1 (if any);
@@ -100,7 +101,7 @@ typedef struct {
     void* user;
 } resist_allocator;
 
-/* Creates a context holding the global ResNet h(W) (Algorithm 1, "randomly initialized ResNet"): He-normal
+/* Creates a context holding the global ResNet h(W) with random initial weights (Algorithm 1, input): He-normal
  * conv and head weights drawn from a splitmix64 stream seeded with `seed`, gamma 1, beta 0, bias 0, running
  * mean 0, running var 1.  arch, opts: host.  alloc may be NULL.  *out receives the context. */
 int resist_init(const resist_arch* arch, const resist_opts* opts, uint64_t seed, const resist_allocator* alloc,
@@ -110,7 +111,7 @@ int resist_destroy(resist_ctx* ctx);
 /* subResNets(h(W), S) of Algorithm 1 (Sec. 2.2): permutes the partitionable block indices with Fisher-Yates
  * driven by splitmix64(round_seed) (i from P-1 down to 1, j = next() mod (i+1)), deals position j of the
  * permutation to sub-ResNet j mod S, gives every other block to all S; then copies the global parameters into
- * the S working copies ("distribute each h_s(W_s) to a different worker") and restarts their momentum.
+ * the S working copies (the step of Algorithm 1 that hands every sub-ResNet to its worker) and restarts their momentum.
  * member_mask: host, [num_blocks], bit s set = block is in sub-ResNet s (may be NULL).
  * Errors: S < 1 or S > 32, or S > P with min_depth == 0 -> RESIST_EINVAL. */
 int resist_partition(resist_ctx* ctx, uint64_t round_seed, int32_t S, uint32_t* member_mask, resist_stream stream);
@@ -242,6 +243,11 @@ int resist_get_profile(resist_ctx* ctx, resist_profile_entry* out, int32_t cap, 
 void resist_splitmix64(uint64_t seed, int64_t n, uint64_t* out);
 
 const char* resist_last_error(resist_ctx* ctx);   /* ctx may be NULL: the last init failure */
+
+/* Test hook: stores `code` in the device status word that a kernel's bounded wait writes when it gives up, so that the next
+ * call that synchronises (resist_aggregate, a parity tap, a layer-level call) returns RESIST_ETIMEOUT and clears the word.
+ * No kernel has to time out for the reporting path to be tested. */
+int resist_debug_set_wait_status(int32_t code);
 
 #ifdef __cplusplus
 }

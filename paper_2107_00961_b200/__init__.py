@@ -85,6 +85,7 @@ def lib():
         L.resist_get_grads.argtypes = [P, I, P]
         L.resist_get_logits.argtypes = [P, I, P]
         L.resist_get_shadow.argtypes = [P, I, P]
+        L.resist_debug_set_wait_status.argtypes = [I]
         L.resist_get_step_info.argtypes = [P, C.POINTER(_StepInfo)]
         L.resist_splitmix64.argtypes = [U64, C.c_int64, P]
         L.resist_splitmix64.restype = None
@@ -105,7 +106,7 @@ def lib():
 
 EXPORTS = ["resist_init", "resist_destroy", "resist_partition", "resist_local_step", "resist_local_step_grouped",
            "resist_aggregate", "resist_eval", "resist_param_count", "resist_get_params", "resist_set_params",
-           "resist_get_grads", "resist_get_logits", "resist_get_shadow", "resist_get_step_info", "resist_splitmix64", "resist_last_error",
+           "resist_get_grads", "resist_get_logits", "resist_get_shadow", "resist_debug_set_wait_status", "resist_get_step_info", "resist_splitmix64", "resist_last_error",
            "resist_set_profiling", "resist_get_profile", "resist_conv2d", "resist_conv2d_bn_relu", "resist_bn_relu_forward", "resist_bn_relu_backward", "resist_layer_last_error",
            "resist_bn_relu_forward_noalloc", "resist_noalloc_last_error"]
 

@@ -1,6 +1,6 @@
 // Bandwidth kernels over the flat parameter arrays: the fused SGD-momentum update (Algorithm 1, the
 // local update W_s = W_s - eta dL/dW_s), the scatter of the global parameters into the S working
-// copies ("distribute each h_s(W_s)"), and the reassembly aggregate(.) (Sec. 2.3, Appendix B).
+// copies (the hand-out step of Algorithm 1), and the reassembly aggregate(.) (Sec. 2.3, Appendix B).
 // Work is described by a table of segments (contiguous runs of parameters treated alike); every CTA
 // owns one 4096-element chunk of one segment, found by binary search, and moves 16 bytes per thread
 // per access when the chunk starts on a 16-byte boundary.

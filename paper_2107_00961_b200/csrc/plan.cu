@@ -723,6 +723,7 @@ static int ensure_workspace(resist_ctx* ctx, int B, std::vector<Needs>& needs) {
     cudaDeviceSynchronize();
     ctx_free(ctx, ctx->d_ws); ctx->d_ws = nullptr; ctx->ws_bytes = 0; ctx->ws_slice = 0;
     for (Plan& p : ctx->plans) p.valid = false;
+    std::fill(ctx->logits_dev.begin(), ctx->logits_dev.end(), nullptr);      // they pointed into the workspace just released
     ctx->d_ws = ctx_alloc(ctx, slice * ctx->S);
     if (!ctx->d_ws) { ctx->err = "allocator returned NULL for the activation workspace"; return RESIST_ENOMEM; }
     ctx->ws_bytes = slice * ctx->S; ctx->ws_slice = slice;
@@ -874,6 +875,7 @@ int resist_local_step(resist_ctx* ctx, int32_t subnet, const void* images, const
                       float* loss_out, resist_stream stream) {
     if (!ctx) return RESIST_EINVAL;
     if (ctx->state < 1) { ctx->err = "local step before partition"; return RESIST_ESTATE; }
+    if (ctx->state == 3) { ctx->err = "local step after aggregate: the working copies are stale until the next partition"; return RESIST_ESTATE; }
     if (subnet < 0 || subnet >= ctx->S) { ctx->err = "subnet out of range"; return RESIST_EINVAL; }
     if (!images || !labels || B < 2 || B > 1024) { ctx->err = "need images, labels and 2 <= B <= 1024"; return RESIST_EINVAL; }
     cudaStream_t st = (cudaStream_t)stream;
@@ -889,6 +891,7 @@ int resist_local_step_grouped(resist_ctx* ctx, const void* const* images, const 
                               float* loss_out, resist_stream stream) {
     if (!ctx) return RESIST_EINVAL;
     if (ctx->state < 1) { ctx->err = "local step before partition"; return RESIST_ESTATE; }
+    if (ctx->state == 3) { ctx->err = "local step after aggregate: the working copies are stale until the next partition"; return RESIST_ESTATE; }
     if (!images || !labels || B < 2 || B > 1024) { ctx->err = "need images, labels and 2 <= B <= 1024"; return RESIST_EINVAL; }
     PatchArgs pa{};
     for (int s = 0; s < ctx->S; ++s) { if (!images[s] || !labels[s]) { ctx->err = "null image or label pointer"; return RESIST_EINVAL; }

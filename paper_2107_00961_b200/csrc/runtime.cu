@@ -77,6 +77,7 @@ void ctx_free(resist_ctx* ctx, void* p) {
 
 void free_plan(resist_ctx* ctx, Plan& p);   // plan.cu
 int conv_tc_read_status();                  // conv_tc.cu
+int* conv_tc_status_word();
 
 // after a synchronisation: did any bounded device-side wait give up?
 static int device_status(resist_ctx* ctx) {
@@ -392,7 +393,15 @@ int resist_aggregate(resist_ctx* ctx, resist_stream stream) {
     ctx->prof.end(st); ctx->prof.collect(st);
     CK(cudaGetLastError());
     CK(cudaStreamSynchronize(st));
+    ctx->state = 3;                                            // the working copies are stale until the next partition
     return device_status(ctx);
+}
+
+// Test hook of the bounded-wait reporting: writes `code` into the status word the kernels' bounded waits write on expiry, so that
+// the next call that synchronises reports RESIST_ETIMEOUT (no kernel has to give up for the mapping to be exercised).
+int resist_debug_set_wait_status(int32_t code) {
+    int* w = conv_tc_status_word();
+    return w && cudaMemcpy(w, &code, 4, cudaMemcpyHostToDevice) == cudaSuccess ? RESIST_OK : RESIST_ECUDA;
 }
 
 }  // extern "C"

@@ -96,7 +96,7 @@ struct resist_ctx {
     resist_allocator alloc{}; bool own_alloc = false;
     int S = 0, S_cap = 0;                                      // current and allocated number of sub-ResNets
     std::vector<uint32_t> mask;                                // member_mask of the current round
-    int state = 0;                                             // 0 = initialised, 1 = partitioned, 2 = stepped
+    int state = 0;                                             // 0 = initialised, 1 = partitioned, 2 = stepped, 3 = aggregated
     unsigned long long generation = 0;                         // bumped by every partition
     resist::ParamArrays pa{};                                  // arrays hold S_cap + 1 copies; the last is the evaluation copy
     void* d_param_blob = nullptr;

@@ -343,6 +343,18 @@ def test_min_depth_partition_and_partial_sharing(lib_mod):
     assert any(m == 3 for m in out_mask[1:])          # one block sits in both sub-ResNets (Fig. 1)
 
 
+def test_init_draws_the_documented_he_normal_stream(lib_mod):
+    """resist_init's own initialiser against the input generator's (same splitmix64 stream, Box-Muller in double, one normal
+    stream in flat parameter order): equal to within one fp32 ulp of the libm functions involved."""
+    for arch, seed in ((synth.tiny_arch(), 3), (small_bottleneck_arch(), 11)):
+        ctx = lib_mod.Context(arch.to_int32(), dtype=lib_mod.F32, seed=seed)
+        p, b = ctx.get_params(-1)
+        p_ref, b_ref = synth.init_params(arch, seed)
+        np.testing.assert_array_equal(b, b_ref)
+        assert max_rel_err(p, p_ref, floor=1e-6) < 1e-6
+        assert (p == p_ref).mean() > 0.99
+
+
 def test_partition_bit_exact_on_all_configs(lib_mod):
     for cfg in (1, 2, 3, 4):
         c = synth.config(cfg)
@@ -407,6 +419,19 @@ def test_error_paths(lib_mod):
         ctx.local_step(0, x[:1], y[:1], 0.1)            # B < 2
     ctx.local_step(0, x, y, 0.1)                        # and the context still works
     torch.cuda.synchronize()
+    ctx.aggregate()
+    with pytest.raises(lib_mod.ResistError) as e:
+        ctx.local_step(0, x, y, 0.1)                    # working copies are stale after aggregate until the next partition
+    assert e.value.code == -2
+    ctx.partition(2, 2)
+    ctx.local_step(0, x, y, 0.1)
+    torch.cuda.synchronize()
+    # a bounded device-side wait that gave up is reported once by the next synchronising call, then the context works again
+    assert lib_mod.lib().resist_debug_set_wait_status(4) == 0
+    with pytest.raises(lib_mod.ResistError) as e:
+        ctx.get_params(0)
+    assert e.value.code == -5 and "wait" in str(e.value)
+    ctx.get_params(0)
     bad = a.copy()
     bad[10 + 2] = 5                                     # first block's cin no longer matches the stem
     with pytest.raises(lib_mod.ResistError):

@@ -147,3 +147,39 @@ def test_bf16_storage_rounding_is_nearest_even():
     y = oracle.conv_fwd(x, w, 1, quant=1)
     ref = torch.from_numpy(x).to(torch.bfloat16).to(torch.float32).numpy()
     np.testing.assert_array_equal(y, ref)
+
+
+def _bf16(x):
+    """nearest-even bf16 rounding by the library routine (torch), back in fp32"""
+    return torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32)).to(torch.bfloat16).to(torch.float32).numpy()
+
+
+def test_bf16_storage_rounding_points_of_the_layer_routines():
+    """quant=1 rounds what a layer STORES (Q15: activations and activation gradients are bf16, every sum is wider) and nothing
+    else: each layer's quant=1 output must be the bf16 rounding of its quant=0 output, element by element, and the statistics
+    a layer returns (mean, 1/std, dgamma, dbeta, running statistics) must not be rounded at all."""
+    a, w = _bf16(rnd(2, 6, 5, 8)), _bf16(rnd(16, 3, 3, 8) * 0.25)
+    add = _bf16(rnd(2, 6, 5, 16))
+    for stride in (1, 2):
+        sub = np.ascontiguousarray(add[:, ::stride, ::stride])        # a residual of the output's shape
+        y0 = oracle.conv_fwd(a, w, stride, add=sub, scale=0.5)
+        y1 = oracle.conv_fwd(a, w, stride, add=sub, scale=0.5, quant=1)
+        np.testing.assert_array_equal(y1, _bf16(y0))
+        dy = _bf16(rnd(*y0.shape))
+        adda = _bf16(rnd(*a.shape))
+        np.testing.assert_array_equal(oracle.conv_dgrad(dy, w, a.shape[1:3], stride, add=adda, quant=1),
+                                      _bf16(oracle.conv_dgrad(dy, w, a.shape[1:3], stride, add=adda)))
+    x = _bf16(rnd(60, 8) * 1.5 + rnd(8)[None, :])
+    g, b = (1 + 0.2 * rnd(8)).astype(np.float32), (0.3 * rnd(8)).astype(np.float32)
+    rm0, rv0, rm1, rv1 = np.zeros(8, np.float32), np.ones(8, np.float32), np.zeros(8, np.float32), np.ones(8, np.float32)
+    a0, mean0, istd0 = oracle.bn_relu_fwd(x, g, b, rm0, rv0)
+    a1, mean1, istd1 = oracle.bn_relu_fwd(x, g, b, rm1, rv1, quant=1)
+    np.testing.assert_array_equal(a1, _bf16(a0))
+    for u, v in ((mean0, mean1), (istd0, istd1), (rm0, rm1), (rv0, rv1)):
+        np.testing.assert_array_equal(u, v)
+    da, skip = _bf16(rnd(60, 8)), _bf16(rnd(60, 8))
+    dx0, dg0, db0 = oracle.bn_relu_bwd(da, x, g, b, mean0, istd0, add=skip)
+    dx1, dg1, db1 = oracle.bn_relu_bwd(da, x, g, b, mean0, istd0, add=skip, quant=1)
+    np.testing.assert_array_equal(dx1, _bf16(dx0))
+    np.testing.assert_array_equal(dg0, dg1)
+    np.testing.assert_array_equal(db0, db1)
