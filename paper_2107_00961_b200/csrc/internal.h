@@ -68,11 +68,11 @@ inline void bn_chunking(BnProb& p, bool bf16, int target_chunks = 0) {
     p.rows_per_chunk = (int)rpc; p.chunks = (int)((m + rpc - 1) / rpc);
 }
 
-// im2col of a few-channel input (C * ksz * ksz <= 32): dst [N*P*Q][32] (bf16, columns (r, s, c), zero beyond), and the
-// layer's weights packed alike: w32 [K][32].
+// im2col of a few-channel input: dst [N*P*Q][cols] (bf16, columns (r, s, c), zero beyond C*ksz*ksz), and the
+// layer's weights packed alike: w32 [K][cols].
 struct ColProb {
     const void* src; void* dst; const void* w; void* w32;
-    int N, H, W, C, ksz, stride, pad, P, Q, K, kk, pad_;
+    int N, H, W, C, ksz, stride, pad, P, Q, K, kk, cols;   // kk = C*ksz*ksz real columns; cols = row pitch (multiple of 8, <= 256)
 };
 
 struct UpProb {           // zero stuffing of a stride-2 layer's dy: src [N,P,Q,K] -> dst [N,H,W,K] (bf16, K % 8 == 0)
@@ -133,6 +133,7 @@ void launch_head_bwd(const HeadProb* d, int nprob, int maxB, int maxC, int max_c
 // statistics, finalisation and apply of BN+ReLU in one cooperative launch (bf16 vector path, training mode); false if the grid cannot be co-resident
 bool launch_bn_fused(const BnProb* d, int nprob, int max_chunks, int backward, cudaStream_t s);   // kernels_ref.cu
 void launch_im2col(const ColProb* d, int nprob, long long max_rows, cudaStream_t s);      // kernels_ref.cu
+void launch_repack_rows(const ConvProb* d, int nprob, int max_elems, cudaStream_t s);     // kernels_ref.cu
 void launch_zero_stuff(const UpProb* d, int nprob, long long max_vecs, cudaStream_t s);   // conv_tc.cu
 
 // ---- launchers (kernels_bw.cu)

@@ -704,18 +704,18 @@ void launch_head_bwd(const HeadProb* d, int nprob, int maxB, int maxC, int max_c
 __global__ void __launch_bounds__(256) im2col_kernel(const ColProb* __restrict__ probs) {
     const ColProb& p = probs[blockIdx.y];
     const __nv_bfloat16* __restrict__ src = (const __nv_bfloat16*)p.src;
-    const long long rows = (long long)p.N * p.P * p.Q, total = rows * 4;
+    const int cols = p.cols, G = cols >> 3;                       // row pitch in columns (a multiple of 8, at most 256), 8-column groups
+    const long long rows = (long long)p.N * p.P * p.Q, total = rows * G;
     // column j of a row = tap (r, s), channel c: the three are looked up, not divided out, for every element
-    __shared__ int s_r[32], s_s[32], s_off[32];
-    if (threadIdx.x < 32) {
-        const int j = threadIdx.x;
+    __shared__ int s_r[256], s_s[256], s_off[256];
+    for (int j = threadIdx.x; j < cols; j += blockDim.x) {
         if (j < p.kk) { const int c = j % p.C, rs = j / p.C, ss = rs % p.ksz, r = rs / p.ksz; s_r[j] = r - p.pad; s_s[j] = ss - p.pad; s_off[j] = ((r - p.pad) * p.W + (ss - p.pad)) * p.C + c; }
         else { s_r[j] = -(1 << 20); s_s[j] = 0; s_off[j] = 0; }   // beyond the taps: never inside the image
     }
     __syncthreads();
     const unsigned short* __restrict__ src16 = reinterpret_cast<const unsigned short*>(src);
     for (long long id = blockIdx.x * (long long)blockDim.x + threadIdx.x; id < total; id += (long long)gridDim.x * blockDim.x) {
-        const int g = (int)(id & 3); const long long row = id >> 2;
+        const int g = G == 4 ? (int)(id & 3) : (int)(id % G); const long long row = G == 4 ? id >> 2 : id / G;
         const int q = (int)(row % p.Q); const long long t = row / p.Q; const int pr = (int)(t % p.P); const int n = (int)(t / p.P);
         const int y0 = pr * p.stride, x0 = q * p.stride;
         const long long base = (((long long)n * p.H + y0) * p.W + x0) * p.C;
@@ -727,20 +727,35 @@ __global__ void __launch_bounds__(256) im2col_kernel(const ColProb* __restrict__
             const bool in = y >= 0 && y < p.H && xx >= 0 && xx < p.W;
             h[e] = in ? src16[base + s_off[j]] : (unsigned short)0;
         }
-        *reinterpret_cast<uint4*>((__nv_bfloat16*)p.dst + row * 32 + g * 8) =
+        *reinterpret_cast<uint4*>((__nv_bfloat16*)p.dst + row * cols + g * 8) =
             make_uint4(h[0] | ((unsigned)h[1] << 16), h[2] | ((unsigned)h[3] << 16), h[4] | ((unsigned)h[5] << 16), h[6] | ((unsigned)h[7] << 16));
-        if (id < (long long)p.K * 4) {                             // weights: w[k][kk] -> w32[k][32]
-            const int kx = (int)(id >> 2);
+        if (id < (long long)p.K * G) {                             // weights: w[k][kk] -> w32[k][cols]
+            const int kx = (int)(id / G);
             __align__(16) __nv_bfloat16 wv[8];
 #pragma unroll
             for (int e = 0; e < 8; ++e) { const int j = g * 8 + e; wv[e] = j < p.kk ? ((const __nv_bfloat16*)p.w)[(long long)kx * p.kk + j] : __float2bfloat16(0.f); }
-            *reinterpret_cast<uint4*>((__nv_bfloat16*)p.w32 + kx * 32 + g * 8) = *reinterpret_cast<const uint4*>(wv);
+            *reinterpret_cast<uint4*>((__nv_bfloat16*)p.w32 + (long long)kx * cols + g * 8) = *reinterpret_cast<const uint4*>(wv);
         }
     }
 }
 void launch_im2col(const ColProb* d, int nprob, long long max_rows, cudaStream_t s) {
     long long gx = (max_rows * 4 + 255) / 256; if (gx > 148 * 16) gx = 148 * 16; if (gx < 1) gx = 1;
     im2col_kernel<<<dim3((unsigned)gx, nprob), 256, 0, s>>>(d);
+}
+
+// dst[r][0..cols) = src[r][0..cols) for rows of different pitch (fp32): the weight gradient of an im2col'ed stem, computed with
+// the padded column count, goes to its place in the gradient vector
+__global__ void repack_rows_kernel(const ConvProb* __restrict__ probs) {
+    const ConvProb& p = probs[blockIdx.y];
+    const float* src = (const float*)p.act; float* dst = (float*)p.out;
+    const int n = p.M * p.Ncol;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+        const int r = i / p.Ncol, c = i - r * p.Ncol;
+        dst[i] = src[(long long)r * p.Kred + c];
+    }
+}
+void launch_repack_rows(const ConvProb* d, int nprob, int max_elems, cudaStream_t s) {
+    repack_rows_kernel<<<dim3(std::max(1, std::min((max_elems + 255) / 256, 148)), nprob), 256, 0, s>>>(d);
 }
 
 }  // namespace resist

@@ -206,37 +206,51 @@ struct Builder {
         o.bn.partial = bn_partial;
     }
 
-    // A stem with few input channels (C * k * k <= 32, bf16): the images are expanded once per step to rows of 32
-    // columns, and forward and wgrad become 1x1 problems with 32 input channels on the warp-MMA kernels.
-    bool stem_as_im2col(const ConvRef& cr) const {
-        return ctx->opts.dtype == RESIST_BF16 && ctx->opts.conv_backend != RESIST_CONV_CUDA_CORES && ctx->opts.conv_backend != RESIST_CONV_TCGEN05 &&
-               cr.cin * cr.k * cr.k <= 32 && cr.cout % 16 == 0 && cr.cout <= 64;
+    // A stem with few input channels (bf16): the images are expanded once per step to rows of (tap, channel) columns, and forward
+    // and wgrad become 1x1 problems on the tensor-core kernels.  Up to 32 columns (3x3 stems of 3 channels): rows of 32 on the
+    // warp-MMA kernels.  More (7x7 stems: 147 columns, pitch 152): on the tcgen05 kernels, whose TMA fills the last 64-column
+    // slab with zeros; the weight gradient is computed at the row pitch and repacked.
+    int stem_cols(const ConvRef& cr) const {
+        if (ctx->opts.dtype != RESIST_BF16 || ctx->opts.conv_backend == RESIST_CONV_CUDA_CORES) return 0;
+        const int kk = cr.cin * cr.k * cr.k, pref = ctx->opts.conv_backend;
+        if (kk <= 32 && cr.cout % 16 == 0 && cr.cout <= 64 && pref != RESIST_CONV_TCGEN05) return 32;
+        if (kk > 32 && kk <= 256 && cr.cin < 8 && cr.cout % 8 == 0 && (pref == RESIST_CONV_AUTO || pref == RESIST_CONV_TCGEN05)) return (kk + 7) / 8 * 8;
+        return 0;
     }
+    bool stem_as_im2col(const ConvRef& cr) const { return stem_cols(cr) != 0; }
+    float* stem_dw = nullptr;                                     // wide stem: weight gradient at the row pitch, before repacking
     void stem_im2col(long long key, const ConvRef& cr, int N, int H, int Wd) {
-        const int P = out_dim(H, cr.k, cr.stride), Q = out_dim(Wd, cr.k, cr.stride);
-        col_buf = (char*)take((size_t)N * P * Q * 64); col_w = (char*)take((size_t)cr.cout * 64);
+        const int P = out_dim(H, cr.k, cr.stride), Q = out_dim(Wd, cr.k, cr.stride), cols = stem_cols(cr);
+        col_buf = (char*)take((size_t)N * P * Q * cols * 2); col_w = (char*)take((size_t)cr.cout * cols * 2);
+        if (cols > 32) stem_dw = (float*)take((size_t)cr.cout * cols * 4);
         Op u{}; u.key = key; u.sub = sub; u.kind = OP_IM2COL;
-        u.col = ColProb{nullptr, col_buf, CW(cr.w), col_w, N, H, Wd, cr.cin, cr.k, cr.stride, (cr.k - 1) / 2, P, Q, cr.cout, cr.cin * cr.k * cr.k, 0};
+        u.col = ColProb{nullptr, col_buf, CW(cr.w), col_w, N, H, Wd, cr.cin, cr.k, cr.stride, (cr.k - 1) / 2, P, Q, cr.cout, cr.cin * cr.k * cr.k, cols};
         ops->push_back(u);
     }
     // the stem as a 1x1 problem on the im2col'ed images: forward (out = y) or wgrad (dy given; dw goes to the stem's gradient)
     void stem_conv(long long key, int mode, const ConvRef& cr, const void* dy, void* out, int N, int H, int Wd) {
-        const int P = out_dim(H, cr.k, cr.stride), Q = out_dim(Wd, cr.k, cr.stride);
+        const int P = out_dim(H, cr.k, cr.stride), Q = out_dim(Wd, cr.k, cr.stride), cols = stem_cols(cr), kk = cr.cin * cr.k * cr.k;
+        const bool wide = cols > 32;
         Op op{}; op.key = key; op.sub = sub; op.kind = mode == CONV_FWD ? OP_CONV_FWD : OP_CONV_WGRAD;
         ConvProb& p = op.conv;
-        p.N = N; p.H = P; p.W = Q; p.C = 32; p.K = cr.cout; p.ksz = 1; p.stride = 1; p.pad = 0; p.P = P; p.Q = Q; p.scale = 1.f;
+        p.N = N; p.H = P; p.W = Q; p.C = cols; p.K = cr.cout; p.ksz = 1; p.stride = 1; p.pad = 0; p.P = P; p.Q = Q; p.scale = 1.f;
         const long long rows = (long long)N * P * Q;
         p.act = col_buf;
-        if (mode == CONV_FWD) { p.wgt = col_w; p.out = out; p.M = (int)rows; p.Ncol = p.K; p.Kred = 32; }
-        else { p.wgt = dy; p.out = G() + cr.w; p.M = p.K; p.Ncol = 32; p.Kred = (int)rows; p.wg_ld = cr.cin * cr.k * cr.k; p.wg_cols = p.wg_ld; }
+        if (mode == CONV_FWD) { p.wgt = col_w; p.out = out; p.M = (int)rows; p.Ncol = p.K; p.Kred = cols; }
+        else { p.wgt = dy; p.out = wide ? stem_dw : G() + cr.w; p.M = p.K; p.Ncol = cols; p.Kred = (int)rows; if (!wide) { p.wg_ld = kk; p.wg_cols = kk; } }
         p.tiles_m = (p.M + 63) / 64; p.tiles_n = (p.Ncol + 63) / 64; p.splits = 1; p.ktiles_per_split = (p.Kred + 15) / 16;
-        flops += 2LL * rows * p.K * cr.k * cr.k * cr.cin;
+        flops += 2LL * rows * p.K * kk;
         size_t pb = 0;
-        op.backend = pick_backend(p, mode, wgrad_target_ctas(ctx), &pb, RESIST_CONV_WARP_MMA);
+        op.backend = pick_backend(p, mode, wgrad_target_ctas(ctx), &pb, wide ? RESIST_CONV_TCGEN05 : RESIST_CONV_WARP_MMA);
         if (mode == CONV_WGRAD) { wgrad_partial_need = std::max(wgrad_partial_need, pb); p.partial = wgrad_partial; }
         ++n_tc;
         ops->push_back(op);
-        if (mode == CONV_FWD) last_fwd_conv = op.backend >= 1000 ? (int)ops->size() - 1 : -1;
+        if (mode == CONV_FWD) { last_fwd_conv = op.backend >= 1000 ? (int)ops->size() - 1 : -1; last_tc_fwd = op.backend == 1 ? (int)ops->size() - 1 : -1; }
+        if (mode == CONV_WGRAD && wide) {                      // [K][cols] -> the stem's [K][k][k][C] in the gradient vector
+            Op r{}; r.key = key + 1; r.sub = sub; r.kind = OP_REPACK;
+            r.conv.act = stem_dw; r.conv.out = G() + cr.w; r.conv.M = cr.cout; r.conv.Ncol = kk; r.conv.Kred = cols;
+            ops->push_back(r);
+        }
     }
 
     // chunks per BN problem that give the fused (cooperative) kernels about two CTAs per SM over all sub-ResNets
@@ -500,11 +514,16 @@ static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool s
             const ConvProb& c = ops[i].conv;
             snprintf(L.label, sizeof(L.label), "%dx%d C%d K%d HW%d s%d%s x%d", c.ksz, c.ksz, c.C, c.K, c.H, c.stride, c.dy_sub == 2 ? "*" : "", L.count);
         } else if (ops[i].kind != OP_HEAD_FWD && ops[i].kind != OP_HEAD_BWD && ops[i].kind != OP_POOL_FWD && ops[i].kind != OP_POOL_BWD &&
-                   ops[i].kind != OP_UPSAMPLE && ops[i].kind != OP_IM2COL && ops[i].kind != OP_SPLITK)
+                   ops[i].kind != OP_UPSAMPLE && ops[i].kind != OP_IM2COL && ops[i].kind != OP_SPLITK && ops[i].kind != OP_REPACK)
             snprintf(L.label, sizeof(L.label), "bn m%lld C%d x%d", ops[i].bn.m, ops[i].bn.C, L.count);
         for (size_t k = i; k < j; ++k) {
             const Op& o = ops[k]; const int slot = single ? 0 : o.sub;
             switch (o.kind) {
+                case OP_REPACK: {
+                    if (k == i) L.first = (int)conv.size();
+                    conv.push_back(o.conv);
+                    L.max_elems = std::max<long long>(L.max_elems, (long long)o.conv.M * o.conv.Ncol); L.bytes += 8.0 * o.conv.M * o.conv.Ncol;
+                    break; }
                 case OP_CONV_FWD: case OP_CONV_DGRAD: case OP_CONV_WGRAD: case OP_SPLITK: {
                     if (o.backend >= 200 && o.kind != OP_SPLITK) {   // warp-level MMA kernels: their own descriptor arrays
                         const ConvProb& p = o.conv;
@@ -597,7 +616,7 @@ static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool s
                     col.push_back(o.col);
                     const double rows = (double)o.col.N * o.col.P * o.col.Q;
                     L.max_elems = std::max<long long>(L.max_elems, (long long)rows);
-                    L.bytes += 64.0 * rows + 2.0 * o.col.N * o.col.H * o.col.W * o.col.C;
+                    L.bytes += 2.0 * o.col.cols * rows + 2.0 * o.col.N * o.col.H * o.col.W * o.col.C;
                     break; }
                 case OP_UPSAMPLE: {
                     if (k == i) L.first = (int)up.size();
@@ -635,7 +654,7 @@ static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool s
                     case OP_CONV_FWD: case OP_CONV_DGRAD: wr.push_back(o.conv.out);
                         if (o.fuse == 1) wr.push_back(o.bn.a); else if (o.fuse == 2) wr.push_back(o.bn.dx);
                         break;
-                    case OP_CONV_WGRAD: case OP_SPLITK: break;
+                    case OP_CONV_WGRAD: case OP_SPLITK: case OP_REPACK: break;
                     case OP_BN_STATS: case OP_BN_BWD_REDUCE: case OP_BN_TILE_STATS: break;
                     case OP_BN_APPLY: case OP_BN_FWD_FUSED: wr.push_back(o.bn.a); break;
                     case OP_BN_BWD_APPLY: case OP_BN_BWD_FUSED: wr.push_back(o.bn.dx); break;
@@ -644,7 +663,7 @@ static int upload_plan(resist_ctx* ctx, Plan& plan, std::vector<Op>& ops, bool s
             }
             L.join_before = false;
             if (L.kind == OP_CONV_WGRAD) { for (size_t k = i; k < j; ++k) { inflight.push_back(ops[k].conv.act); inflight.push_back(ops[k].conv.wgt); } }
-            else if (L.kind != OP_SPLITK && !inflight.empty()) {
+            else if (L.kind != OP_SPLITK && L.kind != OP_REPACK && !inflight.empty()) {
                 bool hit = always;
                 for (const void* w : wr) for (const void* r : inflight) if (w == r) hit = true;
                 if (hit) { L.join_before = true; inflight.clear(); }
@@ -784,7 +803,7 @@ static int run_plan(resist_ctx* ctx, Plan& plan, const PatchArgs& pa, bool updat
     for (const Launch& L : plan.launches) {
         // early start of a warp-MMA convolution: not behind the im2col pass that writes the stem's packed weights, not while profiling
         const bool pdl_ok = !pf.on && prev_kind != OP_IM2COL; prev_kind = L.kind;
-        const bool on_side = overlap && (L.kind == OP_CONV_WGRAD || (L.kind == OP_SPLITK && side_pending));
+        const bool on_side = overlap && (L.kind == OP_CONV_WGRAD || ((L.kind == OP_SPLITK || L.kind == OP_REPACK) && side_pending));
         if (on_side) {
             cudaEventRecord(ctx->ev_fork, main_st); cudaStreamWaitEvent(ctx->side_stream, ctx->ev_fork, 0);
             st = ctx->side_stream;
@@ -797,7 +816,7 @@ static int run_plan(resist_ctx* ctx, Plan& plan, const PatchArgs& pa, bool updat
             case OP_CONV_FWD: pk = (L.backend >= 1000 && ((L.backend - 1000) & MMA_BACKEND_FUSED)) ? PK_CONV_FWD_MMA_BN : L.backend >= 200 ? PK_CONV_FWD_MMA : L.backend ? PK_CONV_FWD_TC : PK_CONV_FWD_CC; break;
             case OP_CONV_DGRAD: pk = (L.backend >= 1000 && ((L.backend - 1000) & MMA_BACKEND_FUSED)) ? PK_CONV_DGRAD_MMA_BN : L.backend >= 200 ? PK_CONV_DGRAD_MMA : L.backend ? PK_CONV_DGRAD_TC : PK_CONV_DGRAD_CC; break;
             case OP_CONV_WGRAD: pk = L.backend >= 200 ? PK_CONV_WGRAD_MMA : L.backend ? PK_CONV_WGRAD_TC : PK_CONV_WGRAD_CC; break;
-            case OP_SPLITK: pk = PK_SPLITK; break;
+            case OP_SPLITK: case OP_REPACK: pk = PK_SPLITK; break;
             case OP_BN_STATS: pk = PK_BN_STATS; nk = 2; break;
             case OP_BN_APPLY: pk = PK_BN_APPLY; break;
             case OP_BN_BWD_REDUCE: pk = PK_BN_BWD_REDUCE; nk = 2; break;
@@ -826,6 +845,7 @@ static int run_plan(resist_ctx* ctx, Plan& plan, const PatchArgs& pa, bool updat
                 else launch_conv_ref(plan.d_conv + L.first, L.count, L.gx, mode, bf, st);
                 ++n_launch; break; }
             case OP_SPLITK: launch_splitk_reduce(plan.d_conv + L.first, L.count, (int)L.max_elems, st); ++n_launch; break;
+            case OP_REPACK: launch_repack_rows(plan.d_conv + L.first, L.count, (int)L.max_elems, st); ++n_launch; break;
             case OP_BN_STATS: launch_bn_stats(plan.d_bn + L.first, L.count, L.gx, L.max_c, bf, st); n_launch += 2; break;
             case OP_BN_APPLY: launch_bn_apply(plan.d_bn + L.first, L.count, L.max_elems, bf, st); ++n_launch; break;
             case OP_BN_BWD_REDUCE: launch_bn_bwd_reduce(plan.d_bn + L.first, L.count, L.gx, L.max_c, bf, st); n_launch += 2; break;

@@ -19,7 +19,7 @@ Layout make_layout(const resist_arch& a, const std::vector<resist_block>& blocks
 
 enum OpKind {
     OP_CONV_FWD, OP_CONV_DGRAD, OP_CONV_WGRAD, OP_SPLITK, OP_BN_STATS, OP_BN_APPLY, OP_BN_BWD_REDUCE, OP_BN_BWD_APPLY,
-    OP_POOL_FWD, OP_POOL_BWD, OP_HEAD_FWD, OP_HEAD_BWD, OP_UPSAMPLE, OP_IM2COL, OP_BN_FWD_FUSED, OP_BN_BWD_FUSED, OP_BN_TILE_STATS
+    OP_POOL_FWD, OP_POOL_BWD, OP_HEAD_FWD, OP_HEAD_BWD, OP_UPSAMPLE, OP_IM2COL, OP_BN_FWD_FUSED, OP_BN_BWD_FUSED, OP_BN_TILE_STATS, OP_REPACK
 };
 
 // One operation of one sub-ResNet, keyed so that equal keys of different sub-ResNets share a launch.
