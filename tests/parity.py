@@ -1,4 +1,7 @@
 """Comparators and drivers shared by the GPU parity tests."""
+import os
+from concurrent.futures import ThreadPoolExecutor
+
 import numpy as np
 import torch
 
@@ -48,7 +51,7 @@ def to_dev(x, dtype):
 
 
 def run_protocol_both(arch, S, B, steps, seed, dtype, quant, grouped, lib_mod, policy_seed=77, lr=LR, mu=MOM,
-                      conv_backend=0):
+                      conv_backend=0, with_oracle=True):
     """One ResIST round on both sides from identical inputs.  Returns a dict of everything comparable."""
     a = arch.to_int32()
     p0, buf0 = synth.perturbed_params(arch, seed)
@@ -81,13 +84,24 @@ def run_protocol_both(arch, S, B, steps, seed, dtype, quant, grouped, lib_mod, p
                 ctx.local_step(s, dx[s], dy[s], lr, loss[s:s + 1])
         torch.cuda.synchronize()
         rec = {"loss_gpu": loss.cpu().numpy(), "subs": []}
+        # the sub-ResNets are independent: the oracle steps them on one host thread each (the C routine releases the interpreter)
+        if not with_oracle:                   # GPU side only (a second backend on inputs the oracle has already seen)
+            rec["subs"] = [{"logits_gpu": ctx.get_logits(s, B), "grads_gpu": ctx.get_grads(s)} for s in range(S)]
+            out["steps"].append(rec)
+            continue
+        with ThreadPoolExecutor(max_workers=max(1, min(S, os.cpu_count() or 1))) as ex:
+            outs = list(ex.map(lambda s: oracle.step(a, oracle.present_of(mask_cpu, s), subs[s], moms[s], bufs[s], xs[s], ys[s], lr=lr, mu=mu,
+                                                     quant=quant), range(S)))
         for s in range(S):
-            o = oracle.step(a, oracle.present_of(mask_cpu, s), subs[s], moms[s], bufs[s], xs[s], ys[s], lr=lr, mu=mu, quant=quant)
+            o = outs[s]
             gp, gb = ctx.get_params(s)
             rec["subs"].append({"loss_cpu": o["loss"], "logits_cpu": o["logits"], "grads_cpu": o["grads"],
                                 "params_cpu": subs[s].copy(), "bufs_cpu": bufs[s].copy(),
                                 "logits_gpu": ctx.get_logits(s, B), "grads_gpu": ctx.get_grads(s), "params_gpu": gp, "bufs_gpu": gb})
         out["steps"].append(rec)
+    out.update(ctx=ctx, info=ctx.step_info())
+    if not with_oracle:
+        return out
     # reassembly: the oracle applied to the GPU's own working copies must match bit for bit
     gsubs = [ctx.get_params(s) for s in range(S)]
     ctx.aggregate()
