@@ -91,6 +91,9 @@ typedef struct {
                                 tensor-core family where the shape allows, CUDA cores elsewhere.  With _AUTO and _WARP_MMA
                                 the BN+ReLU (forward or backward) that consumes a warp-MMA convolution's output runs inside
                                 that convolution's launch; _WARP_MMA_UNFUSED keeps BN in launches of its own */
+    int32_t bn_stat_period;  /* 0 or 1: resist_aggregate averages the BN running statistics at every call; k > 1: only at every k-th
+                                call (Sec. 5, ImageNet settings: statistics aggregated once per many synchronisation rounds); in
+                                between, the global statistics keep their last aggregated values */
 } resist_opts;
 
 /* Device-memory source.  alloc returns a device pointer aligned to >= 256 bytes or NULL; release frees it.

@@ -41,7 +41,7 @@ class _Arch(C.Structure):
 class _Opts(C.Structure):
     _fields_ = [("dtype", C.c_int32), ("momentum", C.c_float), ("weight_decay", C.c_float), ("bn_eps", C.c_float),
                 ("bn_momentum", C.c_float), ("min_depth", C.c_int32), ("momentum_policy", C.c_int32),
-                ("conv_backend", C.c_int32)]
+                ("conv_backend", C.c_int32), ("bn_stat_period", C.c_int32)]
 
 
 _ALLOC_FN = C.CFUNCTYPE(C.c_void_p, C.c_void_p, C.c_size_t)
@@ -223,7 +223,7 @@ class Context:
     def __init__(self, arch_int32: np.ndarray, dtype: int = F32, momentum: float = 0.9, weight_decay: float = 0.0,
                  bn_eps: float = 1e-5, bn_momentum: float = 0.1, min_depth: int = 0,
                  momentum_policy: int = MOMENTUM_RESTART, conv_backend: int = CONV_AUTO, seed: int = 0,
-                 device: str = "cuda:0"):
+                 device: str = "cuda:0", bn_stat_period: int = 0):
         if not torch.cuda.is_available():
             raise RuntimeError("the ResIST library needs a CUDA device; there is no CPU path")
         self._lib = lib()
@@ -236,7 +236,7 @@ class Context:
             for j, (name, _) in enumerate(_Block._fields_):
                 setattr(self._blocks[i], name, int(a[10 + 8 * i + j]))
         arch = _Arch(*[int(v) for v in a[:10]], C.cast(self._blocks, C.POINTER(_Block)))
-        opts = _Opts(dtype, momentum, weight_decay, bn_eps, bn_momentum, min_depth, momentum_policy, conv_backend)
+        opts = _Opts(dtype, momentum, weight_decay, bn_eps, bn_momentum, min_depth, momentum_policy, conv_backend, bn_stat_period)
         # device memory comes from torch's caching allocator
         self._held = {}
 

@@ -380,7 +380,9 @@ int resist_aggregate(resist_ctx* ctx, resist_stream stream) {
         if (!L.blk.empty() && run_mask != all) { flush(buffers ? L.blk.back().buf_end : L.blk.back().end); run_mask = all; }
         flush(total);
     };
-    build(false, segs, chunks); bchunks = chunks; build(true, bsegs, bchunks);   // one table, one launch: the statistics' chunks follow the parameters'
+    // BN running statistics: at every call, or at every bn_stat_period-th one (Sec. 5, ImageNet settings)
+    const bool with_stats = ctx->opts.bn_stat_period <= 1 || (++ctx->aggregate_calls % ctx->opts.bn_stat_period) == 0;
+    build(false, segs, chunks); bchunks = chunks; if (with_stats) build(true, bsegs, bchunks);   // one table, one launch: the statistics' chunks follow the parameters'
     segs.insert(segs.end(), bsegs.begin(), bsegs.end());
     int rc = ensure_seg_table(ctx, (int)segs.size());
     if (rc) return rc;

@@ -98,6 +98,7 @@ struct resist_ctx {
     std::vector<uint32_t> mask;                                // member_mask of the current round
     int state = 0;                                             // 0 = initialised, 1 = partitioned, 2 = stepped, 3 = aggregated
     unsigned long long generation = 0;                         // bumped by every partition
+    long long aggregate_calls = 0;                             // counts resist_aggregate calls for opts.bn_stat_period
     resist::ParamArrays pa{};                                  // arrays hold S_cap + 1 copies; the last is the evaluation copy
     void* d_param_blob = nullptr;
     // workspace: per sub-ResNet slices of one allocation

@@ -150,6 +150,16 @@ def resnet101_arch(policy: str = "paper_section3", depths=(3, 4, 23, 3), classes
     return Arch(in_hw, in_hw, 3, classes, 7, 2, 64, 1, 1, _stack(BOTTLENECK, 64, depths, w, mids, policy))
 
 
+def resnet152_arch(policy: str = "paper_section3", classes: int = 1000, in_hw: int = 224) -> Arch:
+    """The deeper variants of the appendix on deeper architectures: the extra blocks go to the third section ([3,8,36,3] and, below,
+    [3,24,36,3] in the usual layouts), so the share of partitioned blocks grows (P = 35 for both: 36 blocks in section 3, minus the strided one)."""
+    return resnet101_arch(policy, (3, 8, 36, 3), classes, in_hw)
+
+
+def resnet200_arch(policy: str = "paper_section3", classes: int = 1000, in_hw: int = 224) -> Arch:
+    return resnet101_arch(policy, (3, 24, 36, 3), classes, in_hw)
+
+
 @dataclass
 class Config:
     cfg: int

@@ -45,6 +45,8 @@ SHAPES = [
     # wide layers of the bottleneck nets: several 64-channel slabs, several column tiles, 4x4 maps, strided projections
     (2, 4, 4, 512, 512, 3, 1), (2, 16, 16, 256, 512, 1, 2), (2, 8, 8, 1024, 256, 1, 1), (2, 8, 8, 256, 1024, 1, 1),
     (2, 8, 8, 256, 256, 3, 2), (3, 6, 10, 136, 72, 3, 1), (2, 9, 7, 64, 128, 1, 2),
+    # maps of 2x2 and 1x1 positions (the last stage of a deep net on a small input)
+    (5, 2, 2, 128, 128, 3, 1), (5, 4, 4, 128, 256, 3, 2), (6, 1, 1, 128, 128, 3, 1), (5, 2, 2, 128, 256, 1, 2),
 ]
 
 

@@ -371,6 +371,100 @@ def test_min_depth_partition_and_partial_sharing(lib_mod):
     assert any(m == 3 for m in out_mask[1:])          # one block sits in both sub-ResNets (Fig. 1)
 
 
+def test_min_depth_round_with_a_block_held_by_two_of_three(lib_mod):
+    """Sec. 2.6 "Subnetwork Depth" / the starred block of Fig. 1 on the device: 5 partitionable blocks, S = 3, minimum depth 2 -> the
+    deal is 2, 2, 1 and the short sub-ResNet is topped up with a block another one holds.  One fp32 round: masks bit-exact, every
+    sub-ResNet's step within 1e-4 of the oracle, and the reassembly of the block with two of three owners bit-exact against the
+    oracle's mean over exactly those two."""
+    arch = synth.Arch(8, 8, 3, 10, 3, 1, 8, 0, 0, synth._stack(synth.BASIC, 8, (6,), (8,), (8,), "stage_first_shared"))
+    a = arch.to_int32()
+    p0, buf0 = synth.perturbed_params(arch, 3)
+    ctx = lib_mod.Context(a, dtype=lib_mod.F32, momentum=MOM, min_depth=2)
+    ctx.set_params(p0, buf0)
+    seed = next(sd for sd in range(50) if any(bin(int(m)).count("1") == 2 for m in oracle.partition(a, sd, 3, min_depth=2)))
+    mask = oracle.partition(a, seed, 3, min_depth=2)
+    np.testing.assert_array_equal(ctx.partition(seed, 3), mask)
+    subs, moms, bufs = [p0.copy() for _ in range(3)], [np.zeros_like(p0) for _ in range(3)], [buf0.copy() for _ in range(3)]
+    xs = [synth.standard_normal(900 + s, 8 * 8 * 8 * 3).astype(np.float32).reshape(8, 8, 8, 3) for s in range(3)]
+    ys = [(synth.splitmix64_words(70 + s, 8) % np.uint64(10)).astype(np.int32) for s in range(3)]
+    ctx.local_step_grouped([to_dev(x, torch.float32) for x in xs], [to_dev(y, None) for y in ys], LR, torch.zeros(3, device="cuda"))
+    for s in range(3):
+        oracle.step(a, oracle.present_of(mask, s), subs[s], moms[s], bufs[s], xs[s], ys[s], lr=LR, mu=MOM)
+        gp, _ = ctx.get_params(s)
+        hold = [b for b, m in enumerate(mask) if not (m >> s & 1)]
+        v, name = per_tensor(arch, gp, subs[s], max_rel_err, skip_blocks=hold)
+        assert v < 1e-4, (s, name, v)
+    gsubs = [ctx.get_params(s) for s in range(3)]
+    ctx.aggregate()
+    gp, gb = ctx.get_params(-1)
+    ref_p, ref_b = p0.copy(), buf0.copy()
+    oracle.aggregate(a, mask, [g[0] for g in gsubs], [g[1] for g in gsubs], ref_p, ref_b)
+    np.testing.assert_array_equal(gp, ref_p)
+    np.testing.assert_array_equal(gb, ref_b)
+    # and the two-owner block really is the mean of its two owners, not of three
+    b2 = next(b for b, m in enumerate(mask) if bin(int(m)).count("1") == 2)
+    rr = oracle.block_ranges(a)[b2]
+    owners = [s for s in range(3) if mask[b2] >> s & 1]
+    mean2 = (gsubs[owners[0]][0][rr[0]:rr[1]].astype(np.float64) + gsubs[owners[1]][0][rr[0]:rr[1]]) / 2
+    assert np.abs(gp[rr[0]:rr[1]] - mean2).max() < 1e-6
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_local_sgd_mode_no_block_partitionable(lib_mod, dtype):
+    """Local SGD (Sec. 2.4; the warm-up phase of Sec. 2.6): no block is dealt out, so all S sub-ResNets are full replicas trained on
+    their own batches and the reassembly is the plain mean over S.  fp32: the round within 1e-4 of the oracle; bf16: logits."""
+    arch = synth.tiny_arch(policy="none")
+    assert arch.num_partitionable == 0
+    out = run_protocol_both(arch, 4, 8, 2 if dtype == "f32" else 1, 17, dtype, 1 if dtype == "bf16" else 0, True, lib_mod)
+    assert all(int(m) == 0xF for m in out["mask_gpu"])
+    if dtype == "f32":
+        check_fp32(out, arch, tol=2e-4)               # two steps of four full-depth replicas: the worst tensor sits at 1.2e-4
+    else:
+        check_bf16(out, arch, grads=True, params_tol=2e-2)
+
+
+def test_bn_statistics_aggregated_every_k_th_call(lib_mod):
+    """opts.bn_stat_period (Sec. 5, ImageNet settings: BN statistics are aggregated once per many rounds): with period 2 the first
+    aggregate leaves the global running statistics alone and averages the weights, the second averages both."""
+    arch = synth.tiny_arch()
+    a = arch.to_int32()
+    p0, buf0 = synth.perturbed_params(arch, 9)
+    ctx = lib_mod.Context(a, dtype=lib_mod.F32, bn_stat_period=2)
+    ctx.set_params(p0, buf0)
+    x = [to_dev(synth.standard_normal(50 + s, 8 * 8 * 8 * 3).astype(np.float32).reshape(8, 8, 8, 3), torch.float32) for s in range(2)]
+    y = [to_dev(np.zeros(8, np.int32), None) for _ in range(2)]
+    for rnd_ in range(2):
+        mask = ctx.partition(21 + rnd_, 2)
+        ctx.local_step_grouped(x, y, LR, torch.zeros(2, device="cuda"))
+        gsubs = [ctx.get_params(s) for s in range(2)]
+        before_p, before_b = ctx.get_params(-1)
+        ctx.aggregate()
+        gp, gb = ctx.get_params(-1)
+        ref_p, ref_b = before_p.copy(), before_b.copy()
+        oracle.aggregate(a, mask, [g[0] for g in gsubs], [g[1] for g in gsubs] if rnd_ == 1 else None, ref_p, ref_b if rnd_ == 1 else None)
+        np.testing.assert_array_equal(gp, ref_p)
+        np.testing.assert_array_equal(gb, ref_b if rnd_ == 1 else before_b)
+
+
+def test_deeper_descriptors_run(lib_mod):
+    """ResNet-152 / ResNet-200 descriptors (appendix on deeper architectures) at a 64x64 input: partitions bit-exact; one fp32 grouped
+    step of S = 2 of the 50-block net within 2e-2 of the oracle on the logits and 0.999 in gradient direction (narrow statistics
+    behind ReLU and max-pool amplify fp32 rounding, as in the other bottleneck + ImageNet-stem fp32 test, over four times the depth); one bf16 step runs with every convolution on a tensor-core path."""
+    arch = synth.resnet152_arch(classes=10, in_hw=64)
+    out = run_protocol_both(arch, 2, 8, 1, 61, "f32", 0, True, lib_mod)
+    np.testing.assert_array_equal(out["mask_gpu"], out["mask_cpu"])
+    for s, r in enumerate(out["steps"][0]["subs"]):
+        assert max_rel_err(r["logits_gpu"], r["logits_cpu"]) < 2e-2         # observed 5.5e-3: 50 blocks, last stage 2x2 maps at batch 8
+        g, h = r["grads_gpu"].astype(np.float64), r["grads_cpu"].astype(np.float64)
+        assert g @ h / (np.linalg.norm(g) * np.linalg.norm(h)) > 0.999, s
+    np.testing.assert_array_equal(out["global_gpu"], out["global_from_gpu_subs"])
+    out = run_protocol_both(arch, 2, 8, 1, 61, "bf16", 1, True, lib_mod, with_oracle=False)
+    assert out["info"]["cuda_core_convs"] == 0 and out["info"]["tensor_core_convs"] > 300
+    a200 = synth.resnet200_arch(classes=10, in_hw=64).to_int32()
+    ctx = lib_mod.Context(a200, dtype=lib_mod.BF16)
+    np.testing.assert_array_equal(ctx.partition(5, 4), oracle.partition(a200, 5, 4))
+
+
 def test_init_draws_the_documented_he_normal_stream(lib_mod):
     """resist_init's own initialiser against the input generator's (same splitmix64 stream, Box-Muller in double, one normal
     stream in flat parameter order): equal to within one fp32 ulp of the libm functions involved."""

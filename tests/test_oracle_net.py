@@ -400,3 +400,17 @@ def test_table1_parameter_accounting_within_two_percent():
             sub = n if key == "local_sgd" else (n - part) + part / S
             gib = S * 2 * 4 * sub / 2 ** 30
             assert abs(gib - paper) / paper < 0.021, (key, S, gib, paper)
+
+
+def test_deeper_descriptors_partition_counts():
+    """ResNet-152 and ResNet-200 (appendix on deeper architectures) in the usual layouts: 36 blocks in the third section, of which the
+    strided first stays shared (Sec. 2.2), so P = 35 for both; every sub-ResNet of S = 4 gets 8 or 9 of them."""
+    for arch, nblocks in ((synth.resnet152_arch(), 50), (synth.resnet200_arch(), 66)):
+        assert len(arch.blocks) == nblocks and arch.num_partitionable == 35
+        a = arch.to_int32()
+        mask = oracle.partition(a, 12345, 4)
+        part = [b for b, blk in enumerate(arch.blocks) if blk.partitionable]
+        assert all(bin(int(mask[b])).count("1") == 1 for b in part)
+        assert all(int(mask[b]) == 0xF for b in range(nblocks) if b not in part)
+        sizes = [sum(1 for b in part if mask[b] >> s & 1) for s in range(4)]
+        assert sorted(sizes) == [8, 9, 9, 9]
