@@ -47,6 +47,9 @@ WORKLOADS = {
                      "50 local steps per round", 16),
     "imagenet": (4, "configs[3]: ImageNet-shaped ResNet-101, 224x224x3, 1000 classes, S=4 sub-ResNets, batch 64 per sub-ResNet, "
                     "bf16 + fp32 master, 20 local steps per round", 3),
+    # the paper's local-SGD baseline (Sec. 2.4) on the same kernels: no block is dealt out, every sub-ResNet is the full network
+    "wide_localsgd": (3, "configs[2]'s network trained by local SGD (Sec. 2.4): no block dealt out, S=8 full replicas, batch 128 each, "
+                         "bf16 + fp32 master, 50 local steps per round", 4),
 }
 # mean DRAM bytes per launch of a kernel family (ncu, profiles/): workload -> family -> bytes; filled in from the committed captures
 NCU_DRAM_BYTES_PER_LAUNCH = {}
@@ -126,6 +129,18 @@ def make_batches(cfg, n):
     return xs, ys
 
 
+def workload_config(args):
+    cfg = synth.config(WORKLOADS[args.workload][0])
+    if args.workload == "wide_localsgd":
+        cfg.arch = synth.wide_cifar_arch(policy="none")
+    # a smaller case of the same kernels for profiler captures (a few GB on the device): fewer sub-ResNets, smaller batch
+    if args.subnets:
+        cfg.S = args.subnets
+    if args.batch:
+        cfg.batch = args.batch
+    return cfg
+
+
 def bound_of(name: str, v: dict, peaks: dict) -> dict:
     """Roofline of one profile entry: entries named '<family>@tensor' hold the launches whose arithmetic intensity is above the
     ridge (held against the sustained bf16 peak, the kernels being timed inside a long step), the others against HBM bandwidth."""
@@ -149,7 +164,7 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
     torch.cuda.set_device(local)
     dev = torch.device(f"cuda:{local}")
-    cfg = synth.config(WORKLOADS[args.workload][0])
+    cfg = workload_config(args)
     S, B, K, W = cfg.S, cfg.batch, args.steps, args.warmup
     LOCAL_STEPS = cfg.local_steps
     POOL = WORKLOADS[args.workload][2]
@@ -219,7 +234,7 @@ def run_ours(args):
             one_step(e2e)
         blocks, launches, bounds = [], [], []
         total = 0.0
-        while len(blocks) < 3 or (total < 1500.0 and len(blocks) < 200):
+        while len(blocks) < (1 if args.profile_case else 3) or (not args.profile_case and total < 1500.0 and len(blocks) < 200):
             state.update(launches=0, boundaries=0)
             barrier()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -238,6 +253,9 @@ def run_ours(args):
     blocks, launches, bounds = timed(False)
     clocks = sampler.stop()
     info = ctx.step_info()
+    if args.profile_case:                  # profiler capture: the resident pass alone, then a few profiled steps
+        print(json.dumps({"profile_case": True, "workload": args.workload, "S": S, "batch_per_subnet": B, "ms_per_step": float(np.median(blocks)) / K}))
+        return
     blocks_e2e, _, _ = timed(True)
     assert bool(torch.isfinite(h_loss).all()), "the end-to-end pass produced a non-finite loss"
     ms = float(np.median(blocks))
@@ -379,7 +397,7 @@ def run_reference(args):
     if rank != 0:
         return
     import oracle
-    cfg = synth.config(WORKLOADS[args.workload][0])
+    cfg = workload_config(args)
     a = cfg.arch.to_int32()
     mask = oracle.partition(a, cfg.round_seed(0), cfg.S)
     p0, _ = synth.init_params(cfg.arch, cfg.init_seed)
@@ -473,19 +491,42 @@ def run_reassembly(args):
     print(json.dumps(out))
 
 
+def run_micro(args):
+    """tcgen05.mma rate on this device by MMA width, operand layout, number of issuing threads (see resist_micro_mma_rate)."""
+    import torch
+    import paper_2107_00961_b200 as lib
+    torch.cuda.set_device(0)
+    mhz = 1965.0
+    rows = []
+    names = {0: "K-major no swizzle", 1: "K-major 128B swizzle", 2: "K-major 128B swizzle, one 32-byte step", 3: "MN-major 128B swizzle"}
+    for layout in (0, 1, 2, 3):
+        for n in (16, 64, 128, 256):
+            for issuers, alt in ((1, 0), (1, 1), (2, 0), (2, 1)):
+                lib.micro_mma_rate(n, layout, 512, issuers, alt)
+                c = min(lib.micro_mma_rate(n, layout, 4096, issuers, alt) for _ in range(3))
+                rows.append({"layout": names[layout], "n": n, "issuers": issuers, "alternate_accumulators": alt, "cycles_per_mma": c,
+                             "ideal_cycles": n / 2.0, "TFLOPs_per_gpu_at_max_clock": 2.0 * 128 * n * 16 / c * mhz * 1e6 * 148 / 1e12})
+    print(json.dumps({"metric": "tcgen05.mma cycles per 128 x n x 16 MMA", "rows": rows}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="wide", choices=["wide", "resnet110", "imagenet", "reassembly"],
-                    help="wide (default): the headline line; resnet110, imagenet: the other training configurations; "
-                         "reassembly: the synchronisation kernels alone")
+    ap.add_argument("--workload", default="wide", choices=["wide", "resnet110", "imagenet", "wide_localsgd", "reassembly", "micro"],
+                    help="wide (default): the headline line; resnet110, imagenet: the other training configurations; wide_localsgd: the "
+                         "local-SGD baseline on the wide network; reassembly: the synchronisation kernels alone")
     ap.add_argument("--skip-cpu-baseline", action="store_true", help="leave the oracle's timing out of the line (quick kernel work)")
+    ap.add_argument("--subnets", type=int, default=0, help="override S (smaller case of the same kernels for profiler captures)")
+    ap.add_argument("--batch", type=int, default=0, help="override the batch per sub-ResNet (likewise)")
+    ap.add_argument("--profile-case", action="store_true", help="run W warm-up steps and one block of K steps only, print a short line (for ncu)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
-    if args.workload == "reassembly":
+    if args.workload == "micro":
+        run_micro(args)
+    elif args.workload == "reassembly":
         run_reassembly(args)
     elif args.impl == "reference":
         run_reference(args)

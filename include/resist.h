@@ -247,6 +247,14 @@ void resist_splitmix64(uint64_t seed, int64_t n, uint64_t* out);
 
 const char* resist_last_error(resist_ctx* ctx);   /* ctx may be NULL: the last init failure */
 
+/* Micro-benchmark behind the tile shapes of the tensor-core kernels (the paper has no counterpart: a property of the device): every
+ * SM issues `reps` tcgen05 MMAs of shape 128 x n x 16 (bf16 -> fp32) back to back and waits for them; *cycles_per_mma (host)
+ * receives SM clocks per MMA, first issue to completion.  layout: 0 K-major operands without swizzle, 1 K-major with the 128-byte
+ * swizzle (the four 32-byte steps of a row in turn), 2 the same reading one step only, 3 MN-major with the 128-byte swizzle.
+ * issuers: 1 or 2 issuing threads; alternate: 1 = consecutive MMAs accumulate into two different accumulators.  Operand values are
+ * whatever the shared memory holds.  Synchronises the device. */
+int resist_micro_mma_rate(int32_t n, int32_t layout, int32_t reps, int32_t issuers, int32_t alternate, double* cycles_per_mma);
+
 /* Test hook: stores `code` in the device status word that a kernel's bounded wait writes when it gives up, so that the next
  * call that synchronises (resist_aggregate, a parity tap, a layer-level call) returns RESIST_ETIMEOUT and clears the word.
  * No kernel has to time out for the reporting path to be tested. */

@@ -86,6 +86,7 @@ def lib():
         L.resist_get_logits.argtypes = [P, I, P]
         L.resist_get_shadow.argtypes = [P, I, P]
         L.resist_debug_set_wait_status.argtypes = [I]
+        L.resist_micro_mma_rate.argtypes = [I, I, I, I, I, C.POINTER(C.c_double)]
         L.resist_get_step_info.argtypes = [P, C.POINTER(_StepInfo)]
         L.resist_splitmix64.argtypes = [U64, C.c_int64, P]
         L.resist_splitmix64.restype = None
@@ -106,7 +107,7 @@ def lib():
 
 EXPORTS = ["resist_init", "resist_destroy", "resist_partition", "resist_local_step", "resist_local_step_grouped",
            "resist_aggregate", "resist_eval", "resist_param_count", "resist_get_params", "resist_set_params",
-           "resist_get_grads", "resist_get_logits", "resist_get_shadow", "resist_debug_set_wait_status", "resist_get_step_info", "resist_splitmix64", "resist_last_error",
+           "resist_get_grads", "resist_get_logits", "resist_get_shadow", "resist_debug_set_wait_status", "resist_micro_mma_rate", "resist_get_step_info", "resist_splitmix64", "resist_last_error",
            "resist_set_profiling", "resist_get_profile", "resist_conv2d", "resist_conv2d_bn_relu", "resist_bn_relu_forward", "resist_bn_relu_backward", "resist_layer_last_error",
            "resist_bn_relu_forward_noalloc", "resist_noalloc_last_error"]
 
@@ -150,6 +151,15 @@ def resist_conv2d(mode: int, act: torch.Tensor, wgt: torch.Tensor, geom, add: Op
                                      add.data_ptr() if add is not None else None, out.data_ptr(), N, H, W, Cc, K, ksz,
                                      stride, scale, C.addressof(used), _stream_handle(stream)))
     return out, int(used.value)
+
+
+def micro_mma_rate(n: int, layout: int, reps: int = 4096, issuers: int = 1, alternate: int = 0) -> float:
+    """SM clocks per tcgen05 MMA of shape 128 x n x 16 (see resist.h)."""
+    out = C.c_double(0.0)
+    rc = lib().resist_micro_mma_rate(n, layout, reps, issuers, alternate, C.byref(out))
+    if rc:
+        raise ResistError(rc, "resist_micro_mma_rate failed")
+    return float(out.value)
 
 
 def resist_conv2d_bn_relu(mode: int, act: torch.Tensor, wgt: torch.Tensor, geom, gamma, beta, stat=None, x=None, add=None, bn_add=None,
