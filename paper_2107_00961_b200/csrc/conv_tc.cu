@@ -14,11 +14,16 @@
 // and the tensor core reads it back by absolute address, so a descriptor may start at any 128-byte row).  Activations are K-major operands; weights are K-major in forward
 // ([out channel][64 in channels]) and MN-major in dgrad ([64 reduction channels][64 out columns] blocks).
 //
-// Kernel structure (192 threads, one CTA per SM, persistent over the tiles of all problems of the launch):
-// warp 0 = TMA producer (a ring of activation windows and a ring of weight tiles, one weight tile per (slab, tap)),
-// warp 1 = TMEM owner + MMA issuer (two accumulators: the epilogue of tile i overlaps the MMAs of tile i+1),
-// warps 2..5 = epilogue (TMEM -> registers -> scale, residual add, bf16 -> global).  Every wait is bounded: on expiry
-// the kernel records the place in the status word, drains its copies, frees its TMEM and returns.
+// Kernel structure of forward / dgrad (352 threads, one CTA per SM, persistent over the work of all problems of the launch).  A
+// unit of work is a PAIR of neighbouring 128-position tiles times one column tile of up to 256 output channels:
+// warp 0 = TMA producer (a ring of activation windows, two per step, and a ring of weight tiles, one per (slab, tap), shared by
+// the two tiles of the pair); warps 1 and 2 = MMA issuers, one per tile of the pair, each with its own accumulator in TMEM
+// (a single thread issues a tcgen05.mma only every ~150 cycles, see micro.cu, so one issuer cannot keep the tensor core busy);
+// warps 3..10 = two epilogue groups of four warps, one per tile of the pair (TMEM -> registers -> scale, residual add, bf16 ->
+// 16 KB staging slabs of 64 columns -> TMA store or row copy-out, with per-tile column sums for the BN that follows).
+// The weight-gradient kernel (192 threads) has one producer warp, one issuer warp and four epilogue warps.
+// Every wait is bounded: on expiry the kernel records the place in the status word, drains its copies and MMAs, frees its
+// TMEM and returns.
 #include <cuda.h>
 #include <cstdio>
 #include <cstring>
@@ -110,11 +115,11 @@ __device__ __forceinline__ void sts128(uint32_t a, uint4 v) { asm volatile("st.s
 __device__ __forceinline__ uint32_t lds32(uint32_t a) { uint32_t v; asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(a)); return v; }
 
 constexpr int TC_THREADS = 192;              // wgrad kernel: producer warp, MMA warp, four epilogue warps
-constexpr int TC_CONV_THREADS = 320;         // forward / dgrad kernel: producer warp, MMA warp, two groups of four epilogue warps
+constexpr int TC_MAX_ISSUERS = 2;            // forward / dgrad kernel: MMA-issuing warps, one per tile of a pair
+constexpr int TC_CONV_THREADS = 32 * (1 + TC_MAX_ISSUERS + 8);   // forward / dgrad kernel: producer warp, MMA warps, two groups of four epilogue warps
 constexpr int TC_MAX_STAGES = 12;
 constexpr int TILE_M = 128;
 constexpr int SLAB_BYTES = TILE_M * 128;      // 128 rows x 64 channels of bf16
-constexpr size_t TC_RESIDENT_BUDGET = 96 * 1024;   // weights of one column tile that may stay in shared memory
 
 struct TapRef { int wtap; int shift; };       // weight tap index (r*ksz + s); row shift of the operand inside the window
 // One forward / dgrad problem.  The tensor maps come first so that each is 64-byte aligned.
@@ -132,7 +137,7 @@ struct TcHot {                // everything the kernel's loops read: each role k
     int* status;
     int a_flat;               // 1: a window is one box of 128 pixels of the (channel, pixel) map
     int dense;                // 1: position index == output pixel index
-    int add_mode;             // 0 none; 1 fetched by TMA into the staging tile (dense); 2 global loads at the output pixel; 3 global loads from a compact tensor that applies at even (y, x) only
+    int add_mode;             // 0 none; 2 residual read at the output pixel; 3 residual read from a compact tensor that applies at even (y, x) only
     int ngroups; int gbeg[5]; int gxs[4], gys[4];
     int wtap[9], shift[9];    // per tap: weight tap index (r*ksz + s); row shift of the operand inside the window
     int es, pad;
@@ -152,13 +157,13 @@ struct alignas(64) TcProb {
     CUtensorMap map_a;        // activations (forward: a; dgrad: dy): (channel, pixel) or (channel, x, y, image), possibly element-strided
     CUtensorMap map_b;        // weights [K][taps][C] viewed as (C, tap, K)
     CUtensorMap map_out;      // dense problems: the output as (channel, pixel), box 64 x 128
-    CUtensorMap map_add;      // dense problems with a residual: the residual likewise
     TcHot h;
 };
 static_assert(sizeof(TcHot) % 4 == 0, "copied word by word");
 
-struct TcLaunch { int nprob, na, nb, a_stage, b_stage, tmem_cols, acc_stride, n_stg, stg_bytes, b_res, b_region, groups, pg, prefetch; };   // b_res: the weights of a (problem, column tile) stay in shared memory; b_region: bytes of the weight ring or of the resident weights;
-// groups: epilogue groups (they take alternate tiles); pg: staging tiles per group (n_stg = groups * pg); prefetch: some problem's residual is fetched by TMA
+struct TcLaunch { int nprob, na, nb, a_stage, b_stage, tmem_cols, acc_stride, nbuf, groups, pg; };
+// nbuf: accumulators per tile of a pair (2: the next pair's MMAs run under this pair's epilogues); groups: epilogue groups (two: one
+// per tile of a pair; one: it takes both tiles in turn); pg: 16 KB staging buffers (one 64-column slab each) per group
 constexpr int TC_MAX_PROBS = 128;             // descriptors per launch (sub-ResNets x output phases)
 
 __device__ __forceinline__ void copy_hot(TcHot* dst, const TcHot* src, int tid, int nthreads) {
@@ -169,31 +174,35 @@ __device__ __forceinline__ void copy_hot(TcHot* dst, const TcHot* src, int tid, 
 __global__ void __launch_bounds__(TC_CONV_THREADS, 1) conv_tc_kernel(const TcProb* __restrict__ probs, const TcLaunch L) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    __shared__ __align__(8) uint64_t bars[4 * TC_MAX_STAGES + 14];
+    __shared__ __align__(8) uint64_t bars[4 * TC_MAX_STAGES + 10];
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
     __shared__ int pix_s2[2][TILE_M];
     __shared__ float stat_s2[2][4][2][256];
-    __shared__ int tile_end_s[TC_MAX_PROBS];                      // running sum of the problems' tile counts
-    __shared__ TcHot hot_s[4];                                    // the current problem of the producer, the MMA issuer, the two epilogue groups
+    __shared__ int unit_end_s[TC_MAX_PROBS];                      // running sum of the problems' unit counts (a unit: two row tiles x one column tile)
+    __shared__ int tilesm_s[TC_MAX_PROBS], tilesn_s[TC_MAX_PROBS];
+    __shared__ TcHot hot_s[3 + TC_MAX_ISSUERS];                   // the current problem of the producer, the two epilogue groups, the MMA issuers
     const uint32_t a_full = smem_u32(&bars[0]), a_empty = smem_u32(&bars[TC_MAX_STAGES]);
     const uint32_t b_full = smem_u32(&bars[2 * TC_MAX_STAGES]), b_empty = smem_u32(&bars[3 * TC_MAX_STAGES]);
-    const uint32_t acc_full = smem_u32(&bars[4 * TC_MAX_STAGES]), acc_empty = smem_u32(&bars[4 * TC_MAX_STAGES + 2]);
-    const uint32_t add_full = smem_u32(&bars[4 * TC_MAX_STAGES + 4]), stg_free = smem_u32(&bars[4 * TC_MAX_STAGES + 8]);
-    const uint32_t bres_full = smem_u32(&bars[4 * TC_MAX_STAGES + 12]), bres_empty = smem_u32(&bars[4 * TC_MAX_STAGES + 13]);
-    const uint32_t a_ring = smem_u32(smem), b_ring = a_ring + (uint32_t)(L.na * L.a_stage), stg_base = b_ring + (uint32_t)L.b_region;
+    const uint32_t acc_full = smem_u32(&bars[4 * TC_MAX_STAGES]), acc_empty = smem_u32(&bars[4 * TC_MAX_STAGES + 4]);
+    const uint32_t drain = smem_u32(&bars[4 * TC_MAX_STAGES + 8]);
+    const uint32_t a_ring = smem_u32(smem), b_ring = a_ring + (uint32_t)(L.na * L.a_stage), stg_base = b_ring + (uint32_t)(L.nb * L.b_stage);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < TC_MAX_STAGES; ++s) {
-            mbar_init(a_full + 8 * s, 1); mbar_init(a_empty + 8 * s, 1); mbar_init(b_full + 8 * s, 1); mbar_init(b_empty + 8 * s, 1);
+            mbar_init(a_full + 8 * s, 1); mbar_init(a_empty + 8 * s, 1); mbar_init(b_full + 8 * s, 1);
+            mbar_init(b_empty + 8 * s, TC_MAX_ISSUERS);          // a weight tile serves both tiles of a pair: both issuers release it
         }
-        for (int s = 0; s < 2; ++s) { mbar_init(acc_full + 8 * s, 1); mbar_init(acc_empty + 8 * s, 4); }
-        for (int s = 0; s < 4; ++s) { mbar_init(add_full + 8 * s, 1); mbar_init(stg_free + 8 * s, 1); }
-        mbar_init(bres_full, 1); mbar_init(bres_empty, 1);
+        for (int s = 0; s < 4; ++s) { mbar_init(acc_full + 8 * s, 1); mbar_init(acc_empty + 8 * s, 4); }
+        for (int s = 0; s < TC_MAX_ISSUERS; ++s) mbar_init(drain + 8 * s, 1);
         abort_s = 0;
         int run = 0;
-        for (int i = 0; i < L.nprob; ++i) { run += probs[i].h.tiles_m * probs[i].h.tiles_n; tile_end_s[i] = run; }
+        for (int i = 0; i < L.nprob; ++i) {
+            const TcHot* hp = &probs[i].h;
+            run += ((hp->tiles_m + 1) >> 1) * hp->tiles_n; unit_end_s[i] = run;
+            tilesm_s[i] = hp->tiles_m; tilesn_s[i] = hp->tiles_n;
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -204,61 +213,38 @@ __global__ void __launch_bounds__(TC_CONV_THREADS, 1) conv_tc_kernel(const TcPro
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = tmem_base_s;
-    // The tiles of all problems, column tile innermost, are dealt round-robin: the CTAs that run side by side work on neighbouring
-    // tiles, share activation windows and weight tiles in L2 and read HBM as one moving front.  (Contiguous runs per CTA, with the
-    // column tile outermost, were measured too: no faster, and slower for the layers whose weights stream.)
-    const int t_begin = (int)blockIdx.x, t_stop = tile_end_s[L.nprob - 1], t_step = (int)gridDim.x;
+    // A unit of work is a pair of neighbouring row tiles (2 x 128 positions) times one column tile: the two tiles share every weight
+    // tile, which is fetched once, and each has its own MMA-issuing warp and accumulator.  (One thread issues a tcgen05.mma only every
+    // ~150 cycles whatever its N (measured), more than the tensor core needs for it: two issuers keep it busy, and each tile's sum
+    // is still formed by one thread in a fixed order.)  The units of all problems, column tile innermost, are dealt round-robin: the
+    // CTAs that run side by side work on neighbouring tiles, share windows and weight tiles in L2 and read HBM as one moving front.
+    // (Contiguous runs per CTA, with the column tile outermost, were measured too: no faster, and slower where the weights stream.)
+    const int u_begin = (int)blockIdx.x, u_stop = unit_end_s[L.nprob - 1], u_step = (int)gridDim.x;
 
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer
         if (lane == 0) {
-            uint32_t a_cnt = 0, b_cnt = 0, seq = 0, add_use[4] = {0u, 0u, 0u, 0u}; bool ok = true;
+            uint32_t a_cnt = 0, b_cnt = 0; bool ok = true;
             int cur = -1; TcHot& h = hot_s[0];
             int sa = 0, sb_ = 0; uint32_t pha = 0, phb = 0;       // ring positions and phases
-            int cur_unit = -1; uint32_t unit_cnt = 0;
-            for (int t = t_begin; t < t_stop && ok; t += t_step, ++seq) {
-                int pi = 0; while (t >= tile_end_s[pi]) ++pi;
+            for (int u = u_begin; u < u_stop && ok; u += u_step) {
+                int pi = 0; while (u >= unit_end_s[pi]) ++pi;
                 if (pi != cur) { copy_hot(&h, &probs[pi].h, 0, 1); cur = pi; }
                 const TcProb* pp = probs + pi;
-                const int loc = t - (pi ? tile_end_s[pi - 1] : 0);
+                const int loc = u - (pi ? unit_end_s[pi - 1] : 0);
                 const int n_tile = h.n_tile, slabs = h.slabs, ngroups = h.ngroups, a_flat = h.a_flat, nbox = h.nbox,
                           a_box_bytes = h.a_box_bytes, R = h.R, Hp = h.Hp, pad = h.pad, es = h.es, b_bytes = h.b_bytes, mn = h.b_mn_major;
-                const int tiles_n = h.tiles_n, tn = loc % tiles_n, tm = loc / tiles_n;
-                if (L.b_res && (pi << 8 | tn) != cur_unit) {
-                    // new (problem, column tile): all its weight tiles go to the resident region, once the MMAs of the last one have read theirs
-                    if (!mbar_wait(bres_empty, (unit_cnt & 1u) ^ 1u, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(h.status, 8); ok = false; break; }
-                    const int ntaps = h.gbeg[ngroups];
-                    mbar_expect_tx(bres_full, (uint32_t)(slabs * ntaps * b_bytes));
-                    for (int sl = 0; sl < slabs; ++sl)
-                        for (int tap = 0; tap < ntaps; ++tap) {
-                            const uint32_t dst = b_ring + (uint32_t)((sl * ntaps + tap) * ((b_bytes + 1023) & ~1023));
-                            const int wtap = h.wtap[tap];
-                            if (!mn) tma_load_3d(dst, &pp->map_b, bres_full, sl * 64, wtap, tn * n_tile);
-                            else for (int j = 0; j * 64 < n_tile; ++j)
-                                tma_load_3d(dst + (uint32_t)(j * 8192), &pp->map_b, bres_full, tn * n_tile + j * 64, wtap, sl * 64);
-                        }
-                    ++unit_cnt; cur_unit = pi << 8 | tn;
-                }
-                if (h.add_mode == 1) {
-                    // the residual tile goes straight into the staging tile the epilogue will finish in place
-                    const uint32_t grp = L.groups == 2 ? (seq & 1u) : 0u, kk = L.groups == 2 ? (seq >> 1) : seq;
-                    const uint32_t sb = grp * (uint32_t)L.pg + kk % (uint32_t)L.pg, uses = kk / (uint32_t)L.pg;
-                    if (!mbar_wait(stg_free + 8 * sb, (uses & 1u) ^ 1u, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(h.status, 7); ok = false; break; }
-                    mbar_expect_tx(add_full + 8 * sb, (uint32_t)(h.out_slabs * SLAB_BYTES));
-                    for (int j = 0; j < h.out_slabs; ++j)
-                        tma_load_2d(stg_base + sb * (uint32_t)L.stg_bytes + (uint32_t)(j * SLAB_BYTES), &pp->map_add, add_full + 8 * sb, tn * n_tile + j * 64, tm * TILE_M);
-                    ++add_use[sb];
-                }
-                const int bx0 = a_flat ? 0 : floor_div(tm * TILE_M - h.hb, h.box_pos);
+                const int tiles_n = h.tiles_n, tn = loc % tiles_n, tm0 = 2 * (loc / tiles_n), nt = tm0 + 1 < h.tiles_m ? 2 : 1;
                 for (int sl = 0; sl < slabs && ok; ++sl) {
                     for (int g = 0; g < ngroups && ok; ++g) {
-                        {
+                        for (int j = 0; j < nt; ++j) {
                             if (!mbar_wait(a_empty + 8 * sa, pha ^ 1u, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(h.status, 1); ok = false; break; }
+                            const int tm = tm0 + j;
                             const uint32_t dst = a_ring + (uint32_t)(sa * L.a_stage);
                             mbar_expect_tx(a_full + 8 * sa, (uint32_t)(nbox * a_box_bytes));
                             if (a_flat) tma_load_2d(dst, &pp->map_a, a_full + 8 * sa, sl * 64, tm * TILE_M);
                             else {
-                                const int gx = h.gxs[g], gy = h.gys[g];
+                                const int gx = h.gxs[g], gy = h.gys[g], bx0 = floor_div(tm * TILE_M - h.hb, h.box_pos);
                                 for (int i = 0; i < nbox; ++i) {
                                     const int trow = (bx0 + i) * R, img = floor_div(trow, Hp), yy0 = trow - img * Hp;
                                     tma_load_4d(dst + (uint32_t)(i * a_box_bytes), &pp->map_a, a_full + 8 * sa, sl * 64, gx, (yy0 - pad) * es + gy, img);
@@ -266,15 +252,16 @@ __global__ void __launch_bounds__(TC_CONV_THREADS, 1) conv_tc_kernel(const TcPro
                             }
                             ++a_cnt; if (++sa == L.na) { sa = 0; pha ^= 1u; }
                         }
-                        const int t_end = L.b_res ? 0 : h.gbeg[g + 1];
+                        if (!ok) break;
+                        const int t_end = h.gbeg[g + 1];
                         for (int tap = h.gbeg[g]; tap < t_end; ++tap) {
                             if (!mbar_wait(b_empty + 8 * sb_, phb ^ 1u, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(h.status, 2); ok = false; break; }
                             const uint32_t dst = b_ring + (uint32_t)(sb_ * L.b_stage);
                             const int wtap = h.wtap[tap];
                             mbar_expect_tx(b_full + 8 * sb_, (uint32_t)b_bytes);
                             if (!mn) tma_load_3d(dst, &pp->map_b, b_full + 8 * sb_, sl * 64, wtap, tn * n_tile);
-                            else for (int j = 0; j * 64 < n_tile; ++j)
-                                tma_load_3d(dst + (uint32_t)(j * 8192), &pp->map_b, b_full + 8 * sb_, tn * n_tile + j * 64, wtap, sl * 64);
+                            else for (int c = 0; c * 64 < n_tile; ++c)
+                                tma_load_3d(dst + (uint32_t)(c * 8192), &pp->map_b, b_full + 8 * sb_, tn * n_tile + c * 64, wtap, sl * 64);
                             ++b_cnt; if (++sb_ == L.nb) { sb_ = 0; phb ^= 1u; }
                         }
                     }
@@ -286,36 +273,34 @@ __global__ void __launch_bounds__(TC_CONV_THREADS, 1) conv_tc_kernel(const TcPro
                     for (int i = 0; i < 4096 && !mbar_try(a_full + 8 * (c % L.na), (c / L.na) & 1u); ++i) __nanosleep(64);
                 for (uint32_t c = b_cnt > (uint32_t)L.nb ? b_cnt - L.nb : 0; c < b_cnt; ++c)
                     for (int i = 0; i < 4096 && !mbar_try(b_full + 8 * (c % L.nb), (c / L.nb) & 1u); ++i) __nanosleep(64);
-                for (uint32_t sb = 0; sb < 4; ++sb)
-                    if (add_use[sb]) for (int i = 0; i < 4096 && !mbar_try(add_full + 8 * sb, (add_use[sb] - 1u) & 1u); ++i) __nanosleep(64);
             }
         }
-    } else if (warp == 1) {
-        // ---------------------------------------------------------------- MMA issuer
+    } else if (warp <= TC_MAX_ISSUERS) {
+        // ---------------------------------------------------------------- MMA issuers: warp 1 + j runs the reduction of tile j of every
+        // pair into its own accumulator.  Windows are per tile (the pair's two windows sit in consecutive ring stages); a weight stage
+        // is read by both issuers and released by both (an issuer whose pair has no second tile only passes the weight stages on).
+        const int me = warp - 1;
         if (lane == 0) {
-            uint32_t acc_cnt = 0; bool ok = true;
-            int cur = -1; TcHot& h = hot_s[1];
-            int sa = 0, sb = 0; uint32_t pha = 0, phb = 0;
-            int cur_unit = -1; uint32_t unit_cnt = 0;
+            uint32_t a_cnt = 0, cnt = 0; bool ok = true;
+            int cur = -1; TcHot& h = hot_s[3 + me];
+            int sb = 0; uint32_t phb = 0;
             // the constant part of a 128-byte-swizzle descriptor: stride between 8-row groups 1024 bytes, version, swizzle mode
             const uint64_t desc_k = desc_sw128(0, 16, 1024), desc_mn = desc_sw128(0, 8192, 1024);
-            for (int t = t_begin; t < t_stop && ok; t += t_step, ++acc_cnt) {
-                int pi = 0; while (t >= tile_end_s[pi]) ++pi;
+            for (int u = u_begin; u < u_stop && ok; u += u_step) {
+                int pi = 0; while (u >= unit_end_s[pi]) ++pi;
                 if (pi != cur) { copy_hot(&h, &probs[pi].h, 0, 1); cur = pi; }
-                const int loc = t - (pi ? tile_end_s[pi - 1] : 0);
+                const int loc = u - (pi ? unit_end_s[pi - 1] : 0);
                 const int slabs = h.slabs, ngroups = h.ngroups, red = h.red, mn = h.b_mn_major;
-                const int tiles_n = h.tiles_n, tn = loc % tiles_n, tm = loc / tiles_n;
-                const int ntaps = h.gbeg[ngroups], b_stride = (h.b_bytes + 1023) & ~1023;
-                if (L.b_res && (pi << 8 | tn) != cur_unit) {
-                    if (!mbar_wait(bres_full, unit_cnt & 1u, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(h.status, 9); ok = false; break; }
-                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    ++unit_cnt; cur_unit = pi << 8 | tn;
-                }
+                const int tm0 = 2 * (loc / h.tiles_n), nt = tm0 + 1 < h.tiles_m ? 2 : 1, tm = tm0 + me;
+                const bool has = me < nt;
                 const int bx0 = h.a_flat ? 0 : floor_div(tm * TILE_M - h.hb, h.box_pos);
                 const int a_off = h.a_flat ? 0 : tm * TILE_M - h.hb - bx0 * h.box_pos;
-                const uint32_t buf = acc_cnt & 1u, aph = (acc_cnt >> 1) & 1u;
-                if (!mbar_wait(acc_empty + 8 * buf, aph ^ 1u, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(h.status, 3); ok = false; break; }
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t buf = (cnt % (uint32_t)L.nbuf) * 2u + (uint32_t)me, aph = (cnt / (uint32_t)L.nbuf) & 1u;
+                if (has) {
+                    ++cnt;
+                    if (!mbar_wait(acc_empty + 8 * buf, aph ^ 1u, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(h.status, 3); ok = false; break; }
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                }
                 const uint32_t d_tmem = tmem_base + buf * (uint32_t)L.acc_stride;
                 // instruction descriptor: fp32 accumulate, bf16 x bf16, A K-major, B K-major or MN-major, N, M = 128
                 const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)mn << 16) |
@@ -326,80 +311,67 @@ __global__ void __launch_bounds__(TC_CONV_THREADS, 1) conv_tc_kernel(const TcPro
                 for (int sl = 0; sl < slabs && ok; ++sl) {
                     const int ksteps = (min(64, red - sl * 64) + 15) >> 4;
                     for (int g = 0; g < ngroups && ok; ++g) {
-                        if (!mbar_wait(a_full + 8 * sa, pha, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(h.status, 4); ok = false; break; }
-                        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                        const uint32_t a_rows16 = ((a_ring + (uint32_t)(sa * L.a_stage)) >> 4) + (uint32_t)a_off * 8u;   // start address in 16-byte units
+                        const uint32_t ai = a_cnt + (uint32_t)me; a_cnt += (uint32_t)nt;
+                        const uint32_t sa = ai % (uint32_t)L.na, pha = (ai / (uint32_t)L.na) & 1u;
+                        if (has) {
+                            if (!mbar_wait(a_full + 8 * sa, pha, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(h.status, 4); ok = false; break; }
+                            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                        }
+                        const uint32_t a_rows16 = ((a_ring + sa * (uint32_t)L.a_stage) >> 4) + (uint32_t)a_off * 8u;   // start address in 16-byte units
                         const int t_end = h.gbeg[g + 1];
                         for (int tap = h.gbeg[g]; tap < t_end; ++tap) {
-                            const uint32_t a16 = a_rows16 + (uint32_t)h.shift[tap] * 8u;
-                            uint32_t b16;
-                            if (L.b_res) b16 = (b_ring + (uint32_t)((sl * ntaps + tap) * b_stride)) >> 4;
-                            else {
-                                if (!mbar_wait(b_full + 8 * sb, phb, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(h.status, 5); ok = false; break; }
+                            if (!mbar_wait(b_full + 8 * sb, phb, &abort_s)) { atomicExch(&abort_s, 1); atomicExch(h.status, 5); ok = false; break; }
+                            if (has) {
                                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                                b16 = (b_ring + (uint32_t)(sb * L.b_stage)) >> 4;
-                            }
-                            for (int k16 = 0; k16 < ksteps; ++k16) {
-                                umma_bf16(d_tmem, desc_k | (uint64_t)((a16 + 2u * (uint32_t)k16) & 0x3FFFu), b_const | (uint64_t)((b16 + b_step * (uint32_t)k16) & 0x3FFFu), idesc, acc);
-                                acc = 1;
-                            }
-                            if (!L.b_res) {
-                                umma_commit(b_empty + 8 * sb);   // weight tile reusable once these MMAs have read it
-                                if (++sb == L.nb) { sb = 0; phb ^= 1u; }
-                            }
+                                const uint32_t a16 = a_rows16 + (uint32_t)h.shift[tap] * 8u;
+                                const uint32_t b16 = (b_ring + (uint32_t)(sb * L.b_stage)) >> 4;
+                                for (int k16 = 0; k16 < ksteps; ++k16) {
+                                    umma_bf16(d_tmem, desc_k | (uint64_t)((a16 + 2u * (uint32_t)k16) & 0x3FFFu), b_const | (uint64_t)((b16 + b_step * (uint32_t)k16) & 0x3FFFu), idesc, acc);
+                                    acc = 1;
+                                }
+                                umma_commit(b_empty + 8 * sb);   // this issuer's share of the release: once its MMAs have read the weight tile
+                            } else mbar_arrive(b_empty + 8 * sb);
+                            if (++sb == L.nb) { sb = 0; phb ^= 1u; }
                         }
-                        umma_commit(a_empty + 8 * sa);
-                        if (++sa == L.na) { sa = 0; pha ^= 1u; }
+                        if (has && ok) umma_commit(a_empty + 8 * sa);
                     }
                 }
-                if (ok) umma_commit(acc_full + 8 * buf);         // accumulator complete
-                if (ok && L.b_res) {
-                    // last tile of this (problem, column tile) for this CTA: the resident weights may be replaced once these MMAs are done
-                    bool last = t + t_step >= t_stop;
-                    if (!last) { const int t2 = t + t_step; int pn = pi; while (t2 >= tile_end_s[pn]) ++pn; const int l2 = t2 - (pn ? tile_end_s[pn - 1] : 0);
-                        last = pn != pi || l2 % tiles_n != tn; }
-                    if (last) umma_commit(bres_empty);
-                }
+                if (has && ok) umma_commit(acc_full + 8 * buf);  // accumulator complete
+            }
+            if (!ok) {
+                // gave up: the MMAs already issued must have finished before the CTA frees its tensor memory
+                umma_commit(drain + 8 * me);
+                for (int i = 0; i < 65536 && !mbar_try(drain + 8 * me, 0u); ++i) __nanosleep(64);
             }
         }
     } else {
         // ---------------------------------------------------------------- epilogue: two groups of 4 warps (one TMEM lane quadrant each);
-        // group g takes the tiles whose accumulator is buffer g, so two epilogues run side by side
-        const int grp = (warp - 2) >> 2, bid = 1 + grp;
+        // group g takes tile g of every pair, so two epilogues run side by side (a single group takes both tiles in turn)
+        const int grp = (warp - 1 - TC_MAX_ISSUERS) >> 2, bid = 1 + grp;
         const int quad = warp & 3;
         const int m = quad * 32 + lane;                          // row of the tile = TMEM lane
-        const int et = threadIdx.x - 64 - grp * 128;             // 0..127 among the group's threads
+        const int et = threadIdx.x - 32 * (1 + TC_MAX_ISSUERS) - grp * 128;   // 0..127 among the group's threads
         const bool leader = et == 0;
         int* const pix_s = pix_s2[grp];
         float (*const stat_s)[2][256] = stat_s2[grp];
-        uint32_t add_use[4] = {0u, 0u, 0u, 0u}; bool ok = true;
-        int cur = -1; const TcHot& h = hot_s[2 + grp];
-        for (int t = t_begin + grp * t_step; grp < L.groups && t < t_stop && ok; t += L.groups * t_step) {
-            const uint32_t acc_cnt = (uint32_t)((t - t_begin) / t_step), kk = acc_cnt / (uint32_t)L.groups;     // tile number of the CTA, of the group
-            int pi = 0; while (t >= tile_end_s[pi]) ++pi;
-            const TcProb* pp = probs + pi;
-            const int loc = t - (pi ? tile_end_s[pi - 1] : 0);
-            const uint32_t buf = acc_cnt & 1u, aph = (acc_cnt >> 1) & 1u;
-            const uint32_t sb = (uint32_t)(grp * L.pg) + kk % (uint32_t)L.pg;
-            const uint32_t stg = stg_base + sb * (uint32_t)L.stg_bytes;
-            if (leader) {
-                // the staging tile of this tile (and, with a prefetched residual, the next tile's, which the producer is waiting to
-                // fill) must have been read by the bulk store issued from it
-                bulk_wait_read(L.prefetch ? L.pg - 2 : L.pg - 1);
-                if (L.prefetch && kk + 1 >= (uint32_t)L.pg) mbar_arrive(stg_free + 8 * ((uint32_t)(grp * L.pg) + (kk + 1) % (uint32_t)L.pg));
-            }
-            // ... and every warp must have finished its share of the last copy-out
+        bool ok = true;
+        int cur = -1; const TcHot& h = hot_s[1 + grp];
+        uint32_t sc = 0, cnt[2] = {0u, 0u};                      // 64-column slabs this group has staged; tiles taken of each half of the pairs
+        for (int u = u_begin; grp < L.groups && u < u_stop && ok; u += u_step) {
+          int pi = 0; while (u >= unit_end_s[pi]) ++pi;
+          const TcProb* pp = probs + pi;
+          const int loc = u - (pi ? unit_end_s[pi - 1] : 0);
+          const int tn = loc % tilesn_s[pi], tm0 = 2 * (loc / tilesn_s[pi]), nt = tm0 + 1 < tilesm_s[pi] ? 2 : 1;
+          for (int hf = L.groups == 2 ? grp : 0; hf < nt && ok; hf += L.groups == 2 ? 2 : 1) {
+            const int tm = tm0 + hf;
+            const uint32_t buf = (cnt[hf] % (uint32_t)L.nbuf) * 2u + (uint32_t)hf, aph = (cnt[hf] / (uint32_t)L.nbuf) & 1u;
+            ++cnt[hf];
+            // every warp must have finished its share of the last tile's copy-out (it reads the pixel table)
             bar_sync_epi(bid);
-            if (pi != cur) { copy_hot(&hot_s[2 + grp], &probs[pi].h, et, 128); cur = pi; bar_sync_epi(bid); }
-            const int n_tile = h.n_tile, ncol = h.ncol, add_mode = h.add_mode, dense = h.dense, out_slabs = h.out_slabs;
+            if (pi != cur) { copy_hot(&hot_s[1 + grp], &probs[pi].h, et, 128); cur = pi; bar_sync_epi(bid); }
+            const int n_tile = h.n_tile, ncol = h.ncol, add_mode = h.add_mode, dense = h.dense;
             const float scale = h.scale;
             const __nv_bfloat16* addp = h.add; __nv_bfloat16* outp = h.out; float* stat_tiles = h.stat_tiles;
-            const int tiles_n = h.tiles_n, tn = loc % tiles_n, tm = loc / tiles_n;
-            ok = mbar_wait(acc_full + 8 * buf, aph, &abort_s);
-            if (ok && add_mode == 1) { ok = mbar_wait(add_full + 8 * sb, add_use[sb] & 1u, &abort_s); ++add_use[sb]; }
-            ok = bar_and_epi(bid, ok);                           // one decision for the four warps: they share the barriers below
-            if (!ok) { atomicExch(&abort_s, 1); atomicExch(h.status, 6); break; }
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             // position -> output pixel (and the residual's pixel)
             const int pos = tm * TILE_M + m;
             bool valid = pos < h.total_pos;
@@ -414,37 +386,73 @@ __global__ void __launch_bounds__(TC_CONV_THREADS, 1) conv_tc_kernel(const TcPro
             }
             if (add_mode == 2) addpix = pix;
             if (!dense) pix_s[m] = valid ? (int)pix : -1;
-            const uint32_t t_row = tmem_base + buf * (uint32_t)L.acc_stride + ((uint32_t)(quad * 32) << 16);
             const int col0 = tn * n_tile;
-            const uint32_t s_row = stg + (uint32_t)m * 128u;
             const bool gadd = add_mode >= 2 && valid && addpix >= 0;
+            // the residual of a 32-column step is fetched one step ahead of its use (the first one ahead of the accumulator)
+            const __nv_bfloat16* addrow = addp + (gadd ? addpix : 0) * ncol + col0;
+            uint4 ga[4], gn[4];
+#pragma unroll
+            for (int g = 0; g < 4; ++g) gn[g] = (gadd && g * 8 < n_tile && col0 + g * 8 < ncol) ? __ldg(reinterpret_cast<const uint4*>(addrow + g * 8)) : make_uint4(0u, 0u, 0u, 0u);
+            if (add_mode == 2 && dense) {
+                // the residual rows of the group's next tile are asked into L2 now, a whole tile ahead of their use
+                int u2 = u, hf2 = hf + (L.groups == 2 ? 2 : 1);
+                if (hf2 >= nt) { u2 = u + u_step; hf2 = L.groups == 2 ? grp : 0; }
+                if (u2 < unit_end_s[pi]) {                       // same problem (else the next tile's own first loads have to do)
+                    const int loc2 = u2 - (pi ? unit_end_s[pi - 1] : 0);
+                    const int tn2 = loc2 % tilesn_s[pi], tm2 = 2 * (loc2 / tilesn_s[pi]) + hf2;
+                    const long long pos2 = (long long)tm2 * TILE_M + m;
+                    if (tm2 < tilesm_s[pi] && pos2 < h.total_pos) {
+                        const __nv_bfloat16* r2 = addp + pos2 * ncol + tn2 * n_tile;
+                        for (int c = 0; c < n_tile && tn2 * n_tile + c < ncol; c += 64)
+                            asm volatile("prefetch.global.L2 [%0];" ::"l"(r2 + c));
+                    }
+                }
+            }
+            ok = mbar_wait(acc_full + 8 * buf, aph, &abort_s);
+            ok = bar_and_epi(bid, ok);                           // one decision for the four warps: they share the barriers below
+            if (!ok) { atomicExch(&abort_s, 1); atomicExch(h.status, 6); break; }
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t t_row = tmem_base + buf * (uint32_t)L.acc_stride + ((uint32_t)(quad * 32) << 16);
+            // The tile leaves in slabs of 64 columns: a slab is rounded and (with the residual added) written to a 16 KB staging
+            // buffer in the 128-byte-swizzle layout, then stored by TMA (dense problems) or copied out row by row, while the next
+            // slab is staged in the group's other buffer.
             for (int c0 = 0; c0 < n_tile; c0 += 32) {
+                const int slab = c0 >> 6;
+                const bool slab_begin = !(c0 & 32), slab_end = (c0 & 32) || c0 + 32 >= n_tile, last = c0 + 32 >= n_tile;
+                const uint32_t stg = stg_base + ((uint32_t)(grp * L.pg) + sc % (uint32_t)L.pg) * SLAB_BYTES;
+                if (slab_begin) {
+                    if (leader) bulk_wait_read(L.pg - 1);        // the bulk store issued from this buffer has read it
+                    bar_sync_epi(bid);                           // ... and every warp is done with what it last held
+                }
                 uint32_t v[32];
                 tmem_ld32(t_row + (uint32_t)c0, v);
-                uint4 ga[4];
-                if (gadd) {
 #pragma unroll
-                    for (int g = 0; g < 4; ++g)
-                        ga[g] = (c0 + g * 8 < n_tile && col0 + c0 + g * 8 < ncol) ? __ldg(reinterpret_cast<const uint4*>(addp + addpix * ncol + col0 + c0 + g * 8)) : make_uint4(0u, 0u, 0u, 0u);
+                for (int g = 0; g < 4; ++g) {
+                    ga[g] = gn[g];
+                    const int c = c0 + 32 + g * 8;
+                    gn[g] = (gadd && c < n_tile && col0 + c < ncol) ? __ldg(reinterpret_cast<const uint4*>(addrow + c)) : make_uint4(0u, 0u, 0u, 0u);
                 }
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                if (last) {
+                    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(acc_empty + 8 * buf); // this warp has read its quadrant of the accumulator
+                }
+                const uint32_t s_row = stg + (uint32_t)m * 128u;
 #pragma unroll
                 for (int g = 0; g < 4; ++g) {
                     const int c = c0 + g * 8;
                     if (c < n_tile) {
-                        const uint32_t sa = s_row + (uint32_t)(c >> 6) * SLAB_BYTES + ((uint32_t)(((c >> 3) & 7) ^ (m & 7)) << 4);
+                        const uint32_t sa = s_row + ((uint32_t)(((c >> 3) & 7) ^ (m & 7)) << 4);
                         float f[8];
 #pragma unroll
                         for (int k = 0; k < 8; ++k) f[k] = valid ? __uint_as_float(v[g * 8 + k]) * scale : 0.f;
-                        if (add_mode == 1 || gadd) {
-                            const uint4 a0 = add_mode == 1 ? lds128(sa) : ga[g];
-                            const uint32_t aw[4] = {a0.x, a0.y, a0.z, a0.w};
-                            if (valid) {
+                        if (gadd) {
+                            const uint32_t aw[4] = {ga[g].x, ga[g].y, ga[g].z, ga[g].w};
 #pragma unroll
-                                for (int k = 0; k < 4; ++k) {
-                                    f[2 * k] += __uint_as_float(aw[k] << 16);
-                                    f[2 * k + 1] += __uint_as_float(aw[k] & 0xFFFF0000u);
-                                }
+                            for (int k = 0; k < 4; ++k) {
+                                f[2 * k] += __uint_as_float(aw[k] << 16);
+                                f[2 * k + 1] += __uint_as_float(aw[k] & 0xFFFF0000u);
                             }
                         }
                         uint32_t w[4];
@@ -456,31 +464,40 @@ __global__ void __launch_bounds__(TC_CONV_THREADS, 1) conv_tc_kernel(const TcPro
                         sts128(sa, make_uint4(w[0], w[1], w[2], w[3]));
                     }
                 }
-            }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // the bulk store reads what this thread wrote
-            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-            __syncwarp();
-            if (lane == 0) mbar_arrive(acc_empty + 8 * buf);     // this warp has read its quadrant of the accumulator
-            bar_sync_epi(bid);                                   // the staging tile is complete
-            if (dense && leader) {
-                for (int j = 0; j < out_slabs; ++j) tma_store_2d(&pp->map_out, stg + (uint32_t)(j * SLAB_BYTES), col0 + j * 64, tm * TILE_M);
-                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-            }
-            if (stat_tiles) {
-                // column sums of the stored (rounded) values: every warp over its own 32 rows, lane = two neighbouring columns;
-                // the four warps' sums are then added in a fixed order
-                for (int j = 0; j < out_slabs; ++j) {
+                if (!slab_end) continue;
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // the bulk store reads what this thread wrote
+                bar_sync_epi(bid);                               // the slab is complete
+                if (dense && leader) {
+                    tma_store_2d(&pp->map_out, stg, col0 + slab * 64, tm * TILE_M);
+                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                }
+                if (stat_tiles) {
+                    // column sums of the stored (rounded) values: every warp over its own 32 rows, lane = two neighbouring columns;
+                    // the four warps' sums are added in a fixed order once the tile's last slab is through
                     float s0 = 0.f, s1 = 0.f, q0 = 0.f, q1 = 0.f;
 #pragma unroll 8
                     for (int r = 0; r < 32; ++r) {
                         const int row = quad * 32 + r;
-                        const uint32_t u = lds32(stg + (uint32_t)(j * SLAB_BYTES) + (uint32_t)row * 128u + ((uint32_t)((lane >> 2) ^ (row & 7)) << 4) + ((uint32_t)(lane & 3) << 2));
-                        const float lo = __uint_as_float(u << 16), hi = __uint_as_float(u & 0xFFFF0000u);
+                        const uint32_t uu = lds32(stg + (uint32_t)row * 128u + ((uint32_t)((lane >> 2) ^ (row & 7)) << 4) + ((uint32_t)(lane & 3) << 2));
+                        const float lo = __uint_as_float(uu << 16), hi = __uint_as_float(uu & 0xFFFF0000u);
                         s0 += lo; q0 += lo * lo; s1 += hi; q1 += hi * hi;
                     }
-                    stat_s[quad][0][j * 64 + 2 * lane] = s0; stat_s[quad][0][j * 64 + 2 * lane + 1] = s1;
-                    stat_s[quad][1][j * 64 + 2 * lane] = q0; stat_s[quad][1][j * 64 + 2 * lane + 1] = q1;
+                    stat_s[quad][0][slab * 64 + 2 * lane] = s0; stat_s[quad][0][slab * 64 + 2 * lane + 1] = s1;
+                    stat_s[quad][1][slab * 64 + 2 * lane] = q0; stat_s[quad][1][slab * 64 + 2 * lane + 1] = q1;
                 }
+                if (!dense) {
+                    // copy-out of a tall slab: 16-byte chunks, eight consecutive lanes per 128-byte run of one output pixel
+                    for (int idx = et; idx < TILE_M * 8; idx += 128) {
+                        const int ch = idx & 7, row = idx >> 3;
+                        const int c = slab * 64 + ch * 8, px = pix_s[row];
+                        if (px >= 0 && c < n_tile && col0 + c < ncol)
+                            *reinterpret_cast<uint4*>(outp + (long long)px * ncol + col0 + c) =
+                                lds128(stg + (uint32_t)row * 128u + ((uint32_t)(ch ^ (row & 7)) << 4));
+                    }
+                }
+                ++sc;
+            }
+            if (stat_tiles) {
                 bar_sync_epi(bid);
                 for (int c = et; c < n_tile; c += 128) {
                     if (col0 + c < ncol) {
@@ -491,17 +508,7 @@ __global__ void __launch_bounds__(TC_CONV_THREADS, 1) conv_tc_kernel(const TcPro
                     }
                 }
             }
-            if (!dense) {
-                // copy-out of a tall tile: 16-byte chunks, eight consecutive lanes per 128-byte run of one output pixel
-                const int n_chunks = out_slabs * TILE_M * 8;
-                for (int idx = et; idx < n_chunks; idx += 128) {
-                    const int ch = idx & 7, row = (idx >> 3) & (TILE_M - 1), j = idx >> 10;
-                    const int c = j * 64 + ch * 8, px = pix_s[row];
-                    if (px >= 0 && c < n_tile && col0 + c < ncol)
-                        *reinterpret_cast<uint4*>(outp + (long long)px * ncol + col0 + c) =
-                            lds128(stg + (uint32_t)(j * SLAB_BYTES) + (uint32_t)row * 128u + ((uint32_t)(ch ^ (row & 7)) << 4));
-                }
-            }
+          }
         }
         if (leader) bulk_wait_read(0);                           // shared memory stays until the last bulk stores have read it
     }
@@ -923,9 +930,9 @@ int conv_tc_fill(const ConvProb& p, int mode, void* host_tc) {
             if (!encode_tall(&tp.map_a, act, chan_a, p.N, p.P, p.Q, g.Wp, g.box_h, g.box_n, 1)) return 0;
         }
         // residual
-        t.add_mode = !p.add ? 0 : p.add_sub == 2 ? 3 : t.dense ? 1 : 2;
-        // output tiles: up to 256 columns (128 with a prefetched residual: several staging tiles), a multiple of 64 when there are several
-        const int n_cap = t.add_mode == 1 ? 128 : 256;
+        t.add_mode = !p.add ? 0 : p.add_sub == 2 ? 3 : 2;
+        // output tiles: up to 256 columns, a multiple of 64 when there are several
+        const int n_cap = 256;
         const int ntaps = t.gbeg[t.ngroups];
         auto b_tile = [&](int nt) { return mode == CONV_FWD ? nt * 128 : ((nt + 63) / 64) * 8192; };
         auto b_total = [&](int nt) { return (size_t)t.slabs * ntaps * ((b_tile(nt) + 1023) / 1024 * 1024); };
@@ -945,14 +952,14 @@ int conv_tc_fill(const ConvProb& p, int mode, void* host_tc) {
           if (!encode_map(&tp.map_b, p.wgt, 3, dims, st, box)) return 0; }
         if (t.dense) {
             if (!encode_flat(&tp.map_out, p.out, ncol, out_pixels)) return 0;
-            if (t.add_mode == 1 && !encode_flat(&tp.map_add, p.add, ncol, out_pixels)) return 0;
         }
         memcpy((char*)host_tc + (size_t)ph * sizeof(TcProb), &tp, sizeof(tp));
     }
     return count;
 }
 size_t conv_tc_prob_bytes() { return sizeof(TcProb); }
-int conv_tc_tiles(const void* host_tc) { const TcHot* t = &((const TcProb*)host_tc)->h; return t->tiles_m * t->tiles_n; }
+// units of work of a problem: pairs of row tiles x column tiles
+int conv_tc_tiles(const void* host_tc) { const TcHot* t = &((const TcProb*)host_tc)->h; return ((t->tiles_m + 1) / 2) * t->tiles_n; }
 // packs what a launch has to know about its largest problem into one number: window KB (12 bits), weight-tile KB (12), staging
 // tiles (4), KB of all weight tiles of a column tile (16), MMA N (20)
 size_t conv_tc_smem(const void* host_tc) {
@@ -979,38 +986,22 @@ void launch_conv_tc_probs(const void* d_tc, int nprob, int max_tiles, size_t pac
     TcLaunch L{};
     L.nprob = nprob;
     L.a_stage = (int)(packed >> 52) * 1024; L.b_stage = (int)((packed >> 40) & 0xFFF) * 1024;
-    L.prefetch = ((packed >> 36) & 0xF) > 1 ? 1 : 0;
-    const size_t b_total = ((packed >> 20) & 0xFFFF) * 1024;
     const int n_tile = (int)(packed & 0xFFFFF);
-    L.stg_bytes = ((n_tile + 63) / 64) * SLAB_BYTES;
-    // Shared memory.  Staging tiles: two epilogue groups where they fit (they take alternate tiles, so two epilogues run side by
-    // side), each with two tiles when the residual is prefetched into them by TMA, else one; a single group (three tiles behind a
-    // prefetched residual) otherwise.  Weights: resident when all tiles of a column tile are small, else a ring of three tiles.  The
-    // rest goes to the ring of activation windows: an HBM-bound layer runs at the bytes it keeps in flight.
-    L.b_res = b_total <= TC_RESIDENT_BUDGET ? 1 : 0;
-    const size_t kgroups = L.b_stage ? b_total / (size_t)L.b_stage : 1;
-    const size_t b_min = L.b_res ? b_total : 2 * (size_t)L.b_stage;
-    L.groups = 2; L.pg = L.prefetch ? 2 : 1;
-    if (kgroups > 8) L.groups = 1;                             // long reductions: the epilogue is a small share, the smem goes to the rings
-    if (L.groups == 1 || (size_t)L.groups * L.pg * L.stg_bytes + 3 * (size_t)L.a_stage + b_min > TC_SMEM_BUDGET) {
-        L.groups = 1; L.pg = L.prefetch ? 3 : 1;
-        while (L.pg > (L.prefetch ? 2 : 1) && (size_t)L.pg * L.stg_bytes + 2 * (size_t)L.a_stage + b_min > TC_SMEM_BUDGET) --L.pg;
-    }
-    L.n_stg = L.groups * L.pg;
-    const size_t rings = TC_SMEM_BUDGET - (size_t)L.n_stg * L.stg_bytes;
-    if (L.b_res) {
-        L.nb = 0; L.b_region = (int)b_total;
-        L.na = 2; while (L.na < TC_MAX_STAGES && (size_t)(L.na + 1) * L.a_stage + b_total <= rings) ++L.na;
-    } else {
-        L.nb = 3; while (L.nb > 2 && (size_t)L.nb * L.b_stage + 2 * (size_t)L.a_stage > rings) --L.nb;
-        L.na = 2; while (L.na < TC_MAX_STAGES && (size_t)(L.na + 1) * L.a_stage + (size_t)L.nb * L.b_stage <= rings) ++L.na;
-        while (L.nb < 6 && (size_t)L.na * L.a_stage + (size_t)(L.nb + 1) * L.b_stage <= rings) ++L.nb;
-        L.b_region = L.nb * L.b_stage;
-    }
+    // Shared memory.  Two epilogue groups, each with two 16 KB slab buffers (one where the rings need the room).  The windows' ring
+    // gets four stages (two pairs of tiles), the weights' ring what is left, up to eight tiles; any rest goes back to the windows.
+    // A layer runs at the bytes it keeps in flight.
+    const size_t a = (size_t)L.a_stage, b = (size_t)L.b_stage;
+    L.groups = 2; L.pg = 2;
+    if ((size_t)L.groups * L.pg * SLAB_BYTES + 4 * a + 3 * b > TC_SMEM_BUDGET) L.pg = 1;
+    const size_t rings = TC_SMEM_BUDGET - (size_t)L.groups * L.pg * SLAB_BYTES;
+    L.na = 4; while (L.na > 2 && (size_t)L.na * a + 2 * b > rings) --L.na;
+    L.nb = 2; while (L.nb < 8 && (size_t)L.na * a + (size_t)(L.nb + 1) * b <= rings) ++L.nb;
+    while (L.na < TC_MAX_STAGES && (size_t)(L.na + 1) * a + (size_t)L.nb * b <= rings) ++L.na;
     L.acc_stride = (n_tile + 31) / 32 * 32;
-    L.tmem_cols = 32; while (L.tmem_cols < 2 * L.acc_stride) L.tmem_cols *= 2;
+    L.nbuf = L.acc_stride <= 128 ? 2 : 1;
+    L.tmem_cols = 32; while (L.tmem_cols < 2 * L.nbuf * L.acc_stride) L.tmem_cols *= 2;
     // at least 120 KB of shared memory so that two CTAs that allocate tensor memory never share an SM
-    const size_t smem = std::max((size_t)L.na * L.a_stage + (size_t)L.b_region + (size_t)L.n_stg * L.stg_bytes, (size_t)120 * 1024) + 1024;
+    const size_t smem = std::max((size_t)L.na * a + (size_t)L.nb * b + (size_t)L.groups * L.pg * SLAB_BYTES, (size_t)120 * 1024) + 1024;
     const long long total = (long long)max_tiles * nprob;
     const int grid = (int)std::max(1ll, std::min(total, (long long)sms));
     conv_tc_kernel<<<grid, TC_CONV_THREADS, smem, s>>>((const TcProb*)d_tc, L);
