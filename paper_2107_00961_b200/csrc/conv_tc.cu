@@ -114,7 +114,7 @@ __device__ __forceinline__ uint4 lds128(uint32_t a) { uint4 v; asm volatile("ld.
 __device__ __forceinline__ void sts128(uint32_t a, uint4 v) { asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory"); }
 __device__ __forceinline__ uint32_t lds32(uint32_t a) { uint32_t v; asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(a)); return v; }
 
-constexpr int TC_THREADS = 192;              // wgrad kernel: producer warp, MMA warp, four epilogue warps
+constexpr int TC_THREADS = 224;              // wgrad kernel: producer warp, two MMA warps, four epilogue warps
 constexpr int TC_MAX_ISSUERS = 2;            // forward / dgrad kernel: MMA-issuing warps, one per tile of a pair
 constexpr int TC_CONV_THREADS = 32 * (1 + TC_MAX_ISSUERS + 8);   // forward / dgrad kernel: producer warp, MMA warps, two groups of four epilogue warps
 constexpr int TC_MAX_STAGES = 12;
@@ -588,17 +588,18 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_wgrad_tc_kernel(const TcWg
 
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    __shared__ __align__(8) uint64_t bars[2 * TC_MAX_STAGES + 1];
+    __shared__ __align__(8) uint64_t bars[2 * TC_MAX_STAGES + 3];
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
     __shared__ int shift8_s[4], wtap_s[4];                       // the group's taps: row shift in 16-byte units, index in dw
     const uint32_t bar_full = smem_u32(&bars[0]), bar_empty = smem_u32(&bars[TC_MAX_STAGES]), bar_acc = smem_u32(&bars[2 * TC_MAX_STAGES]);
+    const uint32_t bar_drain = smem_u32(&bars[2 * TC_MAX_STAGES + 1]);
     const uint32_t ring = smem_u32(smem);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < TC_MAX_STAGES; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
-        mbar_init(bar_acc, 1);
+        for (int s = 0; s < TC_MAX_STAGES; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 2); }   // both issuers release a stage
+        mbar_init(bar_acc, 2); mbar_init(bar_drain, 1); mbar_init(bar_drain + 8, 1);
         abort_s = 0;
         for (int i = 0; i < ntap; ++i) { shift8_s[i] = p.tap[tap0 + i].shift * 8; wtap_s[i] = p.tap[tap0 + i].wtap; }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -648,8 +649,16 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_wgrad_tc_kernel(const TcWg
                 for (int c = max(0, i - stages); c < i; ++c)
                     for (int w = 0; w < 4096 && !mbar_try(bar_full + 8 * (c % stages), (uint32_t)(c / stages) & 1u); ++w) __nanosleep(64);
         }
-    } else if (warp == 1) {
+    } else if (warp <= 2) {
+        // Two issuing warps (one thread issues a tcgen05.mma only every ~150 cycles, more than the tensor core needs for it).  The
+        // group's taps are split between them; with an odd number of taps the last tap's 128 positions are split instead, each
+        // half into an accumulator of its own (the epilogue adds the two, first half first).  So every accumulator is written
+        // by one thread, in a fixed order.
         if (lane == 0) {
+            const int me = warp - 1, odd = ntap & 1, whole = (ntap - odd) >> 1;
+            int it_tap[3], it_acc[3], it_k0[3], it_k1[3], nit = 0;
+            for (int q = 0; q < whole; ++q) { it_tap[nit] = me * whole + q; it_acc[nit] = me * whole + q; it_k0[nit] = 0; it_k1[nit] = 8; ++nit; }
+            if (odd) { it_tap[nit] = ntap - 1; it_acc[nit] = ntap - 1 + me; it_k0[nit] = me * 4; it_k1[nit] = me * 4 + 4; ++nit; }
             // fp32 accumulate, bf16 x bf16, A and B MN-major, N = n_tile, M = 128
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) | ((uint32_t)(n_tile >> 3) << 17) | ((128u >> 4) << 24);
             const uint64_t dy_const = desc_sw128(0, (uint32_t)dy_slab_bytes, 1024), a_const = desc_sw128(0, (uint32_t)a_slab_bytes, 1024);
@@ -662,17 +671,22 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_wgrad_tc_kernel(const TcWg
                 const int a_off = a_flat ? 0 : pos0 - hb - floor_div(pos0 - hb, box_pos) * box_pos;
                 const uint32_t dy16 = ((ring + (uint32_t)(s * stage_bytes)) >> 4) + (uint32_t)dy_off * 8u;       // start addresses in 16-byte units
                 const uint32_t a16 = ((ring + (uint32_t)(s * stage_bytes) + 2u * (uint32_t)dy_slab_bytes) >> 4) + (uint32_t)a_off * 8u;
-                for (int tt = 0; tt < ntap; ++tt) {
-                    const uint32_t at16 = a16 + (uint32_t)shift8_s[tt];
-                    const uint32_t d_t = tmem_d + (uint32_t)(tt * n_tile);
-#pragma unroll
-                    for (int k16 = 0; k16 < 8; ++k16)          // 16 positions = 16 rows of 128 bytes per step
-                        umma_bf16(d_t, dy_const | (uint64_t)((dy16 + 128u * (uint32_t)k16) & 0x3FFFu), a_const | (uint64_t)((at16 + 128u * (uint32_t)k16) & 0x3FFFu), idesc, (i | k16) ? 1u : 0u);
+                for (int q = 0; q < nit; ++q) {
+                    const uint32_t at16 = a16 + (uint32_t)shift8_s[it_tap[q]];
+                    const uint32_t d_t = tmem_d + (uint32_t)(it_acc[q] * n_tile);
+                    const int k0 = it_k0[q], k1 = it_k1[q];
+                    for (int k16 = k0; k16 < k1; ++k16)        // 16 positions = 16 rows of 128 bytes per step
+                        umma_bf16(d_t, dy_const | (uint64_t)((dy16 + 128u * (uint32_t)k16) & 0x3FFFu), a_const | (uint64_t)((at16 + 128u * (uint32_t)k16) & 0x3FFFu), idesc, (i || k16 != k0) ? 1u : 0u);
                 }
                 umma_commit(bar_empty + 8 * s);
                 if (++s == stages) { s = 0; ph ^= 1u; }
             }
             if (ok) umma_commit(bar_acc);
+            else {
+                // gave up: the MMAs already issued must have finished before the CTA frees its tensor memory
+                umma_commit(bar_drain + 8 * me);
+                for (int w = 0; w < 65536 && !mbar_try(bar_drain + 8 * me, 0u); ++w) __nanosleep(64);
+            }
         }
     } else {
         const int quad = warp & 3, m = quad * 32 + lane;
@@ -690,9 +704,17 @@ __global__ void __launch_bounds__(TC_THREADS, 1) conv_wgrad_tc_kernel(const TcWg
                                         : outp + ((long long)k * taps + wt) * cin + tn * n_tile;
                 for (int c0 = 0; c0 < n_tile; c0 += 32) {
                     uint32_t v[32];
-                    if (nc > 0) { tmem_ld32(tmem_d + ((uint32_t)(quad * 32) << 16) + (uint32_t)(tt * n_tile + c0), v);
-                        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-                    else { for (int j = 0; j < 32; ++j) v[j] = 0u; }
+                    if (nc > 0) {
+                        tmem_ld32(tmem_d + ((uint32_t)(quad * 32) << 16) + (uint32_t)(tt * n_tile + c0), v);
+                        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                        if ((ntap & 1) && tt == ntap - 1) {      // the tap whose positions were split: first half + second half
+                            uint32_t v2[32];
+                            tmem_ld32(tmem_d + ((uint32_t)(quad * 32) << 16) + (uint32_t)(ntap * n_tile + c0), v2);
+                            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) + __uint_as_float(v2[j]));
+                        }
+                    } else { for (int j = 0; j < 32; ++j) v[j] = 0u; }
                     if (k < cout) {
 #pragma unroll
                         for (int j = 0; j < 32; j += 4)
@@ -795,19 +817,19 @@ static bool encode_tall(CUtensorMap* m, const void* base, int chan, int n_img, i
 // one image (R divides Hp), or box_n whole images.  Larger boxes mean fewer TMA issues per window but more rows fetched around it;
 // the choice: at most 96 positions per box, at most 6.5 % of extra rows, then the largest box.
 struct Tall { int Hp, Wp, R, box_pos, box_bytes, box_h, box_n; };
-static bool tall_of(int Hg, int Wg, int pad, int es, Tall& t) {
+static bool tall_of(int Hg, int Wg, int pad, int es, Tall& t, int max_box = 96) {
     t.Wp = Wg + pad;
     const int H0 = Hg + pad;
     if (t.Wp * es > 256) return false;
     int best_r = 1, best_hp = H0;
     for (int r = 1; r <= H0; ++r) {
         const int hp = (H0 + r - 1) / r * r;
-        if (r * t.Wp > 96 || r * es > 256 || (hp - H0) * 200 > 13 * H0 || (pad == 0 && hp != H0)) continue;   // pad = 0: positions are the pixels in order, no extra rows
+        if ((r > 1 && r * t.Wp > max_box) || r * t.Wp > 96 || r * es > 256 || (hp - H0) * 200 > 13 * H0 || (pad == 0 && hp != H0)) continue;   // pad = 0: positions are the pixels in order, no extra rows
         if (r * t.Wp > best_r * t.Wp) { best_r = r; best_hp = hp; }
     }
     t.Hp = best_hp; t.R = best_r; t.box_h = best_r; t.box_n = 1;
     if (best_r == best_hp) {                      // whole images: several per box when they are small
-        int ni = 96 / (t.Hp * t.Wp); if (ni < 1) ni = 1; if (ni > 8) ni = 8;
+        int ni = max_box / (t.Hp * t.Wp); if (ni < 1) ni = 1; if (ni > 8) ni = 8;
         t.box_n = ni; t.R = t.Hp * ni;
     }
     t.box_pos = t.R * t.Wp; t.box_bytes = t.box_pos * 128;
@@ -1010,7 +1032,24 @@ void launch_conv_tc_probs(const void* d_tc, int nprob, int max_tiles, size_t pac
 // ---- wgrad host side
 struct WgGeom { TcWgradProb t; size_t smem, partial_bytes; int box_h, box_n; };
 
+static bool wg_geometry_box(const ConvProb& p, int target_ctas, WgGeom& w, int max_box);
+// Both operands of a 3x3 weight gradient are windows of boxes, so a stage is large and the boxes' rounding decides how many stages
+// fit: the largest boxes that still leave two stages are taken (fewer TMA issues), else the size with the most stages.
 static bool wg_geometry(const ConvProb& p, int target_ctas, WgGeom& w) {
+    if (p.ksz == 1) return wg_geometry_box(p, target_ctas, w, 96);
+    const int caps[5] = {96, 64, 48, 32, 24};
+    WgGeom best; int best_stages = 0;
+    for (int i = 0; i < 5; ++i) {
+        WgGeom g;
+        if (!wg_geometry_box(p, target_ctas, g, caps[i])) continue;
+        if (g.t.stages > best_stages) { best = g; best_stages = g.t.stages; }
+        if (best_stages >= 2) break;
+    }
+    if (!best_stages) return false;
+    w = best;
+    return true;
+}
+static bool wg_geometry_box(const ConvProb& p, int target_ctas, WgGeom& w, int max_box) {
     if (!tc_shape_ok(p)) return false;
     if (((uintptr_t)p.act | (uintptr_t)p.wgt) & 15) return false;
     TcWgradProb& t = w.t; memset(&t, 0, sizeof(t));
@@ -1030,7 +1069,7 @@ static bool wg_geometry(const ConvProb& p, int target_ctas, WgGeom& w) {
         total_pos = (long long)p.N * g.Hp * g.Wp;
         t.tap_groups = 1; t.gbeg[1] = 1; t.tap[0] = TapRef{0, 0};
     } else if (p.stride == 1) {
-        Tall g; if (!tall_of(p.H, p.W, 1, 1, g)) return false;
+        Tall g; if (!tall_of(p.H, p.W, 1, 1, g, max_box)) return false;
         w.box_h = g.box_h; w.box_n = g.box_n;
         t.dy_flat = 0; t.a_flat = 0; t.pad = 1; t.Hp = g.Hp; t.Wp = g.Wp; t.R = g.R; t.box_pos = g.box_pos; t.hb = g.Wp + 1;
         t.nbox_dy = boxes_for(TILE_M, g.box_pos); t.nbox_a = boxes_for(TILE_M + 2 * t.hb, g.box_pos); t.dy_box_bytes = g.box_bytes; t.a_box_bytes = g.box_bytes;
@@ -1038,8 +1077,8 @@ static bool wg_geometry(const ConvProb& p, int target_ctas, WgGeom& w) {
         for (int i = 0; i < 9; ++i) t.tap[i] = TapRef{i, (i / 3) * g.Wp + (i % 3)};
         t.tap_groups = 0;                                // groups of up to three taps: set below, once the column tile is known
     } else {
-        Tall g; if (!tall_of(p.P, p.Q, 1, 2, g)) return false;
-        Tall gd; if (!tall_of(p.P, p.Q, 1, 1, gd)) return false;
+        Tall g; if (!tall_of(p.P, p.Q, 1, 2, g, max_box)) return false;
+        Tall gd; if (!tall_of(p.P, p.Q, 1, 1, gd, max_box)) return false;
         if (gd.R != g.R || gd.Hp != g.Hp) return false;          // both operands walk the same boxes of rows
         w.box_h = g.box_h; w.box_n = g.box_n;
         t.dy_flat = 0; t.a_flat = 0; t.pad = 1; t.es = 2; t.Hp = g.Hp; t.Wp = g.Wp; t.R = g.R; t.box_pos = g.box_pos; t.hb = g.Wp + 1;
@@ -1064,7 +1103,9 @@ static bool wg_geometry(const ConvProb& p, int target_ctas, WgGeom& w) {
     t.a_slabs = (t.n_tile + 63) / 64;
     if (taps == 9 && p.stride == 1) { for (int g = 0; g < 3; ++g) { t.gbeg[g + 1] = 3 * (g + 1); t.gxs[g] = 0; t.gys[g] = 0; } t.tap_groups = 3; }
     int max_group = 0; for (int g = 0; g < t.tap_groups; ++g) max_group = std::max(max_group, t.gbeg[g + 1] - t.gbeg[g]);
-    t.tmem_cols = 32; while (t.tmem_cols < max_group * t.n_tile) t.tmem_cols *= 2;
+    int max_acc = 0; for (int g = 0; g < t.tap_groups; ++g) { const int n = t.gbeg[g + 1] - t.gbeg[g]; max_acc = std::max(max_acc, n + (n & 1)); }   // an odd group's last tap takes two accumulators
+    (void)max_group;
+    t.tmem_cols = 32; while (t.tmem_cols < max_acc * t.n_tile) t.tmem_cols *= 2;
     if (t.tmem_cols > 512) return false;
     t.dy_slab_bytes = (t.nbox_dy * t.dy_box_bytes + 1023) / 1024 * 1024;
     t.a_slab_bytes = (t.nbox_a * t.a_box_bytes + 1023) / 1024 * 1024;
@@ -1072,10 +1113,20 @@ static bool wg_geometry(const ConvProb& p, int target_ctas, WgGeom& w) {
     t.stages = TC_MAX_STAGES; while (t.stages > 1 && (size_t)t.stages * t.stage_bytes > TC_SMEM_BUDGET) --t.stages;
     if ((size_t)t.stages * t.stage_bytes > TC_SMEM_BUDGET) return false;
     w.smem = std::max((size_t)t.stages * t.stage_bytes, (size_t)120 * 1024) + 1024;
+    // Split of the positions.  target_ctas is twice this problem's share of the SMs.  Every CTA pays a fixed cost (set-up, the
+    // accumulators' way out) worth about six chunks, and a launch takes whole waves, so the split is the one that minimises
+    // waves x (chunks per CTA + 6): mostly one full wave.  The partial buffer is sized for the most splits any share could pick.
     const int fixed = t.m_tiles * t.n_tiles * t.tap_groups;
-    int want = std::max(1, target_ctas / fixed); if (want > t.chunks) want = t.chunks; if (want > 256) want = 256;
-    t.chunks_per_split = (t.chunks + want - 1) / want; t.splits = (t.chunks + t.chunks_per_split - 1) / t.chunks_per_split;
-    w.partial_bytes = t.splits > 1 ? (size_t)t.splits * taps * p.K * p.C * 4 : 0;
+    const int want_max = std::max(1, std::min(std::min(t.chunks, 256), target_ctas / fixed));
+    const int share = std::max(1, target_ctas / 2);
+    long long best_cost = -1; int best_cps = t.chunks;
+    for (int sp = 1; sp <= want_max; ++sp) {
+        const int cps = (t.chunks + sp - 1) / sp, eff = (t.chunks + cps - 1) / cps;
+        const long long waves = ((long long)fixed * eff + share - 1) / share, cost = waves * (cps + 6);
+        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_cps = cps; }
+    }
+    t.chunks_per_split = best_cps; t.splits = (t.chunks + best_cps - 1) / best_cps;
+    w.partial_bytes = want_max > 1 ? (size_t)want_max * taps * p.K * p.C * 4 : 0;
     return true;
 }
 
