@@ -190,16 +190,26 @@ __device__ void bn_reduce_vec(const BnProb& p) {
     }
     const uint4* xv = reinterpret_cast<const uint4*>(p.x);
     const uint4* dv = reinterpret_cast<const uint4*>(p.da);
-#pragma unroll 4
-    for (long long row = r0 + r; row < r1; row += R) {
-        float x[8]; unpack8(xv[row * G + g], x);
-        if (MODE == 0) {
+    // four rows of loads in flight per thread; the rows are still added in ascending order
+    for (long long row = r0 + r; row < r1; row += 4 * R) {
+        uint4 xs[4], ds[4];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) { const float d = x[j] - sh[j]; s0[j] += d; s1[j] += d * d; }
-        } else {
-            float d[8]; unpack8(dv[row * G + g], d);
+        for (int u = 0; u < 4; ++u) {
+            const long long rr = row + (long long)u * R;
+            if (rr < r1) { xs[u] = __ldg(xv + rr * G + g); if (MODE == 1) ds[u] = __ldg(dv + rr * G + g); }
+        }
 #pragma unroll
-            for (int j = 0; j < 8; ++j) { const float xh = (x[j] - mean[j]) * istd[j]; const float dz = (xh * ga[j] + be[j] > 0.f) ? d[j] : 0.f; s0[j] += dz; s1[j] += dz * xh; }
+        for (int u = 0; u < 4; ++u) {
+            if (row + (long long)u * R >= r1) break;
+            float x[8]; unpack8(xs[u], x);
+            if (MODE == 0) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) { const float d = x[j] - sh[j]; s0[j] += d; s1[j] += d * d; }
+            } else {
+                float d[8]; unpack8(ds[u], d);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) { const float xh = (x[j] - mean[j]) * istd[j]; const float dz = (xh * ga[j] + be[j] > 0.f) ? d[j] : 0.f; s0[j] += dz; s1[j] += dz * xh; }
+            }
         }
     }
     // lanes of a warp that own the same channel group: fixed-order butterfly in fp32
@@ -230,11 +240,11 @@ __device__ void bn_reduce_vec(const BnProb& p) {
     }
 }
 
-// Streaming form of the elementwise pass (bf16 vector path): a thread keeps ONE group of 8 channels for all its rows, so the
+// Streaming form of the elementwise pass (bf16 vector path; stat: [4][C] as BnProb::stat, in global or shared memory): a thread keeps ONE group of 8 channels for all its rows, so the
 // per-channel constants are loaded once into registers and the loop is loads, arithmetic and a store; a CTA takes at least 16 passes
 // of 256 / G rows (32768 elements), four rows of loads in flight per thread.  MODE 0: a = relu(bn(x)); MODE 1: dx (+ add).
 template <int MODE>
-__device__ void bn_stream_vec(const BnProb& p) {
+__device__ void bn_stream_vec(const BnProb& p, const float* __restrict__ stat) {
     const int C = p.C, G = C >> 3, R = 256 / G;
     const int g = threadIdx.x % G, r = threadIdx.x / G;
     // the grid's CTAs share the rows evenly, in whole passes of 4 * R rows (at least 16 passes of R rows each)
@@ -248,8 +258,8 @@ __device__ void bn_stream_vec(const BnProb& p) {
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
         const int c = g * 8 + j;
-        mean[j] = p.stat[c]; istd[j] = p.stat[C + c]; ga[j] = p.gamma[c]; be[j] = p.beta[c];
-        if (MODE == 1) { sb[j] = p.stat[2 * C + c] * inv_m; sg[j] = p.stat[3 * C + c] * inv_m; }
+        mean[j] = stat[c]; istd[j] = stat[C + c]; ga[j] = p.gamma[c]; be[j] = p.beta[c];
+        if (MODE == 1) { sb[j] = stat[2 * C + c] * inv_m; sg[j] = stat[3 * C + c] * inv_m; }
     }
     const uint4* xv = reinterpret_cast<const uint4*>(p.x);
     const uint4* dv = reinterpret_cast<const uint4*>(p.da);
@@ -288,47 +298,6 @@ __device__ void bn_stream_vec(const BnProb& p) {
                 ov[rr * G + g] = pack8(o);
             }
         }
-    }
-}
-
-template <int MODE>   // 0: forward apply; 1: backward apply.  stat: [4][C] as BnProb::stat, in global or shared memory
-__device__ void bn_apply_vec(const BnProb& p, const float* __restrict__ stat) {
-    const int C = p.C, G = C >> 3;
-    const long long nv = p.m * G;
-    const float inv_m = 1.f / (float)p.m;
-    const uint4* xv = reinterpret_cast<const uint4*>(p.x);
-    const uint4* dv = reinterpret_cast<const uint4*>(p.da);
-    const uint4* av = reinterpret_cast<const uint4*>(p.add);
-    uint4* ov = reinterpret_cast<uint4*>(MODE == 0 ? p.a : p.dx);
-    const long long stride = (long long)gridDim.x * blockDim.x;
-    for (long long v = blockIdx.x * (long long)blockDim.x + threadIdx.x; v < nv; v += stride) {
-        const int c0 = (int)(v & (long long)(G - 1)) * 8;          // G is a power of two
-        float x[8], o[8]; unpack8(xv[v], x);
-        const float4 m0 = *reinterpret_cast<const float4*>(stat + c0), m1 = *reinterpret_cast<const float4*>(stat + c0 + 4);
-        const float4 i0 = *reinterpret_cast<const float4*>(stat + C + c0), i1 = *reinterpret_cast<const float4*>(stat + C + c0 + 4);
-        const float4 g0 = *reinterpret_cast<const float4*>(p.gamma + c0), g1 = *reinterpret_cast<const float4*>(p.gamma + c0 + 4);
-        const float4 b0 = *reinterpret_cast<const float4*>(p.beta + c0), b1 = *reinterpret_cast<const float4*>(p.beta + c0 + 4);
-        const float mean[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w}, istd[8] = {i0.x, i0.y, i0.z, i0.w, i1.x, i1.y, i1.z, i1.w};
-        const float ga[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w}, be[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
-        if (MODE == 0) {
-#pragma unroll
-            for (int j = 0; j < 8; ++j) { const float z = (x[j] - mean[j]) * istd[j] * ga[j] + be[j]; o[j] = z > 0.f ? z : 0.f; }
-        } else {
-            float d[8]; unpack8(dv[v], d);
-            const float4 s0 = *reinterpret_cast<const float4*>(stat + 2 * C + c0), s1 = *reinterpret_cast<const float4*>(stat + 2 * C + c0 + 4);
-            const float4 t0 = *reinterpret_cast<const float4*>(stat + 3 * C + c0), t1 = *reinterpret_cast<const float4*>(stat + 3 * C + c0 + 4);
-            const float sb[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w}, sg[8] = {t0.x, t0.y, t0.z, t0.w, t1.x, t1.y, t1.z, t1.w};
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const float xh = (x[j] - mean[j]) * istd[j];
-                const float dz = (xh * ga[j] + be[j] > 0.f) ? d[j] : 0.f;
-                o[j] = ga[j] * istd[j] * (dz - sb[j] * inv_m - xh * sg[j] * inv_m);
-            }
-            if (av) { float ad[8]; unpack8(av[v], ad);
-#pragma unroll
-                for (int j = 0; j < 8; ++j) o[j] += ad[j]; }
-        }
-        ov[v] = pack8(o);
     }
 }
 
@@ -407,7 +376,7 @@ __global__ void bn_finalize_kernel(const BnProb* __restrict__ probs) {
 template <class T>
 __global__ void __launch_bounds__(256) bn_apply_kernel(const BnProb* __restrict__ probs) {
     const BnProb& p = probs[blockIdx.y];
-    if (p.vec) { bn_stream_vec<0>(p); return; }
+    if (p.vec) { bn_stream_vec<0>(p, p.stat); return; }
     const long long n = p.m * p.C;
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
         const int c = (int)(i % p.C);
@@ -417,9 +386,9 @@ __global__ void __launch_bounds__(256) bn_apply_kernel(const BnProb* __restrict_
 }
 
 template <class T>
-__global__ void __launch_bounds__(256) bn_bwd_apply_kernel(const BnProb* __restrict__ probs) {
+__global__ void __launch_bounds__(256, 2) bn_bwd_apply_kernel(const BnProb* __restrict__ probs) {
     const BnProb& p = probs[blockIdx.y];
-    if (p.vec) { bn_stream_vec<1>(p); return; }
+    if (p.vec) { bn_stream_vec<1>(p, p.stat); return; }
     const long long n = p.m * p.C;
     const float inv_m = 1.f / (float)p.m;
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
@@ -440,7 +409,7 @@ __global__ void __launch_bounds__(256) bn_bwd_apply_kernel(const BnProb* __restr
 // CTA 0 of the problem also stores them) and takes its share of the elementwise pass, whose re-read of x comes
 // from L2.  bf16 vector path, training mode only.
 template <int MODE>
-__global__ void __launch_bounds__(256) bn_fused_kernel(const BnProb* __restrict__ probs) {
+__global__ void __launch_bounds__(256, 2) bn_fused_kernel(const BnProb* __restrict__ probs) {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // a convolution launched behind this kernel may start its prologue
     const BnProb& p = probs[blockIdx.y];
     __shared__ __align__(16) float s_stat[4 * 512];               // callers keep C <= 512
@@ -486,7 +455,7 @@ __global__ void __launch_bounds__(256) bn_fused_kernel(const BnProb* __restrict_
         }
     }
     __syncthreads();
-    bn_apply_vec<MODE>(p, s_stat);
+    bn_stream_vec<MODE>(p, s_stat);
 }
 
 bool launch_bn_fused(const BnProb* d, int nprob, int max_chunks, int backward, cudaStream_t s) {

@@ -57,7 +57,11 @@ int conv_wgrad_mma_pick_variant(const ConvProb& p, int target_ctas);
 // output channels; forward and dgrad: 1000 + the kernel variant, so that the value also separates launches by what
 // the kernel is specialised on).
 static int pick_backend(const ConvProb& p, int mode, int target_ctas, size_t* partial_bytes, int pref = RESIST_CONV_AUTO) {
-    const bool want_mma = pref == RESIST_CONV_AUTO || pref == RESIST_CONV_WARP_MMA || pref == RESIST_CONV_WARP_MMA_UNFUSED, want_tc = pref == RESIST_CONV_AUTO || pref == RESIST_CONV_TCGEN05;
+    bool want_mma = pref == RESIST_CONV_AUTO || pref == RESIST_CONV_WARP_MMA || pref == RESIST_CONV_WARP_MMA_UNFUSED; const bool want_tc = pref == RESIST_CONV_AUTO || pref == RESIST_CONV_TCGEN05;
+    // 3x3 layers of 64 channels and more with many positions run faster on tcgen05 followed by the streaming BN kernels than on
+    // the warp-level MMA kernels with the BN inside (measured at 8 x 128 images of 32 x 32: 450 -> 218 us forward, 668 -> 211 +
+    // 195 us backward); small ones stay (a ResNet-110 stage of 8 x 8 maps measured the same either way)
+    if (pref == RESIST_CONV_AUTO && p.C >= 64 && p.K >= 64 && p.ksz == 3 && (long long)p.N * p.H * p.W >= 65536) want_mma = false;
     if (mode == CONV_WGRAD) {
         if (want_mma && conv_wgrad_mma_supported(p, target_ctas, partial_bytes)) return 200 + conv_wgrad_mma_pick_variant(p, target_ctas);
         if (want_tc && conv_wgrad_tc_supported(p, target_ctas, partial_bytes)) return 1;
@@ -289,8 +293,9 @@ struct Builder {
         BnProb& p = op.bn;
         p.x = x; p.da = da; p.dx = dx; p.add = add; p.gamma = W() + r.g; p.beta = W() + r.b; p.dgamma = G() + r.g; p.dbeta = G() + r.b;
         p.stat = stat; p.m = m; p.C = r.c; p.eps = ctx->opts.bn_eps; p.momentum = ctx->opts.bn_momentum; p.eval = 0;
-        // (measured on 8 x 67 MB tensors, far beyond L2: the single cooperative launch, 794 us, still beats a reduction with many small
-        // chunks followed by a streaming elementwise pass, 308 + 539 us; both move the same six passes over HBM)
+        // (measured on 8 x 67 MB tensors, far beyond L2: the single cooperative launch, 586 us with two CTAs per SM and four rows of
+        // loads in flight per thread in both passes, beats the reduction kernel followed by the streaming elementwise kernel, 683 us;
+        // both move the same five passes over HBM)
         bn_chunking(p, ctx->opts.dtype == RESIST_BF16, fused_chunks());
         bn_partial_need = std::max(bn_partial_need, (size_t)p.chunks * 2 * r.c * 8);
         p.partial = bn_partial;
