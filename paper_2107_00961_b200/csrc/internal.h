@@ -63,7 +63,8 @@ inline void bn_chunking(BnProb& p, bool bf16, int target_chunks = 0) {
     const long long lim = (m + 1023) / 1024; if (rpc < lim) rpc = lim;
     if (p.vec && target_chunks > 0 && (m + rpc - 1) / rpc < target_chunks) {      // more, smaller chunks (whole sweeps of the CTA's rows)
         const int R = 256 / G;
-        rpc = ((m + target_chunks - 1) / target_chunks + R - 1) / R * R; if (rpc < R) rpc = R;
+        rpc = ((m + target_chunks - 1) / target_chunks + R - 1) / R * R;
+        if (rpc < 32 * R) rpc = 32 * R;            // every CTA of the cooperative kernels re-adds all chunks' sums: few chunks for small problems
     }
     p.rows_per_chunk = (int)rpc; p.chunks = (int)((m + rpc - 1) / rpc);
 }
