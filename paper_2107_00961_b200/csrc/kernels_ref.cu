@@ -458,15 +458,19 @@ __global__ void __launch_bounds__(256, 2) bn_fused_kernel(const BnProb* __restri
     bn_stream_vec<MODE>(p, s_stat);
 }
 
-bool launch_bn_fused(const BnProb* d, int nprob, int max_chunks, int backward, cudaStream_t s) {
-    static int cap[2] = {0, 0};                                    // co-resident CTAs of each kernel on this device
+// CTAs of the cooperative kernel that can be resident together on this device (its largest grid)
+int bn_fused_capacity(int backward) {
+    static int cap[2] = {0, 0};
     if (!cap[backward]) {
         int dev = 0, sms = 0, per = 0; cudaGetDevice(&dev); cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         if (backward) cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per, bn_fused_kernel<1>, 256, 0);
         else cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per, bn_fused_kernel<0>, 256, 0);
         cap[backward] = per * sms > 0 ? per * sms : -1;
     }
-    if ((long long)max_chunks * nprob > cap[backward]) return false;
+    return cap[backward];
+}
+bool launch_bn_fused(const BnProb* d, int nprob, int max_chunks, int backward, cudaStream_t s) {
+    if ((long long)max_chunks * nprob > bn_fused_capacity(backward)) return false;
     void* args[] = {(void*)&d};
     const dim3 grid(max_chunks, nprob), block(256);
     const cudaError_t e = backward ? cudaLaunchCooperativeKernel((void*)bn_fused_kernel<1>, grid, block, args, 0, s)

@@ -18,6 +18,7 @@ bool conv_tc_supported(const ConvProb& p, int mode);                            
 int conv_tc_fill(const ConvProb& p, int mode, void* host_tc);
 int conv_tc_count(const ConvProb& p, int mode);
 int conv_tc_stat_tiles(const ConvProb& p);
+int bn_fused_capacity(int backward);                                                    // kernels_ref.cu
 void launch_bn_finalize_tiles(const BnProb* d, int nprob, int max_c, cudaStream_t s);
 size_t conv_tc_prob_bytes();
 int conv_tc_tiles(const void* host_tc);
@@ -283,7 +284,7 @@ struct Builder {
             op.key = key + 1; op.kind = OP_BN_APPLY; ops->push_back(op);
             return stat;
         }
-        if (p.vec && !eval && r.c <= 512) { op.kind = OP_BN_FWD_FUSED; ops->push_back(op); return stat; }   // one cooperative launch
+        if (p.vec && !eval && r.c <= 512 && (long long)p.chunks * ctx->S <= bn_fused_capacity(0)) { op.kind = OP_BN_FWD_FUSED; ops->push_back(op); return stat; }   // one cooperative launch
         ops->push_back(op);
         op.key = key + 1; op.kind = OP_BN_APPLY; ops->push_back(op);
         return stat;
@@ -293,15 +294,18 @@ struct Builder {
         BnProb& p = op.bn;
         p.x = x; p.da = da; p.dx = dx; p.add = add; p.gamma = W() + r.g; p.beta = W() + r.b; p.dgamma = G() + r.g; p.dbeta = G() + r.b;
         p.stat = stat; p.m = m; p.C = r.c; p.eps = ctx->opts.bn_eps; p.momentum = ctx->opts.bn_momentum; p.eval = 0;
-        // (measured on 8 x 67 MB tensors, far beyond L2: the single cooperative launch, 586 us with two CTAs per SM and four rows of
-        // loads in flight per thread in both passes, beats the reduction kernel followed by the streaming elementwise kernel, 683 us;
-        // both move the same five passes over HBM)
+        // (measured on 8 x 67 MB tensors, far beyond L2: reduction + elementwise pass as two streaming launches, each with four rows
+        // of loads in flight per thread and two CTAs per SM, take 586 us; the cooperative kernel with three CTAs per SM and one
+        // row in flight took 794 us; both move the same five passes over HBM, so the cooperative form only pays for tensors that
+        // stay in L2 between its two passes)
         bn_chunking(p, ctx->opts.dtype == RESIST_BF16, fused_chunks());
         bn_partial_need = std::max(bn_partial_need, (size_t)p.chunks * 2 * r.c * 8);
         p.partial = bn_partial;
         const int producer = last_dgrad; last_dgrad = -1;
         if (fusable(producer, da, p)) { fuse_into(producer, p, 2); return; }
-        if (p.vec && r.c <= 512) { op.kind = OP_BN_BWD_FUSED; ops->push_back(op); return; }
+        // one cooperative launch where all sub-ResNets' chunks can be resident together (the kernel holds 128 registers: one CTA
+        // per SM), else the reduction and the elementwise pass as launches of their own
+        if (p.vec && r.c <= 512 && (long long)p.chunks * ctx->S <= bn_fused_capacity(1)) { op.kind = OP_BN_BWD_FUSED; ops->push_back(op); return; }
         ops->push_back(op);
         op.key = key + 1; op.kind = OP_BN_BWD_APPLY; ops->push_back(op);
     }
