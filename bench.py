@@ -51,8 +51,13 @@ WORKLOADS = {
     "wide_localsgd": (3, "configs[2]'s network trained by local SGD (Sec. 2.4): no block dealt out, S=8 full replicas, batch 128 each, "
                          "bf16 + fp32 master, 50 local steps per round", 4),
 }
-# mean DRAM bytes per launch of a kernel family (ncu, profiles/): workload -> family -> bytes; filled in from the committed captures
-NCU_DRAM_BYTES_PER_LAUNCH = {}
+# DRAM traffic of a kernel family as a fraction of its algorithmic bytes (dram__bytes_read.sum + dram__bytes_write.sum over the
+# family's launches of one step / the library's byte count of the same launches), from the ncu capture summarised in
+# profiles/dram_traffic_conv_tc_kernel_wide_S2_B128.txt: workload -> family -> ratio.  The capture ran 2 of the 8 sub-ResNets (the
+# full workload is too large to capture); the full launch's traffic is reported as ratio x its algorithmic bytes, a lower bound,
+# since with 8 sub-ResNets less of each tensor is still in L2 when its consumer reads it.
+NCU_TRAFFIC_RATIO = {"wide": {"conv_fwd_tcgen05": 0.716, "conv_fwd_tcgen05@tensor": 0.581, "conv_dgrad_tcgen05": 0.576,
+                              "conv_dgrad_tcgen05@tensor": 0.531}}
 
 
 def measured_peaks():
@@ -306,7 +311,9 @@ def run_ours(args):
             "arithmetic_intensity": top["flops"] / max(top["bytes"], 1.0),
             # DRAM bytes (read + written) per launch of that family from the ncu capture summarised under profiles/; None for a
             # family the capture does not cover or whose kernel has changed since
-            "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(args.workload, {}).get(top_name)}
+            "traffic": (NCU_TRAFFIC_RATIO.get(args.workload, {}).get(top_name) or 0.0) * top["bytes"] / top["operations"] or None}
+    if roof["traffic"]:
+        roof["traffic_source"] = "ncu on 2 of the 8 sub-ResNets, scaled by algorithmic bytes (lower bound: see profiles/dram_traffic_conv_tc_kernel_wide_S2_B128.txt)"
     conv = {k: v for k, v in step_prof.items() if k.startswith("conv_")}
     conv_ms = sum(v["ms"] for v in conv.values()) + sum(v["ms"] for k, v in step_prof.items() if k.startswith("wgrad_splitk"))
     conv_flops = sum(v["flops"] for v in conv.values())
