@@ -213,7 +213,7 @@ const char* resist_layer_last_error(void);
  *  - Limit: chunks * C <= 262144, where chunks (the number of row chunks reduced by one CTA each) never exceeds
  *    1024: any m with C <= 256 fits.  Larger problems return RESIST_EUNSUPPORTED with the sizes in the message.
  *  - The first call on each device looks up the array's device address (one cudaGetSymbolAddress, with that
- *    device current); make that first call before any stream capture begins.
+ *    device current); later calls on that device reuse it.
  *  - All calls share the one array, and it keeps what the last call left there.  Nothing has to be cleared between
  *    calls (each call writes every slot before reading it), but two calls that overlap on the GPU (different
  *    streams, or different host threads without ordering) race on it: keep them on one stream or order them.

@@ -328,7 +328,7 @@ def test_partition_invariants():
 
 
 def test_resnet101_has_22_partitionable_blocks_and_resnet50_has_five():
-    # Sec. 2.6: "ResNet50 contains only five blocks for partitioning" (its third section has six blocks)
+    # Sec. 2.6 counts five partitionable blocks for ResNet-50 (its third section has six blocks)
     assert synth.resnet101_arch().num_partitionable == 22
     assert synth.resnet101_arch(depths=(3, 4, 6, 3)).num_partitionable == 5
 
