@@ -190,16 +190,18 @@ __device__ void bn_reduce_vec(const BnProb& p) {
     }
     const uint4* xv = reinterpret_cast<const uint4*>(p.x);
     const uint4* dv = reinterpret_cast<const uint4*>(p.da);
-    // four rows of loads in flight per thread; the rows are still added in ascending order
-    for (long long row = r0 + r; row < r1; row += 4 * R) {
-        uint4 xs[4], ds[4];
+    // U rows of loads in flight per thread (backward: x and dy, so six rows = twelve 16-byte loads; forward: eight rows); the rows
+    // are still added in ascending order
+    constexpr int U = MODE == 1 ? 6 : 8;
+    for (long long row = r0 + r; row < r1; row += U * R) {
+        uint4 xs[U], ds[MODE == 1 ? U : 1];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < U; ++u) {
             const long long rr = row + (long long)u * R;
             if (rr < r1) { xs[u] = __ldg(xv + rr * G + g); if (MODE == 1) ds[u] = __ldg(dv + rr * G + g); }
         }
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < U; ++u) {
             if (row + (long long)u * R >= r1) break;
             float x[8]; unpack8(xs[u], x);
             if (MODE == 0) {

@@ -294,8 +294,8 @@ struct Builder {
         BnProb& p = op.bn;
         p.x = x; p.da = da; p.dx = dx; p.add = add; p.gamma = W() + r.g; p.beta = W() + r.b; p.dgamma = G() + r.g; p.dbeta = G() + r.b;
         p.stat = stat; p.m = m; p.C = r.c; p.eps = ctx->opts.bn_eps; p.momentum = ctx->opts.bn_momentum; p.eval = 0;
-        // (measured on 8 x 67 MB tensors, far beyond L2: reduction + elementwise pass as two streaming launches, each with four rows
-        // of loads in flight per thread and two CTAs per SM, take 586 us; the cooperative kernel with three CTAs per SM and one
+        // (measured on 8 x 67 MB tensors, far beyond L2: reduction + elementwise pass as two streaming launches, each with twelve
+        // 16-byte loads in flight per thread and two CTAs per SM, take 194 + 323 us; the cooperative kernel with three CTAs per SM and one
         // row in flight took 794 us; both move the same five passes over HBM, so the cooperative form only pays for tensors that
         // stay in L2 between its two passes)
         bn_chunking(p, ctx->opts.dtype == RESIST_BF16, fused_chunks());
@@ -306,6 +306,14 @@ struct Builder {
         // one cooperative launch where all sub-ResNets' chunks can be resident together (the kernel holds 128 registers: one CTA
         // per SM), else the reduction and the elementwise pass as launches of their own
         if (p.vec && r.c <= 512 && (long long)p.chunks * ctx->S <= bn_fused_capacity(1)) { op.kind = OP_BN_BWD_FUSED; ops->push_back(op); return; }
+        if (p.vec) {
+            // the reduction as a launch of its own: about four waves of CTAs over all sub-ResNets (long enough chunks for the batched
+            // loads to pipeline, enough of them for the SMs to even out the tail)
+            const int R = 256 / (r.c / 8);
+            long long rpc = (m + 4 * fused_chunks() - 1) / (4 * fused_chunks());
+            rpc = (rpc + R - 1) / R * R; if (rpc < 32 * R) rpc = 32 * R;
+            if (rpc > p.rows_per_chunk) { p.rows_per_chunk = (int)rpc; p.chunks = (int)((m + rpc - 1) / rpc); }
+        }
         ops->push_back(op);
         op.key = key + 1; op.kind = OP_BN_BWD_APPLY; ops->push_back(op);
     }
