@@ -117,6 +117,7 @@ struct ParamArrays {      // device pointers of the flat arrays
 };
 
 constexpr int SEG_CHUNK = 4096;   // elements per CTA in the segment kernels
+constexpr int AGG_CHUNK = 8192;   // elements per CTA of the aggregate kernel (two rounds of four 16-byte groups per thread)
 
 // ---- launchers (kernels_ref.cu)
 void launch_conv_ref(const ConvProb* d, int nprob, int max_tiles, int mode, bool bf16, cudaStream_t s);

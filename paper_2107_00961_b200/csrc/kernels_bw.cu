@@ -104,9 +104,15 @@ __device__ __forceinline__ float mean_of_owners(const float* __restrict__ sub, l
 }
 
 // Segment::sub selects the array pair: 0 = parameters, 1 = BN running statistics (one launch serves both).
-__global__ void __launch_bounds__(256, 4) aggregate_kernel(const Segment* __restrict__ segs, int nseg, AggArrays arr, int S) {
+__device__ __forceinline__ void acc_diff(float4& acc, const float4& x, const float4& first) {
+    acc.x = __fadd_rn(acc.x, __fsub_rn(x.x, first.x)); acc.y = __fadd_rn(acc.y, __fsub_rn(x.y, first.y));
+    acc.z = __fadd_rn(acc.z, __fsub_rn(x.z, first.z)); acc.w = __fadd_rn(acc.w, __fsub_rn(x.w, first.w));
+}
+__global__ void __launch_bounds__(256, 3) aggregate_kernel(const Segment* __restrict__ segs, int nseg, AggArrays arr, int S) {
     const Segment& sg = find_segment(segs, nseg, blockIdx.x);
-    const Range r = chunk_range(sg, blockIdx.x);
+    const long long off = ((long long)blockIdx.x - sg.chunk0) * AGG_CHUNK;
+    long long rem = sg.len - off; if (rem > AGG_CHUNK) rem = AGG_CHUNK;
+    const Range r{sg.begin + off, (int)rem};
     const int which = sg.sub != 0;
     const float* __restrict__ sub = which ? arr.sub_b : arr.sub_p; const long long stride = which ? arr.stride_b : arr.stride_p;
     float* __restrict__ global = which ? arr.global_b : arr.global_p;
@@ -115,44 +121,49 @@ __global__ void __launch_bounds__(256, 4) aggregate_kernel(const Segment* __rest
     if (((r.base | stride) & 3) == 0) {
         const int nq = r.len >> 2;
         const int cnt = __popc(mask);
-        // Four 16-byte groups per thread at a time, and for each owner (ascending; the mask is the segment's, so the loop is
-        // uniform over the CTA) their four loads in flight together: the kernel is bound by how many bytes it keeps in flight.
-        // The arithmetic per element is the scalar routine's: first + (sum over the other owners of (w_s - first)) / count.
-        for (int q0 = threadIdx.x; q0 < nq && cnt > 0; q0 += 4 * 256) {
-            float4 first[4], acc[4];
-            unsigned m = mask;
-            const int s0 = __ffs(m) - 1; m &= m - 1;
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int q = q0 + u * 256;
-                first[u] = q < nq ? *reinterpret_cast<const float4*>(sub + (long long)s0 * stride + r.base + 4LL * q) : make_float4(0.f, 0.f, 0.f, 0.f);
-                acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-            while (m) {
-                const int sidx = __ffs(m) - 1; m &= m - 1;
-                float4 x[4];
+        // The kernel is bound by the bytes it keeps in flight: four 16-byte groups per thread at a time, and the loads of TWO
+        // owners (ascending; the mask is the segment's, so the loop is uniform over the CTA) in flight together.  The arithmetic per element is the scalar
+        // routine's, in its order: first + (sum over the other owners of (w_s - first)) / count.
+        if (cnt >= 1) {
+            for (int q0 = threadIdx.x; q0 < nq; q0 += 4 * 256) {
+                float4 first[4], acc[4];
+                unsigned m = mask;
+                const int s0 = __ffs(m) - 1; m &= m - 1;
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
                     const int q = q0 + u * 256;
-                    x[u] = q < nq ? *reinterpret_cast<const float4*>(sub + (long long)sidx * stride + r.base + 4LL * q) : first[u];
+                    first[u] = q < nq ? *reinterpret_cast<const float4*>(sub + (long long)s0 * stride + r.base + 4LL * q) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
                 }
+                while (m) {
+                    const int sa = __ffs(m) - 1; m &= m - 1;
+                    const int sb = m ? __ffs(m) - 1 : -1; if (m) m &= m - 1;
+                    float4 xa[4], xb[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int q = q0 + u * 256;
+                        xa[u] = q < nq ? *reinterpret_cast<const float4*>(sub + (long long)sa * stride + r.base + 4LL * q) : first[u];
+                        xb[u] = (sb >= 0 && q < nq) ? *reinterpret_cast<const float4*>(sub + (long long)sb * stride + r.base + 4LL * q) : first[u];
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) acc_diff(acc[u], xa[u], first[u]);
+                    if (sb >= 0) {
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) acc_diff(acc[u], xb[u], first[u]);
+                    }
+                }
+                const float c = (float)cnt;
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
-                    acc[u].x = __fadd_rn(acc[u].x, __fsub_rn(x[u].x, first[u].x)); acc[u].y = __fadd_rn(acc[u].y, __fsub_rn(x[u].y, first[u].y));
-                    acc[u].z = __fadd_rn(acc[u].z, __fsub_rn(x[u].z, first[u].z)); acc[u].w = __fadd_rn(acc[u].w, __fsub_rn(x[u].w, first[u].w));
-                }
-            }
-            const float c = (float)cnt;
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int q = q0 + u * 256;
-                if (q >= nq) continue;
-                float4 out = first[u];
-                if (cnt > 1) {
+                    const int q = q0 + u * 256;
+                    if (q >= nq) continue;
+                    float4 out = first[u];
+                    if (cnt > 1) {
                     out.x = __fadd_rn(first[u].x, __fdiv_rn(acc[u].x, c)); out.y = __fadd_rn(first[u].y, __fdiv_rn(acc[u].y, c));
                     out.z = __fadd_rn(first[u].z, __fdiv_rn(acc[u].z, c)); out.w = __fadd_rn(first[u].w, __fdiv_rn(acc[u].w, c));
+                    }
+                    *reinterpret_cast<float4*>(global + r.base + 4LL * q) = out;
                 }
-                *reinterpret_cast<float4*>(global + r.base + 4LL * q) = out;
             }
         }
         done = nq << 2;

@@ -370,7 +370,7 @@ int resist_aggregate(resist_ctx* ctx, resist_stream stream) {
     auto build = [&](bool buffers, std::vector<Segment>& out, long long& ch) {
         const long long total = buffers ? L.n_buffers : L.n_params;
         long long run = 0; uint32_t run_mask = all;
-        auto flush = [&](long long end) { if (end > run) { Segment s{run, end - run, ch, run_mask, buffers ? 1 : 0}; ch += (s.len + SEG_CHUNK - 1) / SEG_CHUNK; out.push_back(s); } run = end; };
+        auto flush = [&](long long end) { if (end > run) { Segment s{run, end - run, ch, run_mask, buffers ? 1 : 0}; ch += (s.len + AGG_CHUNK - 1) / AGG_CHUNK; out.push_back(s); } run = end; };
         for (size_t b = 0; b < L.blk.size(); ++b) {
             const long long bb = buffers ? L.blk[b].buf_begin : L.blk[b].begin, be = buffers ? L.blk[b].buf_end : L.blk[b].end;
             if (ctx->mask[b] == run_mask) continue;           // extends the current run (block ranges are contiguous)
