@@ -156,7 +156,7 @@ int resist_get_shadow(resist_ctx* ctx, int32_t subnet, uint16_t* host_bf16);
 typedef struct {
     int64_t kernel_launches;   /* kernels enqueued */
     int64_t conv_flops;        /* 2*M*N*K summed over forward, dgrad and wgrad convolutions */
-    int64_t tensor_core_convs; /* convolution problems run on tcgen05 */
+    int64_t tensor_core_convs; /* convolution problems run on a tensor-core family: tcgen05 or warp-level MMA */
     int64_t cuda_core_convs;   /* convolution problems run on CUDA cores */
     int64_t workspace_bytes;   /* device memory held for activations and scratch */
 } resist_step_info;

@@ -1,11 +1,11 @@
 // Convolutions of NARROW layers (C and K multiples of 16, at most 64) on warp-level MMA (mma.sync m16n8k16, bf16
 // inputs, fp32 accumulation).
 //
-// Why not tcgen05 here: the SM's tensor core takes about 40 cycles per tcgen05.mma with M = 128, K = 16 however
-// small N is (measured: 21 ns per MMA at N = 16 with two issuing threads, 41 ns with one), so a layer with 16
-// output channels uses 1/16 of the array and is bound by that rate below what HBM allows.  The warp-level MMA has
-// no such granularity (n = 8) and was measured at 550 TFLOP/s dense on this GPU, more than these HBM-bound layers
-// need.  Wide layers (more than 64 channels) stay on tcgen05 (conv_tc.cu).
+// Why not tcgen05 here: one thread issues a tcgen05.mma (M = 128, K = 16) only every 114-165 cycles whatever its N, two
+// issuing warps every 57-82 (resist_micro_mma_rate in micro.cu measures it), while the tensor core needs N / 2 cycles: a layer
+// with 16 or 32 output channels would spend 4-10 times its tensor time on issue, and its TMA rows would be 32-64 bytes.  The
+// warp-level MMA has no such granularity (n = 8), cp.async has no per-row cost, and these HBM-bound layers need far less
+// than its rate.  Wider layers, and 64-channel 3x3 layers with many positions, run on tcgen05 (conv_tc.cu).
 //
 // Tiling: a GROUP of G whole images is one tall zero-padded map.  With pad = k/2, image n occupies rows
 // n*Hp .. n*Hp+H-1 (Hp = H + pad) of a map that is Wp = W + pad wide; row H of every image and column W of every
